@@ -1,0 +1,370 @@
+"""CPU oracle for the Ladder-Residual / standard-residual transformer forward.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain definition the CUDA
+library is checked against.  Nothing in the product path may import it; only
+the tests, the smoke check and the CPU-baseline leg of the benchmark do.  It
+shares no code with the CUDA path and never receives a value computed there.
+
+What it follows
+---------------
+* Standard residual recurrence  x_i = h_i(x_{i-1}) + x_{i-1}        (Sec. 2, Eq. 1)
+* Ladder recurrence             x_i = h_i(x_{i-2}) + x_{i-1}        (Sec. 3.1, Eq. 2)
+* The layer routine with pending module outputs                     (Algorithm 1)
+  with the asynchronous all-reduce and its handle being the identity on a
+  single device.
+* "Llama-3's model architecture" (Sec. 3.3.1): pre-norm RMSNorm, rotary
+  position embedding on interleaved pairs, grouped-query causal attention,
+  SwiGLU MLP, final RMSNorm, untied LM head, no biases.
+
+Readings taken where the paper is silent (both sides of every parity test use
+the same ones):
+* initial pending outputs of Algorithm 1 are zero, so modules 1 and 2 both read x_0;
+* the two outputs still pending after the last layer are added before the
+  final norm (Eq. 2 adds every h_i into the stream);
+* a standard layer first adds whatever is pending and leaves nothing pending
+  (hybrid models: the first ladder attention after a standard layer reads the
+  complete stream) -- PARITY UNPINNED by the paper for this hybrid boundary rule;
+* greedy argmax takes the lowest index among equal maxima.
+
+Arithmetic: every array is ``dtype`` (float64 by default, float32 for the large
+workloads); rotary angles, cos and sin are always formed in float64.  With
+``bf16_storage=True`` the values the CUDA path stores as bf16 (normalised
+activations, q/k/v, attention output, SwiGLU output) are rounded to bf16 too;
+this is a diagnostic switch that separates bf16 noise from bugs, not the
+definition.
+
+Pins (tests/test_oracle_pins.py): single-module ladder == standard, cached
+decode == recomputation, softmax rows, brute-force attention, Eq.-2 form ==
+Algorithm-1 form, staleness, telescoping sum, single live module, closed forms
+for zeroed projections, RoPE relative-position property, RMSNorm textbook
+formula, GQA == MHA with repeated heads, causality, batch independence,
+linear layers vs float64 matmul written out in the test.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Callable, Dict, List, Optional, Sequence
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------- config
+@dataclass
+class OracleConfig:
+    d_model: int
+    n_layers: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    d_ff: int
+    vocab_size: int
+    rms_eps: float = 1e-5
+    rope_theta: float = 10000.0
+    layer_is_ladder: Optional[Sequence[bool]] = None  # None = every layer ladder
+
+    def ladder(self, layer: int) -> bool:
+        if self.layer_is_ladder is None:
+            return True
+        return bool(self.layer_is_ladder[layer])
+
+
+class OracleWeights:
+    """Logical (unpacked) weights.  ``get(name, layer)`` returns a float array.
+
+    names: tok_embedding [V,d], final_norm [d], lm_head [V,d] (layer=None) and per
+    layer attn_norm [d], wq [Hq*Dh,d], wk [Hkv*Dh,d], wv [Hkv*Dh,d], wo [d,Hq*Dh],
+    mlp_norm [d], w_gate [F,d], w_up [F,d], w_down [d,F].  A provider callback lets
+    a caller stream one layer at a time for models larger than host memory.
+    """
+
+    def __init__(self, tensors: Optional[Dict] = None,
+                 provider: Optional[Callable[[str, Optional[int]], np.ndarray]] = None):
+        self._t = tensors or {}
+        self._p = provider
+
+    def get(self, name: str, layer: Optional[int] = None) -> np.ndarray:
+        key = (name, layer)
+        if key in self._t:
+            return self._t[key]
+        if self._p is None:
+            raise KeyError(key)
+        return self._p(name, layer)
+
+
+# --------------------------------------------------------------------------- helpers
+def bf16_round(a: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even to bfloat16 precision, returned in a's dtype."""
+    f = np.ascontiguousarray(a, dtype=np.float32)
+    u = f.view(np.uint32)
+    lsb = (u >> np.uint32(16)) & np.uint32(1)
+    r = (u + np.uint32(0x7FFF) + lsb) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(a.dtype)
+
+
+def _store(a: np.ndarray, bf16_storage: bool) -> np.ndarray:
+    return bf16_round(a) if bf16_storage else a
+
+
+def rmsnorm(x: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
+    """y_i = x_i / sqrt(mean_j x_j^2 + eps) * g_i over the last axis."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + x.dtype.type(eps)) * g.astype(x.dtype)
+
+
+def rope_angles(positions: np.ndarray, head_dim: int, theta: float):
+    """cos/sin [T, Dh/2] in float64: angle = p * theta^(-2j/Dh)."""
+    j = np.arange(head_dim // 2, dtype=np.float64)
+    inv_freq = np.float64(theta) ** (-2.0 * j / head_dim)
+    ang = positions.astype(np.float64)[:, None] * inv_freq[None, :]
+    return np.cos(ang), np.sin(ang)
+
+
+def rope(u: np.ndarray, positions: np.ndarray, theta: float) -> np.ndarray:
+    """Rotate interleaved pairs (u_{2j}, u_{2j+1}) of u[..., T, H, Dh] by position."""
+    dh = u.shape[-1]
+    cos, sin = rope_angles(positions, dh, theta)          # [T, Dh/2]
+    cos = cos[:, None, :].astype(u.dtype)
+    sin = sin[:, None, :].astype(u.dtype)
+    ue, uo = u[..., 0::2], u[..., 1::2]
+    out = np.empty_like(u)
+    out[..., 0::2] = ue * cos - uo * sin
+    out[..., 1::2] = ue * sin + uo * cos
+    return out
+
+
+def softmax_rows(s: np.ndarray) -> np.ndarray:
+    """Softmax over the last axis with max subtraction; -inf entries give exactly 0."""
+    m = np.max(s, axis=-1, keepdims=True)
+    e = np.exp(s - m)
+    return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def causal_attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, q_pos0: int,
+                     return_probs: bool = False):
+    """Grouped-query causal attention for one sequence.
+
+    q [T, Hq, Dh] holds queries at absolute positions q_pos0 .. q_pos0+T-1;
+    k, v [L, Hkv, Dh] hold keys/values at absolute positions 0 .. L-1.
+    Query head h uses kv head h // (Hq // Hkv).  Query at position p attends to
+    keys t <= p.  Returns o [T, Hq, Dh] (and the probabilities [Hq, T, L]).
+    """
+    T, Hq, Dh = q.shape
+    L, Hkv, _ = k.shape
+    group = Hq // Hkv
+    scale = q.dtype.type(1.0 / np.sqrt(Dh))
+    o = np.empty_like(q)
+    probs = np.empty((Hq, T, L), dtype=q.dtype) if return_probs else None
+    p_idx = q_pos0 + np.arange(T)[:, None]
+    t_idx = np.arange(L)[None, :]
+    masked = t_idx > p_idx                                   # [T, L]
+    for h in range(Hq):
+        kh = h // group
+        s = (q[:, h, :] @ k[:, kh, :].T) * scale             # [T, L]
+        s = np.where(masked, -np.inf, s)
+        pr = softmax_rows(s)
+        o[:, h, :] = pr @ v[:, kh, :]
+        if return_probs:
+            probs[h] = pr
+    return (o, probs) if return_probs else o
+
+
+def silu(z: np.ndarray) -> np.ndarray:
+    return z / (1.0 + np.exp(-z))
+
+
+# --------------------------------------------------------------------------- cache
+class OracleCache:
+    """K (post-RoPE) and V for every layer: [n_layers][B][max_seq][Hkv][Dh]."""
+
+    def __init__(self, cfg: OracleConfig, batch: int, max_seq_len: int, dtype=np.float64):
+        shp = (cfg.n_layers, batch, max_seq_len, cfg.n_kv_heads, cfg.head_dim)
+        self.k = np.zeros(shp, dtype=dtype)
+        self.v = np.zeros(shp, dtype=dtype)
+        self.seq_len = 0
+        self.max_seq_len = max_seq_len
+
+
+# --------------------------------------------------------------------------- modules
+def attention_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndarray,
+                     pos0: int, cache: Optional[OracleCache], bf16_storage: bool = False):
+    """h(n) for the attention module of ``layer``.
+
+    n [B, T, d] is the normalised input at absolute positions pos0..pos0+T-1.
+    With a cache, the new K/V rows are appended at those positions first and
+    attention then runs over positions 0..pos0+T-1 (append, then attend).
+    """
+    B, T, d = n.shape
+    Hq, Hkv, Dh = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    dt = n.dtype
+    wq = W.get("wq", layer).astype(dt)
+    wk = W.get("wk", layer).astype(dt)
+    wv = W.get("wv", layer).astype(dt)
+    wo = W.get("wo", layer).astype(dt)
+    positions = pos0 + np.arange(T)
+    q = (n @ wq.T).reshape(B, T, Hq, Dh)
+    k = (n @ wk.T).reshape(B, T, Hkv, Dh)
+    v = (n @ wv.T).reshape(B, T, Hkv, Dh)
+    q = _store(rope(q, positions, cfg.rope_theta), bf16_storage)
+    k = _store(rope(k, positions, cfg.rope_theta), bf16_storage)
+    v = _store(v, bf16_storage)
+    o = np.empty((B, T, Hq, Dh), dtype=dt)
+    for b in range(B):
+        if cache is not None:
+            cache.k[layer, b, pos0:pos0 + T] = k[b]
+            cache.v[layer, b, pos0:pos0 + T] = v[b]
+            kk = cache.k[layer, b, :pos0 + T].astype(dt)
+            vv = cache.v[layer, b, :pos0 + T].astype(dt)
+        else:
+            assert pos0 == 0
+            kk, vv = k[b], v[b]
+        o[b] = causal_attention(q[b], kk, vv, pos0)
+    o = _store(o.reshape(B, T, Hq * Dh), bf16_storage)
+    return o @ wo.T
+
+
+def mlp_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndarray,
+               bf16_storage: bool = False):
+    """h(n) = W_down ( silu(W_gate n) * (W_up n) )."""
+    dt = n.dtype
+    wg = W.get("w_gate", layer).astype(dt)
+    wu = W.get("w_up", layer).astype(dt)
+    wd = W.get("w_down", layer).astype(dt)
+    h = _store(silu(n @ wg.T) * (n @ wu.T), bf16_storage)
+    return h @ wd.T
+
+
+# --------------------------------------------------------------------------- forward
+@dataclass
+class ForwardResult:
+    x_final: np.ndarray                 # [B, T, d]   residual stream after the last add
+    hidden: np.ndarray                  # [B, T, d]   after the final RMSNorm
+    logits: Optional[np.ndarray]        # [B, T', V]  (T' = T, or 1 when last_only)
+    next_tokens: Optional[np.ndarray]   # [B, T']
+    module_inputs: List[np.ndarray] = field(default_factory=list)   # residual each module read
+    module_outputs: List[np.ndarray] = field(default_factory=list)  # h_m(.)
+
+
+def greedy(logits: np.ndarray) -> np.ndarray:
+    """argmax over the last axis; numpy returns the first (lowest) index on ties."""
+    return np.argmax(logits, axis=-1).astype(np.int64)
+
+
+def run_layers(cfg: OracleConfig, W: OracleWeights, x: np.ndarray, pos0: int,
+               cache: Optional[OracleCache], bf16_storage: bool = False,
+               record: Optional[ForwardResult] = None, n_layers: Optional[int] = None):
+    """The layer stack in Algorithm-1 form, then the final flush.  x [B,T,d]."""
+    a_p = np.zeros_like(x)              # pending attention output (attn_out)
+    m_p = np.zeros_like(x)              # pending MLP output       (mlp_out)
+    L = cfg.n_layers if n_layers is None else n_layers
+    for l in range(L):
+        g_a = W.get("attn_norm", l)
+        g_m = W.get("mlp_norm", l)
+        if cfg.ladder(l):
+            x = x + a_p                                                  # residual += attn_out
+            n = _store(rmsnorm(x, g_a, cfg.rms_eps), bf16_storage)       # AttentionNorm
+            if record is not None:
+                record.module_inputs.append(x.copy())
+            a_p = attention_module(cfg, W, l, n, pos0, cache, bf16_storage)
+            x = x + m_p                                                  # residual += mlp_out
+            n = _store(rmsnorm(x, g_m, cfg.rms_eps), bf16_storage)       # MLPNorm
+            if record is not None:
+                record.module_inputs.append(x.copy())
+            m_p = mlp_module(cfg, W, l, n, bf16_storage)
+            if record is not None:
+                record.module_outputs += [a_p.copy(), m_p.copy()]
+        else:
+            x = x + a_p + m_p                                            # nothing stays pending
+            a_p = np.zeros_like(x)
+            m_p = np.zeros_like(x)
+            n = _store(rmsnorm(x, g_a, cfg.rms_eps), bf16_storage)
+            if record is not None:
+                record.module_inputs.append(x.copy())
+            a = attention_module(cfg, W, l, n, pos0, cache, bf16_storage)
+            x = x + a
+            n = _store(rmsnorm(x, g_m, cfg.rms_eps), bf16_storage)
+            if record is not None:
+                record.module_inputs.append(x.copy())
+            m = mlp_module(cfg, W, l, n, bf16_storage)
+            x = x + m
+            if record is not None:
+                record.module_outputs += [a.copy(), m.copy()]
+    return x + a_p + m_p
+
+
+def embed(W: OracleWeights, tokens: np.ndarray, dtype) -> np.ndarray:
+    E = W.get("tok_embedding")
+    return E[np.asarray(tokens, dtype=np.int64)].astype(dtype)
+
+
+def head(cfg: OracleConfig, W: OracleWeights, x: np.ndarray, bf16_storage: bool = False):
+    hidden = rmsnorm(x, W.get("final_norm"), cfg.rms_eps)
+    logits = _store(hidden, bf16_storage) @ W.get("lm_head").astype(x.dtype).T
+    return hidden, logits
+
+
+def forward(cfg: OracleConfig, W: OracleWeights, tokens: np.ndarray, dtype=np.float64,
+            cache: Optional[OracleCache] = None, pos0: int = 0, last_only: bool = False,
+            bf16_storage: bool = False, record: bool = False,
+            with_logits: bool = True, n_layers: Optional[int] = None) -> ForwardResult:
+    """Full forward over tokens [B, T] at positions pos0..pos0+T-1.
+
+    Without a cache pos0 must be 0 and the whole sequence is recomputed.  With a
+    cache the new rows are appended and ``cache.seq_len`` advances by T.
+    """
+    tokens = np.asarray(tokens)
+    res = ForwardResult(None, None, None, None)
+    x = embed(W, tokens, dtype)
+    x = run_layers(cfg, W, x, pos0, cache, bf16_storage, res if record else None, n_layers)
+    if cache is not None:
+        assert cache.seq_len == pos0
+        cache.seq_len = pos0 + tokens.shape[1]
+    res.x_final = x
+    xs = x[:, -1:, :] if last_only else x
+    if with_logits:
+        hidden, logits = head(cfg, W, xs, bf16_storage)
+        res.logits = logits
+        res.next_tokens = greedy(logits)
+    else:
+        hidden = rmsnorm(xs, W.get("final_norm"), cfg.rms_eps)
+    res.hidden = hidden
+    return res
+
+
+def prefill(cfg, W, tokens, cache: OracleCache, dtype=np.float64, bf16_storage=False,
+            n_layers=None) -> ForwardResult:
+    """Prompt pass: fills cache rows 0..S-1, returns hidden/logits at position S-1."""
+    assert cache.seq_len == 0
+    return forward(cfg, W, tokens, dtype, cache, 0, last_only=True,
+                   bf16_storage=bf16_storage, n_layers=n_layers)
+
+
+def decode_step(cfg, W, tokens, cache: OracleCache, dtype=np.float64, bf16_storage=False,
+                n_layers=None) -> ForwardResult:
+    """One token per sequence at position cache.seq_len (append, then attend)."""
+    tokens = np.asarray(tokens).reshape(-1, 1)
+    return forward(cfg, W, tokens, dtype, cache, cache.seq_len, last_only=True,
+                   bf16_storage=bf16_storage, n_layers=n_layers)
+
+
+def generate(cfg, W, prompt: np.ndarray, n_steps: int, max_seq_len: int, dtype=np.float64,
+             forced: Optional[np.ndarray] = None, bf16_storage=False):
+    """prefill + n_steps decode steps.
+
+    Returns (tokens [B, n_steps+1], hiddens [B, n_steps+1, d]): entry 0 comes from
+    the prefill (token at position S), entry j+1 from decode step j.  With
+    ``forced`` [B, n_steps+1] the fed-back tokens are taken from it instead of the
+    oracle's own argmax (teacher forcing), while the returned tokens stay the
+    oracle's own choices.
+    """
+    prompt = np.asarray(prompt)
+    B, S = prompt.shape
+    cache = OracleCache(cfg, B, max_seq_len, dtype)
+    r = prefill(cfg, W, prompt, cache, dtype, bf16_storage)
+    toks = [r.next_tokens[:, 0]]
+    hids = [r.hidden[:, 0]]
+    for j in range(n_steps):
+        feed = toks[-1] if forced is None else np.asarray(forced)[:, j]
+        r = decode_step(cfg, W, feed, cache, dtype, bf16_storage)
+        toks.append(r.next_tokens[:, 0])
+        hids.append(r.hidden[:, 0])
+    return np.stack(toks, axis=1), np.stack(hids, axis=1)

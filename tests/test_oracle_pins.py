@@ -1,0 +1,376 @@
+"""Pins for the CPU oracle: every check compares it with something other than itself --
+a closed form, a textbook formula written out here, brute force in scalar loops, or an
+invariant the paper fixes (Sec. 2 Eq. 1, Sec. 3.1 Eq. 2, Algorithm 1)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ladder_oracle as O
+from tests.helpers import W, rand_weights, small_cfg
+
+TOK = np.array([[3, 17, 5, 9, 60, 1], [8, 8, 2, 33, 4, 50]])
+
+
+def _x0(t, tokens):
+    return t[("tok_embedding", None)][tokens]
+
+
+# ---------------------------------------------------------------- elementary operations
+def test_rmsnorm_textbook_formula():
+    rng = np.random.default_rng(1)
+    x = rng.normal(size=(3, 10))
+    g = rng.uniform(0.5, 1.5, 10)
+    y = O.rmsnorm(x, g, 1e-5)
+    for r in range(3):
+        ms = sum(float(v) ** 2 for v in x[r]) / 10
+        for i in range(10):
+            assert abs(y[r, i] - x[r, i] / math.sqrt(ms + 1e-5) * g[i]) < 1e-12
+    # scale invariance and unit rms for g = 1, eps -> 0
+    y1 = O.rmsnorm(x, np.ones(10), 0.0)
+    assert np.allclose(np.sqrt(np.mean(y1 ** 2, -1)), 1.0, atol=1e-12)
+    assert np.allclose(O.rmsnorm(7.5 * x, g, 0.0), O.rmsnorm(x, g, 0.0), atol=1e-12)
+
+
+def test_rope_is_complex_rotation_of_interleaved_pairs():
+    rng = np.random.default_rng(2)
+    T, H, Dh, theta = 5, 2, 8, 10000.0
+    u = rng.normal(size=(T, H, Dh))
+    pos = np.array([0, 1, 2, 7, 100])
+    out = O.rope(u, pos, theta)
+    for t in range(T):
+        for h in range(H):
+            for j in range(Dh // 2):
+                z = complex(u[t, h, 2 * j], u[t, h, 2 * j + 1])
+                ang = pos[t] * theta ** (-2.0 * j / Dh)
+                zr = z * complex(math.cos(ang), math.sin(ang))
+                assert abs(out[t, h, 2 * j] - zr.real) < 1e-12
+                assert abs(out[t, h, 2 * j + 1] - zr.imag) < 1e-12
+    assert np.array_equal(out[0], u[0])                                # position 0 is the identity
+    assert np.allclose(np.linalg.norm(out, axis=-1), np.linalg.norm(u, axis=-1), atol=1e-12)
+
+
+def test_rope_scores_depend_on_relative_position_only():
+    rng = np.random.default_rng(3)
+    q = rng.normal(size=(1, 1, 16))
+    k = rng.normal(size=(1, 1, 16))
+    def score(p, t):
+        return float(np.sum(O.rope(q, np.array([p]), 500000.0) * O.rope(k, np.array([t]), 500000.0)))
+    assert abs(score(9, 4) - score(9 + 37, 4 + 37)) < 1e-10
+    assert abs(score(9, 4) - score(8, 4)) > 1e-6
+
+
+def test_silu_and_swiglu_scalar_formula():
+    rng = np.random.default_rng(4)
+    cfg = small_cfg(n_layers=1)
+    t = rand_weights(cfg, 4)
+    n = rng.normal(size=(1, 2, cfg.d_model))
+    out = O.mlp_module(cfg, W(t), 0, n)
+    wg, wu, wd = t[("w_gate", 0)], t[("w_up", 0)], t[("w_down", 0)]
+    for p in range(2):
+        h = []
+        for j in range(cfg.d_ff):
+            zg = sum(wg[j, i] * n[0, p, i] for i in range(cfg.d_model))
+            zu = sum(wu[j, i] * n[0, p, i] for i in range(cfg.d_model))
+            h.append(zg / (1.0 + math.exp(-zg)) * zu)
+        for i in range(cfg.d_model):
+            ref = sum(wd[i, j] * h[j] for j in range(cfg.d_ff))
+            assert abs(out[0, p, i] - ref) < 1e-10
+
+
+def test_bf16_round_matches_library_conversion():
+    rng = np.random.default_rng(5)
+    a = np.concatenate([rng.normal(size=1000), [0.0, 1.0, -1.0, 1.00390625, 3.0e-5, 65504.0]]).astype(np.float32)
+    ref = torch.from_numpy(a).to(torch.bfloat16).to(torch.float32).numpy()
+    assert np.array_equal(O.bf16_round(a), ref)
+
+
+# ---------------------------------------------------------------- attention
+def _brute_attention(q, k, v, pos0):
+    """Scalar loops, explicit K/V replication per query head, explicit mask."""
+    T, Hq, Dh = q.shape
+    L, Hkv, _ = k.shape
+    rep = Hq // Hkv
+    k_rep = [[k[t][h // rep] for h in range(Hq)] for t in range(L)]
+    v_rep = [[v[t][h // rep] for h in range(Hq)] for t in range(L)]
+    out = np.zeros((T, Hq, Dh))
+    for p in range(T):
+        for h in range(Hq):
+            s = []
+            for t in range(L):
+                if t <= pos0 + p:
+                    s.append(sum(q[p, h, i] * k_rep[t][h][i] for i in range(Dh)) / math.sqrt(Dh))
+            m = max(s)
+            e = [math.exp(v_ - m) for v_ in s]
+            z = sum(e)
+            for t in range(len(s)):
+                for i in range(Dh):
+                    out[p, h, i] += e[t] / z * v_rep[t][h][i]
+    return out
+
+
+@pytest.mark.parametrize("hq,hkv,pos0,T", [(4, 2, 0, 5), (4, 4, 0, 4), (6, 1, 3, 2), (2, 2, 6, 1)])
+def test_attention_brute_force(hq, hkv, pos0, T):
+    rng = np.random.default_rng(6)
+    Dh, L = 4, pos0 + T
+    q = rng.normal(size=(T, hq, Dh))
+    k = rng.normal(size=(L, hkv, Dh))
+    v = rng.normal(size=(L, hkv, Dh))
+    assert np.allclose(O.causal_attention(q, k, v, pos0), _brute_attention(q, k, v, pos0), atol=1e-12)
+
+
+def test_softmax_rows_sum_to_one_and_mask_is_exact():
+    rng = np.random.default_rng(7)
+    q = rng.normal(size=(6, 4, 8)) * 3
+    k = rng.normal(size=(6, 2, 8)) * 3
+    v = rng.normal(size=(6, 2, 8))
+    _, p = O.causal_attention(q, k, v, 0, return_probs=True)
+    assert np.all(p >= 0)
+    assert np.allclose(p.sum(-1), 1.0, atol=1e-12)
+    for a in range(6):
+        assert np.all(p[:, a, a + 1:] == 0.0)
+        assert np.all(p[:, a, :a + 1] > 0.0)
+
+
+def test_zero_query_gives_causal_running_mean_of_values():
+    cfg = small_cfg(n_layers=1)
+    t = rand_weights(cfg, 8)
+    t[("wq", 0)] = np.zeros_like(t[("wq", 0)])
+    rng = np.random.default_rng(8)
+    n = rng.normal(size=(1, 5, cfg.d_model))
+    out = O.attention_module(cfg, W(t), 0, n, 0, None)
+    v = (n[0] @ t[("wv", 0)].T).reshape(5, cfg.n_kv_heads, cfg.head_dim)
+    run = np.cumsum(v, axis=0) / np.arange(1, 6)[:, None, None]
+    rep = cfg.n_q_heads // cfg.n_kv_heads
+    o = np.repeat(run, rep, axis=1).reshape(5, -1)
+    assert np.allclose(out[0], o @ t[("wo", 0)].T, atol=1e-12)
+
+
+def test_gqa_equals_mha_with_repeated_kv_heads():
+    cfg_g = small_cfg(n_layers=2, hq=4, hkv=2)
+    cfg_m = small_cfg(n_layers=2, hq=4, hkv=4)
+    t = rand_weights(cfg_g, 9)
+    tm = dict(t)
+    for l in range(2):
+        for nm in ("wk", "wv"):
+            w = t[(nm, l)].reshape(2, cfg_g.head_dim, -1)
+            tm[(nm, l)] = np.repeat(w, 2, axis=0).reshape(4 * cfg_g.head_dim, -1)
+    a = O.forward(cfg_g, W(t), TOK)
+    b = O.forward(cfg_m, W(tm), TOK)
+    assert np.allclose(a.hidden, b.hidden, atol=1e-12)
+
+
+def test_linear_layers_match_float64_matmul_written_here():
+    cfg = small_cfg(n_layers=1, hq=2, hkv=2)
+    t = rand_weights(cfg, 10)
+    rng = np.random.default_rng(10)
+    n = rng.normal(size=(1, 1, cfg.d_model))
+    out = O.attention_module(cfg, W(t), 0, n, 0, None)
+    # one token at position 0: RoPE is the identity, softmax over one key is 1, so out = Wo Wv n
+    v = np.array([sum(t[("wv", 0)][r, i] * n[0, 0, i] for i in range(cfg.d_model))
+                  for r in range(cfg.n_kv_heads * cfg.head_dim)])
+    ref = np.array([sum(t[("wo", 0)][r, c] * v[c] for c in range(v.size)) for r in range(cfg.d_model)])
+    assert np.allclose(out[0, 0], ref, atol=1e-12)
+
+
+# ---------------------------------------------------------------- routing (Eq. 1, Eq. 2, Algorithm 1)
+def _modules(cfg, t):
+    """h_m for m = 1..2N acting on a residual value, built from the oracle's module functions."""
+    Wt = W(t)
+    mods = []
+    for l in range(cfg.n_layers):
+        mods.append(lambda x, l=l: O.attention_module(
+            cfg, Wt, l, O.rmsnorm(x, t[("attn_norm", l)], cfg.rms_eps), 0, None))
+        mods.append(lambda x, l=l: O.mlp_module(
+            cfg, Wt, l, O.rmsnorm(x, t[("mlp_norm", l)], cfg.rms_eps)))
+    return mods
+
+
+def test_algorithm1_form_equals_equation2_form():
+    cfg = small_cfg(n_layers=3)
+    t = rand_weights(cfg, 11)
+    mods = _modules(cfg, t)
+    xs = [_x0(t, TOK)]
+    for m in range(1, 2 * cfg.n_layers + 1):
+        xs.append(xs[m - 1] + mods[m - 1](xs[max(m - 2, 0)]))           # Eq. 2
+    r = O.forward(cfg, W(t), TOK, record=True)
+    assert np.allclose(r.x_final, xs[-1], atol=1e-11)
+    for m in range(1, 2 * cfg.n_layers + 1):
+        assert np.allclose(r.module_inputs[m - 1], xs[max(m - 2, 0)], atol=1e-11)
+
+
+def test_standard_mask_equals_equation1():
+    cfg = small_cfg(n_layers=3, ladder=[0, 0, 0])
+    t = rand_weights(cfg, 12)
+    mods = _modules(cfg, t)
+    x = _x0(t, TOK)
+    for h in mods:
+        x = x + h(x)                                                     # Eq. 1
+    r = O.forward(cfg, W(t), TOK)
+    assert np.allclose(r.x_final, x, atol=1e-11)
+    lad = O.forward(small_cfg(n_layers=3), W(t), TOK)
+    assert not np.allclose(lad.x_final, x, atol=1e-3)                    # the two really differ
+
+
+def test_hybrid_boundary_reading():
+    # layers: standard, ladder, ladder, standard.  Inputs each module must read (x_k = stream after k adds):
+    cfg = small_cfg(n_layers=4, ladder=[0, 1, 1, 0])
+    t = rand_weights(cfg, 13)
+    mods = _modules(cfg, t)
+    reads = [0, 1, 2, 2, 3, 4, 6, 7]        # m=3 reads the complete stream, m=4..6 are stale, m=7,8 complete
+    xs = [_x0(t, TOK)]
+    for m in range(1, 9):
+        xs.append(xs[m - 1] + mods[m - 1](xs[reads[m - 1]]))
+    r = O.forward(cfg, W(t), TOK, record=True)
+    assert np.allclose(r.x_final, xs[-1], atol=1e-11)
+
+
+def test_single_live_module_ladder_equals_standard_bitwise():
+    for dead in ("w_down", "wo"):
+        cfg_l = small_cfg(n_layers=1)
+        cfg_s = small_cfg(n_layers=1, ladder=[0])
+        t = rand_weights(cfg_l, 14)
+        t[(dead, 0)] = np.zeros_like(t[(dead, 0)])
+        a = O.forward(cfg_l, W(t), TOK)
+        b = O.forward(cfg_s, W(t), TOK)
+        assert np.array_equal(a.hidden, b.hidden)
+        assert np.array_equal(a.logits, b.logits)
+
+
+def test_only_module_k_live_gives_x0_plus_hk_x0():
+    cfg = small_cfg(n_layers=3)
+    base = rand_weights(cfg, 15)
+    for k in range(1, 7):
+        t = dict(base)
+        for l in range(3):
+            if 2 * l + 1 != k:
+                t[("wo", l)] = np.zeros_like(base[("wo", l)])
+            if 2 * l + 2 != k:
+                t[("w_down", l)] = np.zeros_like(base[("w_down", l)])
+        x0 = _x0(t, TOK)
+        want = x0 + _modules(cfg, t)[k - 1](x0)
+        for ladder in (None, [0, 0, 0]):
+            cfg.layer_is_ladder = ladder
+            assert np.allclose(O.forward(cfg, W(t), TOK).x_final, want, atol=1e-11)
+        cfg.layer_is_ladder = None
+
+
+def test_telescoping_sum_of_module_outputs():
+    for ladder in (None, [0, 0, 0], [0, 1, 1]):
+        cfg = small_cfg(n_layers=3, ladder=ladder)
+        t = rand_weights(cfg, 16)
+        r = O.forward(cfg, W(t), TOK, record=True)
+        assert len(r.module_outputs) == 6
+        assert np.allclose(r.x_final, _x0(t, TOK) + sum(r.module_outputs), atol=1e-11)
+
+
+def test_staleness_is_one_module():
+    cfg = small_cfg(n_layers=3)
+    t = rand_weights(cfg, 17)
+    t2 = dict(t)
+    t2[("wo", 1)] = rand_weights(cfg, 99)[("wo", 1)]     # module 3 = attention of layer 1
+    for ladder, same_next in ((None, True), ([0, 0, 0], False)):
+        cfg.layer_is_ladder = ladder
+        a = O.forward(cfg, W(t), TOK, record=True).module_inputs
+        b = O.forward(cfg, W(t2), TOK, record=True).module_inputs
+        assert np.array_equal(a[2], b[2])                  # module 3 itself reads nothing it wrote
+        assert np.array_equal(a[3], b[3]) == same_next     # module 4: unchanged only under ladder
+        assert not np.array_equal(a[4], b[4])              # module 5 sees it in both
+    cfg.layer_is_ladder = None
+
+
+def test_zeroed_output_projections_closed_form():
+    cfg = small_cfg(n_layers=2)
+    t = rand_weights(cfg, 18)
+    for l in range(2):
+        t[("wo", l)] = np.zeros_like(t[("wo", l)])
+        t[("w_down", l)] = np.zeros_like(t[("w_down", l)])
+    r = O.forward(cfg, W(t), TOK)
+    x0 = _x0(t, TOK)
+    hid = x0 / np.sqrt((x0 ** 2).mean(-1, keepdims=True) + 1e-5) * t[("final_norm", None)]
+    assert np.allclose(r.hidden, hid, atol=1e-12)
+    logits = np.einsum("btd,vd->btv", hid, t[("lm_head", None)])
+    assert np.allclose(r.logits, logits, atol=1e-11)
+    assert np.array_equal(r.next_tokens, logits.argmax(-1))
+
+
+def test_greedy_lowest_index_on_ties():
+    assert O.greedy(np.array([[0.5, 2.0, 2.0, -1.0, 2.0]]))[0] == 1
+
+
+# ---------------------------------------------------------------- cache, causality, batching
+@pytest.mark.parametrize("ladder", [None, [0, 0, 0], [0, 1, 1]])
+def test_cached_decode_equals_full_recomputation(ladder):
+    cfg = small_cfg(n_layers=3, ladder=ladder)
+    t = rand_weights(cfg, 19)
+    S, steps = 4, 5
+    rng = np.random.default_rng(19)
+    seq = rng.integers(0, cfg.vocab_size, size=(2, S + steps))
+    cache = O.OracleCache(cfg, 2, S + steps)
+    r = O.prefill(cfg, W(t), seq[:, :S], cache)
+    full = O.forward(cfg, W(t), seq)
+    assert np.allclose(r.hidden[:, 0], full.hidden[:, S - 1], atol=1e-10)
+    for j in range(steps):
+        r = O.decode_step(cfg, W(t), seq[:, S + j], cache)
+        assert cache.seq_len == S + j + 1
+        assert np.allclose(r.hidden[:, 0], full.hidden[:, S + j], atol=1e-10)
+        assert np.allclose(r.logits[:, 0], full.logits[:, S + j], atol=1e-10)
+
+
+def test_generate_is_consistent_with_recomputation_and_teacher_forcing():
+    cfg = small_cfg(n_layers=2)
+    t = rand_weights(cfg, 20)
+    prompt = TOK[:, :4]
+    toks, hid = O.generate(cfg, W(t), prompt, 5, 16)
+    seq = np.concatenate([prompt, toks[:, :-1]], axis=1)
+    full = O.forward(cfg, W(t), seq)
+    assert np.array_equal(full.next_tokens[:, 3:], toks)
+    assert np.allclose(full.hidden[:, 3:], hid, atol=1e-10)
+    forced = np.array(toks)
+    forced[:, 2] = (forced[:, 2] + 1) % cfg.vocab_size
+    toks_f, _ = O.generate(cfg, W(t), prompt, 5, 16, forced=forced)
+    assert np.array_equal(toks_f[:, :3], toks[:, :3])      # history identical up to the forced change
+    seq_f = np.concatenate([prompt, forced[:, :-1]], axis=1)
+    assert np.array_equal(O.forward(cfg, W(t), seq_f).next_tokens[:, 3:], toks_f)
+
+
+def test_causality_bitwise():
+    cfg = small_cfg(n_layers=2)
+    t = rand_weights(cfg, 21)
+    a = O.forward(cfg, W(t), TOK)
+    tok2 = TOK.copy()
+    tok2[:, 4] = (tok2[:, 4] + 7) % cfg.vocab_size
+    b = O.forward(cfg, W(t), tok2)
+    assert np.array_equal(a.hidden[:, :4], b.hidden[:, :4])
+    assert not np.allclose(a.hidden[:, 4:], b.hidden[:, 4:])
+
+
+def test_batch_rows_are_independent():
+    cfg = small_cfg(n_layers=2)
+    t = rand_weights(cfg, 22)
+    both = O.forward(cfg, W(t), TOK)
+    for b in range(2):
+        one = O.forward(cfg, W(t), TOK[b:b + 1])
+        assert np.allclose(both.hidden[b], one.hidden[0], atol=1e-12)
+
+
+def test_float32_mode_tracks_float64():
+    cfg = small_cfg(n_layers=3)
+    t = rand_weights(cfg, 23)
+    a = O.forward(cfg, W(t), TOK, dtype=np.float64)
+    b = O.forward(cfg, W(t), TOK, dtype=np.float32)
+    assert b.hidden.dtype == np.float32
+    assert np.max(np.abs(a.hidden - b.hidden)) < 1e-4
+
+
+# ---------------------------------------------------------------- the paper's own arithmetic (Tab. 2)
+def test_table2_reading_latency_reduction_vs_throughput_gain():
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "table2_improvements.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    assert len(rows) == 6
+    for name, prefill, decode, toks in rows:
+        gain = 100.0 * (1.0 / (1.0 - float(decode) / 100.0) - 1.0)
+        # tokens/s gain is dominated by the decode latency reduction r: about 1/(1-r) - 1
+        assert abs(gain - float(toks)) < 1.0, (name, gain, toks)

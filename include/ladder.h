@@ -1,0 +1,199 @@
+/* libladder -- bf16 forward (prefill + autoregressive decode) of a Ladder-Residual /
+ * standard-residual / hybrid Llama-shaped transformer on ONE NVIDIA B200 (sm_100a).
+ *
+ * Plain C ABI: no C++ or torch types cross this boundary.  Unless a parameter says
+ * HOST, every data pointer is a DEVICE pointer on the current CUDA device.  All work is
+ * enqueued stream-ordered on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
+ * legacy default stream); an internal second stream, when enabled, is forked from and
+ * joined back to it with events, so callers see ordinary stream semantics.  No call
+ * synchronises the device unless its comment says so.
+ *
+ * Residual rules implemented (m = 1..2N indexes modules, odd = attention, even = MLP):
+ *   standard layer :  x_m = x_{m-1} + h_m(x_{m-1})                      (paper Sec. 2, Eq. 1)
+ *   ladder layer   :  x_m = x_{m-1} + h_m(x_{m-2})                      (paper Sec. 3.1, Eq. 2)
+ * in the pending-output form of the paper's Algorithm 1 with the all-reduce removed:
+ * initial pending outputs are zero (modules 1 and 2 both read x_0), outputs still pending
+ * after the last layer are added before the final norm, and a standard layer first adds
+ * whatever is pending and leaves nothing pending.  Each module h_m is pre-norm RMSNorm
+ * followed by grouped-query causal attention with rotary embedding on interleaved pairs,
+ * or by a SwiGLU MLP ("Llama-3's model architecture", paper Sec. 3.3.1).
+ *
+ * Numerics: bf16 weights, bf16 KV cache, bf16 GEMM operands, fp32 accumulation, fp32
+ * softmax, fp32 residual stream, fp32 logits.  Greedy argmax picks the lowest index on ties.
+ *
+ * Errors: every function returns a ladder_status_t; argument errors are detected on the
+ * host before anything is launched; nothing aborts, traps or hangs the device.
+ * A model object is not thread-safe; distinct objects are independent.
+ */
+#ifndef LADDER_H_
+#define LADDER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ladder_model ladder_model_t; /* opaque, owned by the library */
+
+typedef enum {
+  LADDER_OK = 0,
+  LADDER_ERR_INVALID_ARG = 1, /* NULL / out-of-range argument                          */
+  LADDER_ERR_UNSUPPORTED = 2, /* shape outside what the kernels handle (see create)    */
+  LADDER_ERR_OOM = 3,         /* workspace allocation failed                           */
+  LADDER_ERR_CUDA = 4,        /* a CUDA call failed (sticky; see ladder_last_error)    */
+  LADDER_ERR_STATE = 5        /* cache overflow, batch > max_batch, prefill on a non-empty position */
+} ladder_status_t;
+
+/* Bits of the device status word (ladder_device_status). */
+#define LADDER_DEV_BAD_TOKEN 1      /* a token id was outside [0, vocab): row treated as id 0 */
+#define LADDER_DEV_CACHE_OVERFLOW 2 /* a position >= max_seq_len reached a kernel: store skipped */
+
+typedef struct {
+  uint32_t struct_size; /* sizeof(ladder_config_t), for ABI versioning */
+  int32_t d_model, n_layers, n_q_heads, n_kv_heads, head_dim, d_ff, vocab_size;
+  float rms_eps, rope_theta;
+  int32_t max_batch;        /* largest batch of any call (decode kernels: <= 64)          */
+  int32_t max_seq_len;      /* cache capacity per sequence (prompt + generated)           */
+  int32_t max_prefill_tokens; /* largest batch*seq_len of a prefill call; 0 = max_batch*max_seq_len */
+  const uint8_t* layer_is_ladder; /* HOST, n_layers bytes, copied. NULL = all ladder; 0 = standard layer */
+} ladder_config_t;
+/* Shape limits (else LADDER_ERR_UNSUPPORTED): head_dim 64 or 128; n_q_heads % n_kv_heads == 0;
+ * d_model, n_q_heads*head_dim and d_ff multiples of 8; (n_q_heads+2 n_kv_heads)*head_dim,
+ * 2*d_ff, d_model and vocab_size multiples of 8. */
+
+/* Weights: bf16, row-major with the input (K) dimension contiguous, 16-byte aligned.
+ * BORROWED: the caller owns them and keeps them alive and unchanged until ladder_destroy;
+ * the library never writes, frees or copies them (a 70B model is ~141 GB). */
+typedef struct {
+  const void* tok_embedding;    /* [vocab, d_model]                                        */
+  const void* final_norm;       /* [d_model]                                               */
+  const void* lm_head;          /* [vocab, d_model] (untied)                               */
+  const void* const* attn_norm; /* HOST array[n_layers] of device ptrs, each [d_model]     */
+  const void* const* w_qkv;     /* [(Hq+2Hkv)*Dh, d_model]: Q heads, then K heads, then V  */
+  const void* const* w_o;       /* [d_model, Hq*Dh]                                        */
+  const void* const* mlp_norm;  /* [d_model]                                               */
+  const void* const* w_gate_up; /* [2*d_ff, d_model]: row 2j = gate_j, row 2j+1 = up_j      */
+  const void* const* w_down;    /* [d_model, d_ff]                                         */
+} ladder_weights_t;
+
+/* KV cache: caller-allocated, library reads and writes.  K holds post-rotation keys. */
+typedef struct {
+  void* k;           /* bf16 [n_layers][max_batch][n_kv_heads][max_seq_len][head_dim] */
+  void* v;           /* same shape                                                    */
+  int32_t* seq_lens; /* int32 [max_batch]: tokens cached per sequence; prefill sets it,
+                        each decode step reads the position from it and adds one        */
+} ladder_kv_cache_t;
+
+/* Outputs: all optional (NULL = not wanted), caller-owned device buffers. */
+typedef struct {
+  int32_t* next_tokens; /* [batch] greedy token                                            */
+  float* final_hidden;  /* [batch, d_model] final RMSNorm output at the last/current position */
+  float* logits;        /* [batch, vocab]                                                  */
+  float* all_hidden;    /* prefill only: [batch, seq_len, d_model] final RMSNorm at every position */
+} ladder_outputs_t;
+
+/* Bytes of ONE of the two cache buffers (k or v) for this configuration. */
+size_t ladder_kv_cache_bytes(const ladder_config_t* cfg);
+
+/* Validates the configuration, allocates the workspace (two fp32 residual buffers of
+ * max(max_batch, max_prefill_tokens) rows, activation scratch, split-KV partials, the
+ * rotary table), creates the second stream and events.  Allocates device memory and may
+ * synchronise.  On failure *out is NULL. */
+ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_weights_t* weights,
+                                    ladder_model_t** out);
+
+/* Decode scheduling (paper Sec. 3.2: side stream, CUDA graphs).
+ *   n_streams 1|2 : with 2, attention modules and MLP modules of ladder layers run on two
+ *                   streams with the event edges the ladder rule allows (module m's last GEMM
+ *                   waits for module m-1; everything before it does not); standard layers serialise.
+ *   use_graph 0|1 : capture one decode step as a CUDA graph and replay it.
+ *   use_pdl   0|1 : launch consecutive kernels of a stream with programmatic dependent launch so a
+ *                   kernel's weight prefetch starts before its predecessor has drained.
+ * Defaults: 2, 1, 1.  Results are bit-identical across all settings. */
+ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, int32_t use_graph, int32_t use_pdl);
+
+/* Prompt pass.  d_tokens int32 [batch, seq_len]; every sequence has the same length.
+ * Writes cache rows 0..seq_len-1 of sequences 0..batch-1, sets seq_lens[b] = seq_len, and
+ * produces outputs for position seq_len-1 (next_tokens = the first generated token).
+ * batch*seq_len <= max_prefill_tokens, seq_len <= max_seq_len, else LADDER_ERR_STATE. */
+ladder_status_t ladder_prefill(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                               int32_t batch, int32_t seq_len, const ladder_outputs_t* out, void* cuda_stream);
+
+/* One autoregressive step: consumes d_tokens int32 [batch] at position seq_lens[b] (read on
+ * the device), appends K/V there, attends over positions 0..seq_lens[b], writes the outputs and
+ * adds one to seq_lens[b].  d_tokens may alias out->next_tokens (device-side feedback loop).
+ * The library tracks the common length on the host (set by prefill / ladder_set_position) and
+ * returns LADDER_ERR_STATE instead of overflowing the cache. */
+ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                                   int32_t batch, const ladder_outputs_t* out, void* cuda_stream);
+
+/* Same step with HOST token buffers: copies h_tokens [batch] to the device, runs the step,
+ * copies the greedy tokens back to h_next_tokens [batch] and SYNCHRONISES the stream.
+ * Pinned host memory makes the copies asynchronous up to that final sync. */
+ladder_status_t ladder_decode_step_host(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* h_tokens,
+                                        int32_t batch, int32_t* h_next_tokens, void* cuda_stream);
+/* Prompt pass with HOST token buffers [batch, seq_len]; synchronises like the call above. */
+ladder_status_t ladder_prefill_host(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* h_tokens,
+                                    int32_t batch, int32_t seq_len, int32_t* h_next_tokens, void* cuda_stream);
+
+/* Tell the library that every sequence of the cache now holds `len` tokens (e.g. after the
+ * caller restored a cache snapshot or rewound seq_lens itself).  Host-side only. */
+ladder_status_t ladder_set_position(ladder_model_t* m, int32_t len);
+
+/* Synchronises `cuda_stream`, returns the device status word (LADDER_DEV_* bits) and clears it. */
+ladder_status_t ladder_device_status(ladder_model_t* m, int32_t* flags, void* cuda_stream);
+
+/* Number of kernels this model has enqueued so far (graph replays count their kernel nodes). */
+int64_t ladder_kernel_launches(const ladder_model_t* m);
+
+ladder_status_t ladder_destroy(ladder_model_t* m); /* NULL is fine */
+const char* ladder_status_string(ladder_status_t s);
+const char* ladder_last_error(const ladder_model_t* m); /* library-owned string; NULL model = last create error */
+
+/* ------------------------------------------------------------------------------------------
+ * Single-kernel entry points: the same kernels the model calls, exposed so each can be tested
+ * and profiled at its true shape.  They allocate nothing and do not synchronise.
+ * ------------------------------------------------------------------------------------------ */
+
+/* Weight-streaming small-M GEMM  acc[b,n] = sum_k act[b,k] * W[n,k]  (decode: M = batch <= 64),
+ * with the activation staging and the epilogue of one step of the decode path.
+ *   act_mode 0: act = bf16 [batch, K]                              (steps: output / down projection)
+ *            1: act = fp32 residual [batch, K]; the kernel applies RMSNorm with gain `gain`
+ *               bf16 [K] and eps (steps: fused RMSNorm + QKV / gate-up projection, LM head)
+ *   epi_mode 0: out_f32[b,n] = addend[b,n] + acc            (residual add; addend may equal out_f32)
+ *            1: out_bf16[b,j] = silu(acc[b,2j]) * acc[b,2j+1]      (SwiGLU over interleaved rows)
+ *            2: out_f32[b,n] = acc                                   (plain, e.g. logits)
+ * W bf16 [N,K] row-major; N % 8 == 0, K % 8 == 0, 1 <= batch <= 64. */
+ladder_status_t ladder_op_smallm_gemm(const void* W, int32_t N, int32_t K, const void* act, int32_t act_mode,
+                                      const void* gain, float eps, int32_t batch, int32_t epi_mode,
+                                      const float* addend, void* out, void* cuda_stream);
+
+/* Split-KV grouped-query decode attention for one layer.
+ *   q fp32 [batch, Hq*Dh] (already rotated); k,v bf16 [max_batch][Hkv][max_seq_len][Dh] (one layer);
+ *   kv_len int32 [batch] = number of keys to attend (positions 0..kv_len-1);
+ *   scratch fp32, at least ladder_decode_attention_scratch_bytes(...) bytes;
+ *   o bf16 [batch, Hq*Dh].  softmax(q.k/sqrt(Dh)) v per head, fp32 softmax and accumulation. */
+size_t ladder_decode_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim, int32_t max_seq_len);
+ladder_status_t ladder_op_decode_attention(const float* q, const void* k, const void* v, const int32_t* kv_len,
+                                           int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                           int32_t max_seq_len, float* scratch, void* o, void* cuda_stream);
+
+/* Large-M GEMM of the prefill path: C[m,n] = sum_k A[m,k] * W[n,k], A bf16 [M,K], W bf16 [N,K].
+ *   epi_mode 0: out_f32[m,n] = addend[m,n] + acc;  1: SwiGLU -> out_bf16 [M, N/2];
+ *            2: out_f32 = acc;  3: out_bf16[m,n] = acc.   K % 8 == 0, N % 8 == 0. */
+ladder_status_t ladder_op_prefill_gemm(const void* A, const void* W, int32_t M, int32_t N, int32_t K,
+                                       int32_t epi_mode, const float* addend, void* out, void* cuda_stream);
+
+/* Causal grouped-query attention of the prefill path for one layer:
+ *   q bf16 [batch, seq_len, Hq*Dh] (rotated); k,v bf16 cache of one layer as above, rows 0..seq_len-1
+ *   valid; o bf16 [batch, seq_len, Hq*Dh].  Query p attends keys t <= p. */
+ladder_status_t ladder_op_prefill_attention(const void* q, const void* k, const void* v, int32_t batch,
+                                            int32_t seq_len, int32_t n_q_heads, int32_t n_kv_heads,
+                                            int32_t head_dim, int32_t max_seq_len, void* o, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LADDER_H_ */

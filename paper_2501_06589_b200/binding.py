@@ -1,0 +1,257 @@
+"""ctypes binding of libladder.so: argument marshalling only.
+
+Every function here forwards to the C entry point of the same name declared in
+``include/ladder.h``; tensors are torch CUDA tensors used purely as device
+memory, and the CUDA stream is torch's current stream.  There is no fallback:
+if the library is missing, importing :func:`lib` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+from .synth import AbiWeights, ModelShape
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libladder.so")
+
+EXPORTS = [
+    "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_prefill",
+    "ladder_decode_step", "ladder_decode_step_host", "ladder_prefill_host", "ladder_set_position",
+    "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
+    "ladder_last_error", "ladder_op_smallm_gemm", "ladder_decode_attention_scratch_bytes",
+    "ladder_op_decode_attention", "ladder_op_prefill_gemm", "ladder_op_prefill_attention",
+]
+
+
+class LadderError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"libladder status {status}: {msg}")
+        self.status = status
+
+
+class ladder_config_t(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("d_model", C.c_int32), ("n_layers", C.c_int32),
+                ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("d_ff", C.c_int32), ("vocab_size", C.c_int32), ("rms_eps", C.c_float),
+                ("rope_theta", C.c_float), ("max_batch", C.c_int32), ("max_seq_len", C.c_int32),
+                ("max_prefill_tokens", C.c_int32), ("layer_is_ladder", C.POINTER(C.c_uint8))]
+
+
+class ladder_weights_t(C.Structure):
+    _fields_ = [("tok_embedding", C.c_void_p), ("final_norm", C.c_void_p), ("lm_head", C.c_void_p),
+                ("attn_norm", C.POINTER(C.c_void_p)), ("w_qkv", C.POINTER(C.c_void_p)),
+                ("w_o", C.POINTER(C.c_void_p)), ("mlp_norm", C.POINTER(C.c_void_p)),
+                ("w_gate_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p))]
+
+
+class ladder_kv_cache_t(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("seq_lens", C.c_void_p)]
+
+
+class ladder_outputs_t(C.Structure):
+    _fields_ = [("next_tokens", C.c_void_p), ("final_hidden", C.c_void_p), ("logits", C.c_void_p),
+                ("all_hidden", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libladder.so (built in-tree by paper_2501_06589_b200.build); fails loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} not built: run `python -m paper_2501_06589_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        L.ladder_kv_cache_bytes.restype = C.c_size_t
+        L.ladder_kv_cache_bytes.argtypes = [C.POINTER(ladder_config_t)]
+        L.ladder_model_create.argtypes = [C.POINTER(ladder_config_t), C.POINTER(ladder_weights_t),
+                                          C.POINTER(C.c_void_p)]
+        L.ladder_model_set_schedule.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32]
+        L.ladder_prefill.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32, C.c_int32,
+                                     C.POINTER(ladder_outputs_t), C.c_void_p]
+        L.ladder_decode_step.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32,
+                                         C.POINTER(ladder_outputs_t), C.c_void_p]
+        L.ladder_decode_step_host.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32,
+                                              C.c_void_p, C.c_void_p]
+        L.ladder_prefill_host.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32,
+                                          C.c_int32, C.c_void_p, C.c_void_p]
+        L.ladder_set_position.argtypes = [C.c_void_p, C.c_int32]
+        L.ladder_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.c_void_p]
+        L.ladder_kernel_launches.restype = C.c_int64
+        L.ladder_kernel_launches.argtypes = [C.c_void_p]
+        L.ladder_destroy.argtypes = [C.c_void_p]
+        L.ladder_status_string.restype = C.c_char_p
+        L.ladder_status_string.argtypes = [C.c_int]
+        L.ladder_last_error.restype = C.c_char_p
+        L.ladder_last_error.argtypes = [C.c_void_p]
+        L.ladder_op_smallm_gemm.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
+                                            C.c_float, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ladder_decode_attention_scratch_bytes.restype = C.c_size_t
+        L.ladder_decode_attention_scratch_bytes.argtypes = [C.c_int32] * 4
+        L.ladder_op_decode_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                                 C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                                 C.c_void_p, C.c_void_p]
+        L.ladder_op_prefill_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                             C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ladder_op_prefill_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                                  C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                                  C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(status: int, model=None):
+    if status != 0:
+        L = lib()
+        msg = L.ladder_status_string(status).decode()
+        detail = L.ladder_last_error(model).decode() if True else ""
+        raise LadderError(status, f"{msg}: {detail}")
+
+
+def make_config(shape: ModelShape, max_batch: int, max_seq_len: int, max_prefill_tokens: int = 0):
+    mask = (C.c_uint8 * shape.n_layers)(*shape.ladder_mask())
+    cfg = ladder_config_t(C.sizeof(ladder_config_t), shape.d_model, shape.n_layers, shape.n_q_heads,
+                          shape.n_kv_heads, shape.head_dim, shape.d_ff, shape.vocab_size, shape.rms_eps,
+                          shape.rope_theta, max_batch, max_seq_len, max_prefill_tokens,
+                          C.cast(mask, C.POINTER(C.c_uint8)))
+    cfg._keep = mask
+    return cfg
+
+
+class KVCache:
+    """Caller-owned cache buffers (torch device memory) for one model configuration."""
+
+    def __init__(self, shape: ModelShape, max_batch: int, max_seq_len: int, device="cuda", fill: Optional[int] = None):
+        n = shape.n_layers * max_batch * shape.n_kv_heads * max_seq_len * shape.head_dim
+        self.k = torch.empty(n, dtype=torch.bfloat16, device=device)
+        self.v = torch.empty(n, dtype=torch.bfloat16, device=device)
+        if fill is not None:       # canary pattern for indexing tests
+            self.k.view(torch.int16).fill_(fill)
+            self.v.view(torch.int16).fill_(fill)
+        self.seq_lens = torch.zeros(max_batch, dtype=torch.int32, device=device)
+        self.dims = (shape.n_layers, max_batch, shape.n_kv_heads, max_seq_len, shape.head_dim)
+        self.c = ladder_kv_cache_t(self.k.data_ptr(), self.v.data_ptr(), self.seq_lens.data_ptr())
+
+    def k5(self) -> torch.Tensor:
+        return self.k.view(*self.dims)
+
+    def v5(self) -> torch.Tensor:
+        return self.v.view(*self.dims)
+
+
+class Model:
+    """Owns a ladder_model_t; keeps the borrowed weight tensors alive."""
+
+    def __init__(self, weights: AbiWeights, max_batch: int, max_seq_len: int, max_prefill_tokens: int = 0):
+        L = lib()
+        s = weights.shape
+        self.shape, self.weights = s, weights
+        self.max_batch, self.max_seq_len = max_batch, max_seq_len
+        self._cfg = make_config(s, max_batch, max_seq_len, max_prefill_tokens)
+
+        def arr(ts: Sequence[torch.Tensor]):
+            return (C.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+
+        self._arrs = [arr(weights.attn_norm), arr(weights.w_qkv), arr(weights.w_o), arr(weights.mlp_norm),
+                      arr(weights.w_gate_up), arr(weights.w_down)]
+        w = ladder_weights_t(weights.tok_embedding.data_ptr(), weights.final_norm.data_ptr(),
+                             weights.lm_head.data_ptr(), *[C.cast(a, C.POINTER(C.c_void_p)) for a in self._arrs])
+        h = C.c_void_p()
+        _check(L.ladder_model_create(C.byref(self._cfg), C.byref(w), C.byref(h)))
+        self.h = h
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().ladder_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_schedule(self, n_streams: int = 2, use_graph: bool = True, use_pdl: bool = True):
+        _check(lib().ladder_model_set_schedule(self.h, n_streams, int(use_graph), int(use_pdl)), self.h)
+
+    def set_position(self, length: int):
+        _check(lib().ladder_set_position(self.h, length), self.h)
+
+    def device_status(self) -> int:
+        f = C.c_int32(0)
+        _check(lib().ladder_device_status(self.h, C.byref(f), _stream()), self.h)
+        return f.value
+
+    def kernel_launches(self) -> int:
+        return int(lib().ladder_kernel_launches(self.h))
+
+    @staticmethod
+    def _outs(next_tokens=None, final_hidden=None, logits=None, all_hidden=None):
+        return ladder_outputs_t(_ptr(next_tokens), _ptr(final_hidden), _ptr(logits), _ptr(all_hidden))
+
+    def prefill(self, cache: KVCache, tokens: torch.Tensor, next_tokens=None, final_hidden=None, logits=None,
+                all_hidden=None):
+        assert tokens.dtype == torch.int32 and tokens.is_cuda and tokens.dim() == 2
+        o = self._outs(next_tokens, final_hidden, logits, all_hidden)
+        _check(lib().ladder_prefill(self.h, C.byref(cache.c), _ptr(tokens), tokens.shape[0], tokens.shape[1],
+                                    C.byref(o), _stream()), self.h)
+
+    def decode_step(self, cache: KVCache, tokens: torch.Tensor, next_tokens=None, final_hidden=None, logits=None):
+        assert tokens.dtype == torch.int32 and tokens.is_cuda
+        o = self._outs(next_tokens, final_hidden, logits)
+        _check(lib().ladder_decode_step(self.h, C.byref(cache.c), _ptr(tokens), tokens.numel(), C.byref(o),
+                                        _stream()), self.h)
+
+    def decode_step_host(self, cache: KVCache, h_tokens: torch.Tensor, h_next: torch.Tensor):
+        assert not h_tokens.is_cuda and not h_next.is_cuda and h_tokens.dtype == torch.int32
+        _check(lib().ladder_decode_step_host(self.h, C.byref(cache.c), h_tokens.data_ptr(), h_tokens.numel(),
+                                             h_next.data_ptr(), _stream()), self.h)
+
+    def prefill_host(self, cache: KVCache, h_tokens: torch.Tensor, h_next: torch.Tensor):
+        assert not h_tokens.is_cuda and h_tokens.dtype == torch.int32 and h_tokens.dim() == 2
+        _check(lib().ladder_prefill_host(self.h, C.byref(cache.c), h_tokens.data_ptr(), h_tokens.shape[0],
+                                         h_tokens.shape[1], h_next.data_ptr(), _stream()), self.h)
+
+
+# ----------------------------------------------------------------------------- single-kernel entry points
+def op_smallm_gemm(W: torch.Tensor, act: torch.Tensor, act_mode: int, epi_mode: int, out: torch.Tensor,
+                   gain: Optional[torch.Tensor] = None, eps: float = 1e-5, addend: Optional[torch.Tensor] = None):
+    N, K = W.shape
+    _check(lib().ladder_op_smallm_gemm(_ptr(W), N, K, _ptr(act), act_mode, _ptr(gain), eps, act.shape[0], epi_mode,
+                                       _ptr(addend), _ptr(out), _stream()))
+
+
+def decode_attention_scratch_bytes(batch: int, n_q_heads: int, head_dim: int, max_seq_len: int) -> int:
+    return int(lib().ladder_decode_attention_scratch_bytes(batch, n_q_heads, head_dim, max_seq_len))
+
+
+def op_decode_attention(q, k, v, kv_len, n_q_heads, n_kv_heads, head_dim, max_seq_len, scratch, o):
+    _check(lib().ladder_op_decode_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_len), q.shape[0], n_q_heads,
+                                            n_kv_heads, head_dim, max_seq_len, _ptr(scratch), _ptr(o), _stream()))
+
+
+def op_prefill_gemm(A, W, epi_mode: int, out, addend=None):
+    M, K = A.shape
+    N = W.shape[0]
+    _check(lib().ladder_op_prefill_gemm(_ptr(A), _ptr(W), M, N, K, epi_mode, _ptr(addend), _ptr(out), _stream()))
+
+
+def op_prefill_attention(q, k, v, batch, seq_len, n_q_heads, n_kv_heads, head_dim, max_seq_len, o):
+    _check(lib().ladder_op_prefill_attention(_ptr(q), _ptr(k), _ptr(v), batch, seq_len, n_q_heads, n_kv_heads,
+                                             head_dim, max_seq_len, _ptr(o), _stream()))

@@ -1,0 +1,839 @@
+// C ABI of libladder: model object, module scheduler (residual routing, two streams,
+// CUDA graph of the decode step) and the single-kernel entry points.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/ladder.h"
+#include "kernels.h"
+
+using namespace ladder;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+bool g_kernels_ready = false;
+cudaError_t kernels_ready() {  // opt-in to large dynamic shared memory, once per process
+  if (g_kernels_ready) return cudaSuccess;
+  cudaError_t e = smallm_gemm_init();
+  if (e == cudaSuccess) e = largem_gemm_init();
+  if (e == cudaSuccess) e = prefill_attention_init();
+  if (e == cudaSuccess) g_kernels_ready = true;
+  return e;
+}
+
+struct GraphKey {
+  int batch = 0, n_streams = 0, pdl = 0;
+  const void *k = nullptr, *v = nullptr, *lens = nullptr, *tok = nullptr;
+  const void *o_next = nullptr, *o_hid = nullptr, *o_logits = nullptr;
+  bool operator==(const GraphKey& o) const {
+    return batch == o.batch && n_streams == o.n_streams && pdl == o.pdl && k == o.k && v == o.v && lens == o.lens &&
+           tok == o.tok && o_next == o.o_next && o_hid == o.o_hid && o_logits == o.o_logits;
+  }
+};
+
+}  // namespace
+
+struct ladder_model {
+  ladder_config_t cfg;
+  std::vector<uint8_t> is_ladder;
+  const __nv_bfloat16 *tok_embedding, *final_norm, *lm_head;
+  std::vector<const __nv_bfloat16*> attn_norm, w_qkv, w_o, mlp_norm, w_gate_up, w_down;
+  int sm_count = 0;
+  int max_rows = 0;  // rows of the residual buffers
+  // workspace (device)
+  float* R[2] = {nullptr, nullptr};
+  float* q_f32 = nullptr;           // decode [max_batch, Hq*Dh]
+  __nv_bfloat16* o_dec = nullptr;   // decode [max_batch, Hq*Dh]
+  __nv_bfloat16* h_dec = nullptr;   // decode [max_batch, F]
+  float* attn_scratch = nullptr;
+  int attn_splits = 1;
+  float* logits_ws = nullptr;       // [max_batch, V]
+  float* last_x = nullptr;          // [max_batch, d]
+  __nv_bfloat16 *n_pf = nullptr, *q_pf = nullptr, *o_pf = nullptr, *h_pf = nullptr;  // prefill activations
+  float2* rope = nullptr;
+  int32_t* status = nullptr;
+  int32_t *tok_tmp = nullptr, *next_tmp = nullptr;
+  // scheduling
+  cudaStream_t side = nullptr, cap = nullptr;
+  std::vector<cudaEvent_t> ev;  // ev[m] = end of module m (m = 0: embedding)
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  int n_streams = 2, use_graph = 1, use_pdl = 1;
+  cudaGraphExec_t graph_exec = nullptr;
+  GraphKey graph_key;
+  int64_t graph_kernels = 0;
+  // state
+  int host_len = 0;
+  int64_t launches = 0;
+  std::string err;
+  bool sticky_cuda = false;
+};
+
+namespace {
+
+ladder_status_t fail(ladder_model* m, ladder_status_t s, const std::string& msg) {
+  if (m) m->err = msg;
+  else g_create_error = msg;
+  return s;
+}
+
+#define CK(m, call)                                                                                   \
+  do {                                                                                                \
+    cudaError_t e_ = (call);                                                                          \
+    if (e_ != cudaSuccess) {                                                                          \
+      if (m) (m)->sticky_cuda = true;                                                                 \
+      return fail(m, LADDER_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_));            \
+    }                                                                                                 \
+  } while (0)
+
+template <typename T>
+cudaError_t dev_alloc(T** p, size_t count) {
+  return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T) + 256);
+}
+
+const char* check_shape(const ladder_config_t& c) {
+  if (c.d_model <= 0 || c.n_layers <= 0 || c.n_q_heads <= 0 || c.n_kv_heads <= 0 || c.d_ff <= 0 || c.vocab_size <= 0)
+    return "non-positive dimension";
+  if (c.head_dim != 64 && c.head_dim != 128) return "head_dim must be 64 or 128";
+  if (c.n_q_heads % c.n_kv_heads) return "n_q_heads must be a multiple of n_kv_heads";
+  if (c.d_model % 8 || c.d_ff % 8 || c.vocab_size % 8) return "d_model, d_ff and vocab_size must be multiples of 8";
+  if (c.max_batch < 1 || c.max_batch > 64) return "max_batch must be in [1, 64]";
+  if (c.max_seq_len < 1) return "max_seq_len must be positive";
+  if (!(c.rms_eps >= 0.f) || !(c.rope_theta > 0.f)) return "bad rms_eps / rope_theta";
+  return nullptr;
+}
+
+// Residual routing (Eq. 1 / Eq. 2 of the paper on two ping-pong buffers).
+struct Router {
+  int cur = 0, stale = -1;  // buffer holding x_{m-1}; buffer holding x_{m-2} (or -1)
+  int writer[2] = {0, -1};  // module that last wrote each buffer
+  struct Route {
+    int in, add, dst, in_writer;
+  };
+  Route next(bool ladder, int module) {
+    Route r;
+    if (ladder && stale >= 0) {
+      r = {stale, cur, stale, writer[stale]};
+      const int old_cur = cur;
+      cur = stale;
+      stale = old_cur;
+    } else if (ladder) {
+      r = {cur, cur, cur ^ 1, writer[cur]};
+      stale = cur;
+      cur ^= 1;
+    } else {
+      r = {cur, cur, cur, writer[cur]};
+      stale = -1;
+    }
+    writer[r.dst] = module;
+    return r;
+  }
+};
+
+struct Enqueue {
+  ladder_model* m;
+  cudaStream_t sA, sB;
+  bool two;
+  bool pdl_ok[2] = {false, false};  // previous op on the stream was a kernel (programmatic edge possible)
+  int64_t kernels = 0;
+  cudaError_t err = cudaSuccess;
+
+  cudaStream_t stream(int s) const { return s ? sB : sA; }
+  bool pdl(int s) const { return m->use_pdl && pdl_ok[two ? s : 0]; }
+  void launched(int s, cudaError_t e) {
+    if (err == cudaSuccess) err = e;
+    pdl_ok[two ? s : 0] = true;
+    ++kernels;
+  }
+  void wait(int s, cudaEvent_t ev_from_other) {
+    if (!two) return;
+    cudaError_t e = cudaStreamWaitEvent(stream(s), ev_from_other, 0);
+    if (err == cudaSuccess) err = e;
+    pdl_ok[s] = false;
+  }
+  void record(int s, cudaEvent_t e) {
+    if (!two) return;
+    cudaError_t r = cudaEventRecord(e, stream(s));
+    if (err == cudaSuccess) err = r;
+  }
+};
+
+// One decode step: enqueue every kernel on sA (attention modules, head) and sB (MLP modules).
+cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int batch,
+                           const ladder_outputs_t* out, cudaStream_t sA, cudaStream_t sB, int64_t* n_kernels) {
+  const ladder_config_t& c = m->cfg;
+  Enqueue q{m, sA, sB, sA != sB};
+  const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff;
+  const size_t layer_elems = static_cast<size_t>(c.max_batch) * Hkv * c.max_seq_len * Dh;
+
+  q.launched(0, launch_embed(d_tokens, m->tok_embedding, batch, d, c.vocab_size, m->R[0], m->status, sA, false));
+  q.pdl_ok[0] = true;
+  q.record(0, m->ev[0]);
+  bool b_joined = false;  // has sB been ordered after the embedding yet
+
+  Router rt;
+  int last_wait[2] = {0, -1};  // latest module each stream has (transitively) waited for
+  auto need = [&](int s, int module) {
+    // make stream s wait for the end of `module` unless that is already implied
+    if (!q.two) return;
+    const int owner = module == 0 ? 0 : ((module & 1) ? 0 : 1);
+    if (owner == s) return;  // same stream: program order
+    if (last_wait[s] >= module) return;
+    q.wait(s, m->ev[module]);
+    last_wait[s] = module;
+    if (s == 1) b_joined = true;
+  };
+
+  for (int l = 0; l < c.n_layers; ++l) {
+    const bool lad = m->is_ladder[l] != 0;
+    // ---------------- attention module (module index 2l+1) on stream A
+    {
+      const int mod = 2 * l + 1;
+      const Router::Route r = rt.next(lad, mod);
+      need(0, r.in_writer);
+      SmallMParams p = {};
+      p.W = m->w_qkv[l];
+      p.N = (Hq + 2 * Hkv) * Dh;
+      p.K = d;
+      p.act = m->R[r.in];
+      p.act_mode = ACT_F32_NORM;
+      p.gain = m->attn_norm[l];
+      p.eps = c.rms_eps;
+      p.batch = batch;
+      p.epi_mode = EPI_QKV_ROPE;
+      p.qkv.q_out_f32 = m->q_f32;
+      p.qkv.k_cache = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
+      p.qkv.v_cache = static_cast<__nv_bfloat16*>(cache->v) + l * layer_elems;
+      p.qkv.seq_lens = cache->seq_lens;
+      p.qkv.rope = m->rope;
+      p.qkv.n_q_heads = Hq;
+      p.qkv.n_kv_heads = Hkv;
+      p.qkv.head_dim = Dh;
+      p.qkv.max_seq_len = c.max_seq_len;
+      p.status = m->status;
+      q.launched(0, launch_smallm_gemm(p, sA, q.pdl(0), m->sm_count));
+
+      DecodeAttnParams a = {};
+      a.q = m->q_f32;
+      a.k = p.qkv.k_cache;
+      a.v = p.qkv.v_cache;
+      a.kv_len = cache->seq_lens;
+      a.kv_len_offset = 1;
+      a.batch = batch;
+      a.n_q_heads = Hq;
+      a.n_kv_heads = Hkv;
+      a.head_dim = Dh;
+      a.max_seq_len = c.max_seq_len;
+      a.n_splits = m->attn_splits;
+      a.max_len = c.max_seq_len;
+      a.scratch = m->attn_scratch;
+      a.o = m->o_dec;
+      q.launched(0, launch_decode_attention(a, sA, q.pdl(0)));
+
+      need(0, mod - 1);  // the epilogue reads x_{m-1} and overwrites the buffer of x_{m-2}
+      SmallMParams o = {};
+      o.W = m->w_o[l];
+      o.N = d;
+      o.K = Hq * Dh;
+      o.act = m->o_dec;
+      o.act_mode = ACT_BF16;
+      o.batch = batch;
+      o.epi_mode = EPI_RESID;
+      o.addend = m->R[r.add];
+      o.out = m->R[r.dst];
+      o.status = m->status;
+      q.launched(0, launch_smallm_gemm(o, sA, q.pdl(0), m->sm_count));
+      q.record(0, m->ev[mod]);
+    }
+    // ---------------- MLP module (module index 2l+2) on stream B
+    {
+      const int mod = 2 * l + 2;
+      const Router::Route r = rt.next(lad, mod);
+      need(1, r.in_writer);
+      if (q.two && !b_joined) {  // first use of sB in this step: order it after the embedding
+        q.wait(1, m->ev[0]);
+        b_joined = true;
+      }
+      SmallMParams p = {};
+      p.W = m->w_gate_up[l];
+      p.N = 2 * F;
+      p.K = d;
+      p.act = m->R[r.in];
+      p.act_mode = ACT_F32_NORM;
+      p.gain = m->mlp_norm[l];
+      p.eps = c.rms_eps;
+      p.batch = batch;
+      p.epi_mode = EPI_SWIGLU;
+      p.out = m->h_dec;
+      p.status = m->status;
+      q.launched(1, launch_smallm_gemm(p, q.stream(1), q.pdl(1), m->sm_count));
+
+      need(1, mod - 1);
+      SmallMParams o = {};
+      o.W = m->w_down[l];
+      o.N = d;
+      o.K = F;
+      o.act = m->h_dec;
+      o.act_mode = ACT_BF16;
+      o.batch = batch;
+      o.epi_mode = EPI_RESID;
+      o.addend = m->R[r.add];
+      o.out = m->R[r.dst];
+      o.status = m->status;
+      q.launched(1, launch_smallm_gemm(o, q.stream(1), q.pdl(1), m->sm_count));
+      q.record(1, m->ev[mod]);
+    }
+  }
+  // ---------------- head on stream A (joins stream B)
+  need(0, 2 * c.n_layers);
+  const float* xf = m->R[rt.cur];
+  float* logits = (out && out->logits) ? out->logits : m->logits_ws;
+  SmallMParams h = {};
+  h.W = m->lm_head;
+  h.N = c.vocab_size;
+  h.K = d;
+  h.act = xf;
+  h.act_mode = ACT_F32_NORM;
+  h.gain = m->final_norm;
+  h.eps = c.rms_eps;
+  h.batch = batch;
+  h.epi_mode = EPI_PLAIN;
+  h.out = logits;
+  h.status = m->status;
+  q.launched(0, launch_smallm_gemm(h, sA, q.pdl(0), m->sm_count));
+  if (out && out->final_hidden)
+    q.launched(0, launch_rmsnorm_f32(xf, m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, sA, q.pdl(0)));
+  q.launched(0, launch_argmax_advance(logits, batch, c.vocab_size, out ? out->next_tokens : nullptr, cache->seq_lens, 1,
+                                      -1, sA, q.pdl(0)));
+  *n_kernels = q.kernels;
+  return q.err;
+}
+
+cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int batch, int S,
+                            const ladder_outputs_t* out, cudaStream_t st, int64_t* n_kernels) {
+  const ladder_config_t& c = m->cfg;
+  const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff;
+  const int M = batch * S;
+  const size_t layer_elems = static_cast<size_t>(c.max_batch) * Hkv * c.max_seq_len * Dh;
+  int64_t k = 0;
+  cudaError_t err = cudaSuccess;
+  auto did = [&](cudaError_t e) {
+    if (err == cudaSuccess) err = e;
+    ++k;
+  };
+  did(launch_embed(d_tokens, m->tok_embedding, M, d, c.vocab_size, m->R[0], m->status, st, false));
+  Router rt;
+  for (int l = 0; l < c.n_layers; ++l) {
+    const bool lad = m->is_ladder[l] != 0;
+    {
+      const Router::Route r = rt.next(lad, 2 * l + 1);
+      did(launch_rmsnorm_bf16(m->R[r.in], m->attn_norm[l], c.rms_eps, M, d, m->n_pf, st));
+      LargeMParams p = {};
+      p.A = m->n_pf;
+      p.W = m->w_qkv[l];
+      p.M = M;
+      p.N = (Hq + 2 * Hkv) * Dh;
+      p.K = d;
+      p.epi_mode = EPI_QKV_ROPE;
+      p.qkv.q_out_bf16 = m->q_pf;
+      p.qkv.k_cache = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
+      p.qkv.v_cache = static_cast<__nv_bfloat16*>(cache->v) + l * layer_elems;
+      p.qkv.rope = m->rope;
+      p.qkv.n_q_heads = Hq;
+      p.qkv.n_kv_heads = Hkv;
+      p.qkv.head_dim = Dh;
+      p.qkv.max_seq_len = c.max_seq_len;
+      p.qkv.prefill_seq_len = S;
+      did(launch_largem_gemm(p, st));
+      did(launch_prefill_attention(m->q_pf, p.qkv.k_cache, p.qkv.v_cache, batch, S, Hq, Hkv, Dh, c.max_seq_len, m->o_pf,
+                                   st));
+      LargeMParams o = {};
+      o.A = m->o_pf;
+      o.W = m->w_o[l];
+      o.M = M;
+      o.N = d;
+      o.K = Hq * Dh;
+      o.epi_mode = EPI_RESID;
+      o.addend = m->R[r.add];
+      o.out = m->R[r.dst];
+      did(launch_largem_gemm(o, st));
+    }
+    {
+      const Router::Route r = rt.next(lad, 2 * l + 2);
+      did(launch_rmsnorm_bf16(m->R[r.in], m->mlp_norm[l], c.rms_eps, M, d, m->n_pf, st));
+      LargeMParams p = {};
+      p.A = m->n_pf;
+      p.W = m->w_gate_up[l];
+      p.M = M;
+      p.N = 2 * F;
+      p.K = d;
+      p.epi_mode = EPI_SWIGLU;
+      p.out = m->h_pf;
+      did(launch_largem_gemm(p, st));
+      LargeMParams o = {};
+      o.A = m->h_pf;
+      o.W = m->w_down[l];
+      o.M = M;
+      o.N = d;
+      o.K = F;
+      o.epi_mode = EPI_RESID;
+      o.addend = m->R[r.add];
+      o.out = m->R[r.dst];
+      did(launch_largem_gemm(o, st));
+    }
+  }
+  const float* xf = m->R[rt.cur];
+  if (out && out->all_hidden) did(launch_rmsnorm_f32(xf, m->final_norm, c.rms_eps, M, d, d, out->all_hidden, st, false));
+  did(launch_gather_rows(xf, batch, d, S, S - 1, m->last_x, st));
+  float* logits = (out && out->logits) ? out->logits : m->logits_ws;
+  SmallMParams h = {};
+  h.W = m->lm_head;
+  h.N = c.vocab_size;
+  h.K = d;
+  h.act = m->last_x;
+  h.act_mode = ACT_F32_NORM;
+  h.gain = m->final_norm;
+  h.eps = c.rms_eps;
+  h.batch = batch;
+  h.epi_mode = EPI_PLAIN;
+  h.out = logits;
+  h.status = m->status;
+  did(launch_smallm_gemm(h, st, false, m->sm_count));
+  if (out && out->final_hidden)
+    did(launch_rmsnorm_f32(m->last_x, m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, st, false));
+  did(launch_argmax_advance(logits, batch, c.vocab_size, out ? out->next_tokens : nullptr, cache->seq_lens, 0, S, st,
+                            false));
+  *n_kernels = k;
+  return err;
+}
+
+void drop_graph(ladder_model* m) {
+  if (m->graph_exec) cudaGraphExecDestroy(m->graph_exec);
+  m->graph_exec = nullptr;
+  m->graph_key = GraphKey();
+}
+
+}  // namespace
+
+// =========================================================================== C ABI
+extern "C" {
+
+const char* ladder_status_string(ladder_status_t s) {
+  switch (s) {
+    case LADDER_OK: return "ok";
+    case LADDER_ERR_INVALID_ARG: return "invalid argument";
+    case LADDER_ERR_UNSUPPORTED: return "unsupported configuration";
+    case LADDER_ERR_OOM: return "out of device memory";
+    case LADDER_ERR_CUDA: return "CUDA error";
+    case LADDER_ERR_STATE: return "invalid state (cache overflow / batch too large)";
+    default: return "unknown status";
+  }
+}
+
+const char* ladder_last_error(const ladder_model_t* m) { return m ? m->err.c_str() : g_create_error.c_str(); }
+
+size_t ladder_kv_cache_bytes(const ladder_config_t* c) {
+  if (!c) return 0;
+  return static_cast<size_t>(c->n_layers) * c->max_batch * c->n_kv_heads * c->max_seq_len * c->head_dim * 2;
+}
+
+ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_weights_t* w, ladder_model_t** out) {
+  if (out) *out = nullptr;
+  if (!cfg || !w || !out) return fail(nullptr, LADDER_ERR_INVALID_ARG, "NULL argument");
+  if (cfg->struct_size != sizeof(ladder_config_t)) return fail(nullptr, LADDER_ERR_INVALID_ARG, "struct_size mismatch");
+  if (const char* why = check_shape(*cfg)) return fail(nullptr, LADDER_ERR_UNSUPPORTED, why);
+  if (!w->tok_embedding || !w->final_norm || !w->lm_head || !w->attn_norm || !w->w_qkv || !w->w_o || !w->mlp_norm ||
+      !w->w_gate_up || !w->w_down)
+    return fail(nullptr, LADDER_ERR_INVALID_ARG, "NULL weight pointer");
+  ladder_model* m = new ladder_model();
+  m->cfg = *cfg;
+  m->cfg.layer_is_ladder = nullptr;
+  const int L = cfg->n_layers;
+  m->is_ladder.assign(L, 1);
+  if (cfg->layer_is_ladder)
+    for (int l = 0; l < L; ++l) m->is_ladder[l] = cfg->layer_is_ladder[l] ? 1 : 0;
+  m->tok_embedding = static_cast<const __nv_bfloat16*>(w->tok_embedding);
+  m->final_norm = static_cast<const __nv_bfloat16*>(w->final_norm);
+  m->lm_head = static_cast<const __nv_bfloat16*>(w->lm_head);
+  auto grab = [&](const void* const* src, std::vector<const __nv_bfloat16*>& dst) -> bool {
+    dst.resize(L);
+    for (int l = 0; l < L; ++l) {
+      dst[l] = static_cast<const __nv_bfloat16*>(src[l]);
+      if (!dst[l] || (reinterpret_cast<uintptr_t>(dst[l]) & 15)) return false;
+    }
+    return true;
+  };
+  if (!grab(w->attn_norm, m->attn_norm) || !grab(w->w_qkv, m->w_qkv) || !grab(w->w_o, m->w_o) ||
+      !grab(w->mlp_norm, m->mlp_norm) || !grab(w->w_gate_up, m->w_gate_up) || !grab(w->w_down, m->w_down)) {
+    delete m;
+    return fail(nullptr, LADDER_ERR_INVALID_ARG, "NULL or misaligned (16 B) per-layer weight pointer");
+  }
+  if ((reinterpret_cast<uintptr_t>(m->tok_embedding) | reinterpret_cast<uintptr_t>(m->final_norm) |
+       reinterpret_cast<uintptr_t>(m->lm_head)) & 15) {
+    delete m;
+    return fail(nullptr, LADDER_ERR_INVALID_ARG, "misaligned (16 B) weight pointer");
+  }
+  const ladder_config_t& c = m->cfg;
+  if (m->cfg.max_prefill_tokens <= 0) m->cfg.max_prefill_tokens = c.max_batch * c.max_seq_len;
+  m->max_rows = c.max_prefill_tokens > c.max_batch ? c.max_prefill_tokens : c.max_batch;
+
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&m->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  int smem_optin = 0;
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e == cudaSuccess) e = kernels_ready();
+  if (e != cudaSuccess) {
+    delete m;
+    return fail(nullptr, LADDER_ERR_CUDA, std::string("device query: ") + cudaGetErrorString(e));
+  }
+  if (static_cast<size_t>(smem_optin) < smallm_gemm_smem_bytes(c.max_batch)) {
+    delete m;
+    return fail(nullptr, LADDER_ERR_UNSUPPORTED, "device has too little shared memory per block (needs sm_100-class)");
+  }
+
+  const size_t rows = m->max_rows, d = c.d_model, qd = static_cast<size_t>(c.n_q_heads) * c.head_dim, F = c.d_ff;
+  const size_t MB = c.max_batch, MP = c.max_prefill_tokens;
+  m->attn_splits = decode_attention_splits(c.max_batch, c.n_kv_heads, c.max_seq_len, m->sm_count);
+  const size_t scratch_floats = decode_attention_scratch_floats(c.max_batch, c.n_q_heads, c.head_dim, m->attn_splits);
+  bool oom = false;
+  auto A = [&](cudaError_t r) {
+    if (r != cudaSuccess) oom = true;
+  };
+  A(dev_alloc(&m->R[0], rows * d));
+  A(dev_alloc(&m->R[1], rows * d));
+  A(dev_alloc(&m->q_f32, MB * qd));
+  A(dev_alloc(&m->o_dec, MB * qd));
+  A(dev_alloc(&m->h_dec, MB * F));
+  A(dev_alloc(&m->attn_scratch, scratch_floats));
+  A(dev_alloc(&m->logits_ws, MB * c.vocab_size));
+  A(dev_alloc(&m->last_x, MB * d));
+  A(dev_alloc(&m->n_pf, MP * d));
+  A(dev_alloc(&m->q_pf, MP * qd));
+  A(dev_alloc(&m->o_pf, MP * qd));
+  A(dev_alloc(&m->h_pf, MP * F));
+  A(dev_alloc(&m->rope, static_cast<size_t>(c.max_seq_len) * (c.head_dim / 2)));
+  A(dev_alloc(&m->status, 4));
+  A(dev_alloc(&m->tok_tmp, MP > MB ? MP : MB));
+  A(dev_alloc(&m->next_tmp, MB));
+  if (oom) {
+    cudaGetLastError();
+    ladder_destroy(m);
+    return fail(nullptr, LADDER_ERR_OOM, "workspace allocation failed");
+  }
+  // rotary table in double precision: angle = p * theta^(-2j/Dh)
+  {
+    const int half = c.head_dim / 2;
+    std::vector<float2> tab(static_cast<size_t>(c.max_seq_len) * half);
+    for (int j = 0; j < half; ++j) {
+      const double inv = pow(static_cast<double>(c.rope_theta), -2.0 * j / c.head_dim);
+      for (int p = 0; p < c.max_seq_len; ++p) {
+        const double a = p * inv;
+        tab[static_cast<size_t>(p) * half + j] = make_float2(static_cast<float>(cos(a)), static_cast<float>(sin(a)));
+      }
+    }
+    e = cudaMemcpy(m->rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice);
+  }
+  if (e == cudaSuccess) e = cudaMemset(m->status, 0, 16);
+  if (e == cudaSuccess) e = cudaMemset(m->attn_scratch, 0, scratch_floats * sizeof(float));
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&m->cap, cudaStreamNonBlocking);
+  m->ev.resize(2 * L + 1, nullptr);
+  for (auto& ev : m->ev)
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming);
+  if (e != cudaSuccess) {
+    std::string msg = std::string("set-up: ") + cudaGetErrorString(e);
+    ladder_destroy(m);
+    return fail(nullptr, LADDER_ERR_CUDA, msg);
+  }
+  *out = m;
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_destroy(ladder_model_t* m) {
+  if (!m) return LADDER_OK;
+  drop_graph(m);
+  for (auto ev : m->ev)
+    if (ev) cudaEventDestroy(ev);
+  if (m->ev_fork) cudaEventDestroy(m->ev_fork);
+  if (m->ev_join) cudaEventDestroy(m->ev_join);
+  if (m->side) cudaStreamDestroy(m->side);
+  if (m->cap) cudaStreamDestroy(m->cap);
+  void* bufs[] = {m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
+                  m->n_pf, m->q_pf,  m->o_pf,  m->h_pf,  m->rope,  m->status,       m->tok_tmp,   m->next_tmp};
+  for (void* b : bufs)
+    if (b) cudaFree(b);
+  delete m;
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, int32_t use_graph, int32_t use_pdl) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  if (n_streams != 1 && n_streams != 2) return fail(m, LADDER_ERR_INVALID_ARG, "n_streams must be 1 or 2");
+  m->n_streams = n_streams;
+  m->use_graph = use_graph ? 1 : 0;
+  m->use_pdl = use_pdl ? 1 : 0;
+  drop_graph(m);
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_set_position(ladder_model_t* m, int32_t len) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  if (len < 0 || len > m->cfg.max_seq_len) return fail(m, LADDER_ERR_INVALID_ARG, "length outside [0, max_seq_len]");
+  m->host_len = len;
+  return LADDER_OK;
+}
+
+int64_t ladder_kernel_launches(const ladder_model_t* m) { return m ? m->launches : 0; }
+
+ladder_status_t ladder_device_status(ladder_model_t* m, int32_t* flags, void* cuda_stream) {
+  if (!m || !flags) return LADDER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CK(m, cudaStreamSynchronize(st));
+  CK(m, cudaMemcpy(flags, m->status, sizeof(int32_t), cudaMemcpyDeviceToHost));
+  CK(m, cudaMemset(m->status, 0, sizeof(int32_t)));
+  return LADDER_OK;
+}
+
+static ladder_status_t check_call(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* tokens, int batch) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  if (m->sticky_cuda) return fail(m, LADDER_ERR_CUDA, "an earlier CUDA call failed: " + m->err);
+  if (!cache || !cache->k || !cache->v || !cache->seq_lens || !tokens) return fail(m, LADDER_ERR_INVALID_ARG, "NULL argument");
+  if (batch < 1) return fail(m, LADDER_ERR_INVALID_ARG, "batch must be >= 1");
+  if (batch > m->cfg.max_batch) return fail(m, LADDER_ERR_STATE, "batch exceeds max_batch");
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_prefill(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int32_t batch,
+                               int32_t seq_len, const ladder_outputs_t* out, void* cuda_stream) {
+  ladder_status_t s = check_call(m, cache, d_tokens, batch);
+  if (s != LADDER_OK) return s;
+  if (seq_len < 1) return fail(m, LADDER_ERR_INVALID_ARG, "seq_len must be >= 1");
+  if (seq_len > m->cfg.max_seq_len) return fail(m, LADDER_ERR_STATE, "seq_len exceeds max_seq_len");
+  if (static_cast<int64_t>(batch) * seq_len > m->cfg.max_prefill_tokens)
+    return fail(m, LADDER_ERR_STATE, "batch*seq_len exceeds max_prefill_tokens");
+  int64_t k = 0;
+  CK(m, enqueue_prefill(m, cache, d_tokens, batch, seq_len, out, static_cast<cudaStream_t>(cuda_stream), &k));
+  m->launches += k;
+  m->host_len = seq_len;
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                                   int32_t batch, const ladder_outputs_t* out, void* cuda_stream) {
+  ladder_status_t s = check_call(m, cache, d_tokens, batch);
+  if (s != LADDER_OK) return s;
+  if (m->host_len + 1 > m->cfg.max_seq_len) return fail(m, LADDER_ERR_STATE, "KV cache is full");
+  if (out && out->all_hidden) return fail(m, LADDER_ERR_INVALID_ARG, "all_hidden is a prefill-only output");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const bool two = m->n_streams == 2;
+
+  if (!m->use_graph) {
+    int64_t k = 0;
+    if (two) {
+      // the side stream may only start after everything already queued on the caller's stream
+      CK(m, cudaEventRecord(m->ev_fork, st));
+      CK(m, cudaStreamWaitEvent(m->side, m->ev_fork, 0));
+    }
+    CK(m, enqueue_decode(m, cache, d_tokens, batch, out, st, two ? m->side : st, &k));
+    m->launches += k;
+  } else {
+    GraphKey key;
+    key.batch = batch;
+    key.n_streams = m->n_streams;
+    key.pdl = m->use_pdl;
+    key.k = cache->k;
+    key.v = cache->v;
+    key.lens = cache->seq_lens;
+    key.tok = d_tokens;
+    key.o_next = out ? out->next_tokens : nullptr;
+    key.o_hid = out ? out->final_hidden : nullptr;
+    key.o_logits = out ? out->logits : nullptr;
+    if (!m->graph_exec || !(key == m->graph_key)) {
+      drop_graph(m);
+      for (int attempt = 0; attempt < 2 && !m->graph_exec; ++attempt) {
+        cudaGraph_t graph = nullptr;
+        int64_t k = 0;
+        CK(m, cudaStreamBeginCapture(m->cap, cudaStreamCaptureModeRelaxed));
+        cudaError_t e = enqueue_decode(m, cache, d_tokens, batch, out, m->cap, two ? m->side : m->cap, &k);
+        cudaError_t e2 = cudaStreamEndCapture(m->cap, &graph);
+        if (e == cudaSuccess) e = e2;
+        if (e == cudaSuccess) e = cudaGraphInstantiate(&m->graph_exec, graph, 0);
+        if (graph) cudaGraphDestroy(graph);
+        if (e != cudaSuccess) {
+          cudaGetLastError();
+          m->graph_exec = nullptr;
+          if (attempt == 0 && m->use_pdl) {  // retry once without programmatic edges
+            m->use_pdl = 0;
+            key.pdl = 0;
+            continue;
+          }
+          m->sticky_cuda = true;
+          return fail(m, LADDER_ERR_CUDA, std::string("graph capture: ") + cudaGetErrorString(e));
+        }
+        m->graph_kernels = k;
+      }
+      m->graph_key = key;
+    }
+    CK(m, cudaGraphLaunch(m->graph_exec, st));
+    m->launches += m->graph_kernels;
+  }
+  m->host_len += 1;
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_decode_step_host(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* h_tokens,
+                                        int32_t batch, int32_t* h_next_tokens, void* cuda_stream) {
+  if (!m || !h_tokens || !h_next_tokens) return LADDER_ERR_INVALID_ARG;
+  if (batch < 1 || batch > m->cfg.max_batch) return fail(m, LADDER_ERR_STATE, "batch outside [1, max_batch]");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CK(m, cudaMemcpyAsync(m->tok_tmp, h_tokens, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  ladder_outputs_t out = {};
+  out.next_tokens = m->next_tmp;
+  ladder_status_t s = ladder_decode_step(m, cache, m->tok_tmp, batch, &out, cuda_stream);
+  if (s != LADDER_OK) return s;
+  CK(m, cudaMemcpyAsync(h_next_tokens, m->next_tmp, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  CK(m, cudaStreamSynchronize(st));
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_prefill_host(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* h_tokens,
+                                    int32_t batch, int32_t seq_len, int32_t* h_next_tokens, void* cuda_stream) {
+  if (!m || !h_tokens || !h_next_tokens) return LADDER_ERR_INVALID_ARG;
+  if (batch < 1 || batch > m->cfg.max_batch) return fail(m, LADDER_ERR_STATE, "batch outside [1, max_batch]");
+  if (seq_len < 1 || static_cast<int64_t>(batch) * seq_len > m->cfg.max_prefill_tokens)
+    return fail(m, LADDER_ERR_STATE, "batch*seq_len outside [1, max_prefill_tokens]");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CK(m, cudaMemcpyAsync(m->tok_tmp, h_tokens, static_cast<size_t>(batch) * seq_len * sizeof(int32_t),
+                        cudaMemcpyHostToDevice, st));
+  ladder_outputs_t out = {};
+  out.next_tokens = m->next_tmp;
+  ladder_status_t s = ladder_prefill(m, cache, m->tok_tmp, batch, seq_len, &out, cuda_stream);
+  if (s != LADDER_OK) return s;
+  CK(m, cudaMemcpyAsync(h_next_tokens, m->next_tmp, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  CK(m, cudaStreamSynchronize(st));
+  return LADDER_OK;
+}
+
+// --------------------------------------------------------------------------- single-kernel entry points
+static int g_sm_count = 0;
+static int sm_count_cached() {
+  if (!g_sm_count) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess)
+      g_sm_count = n;
+  }
+  return g_sm_count > 0 ? g_sm_count : 148;
+}
+
+ladder_status_t ladder_op_smallm_gemm(const void* W, int32_t N, int32_t K, const void* act, int32_t act_mode,
+                                      const void* gain, float eps, int32_t batch, int32_t epi_mode, const float* addend,
+                                      void* out, void* cuda_stream) {
+  if (!W || !act || !out || N < 8 || K < 8 || (N % 8) || (K % 8) || batch < 1 || batch > 64) return LADDER_ERR_INVALID_ARG;
+  if (act_mode != ACT_BF16 && act_mode != ACT_F32_NORM) return LADDER_ERR_INVALID_ARG;
+  if (act_mode == ACT_F32_NORM && !gain) return LADDER_ERR_INVALID_ARG;
+  if (epi_mode != EPI_RESID && epi_mode != EPI_SWIGLU && epi_mode != EPI_PLAIN) return LADDER_ERR_INVALID_ARG;
+  if (epi_mode == EPI_RESID && !addend) return LADDER_ERR_INVALID_ARG;
+  SmallMParams p = {};
+  p.W = static_cast<const __nv_bfloat16*>(W);
+  p.N = N;
+  p.K = K;
+  p.act = act;
+  p.act_mode = act_mode;
+  p.gain = static_cast<const __nv_bfloat16*>(gain);
+  p.eps = eps;
+  p.batch = batch;
+  p.epi_mode = epi_mode;
+  p.addend = addend;
+  p.out = out;
+  if (kernels_ready() != cudaSuccess) return LADDER_ERR_CUDA;
+  cudaError_t e = launch_smallm_gemm(p, static_cast<cudaStream_t>(cuda_stream), false, sm_count_cached());
+  return e == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
+}
+
+static int op_attn_splits(int batch, int n_kv_heads, int max_seq_len) {
+  return decode_attention_splits(batch, n_kv_heads, max_seq_len, sm_count_cached());
+}
+
+size_t ladder_decode_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim, int32_t max_seq_len) {
+  if (batch < 1 || n_q_heads < 1 || max_seq_len < 1) return 0;
+  // sized for the finest split any kv-head count can ask for (n_kv_heads = 1 gives the most splits)
+  const int splits = op_attn_splits(batch, 1, max_seq_len);
+  return decode_attention_scratch_floats(batch, n_q_heads, head_dim, splits) * sizeof(float);
+}
+
+ladder_status_t ladder_op_decode_attention(const float* q, const void* k, const void* v, const int32_t* kv_len,
+                                           int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                           int32_t max_seq_len, float* scratch, void* o, void* cuda_stream) {
+  if (!q || !k || !v || !kv_len || !scratch || !o) return LADDER_ERR_INVALID_ARG;
+  if (batch < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads || (head_dim != 64 && head_dim != 128) || max_seq_len < 1)
+    return LADDER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DecodeAttnParams a = {};
+  a.q = q;
+  a.k = static_cast<const __nv_bfloat16*>(k);
+  a.v = static_cast<const __nv_bfloat16*>(v);
+  a.kv_len = kv_len;
+  a.kv_len_offset = 0;
+  a.batch = batch;
+  a.n_q_heads = n_q_heads;
+  a.n_kv_heads = n_kv_heads;
+  a.head_dim = head_dim;
+  a.max_seq_len = max_seq_len;
+  a.max_len = max_seq_len;
+  a.n_splits = op_attn_splits(batch, n_kv_heads, max_seq_len);
+  a.scratch = scratch;
+  a.o = static_cast<__nv_bfloat16*>(o);
+  // ticket counters at the head of the scratch must start at zero
+  const size_t counters = (static_cast<size_t>(batch) * n_q_heads + 63) / 64 * 64;
+  if (cudaMemsetAsync(scratch, 0, counters * sizeof(float), st) != cudaSuccess) return LADDER_ERR_CUDA;
+  return launch_decode_attention(a, st, false) == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
+}
+
+ladder_status_t ladder_op_prefill_gemm(const void* A, const void* W, int32_t M, int32_t N, int32_t K, int32_t epi_mode,
+                                       const float* addend, void* out, void* cuda_stream) {
+  if (!A || !W || !out || M < 1 || N < 8 || K < 8 || (N % 8) || (K % 8)) return LADDER_ERR_INVALID_ARG;
+  int mode;
+  switch (epi_mode) {
+    case 0: mode = EPI_RESID; break;
+    case 1: mode = EPI_SWIGLU; break;
+    case 2: mode = EPI_PLAIN; break;
+    case 3: mode = EPI_BF16; break;
+    default: return LADDER_ERR_INVALID_ARG;
+  }
+  if (mode == EPI_RESID && !addend) return LADDER_ERR_INVALID_ARG;
+  LargeMParams p = {};
+  p.A = static_cast<const __nv_bfloat16*>(A);
+  p.W = static_cast<const __nv_bfloat16*>(W);
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  p.epi_mode = mode;
+  p.addend = addend;
+  p.out = out;
+  if (kernels_ready() != cudaSuccess) return LADDER_ERR_CUDA;
+  return launch_largem_gemm(p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
+}
+
+ladder_status_t ladder_op_prefill_attention(const void* q, const void* k, const void* v, int32_t batch, int32_t seq_len,
+                                            int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t max_seq_len,
+                                            void* o, void* cuda_stream) {
+  if (!q || !k || !v || !o || batch < 1 || seq_len < 1 || seq_len > max_seq_len || n_kv_heads < 1 ||
+      n_q_heads % n_kv_heads || (head_dim != 64 && head_dim != 128))
+    return LADDER_ERR_INVALID_ARG;
+  if (kernels_ready() != cudaSuccess) return LADDER_ERR_CUDA;
+  cudaError_t e = launch_prefill_attention(static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
+                                           static_cast<const __nv_bfloat16*>(v), batch, seq_len, n_q_heads, n_kv_heads,
+                                           head_dim, max_seq_len, static_cast<__nv_bfloat16*>(o),
+                                           static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
+}
+
+}  // extern "C"

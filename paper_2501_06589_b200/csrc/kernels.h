@@ -1,0 +1,94 @@
+// Host-side launch interface of the kernels (internal to libladder; no torch types).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ladder {
+
+enum ActMode { ACT_BF16 = 0, ACT_F32_NORM = 1 };
+enum EpiMode { EPI_RESID = 0, EPI_SWIGLU = 1, EPI_PLAIN = 2, EPI_QKV_ROPE = 3, EPI_BF16 = 4 };
+
+// Rotary / KV-append epilogue description shared by the decode and prefill QKV projections.
+struct QkvEpilogue {
+  float* q_out_f32;            // decode: fp32 [batch, Hq*Dh]
+  __nv_bfloat16* q_out_bf16;   // prefill: bf16 [M, Hq*Dh]
+  __nv_bfloat16* k_cache;      // one layer: [max_batch][Hkv][max_seq][Dh]
+  __nv_bfloat16* v_cache;
+  const int32_t* seq_lens;     // decode: position of row b = seq_lens[b]; prefill: NULL (position = m % seq_len)
+  const float2* rope;          // [max_seq][Dh/2] (cos, sin)
+  int n_q_heads, n_kv_heads, head_dim, max_seq_len;
+  int prefill_seq_len;         // prefill: rows are [batch, seq_len] flattened
+};
+
+struct SmallMParams {
+  const __nv_bfloat16* W;  // [N, K]
+  int N, K;
+  const void* act;         // ACT_BF16: bf16 [batch, K]; ACT_F32_NORM: fp32 [batch, K]
+  int act_mode;
+  const __nv_bfloat16* gain;  // [K] (ACT_F32_NORM)
+  float eps;
+  int batch;
+  int epi_mode;
+  const float* addend;     // EPI_RESID: fp32 [batch, N]
+  void* out;               // EPI_RESID / EPI_PLAIN: fp32 [batch, N]; EPI_SWIGLU: bf16 [batch, N/2]
+  QkvEpilogue qkv;         // EPI_QKV_ROPE
+  int32_t* status;         // device status word (may be NULL)
+};
+
+cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);
+size_t smallm_gemm_smem_bytes(int batch);
+
+// Decode attention (split over the cache) and its combine step.
+struct DecodeAttnParams {
+  const float* q;               // [batch, Hq*Dh]
+  const __nv_bfloat16* k;       // one layer
+  const __nv_bfloat16* v;
+  const int32_t* kv_len;        // [batch]
+  int kv_len_offset;            // keys attended = kv_len[b] + kv_len_offset (decode passes seq_lens and 1)
+  int batch, n_q_heads, n_kv_heads, head_dim, max_seq_len;
+  int n_splits;                 // CTAs per (b, kv head); each covers ceil(max_len / n_splits) keys
+  int max_len;                  // host upper bound on keys attended (sizes the split)
+  float* scratch;               // [batch][Hq][n_splits][Dh + 2]
+  __nv_bfloat16* o;             // [batch, Hq*Dh]
+};
+int decode_attention_splits(int batch, int n_kv_heads, int max_len, int sm_count);
+size_t decode_attention_scratch_floats(int batch, int n_q_heads, int head_dim, int n_splits);
+cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stream, bool pdl);
+
+// Prefill kernels.
+struct LargeMParams {
+  const __nv_bfloat16* A;  // [M, K]
+  const __nv_bfloat16* W;  // [N, K]
+  int M, N, K;
+  int epi_mode;
+  const float* addend;     // EPI_RESID
+  void* out;
+  QkvEpilogue qkv;
+};
+cudaError_t launch_largem_gemm(const LargeMParams& p, cudaStream_t stream);
+
+cudaError_t launch_prefill_attention(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                     int batch, int seq_len, int n_q_heads, int n_kv_heads, int head_dim,
+                                     int max_seq_len, __nv_bfloat16* o, cudaStream_t stream);
+
+// Small element-wise / gather kernels.
+cudaError_t launch_embed(const int32_t* tokens, const __nv_bfloat16* table, int rows, int d, int vocab, float* x,
+                         int32_t* status, cudaStream_t stream, bool pdl);
+cudaError_t launch_rmsnorm_bf16(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d,
+                                __nv_bfloat16* out, cudaStream_t stream);
+cudaError_t launch_rmsnorm_f32(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, int row_stride,
+                               float* out, cudaStream_t stream, bool pdl);
+cudaError_t launch_gather_rows(const float* x, int rows, int d, int src_stride_rows, int src_offset_rows, float* out,
+                               cudaStream_t stream);
+// argmax over logits [batch, vocab] (lowest index on ties) -> next_tokens; adds `advance` to seq_lens[b].
+cudaError_t launch_argmax_advance(const float* logits, int batch, int vocab, int32_t* next_tokens, int32_t* seq_lens,
+                                  int advance, int set_len, cudaStream_t stream, bool pdl);
+
+// One-time opt-in to large dynamic shared memory for every kernel (call once per process/device,
+// outside any stream capture).
+cudaError_t smallm_gemm_init();
+cudaError_t largem_gemm_init();
+cudaError_t prefill_attention_init();
+
+}  // namespace ladder

@@ -1,0 +1,166 @@
+// Small gather / normalisation / argmax kernels around the GEMMs.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace ladder {
+namespace {
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, bool pdl, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+// x[r, :] = float(table[tok[r], :]); an id outside [0, vocab) is reported and read as id 0.
+__global__ void embed_kernel(const int32_t* tokens, const __nv_bfloat16* table, int d, int vocab, float* x,
+                             int32_t* status) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  int t = tokens[r];
+  if (t < 0 || t >= vocab) {
+    if (threadIdx.x == 0 && status) atomicOr(status, LADDER_DEV_BAD_TOKEN);
+    t = 0;
+  }
+  const uint4* src = reinterpret_cast<const uint4*>(table + static_cast<size_t>(t) * d);
+  float4* dst = reinterpret_cast<float4*>(x + static_cast<size_t>(r) * d);
+  for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
+    const uint4 u = __ldg(src + i);
+    dst[2 * i] = make_float4(bf16_lo(u.x), bf16_hi(u.x), bf16_lo(u.y), bf16_hi(u.y));
+    dst[2 * i + 1] = make_float4(bf16_lo(u.z), bf16_hi(u.z), bf16_lo(u.w), bf16_hi(u.w));
+  }
+}
+
+__device__ __forceinline__ float block_sum(float v, float* sh) {
+  v = warp_sum(v);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) sh[warp] = v;
+  __syncthreads();
+  float t = 0.f;
+  const int nw = (blockDim.x + 31) >> 5;
+  for (int w = 0; w < nw; ++w) t += sh[w];
+  __syncthreads();
+  return t;
+}
+
+// y = x / sqrt(mean(x^2) + eps) * gain, one CTA per row; OUT = bf16 or fp32.
+template <typename OUT>
+__global__ void rmsnorm_kernel(const float* x, const __nv_bfloat16* gain, float eps, int d, int row_stride, OUT* out) {
+  __shared__ float sh[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const float* xr = x + static_cast<size_t>(blockIdx.x) * row_stride;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
+    const float4 v = reinterpret_cast<const float4*>(xr)[i];
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  const float rstd = rsqrtf(block_sum(ss, sh) / static_cast<float>(d) + eps);
+  OUT* o = out + static_cast<size_t>(blockIdx.x) * d;
+  for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
+    const float4 v = reinterpret_cast<const float4*>(xr)[i];
+    const uint2 gq = __ldg(reinterpret_cast<const uint2*>(gain) + i);
+    const float y0 = v.x * rstd * bf16_lo(gq.x), y1 = v.y * rstd * bf16_hi(gq.x);
+    const float y2 = v.z * rstd * bf16_lo(gq.y), y3 = v.w * rstd * bf16_hi(gq.y);
+    if (sizeof(OUT) == 2) {
+      reinterpret_cast<uint2*>(o)[i] = make_uint2(pack_bf16x2(y0, y1), pack_bf16x2(y2, y3));
+    } else {
+      reinterpret_cast<float4*>(o)[i] = make_float4(y0, y1, y2, y3);
+    }
+  }
+}
+
+// out[r, :] = x[(r * stride + offset), :]
+__global__ void gather_rows_kernel(const float* x, int d, int stride, int offset, float* out) {
+  const float4* src = reinterpret_cast<const float4*>(x + (static_cast<size_t>(blockIdx.x) * stride + offset) * d);
+  float4* dst = reinterpret_cast<float4*>(out + static_cast<size_t>(blockIdx.x) * d);
+  for (int i = threadIdx.x; i < d / 4; i += blockDim.x) dst[i] = src[i];
+}
+
+// Greedy token per row (lowest index among equal maxima), then the length update.
+__global__ void argmax_advance_kernel(const float* logits, int vocab, int32_t* next_tokens, int32_t* seq_lens,
+                                      int advance, int set_len) {
+  __shared__ float bv[32];
+  __shared__ int bi[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int b = blockIdx.x;
+  if (next_tokens) {
+    const float* row = logits + static_cast<size_t>(b) * vocab;
+    float best = -INFINITY;
+    int idx = 0x7fffffff;
+    for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
+      const float v = row[i];
+      if (v > best || (v == best && i < idx)) {
+        best = v;
+        idx = i;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+      if (ov > best || (ov == best && oi < idx)) {
+        best = ov;
+        idx = oi;
+      }
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) {
+      bv[warp] = best;
+      bi[warp] = idx;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const int nw = (blockDim.x + 31) >> 5;
+      for (int w = 1; w < nw; ++w)
+        if (bv[w] > best || (bv[w] == best && bi[w] < idx)) {
+          best = bv[w];
+          idx = bi[w];
+        }
+      next_tokens[b] = idx == 0x7fffffff ? 0 : idx;  // all-NaN row: defined result
+    }
+  }
+  if (threadIdx.x == 0 && seq_lens) {
+    if (set_len >= 0) seq_lens[b] = set_len;
+    else seq_lens[b] += advance;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_embed(const int32_t* tokens, const __nv_bfloat16* table, int rows, int d, int vocab, float* x,
+                         int32_t* status, cudaStream_t stream, bool pdl) {
+  return launch(embed_kernel, dim3(rows), dim3(256), stream, pdl, tokens, table, d, vocab, x, status);
+}
+
+cudaError_t launch_rmsnorm_bf16(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d,
+                                __nv_bfloat16* out, cudaStream_t stream) {
+  return launch(rmsnorm_kernel<__nv_bfloat16>, dim3(rows), dim3(256), stream, false, x, gain, eps, d, d, out);
+}
+
+cudaError_t launch_rmsnorm_f32(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, int row_stride,
+                               float* out, cudaStream_t stream, bool pdl) {
+  return launch(rmsnorm_kernel<float>, dim3(rows), dim3(256), stream, pdl, x, gain, eps, d, row_stride, out);
+}
+
+cudaError_t launch_gather_rows(const float* x, int rows, int d, int src_stride_rows, int src_offset_rows, float* out,
+                               cudaStream_t stream) {
+  return launch(gather_rows_kernel, dim3(rows), dim3(256), stream, false, x, d, src_stride_rows, src_offset_rows, out);
+}
+
+cudaError_t launch_argmax_advance(const float* logits, int batch, int vocab, int32_t* next_tokens, int32_t* seq_lens,
+                                  int advance, int set_len, cudaStream_t stream, bool pdl) {
+  return launch(argmax_advance_kernel, dim3(batch), dim3(1024), stream, pdl, logits, vocab, next_tokens, seq_lens,
+                advance, set_len);
+}
+
+}  // namespace ladder

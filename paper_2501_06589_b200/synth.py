@@ -172,16 +172,27 @@ def _np(t: torch.Tensor, dtype) -> np.ndarray:
     return t.detach().to(torch.float32).cpu().numpy().astype(dtype, copy=False)
 
 
-def logical_provider(w: AbiWeights, dtype=np.float32):
+def logical_provider(w: AbiWeights, dtype=np.float32, keep: bool = True):
     """Callable (name, layer) -> ndarray giving the *logical* tensors
-    (wq, wk, wv, wo, w_gate, w_up, w_down, norms, embedding, head) as views of the
+    (wq, wk, wv, wo, w_gate, w_up, w_down, norms, embedding, head) as slices of the
     packed bf16 data widened to ``dtype``.  Pure indexing and widening; tensors
-    that live on a GPU are downloaded one at a time."""
+    that live on a GPU are downloaded one at a time.  With ``keep`` the widened
+    copies are remembered (host memory = model size in ``dtype``); without it
+    every request converts again, which lets models larger than host memory stream."""
     s = w.shape
     nq = s.n_q_heads * s.head_dim
     nkv = s.n_kv_heads * s.head_dim
+    memo: Dict = {}
 
     def get(name: str, layer: Optional[int] = None) -> np.ndarray:
+        if not keep:
+            return fetch(name, layer)
+        key = (name, layer)
+        if key not in memo:
+            memo[key] = fetch(name, layer)
+        return memo[key]
+
+    def fetch(name: str, layer: Optional[int] = None) -> np.ndarray:
         if name == "tok_embedding":
             return _np(w.tok_embedding, dtype)
         if name == "final_norm":

@@ -1,0 +1,212 @@
+"""End-to-end parity of the CUDA library (through the C ABI) against the CPU oracle:
+final hidden states, greedy tokens (teacher-forced), KV-cache indexing, schedule invariance."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ladder_oracle as O
+from paper_2501_06589_b200 import synth
+from tests.helpers import rel_err
+
+pytestmark = pytest.mark.gpu
+
+HIDDEN_TOL = 2e-2          # max_i |g_i - o_i| / max_i |o_i| per (sequence, position), bf16 path vs oracle
+CANARY = 0x7F7F            # bf16 bit pattern pre-filled into the cache (a huge finite value)
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2501_06589_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+def oracle_cfg(s: synth.ModelShape) -> O.OracleConfig:
+    return O.OracleConfig(s.d_model, s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.vocab_size,
+                          s.rms_eps, s.rope_theta, None if s.layer_is_ladder is None else list(s.layer_is_ladder))
+
+
+def gpu_generate(B, model, cache, prompt: np.ndarray, steps: int, want_hidden=True):
+    """prefill + `steps` greedy decode steps on the device. Returns tokens [B, steps+1], hiddens."""
+    bsz = prompt.shape[0]
+    d = model.shape.d_model
+    tok = torch.from_numpy(prompt).cuda()
+    nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+    hid = torch.zeros(bsz, d, device="cuda") if want_hidden else None
+    toks, hids = [], []
+    model.prefill(cache, tok, next_tokens=nxt, final_hidden=hid)
+    toks.append(nxt.clone())
+    if want_hidden:
+        hids.append(hid.clone())
+    for _ in range(steps):
+        model.decode_step(cache, nxt, next_tokens=nxt, final_hidden=hid)     # token feedback stays on the device
+        toks.append(nxt.clone())
+        if want_hidden:
+            hids.append(hid.clone())
+    torch.cuda.synchronize()
+    toks = torch.stack(toks, 1).cpu().numpy()
+    hids = torch.stack(hids, 1).cpu().numpy() if want_hidden else None
+    return toks, hids
+
+
+def check_generation(B, shape, steps, dtype, gains="ones", schedule=None, min_agree=0.99, batch=None, prompt_len=None):
+    w = synth.make_weights(shape, device="cuda", gains=gains)
+    bsz = shape.batch if batch is None else batch
+    S = shape.prompt_len if prompt_len is None else prompt_len
+    prompt = synth.make_tokens(shape, bsz, S)
+    max_seq = S + steps + 3
+    model = B.Model(w, bsz, max_seq, bsz * S)
+    if schedule is not None:
+        model.set_schedule(*schedule)
+    cache = B.KVCache(shape, bsz, max_seq, fill=CANARY)
+    toks, hids = gpu_generate(B, model, cache, prompt, steps)
+    assert model.device_status() == 0
+    # --- oracle, fed the GPU's token history (teacher forcing)
+    cfg = oracle_cfg(shape)
+    OW = O.OracleWeights(provider=synth.logical_provider(w, dtype))
+    o_toks, o_hids = O.generate(cfg, OW, prompt, steps, max_seq, dtype=dtype, forced=toks)
+    err = rel_err(hids, o_hids)
+    agree = float(np.mean(toks == o_toks))
+    # --- KV cache indexing
+    used = S + steps
+    assert cache.seq_lens.cpu().tolist() == [used] * bsz
+    k5, v5 = cache.k5().view(torch.int16), cache.v5().view(torch.int16)
+    assert bool((k5[:, :, :, used:, :] == CANARY).all()) and bool((v5[:, :, :, used:, :] == CANARY).all())
+    assert not bool((k5[:, :, :, :used, :] == CANARY).any()) and not bool((v5[:, :, :, :used, :] == CANARY).any())
+    model.close()
+    return err, agree, toks, hids, cache
+
+
+@pytest.mark.parametrize("variant", ["ladder", "standard", "hybrid"])
+def test_tiny_config_full(B, variant):
+    s = synth.SHAPES["tiny"]
+    if variant == "standard":
+        s = s.as_standard()
+    elif variant == "hybrid":
+        s = synth.replace(s, layer_is_ladder=(0, 1, 1, 0))
+    err, agree, *_ = check_generation(B, s, 16, np.float64, gains="uniform", batch=4)
+    assert err < HIDDEN_TOL, err
+    assert agree >= 0.99, agree
+
+
+def test_tiny_cache_values_match_oracle(B):
+    s = synth.SHAPES["tiny"]
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    prompt = synth.make_tokens(s, 2, 16)
+    model = B.Model(w, 2, 40, 32)
+    cache = B.KVCache(s, 2, 40, fill=CANARY)
+    toks, _ = gpu_generate(B, model, cache, prompt, 8)
+    cfg = oracle_cfg(s)
+    OW = O.OracleWeights(provider=synth.logical_provider(w, np.float64))
+    oc = O.OracleCache(cfg, 2, 40)
+    O.prefill(cfg, OW, prompt, oc)
+    for j in range(8):
+        O.decode_step(cfg, OW, toks[:, j], oc)
+    gk = cache.k5()[:, :, :, :24].float().cpu().numpy().transpose(0, 1, 3, 2, 4)     # -> [l][b][pos][h][d]
+    gv = cache.v5()[:, :, :, :24].float().cpu().numpy().transpose(0, 1, 3, 2, 4)
+    assert rel_err(gk, oc.k[:, :, :24]) < 2e-2
+    assert rel_err(gv, oc.v[:, :, :24]) < 2e-2
+
+
+def test_schedules_are_bit_identical(B):
+    s = synth.replace(synth.SHAPES["tiny"], layer_is_ladder=(1, 1, 0, 1))
+    ref = None
+    for sched in [(1, False, False), (1, True, False), (2, False, False), (2, True, False), (1, False, True),
+                  (2, False, True), (2, True, True)]:
+        _, _, toks, hids, cache = check_generation(B, s, 12, np.float64, schedule=sched, batch=3, min_agree=0.0)
+        cur = (toks, hids, cache.k.clone(), cache.v.clone())
+        if ref is None:
+            ref = cur
+        else:
+            assert np.array_equal(ref[0], cur[0]), sched
+            assert np.array_equal(ref[1], cur[1]), sched
+            assert torch.equal(ref[2], cur[2]) and torch.equal(ref[3], cur[3]), sched
+
+
+def test_decode_equals_prefill_recomputation_on_gpu(B):
+    """KV-cached decode == full-sequence prefill of the same tokens, within bf16 tolerance."""
+    s = synth.SHAPES["tiny"]
+    w = synth.make_weights(s, device="cuda")
+    prompt = synth.make_tokens(s, 2, 16)
+    model = B.Model(w, 2, 64, 128)
+    cache = B.KVCache(s, 2, 64)
+    toks, hids = gpu_generate(B, model, cache, prompt, 10)
+    full = np.concatenate([prompt, toks[:, :10]], axis=1).astype(np.int32)
+    cache2 = B.KVCache(s, 2, 64)
+    allh = torch.zeros(2, 26, s.d_model, device="cuda")
+    model.prefill(cache2, torch.from_numpy(full).cuda(), all_hidden=allh)
+    torch.cuda.synchronize()
+    assert rel_err(allh[:, 15:].cpu().numpy(), hids) < HIDDEN_TOL
+    model.close()
+
+
+def test_host_buffer_entry_points(B):
+    s = synth.SHAPES["tiny"]
+    w = synth.make_weights(s, device="cuda")
+    prompt = synth.make_tokens(s, 2, 16)
+    model = B.Model(w, 2, 40, 32)
+    c1, c2 = B.KVCache(s, 2, 40), B.KVCache(s, 2, 40)
+    toks, _ = gpu_generate(B, model, c1, prompt, 6, want_hidden=False)
+    h_tok = torch.from_numpy(prompt).pin_memory()
+    h_next = torch.zeros(2, dtype=torch.int32).pin_memory()
+    model.prefill_host(c2, h_tok, h_next)
+    got = [h_next.clone().numpy()]
+    for _ in range(6):
+        h_in = h_next.clone().pin_memory()
+        model.decode_step_host(c2, h_in, h_next)
+        got.append(h_next.clone().numpy())
+    assert np.array_equal(np.stack(got, 1), toks)
+    model.close()
+
+
+def test_state_errors_and_bad_tokens(B):
+    s = synth.SHAPES["tiny"]
+    w = synth.make_weights(s, device="cuda")
+    model = B.Model(w, 2, 18, 32)
+    cache = B.KVCache(s, 2, 18)
+    tok = torch.from_numpy(synth.make_tokens(s, 2, 16)).cuda()
+    nxt = torch.zeros(2, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.LadderError) as e:
+        model.prefill(cache, torch.zeros(3, 4, dtype=torch.int32, device="cuda"))
+    assert e.value.status == 5                                  # batch > max_batch
+    model.prefill(cache, tok, next_tokens=nxt)
+    model.decode_step(cache, nxt, next_tokens=nxt)
+    model.decode_step(cache, nxt, next_tokens=nxt)
+    with pytest.raises(B.LadderError) as e:
+        model.decode_step(cache, nxt, next_tokens=nxt)          # 16 + 2 == max_seq_len: cache full
+    assert e.value.status == 5
+    assert model.device_status() == 0
+    model.set_position(16)
+    cache.seq_lens.fill_(16)
+    bad = torch.tensor([5, 99999], dtype=torch.int32, device="cuda")
+    model.decode_step(cache, bad, next_tokens=nxt)
+    assert model.device_status() & 1                            # LADDER_DEV_BAD_TOKEN, no fault
+    assert model.device_status() == 0
+    model.close()
+
+
+def test_config_1p2b_full(B):
+    """Second benchmark configuration in full: 512-token prompt, 64 greedy steps, oracle in float32."""
+    s = synth.SHAPES["1p2b"]
+    err, agree, *_ = check_generation(B, s, 64, np.float32)
+    assert err < HIDDEN_TOL, err
+    assert agree >= 0.99, agree
+
+
+def test_70b_shape_shallow_full_context(B):
+    """First 2 layers of the 70B shape, batch 4, 1024-token prompts, 8 decode steps:
+    long-cache indexing, the split over the cache, M = 4096 prefill tiles."""
+    s = synth.SHAPES["70b"].with_layers(2)
+    err, agree, *_ = check_generation(B, s, 8, np.float32)
+    assert err < HIDDEN_TOL, err
+    assert agree >= 0.97, agree          # 36 comparisons: allow one near-tie flip
+
+
+def test_8b_hybrid_shape_short_context(B):
+    """The 8B hybrid shape (GQA 32/8, theta 500000) cut to 4 standard + 4 ladder layers so the
+    float32 oracle copy fits any host; 16-token prompts, 8 steps."""
+    s = synth.replace(synth.SHAPES["8b_hybrid"].with_layers(8), layer_is_ladder=(0, 0, 0, 0, 1, 1, 1, 1))
+    err, agree, *_ = check_generation(B, s, 8, np.float32, batch=2, prompt_len=16)
+    assert err < HIDDEN_TOL, err
+    assert agree >= 0.94, agree          # 18 comparisons

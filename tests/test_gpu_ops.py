@@ -1,0 +1,167 @@
+"""Per-kernel parity: each CUDA kernel, called through the C ABI, against the oracle's
+operation on the same seeded inputs, at shapes that span several tiles and a ragged tail
+and at the true 70B decode shapes."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ladder_oracle as O
+from tests.helpers import rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2501_06589_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+def _bf16(shape, seed, std=1.0, device="cuda"):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    return (torch.randn(shape, generator=g) * std).to(torch.bfloat16).to(device)
+
+
+def _f64(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+# tolerance of a bf16-operand, fp32-accumulate dot product against float64 on the same operands:
+# the only error is the bf16 rounding of the normalised activation (2^-9 relative per element,
+# random sign) and fp32 summation, both far below 1e-2 of the row maximum.
+TOL_GEMM = 1e-2
+
+
+@pytest.mark.parametrize("N,K,batch", [(256, 256, 1), (1376, 256, 4), (256, 688, 3), (1024, 2048, 8),
+                                       (10240, 8192, 4), (4104, 1024, 16), (2048, 1280, 33), (1000, 520, 64)])
+def test_smallm_gemm_norm_plain(B, N, K, batch):
+    W = _bf16((N, K), 1, 0.02)
+    x = torch.randn(batch, K, generator=torch.Generator().manual_seed(2)).cuda() * 3.0
+    g = (torch.rand(K, generator=torch.Generator().manual_seed(3)) + 0.5).to(torch.bfloat16).cuda()
+    out = torch.full((batch, N), float("nan"), device="cuda")
+    B.op_smallm_gemm(W, x, 1, 2, out, gain=g, eps=1e-5)
+    torch.cuda.synchronize()
+    ref = O.rmsnorm(_f64(x), _f64(g), 1e-5) @ _f64(W).T
+    assert rel_err(out.cpu().numpy(), ref) < TOL_GEMM
+
+
+@pytest.mark.parametrize("N,K,batch", [(256, 688, 1), (8192, 8192, 4), (8192, 28672, 4), (512, 1032, 7), (776, 3584, 16)])
+def test_smallm_gemm_bf16_residual(B, N, K, batch):
+    W = _bf16((N, K), 4, 0.02)
+    a = _bf16((batch, K), 5, 1.0)
+    addend = torch.randn(batch, N, generator=torch.Generator().manual_seed(6)).cuda()
+    out = torch.empty_like(addend)
+    B.op_smallm_gemm(W, a, 0, 0, out, addend=addend)
+    torch.cuda.synchronize()
+    ref = _f64(addend) + _f64(a) @ _f64(W).T
+    assert rel_err(out.cpu().numpy(), ref) < 1e-3
+    # in place (standard-residual layers): destination == addend
+    inplace = addend.clone()
+    B.op_smallm_gemm(W, a, 0, 0, inplace, addend=inplace)
+    torch.cuda.synchronize()
+    assert torch.equal(inplace, out)
+
+
+@pytest.mark.parametrize("F,K,batch", [(688, 256, 1), (28672 // 8, 8192, 4), (1004, 520, 5)])
+def test_smallm_gemm_swiglu(B, F, K, batch):
+    W = _bf16((2 * F, K), 7, 0.05)
+    x = torch.randn(batch, K, generator=torch.Generator().manual_seed(8)).cuda()
+    g = torch.ones(K, dtype=torch.bfloat16, device="cuda")
+    out = torch.empty(batch, F, dtype=torch.bfloat16, device="cuda")
+    B.op_smallm_gemm(W, x, 1, 1, out, gain=g, eps=1e-5)
+    torch.cuda.synchronize()
+    n = O.rmsnorm(_f64(x), _f64(g), 1e-5)
+    w = _f64(W)
+    ref = O.silu(n @ w[0::2].T) * (n @ w[1::2].T)
+    assert rel_err(_f64(out), ref) < 2e-2
+
+
+def test_smallm_gemm_is_deterministic_and_batch_invariant(B):
+    N, K = 2048, 4096
+    W = _bf16((N, K), 9, 0.02)
+    x = torch.randn(4, K, generator=torch.Generator().manual_seed(10)).cuda()
+    g = torch.ones(K, dtype=torch.bfloat16, device="cuda")
+    o1 = torch.empty(4, N, device="cuda")
+    o2 = torch.empty(4, N, device="cuda")
+    B.op_smallm_gemm(W, x, 1, 2, o1, gain=g)
+    B.op_smallm_gemm(W, x, 1, 2, o2, gain=g)
+    o3 = torch.empty(1, N, device="cuda")
+    B.op_smallm_gemm(W, x[2:3].contiguous(), 1, 2, o3, gain=g)
+    torch.cuda.synchronize()
+    assert torch.equal(o1, o2)
+    assert torch.equal(o1[2:3], o3)          # row b of a batch == the same row run alone
+
+
+@pytest.mark.parametrize("batch,Hq,Hkv,Dh,max_seq,lens", [
+    (1, 4, 4, 64, 32, [17]),
+    (2, 16, 16, 128, 640, [513, 640]),
+    (4, 64, 8, 128, 1536, [1025, 1300, 1536, 1]),
+    (3, 32, 8, 128, 300, [0, 299, 37]),
+    (2, 8, 1, 128, 2048, [2048, 2047]),
+    (2, 6, 3, 64, 100, [100, 31]),
+])
+def test_decode_attention(B, batch, Hq, Hkv, Dh, max_seq, lens):
+    q = torch.randn(batch, Hq * Dh, generator=torch.Generator().manual_seed(11)).cuda()
+    k = _bf16((batch, Hkv, max_seq, Dh), 12, 1.0)
+    v = _bf16((batch, Hkv, max_seq, Dh), 13, 1.0)
+    kv_len = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    scratch = torch.empty(B.decode_attention_scratch_bytes(batch, Hq, Dh, max_seq) // 4, device="cuda")
+    o = torch.full((batch, Hq * Dh), float("nan"), dtype=torch.bfloat16, device="cuda")
+    for _ in range(2):                       # twice: the ticket counters must clean themselves up
+        B.op_decode_attention(q, k, v, kv_len, Hq, Hkv, Dh, max_seq, scratch, o)
+    torch.cuda.synchronize()
+    got = _f64(o).reshape(batch, Hq, Dh)
+    qb = O.bf16_round(_f64(q)).reshape(batch, 1, Hq, Dh)          # the kernel feeds q to the MMA as bf16
+    for b in range(batch):
+        L = lens[b]
+        if L == 0:
+            assert np.all(got[b] == 0.0)
+            continue
+        kk = _f64(k[b, :, :L]).transpose(1, 0, 2)
+        vv = _f64(v[b, :, :L]).transpose(1, 0, 2)
+        ref = O.causal_attention(qb[b], kk, vv, L - 1)[0]
+        assert rel_err(got[b], ref) < 1e-2, b
+
+
+@pytest.mark.parametrize("M,N,K,mode", [(16, 768, 256, 3), (300, 1376, 256, 1), (512, 256, 688, 0),
+                                        (1000, 520, 264, 2), (4096, 1024, 1024, 0)])
+def test_prefill_gemm(B, M, N, K, mode):
+    A = _bf16((M, K), 14, 1.0)
+    W = _bf16((N, K), 15, 0.05)
+    acc = _f64(A) @ _f64(W).T
+    if mode == 0:
+        addend = torch.randn(M, N, generator=torch.Generator().manual_seed(16)).cuda()
+        out = torch.empty_like(addend)
+        B.op_prefill_gemm(A, W, 0, out, addend=addend)
+        ref = _f64(addend) + acc
+    elif mode == 1:
+        out = torch.empty(M, N // 2, dtype=torch.bfloat16, device="cuda")
+        B.op_prefill_gemm(A, W, 1, out)
+        ref = O.silu(acc[:, 0::2]) * acc[:, 1::2]
+    elif mode == 2:
+        out = torch.empty(M, N, device="cuda")
+        B.op_prefill_gemm(A, W, 2, out)
+        ref = acc
+    else:
+        out = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+        B.op_prefill_gemm(A, W, 3, out)
+        ref = acc
+    torch.cuda.synchronize()
+    assert rel_err(_f64(out), ref) < (1e-3 if mode in (0, 2) else 1e-2)
+
+
+@pytest.mark.parametrize("batch,S,Hq,Hkv,Dh,max_seq", [(1, 16, 4, 4, 64, 32), (2, 200, 8, 2, 128, 256),
+                                                       (1, 1024, 8, 1, 128, 1536), (2, 65, 6, 3, 64, 70)])
+def test_prefill_attention(B, batch, S, Hq, Hkv, Dh, max_seq):
+    q = _bf16((batch, S, Hq * Dh), 17, 1.0)
+    k = _bf16((batch, Hkv, max_seq, Dh), 18, 1.0)
+    v = _bf16((batch, Hkv, max_seq, Dh), 19, 1.0)
+    o = torch.full((batch, S, Hq * Dh), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.op_prefill_attention(q, k, v, batch, S, Hq, Hkv, Dh, max_seq, o)
+    torch.cuda.synchronize()
+    for b in range(batch):
+        ref = O.causal_attention(_f64(q[b]).reshape(S, Hq, Dh), _f64(k[b, :, :S]).transpose(1, 0, 2),
+                                 _f64(v[b, :, :S]).transpose(1, 0, 2), 0)
+        assert rel_err(_f64(o[b]).reshape(S, Hq, Dh), ref) < 2e-2, b

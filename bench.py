@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of the Ladder-Residual decode path on B200: decode tokens/s and the fraction of
+the HBM roofline, 70B shape, batch 4, 1024-token prompts, 512 decode steps (paper Sec. 3.3.1
+workload; seeded synthetic weights and tokens).
+
+A *step* is one autoregressive decode step of the whole model over the batch (embedding,
+80 x [RMSNorm+QKV+RoPE+KV append, split-KV attention, output projection + ladder add,
+RMSNorm+gate/up+SwiGLU, down projection + ladder add], final norm, LM head, argmax), replayed
+as one CUDA graph with the token fed back on the device.  The prompt pass runs before the
+timed region and is reported separately as `prefill`.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 70b] [--impl reference]
+
+N > 1 runs N independent replicas (one process per GPU under torch.distributed; no data-path
+collective: the path does not shard) and reports the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return float(j["hbm_gbs"]), float(j.get("bf16_tflops_sustained", j["bf16_tflops"])), "measured"
+    return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_decode_sample(shape, weights, kv_len, n_layers_sample, dtype_name="float32"):
+    """Time the CPU oracle on a bounded sample of one decode step: `n_layers_sample` layers of
+    the stack at KV length `kv_len` plus the LM head; returns (seconds for the sample's layers,
+    seconds for the head, threads).  The cache content is seeded noise (timing only)."""
+    import numpy as np
+    from oracle import ladder_oracle as O
+    from paper_2501_06589_b200 import synth
+    dt = getattr(np, dtype_name)
+    sub = shape.with_layers(n_layers_sample)
+    cfg = O.OracleConfig(sub.d_model, sub.n_layers, sub.n_q_heads, sub.n_kv_heads, sub.head_dim, sub.d_ff,
+                         sub.vocab_size, sub.rms_eps, sub.rope_theta,
+                         None if sub.layer_is_ladder is None else list(sub.layer_is_ladder))
+    prov = synth.logical_provider(weights, dt)
+    W = O.OracleWeights(provider=prov)
+    for l in range(n_layers_sample):                       # widen the sample's weights outside the timed part
+        for nm in ("attn_norm", "mlp_norm", "wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down"):
+            W.get(nm, l)
+    for nm in ("tok_embedding", "final_norm", "lm_head"):
+        W.get(nm)
+    B = shape.batch
+    cache = O.OracleCache(cfg, B, kv_len + 1, dt)
+    rng = np.random.default_rng(7)
+    cache.k[:, :, :kv_len] = rng.standard_normal(cache.k[:, :, :kv_len].shape, dtype=np.float32).astype(dt)
+    cache.v[:, :, :kv_len] = rng.standard_normal(cache.v[:, :, :kv_len].shape, dtype=np.float32).astype(dt)
+    cache.seq_len = kv_len
+    toks = synth.make_tokens(shape, B, 1)[:, 0]
+    t0 = time.perf_counter()
+    x = O.embed(W, toks.reshape(-1, 1), dt)
+    x = O.run_layers(cfg, W, x, kv_len, cache)
+    t1 = time.perf_counter()
+    O.head(cfg, W, x)
+    t2 = time.perf_counter()
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    return t1 - t0, t2 - t1, threads
+
+
+def cpu_baseline(shape, weights, kv_len):
+    n_sample = min(2, shape.n_layers)
+    t_layers, t_head, threads = oracle_decode_sample(shape, weights, kv_len, n_sample)
+    t_step = t_layers * (shape.n_layers / n_sample) + t_head
+    return {"value": shape.batch / t_step, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+            "sample": (f"one decode step at KV length {kv_len}, batch {shape.batch}: {n_sample} of {shape.n_layers} "
+                       f"layers ({t_layers:.2f} s) + LM head ({t_head:.2f} s) in float32, layer time extrapolated "
+                       f"x{shape.n_layers / n_sample:g}")}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import torch
+    from paper_2501_06589_b200 import synth
+    shape = synth.SHAPES[args.config]
+    n_sample = min(2, shape.n_layers)
+    w = synth.make_weights(shape.with_layers(n_sample), device="cpu")
+    kv_len = shape.prompt_len
+    times = []
+    for i in range(args.warmup + args.steps):
+        t_layers, t_head, threads = oracle_decode_sample(shape, w, kv_len, n_sample)
+        if i >= args.warmup:
+            times.append(t_layers * (shape.n_layers / n_sample) + t_head)
+    t = statistics.mean(times)
+    sample = (f"per step: one decode step at KV length {kv_len}, batch {shape.batch}, {n_sample} of {shape.n_layers} "
+              f"layers + LM head in float32, layer time extrapolated x{shape.n_layers / n_sample:g}")
+    val = shape.batch / t
+    line = {"impl": "reference", "metric": "decode_tokens_per_s", "value": val, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(shape, args),
+            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(shape, args):
+    return {"workload": f"{shape.name}: d_model {shape.d_model}, {shape.n_layers} layers "
+                        f"({'all ladder' if shape.layer_is_ladder is None else 'hybrid mask'}), "
+                        f"{shape.n_q_heads}q/{shape.n_kv_heads}kv heads x {shape.head_dim}, ffn {shape.d_ff}, "
+                        f"vocab {shape.vocab_size}",
+            "batch": shape.batch, "prompt_len": shape.prompt_len, "decode_steps": args.steps,
+            "l2": "inputs larger than L2 (every step streams all weights, far above 126 MB)",
+            "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=512)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="70b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--streams", type=int, default=None)
+    ap.add_argument("--graph", type=int, default=None)
+    ap.add_argument("--pdl", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill-timing", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    from paper_2501_06589_b200 import binding as B
+    from paper_2501_06589_b200 import build, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if dist:
+        dist.barrier()
+    B.lib()
+
+    shape = synth.SHAPES[args.config]
+    steps, warm = args.steps, max(args.warmup, 0)
+    S, bsz = shape.prompt_len, shape.batch
+    max_seq = S + max(steps, warm)
+    hbm_peak, bf16_peak, peak_src = measured_peaks()
+
+    t0 = time.time()
+    w = synth.make_weights(shape, device="cuda")
+    torch.cuda.synchronize()
+    t_gen = time.time() - t0
+    model = B.Model(w, bsz, max_seq, bsz * S)
+    if args.streams is not None or args.graph is not None or args.pdl is not None:
+        model.set_schedule(2 if args.streams is None else args.streams, 1 if args.graph is None else args.graph,
+                           1 if args.pdl is None else args.pdl)
+    cache = B.KVCache(shape, bsz, max_seq)
+    prompt = torch.from_numpy(synth.make_tokens(shape, bsz, S)).cuda()
+    nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+    first = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- prefill: once untimed (warm-up), once timed
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    model.prefill(cache, prompt, next_tokens=first)
+    torch.cuda.synchronize()
+    prefill_ms = None
+    if not args.no_prefill_timing:
+        ev[0].record()
+        model.prefill(cache, prompt, next_tokens=first)
+        ev[1].record()
+        torch.cuda.synchronize()
+        prefill_ms = ev[0].elapsed_time(ev[1])
+
+    def rewind():
+        cache.seq_lens.fill_(S)
+        model.set_position(S)
+        nxt.copy_(first)
+
+    # ---- decode: warm-up, then K timed steps (token fed back on the device, no host sync inside)
+    rewind()
+    for _ in range(warm):
+        model.decode_step(cache, nxt, next_tokens=nxt)
+    rewind()
+    sync_all()
+    launches0 = model.kernel_launches()
+    with ClockSampler(local) as clocks:
+        ev[2].record()
+        for _ in range(steps):
+            model.decode_step(cache, nxt, next_tokens=nxt)
+        ev[3].record()
+        sync_all()
+    dev_ms = ev[2].elapsed_time(ev[3])
+    launches = model.kernel_launches() - launches0
+    status = model.device_status()
+
+    # ---- end to end: host token buffers in, host tokens out, every step (pinned memory)
+    rewind()
+    h_in = first.cpu().pin_memory()
+    h_out = torch.zeros(bsz, dtype=torch.int32).pin_memory()
+    sync_all()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        model.decode_step_host(cache, h_in, h_out)
+        h_in.copy_(h_out)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+
+    # ---- dominant kernel alone: the gate/up weight-streaming GEMM over every layer's weights
+    x_act = torch.randn(bsz, shape.d_model, device="cuda")
+    h_out_buf = torch.empty(bsz, shape.d_ff, device="cuda")
+    n_l = shape.n_layers
+    for l in range(min(3, n_l)):
+        B.op_smallm_gemm(w.w_gate_up[l], x_act, 1, 1, h_out_buf, gain=w.mlp_norm[l], eps=shape.rms_eps)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for l in range(n_l):
+        B.op_smallm_gemm(w.w_gate_up[l], x_act, 1, 1, h_out_buf, gain=w.mlp_norm[l], eps=shape.rms_eps)
+    e1.record()
+    torch.cuda.synchronize()
+    k_ms = e0.elapsed_time(e1) / n_l
+    k_bytes = 2.0 * 2 * shape.d_ff * shape.d_model
+    k_gbs = k_bytes / (k_ms * 1e-3) / 1e9
+
+    # ---- reduce over ranks (max time), aggregate value
+    t_dev = torch.tensor([dev_ms, e2e_s * 1e3, prefill_ms or 0.0], device="cuda", dtype=torch.float64)
+    if dist:
+        dist.all_reduce(t_dev, op=dist.ReduceOp.MAX)
+    dev_ms, e2e_ms, prefill_ms_max = [float(v) for v in t_dev.tolist()]
+    ms_per_step = dev_ms / steps
+    value = world * bsz * steps / (dev_ms * 1e-3)
+    e2e_value = world * bsz * steps / (e2e_ms * 1e-3)
+    mean_kv = S + (steps + 1) / 2.0
+    step_bytes = shape.decode_step_bytes(mean_kv)
+    step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+
+    line = {
+        "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps,
+        "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(shape, args),
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": 4 * bsz, "d2h_bytes_per_step": 4 * bsz},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "smallm_gemm (RMSNorm + gate/up projection + SwiGLU)",
+                     "achieved": k_gbs, "peak": hbm_peak, "peak_source": peak_src, "unit": "GB/s",
+                     "frac": k_gbs / hbm_peak, "bytes_per_launch": k_bytes, "ms_per_launch": k_ms, "traffic": None},
+        "step_roofline": {"bytes_per_step": step_bytes, "achieved_gbs": step_gbs,
+                          "frac_of_measured_copy_peak": step_gbs / hbm_peak,
+                          "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS, "mean_kv_len": mean_kv},
+        "clocks": clocks.summary(),
+        "device_status": status,
+        "schedule": {"streams": args.streams, "graph": args.graph, "pdl": args.pdl},
+        "weights_gb": w.nbytes() / 1e9, "weight_gen_s": t_gen,
+    }
+    if prefill_ms_max:
+        flops = prefill_flops(shape, bsz, S)
+        line["prefill"] = {"tokens_per_s": world * bsz * S / (prefill_ms_max * 1e-3), "ms": prefill_ms_max,
+                           "tflops": flops / (prefill_ms_max * 1e-3) / 1e12,
+                           "frac_of_bf16_peak": flops / (prefill_ms_max * 1e-3) / 1e12 / bf16_peak,
+                           "peak_tflops": bf16_peak, "peak_source": peak_src}
+    tr = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tr):
+        try:
+            line["roofline"]["traffic"] = json.load(open(tr)).get("smallm_gemm_gate_up_bytes_per_launch")
+        except Exception:
+            pass
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(shape, w, S)
+    if rank == 0:
+        print(json.dumps(line))
+    model.close()
+    if dist:
+        dist.destroy_process_group()
+    return 0
+
+
+def prefill_flops(shape, bsz, S):
+    d, F = shape.d_model, shape.d_ff
+    per_tok_layer = 2 * (shape.qkv_rows * d + d * shape.n_q_heads * shape.head_dim + 3 * F * d)
+    attn = 2 * 2 * shape.n_q_heads * shape.head_dim * (S * (S + 1) / 2)       # QK^T and PV, causal
+    return shape.n_layers * (bsz * S * per_tok_layer + bsz * attn) + 2 * bsz * shape.vocab_size * d
+
+
+if __name__ == "__main__":
+    sys.exit(main())

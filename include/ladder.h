@@ -18,8 +18,12 @@
  * followed by grouped-query causal attention with rotary embedding on interleaved pairs,
  * or by a SwiGLU MLP ("Llama-3's model architecture", paper Sec. 3.3.1).
  *
- * Numerics: bf16 weights, bf16 KV cache, bf16 GEMM operands, fp32 accumulation, fp32
- * softmax, fp32 residual stream, fp32 logits.  Greedy argmax picks the lowest index on ties.
+ * Numerics: bf16 weights, bf16 KV cache, bf16 tensor-core operands, fp32 accumulation, fp32
+ * softmax, fp32 residual stream, fp32 logits.  In the decode path activations enter the
+ * tensor cores as a bf16 high + low pair (about 16 mantissa bits; free in a bandwidth-bound
+ * kernel) for batch <= 16, and so do the prefill GEMMs and the prefill query (two MMAs per
+ * weight tile): what is left of bf16 in the activations is the KV cache itself.
+ * Greedy argmax picks the lowest index on ties.
  *
  * Errors: every function returns a ladder_status_t; argument errors are detected on the
  * host before anything is launched; nothing aborts, traps or hangs the device.
@@ -159,11 +163,12 @@ const char* ladder_last_error(const ladder_model_t* m); /* library-owned string;
 
 /* Weight-streaming small-M GEMM  acc[b,n] = sum_k act[b,k] * W[n,k]  (decode: M = batch <= 64),
  * with the activation staging and the epilogue of one step of the decode path.
- *   act_mode 0: act = bf16 [batch, K]                              (steps: output / down projection)
- *            1: act = fp32 residual [batch, K]; the kernel applies RMSNorm with gain `gain`
- *               bf16 [K] and eps (steps: fused RMSNorm + QKV / gate-up projection, LM head)
+ *   act      fp32 [batch, K]
+ *   act_mode 0: used as is                                         (steps: output / down projection)
+ *            1: the kernel applies RMSNorm with gain `gain` bf16 [K] and eps to it
+ *               (steps: fused RMSNorm + QKV / gate-up projection, LM head)
  *   epi_mode 0: out_f32[b,n] = addend[b,n] + acc            (residual add; addend may equal out_f32)
- *            1: out_bf16[b,j] = silu(acc[b,2j]) * acc[b,2j+1]      (SwiGLU over interleaved rows)
+ *            1: out_f32[b,j] = silu(acc[b,2j]) * acc[b,2j+1]       (SwiGLU over interleaved rows)
  *            2: out_f32[b,n] = acc                                   (plain, e.g. logits)
  * W bf16 [N,K] row-major; N % 8 == 0, K % 8 == 0, 1 <= batch <= 64. */
 ladder_status_t ladder_op_smallm_gemm(const void* W, int32_t N, int32_t K, const void* act, int32_t act_mode,
@@ -174,24 +179,28 @@ ladder_status_t ladder_op_smallm_gemm(const void* W, int32_t N, int32_t K, const
  *   q fp32 [batch, Hq*Dh] (already rotated); k,v bf16 [max_batch][Hkv][max_seq_len][Dh] (one layer);
  *   kv_len int32 [batch] = number of keys to attend (positions 0..kv_len-1);
  *   scratch fp32, at least ladder_decode_attention_scratch_bytes(...) bytes;
- *   o bf16 [batch, Hq*Dh].  softmax(q.k/sqrt(Dh)) v per head, fp32 softmax and accumulation. */
+ *   o fp32 [batch, Hq*Dh].  softmax(q.k/sqrt(Dh)) v per head, fp32 softmax and accumulation. */
 size_t ladder_decode_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim, int32_t max_seq_len);
 ladder_status_t ladder_op_decode_attention(const float* q, const void* k, const void* v, const int32_t* kv_len,
                                            int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
                                            int32_t max_seq_len, float* scratch, void* o, void* cuda_stream);
 
-/* Large-M GEMM of the prefill path: C[m,n] = sum_k A[m,k] * W[n,k], A bf16 [M,K], W bf16 [N,K].
+/* Large-M GEMM of the prefill path: C[m,n] = sum_k (A[m,k] + A_lo[m,k]) * W[n,k], A bf16 [M,K], W bf16 [N,K].
+ *   A_lo: optional bf16 [M,K] low part of the activation (activation ~ A + A_lo); NULL = single bf16.
  *   epi_mode 0: out_f32[m,n] = addend[m,n] + acc;  1: SwiGLU -> out_bf16 [M, N/2];
- *            2: out_f32 = acc;  3: out_bf16[m,n] = acc.   K % 8 == 0, N % 8 == 0. */
-ladder_status_t ladder_op_prefill_gemm(const void* A, const void* W, int32_t M, int32_t N, int32_t K,
-                                       int32_t epi_mode, const float* addend, void* out, void* cuda_stream);
+ *            2: out_f32 = acc;  3: out_bf16[m,n] = acc.   K % 8 == 0, N % 8 == 0.
+ *   out_lo: optional (modes 1 and 3) bf16 buffer of out's shape receiving value - bf16(value). */
+ladder_status_t ladder_op_prefill_gemm(const void* A, const void* A_lo, const void* W, int32_t M, int32_t N, int32_t K,
+                                       int32_t epi_mode, const float* addend, void* out, void* out_lo,
+                                       void* cuda_stream);
 
 /* Causal grouped-query attention of the prefill path for one layer:
- *   q bf16 [batch, seq_len, Hq*Dh] (rotated); k,v bf16 cache of one layer as above, rows 0..seq_len-1
- *   valid; o bf16 [batch, seq_len, Hq*Dh].  Query p attends keys t <= p. */
-ladder_status_t ladder_op_prefill_attention(const void* q, const void* k, const void* v, int32_t batch,
-                                            int32_t seq_len, int32_t n_q_heads, int32_t n_kv_heads,
-                                            int32_t head_dim, int32_t max_seq_len, void* o, void* cuda_stream);
+ *   q bf16 [batch, seq_len, Hq*Dh] (rotated), q_lo its optional low part; k,v bf16 cache of one layer
+ *   as above, rows 0..seq_len-1 valid; o bf16 [batch, seq_len, Hq*Dh], o_lo its low part (given iff
+ *   q_lo is).  Query p attends keys t <= p. */
+ladder_status_t ladder_op_prefill_attention(const void* q, const void* q_lo, const void* k, const void* v, int32_t batch,
+                                            int32_t seq_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                            int32_t max_seq_len, void* o, void* o_lo, void* cuda_stream);
 
 #ifdef __cplusplus
 }

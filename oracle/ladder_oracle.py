@@ -108,7 +108,7 @@ def _store(a: np.ndarray, bf16_storage: bool) -> np.ndarray:
 def rmsnorm(x: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
     """y_i = x_i / sqrt(mean_j x_j^2 + eps) * g_i over the last axis."""
     ms = np.mean(x * x, axis=-1, keepdims=True)
-    return x / np.sqrt(ms + x.dtype.type(eps)) * g.astype(x.dtype)
+    return x / np.sqrt(ms + x.dtype.type(eps)) * g.astype(x.dtype, copy=False)
 
 
 def rope_angles(positions: np.ndarray, head_dim: int, theta: float):
@@ -196,10 +196,10 @@ def attention_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndar
     B, T, d = n.shape
     Hq, Hkv, Dh = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
     dt = n.dtype
-    wq = W.get("wq", layer).astype(dt)
-    wk = W.get("wk", layer).astype(dt)
-    wv = W.get("wv", layer).astype(dt)
-    wo = W.get("wo", layer).astype(dt)
+    wq = W.get("wq", layer).astype(dt, copy=False)
+    wk = W.get("wk", layer).astype(dt, copy=False)
+    wv = W.get("wv", layer).astype(dt, copy=False)
+    wo = W.get("wo", layer).astype(dt, copy=False)
     positions = pos0 + np.arange(T)
     q = (n @ wq.T).reshape(B, T, Hq, Dh)
     k = (n @ wk.T).reshape(B, T, Hkv, Dh)
@@ -212,8 +212,8 @@ def attention_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndar
         if cache is not None:
             cache.k[layer, b, pos0:pos0 + T] = k[b]
             cache.v[layer, b, pos0:pos0 + T] = v[b]
-            kk = cache.k[layer, b, :pos0 + T].astype(dt)
-            vv = cache.v[layer, b, :pos0 + T].astype(dt)
+            kk = cache.k[layer, b, :pos0 + T].astype(dt, copy=False)
+            vv = cache.v[layer, b, :pos0 + T].astype(dt, copy=False)
         else:
             assert pos0 == 0
             kk, vv = k[b], v[b]
@@ -226,9 +226,9 @@ def mlp_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndarray,
                bf16_storage: bool = False):
     """h(n) = W_down ( silu(W_gate n) * (W_up n) )."""
     dt = n.dtype
-    wg = W.get("w_gate", layer).astype(dt)
-    wu = W.get("w_up", layer).astype(dt)
-    wd = W.get("w_down", layer).astype(dt)
+    wg = W.get("w_gate", layer).astype(dt, copy=False)
+    wu = W.get("w_up", layer).astype(dt, copy=False)
+    wd = W.get("w_down", layer).astype(dt, copy=False)
     h = _store(silu(n @ wg.T) * (n @ wu.T), bf16_storage)
     return h @ wd.T
 
@@ -298,7 +298,7 @@ def embed(W: OracleWeights, tokens: np.ndarray, dtype) -> np.ndarray:
 
 def head(cfg: OracleConfig, W: OracleWeights, x: np.ndarray, bf16_storage: bool = False):
     hidden = rmsnorm(x, W.get("final_norm"), cfg.rms_eps)
-    logits = _store(hidden, bf16_storage) @ W.get("lm_head").astype(x.dtype).T
+    logits = _store(hidden, bf16_storage) @ W.get("lm_head").astype(x.dtype, copy=False).T
     return hidden, logits
 
 

@@ -96,11 +96,11 @@ def lib() -> C.CDLL:
         L.ladder_op_decode_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                                  C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
                                                  C.c_void_p, C.c_void_p]
-        L.ladder_op_prefill_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
-                                             C.c_void_p, C.c_void_p, C.c_void_p]
-        L.ladder_op_prefill_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
-                                                  C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
-                                                  C.c_void_p]
+        L.ladder_op_prefill_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                             C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ladder_op_prefill_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                                  C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                                  C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -246,12 +246,14 @@ def op_decode_attention(q, k, v, kv_len, n_q_heads, n_kv_heads, head_dim, max_se
                                             n_kv_heads, head_dim, max_seq_len, _ptr(scratch), _ptr(o), _stream()))
 
 
-def op_prefill_gemm(A, W, epi_mode: int, out, addend=None):
+def op_prefill_gemm(A, W, epi_mode: int, out, addend=None, A_lo=None, out_lo=None):
     M, K = A.shape
     N = W.shape[0]
-    _check(lib().ladder_op_prefill_gemm(_ptr(A), _ptr(W), M, N, K, epi_mode, _ptr(addend), _ptr(out), _stream()))
+    _check(lib().ladder_op_prefill_gemm(_ptr(A), _ptr(A_lo), _ptr(W), M, N, K, epi_mode, _ptr(addend), _ptr(out),
+                                        _ptr(out_lo), _stream()))
 
 
-def op_prefill_attention(q, k, v, batch, seq_len, n_q_heads, n_kv_heads, head_dim, max_seq_len, o):
-    _check(lib().ladder_op_prefill_attention(_ptr(q), _ptr(k), _ptr(v), batch, seq_len, n_q_heads, n_kv_heads,
-                                             head_dim, max_seq_len, _ptr(o), _stream()))
+def op_prefill_attention(q, k, v, batch, seq_len, n_q_heads, n_kv_heads, head_dim, max_seq_len, o, q_lo=None,
+                         o_lo=None):
+    _check(lib().ladder_op_prefill_attention(_ptr(q), _ptr(q_lo), _ptr(k), _ptr(v), batch, seq_len, n_q_heads,
+                                             n_kv_heads, head_dim, max_seq_len, _ptr(o), _ptr(o_lo), _stream()))

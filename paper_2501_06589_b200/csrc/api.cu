@@ -48,13 +48,15 @@ struct ladder_model {
   // workspace (device)
   float* R[2] = {nullptr, nullptr};
   float* q_f32 = nullptr;           // decode [max_batch, Hq*Dh]
-  __nv_bfloat16* o_dec = nullptr;   // decode [max_batch, Hq*Dh]
-  __nv_bfloat16* h_dec = nullptr;   // decode [max_batch, F]
+  float* o_dec = nullptr;           // decode [max_batch, Hq*Dh]
+  float* h_dec = nullptr;           // decode [max_batch, F]
   float* attn_scratch = nullptr;
   int attn_splits = 1;
   float* logits_ws = nullptr;       // [max_batch, V]
   float* last_x = nullptr;          // [max_batch, d]
-  __nv_bfloat16 *n_pf = nullptr, *q_pf = nullptr, *o_pf = nullptr, *h_pf = nullptr;  // prefill activations
+  // prefill activations, each a bf16 hi part followed by a lo part (value ~ hi + lo)
+  __nv_bfloat16 *n_pf = nullptr, *q_pf = nullptr, *o_pf = nullptr, *h_pf = nullptr;
+  size_t n_lo = 0, q_lo = 0, h_lo = 0;  // element offsets of the lo parts
   float2* rope = nullptr;
   int32_t* status = nullptr;
   int32_t *tok_tmp = nullptr, *next_tmp = nullptr;
@@ -240,7 +242,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       o.N = d;
       o.K = Hq * Dh;
       o.act = m->o_dec;
-      o.act_mode = ACT_BF16;
+      o.act_mode = ACT_F32;
       o.batch = batch;
       o.epi_mode = EPI_RESID;
       o.addend = m->R[r.add];
@@ -278,7 +280,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       o.N = d;
       o.K = F;
       o.act = m->h_dec;
-      o.act_mode = ACT_BF16;
+      o.act_mode = ACT_F32;
       o.batch = batch;
       o.epi_mode = EPI_RESID;
       o.addend = m->R[r.add];
@@ -331,15 +333,17 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
     const bool lad = m->is_ladder[l] != 0;
     {
       const Router::Route r = rt.next(lad, 2 * l + 1);
-      did(launch_rmsnorm_bf16(m->R[r.in], m->attn_norm[l], c.rms_eps, M, d, m->n_pf, st));
+      did(launch_rmsnorm_bf16(m->R[r.in], m->attn_norm[l], c.rms_eps, M, d, m->n_pf, m->n_pf + m->n_lo, st));
       LargeMParams p = {};
       p.A = m->n_pf;
+      p.A_lo = m->n_pf + m->n_lo;
       p.W = m->w_qkv[l];
       p.M = M;
       p.N = (Hq + 2 * Hkv) * Dh;
       p.K = d;
       p.epi_mode = EPI_QKV_ROPE;
       p.qkv.q_out_bf16 = m->q_pf;
+      p.qkv.q_out_lo = m->q_pf + m->q_lo;
       p.qkv.k_cache = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
       p.qkv.v_cache = static_cast<__nv_bfloat16*>(cache->v) + l * layer_elems;
       p.qkv.rope = m->rope;
@@ -349,10 +353,11 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       p.qkv.max_seq_len = c.max_seq_len;
       p.qkv.prefill_seq_len = S;
       did(launch_largem_gemm(p, st));
-      did(launch_prefill_attention(m->q_pf, p.qkv.k_cache, p.qkv.v_cache, batch, S, Hq, Hkv, Dh, c.max_seq_len, m->o_pf,
-                                   st));
+      did(launch_prefill_attention(m->q_pf, m->q_pf + m->q_lo, p.qkv.k_cache, p.qkv.v_cache, batch, S, Hq, Hkv, Dh,
+                                   c.max_seq_len, m->o_pf, m->o_pf + m->q_lo, st));
       LargeMParams o = {};
       o.A = m->o_pf;
+      o.A_lo = m->o_pf + m->q_lo;
       o.W = m->w_o[l];
       o.M = M;
       o.N = d;
@@ -364,18 +369,21 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
     }
     {
       const Router::Route r = rt.next(lad, 2 * l + 2);
-      did(launch_rmsnorm_bf16(m->R[r.in], m->mlp_norm[l], c.rms_eps, M, d, m->n_pf, st));
+      did(launch_rmsnorm_bf16(m->R[r.in], m->mlp_norm[l], c.rms_eps, M, d, m->n_pf, m->n_pf + m->n_lo, st));
       LargeMParams p = {};
       p.A = m->n_pf;
+      p.A_lo = m->n_pf + m->n_lo;
       p.W = m->w_gate_up[l];
       p.M = M;
       p.N = 2 * F;
       p.K = d;
       p.epi_mode = EPI_SWIGLU;
       p.out = m->h_pf;
+      p.out_lo = m->h_pf + m->h_lo;
       did(launch_largem_gemm(p, st));
       LargeMParams o = {};
       o.A = m->h_pf;
+      o.A_lo = m->h_pf + m->h_lo;
       o.W = m->w_down[l];
       o.M = M;
       o.N = d;
@@ -512,10 +520,13 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   A(dev_alloc(&m->attn_scratch, scratch_floats));
   A(dev_alloc(&m->logits_ws, MB * c.vocab_size));
   A(dev_alloc(&m->last_x, MB * d));
-  A(dev_alloc(&m->n_pf, MP * d));
-  A(dev_alloc(&m->q_pf, MP * qd));
-  A(dev_alloc(&m->o_pf, MP * qd));
-  A(dev_alloc(&m->h_pf, MP * F));
+  m->n_lo = MP * d;
+  m->q_lo = MP * qd;
+  m->h_lo = MP * F;
+  A(dev_alloc(&m->n_pf, 2 * MP * d));
+  A(dev_alloc(&m->q_pf, 2 * MP * qd));
+  A(dev_alloc(&m->o_pf, 2 * MP * qd));
+  A(dev_alloc(&m->h_pf, 2 * MP * F));
   A(dev_alloc(&m->rope, static_cast<size_t>(c.max_seq_len) * (c.head_dim / 2)));
   A(dev_alloc(&m->status, 4));
   A(dev_alloc(&m->tok_tmp, MP > MB ? MP : MB));
@@ -737,7 +748,7 @@ ladder_status_t ladder_op_smallm_gemm(const void* W, int32_t N, int32_t K, const
                                       const void* gain, float eps, int32_t batch, int32_t epi_mode, const float* addend,
                                       void* out, void* cuda_stream) {
   if (!W || !act || !out || N < 8 || K < 8 || (N % 8) || (K % 8) || batch < 1 || batch > 64) return LADDER_ERR_INVALID_ARG;
-  if (act_mode != ACT_BF16 && act_mode != ACT_F32_NORM) return LADDER_ERR_INVALID_ARG;
+  if (act_mode != ACT_F32 && act_mode != ACT_F32_NORM) return LADDER_ERR_INVALID_ARG;
   if (act_mode == ACT_F32_NORM && !gain) return LADDER_ERR_INVALID_ARG;
   if (epi_mode != EPI_RESID && epi_mode != EPI_SWIGLU && epi_mode != EPI_PLAIN) return LADDER_ERR_INVALID_ARG;
   if (epi_mode == EPI_RESID && !addend) return LADDER_ERR_INVALID_ARG;
@@ -790,15 +801,16 @@ ladder_status_t ladder_op_decode_attention(const float* q, const void* k, const 
   a.max_len = max_seq_len;
   a.n_splits = op_attn_splits(batch, n_kv_heads, max_seq_len);
   a.scratch = scratch;
-  a.o = static_cast<__nv_bfloat16*>(o);
+  a.o = static_cast<float*>(o);
   // ticket counters at the head of the scratch must start at zero
   const size_t counters = (static_cast<size_t>(batch) * n_q_heads + 63) / 64 * 64;
   if (cudaMemsetAsync(scratch, 0, counters * sizeof(float), st) != cudaSuccess) return LADDER_ERR_CUDA;
   return launch_decode_attention(a, st, false) == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
 }
 
-ladder_status_t ladder_op_prefill_gemm(const void* A, const void* W, int32_t M, int32_t N, int32_t K, int32_t epi_mode,
-                                       const float* addend, void* out, void* cuda_stream) {
+ladder_status_t ladder_op_prefill_gemm(const void* A, const void* A_lo, const void* W, int32_t M, int32_t N, int32_t K,
+                                       int32_t epi_mode, const float* addend, void* out, void* out_lo,
+                                       void* cuda_stream) {
   if (!A || !W || !out || M < 1 || N < 8 || K < 8 || (N % 8) || (K % 8)) return LADDER_ERR_INVALID_ARG;
   int mode;
   switch (epi_mode) {
@@ -811,6 +823,8 @@ ladder_status_t ladder_op_prefill_gemm(const void* A, const void* W, int32_t M, 
   if (mode == EPI_RESID && !addend) return LADDER_ERR_INVALID_ARG;
   LargeMParams p = {};
   p.A = static_cast<const __nv_bfloat16*>(A);
+  p.A_lo = static_cast<const __nv_bfloat16*>(A_lo);
+  p.out_lo = static_cast<__nv_bfloat16*>(out_lo);
   p.W = static_cast<const __nv_bfloat16*>(W);
   p.M = M;
   p.N = N;
@@ -822,17 +836,18 @@ ladder_status_t ladder_op_prefill_gemm(const void* A, const void* W, int32_t M, 
   return launch_largem_gemm(p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
 }
 
-ladder_status_t ladder_op_prefill_attention(const void* q, const void* k, const void* v, int32_t batch, int32_t seq_len,
-                                            int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t max_seq_len,
-                                            void* o, void* cuda_stream) {
+ladder_status_t ladder_op_prefill_attention(const void* q, const void* q_lo, const void* k, const void* v, int32_t batch,
+                                            int32_t seq_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                            int32_t max_seq_len, void* o, void* o_lo, void* cuda_stream) {
   if (!q || !k || !v || !o || batch < 1 || seq_len < 1 || seq_len > max_seq_len || n_kv_heads < 1 ||
       n_q_heads % n_kv_heads || (head_dim != 64 && head_dim != 128))
     return LADDER_ERR_INVALID_ARG;
   if (kernels_ready() != cudaSuccess) return LADDER_ERR_CUDA;
-  cudaError_t e = launch_prefill_attention(static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
-                                           static_cast<const __nv_bfloat16*>(v), batch, seq_len, n_q_heads, n_kv_heads,
-                                           head_dim, max_seq_len, static_cast<__nv_bfloat16*>(o),
-                                           static_cast<cudaStream_t>(cuda_stream));
+  if ((q_lo == nullptr) != (o_lo == nullptr)) return LADDER_ERR_INVALID_ARG;
+  cudaError_t e = launch_prefill_attention(
+      static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(q_lo), static_cast<const __nv_bfloat16*>(k),
+      static_cast<const __nv_bfloat16*>(v), batch, seq_len, n_q_heads, n_kv_heads, head_dim, max_seq_len,
+      static_cast<__nv_bfloat16*>(o), static_cast<__nv_bfloat16*>(o_lo), static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
 }
 

@@ -8,7 +8,7 @@
 //   3. accumulates P.V on the CUDA cores (each warp walks keys, each lane owns Dh/32 dims),
 //   4. writes (o, m, l) partials to an L2-resident scratch, and the LAST CTA of a head group to
 //      arrive (atomic ticket, no spinning) merges the partials by log-sum-exp in a fixed order
-//      and writes o as bf16.  The ticket counters clean themselves up for the next launch.
+//      and writes o in fp32.  The ticket counters clean themselves up for the next launch.
 // The kernel is latency- not bandwidth-bound (KV is ~1 % of the bytes of a decode step); its
 // shared-memory footprint is kept small so it can co-reside with a weight-streaming GEMM CTA.
 #include "common.cuh"
@@ -51,7 +51,8 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
   const float scale = rsqrtf(static_cast<float>(DH));
 
   // ---- 1. scores
-  uint32_t qa[KJ][2][2];  // [j][half][pair]: bf16x2 of q[head0+g][j*32 + tig*8 + half*4 + 2*pair ..+1]
+  // q as a bf16 hi + lo pair (q ~ hi + lo), so the fp32 query loses nothing on its way into the MMA
+  uint32_t qa[KJ][2][2], ql[KJ][2][2];  // [j][half][pair]: q[head0+g][j*32 + tig*8 + half*4 + 2*pair ..+1]
 #pragma unroll
   for (int j = 0; j < KJ; ++j)
 #pragma unroll
@@ -62,6 +63,8 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
                                              tig * 8 + h * 4);
       qa[j][h][0] = pack_bf16x2(v.x, v.y);
       qa[j][h][1] = pack_bf16x2(v.z, v.w);
+      ql[j][h][0] = pack_bf16x2(v.x - bf16_lo(qa[j][h][0]), v.y - bf16_hi(qa[j][h][0]));
+      ql[j][h][1] = pack_bf16x2(v.z - bf16_lo(qa[j][h][1]), v.w - bf16_hi(qa[j][h][1]));
     }
   for (int kb = warp * 8; kb < nk; kb += 32) {
     const int key = k_begin + kb + g;
@@ -75,6 +78,8 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
     for (int j = 0; j < KJ; ++j) {
       mma_bf16_16816(c, qa[j][0][0], 0u, qa[j][0][1], 0u, kf[j].x, kf[j].y);
       mma_bf16_16816(c, qa[j][1][0], 0u, qa[j][1][1], 0u, kf[j].z, kf[j].w);
+      mma_bf16_16816(c, ql[j][0][0], 0u, ql[j][0][1], 0u, kf[j].x, kf[j].y);
+      mma_bf16_16816(c, ql[j][1][0], 0u, ql[j][1][1], 0u, kf[j].z, kf[j].w);
     }
     if (g < GT) {
       const int c0 = kb + 2 * tig;
@@ -173,7 +178,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
       lsum += w * __ldcg(base + s * stride + DH + 1);
       o += w * __ldcg(base + s * stride + d);
     }
-    p.o[(static_cast<size_t>(b) * p.n_q_heads + head0 + h) * DH + d] = __float2bfloat16_rn(lsum > 0.f ? o / lsum : 0.f);
+    p.o[(static_cast<size_t>(b) * p.n_q_heads + head0 + h) * DH + d] = lsum > 0.f ? o / lsum : 0.f;
   }
 }
 

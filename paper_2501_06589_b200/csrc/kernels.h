@@ -6,13 +6,14 @@
 
 namespace ladder {
 
-enum ActMode { ACT_BF16 = 0, ACT_F32_NORM = 1 };
+enum ActMode { ACT_F32 = 0, ACT_F32_NORM = 1 };  // activations are fp32 [batch, K]; NORM applies RMSNorm
 enum EpiMode { EPI_RESID = 0, EPI_SWIGLU = 1, EPI_PLAIN = 2, EPI_QKV_ROPE = 3, EPI_BF16 = 4 };
 
 // Rotary / KV-append epilogue description shared by the decode and prefill QKV projections.
 struct QkvEpilogue {
   float* q_out_f32;            // decode: fp32 [batch, Hq*Dh]
-  __nv_bfloat16* q_out_bf16;   // prefill: bf16 [M, Hq*Dh]
+  __nv_bfloat16* q_out_bf16;   // prefill: bf16 [M, Hq*Dh] (hi part)
+  __nv_bfloat16* q_out_lo;     // prefill: lo part (q ~ hi + lo), may be NULL
   __nv_bfloat16* k_cache;      // one layer: [max_batch][Hkv][max_seq][Dh]
   __nv_bfloat16* v_cache;
   const int32_t* seq_lens;     // decode: position of row b = seq_lens[b]; prefill: NULL (position = m % seq_len)
@@ -24,14 +25,14 @@ struct QkvEpilogue {
 struct SmallMParams {
   const __nv_bfloat16* W;  // [N, K]
   int N, K;
-  const void* act;         // ACT_BF16: bf16 [batch, K]; ACT_F32_NORM: fp32 [batch, K]
+  const void* act;         // fp32 [batch, K]
   int act_mode;
   const __nv_bfloat16* gain;  // [K] (ACT_F32_NORM)
   float eps;
   int batch;
   int epi_mode;
   const float* addend;     // EPI_RESID: fp32 [batch, N]
-  void* out;               // EPI_RESID / EPI_PLAIN: fp32 [batch, N]; EPI_SWIGLU: bf16 [batch, N/2]
+  void* out;               // EPI_RESID / EPI_PLAIN: fp32 [batch, N]; EPI_SWIGLU: fp32 [batch, N/2]
   QkvEpilogue qkv;         // EPI_QKV_ROPE
   int32_t* status;         // device status word (may be NULL)
 };
@@ -50,7 +51,7 @@ struct DecodeAttnParams {
   int n_splits;                 // CTAs per (b, kv head); each covers ceil(max_len / n_splits) keys
   int max_len;                  // host upper bound on keys attended (sizes the split)
   float* scratch;               // [batch][Hq][n_splits][Dh + 2]
-  __nv_bfloat16* o;             // [batch, Hq*Dh]
+  float* o;                     // [batch, Hq*Dh]
 };
 int decode_attention_splits(int batch, int n_kv_heads, int max_len, int sm_count);
 size_t decode_attention_scratch_floats(int batch, int n_q_heads, int head_dim, int n_splits);
@@ -58,25 +59,29 @@ cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stre
 
 // Prefill kernels.
 struct LargeMParams {
-  const __nv_bfloat16* A;  // [M, K]
+  const __nv_bfloat16* A;  // [M, K] (hi part)
+  const __nv_bfloat16* A_lo;  // [M, K] lo part with activation ~ A + A_lo, or NULL (single bf16)
   const __nv_bfloat16* W;  // [N, K]
   int M, N, K;
   int epi_mode;
   const float* addend;     // EPI_RESID
   void* out;
+  __nv_bfloat16* out_lo;   // EPI_SWIGLU / EPI_BF16: lo part of the bf16 output, or NULL
   QkvEpilogue qkv;
 };
 cudaError_t launch_largem_gemm(const LargeMParams& p, cudaStream_t stream);
 
-cudaError_t launch_prefill_attention(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                                     int batch, int seq_len, int n_q_heads, int n_kv_heads, int head_dim,
-                                     int max_seq_len, __nv_bfloat16* o, cudaStream_t stream);
+// q_lo / o_lo: optional lo parts (value ~ hi + lo) of the query input and the attention output.
+cudaError_t launch_prefill_attention(const __nv_bfloat16* q, const __nv_bfloat16* q_lo, const __nv_bfloat16* k,
+                                     const __nv_bfloat16* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
+                                     int head_dim, int max_seq_len, __nv_bfloat16* o, __nv_bfloat16* o_lo,
+                                     cudaStream_t stream);
 
 // Small element-wise / gather kernels.
 cudaError_t launch_embed(const int32_t* tokens, const __nv_bfloat16* table, int rows, int d, int vocab, float* x,
                          int32_t* status, cudaStream_t stream, bool pdl);
 cudaError_t launch_rmsnorm_bf16(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d,
-                                __nv_bfloat16* out, cudaStream_t stream);
+                                __nv_bfloat16* out, __nv_bfloat16* out_lo, cudaStream_t stream);
 cudaError_t launch_rmsnorm_f32(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, int row_stride,
                                float* out, cudaStream_t stream, bool pdl);
 cudaError_t launch_gather_rows(const float* x, int rows, int d, int src_stride_rows, int src_offset_rows, float* out,

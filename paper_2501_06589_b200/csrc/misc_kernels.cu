@@ -52,8 +52,10 @@ __device__ __forceinline__ float block_sum(float v, float* sh) {
 }
 
 // y = x / sqrt(mean(x^2) + eps) * gain, one CTA per row; OUT = bf16 or fp32.
+// bf16 output is written as a hi part and (if out_lo) a lo part with y ~ hi + lo.
 template <typename OUT>
-__global__ void rmsnorm_kernel(const float* x, const __nv_bfloat16* gain, float eps, int d, int row_stride, OUT* out) {
+__global__ void rmsnorm_kernel(const float* x, const __nv_bfloat16* gain, float eps, int d, int row_stride, OUT* out,
+                               OUT* out_lo) {
   __shared__ float sh[32];
   pdl_launch_dependents();
   pdl_wait();
@@ -71,7 +73,12 @@ __global__ void rmsnorm_kernel(const float* x, const __nv_bfloat16* gain, float 
     const float y0 = v.x * rstd * bf16_lo(gq.x), y1 = v.y * rstd * bf16_hi(gq.x);
     const float y2 = v.z * rstd * bf16_lo(gq.y), y3 = v.w * rstd * bf16_hi(gq.y);
     if (sizeof(OUT) == 2) {
-      reinterpret_cast<uint2*>(o)[i] = make_uint2(pack_bf16x2(y0, y1), pack_bf16x2(y2, y3));
+      const uint2 hi = make_uint2(pack_bf16x2(y0, y1), pack_bf16x2(y2, y3));
+      reinterpret_cast<uint2*>(o)[i] = hi;
+      if (out_lo)
+        reinterpret_cast<uint2*>(out_lo + static_cast<size_t>(blockIdx.x) * d)[i] =
+            make_uint2(pack_bf16x2(y0 - bf16_lo(hi.x), y1 - bf16_hi(hi.x)),
+                       pack_bf16x2(y2 - bf16_lo(hi.y), y3 - bf16_hi(hi.y)));
     } else {
       reinterpret_cast<float4*>(o)[i] = make_float4(y0, y1, y2, y3);
     }
@@ -143,13 +150,14 @@ cudaError_t launch_embed(const int32_t* tokens, const __nv_bfloat16* table, int 
 }
 
 cudaError_t launch_rmsnorm_bf16(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d,
-                                __nv_bfloat16* out, cudaStream_t stream) {
-  return launch(rmsnorm_kernel<__nv_bfloat16>, dim3(rows), dim3(256), stream, false, x, gain, eps, d, d, out);
+                                __nv_bfloat16* out, __nv_bfloat16* out_lo, cudaStream_t stream) {
+  return launch(rmsnorm_kernel<__nv_bfloat16>, dim3(rows), dim3(256), stream, false, x, gain, eps, d, d, out, out_lo);
 }
 
 cudaError_t launch_rmsnorm_f32(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, int row_stride,
                                float* out, cudaStream_t stream, bool pdl) {
-  return launch(rmsnorm_kernel<float>, dim3(rows), dim3(256), stream, pdl, x, gain, eps, d, row_stride, out);
+  return launch(rmsnorm_kernel<float>, dim3(rows), dim3(256), stream, pdl, x, gain, eps, d, row_stride, out,
+                static_cast<float*>(nullptr));
 }
 
 cudaError_t launch_gather_rows(const float* x, int rows, int d, int src_stride_rows, int src_offset_rows, float* out,

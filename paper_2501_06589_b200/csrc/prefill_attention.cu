@@ -27,23 +27,26 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
                : "r"(addr));
 }
 
-template <int DH>
+// SPLIT: the query comes as a bf16 hi + lo pair and the output is written as one (value ~ hi + lo).
+template <int DH, bool SPLIT>
 __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __nv_bfloat16* __restrict__ q,
+                                                                       const __nv_bfloat16* __restrict__ q_lo,
                                                                        const __nv_bfloat16* __restrict__ kc,
                                                                        const __nv_bfloat16* __restrict__ vc, int seq_len,
                                                                        int n_q_heads, int n_kv_heads, int max_seq_len,
-                                                                       __nv_bfloat16* __restrict__ o) {
+                                                                       __nv_bfloat16* __restrict__ o,
+                                                                       __nv_bfloat16* __restrict__ o_lo) {
   constexpr int P = DH + 8;  // smem pitch in elements
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __nv_bfloat16* sQ = reinterpret_cast<__nv_bfloat16*>(smem_raw);
   __nv_bfloat16* sK = sQ + kQT * P;
   __nv_bfloat16* sV = sK + kKT * P;
+  __nv_bfloat16* sQl = sV + kKT * P;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tig = lane & 3;
   const int q0 = blockIdx.x * kQT, h = blockIdx.y, b = blockIdx.z;
   const int kvh = h / (n_q_heads / n_kv_heads);
   const size_t qrow_stride = static_cast<size_t>(n_q_heads) * DH;
-  const __nv_bfloat16* qg = q + (static_cast<size_t>(b) * seq_len) * qrow_stride + static_cast<size_t>(h) * DH;
   const __nv_bfloat16* kg = kc + (static_cast<size_t>(b) * n_kv_heads + kvh) * max_seq_len * DH;
   const __nv_bfloat16* vg = vc + (static_cast<size_t>(b) * n_kv_heads + kvh) * max_seq_len * DH;
   constexpr int CPR = DH / 8;  // 16-byte chunks per row
@@ -51,7 +54,10 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
   for (int i = tid; i < kQT * CPR; i += kPfThreads) {
     const int r = i / CPR, c = i % CPR;
     const bool v = q0 + r < seq_len;
-    cp16(smem_u32(sQ + r * P + c * 8), qg + (v ? static_cast<size_t>(q0 + r) * qrow_stride + c * 8 : 0), v);
+    const size_t off = (static_cast<size_t>(b) * seq_len) * qrow_stride + static_cast<size_t>(h) * DH +
+                       (v ? static_cast<size_t>(q0 + r) * qrow_stride + c * 8 : 0);
+    cp16(smem_u32(sQ + r * P + c * 8), q + off, v);
+    if (SPLIT) cp16(smem_u32(sQl + r * P + c * 8), q_lo + off, v);
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
 
@@ -87,14 +93,19 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
       for (int c = 0; c < 4; ++c) s[i][c] = 0.f;
 #pragma unroll
     for (int ks = 0; ks < DH; ks += 16) {
-      uint32_t a0, a1, a2, a3;
+      uint32_t a0, a1, a2, a3, l0 = 0, l1 = 0, l2 = 0, l3 = 0;
       ldsm_x4(smem_u32(sQ + (warp * 16 + (lane & 15)) * P + ks + (lane >> 4) * 8), a0, a1, a2, a3);
+      if (SPLIT) ldsm_x4(smem_u32(sQl + (warp * 16 + (lane & 15)) * P + ks + (lane >> 4) * 8), l0, l1, l2, l3);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         uint32_t b0, b1, b2, b3;
         ldsm_x4(smem_u32(sK + (j * 16 + (lane & 7) + (lane >> 4) * 8) * P + ks + ((lane >> 3) & 1) * 8), b0, b1, b2, b3);
         mma_bf16_16816(s[2 * j], a0, a1, a2, a3, b0, b1);
         mma_bf16_16816(s[2 * j + 1], a0, a1, a2, a3, b2, b3);
+        if (SPLIT) {
+          mma_bf16_16816(s[2 * j], l0, l1, l2, l3, b0, b1);
+          mma_bf16_16816(s[2 * j + 1], l0, l1, l2, l3, b2, b3);
+        }
       }
     }
 
@@ -169,37 +180,55 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
     const int qi = q0 + warp * 16 + g + r * 8;
     if (qi >= seq_len) continue;
     const float inv = l_run[r] > 0.f ? 1.f / l_run[r] : 0.f;
-    __nv_bfloat16* dst = o + (static_cast<size_t>(b) * seq_len + qi) * qrow_stride + static_cast<size_t>(h) * DH;
+    const size_t doff = (static_cast<size_t>(b) * seq_len + qi) * qrow_stride + static_cast<size_t>(h) * DH;
 #pragma unroll
-    for (int i = 0; i < DH / 8; ++i)
-      *reinterpret_cast<uint32_t*>(dst + i * 8 + tig * 2) = pack_bf16x2(oacc[i][2 * r] * inv, oacc[i][2 * r + 1] * inv);
+    for (int i = 0; i < DH / 8; ++i) {
+      const float v0 = oacc[i][2 * r] * inv, v1 = oacc[i][2 * r + 1] * inv;
+      const uint32_t hi = pack_bf16x2(v0, v1);
+      *reinterpret_cast<uint32_t*>(o + doff + i * 8 + tig * 2) = hi;
+      if (SPLIT) *reinterpret_cast<uint32_t*>(o_lo + doff + i * 8 + tig * 2) = pack_bf16x2(v0 - bf16_lo(hi), v1 - bf16_hi(hi));
+    }
   }
 }
 
-template <int DH>
-cudaError_t launch_dh(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v, int batch, int seq_len,
-                      int n_q_heads, int n_kv_heads, int max_seq_len, __nv_bfloat16* o, cudaStream_t stream) {
-  constexpr int smem = 3 * 64 * (DH + 8) * 2;
+template <int DH, bool SPLIT>
+cudaError_t launch_dh(const __nv_bfloat16* q, const __nv_bfloat16* q_lo, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                      int batch, int seq_len, int n_q_heads, int n_kv_heads, int max_seq_len, __nv_bfloat16* o,
+                      __nv_bfloat16* o_lo, cudaStream_t stream) {
+  constexpr int smem = 4 * 64 * (DH + 8) * 2;
   dim3 grid((seq_len + kQT - 1) / kQT, n_q_heads, batch);
-  prefill_attention_kernel<DH><<<grid, kPfThreads, smem, stream>>>(q, k, v, seq_len, n_q_heads, n_kv_heads, max_seq_len, o);
+  prefill_attention_kernel<DH, SPLIT><<<grid, kPfThreads, smem, stream>>>(q, q_lo, k, v, seq_len, n_q_heads, n_kv_heads,
+                                                                          max_seq_len, o, o_lo);
   return cudaGetLastError();
+}
+
+template <int DH, bool SPLIT>
+cudaError_t init_dh() {
+  return cudaFuncSetAttribute(prefill_attention_kernel<DH, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              4 * 64 * (DH + 8) * 2);
 }
 
 }  // namespace
 
 cudaError_t prefill_attention_init() {
-  cudaError_t e = cudaFuncSetAttribute(prefill_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       3 * 64 * (128 + 8) * 2);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(prefill_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              3 * 64 * (64 + 8) * 2);
+  cudaError_t e = init_dh<128, true>();
+  if (e == cudaSuccess) e = init_dh<128, false>();
+  if (e == cudaSuccess) e = init_dh<64, true>();
+  if (e == cudaSuccess) e = init_dh<64, false>();
+  return e;
 }
 
-cudaError_t launch_prefill_attention(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v, int batch,
-                                     int seq_len, int n_q_heads, int n_kv_heads, int head_dim, int max_seq_len,
-                                     __nv_bfloat16* o, cudaStream_t stream) {
-  if (head_dim == 128) return launch_dh<128>(q, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, stream);
-  if (head_dim == 64) return launch_dh<64>(q, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, stream);
+cudaError_t launch_prefill_attention(const __nv_bfloat16* q, const __nv_bfloat16* q_lo, const __nv_bfloat16* k,
+                                     const __nv_bfloat16* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
+                                     int head_dim, int max_seq_len, __nv_bfloat16* o, __nv_bfloat16* o_lo,
+                                     cudaStream_t stream) {
+  const bool split = q_lo != nullptr && o_lo != nullptr;
+  if (head_dim == 128)
+    return split ? launch_dh<128, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream)
+                 : launch_dh<128, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream);
+  if (head_dim == 64)
+    return split ? launch_dh<64, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream)
+                 : launch_dh<64, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream);
   return cudaErrorInvalidValue;
 }
 

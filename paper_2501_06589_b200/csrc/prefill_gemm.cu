@@ -2,6 +2,9 @@
 // with the fused epilogues of the layer: residual add (Eq. 1 / Eq. 2 of the paper), SwiGLU over
 // interleaved gate/up rows, rotary embedding + KV-cache append, plain stores.
 //
+// Activations may come as a bf16 hi + lo pair (a ~ hi + lo): both tiles are staged and multiplied
+// with the same weight tile, which removes the activation rounding error at twice the MMA count.
+//
 // This file holds the warp-level (mma.sync) implementation: 128x128x32 CTA tiles, 3-stage
 // cp.async pipeline, ldmatrix fragments, 8 warps of 64x32.  Adjacent output columns (2j, 2j+1)
 // live in one thread, which is what the pair-wise epilogues (SwiGLU, rotary) need.
@@ -14,7 +17,7 @@ namespace {
 constexpr int BM = 128, BN = 128, BK = 32, STAGES = 3, PITCH = BK + 8;  // pitch in elements (80 bytes)
 constexpr int kGemmThreads = 256;
 constexpr int kTileElems = BM * PITCH;
-constexpr int kSmemBytes = STAGES * 2 * kTileElems * 2;
+constexpr int kSmemBytes = STAGES * 3 * kTileElems * 2;  // A hi, A lo, W
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
   const int sz = valid ? 16 : 0;  // zero-fill when out of range
@@ -42,16 +45,22 @@ __device__ __forceinline__ void epilogue_pair(const LargeMParams& p, int m, int 
     }
     case EPI_SWIGLU: {
       const float h = v0 / (1.f + __expf(-v0)) * v1;
-      static_cast<__nv_bfloat16*>(p.out)[static_cast<size_t>(m) * (p.N >> 1) + (n >> 1)] = __float2bfloat16_rn(h);
+      const size_t o = static_cast<size_t>(m) * (p.N >> 1) + (n >> 1);
+      const __nv_bfloat16 hi = __float2bfloat16_rn(h);
+      static_cast<__nv_bfloat16*>(p.out)[o] = hi;
+      if (p.out_lo) p.out_lo[o] = __float2bfloat16_rn(h - __bfloat162float(hi));
       break;
     }
     case EPI_PLAIN:
       *reinterpret_cast<float2*>(static_cast<float*>(p.out) + static_cast<size_t>(m) * p.N + n) = make_float2(v0, v1);
       break;
-    case EPI_BF16:
-      *reinterpret_cast<uint32_t*>(static_cast<__nv_bfloat16*>(p.out) + static_cast<size_t>(m) * p.N + n) =
-          pack_bf16x2(v0, v1);
+    case EPI_BF16: {
+      const size_t o = static_cast<size_t>(m) * p.N + n;
+      const uint32_t hi = pack_bf16x2(v0, v1);
+      *reinterpret_cast<uint32_t*>(static_cast<__nv_bfloat16*>(p.out) + o) = hi;
+      if (p.out_lo) *reinterpret_cast<uint32_t*>(p.out_lo + o) = pack_bf16x2(v0 - bf16_lo(hi), v1 - bf16_hi(hi));
       break;
+    }
     case EPI_QKV_ROPE: {
       const QkvEpilogue& e = p.qkv;
       const int Dh = e.head_dim, nq = e.n_q_heads * Dh, nk = e.n_kv_heads * Dh;
@@ -63,7 +72,11 @@ __device__ __forceinline__ void epilogue_pair(const LargeMParams& p, int m, int 
         v1 = a1;
       }
       if (n < nq) {
-        *reinterpret_cast<uint32_t*>(e.q_out_bf16 + static_cast<size_t>(m) * nq + n) = pack_bf16x2(v0, v1);
+        const uint32_t hi = pack_bf16x2(v0, v1);
+        *reinterpret_cast<uint32_t*>(e.q_out_bf16 + static_cast<size_t>(m) * nq + n) = hi;
+        if (e.q_out_lo)
+          *reinterpret_cast<uint32_t*>(e.q_out_lo + static_cast<size_t>(m) * nq + n) =
+              pack_bf16x2(v0 - bf16_lo(hi), v1 - bf16_hi(hi));
       } else {
         const int nn = n < nq + nk ? n - nq : n - nq - nk;
         __nv_bfloat16* cache = n < nq + nk ? e.k_cache : e.v_cache;
@@ -76,10 +89,12 @@ __device__ __forceinline__ void epilogue_pair(const LargeMParams& p, int m, int 
   }
 }
 
+template <bool SPLIT>
 __global__ void __launch_bounds__(kGemmThreads) largem_gemm_kernel(const LargeMParams p) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __nv_bfloat16* sA = reinterpret_cast<__nv_bfloat16*>(smem_raw);
   __nv_bfloat16* sB = sA + STAGES * kTileElems;
+  __nv_bfloat16* sL = sB + STAGES * kTileElems;  // lo part of A
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int wm = warp >> 2, wn = warp & 3;  // 2 x 4 warps, warp tile 64 x 32
@@ -99,6 +114,10 @@ __global__ void __launch_bounds__(kGemmThreads) largem_gemm_kernel(const LargeMP
       const __nv_bfloat16* gb = p.W + (vb ? static_cast<size_t>(n) * p.K + kc : 0);
       cp_async16(smem_u32(sA + st * kTileElems + r * PITCH + (tid & 3) * 8), ga, va);
       cp_async16(smem_u32(sB + st * kTileElems + r * PITCH + (tid & 3) * 8), gb, vb);
+      if (SPLIT) {
+        const __nv_bfloat16* gl = p.A_lo + (va ? static_cast<size_t>(m) * p.K + kc : 0);
+        cp_async16(smem_u32(sL + st * kTileElems + r * PITCH + (tid & 3) * 8), gl, va);
+      }
     }
   };
 
@@ -122,23 +141,28 @@ __global__ void __launch_bounds__(kGemmThreads) largem_gemm_kernel(const LargeMP
     cp_async_commit();
     const __nv_bfloat16* a = sA + (kt % STAGES) * kTileElems;
     const __nv_bfloat16* b = sB + (kt % STAGES) * kTileElems;
+    const __nv_bfloat16* al = sL + (kt % STAGES) * kTileElems;
 #pragma unroll
     for (int ks = 0; ks < BK; ks += 16) {
       uint32_t af[4][4], bfr[2][4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        ldmatrix_x4(smem_u32(a + (wm * 64 + i * 16 + (lane & 15)) * PITCH + ks + (lane >> 4) * 8), af[i][0], af[i][1],
-                    af[i][2], af[i][3]);
 #pragma unroll
       for (int j = 0; j < 2; ++j)
         ldmatrix_x4(smem_u32(b + (wn * 32 + j * 16 + (lane & 7) + (lane >> 4) * 8) * PITCH + ks + ((lane >> 3) & 1) * 8),
                     bfr[j][0], bfr[j][1], bfr[j][2], bfr[j][3]);
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int part = 0; part < (SPLIT ? 2 : 1); ++part) {
+        const __nv_bfloat16* src = part ? al : a;
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-          mma_bf16_16816(acc[i][j], af[i][0], af[i][1], af[i][2], af[i][3], bfr[j >> 1][(j & 1) * 2],
-                         bfr[j >> 1][(j & 1) * 2 + 1]);
+        for (int i = 0; i < 4; ++i)
+          ldmatrix_x4(smem_u32(src + (wm * 64 + i * 16 + (lane & 15)) * PITCH + ks + (lane >> 4) * 8), af[i][0],
+                      af[i][1], af[i][2], af[i][3]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            mma_bf16_16816(acc[i][j], af[i][0], af[i][1], af[i][2], af[i][3], bfr[j >> 1][(j & 1) * 2],
+                           bfr[j >> 1][(j & 1) * 2 + 1]);
+      }
     }
   }
   cp_async_wait<0>();
@@ -158,12 +182,15 @@ __global__ void __launch_bounds__(kGemmThreads) largem_gemm_kernel(const LargeMP
 }  // namespace
 
 cudaError_t largem_gemm_init() {
-  return cudaFuncSetAttribute(largem_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(largem_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(largem_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
 cudaError_t launch_largem_gemm(const LargeMParams& p, cudaStream_t stream) {
   dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM);
-  largem_gemm_kernel<<<grid, kGemmThreads, kSmemBytes, stream>>>(p);
+  if (p.A_lo) largem_gemm_kernel<true><<<grid, kGemmThreads, kSmemBytes, stream>>>(p);
+  else largem_gemm_kernel<false><<<grid, kGemmThreads, kSmemBytes, stream>>>(p);
   return cudaGetLastError();
 }
 

@@ -11,9 +11,12 @@
 //     contiguous bytes of a weight row and the matching 16 bytes of an activation row: the K
 //     index inside an MMA is permuted the same way for both operands, so no ldmatrix and no
 //     swizzle are needed; a row pitch of 64 mod 128 bytes keeps the 128-bit loads conflict-free;
-//   * activations are staged per K-chunk by the consumer warps (fp32 residual x gain -> bf16,
-//     sum of squares accumulated on the way, so RMSNorm costs one pass and its 1/rms factor is
-//     applied to the accumulators in the epilogue);
+//   * activations are fp32 in global memory and are staged per K-chunk by the consumer warps:
+//     (x * gain) is split into a bf16 high part and a bf16 low part (x ~ hi + lo, ~16 mantissa
+//     bits) and both are multiplied with the weight fragment, so the tensor-core operands are
+//     bf16 while the activation rounding error all but disappears -- the extra MMAs are free in
+//     a bandwidth-bound kernel.  The sum of squares is accumulated on the way, so RMSNorm costs
+//     one pass and its 1/rms factor is applied to the accumulators in the epilogue;
 //   * everything that does not depend on the previous kernel (barrier set-up, the first ring
 //     fill of weights) happens before griddepcontrol.wait, so with programmatic dependent
 //     launch the weight stream never drains between kernels;
@@ -28,38 +31,42 @@ namespace {
 
 constexpr int kThreads = 160;  // warp 0 = producer, warps 1..4 = consumers
 
-template <int NB>
+template <int NB, bool R4>
 struct Cfg {
   static constexpr int TK = NB == 1 ? 1024 : (NB == 2 ? 512 : 256);  // K elements per chunk
-  static constexpr int STAGES = NB == 1 ? 4 : (NB == 2 ? 8 : 12);
+  static constexpr int STAGES = NB == 1 ? 4 : (NB == 2 ? 7 : 12);
   static constexpr int PITCH = TK * 2 + 64;  // bytes between weight rows in a stage (64 mod 128)
   static constexpr int STAGE_BYTES = 16 * PITCH;
   static constexpr int APITCH = TK * 2 + 64;
-  static constexpr int ACT_ROWS = 8 * NB;
+  static constexpr bool SPLIT = NB <= 2;     // activations as bf16 hi + lo pair (batch <= 16)
+  static constexpr int PARTS = SPLIT ? 2 : 1;
+  static constexpr int ACT_ROWS = R4 ? 4 : 8 * NB;  // R4: batch <= 4 needs only 4 staged rows
   static constexpr int ACT_BYTES = ACT_ROWS * APITCH;
   static constexpr int RG_MAX = 8 / NB;    // 16-row groups whose accumulators live in registers at once
   static constexpr int SPW = TK / 32 / 4;  // 32-wide K slabs per consumer warp per chunk
   static constexpr int KQ = TK / 8;        // 16-byte units per activation row per chunk
   static constexpr int RL = 128 / KQ;      // consumer threads side by side along the batch
-  static constexpr int RPT = ACT_ROWS / RL;  // activation rows per thread
+  static constexpr int RPT = (ACT_ROWS + RL - 1) / RL;  // activation rows per thread
   static constexpr int PF = RPT < 4 ? RPT : 4;  // rows prefetched into registers one chunk ahead
   static constexpr int RED_FLOATS = 4 * RG_MAX * NB * 4 * 32;
-  static constexpr int SMEM = STAGES * STAGE_BYTES + 2 * ACT_BYTES + RED_FLOATS * 4 + (4 * 16 + 64) * 4 +
+  static constexpr int SMEM = STAGES * STAGE_BYTES + 2 * PARTS * ACT_BYTES + RED_FLOATS * 4 + (4 * 16 + 64) * 4 +
                               2 * STAGES * 8 + 16 + 128;
+  static_assert(!R4 || NB == 1, "R4 is a variant of the batch <= 8 kernel");
+  static_assert(SMEM <= 232448, "exceeds the 227 KB of shared memory a CTA can opt in to");
 };
 
 struct F8 {
   float4 a, b;
 };
 
-template <int NB, int ACT>
+template <int NB, bool R4, bool NORM>
 __global__ void __launch_bounds__(kThreads, 1) smallm_gemm_kernel(const SmallMParams p) {
-  using C = Cfg<NB>;
+  using C = Cfg<NB, R4>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   uint8_t* ring = smem;
   uint8_t* act = ring + C::STAGES * C::STAGE_BYTES;
-  float* red = reinterpret_cast<float*>(act + 2 * C::ACT_BYTES);
+  float* red = reinterpret_cast<float*>(act + 2 * C::PARTS * C::ACT_BYTES);
   float* ssq_s = red + C::RED_FLOATS;  // [4 warps][16]
   float* rstd_s = ssq_s + 64;          // [64]
   uint64_t* full = reinterpret_cast<uint64_t*>(rstd_s + 64);
@@ -157,79 +164,67 @@ __global__ void __launch_bounds__(kThreads, 1) smallm_gemm_kernel(const SmallMPa
 #pragma unroll
     for (int i = 0; i < C::RPT; ++i) ssq[i] = 0.f;
 
-    // register prefetch of the raw activation chunk
+    // register prefetch of the raw fp32 activation chunk
     F8 pf_x[C::PF];
-    uint4 pf_h[C::PF];
-    uint4 pf_g = make_uint4(0, 0, 0, 0);
+    uint4 pf_g = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);  // gain 1.0
+    const float* actf = static_cast<const float*>(p.act);
+    auto load_x = [&](int b, int k, bool kv) -> F8 {
+      F8 x;
+      x.a = x.b = make_float4(0, 0, 0, 0);
+      if (kv && b < batch) {
+        const float4* src = reinterpret_cast<const float4*>(actf + static_cast<size_t>(b) * p.K + k);
+        x.a = src[0];
+        x.b = src[1];
+      }
+      return x;
+    };
     auto prefetch = [&](int ch) {
       const int k = ch * C::TK + kq * 8;
       const bool kv = k < p.K;
-      if (ACT == ACT_F32_NORM) {
-        pf_g = kv ? __ldg(reinterpret_cast<const uint4*>(p.gain + k)) : make_uint4(0, 0, 0, 0);
+      if (NORM) pf_g = kv ? __ldg(reinterpret_cast<const uint4*>(p.gain + k)) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-        for (int i = 0; i < C::PF; ++i) {
-          const int b = rl + i * C::RL;
-          if (kv && b < batch) {
-            const float4* src = reinterpret_cast<const float4*>(static_cast<const float*>(p.act) +
-                                                                static_cast<size_t>(b) * p.K + k);
-            pf_x[i].a = src[0];
-            pf_x[i].b = src[1];
-          } else {
-            pf_x[i].a = make_float4(0, 0, 0, 0);
-            pf_x[i].b = make_float4(0, 0, 0, 0);
-          }
-        }
-      } else {
-#pragma unroll
-        for (int i = 0; i < C::PF; ++i) {
-          const int b = rl + i * C::RL;
-          pf_h[i] = (kv && b < batch)
-                        ? *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.act) +
-                                                          static_cast<size_t>(b) * p.K + k)
-                        : make_uint4(0, 0, 0, 0);
-        }
+      for (int i = 0; i < C::PF; ++i) pf_x[i] = load_x(rl + i * C::RL, k, kv);
+    };
+    // y = x * gain, written as bf16 hi (and lo = bf16(y - hi)); sum of squares of x on the way
+    auto stage_row = [&](const F8& x, const uint4& gq, float& ss, uint32_t dst) {
+      float y[8] = {x.a.x, x.a.y, x.a.z, x.a.w, x.b.x, x.b.y, x.b.z, x.b.w};
+      if (NORM) {
+        ss += y[0] * y[0] + y[1] * y[1] + y[2] * y[2] + y[3] * y[3] + y[4] * y[4] + y[5] * y[5] + y[6] * y[6] +
+              y[7] * y[7];
+        y[0] *= bf16_lo(gq.x);
+        y[1] *= bf16_hi(gq.x);
+        y[2] *= bf16_lo(gq.y);
+        y[3] *= bf16_hi(gq.y);
+        y[4] *= bf16_lo(gq.z);
+        y[5] *= bf16_hi(gq.z);
+        y[6] *= bf16_lo(gq.w);
+        y[7] *= bf16_hi(gq.w);
+      }
+      uint4 hi;
+      hi.x = pack_bf16x2(y[0], y[1]);
+      hi.y = pack_bf16x2(y[2], y[3]);
+      hi.z = pack_bf16x2(y[4], y[5]);
+      hi.w = pack_bf16x2(y[6], y[7]);
+      sts128(dst, hi);
+      if (C::SPLIT) {
+        uint4 lo;
+        lo.x = pack_bf16x2(y[0] - bf16_lo(hi.x), y[1] - bf16_hi(hi.x));
+        lo.y = pack_bf16x2(y[2] - bf16_lo(hi.y), y[3] - bf16_hi(hi.y));
+        lo.z = pack_bf16x2(y[4] - bf16_lo(hi.z), y[5] - bf16_hi(hi.z));
+        lo.w = pack_bf16x2(y[6] - bf16_lo(hi.w), y[7] - bf16_hi(hi.w));
+        sts128(dst + C::ACT_BYTES, lo);
       }
     };
-    auto norm_pack = [&](const F8& x, const uint4& gq, float& ss) -> uint4 {
-      ss += x.a.x * x.a.x + x.a.y * x.a.y + x.a.z * x.a.z + x.a.w * x.a.w + x.b.x * x.b.x + x.b.y * x.b.y +
-            x.b.z * x.b.z + x.b.w * x.b.w;
-      uint4 o;
-      o.x = pack_bf16x2(x.a.x * bf16_lo(gq.x), x.a.y * bf16_hi(gq.x));
-      o.y = pack_bf16x2(x.a.z * bf16_lo(gq.y), x.a.w * bf16_hi(gq.y));
-      o.z = pack_bf16x2(x.b.x * bf16_lo(gq.z), x.b.y * bf16_hi(gq.z));
-      o.w = pack_bf16x2(x.b.z * bf16_lo(gq.w), x.b.w * bf16_hi(gq.w));
-      return o;
-    };
     auto stage_act = [&](int ch) {
-      const uint32_t dst = act_u32 + (ch & 1) * C::ACT_BYTES + kq * 16;
+      const uint32_t dst = act_u32 + (ch & 1) * C::PARTS * C::ACT_BYTES + kq * 16;
       const int k = ch * C::TK + kq * 8;
       const bool kv = k < p.K;
 #pragma unroll
       for (int i = 0; i < C::RPT; ++i) {
         const int b = rl + i * C::RL;
-        if (b >= batch) break;
-        uint4 o;
-        if (i < C::PF) {
-          if (ACT == ACT_F32_NORM) o = norm_pack(pf_x[i < C::PF ? i : 0], pf_g, ssq[i]);
-          else o = pf_h[i < C::PF ? i : 0];
-        } else {
-          if (ACT == ACT_F32_NORM) {
-            F8 x;
-            x.a = x.b = make_float4(0, 0, 0, 0);
-            if (kv) {
-              const float4* src = reinterpret_cast<const float4*>(static_cast<const float*>(p.act) +
-                                                                  static_cast<size_t>(b) * p.K + k);
-              x.a = src[0];
-              x.b = src[1];
-            }
-            o = norm_pack(x, pf_g, ssq[i]);
-          } else {
-            o = kv ? *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(p.act) +
-                                                     static_cast<size_t>(b) * p.K + k)
-                   : make_uint4(0, 0, 0, 0);
-          }
-        }
-        sts128(dst + b * C::APITCH, o);
+        if (b >= batch || b >= C::ACT_ROWS) break;
+        if (i < C::PF) stage_row(pf_x[i < C::PF ? i : 0], pf_g, ssq[i], dst + b * C::APITCH);
+        else stage_row(load_x(b, k, kv), pf_g, ssq[i], dst + b * C::APITCH);
       }
     };
 
@@ -240,17 +235,20 @@ __global__ void __launch_bounds__(kThreads, 1) smallm_gemm_kernel(const SmallMPa
       if (ch + 1 < nchunk) prefetch(ch + 1);
 
       // activation fragments of this warp's K slabs (reused by every row group of the pass)
-      uint4 bf[C::SPW][NB];
+      uint4 bf[C::PARTS][C::SPW][NB];
       const int k0 = ch * C::TK;
 #pragma unroll
-      for (int j = 0; j < C::SPW; ++j)
+      for (int pt = 0; pt < C::PARTS; ++pt)
 #pragma unroll
-        for (int nt = 0; nt < NB; ++nt) {
-          const int brow = nt * 8 + g;
-          bf[j][nt] = brow < batch ? lds128(act_u32 + (ch & 1) * C::ACT_BYTES + brow * C::APITCH +
-                                            (cw * C::SPW + j) * 64 + tig * 16)
-                                   : make_uint4(0, 0, 0, 0);
-        }
+        for (int j = 0; j < C::SPW; ++j)
+#pragma unroll
+          for (int nt = 0; nt < NB; ++nt) {
+            const int brow = nt * 8 + g;
+            bf[pt][j][nt] = (brow < batch && brow < C::ACT_ROWS)
+                                ? lds128(act_u32 + ((ch & 1) * C::PARTS + pt) * C::ACT_BYTES + brow * C::APITCH +
+                                         (cw * C::SPW + j) * 64 + tig * 16)
+                                : make_uint4(0, 0, 0, 0);
+          }
 
 #pragma unroll
       for (int rgi = 0; rgi < C::RG_MAX; ++rgi) {
@@ -269,10 +267,12 @@ __global__ void __launch_bounds__(kThreads, 1) smallm_gemm_kernel(const SmallMPa
             hi = lds128(base + 8 * C::PITCH + slab * 64);
           }
 #pragma unroll
-          for (int nt = 0; nt < NB; ++nt) {
-            mma_bf16_16816(acc[rgi][nt], lo.x, hi.x, lo.y, hi.y, bf[j][nt].x, bf[j][nt].y);
-            mma_bf16_16816(acc[rgi][nt], lo.z, hi.z, lo.w, hi.w, bf[j][nt].z, bf[j][nt].w);
-          }
+          for (int nt = 0; nt < NB; ++nt)
+#pragma unroll
+            for (int pt = 0; pt < C::PARTS; ++pt) {
+              mma_bf16_16816(acc[rgi][nt], lo.x, hi.x, lo.y, hi.y, bf[pt][j][nt].x, bf[pt][j][nt].y);
+              mma_bf16_16816(acc[rgi][nt], lo.z, hi.z, lo.w, hi.w, bf[pt][j][nt].z, bf[pt][j][nt].w);
+            }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[st]);
@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(kThreads, 1) smallm_gemm_kernel(const SmallMPa
       for (int nt = 0; nt < NB; ++nt)
 #pragma unroll
         for (int c = 0; c < 4; ++c) red[(((cw * C::RG_MAX + a) * NB + nt) * 4 + c) * 32 + lane] = acc[a][nt][c];
-    if (ACT == ACT_F32_NORM) {
+    if (NORM) {
 #pragma unroll
       for (int i = 0; i < C::RPT; ++i) {
         const float s = warp_sum(ssq[i]);
@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(kThreads, 1) smallm_gemm_kernel(const SmallMPa
       }
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");
-    if (ACT == ACT_F32_NORM) {
+    if (NORM) {
       if (ct < batch) {
         // row b = rl' + i*RL is staged by the warps whose threads have rl == rl'
         const int rlb = ct % C::RL, i = ct / C::RL;
@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(kThreads, 1) smallm_gemm_kernel(const SmallMPa
       float s = 0.f;
 #pragma unroll
       for (int w = 0; w < 4; ++w) s += red[w * (C::RG_MAX * NB * 128) + idx];
-      if (ACT == ACT_F32_NORM) s *= rstd_s[b];
+      if (NORM) s *= rstd_s[b];
       return s;
     };
 
@@ -329,13 +329,12 @@ __global__ void __launch_bounds__(kThreads, 1) smallm_gemm_kernel(const SmallMPa
         out[o] = v;
       }
     } else if (p.epi_mode == EPI_SWIGLU) {
-      __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.out);
+      float* out = static_cast<float*>(p.out);
       const int half = prow >> 1;
       for (int idx = ct; idx < half * batch; idx += 128) {
         const int pr = idx % half, b = idx / half;
         const float gt = value(2 * pr, b), up = value(2 * pr + 1, b);
-        const float h = gt / (1.f + __expf(-gt)) * up;
-        out[static_cast<size_t>(b) * (p.N >> 1) + ((nbase >> 1) + pr)] = __float2bfloat16_rn(h);
+        out[static_cast<size_t>(b) * (p.N >> 1) + ((nbase >> 1) + pr)] = gt / (1.f + __expf(-gt)) * up;
       }
     } else if (p.epi_mode == EPI_QKV_ROPE) {
       const QkvEpilogue& e = p.qkv;
@@ -372,10 +371,10 @@ __global__ void __launch_bounds__(kThreads, 1) smallm_gemm_kernel(const SmallMPa
   if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
 }
 
-template <int NB>
+template <int NB, bool R4>
 cudaError_t launch_nb(const SmallMParams& p, cudaStream_t stream, bool pdl, int grid) {
-  using C = Cfg<NB>;
-  auto kern = p.act_mode == ACT_F32_NORM ? smallm_gemm_kernel<NB, ACT_F32_NORM> : smallm_gemm_kernel<NB, ACT_BF16>;
+  using C = Cfg<NB, R4>;
+  auto kern = p.act_mode == ACT_F32_NORM ? smallm_gemm_kernel<NB, R4, true> : smallm_gemm_kernel<NB, R4, false>;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kThreads);
@@ -389,39 +388,42 @@ cudaError_t launch_nb(const SmallMParams& p, cudaStream_t stream, bool pdl, int 
   return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
-template <int NB>
+template <int NB, bool R4>
 cudaError_t init_nb() {
-  cudaError_t e = cudaFuncSetAttribute(smallm_gemm_kernel<NB, ACT_F32_NORM>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<NB>::SMEM);
+  cudaError_t e = cudaFuncSetAttribute(smallm_gemm_kernel<NB, R4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       Cfg<NB, R4>::SMEM);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(smallm_gemm_kernel<NB, ACT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Cfg<NB>::SMEM);
+  return cudaFuncSetAttribute(smallm_gemm_kernel<NB, R4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<NB, R4>::SMEM);
 }
 
 }  // namespace
 
 cudaError_t smallm_gemm_init() {
-  cudaError_t e = init_nb<1>();
-  if (e == cudaSuccess) e = init_nb<2>();
-  if (e == cudaSuccess) e = init_nb<4>();
-  if (e == cudaSuccess) e = init_nb<8>();
+  cudaError_t e = init_nb<1, true>();
+  if (e == cudaSuccess) e = init_nb<1, false>();
+  if (e == cudaSuccess) e = init_nb<2, false>();
+  if (e == cudaSuccess) e = init_nb<4, false>();
+  if (e == cudaSuccess) e = init_nb<8, false>();
   return e;
 }
 
 size_t smallm_gemm_smem_bytes(int batch) {
-  if (batch <= 8) return Cfg<1>::SMEM;
-  if (batch <= 16) return Cfg<2>::SMEM;
-  if (batch <= 32) return Cfg<4>::SMEM;
-  return Cfg<8>::SMEM;
+  if (batch <= 4) return Cfg<1, true>::SMEM;
+  if (batch <= 8) return Cfg<1, false>::SMEM;
+  if (batch <= 16) return Cfg<2, false>::SMEM;
+  if (batch <= 32) return Cfg<4, false>::SMEM;
+  return Cfg<8, false>::SMEM;
 }
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
   const int units = p.N >> 3;
   const int grid = units < sm_count ? units : sm_count;
-  if (p.batch <= 8) return launch_nb<1>(p, stream, pdl, grid);
-  if (p.batch <= 16) return launch_nb<2>(p, stream, pdl, grid);
-  if (p.batch <= 32) return launch_nb<4>(p, stream, pdl, grid);
-  return launch_nb<8>(p, stream, pdl, grid);
+  if (p.batch <= 4) return launch_nb<1, true>(p, stream, pdl, grid);
+  if (p.batch <= 8) return launch_nb<1, false>(p, stream, pdl, grid);
+  if (p.batch <= 16) return launch_nb<2, false>(p, stream, pdl, grid);
+  if (p.batch <= 32) return launch_nb<4, false>(p, stream, pdl, grid);
+  return launch_nb<8, false>(p, stream, pdl, grid);
 }
 
 }  // namespace ladder

@@ -74,7 +74,7 @@ def test_null_model_calls_are_rejected(L):
 def test_op_entry_points_validate_arguments(L):
     assert L.ladder_op_smallm_gemm(None, 8, 8, None, 0, None, 0.0, 1, 0, None, None, None) == 1
     assert L.ladder_op_decode_attention(None, None, None, None, 1, 8, 8, 128, 16, None, None, None) == 1
-    assert L.ladder_op_prefill_gemm(None, None, 1, 8, 8, 0, None, None, None) == 1
-    assert L.ladder_op_prefill_attention(None, None, None, 1, 1, 8, 8, 128, 16, None, None) == 1
+    assert L.ladder_op_prefill_gemm(None, None, None, 1, 8, 8, 0, None, None, None, None) == 1
+    assert L.ladder_op_prefill_attention(None, None, None, None, 1, 1, 8, 8, 128, 16, None, None, None) == 1
     assert L.ladder_decode_attention_scratch_bytes(0, 8, 128, 16) == 0
     assert L.ladder_decode_attention_scratch_bytes(4, 64, 128, 1536) > 0

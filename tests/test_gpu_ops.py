@@ -28,10 +28,11 @@ def _f64(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-# tolerance of a bf16-operand, fp32-accumulate dot product against float64 on the same operands:
-# the only error is the bf16 rounding of the normalised activation (2^-9 relative per element,
-# random sign) and fp32 summation, both far below 1e-2 of the row maximum.
-TOL_GEMM = 1e-2
+# Decode GEMMs feed the activation as a bf16 hi+lo pair (batch <= 16): what is left is fp32
+# accumulation error, ~1e-5 of the row maximum.  Above batch 16 the activation is a single
+# bf16 (2^-9 relative rounding per element, random sign), ~1e-3 of the row maximum.
+def tol_gemm(batch):
+    return 2e-4 if batch <= 16 else 1e-2
 
 
 @pytest.mark.parametrize("N,K,batch", [(256, 256, 1), (1376, 256, 4), (256, 688, 3), (1024, 2048, 8),
@@ -44,19 +45,19 @@ def test_smallm_gemm_norm_plain(B, N, K, batch):
     B.op_smallm_gemm(W, x, 1, 2, out, gain=g, eps=1e-5)
     torch.cuda.synchronize()
     ref = O.rmsnorm(_f64(x), _f64(g), 1e-5) @ _f64(W).T
-    assert rel_err(out.cpu().numpy(), ref) < TOL_GEMM
+    assert rel_err(out.cpu().numpy(), ref) < tol_gemm(batch)
 
 
 @pytest.mark.parametrize("N,K,batch", [(256, 688, 1), (8192, 8192, 4), (8192, 28672, 4), (512, 1032, 7), (776, 3584, 16)])
 def test_smallm_gemm_bf16_residual(B, N, K, batch):
     W = _bf16((N, K), 4, 0.02)
-    a = _bf16((batch, K), 5, 1.0)
+    a = torch.randn(batch, K, generator=torch.Generator().manual_seed(5)).cuda()
     addend = torch.randn(batch, N, generator=torch.Generator().manual_seed(6)).cuda()
     out = torch.empty_like(addend)
     B.op_smallm_gemm(W, a, 0, 0, out, addend=addend)
     torch.cuda.synchronize()
     ref = _f64(addend) + _f64(a) @ _f64(W).T
-    assert rel_err(out.cpu().numpy(), ref) < 1e-3
+    assert rel_err(out.cpu().numpy(), ref) < tol_gemm(batch)
     # in place (standard-residual layers): destination == addend
     inplace = addend.clone()
     B.op_smallm_gemm(W, a, 0, 0, inplace, addend=inplace)
@@ -69,13 +70,13 @@ def test_smallm_gemm_swiglu(B, F, K, batch):
     W = _bf16((2 * F, K), 7, 0.05)
     x = torch.randn(batch, K, generator=torch.Generator().manual_seed(8)).cuda()
     g = torch.ones(K, dtype=torch.bfloat16, device="cuda")
-    out = torch.empty(batch, F, dtype=torch.bfloat16, device="cuda")
+    out = torch.empty(batch, F, device="cuda")
     B.op_smallm_gemm(W, x, 1, 1, out, gain=g, eps=1e-5)
     torch.cuda.synchronize()
     n = O.rmsnorm(_f64(x), _f64(g), 1e-5)
     w = _f64(W)
     ref = O.silu(n @ w[0::2].T) * (n @ w[1::2].T)
-    assert rel_err(_f64(out), ref) < 2e-2
+    assert rel_err(_f64(out), ref) < 5e-4
 
 
 def test_smallm_gemm_is_deterministic_and_batch_invariant(B):
@@ -108,12 +109,12 @@ def test_decode_attention(B, batch, Hq, Hkv, Dh, max_seq, lens):
     v = _bf16((batch, Hkv, max_seq, Dh), 13, 1.0)
     kv_len = torch.tensor(lens, dtype=torch.int32, device="cuda")
     scratch = torch.empty(B.decode_attention_scratch_bytes(batch, Hq, Dh, max_seq) // 4, device="cuda")
-    o = torch.full((batch, Hq * Dh), float("nan"), dtype=torch.bfloat16, device="cuda")
+    o = torch.full((batch, Hq * Dh), float("nan"), device="cuda")
     for _ in range(2):                       # twice: the ticket counters must clean themselves up
         B.op_decode_attention(q, k, v, kv_len, Hq, Hkv, Dh, max_seq, scratch, o)
     torch.cuda.synchronize()
     got = _f64(o).reshape(batch, Hq, Dh)
-    qb = O.bf16_round(_f64(q)).reshape(batch, 1, Hq, Dh)          # the kernel feeds q to the MMA as bf16
+    qb = _f64(q).reshape(batch, 1, Hq, Dh)
     for b in range(batch):
         L = lens[b]
         if L == 0:
@@ -122,46 +123,66 @@ def test_decode_attention(B, batch, Hq, Hkv, Dh, max_seq, lens):
         kk = _f64(k[b, :, :L]).transpose(1, 0, 2)
         vv = _f64(v[b, :, :L]).transpose(1, 0, 2)
         ref = O.causal_attention(qb[b], kk, vv, L - 1)[0]
-        assert rel_err(got[b], ref) < 1e-2, b
+        assert rel_err(got[b], ref) < 1e-3, b
 
 
+def _split(shape, seed, std=1.0):
+    """fp32 values and their bf16 hi / lo parts (value ~ hi + lo)."""
+    f = torch.randn(shape, generator=torch.Generator().manual_seed(seed)) * std
+    hi = f.to(torch.bfloat16)
+    lo = (f - hi.float()).to(torch.bfloat16)
+    return f.cuda(), hi.cuda(), lo.cuda()
+
+
+@pytest.mark.parametrize("split", [False, True])
 @pytest.mark.parametrize("M,N,K,mode", [(16, 768, 256, 3), (300, 1376, 256, 1), (512, 256, 688, 0),
                                         (1000, 520, 264, 2), (4096, 1024, 1024, 0)])
-def test_prefill_gemm(B, M, N, K, mode):
-    A = _bf16((M, K), 14, 1.0)
+def test_prefill_gemm(B, M, N, K, mode, split):
+    Af, A, A_lo = _split((M, K), 14)
     W = _bf16((N, K), 15, 0.05)
-    acc = _f64(A) @ _f64(W).T
+    acc = (_f64(Af) if split else _f64(A)) @ _f64(W).T
+    lo_in = A_lo if split else None
+    out_lo = None
     if mode == 0:
         addend = torch.randn(M, N, generator=torch.Generator().manual_seed(16)).cuda()
         out = torch.empty_like(addend)
-        B.op_prefill_gemm(A, W, 0, out, addend=addend)
+        B.op_prefill_gemm(A, W, 0, out, addend=addend, A_lo=lo_in)
         ref = _f64(addend) + acc
     elif mode == 1:
         out = torch.empty(M, N // 2, dtype=torch.bfloat16, device="cuda")
-        B.op_prefill_gemm(A, W, 1, out)
+        out_lo = torch.empty_like(out) if split else None
+        B.op_prefill_gemm(A, W, 1, out, A_lo=lo_in, out_lo=out_lo)
         ref = O.silu(acc[:, 0::2]) * acc[:, 1::2]
     elif mode == 2:
         out = torch.empty(M, N, device="cuda")
-        B.op_prefill_gemm(A, W, 2, out)
+        B.op_prefill_gemm(A, W, 2, out, A_lo=lo_in)
         ref = acc
     else:
         out = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
-        B.op_prefill_gemm(A, W, 3, out)
+        out_lo = torch.empty_like(out) if split else None
+        B.op_prefill_gemm(A, W, 3, out, A_lo=lo_in, out_lo=out_lo)
         ref = acc
     torch.cuda.synchronize()
-    assert rel_err(_f64(out), ref) < (1e-3 if mode in (0, 2) else 1e-2)
+    got = _f64(out) + (_f64(out_lo) if out_lo is not None else 0.0)
+    # fp32 outputs / hi+lo outputs carry only accumulation error; a single bf16 output rounds at 2^-9
+    tol = 2e-4 if (mode in (0, 2) or out_lo is not None) else 1e-2
+    assert rel_err(got, ref) < tol
 
 
+@pytest.mark.parametrize("split", [False, True])
 @pytest.mark.parametrize("batch,S,Hq,Hkv,Dh,max_seq", [(1, 16, 4, 4, 64, 32), (2, 200, 8, 2, 128, 256),
                                                        (1, 1024, 8, 1, 128, 1536), (2, 65, 6, 3, 64, 70)])
-def test_prefill_attention(B, batch, S, Hq, Hkv, Dh, max_seq):
-    q = _bf16((batch, S, Hq * Dh), 17, 1.0)
+def test_prefill_attention(B, batch, S, Hq, Hkv, Dh, max_seq, split):
+    qf, q, q_lo = _split((batch, S, Hq * Dh), 17)
     k = _bf16((batch, Hkv, max_seq, Dh), 18, 1.0)
     v = _bf16((batch, Hkv, max_seq, Dh), 19, 1.0)
     o = torch.full((batch, S, Hq * Dh), float("nan"), dtype=torch.bfloat16, device="cuda")
-    B.op_prefill_attention(q, k, v, batch, S, Hq, Hkv, Dh, max_seq, o)
+    o_lo = torch.zeros_like(o) if split else None
+    B.op_prefill_attention(q, k, v, batch, S, Hq, Hkv, Dh, max_seq, o, q_lo=q_lo if split else None, o_lo=o_lo)
     torch.cuda.synchronize()
+    got = _f64(o) + (_f64(o_lo) if split else 0.0)
     for b in range(batch):
-        ref = O.causal_attention(_f64(q[b]).reshape(S, Hq, Dh), _f64(k[b, :, :S]).transpose(1, 0, 2),
-                                 _f64(v[b, :, :S]).transpose(1, 0, 2), 0)
-        assert rel_err(_f64(o[b]).reshape(S, Hq, Dh), ref) < 2e-2, b
+        ref = O.causal_attention(_f64(qf[b] if split else q[b]).reshape(S, Hq, Dh),
+                                 _f64(k[b, :, :S]).transpose(1, 0, 2), _f64(v[b, :, :S]).transpose(1, 0, 2), 0)
+        # the probabilities enter the P.V MMA as single bf16 values (2^-9 relative each, averaged over keys)
+        assert rel_err(got[b].reshape(S, Hq, Dh), ref) < (5e-3 if split else 2e-2), b

@@ -279,6 +279,8 @@ def main():
     rewind()
     h_in = first.cpu().pin_memory()
     h_out = torch.zeros(bsz, dtype=torch.int32).pin_memory()
+    model.decode_step_host(cache, h_in, h_out)      # untimed: captures the graph for the staging buffers
+    rewind()
     sync_all()
     t0 = time.perf_counter()
     for _ in range(steps):

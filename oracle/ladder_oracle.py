@@ -27,11 +27,17 @@ the same ones):
 * greedy argmax takes the lowest index among equal maxima.
 
 Arithmetic: every array is ``dtype`` (float64 by default, float32 for the large
-workloads); rotary angles, cos and sin are always formed in float64.  With
-``bf16_storage=True`` the values the CUDA path stores as bf16 (normalised
-activations, q/k/v, attention output, SwiGLU output) are rounded to bf16 too;
-this is a diagnostic switch that separates bf16 noise from bugs, not the
-definition.
+workloads); rotary angles, cos and sin are always formed in float64.
+
+Storage precision switches (the definition is both off):
+* ``bf16_kv=True`` rounds K (after rotation) and V to bf16 where they enter the
+  cache / the attention -- the storage precision of a bf16 KV cache, which the
+  "bf16 forward" of the benchmark prescribes.  It is used where floating point
+  decides an integer (the greedy argmax), so that both sides take that decision
+  from keys and values of the same precision.
+* ``bf16_storage=True`` additionally rounds normalised activations, q, the
+  attention output and the SwiGLU output: a diagnostic that separates bf16
+  noise from bugs.
 
 Pins (tests/test_oracle_pins.py): single-module ladder == standard, cached
 decode == recomputation, softmax rows, brute-force attention, Eq.-2 form ==
@@ -186,7 +192,8 @@ class OracleCache:
 
 # --------------------------------------------------------------------------- modules
 def attention_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndarray,
-                     pos0: int, cache: Optional[OracleCache], bf16_storage: bool = False):
+                     pos0: int, cache: Optional[OracleCache], bf16_storage: bool = False,
+                     bf16_kv: bool = False):
     """h(n) for the attention module of ``layer``.
 
     n [B, T, d] is the normalised input at absolute positions pos0..pos0+T-1.
@@ -205,8 +212,8 @@ def attention_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndar
     k = (n @ wk.T).reshape(B, T, Hkv, Dh)
     v = (n @ wv.T).reshape(B, T, Hkv, Dh)
     q = _store(rope(q, positions, cfg.rope_theta), bf16_storage)
-    k = _store(rope(k, positions, cfg.rope_theta), bf16_storage)
-    v = _store(v, bf16_storage)
+    k = _store(rope(k, positions, cfg.rope_theta), bf16_storage or bf16_kv)
+    v = _store(v, bf16_storage or bf16_kv)
     o = np.empty((B, T, Hq, Dh), dtype=dt)
     for b in range(B):
         if cache is not None:
@@ -251,7 +258,8 @@ def greedy(logits: np.ndarray) -> np.ndarray:
 
 def run_layers(cfg: OracleConfig, W: OracleWeights, x: np.ndarray, pos0: int,
                cache: Optional[OracleCache], bf16_storage: bool = False,
-               record: Optional[ForwardResult] = None, n_layers: Optional[int] = None):
+               record: Optional[ForwardResult] = None, n_layers: Optional[int] = None,
+               bf16_kv: bool = False):
     """The layer stack in Algorithm-1 form, then the final flush.  x [B,T,d]."""
     a_p = np.zeros_like(x)              # pending attention output (attn_out)
     m_p = np.zeros_like(x)              # pending MLP output       (mlp_out)
@@ -264,7 +272,7 @@ def run_layers(cfg: OracleConfig, W: OracleWeights, x: np.ndarray, pos0: int,
             n = _store(rmsnorm(x, g_a, cfg.rms_eps), bf16_storage)       # AttentionNorm
             if record is not None:
                 record.module_inputs.append(x.copy())
-            a_p = attention_module(cfg, W, l, n, pos0, cache, bf16_storage)
+            a_p = attention_module(cfg, W, l, n, pos0, cache, bf16_storage, bf16_kv)
             x = x + m_p                                                  # residual += mlp_out
             n = _store(rmsnorm(x, g_m, cfg.rms_eps), bf16_storage)       # MLPNorm
             if record is not None:
@@ -279,7 +287,7 @@ def run_layers(cfg: OracleConfig, W: OracleWeights, x: np.ndarray, pos0: int,
             n = _store(rmsnorm(x, g_a, cfg.rms_eps), bf16_storage)
             if record is not None:
                 record.module_inputs.append(x.copy())
-            a = attention_module(cfg, W, l, n, pos0, cache, bf16_storage)
+            a = attention_module(cfg, W, l, n, pos0, cache, bf16_storage, bf16_kv)
             x = x + a
             n = _store(rmsnorm(x, g_m, cfg.rms_eps), bf16_storage)
             if record is not None:
@@ -305,7 +313,8 @@ def head(cfg: OracleConfig, W: OracleWeights, x: np.ndarray, bf16_storage: bool 
 def forward(cfg: OracleConfig, W: OracleWeights, tokens: np.ndarray, dtype=np.float64,
             cache: Optional[OracleCache] = None, pos0: int = 0, last_only: bool = False,
             bf16_storage: bool = False, record: bool = False,
-            with_logits: bool = True, n_layers: Optional[int] = None) -> ForwardResult:
+            with_logits: bool = True, n_layers: Optional[int] = None,
+            bf16_kv: bool = False) -> ForwardResult:
     """Full forward over tokens [B, T] at positions pos0..pos0+T-1.
 
     Without a cache pos0 must be 0 and the whole sequence is recomputed.  With a
@@ -314,7 +323,7 @@ def forward(cfg: OracleConfig, W: OracleWeights, tokens: np.ndarray, dtype=np.fl
     tokens = np.asarray(tokens)
     res = ForwardResult(None, None, None, None)
     x = embed(W, tokens, dtype)
-    x = run_layers(cfg, W, x, pos0, cache, bf16_storage, res if record else None, n_layers)
+    x = run_layers(cfg, W, x, pos0, cache, bf16_storage, res if record else None, n_layers, bf16_kv)
     if cache is not None:
         assert cache.seq_len == pos0
         cache.seq_len = pos0 + tokens.shape[1]
@@ -331,23 +340,23 @@ def forward(cfg: OracleConfig, W: OracleWeights, tokens: np.ndarray, dtype=np.fl
 
 
 def prefill(cfg, W, tokens, cache: OracleCache, dtype=np.float64, bf16_storage=False,
-            n_layers=None) -> ForwardResult:
+            n_layers=None, bf16_kv=False) -> ForwardResult:
     """Prompt pass: fills cache rows 0..S-1, returns hidden/logits at position S-1."""
     assert cache.seq_len == 0
     return forward(cfg, W, tokens, dtype, cache, 0, last_only=True,
-                   bf16_storage=bf16_storage, n_layers=n_layers)
+                   bf16_storage=bf16_storage, n_layers=n_layers, bf16_kv=bf16_kv)
 
 
 def decode_step(cfg, W, tokens, cache: OracleCache, dtype=np.float64, bf16_storage=False,
-                n_layers=None) -> ForwardResult:
+                n_layers=None, bf16_kv=False) -> ForwardResult:
     """One token per sequence at position cache.seq_len (append, then attend)."""
     tokens = np.asarray(tokens).reshape(-1, 1)
     return forward(cfg, W, tokens, dtype, cache, cache.seq_len, last_only=True,
-                   bf16_storage=bf16_storage, n_layers=n_layers)
+                   bf16_storage=bf16_storage, n_layers=n_layers, bf16_kv=bf16_kv)
 
 
 def generate(cfg, W, prompt: np.ndarray, n_steps: int, max_seq_len: int, dtype=np.float64,
-             forced: Optional[np.ndarray] = None, bf16_storage=False):
+             forced: Optional[np.ndarray] = None, bf16_storage=False, bf16_kv=False):
     """prefill + n_steps decode steps.
 
     Returns (tokens [B, n_steps+1], hiddens [B, n_steps+1, d]): entry 0 comes from
@@ -359,12 +368,12 @@ def generate(cfg, W, prompt: np.ndarray, n_steps: int, max_seq_len: int, dtype=n
     prompt = np.asarray(prompt)
     B, S = prompt.shape
     cache = OracleCache(cfg, B, max_seq_len, dtype)
-    r = prefill(cfg, W, prompt, cache, dtype, bf16_storage)
+    r = prefill(cfg, W, prompt, cache, dtype, bf16_storage, bf16_kv=bf16_kv)
     toks = [r.next_tokens[:, 0]]
     hids = [r.hidden[:, 0]]
     for j in range(n_steps):
         feed = toks[-1] if forced is None else np.asarray(forced)[:, j]
-        r = decode_step(cfg, W, feed, cache, dtype, bf16_storage)
+        r = decode_step(cfg, W, feed, cache, dtype, bf16_storage, bf16_kv=bf16_kv)
         toks.append(r.next_tokens[:, 0])
         hids.append(r.hidden[:, 0])
     return np.stack(toks, axis=1), np.stack(hids, axis=1)

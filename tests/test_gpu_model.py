@@ -10,7 +10,10 @@ from tests.helpers import rel_err
 
 pytestmark = pytest.mark.gpu
 
-HIDDEN_TOL = 2e-2          # max_i |g_i - o_i| / max_i |o_i| per (sequence, position), bf16 path vs oracle
+# Final hidden state: max_i |g_i - o_i| / max_i |o_i| per (sequence, position), bf16 path vs the exact
+# oracle.  Greedy tokens: teacher-forced (the oracle is fed the GPU's history) and, because floating
+# point decides an integer there, taken with both sides at the KV cache's bf16 storage precision.
+HIDDEN_TOL = 2e-2
 CANARY = 0x7F7F            # bf16 bit pattern pre-filled into the cache (a huge finite value)
 
 
@@ -67,7 +70,11 @@ def check_generation(B, shape, steps, dtype, gains="ones", schedule=None, min_ag
     OW = O.OracleWeights(provider=synth.logical_provider(w, dtype))
     o_toks, o_hids = O.generate(cfg, OW, prompt, steps, max_seq, dtype=dtype, forced=toks)
     err = rel_err(hids, o_hids)
-    agree = float(np.mean(toks == o_toks))
+    # the argmax decision is compared with both sides holding K/V at the cache's bf16 precision
+    k_toks, _ = O.generate(cfg, OW, prompt, steps, max_seq, dtype=dtype, forced=toks, bf16_kv=True)
+    agree = float(np.mean(toks == k_toks))
+    print(f"[{shape.name} L{shape.n_layers}] hidden max-rel-err {err:.3e}; greedy agreement {agree:.4f} "
+          f"(oracle with bf16 KV), {float(np.mean(toks == o_toks)):.4f} (exact oracle), {toks.size} comparisons")
     # --- KV cache indexing
     used = S + steps
     assert cache.seq_lens.cpu().tolist() == [used] * bsz
@@ -85,7 +92,7 @@ def test_tiny_config_full(B, variant):
         s = s.as_standard()
     elif variant == "hybrid":
         s = synth.replace(s, layer_is_ladder=(0, 1, 1, 0))
-    err, agree, *_ = check_generation(B, s, 16, np.float64, gains="uniform", batch=4)
+    err, agree, *_ = check_generation(B, s, 64, np.float64, gains="uniform", batch=4)     # 4 x 65 comparisons
     assert err < HIDDEN_TOL, err
     assert agree >= 0.99, agree
 
@@ -200,13 +207,13 @@ def test_70b_shape_shallow_full_context(B):
     s = synth.SHAPES["70b"].with_layers(2)
     err, agree, *_ = check_generation(B, s, 8, np.float32)
     assert err < HIDDEN_TOL, err
-    assert agree >= 0.97, agree          # 36 comparisons: allow one near-tie flip
+    assert agree >= 0.97, agree          # 36 comparisons: at most one flip
 
 
 def test_8b_hybrid_shape_short_context(B):
     """The 8B hybrid shape (GQA 32/8, theta 500000) cut to 4 standard + 4 ladder layers so the
-    float32 oracle copy fits any host; 16-token prompts, 8 steps."""
+    float32 oracle copy fits any host; 64-token prompts, 64 greedy steps."""
     s = synth.replace(synth.SHAPES["8b_hybrid"].with_layers(8), layer_is_ladder=(0, 0, 0, 0, 1, 1, 1, 1))
-    err, agree, *_ = check_generation(B, s, 8, np.float32, batch=2, prompt_len=16)
+    err, agree, *_ = check_generation(B, s, 64, np.float32, batch=4, prompt_len=64)       # 260 comparisons
     assert err < HIDDEN_TOL, err
-    assert agree >= 0.94, agree          # 18 comparisons
+    assert agree >= 0.99, agree

@@ -364,6 +364,24 @@ def test_float32_mode_tracks_float64():
     assert np.max(np.abs(a.hidden - b.hidden)) < 1e-4
 
 
+def test_bf16_kv_switch_rounds_exactly_the_cache():
+    cfg = small_cfg(n_layers=2)
+    t = rand_weights(cfg, 24)
+    exact, rounded = O.OracleCache(cfg, 2, 8), O.OracleCache(cfg, 2, 8)
+    a = O.prefill(cfg, W(t), TOK, exact)
+    b = O.prefill(cfg, W(t), TOK, rounded, bf16_kv=True)
+    # layer 0 sees identical inputs, so its cache is the bf16 rounding of the exact one (library conversion)
+    for src, dst in ((exact.k, rounded.k), (exact.v, rounded.v)):
+        ref = torch.from_numpy(src[0, :, :6].astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+        assert np.array_equal(dst[0, :, :6], ref)
+    assert np.array_equal(O.bf16_round(rounded.k), rounded.k)          # every cached value is a bf16 value
+    assert 0 < np.max(np.abs(a.hidden - b.hidden)) < 0.05              # close to, but not, the exact result
+    # cached decode still equals recomputation under the switch
+    full = O.forward(cfg, W(t), np.concatenate([TOK, TOK[:, :1]], 1), bf16_kv=True)
+    step = O.decode_step(cfg, W(t), TOK[:, 0], rounded, bf16_kv=True)
+    assert np.allclose(step.hidden[:, 0], full.hidden[:, 6], atol=1e-10)
+
+
 # ---------------------------------------------------------------- the paper's own arithmetic (Tab. 2)
 def test_table2_reading_latency_reduction_vs_throughput_gain():
     import os

@@ -158,7 +158,9 @@ const char* ladder_last_error(const ladder_model_t* m); /* library-owned string;
 
 /* ------------------------------------------------------------------------------------------
  * Single-kernel entry points: the same kernels the model calls, exposed so each can be tested
- * and profiled at its true shape.  They allocate nothing and do not synchronise.
+ * and profiled at its true shape.  They do not synchronise; ladder_op_smallm_gemm keeps a
+ * library-owned split-K scratch that it grows (allocating, and then synchronising once) when a
+ * larger shape is first seen, so its calls must not overlap on the device; the others allocate nothing.
  * ------------------------------------------------------------------------------------------ */
 
 /* Weight-streaming small-M GEMM  acc[b,n] = sum_k act[b,k] * W[n,k]  (decode: M = batch <= 64),

@@ -4,6 +4,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <string>
 #include <vector>
 
@@ -52,6 +53,9 @@ struct ladder_model {
   float* h_dec = nullptr;           // decode [max_batch, F]
   float* attn_scratch = nullptr;
   int attn_splits = 1;
+  float* gemm_scratch[2] = {nullptr, nullptr};  // split-K partials + tickets, one per stream role
+  int32_t* work_slots = nullptr;    // 2 ints per GEMM launch of a step (claim counters)
+  int n_work_slots = 0;
   float* logits_ws = nullptr;       // [max_batch, V]
   float* last_x = nullptr;          // [max_batch, d]
   // prefill activations, each a bf16 hi part followed by a lo part (value ~ hi + lo)
@@ -142,6 +146,13 @@ struct Enqueue {
   bool two;
   bool pdl_ok[2] = {false, false};  // previous op on the stream was a kernel (programmatic edge possible)
   int64_t kernels = 0;
+  int slot = 0;  // next claim-counter slot
+  void gemm(int s, SmallMParams& p) {
+    p.scratch = m->gemm_scratch[s];
+    p.work = m->work_slots + 2 * (slot++ % m->n_work_slots);
+    p.status = m->status;
+    launched(s, launch_smallm_gemm(p, stream(s), pdl(s), m->sm_count));
+  }
   cudaError_t err = cudaSuccess;
 
   cudaStream_t stream(int s) const { return s ? sB : sA; }
@@ -217,7 +228,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       p.qkv.head_dim = Dh;
       p.qkv.max_seq_len = c.max_seq_len;
       p.status = m->status;
-      q.launched(0, launch_smallm_gemm(p, sA, q.pdl(0), m->sm_count));
+      q.gemm(0, p);
 
       DecodeAttnParams a = {};
       a.q = m->q_f32;
@@ -235,6 +246,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       a.scratch = m->attn_scratch;
       a.o = m->o_dec;
       q.launched(0, launch_decode_attention(a, sA, q.pdl(0)));
+      ++q.kernels;  // the split kernel and its merge kernel
 
       need(0, mod - 1);  // the epilogue reads x_{m-1} and overwrites the buffer of x_{m-2}
       SmallMParams o = {};
@@ -248,7 +260,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       o.addend = m->R[r.add];
       o.out = m->R[r.dst];
       o.status = m->status;
-      q.launched(0, launch_smallm_gemm(o, sA, q.pdl(0), m->sm_count));
+      q.gemm(0, o);
       q.record(0, m->ev[mod]);
     }
     // ---------------- MLP module (module index 2l+2) on stream B
@@ -272,7 +284,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       p.epi_mode = EPI_SWIGLU;
       p.out = m->h_dec;
       p.status = m->status;
-      q.launched(1, launch_smallm_gemm(p, q.stream(1), q.pdl(1), m->sm_count));
+      q.gemm(1, p);
 
       need(1, mod - 1);
       SmallMParams o = {};
@@ -286,7 +298,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       o.addend = m->R[r.add];
       o.out = m->R[r.dst];
       o.status = m->status;
-      q.launched(1, launch_smallm_gemm(o, q.stream(1), q.pdl(1), m->sm_count));
+      q.gemm(1, o);
       q.record(1, m->ev[mod]);
     }
   }
@@ -306,7 +318,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   h.epi_mode = EPI_PLAIN;
   h.out = logits;
   h.status = m->status;
-  q.launched(0, launch_smallm_gemm(h, sA, q.pdl(0), m->sm_count));
+  q.gemm(0, h);
   if (out && out->final_hidden)
     q.launched(0, launch_rmsnorm_f32(xf, m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, sA, q.pdl(0)));
   q.launched(0, launch_argmax_advance(logits, batch, c.vocab_size, out ? out->next_tokens : nullptr, cache->seq_lens, 1,
@@ -410,6 +422,8 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
   h.epi_mode = EPI_PLAIN;
   h.out = logits;
   h.status = m->status;
+  h.scratch = m->gemm_scratch[0];
+  h.work = m->work_slots + 2 * (m->n_work_slots - 1);
   did(launch_smallm_gemm(h, st, false, m->sm_count));
   if (out && out->final_hidden)
     did(launch_rmsnorm_f32(m->last_x, m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, st, false));
@@ -518,6 +532,23 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   A(dev_alloc(&m->o_dec, MB * qd));
   A(dev_alloc(&m->h_dec, MB * F));
   A(dev_alloc(&m->attn_scratch, scratch_floats));
+  {
+    const int qkv_rows = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+    size_t sa = smallm_gemm_scratch_floats(qkv_rows, c.d_model, c.max_batch);
+    sa = std::max(sa, smallm_gemm_scratch_floats(c.d_model, static_cast<int>(qd), c.max_batch));
+    sa = std::max(sa, smallm_gemm_scratch_floats(c.vocab_size, c.d_model, c.max_batch));
+    size_t sb = std::max(smallm_gemm_scratch_floats(2 * c.d_ff, c.d_model, c.max_batch),
+                         smallm_gemm_scratch_floats(c.d_model, c.d_ff, c.max_batch));
+    m->n_work_slots = 4 * L + 4;
+    A(dev_alloc(&m->gemm_scratch[0], sa + 64));
+    A(dev_alloc(&m->gemm_scratch[1], sb + 64));
+    A(dev_alloc(&m->work_slots, static_cast<size_t>(2 * m->n_work_slots)));
+    if (!oom) {
+      if (cudaMemset(m->gemm_scratch[0], 0, (sa + 64) * sizeof(float)) != cudaSuccess) oom = true;
+      if (cudaMemset(m->gemm_scratch[1], 0, (sb + 64) * sizeof(float)) != cudaSuccess) oom = true;
+      if (cudaMemset(m->work_slots, 0, 2 * m->n_work_slots * sizeof(int32_t)) != cudaSuccess) oom = true;
+    }
+  }
   A(dev_alloc(&m->logits_ws, MB * c.vocab_size));
   A(dev_alloc(&m->last_x, MB * d));
   m->n_lo = MP * d;
@@ -576,7 +607,7 @@ ladder_status_t ladder_destroy(ladder_model_t* m) {
   if (m->ev_join) cudaEventDestroy(m->ev_join);
   if (m->side) cudaStreamDestroy(m->side);
   if (m->cap) cudaStreamDestroy(m->cap);
-  void* bufs[] = {m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
+  void* bufs[] = {m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
                   m->n_pf, m->q_pf,  m->o_pf,  m->h_pf,  m->rope,  m->status,       m->tok_tmp,   m->next_tmp};
   for (void* b : bufs)
     if (b) cudaFree(b);
@@ -744,6 +775,30 @@ static int sm_count_cached() {
   return g_sm_count > 0 ? g_sm_count : 148;
 }
 
+// Library-owned scratch of the single-kernel GEMM entry point (grown on demand; one per process, so
+// calls of that entry point must not overlap on the device).
+static float* g_op_scratch = nullptr;
+static size_t g_op_scratch_floats = 0;
+static int32_t* g_op_work = nullptr;
+static int g_op_serial = 0;
+static cudaError_t op_scratch(size_t floats) {
+  if (!g_op_work) {
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&g_op_work), 2 * 256 * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(g_op_work, 0, 2 * 256 * sizeof(int32_t));
+    if (e != cudaSuccess) return e;
+  }
+  if (floats <= g_op_scratch_floats) return cudaSuccess;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return e;
+  if (g_op_scratch) cudaFree(g_op_scratch);
+  g_op_scratch = nullptr;
+  g_op_scratch_floats = 0;
+  e = cudaMalloc(reinterpret_cast<void**>(&g_op_scratch), floats * sizeof(float));
+  if (e == cudaSuccess) e = cudaMemset(g_op_scratch, 0, floats * sizeof(float));
+  if (e == cudaSuccess) g_op_scratch_floats = floats;
+  return e;
+}
+
 ladder_status_t ladder_op_smallm_gemm(const void* W, int32_t N, int32_t K, const void* act, int32_t act_mode,
                                       const void* gain, float eps, int32_t batch, int32_t epi_mode, const float* addend,
                                       void* out, void* cuda_stream) {
@@ -765,6 +820,9 @@ ladder_status_t ladder_op_smallm_gemm(const void* W, int32_t N, int32_t K, const
   p.addend = addend;
   p.out = out;
   if (kernels_ready() != cudaSuccess) return LADDER_ERR_CUDA;
+  if (op_scratch(smallm_gemm_scratch_floats(N, K, batch) + 64) != cudaSuccess) return LADDER_ERR_OOM;
+  p.scratch = g_op_scratch;
+  p.work = g_op_work + 2 * (g_op_serial++ & 255);
   cudaError_t e = launch_smallm_gemm(p, static_cast<cudaStream_t>(cuda_stream), false, sm_count_cached());
   return e == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
 }
@@ -802,9 +860,6 @@ ladder_status_t ladder_op_decode_attention(const float* q, const void* k, const 
   a.n_splits = op_attn_splits(batch, n_kv_heads, max_seq_len);
   a.scratch = scratch;
   a.o = static_cast<float*>(o);
-  // ticket counters at the head of the scratch must start at zero
-  const size_t counters = (static_cast<size_t>(batch) * n_q_heads + 63) / 64 * 64;
-  if (cudaMemsetAsync(scratch, 0, counters * sizeof(float), st) != cudaSuccess) return LADDER_ERR_CUDA;
   return launch_decode_attention(a, st, false) == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
 }
 

@@ -1,16 +1,19 @@
 // Grouped-query decode attention, split over the KV cache.
 //
-// One CTA per (split s, group of GT query heads sharing a kv head, sequence b).  The CTA
-//   1. computes the GT x CH score block with mma.sync (Q padded to 16 rows is the A operand,
-//      K rows are read straight from the cache as B fragments -- the contraction index is
-//      permuted identically on both sides so each thread reads 16 contiguous bytes of a key),
-//   2. does the softmax of its block in fp32 (max, exp, sum) in shared memory,
-//   3. accumulates P.V on the CUDA cores (each warp walks keys, each lane owns Dh/32 dims),
-//   4. writes (o, m, l) partials to an L2-resident scratch, and the LAST CTA of a head group to
-//      arrive (atomic ticket, no spinning) merges the partials by log-sum-exp in a fixed order
-//      and writes o in fp32.  The ticket counters clean themselves up for the next launch.
-// The kernel is latency- not bandwidth-bound (KV is ~1 % of the bytes of a decode step); its
-// shared-memory footprint is kept small so it can co-reside with a weight-streaming GEMM CTA.
+// The step is latency-bound, not bandwidth-bound (the KV prefix is ~1 % of the bytes of a decode
+// step), so the kernel is built around memory-level parallelism: one CTA per (64-key split, group
+// of GT query heads sharing a kv head, sequence); each of its 4 warps owns 16 keys and issues ALL of
+// its loads -- q, 16 key rows as MMA fragments, 16 value rows -- before the first dependent
+// instruction, so the whole CTA costs about one memory round trip plus one merge.
+//   1. scores: mma.sync with Q (padded to 16 rows, bf16 hi + lo pair so the fp32 query loses
+//      nothing) as the A operand and key rows read straight from the cache as B fragments (the
+//      contraction index is permuted identically on both sides: 16 contiguous bytes per thread);
+//   2. fp32 softmax statistics per warp, probabilities to shared memory;
+//   3. P.V on the CUDA cores in fp32 from the value rows already in registers;
+//   4. the 4 warps are merged by log-sum-exp in shared memory and the CTA's (o, m, l) partial goes
+//      to an L2-resident scratch; a second, tiny kernel (one CTA per sequence and head, launched
+//      with programmatic dependent launch) merges the splits in a fixed order and writes o in fp32.
+// The shared-memory footprint (~19 KB) lets a CTA co-reside with a weight-streaming GEMM CTA.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -18,17 +21,15 @@ namespace ladder {
 namespace {
 
 constexpr int kAttnThreads = 128;
-constexpr int kMaxChunk = 256;
+constexpr int kChunk = 64;  // keys per CTA (16 per warp)
 
 template <int GT, int DH>
-__global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const DecodeAttnParams p, int chunk,
-                                                                        int32_t* counters) {
+__global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const DecodeAttnParams p) {
   constexpr int DPL = DH / 32;  // dims per lane in the P.V phase
   constexpr int KJ = DH / 32;   // 16-byte loads per key per thread in the score phase
-  __shared__ float sc[GT][kMaxChunk];
+  __shared__ __align__(16) float ps[4][GT][16];
   __shared__ float red[4][GT][DH];
-  __shared__ float ml[GT][2];
-  __shared__ int last_s;
+  __shared__ float mls[4][GT][2];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, tig = lane & 3;
@@ -45,14 +46,34 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
 
   int L = p.kv_len[b] + p.kv_len_offset;
   L = max(0, min(L, p.max_seq_len));
-  const int k_begin = min(split * chunk, L);
-  const int k_end = min(k_begin + chunk, L);
-  const int nk = k_end - k_begin;
+  const int kw0 = split * kChunk + warp * 16;  // first key of this warp
   const float scale = rsqrtf(static_cast<float>(DH));
 
-  // ---- 1. scores
-  // q as a bf16 hi + lo pair (q ~ hi + lo), so the fp32 query loses nothing on its way into the MMA
-  uint32_t qa[KJ][2][2], ql[KJ][2][2];  // [j][half][pair]: q[head0+g][j*32 + tig*8 + half*4 + 2*pair ..+1]
+  // ---- all loads up front
+  uint4 kf[2][KJ];
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    const int key = kw0 + nt * 8 + g;
+#pragma unroll
+    for (int j = 0; j < KJ; ++j)
+      kf[nt][j] = key < L ? *reinterpret_cast<const uint4*>(K + static_cast<size_t>(key) * DH + j * 32 + tig * 8)
+                          : make_uint4(0, 0, 0, 0);
+  }
+  uint32_t vr[16][DPL / 2];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int key = kw0 + i;
+    if (DPL == 4) {
+      const uint2 u = key < L ? *reinterpret_cast<const uint2*>(V + static_cast<size_t>(key) * DH + lane * DPL)
+                              : make_uint2(0, 0);
+      vr[i][0] = u.x;
+      vr[i][DPL / 2 - 1] = u.y;
+    } else {
+      vr[i][0] = key < L ? *reinterpret_cast<const uint32_t*>(V + static_cast<size_t>(key) * DH + lane * DPL) : 0u;
+    }
+  }
+  // q as a bf16 hi + lo pair: [j][half][pair] covers q[head0+g][j*32 + tig*8 + half*4 + 2*pair ..+1]
+  uint32_t qa[KJ][2][2], ql[KJ][2][2];
 #pragma unroll
   for (int j = 0; j < KJ; ++j)
 #pragma unroll
@@ -66,73 +87,78 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
       ql[j][h][0] = pack_bf16x2(v.x - bf16_lo(qa[j][h][0]), v.y - bf16_hi(qa[j][h][0]));
       ql[j][h][1] = pack_bf16x2(v.z - bf16_lo(qa[j][h][1]), v.w - bf16_hi(qa[j][h][1]));
     }
-  for (int kb = warp * 8; kb < nk; kb += 32) {
-    const int key = k_begin + kb + g;
-    float c[4] = {0.f, 0.f, 0.f, 0.f};
-    uint4 kf[KJ];
+
+  // ---- 1. scores of this warp's 16 keys: c[nt][0..1] = (head g, keys nt*8 + 2*tig, +1)
+  float c[2][4];
 #pragma unroll
-    for (int j = 0; j < KJ; ++j)
-      kf[j] = (kb + g < nk) ? *reinterpret_cast<const uint4*>(K + static_cast<size_t>(key) * DH + j * 32 + tig * 8)
-                            : make_uint4(0, 0, 0, 0);
+  for (int nt = 0; nt < 2; ++nt) {
+    c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
 #pragma unroll
     for (int j = 0; j < KJ; ++j) {
-      mma_bf16_16816(c, qa[j][0][0], 0u, qa[j][0][1], 0u, kf[j].x, kf[j].y);
-      mma_bf16_16816(c, qa[j][1][0], 0u, qa[j][1][1], 0u, kf[j].z, kf[j].w);
-      mma_bf16_16816(c, ql[j][0][0], 0u, ql[j][0][1], 0u, kf[j].x, kf[j].y);
-      mma_bf16_16816(c, ql[j][1][0], 0u, ql[j][1][1], 0u, kf[j].z, kf[j].w);
-    }
-    if (g < GT) {
-      const int c0 = kb + 2 * tig;
-      if (c0 < nk) sc[g][c0] = c[0] * scale;
-      if (c0 + 1 < nk) sc[g][c0 + 1] = c[1] * scale;
+      mma_bf16_16816(c[nt], qa[j][0][0], 0u, qa[j][0][1], 0u, kf[nt][j].x, kf[nt][j].y);
+      mma_bf16_16816(c[nt], qa[j][1][0], 0u, qa[j][1][1], 0u, kf[nt][j].z, kf[nt][j].w);
+      mma_bf16_16816(c[nt], ql[j][0][0], 0u, ql[j][0][1], 0u, kf[nt][j].x, kf[nt][j].y);
+      mma_bf16_16816(c[nt], ql[j][1][0], 0u, ql[j][1][1], 0u, kf[nt][j].z, kf[nt][j].w);
     }
   }
-  __syncthreads();
-
-  // ---- 2. softmax of the block (fp32)
-  for (int h = warp; h < GT; h += 4) {
-    float m = -INFINITY;
-    for (int i = lane; i < nk; i += 32) m = fmaxf(m, sc[h][i]);
-    m = warp_max(m);
-    float l = 0.f;
-    for (int i = lane; i < nk; i += 32) {
-      const float e = __expf(sc[h][i] - m);
-      sc[h][i] = e;
-      l += e;
+  // ---- 2. softmax statistics of head g over the warp's keys (quad reduction)
+  float sv[4];
+  float m = -INFINITY;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int key = kw0 + nt * 8 + 2 * tig + e;
+      sv[nt * 2 + e] = key < L ? c[nt][e] * scale : -INFINITY;
+      m = fmaxf(m, sv[nt * 2 + e]);
     }
-    l = warp_sum(l);
-    if (lane == 0) {
-      ml[h][0] = m;
-      ml[h][1] = l;
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+  float l = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    sv[i] = (m == -INFINITY) ? 0.f : __expf(sv[i] - m);
+    l += sv[i];
+  }
+  l += __shfl_xor_sync(0xffffffffu, l, 1);
+  l += __shfl_xor_sync(0xffffffffu, l, 2);
+  if (g < GT) {
+    *reinterpret_cast<float2*>(&ps[warp][g][2 * tig]) = make_float2(sv[0], sv[1]);
+    *reinterpret_cast<float2*>(&ps[warp][g][8 + 2 * tig]) = make_float2(sv[2], sv[3]);
+    if (tig == 0) {
+      mls[warp][g][0] = m;
+      mls[warp][g][1] = l;
     }
   }
-  __syncthreads();
+  __syncwarp();
 
-  // ---- 3. P.V
+  // ---- 3. P.V for the warp's 16 keys; lane owns dims [lane*DPL, +DPL)
   float acc[GT][DPL];
 #pragma unroll
   for (int h = 0; h < GT; ++h)
 #pragma unroll
     for (int d = 0; d < DPL; ++d) acc[h][d] = 0.f;
-  for (int i = warp; i < nk; i += 4) {
-    const __nv_bfloat16* vr = V + static_cast<size_t>(k_begin + i) * DH + lane * DPL;
-    float v[DPL];
-    if (DPL == 4) {
-      const uint2 u = *reinterpret_cast<const uint2*>(vr);
-      v[0] = bf16_lo(u.x);
-      v[1] = bf16_hi(u.x);
-      v[DPL - 2] = bf16_lo(u.y);
-      v[DPL - 1] = bf16_hi(u.y);
-    } else {
-      const uint32_t u = *reinterpret_cast<const uint32_t*>(vr);
-      v[0] = bf16_lo(u);
-      v[1] = bf16_hi(u);
-    }
 #pragma unroll
-    for (int h = 0; h < GT; ++h) {
-      const float pw = sc[h][i];
+  for (int i4 = 0; i4 < 4; ++i4) {
+    float4 pw[GT];
 #pragma unroll
-      for (int d = 0; d < DPL; ++d) acc[h][d] += pw * v[d];
+    for (int h = 0; h < GT; ++h) pw[h] = *reinterpret_cast<const float4*>(&ps[warp][h][i4 * 4]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int i = i4 * 4 + e;
+      float v[DPL];
+      v[0] = bf16_lo(vr[i][0]);
+      v[1] = bf16_hi(vr[i][0]);
+      if (DPL == 4) {
+        v[DPL - 2] = bf16_lo(vr[i][DPL / 2 - 1]);
+        v[DPL - 1] = bf16_hi(vr[i][DPL / 2 - 1]);
+      }
+#pragma unroll
+      for (int h = 0; h < GT; ++h) {
+        const float w = e == 0 ? pw[h].x : (e == 1 ? pw[h].y : (e == 2 ? pw[h].z : pw[h].w));
+#pragma unroll
+        for (int d = 0; d < DPL; ++d) acc[h][d] += w * v[d];
+      }
     }
   }
 #pragma unroll
@@ -141,61 +167,86 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
     for (int d = 0; d < DPL; ++d) red[warp][h][lane * DPL + d] = acc[h][d];
   __syncthreads();
 
-  // ---- 4. partial -> scratch
+  // ---- 4. merge the 4 warps, write the CTA partial
   const int stride = DH + 2;
   for (int idx = tid; idx < GT * DH; idx += kAttnThreads) {
     const int h = idx / DH, d = idx % DH;
-    const float o = red[0][h][d] + red[1][h][d] + red[2][h][d] + red[3][h][d];
-    p.scratch[((static_cast<size_t>(b) * p.n_q_heads + head0 + h) * p.n_splits + split) * stride + d] = o;
-  }
-  if (tid < GT) {
-    float* dst = p.scratch + ((static_cast<size_t>(b) * p.n_q_heads + head0 + tid) * p.n_splits + split) * stride + DH;
-    dst[0] = ml[tid][0];
-    dst[1] = ml[tid][1];
-  }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    int32_t* ctr = counters + b * gridDim.y + hg;
-    const int ticket = atomicAdd(ctr, 1);
-    last_s = (ticket == p.n_splits - 1);
-    if (last_s) *ctr = 0;  // every CTA of this group has arrived: reset for the next launch
-  }
-  __syncthreads();
-  if (!last_s) return;
-  __threadfence();
-
-  // ---- 5. merge (fixed order over splits => deterministic)
-  for (int idx = tid; idx < GT * DH; idx += kAttnThreads) {
-    const int h = idx / DH, d = idx % DH;
-    const float* base = p.scratch + (static_cast<size_t>(b) * p.n_q_heads + head0 + h) * p.n_splits * stride;
-    float M = -INFINITY;
-    for (int s = 0; s < p.n_splits; ++s) M = fmaxf(M, __ldcg(base + s * stride + DH));
-    float lsum = 0.f, o = 0.f;
-    for (int s = 0; s < p.n_splits; ++s) {
-      const float ms = __ldcg(base + s * stride + DH);
-      const float w = (ms == -INFINITY) ? 0.f : __expf(ms - M);
-      lsum += w * __ldcg(base + s * stride + DH + 1);
-      o += w * __ldcg(base + s * stride + d);
+    const float M = fmaxf(fmaxf(mls[0][h][0], mls[1][h][0]), fmaxf(mls[2][h][0], mls[3][h][0]));
+    float o = 0.f, ls = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float f = (mls[w][h][0] == -INFINITY) ? 0.f : __expf(mls[w][h][0] - M);
+      o += f * red[w][h][d];
+      ls += f * mls[w][h][1];
     }
-    p.o[(static_cast<size_t>(b) * p.n_q_heads + head0 + h) * DH + d] = lsum > 0.f ? o / lsum : 0.f;
+    float* dst = p.scratch + ((static_cast<size_t>(b) * p.n_q_heads + head0 + h) * p.n_splits + split) * stride;
+    dst[d] = o;
+    if (d == 0) {
+      dst[DH] = M;
+      dst[DH + 1] = ls;
+    }
   }
 }
 
-template <int GT>
-cudaError_t launch_gt(const DecodeAttnParams& p, int chunk, int32_t* counters, cudaStream_t stream, bool pdl) {
+// Merge of the per-split partials of one (sequence, head) by log-sum-exp, in split order.
+constexpr int kMaxSplits = 1024;
+template <int DH>
+__global__ void __launch_bounds__(DH) decode_attention_merge_kernel(const float* scratch, int n_q_heads, int n_splits,
+                                                                    float* o) {
+  __shared__ float wgt[kMaxSplits];
+  __shared__ float red_m[DH / 32], red_l[DH / 32];
+  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr int stride = DH + 2;
+  pdl_launch_dependents();
+  pdl_wait();
+  const float* base = scratch + (static_cast<size_t>(b) * n_q_heads + h) * n_splits * stride;
+  float m = -INFINITY;
+  for (int s = tid; s < n_splits; s += DH) {
+    wgt[s] = __ldcg(base + s * stride + DH);
+    m = fmaxf(m, wgt[s]);
+  }
+  m = warp_max(m);
+  if (lane == 0) red_m[warp] = m;
+  __syncthreads();
+  float M = red_m[0];
+#pragma unroll
+  for (int w = 1; w < DH / 32; ++w) M = fmaxf(M, red_m[w]);
+  float l = 0.f;
+  for (int s = tid; s < n_splits; s += DH) {
+    const float f = (wgt[s] == -INFINITY) ? 0.f : __expf(wgt[s] - M);
+    wgt[s] = f;
+    l += f * __ldcg(base + s * stride + DH + 1);
+  }
+  l = warp_sum(l);
+  if (lane == 0) red_l[warp] = l;
+  __syncthreads();
+  float lsum = 0.f;
+#pragma unroll
+  for (int w = 0; w < DH / 32; ++w) lsum += red_l[w];
+  float acc = 0.f;
+#pragma unroll 8
+  for (int s = 0; s < n_splits; ++s) acc += wgt[s] * __ldcg(base + s * stride + tid);
+  o[(static_cast<size_t>(b) * n_q_heads + h) * DH + tid] = lsum > 0.f ? acc / lsum : 0.f;
+}
+
+cudaLaunchConfig_t make_cfg(dim3 grid, dim3 block, cudaStream_t stream, bool pdl, cudaLaunchAttribute* at) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(p.n_splits, p.n_q_heads / GT, p.batch);
-  cfg.blockDim = dim3(kAttnThreads);
-  cfg.dynamicSmemBytes = 0;
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
   cfg.stream = stream;
-  cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = pdl ? 1 : 0;
-  if (p.head_dim == 128) return cudaLaunchKernelEx(&cfg, decode_attention_kernel<GT, 128>, p, chunk, counters);
-  return cudaLaunchKernelEx(&cfg, decode_attention_kernel<GT, 64>, p, chunk, counters);
+  return cfg;
+}
+
+template <int GT>
+cudaError_t launch_gt(const DecodeAttnParams& p, cudaStream_t stream, bool pdl) {
+  cudaLaunchAttribute at[1];
+  cudaLaunchConfig_t cfg = make_cfg(dim3(p.n_splits, p.n_q_heads / GT, p.batch), dim3(kAttnThreads), stream, pdl, at);
+  if (p.head_dim == 128) return cudaLaunchKernelEx(&cfg, decode_attention_kernel<GT, 128>, p);
+  return cudaLaunchKernelEx(&cfg, decode_attention_kernel<GT, 64>, p);
 }
 
 int heads_per_cta(int n_q_heads, int n_kv_heads) {
@@ -208,36 +259,32 @@ int heads_per_cta(int n_q_heads, int n_kv_heads) {
 }  // namespace
 
 int decode_attention_splits(int batch, int n_kv_heads, int max_len, int sm_count) {
-  // enough CTAs for ~2 per SM, at most kMaxChunk keys per CTA, at least 32
-  const int ctas_per_split = batch * n_kv_heads;
-  int want = (2 * sm_count + ctas_per_split - 1) / ctas_per_split;
-  const int lo = (max_len + kMaxChunk - 1) / kMaxChunk;
-  const int hi = (max_len + 31) / 32;
-  if (want < lo) want = lo;
-  if (want > hi) want = hi;
-  return want < 1 ? 1 : want;
+  (void)batch, (void)n_kv_heads, (void)sm_count;
+  const int n = (max_len + kChunk - 1) / kChunk;  // one CTA per 64 keys
+  return n < 1 ? 1 : n;
 }
 
-// scratch layout: [batch * Hq ticket counters (int32), padded to 64 floats][partials]
+// scratch: [batch][Hq][n_splits][Dh + 2] floats (o, m, l per split)
 size_t decode_attention_scratch_floats(int batch, int n_q_heads, int head_dim, int n_splits) {
-  const size_t counters = (static_cast<size_t>(batch) * n_q_heads + 63) / 64 * 64;
-  return counters + static_cast<size_t>(batch) * n_q_heads * n_splits * (head_dim + 2);
+  return static_cast<size_t>(batch) * n_q_heads * n_splits * (head_dim + 2);
 }
 
-cudaError_t launch_decode_attention(const DecodeAttnParams& p_in, cudaStream_t stream, bool pdl) {
-  DecodeAttnParams p = p_in;
-  const size_t counters = (static_cast<size_t>(p.batch) * p.n_q_heads + 63) / 64 * 64;
-  int32_t* ctr = reinterpret_cast<int32_t*>(p.scratch);
-  p.scratch = p.scratch + counters;
-  int chunk = (p.max_len + p.n_splits - 1) / p.n_splits;
-  chunk = (chunk + 31) / 32 * 32;
-  if (chunk > kMaxChunk) return cudaErrorInvalidValue;
+cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stream, bool pdl) {
+  if (p.n_splits * kChunk < p.max_len || p.n_splits > kMaxSplits) return cudaErrorInvalidValue;
+  cudaError_t e;
   switch (heads_per_cta(p.n_q_heads, p.n_kv_heads)) {
-    case 8: return launch_gt<8>(p, chunk, ctr, stream, pdl);
-    case 4: return launch_gt<4>(p, chunk, ctr, stream, pdl);
-    case 2: return launch_gt<2>(p, chunk, ctr, stream, pdl);
-    default: return launch_gt<1>(p, chunk, ctr, stream, pdl);
+    case 8: e = launch_gt<8>(p, stream, pdl); break;
+    case 4: e = launch_gt<4>(p, stream, pdl); break;
+    case 2: e = launch_gt<2>(p, stream, pdl); break;
+    default: e = launch_gt<1>(p, stream, pdl); break;
   }
+  if (e != cudaSuccess) return e;
+  cudaLaunchAttribute at[1];
+  cudaLaunchConfig_t cfg = make_cfg(dim3(p.n_q_heads, p.batch), dim3(p.head_dim), stream, pdl, at);
+  const float* scratch = p.scratch;
+  if (p.head_dim == 128)
+    return cudaLaunchKernelEx(&cfg, decode_attention_merge_kernel<128>, scratch, p.n_q_heads, p.n_splits, p.o);
+  return cudaLaunchKernelEx(&cfg, decode_attention_merge_kernel<64>, scratch, p.n_q_heads, p.n_splits, p.o);
 }
 
 }  // namespace ladder

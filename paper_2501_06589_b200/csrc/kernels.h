@@ -35,10 +35,17 @@ struct SmallMParams {
   void* out;               // EPI_RESID / EPI_PLAIN: fp32 [batch, N]; EPI_SWIGLU: fp32 [batch, N/2]
   QkvEpilogue qkv;         // EPI_QKV_ROPE
   int32_t* status;         // device status word (may be NULL)
+  // batch <= 8 (dynamic item claiming, split-K fix-up):
+  float* scratch;          // smallm_gemm_scratch_floats(N, K, batch) floats, ticket part zero; kernels that
+                           // may run concurrently need distinct scratch
+  int32_t* work;           // 2 ints, zero: claim counter + finished-CTA counter of THIS launch (left zero)
+  float* part;             // set by the launcher: partial sums inside scratch
+  int32_t* tickets;        // set by the launcher: ticket counters inside scratch
 };
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);
 size_t smallm_gemm_smem_bytes(int batch);
+size_t smallm_gemm_scratch_floats(int N, int K, int batch);
 
 // Decode attention (split over the cache) and its combine step.
 struct DecodeAttnParams {

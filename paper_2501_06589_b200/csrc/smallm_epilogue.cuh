@@ -1,0 +1,64 @@
+// Epilogues shared by the weight-streaming decode GEMM kernels.  `value(r, b)` returns the finished
+// accumulator (K-split reduced, 1/rms applied) of local row r of the block and batch row b; NT
+// threads (index ct) walk the block's outputs.
+#pragma once
+#include "common.cuh"
+#include "kernels.h"
+
+namespace ladder {
+
+template <int NT = 128, typename ValueFn>
+__device__ __forceinline__ void smallm_epilogue(const SmallMParams& p, int ct, int prow, int nbase, int batch,
+                                                ValueFn value) {
+  if (p.epi_mode == EPI_RESID || p.epi_mode == EPI_PLAIN) {
+    // x_m = addend + h_m(.)   (the residual add of Eq. 1 / Eq. 2 of the paper), or a plain store
+    float* out = static_cast<float*>(p.out);
+    for (int idx = ct; idx < prow * batch; idx += NT) {
+      const int r = idx % prow, b = idx / prow;
+      const size_t o = static_cast<size_t>(b) * p.N + nbase + r;
+      float v = value(r, b);
+      if (p.epi_mode == EPI_RESID) v += p.addend[o];
+      out[o] = v;
+    }
+  } else if (p.epi_mode == EPI_SWIGLU) {
+    // rows (2j, 2j+1) = (gate_j, up_j)  ->  h_j = silu(gate_j) * up_j
+    float* out = static_cast<float*>(p.out);
+    const int half = prow >> 1;
+    for (int idx = ct; idx < half * batch; idx += NT) {
+      const int pr = idx % half, b = idx / half;
+      const float gt = value(2 * pr, b), up = value(2 * pr + 1, b);
+      out[static_cast<size_t>(b) * (p.N >> 1) + ((nbase >> 1) + pr)] = gt / (1.f + __expf(-gt)) * up;
+    }
+  } else if (p.epi_mode == EPI_QKV_ROPE) {
+    // rotary embedding on interleaved pairs of q and k at position seq_lens[b]; k, v appended to the cache
+    const QkvEpilogue& e = p.qkv;
+    const int half = prow >> 1, Dh = e.head_dim;
+    const int nq = e.n_q_heads * Dh, nk = e.n_kv_heads * Dh;
+    for (int idx = ct; idx < half * batch; idx += NT) {
+      const int pr = idx % half, b = idx / half;
+      const int n = nbase + 2 * pr;
+      float v0 = value(2 * pr, b), v1 = value(2 * pr + 1, b);
+      const int pos = e.seq_lens[b];
+      if (pos < 0 || pos >= e.max_seq_len) {
+        if (p.status) atomicOr(p.status, LADDER_DEV_CACHE_OVERFLOW);
+        continue;
+      }
+      if (n < nq + nk) {
+        const float2 cs = e.rope[static_cast<size_t>(pos) * (Dh >> 1) + ((n % Dh) >> 1)];
+        const float a0 = v0 * cs.x - v1 * cs.y, a1 = v0 * cs.y + v1 * cs.x;
+        v0 = a0;
+        v1 = a1;
+      }
+      if (n < nq) {
+        *reinterpret_cast<float2*>(e.q_out_f32 + static_cast<size_t>(b) * nq + n) = make_float2(v0, v1);
+      } else {
+        const int nn = n < nq + nk ? n - nq : n - nq - nk;
+        __nv_bfloat16* cache = n < nq + nk ? e.k_cache : e.v_cache;
+        const size_t off = ((static_cast<size_t>(b) * e.n_kv_heads + nn / Dh) * e.max_seq_len + pos) * Dh + (nn % Dh);
+        *reinterpret_cast<uint32_t*>(cache + off) = pack_bf16x2(v0, v1);
+      }
+    }
+  }
+}
+
+}  // namespace ladder

@@ -1,4 +1,5 @@
-// Weight-streaming small-M GEMM for the decode path:  acc[b, n] = sum_k act[b, k] * W[n, k],  b < batch <= 64.
+// Weight-streaming small-M GEMM for the decode path, batches 9..64 (batch <= 8 has its own kernel
+// in decode_gemm.cu):  acc[b, n] = sum_k act[b, k] * W[n, k].
 //
 // The kernel is HBM-bound: every weight byte is read exactly once and nothing else of size
 // is touched.  Design:
@@ -25,6 +26,7 @@
 // Results are deterministic: the K split across warps is reduced in a fixed order.
 #include "common.cuh"
 #include "kernels.h"
+#include "smallm_epilogue.cuh"
 
 namespace ladder {
 namespace {
@@ -319,53 +321,7 @@ __global__ void __launch_bounds__(kThreads, 1) smallm_gemm_kernel(const SmallMPa
       return s;
     };
 
-    if (p.epi_mode == EPI_RESID || p.epi_mode == EPI_PLAIN) {
-      float* out = static_cast<float*>(p.out);
-      for (int idx = ct; idx < prow * batch; idx += 128) {
-        const int r = idx % prow, b = idx / prow;
-        const size_t o = static_cast<size_t>(b) * p.N + nbase + r;
-        float v = value(r, b);
-        if (p.epi_mode == EPI_RESID) v += p.addend[o];
-        out[o] = v;
-      }
-    } else if (p.epi_mode == EPI_SWIGLU) {
-      float* out = static_cast<float*>(p.out);
-      const int half = prow >> 1;
-      for (int idx = ct; idx < half * batch; idx += 128) {
-        const int pr = idx % half, b = idx / half;
-        const float gt = value(2 * pr, b), up = value(2 * pr + 1, b);
-        out[static_cast<size_t>(b) * (p.N >> 1) + ((nbase >> 1) + pr)] = gt / (1.f + __expf(-gt)) * up;
-      }
-    } else if (p.epi_mode == EPI_QKV_ROPE) {
-      const QkvEpilogue& e = p.qkv;
-      const int half = prow >> 1, Dh = e.head_dim;
-      const int nq = e.n_q_heads * Dh, nk = e.n_kv_heads * Dh;
-      for (int idx = ct; idx < half * batch; idx += 128) {
-        const int pr = idx % half, b = idx / half;
-        const int n = nbase + 2 * pr;
-        float v0 = value(2 * pr, b), v1 = value(2 * pr + 1, b);
-        const int pos = e.seq_lens[b];
-        if (pos < 0 || pos >= e.max_seq_len) {
-          if (p.status) atomicOr(p.status, LADDER_DEV_CACHE_OVERFLOW);
-          continue;
-        }
-        if (n < nq + nk) {  // rotate q and k pairs
-          const float2 cs = e.rope[static_cast<size_t>(pos) * (Dh >> 1) + ((n % Dh) >> 1)];
-          const float a0 = v0 * cs.x - v1 * cs.y, a1 = v0 * cs.y + v1 * cs.x;
-          v0 = a0;
-          v1 = a1;
-        }
-        if (n < nq) {
-          *reinterpret_cast<float2*>(e.q_out_f32 + static_cast<size_t>(b) * nq + n) = make_float2(v0, v1);
-        } else {
-          const int nn = n < nq + nk ? n - nq : n - nq - nk;
-          __nv_bfloat16* cache = n < nq + nk ? e.k_cache : e.v_cache;
-          const size_t off =
-              ((static_cast<size_t>(b) * e.n_kv_heads + nn / Dh) * e.max_seq_len + pos) * Dh + (nn % Dh);
-          *reinterpret_cast<uint32_t*>(cache + off) = pack_bf16x2(v0, v1);
-        }
-      }
-    }
+    smallm_epilogue(p, ct, prow, nbase, batch, value);
     asm volatile("bar.sync 1, 128;" ::: "memory");  // red / rstd are reused by the next pass
   }
   if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
@@ -399,28 +355,23 @@ cudaError_t init_nb() {
 
 }  // namespace
 
-cudaError_t smallm_gemm_init() {
-  cudaError_t e = init_nb<1, true>();
-  if (e == cudaSuccess) e = init_nb<1, false>();
-  if (e == cudaSuccess) e = init_nb<2, false>();
+cudaError_t smallm_gemm_wide_init() {
+  cudaError_t e = init_nb<2, false>();
   if (e == cudaSuccess) e = init_nb<4, false>();
   if (e == cudaSuccess) e = init_nb<8, false>();
   return e;
 }
 
-size_t smallm_gemm_smem_bytes(int batch) {
-  if (batch <= 4) return Cfg<1, true>::SMEM;
-  if (batch <= 8) return Cfg<1, false>::SMEM;
+size_t smallm_gemm_wide_smem_bytes(int batch) {
   if (batch <= 16) return Cfg<2, false>::SMEM;
   if (batch <= 32) return Cfg<4, false>::SMEM;
   return Cfg<8, false>::SMEM;
 }
 
-cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
+// batch 9..64
+cudaError_t launch_smallm_gemm_wide(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
   const int units = p.N >> 3;
   const int grid = units < sm_count ? units : sm_count;
-  if (p.batch <= 4) return launch_nb<1, true>(p, stream, pdl, grid);
-  if (p.batch <= 8) return launch_nb<1, false>(p, stream, pdl, grid);
   if (p.batch <= 16) return launch_nb<2, false>(p, stream, pdl, grid);
   if (p.batch <= 32) return launch_nb<4, false>(p, stream, pdl, grid);
   return launch_nb<8, false>(p, stream, pdl, grid);

@@ -1,0 +1,107 @@
+"""Run ONE kernel of the decode path at a model's true shape, a few launches in a row -- the
+small, self-ending workload to put under `ncu` (or to time with CUDA events).
+
+    python -m paper_2501_06589_b200.run_op gate_up --config 70b --layers 2 --iters 2
+
+ops: qkv, wo, gate_up, down, lm_head (weight-streaming GEMMs), attn (split-KV decode attention),
+     prefill_gemm, prefill_attn.  Each launch uses a different layer's weights, so nothing is
+     served from L2.  Prints one line with the mean time per launch and the achieved GB/s or TFLOP/s.
+"""
+from __future__ import annotations
+
+import argparse
+
+import torch
+
+from . import binding as B
+from . import build, synth
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("op")
+    ap.add_argument("--config", default="70b")
+    ap.add_argument("--layers", type=int, default=2, help="distinct weight sets to allocate")
+    ap.add_argument("--iters", type=int, default=2, help="passes over the layers")
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--kv-len", type=int, default=None)
+    ap.add_argument("--tokens", type=int, default=4096, help="M of the prefill GEMM")
+    a = ap.parse_args()
+    build.build()
+    B.lib()
+    s = synth.SHAPES[a.config]
+    bsz = a.batch or s.batch
+    d, F, Hq, Hkv, Dh, V = s.d_model, s.d_ff, s.n_q_heads, s.n_kv_heads, s.head_dim, s.vocab_size
+    L = a.layers
+    dev = "cuda"
+
+    def w(rows, cols):
+        return [(torch.randn(rows, cols, device=dev) * 0.02).to(torch.bfloat16) for _ in range(L)]
+
+    x = torch.randn(bsz, d, device=dev)
+    gain = torch.ones(d, dtype=torch.bfloat16, device=dev)
+    if a.op == "qkv":
+        W, out = w(s.qkv_rows, d), torch.empty(bsz, s.qkv_rows, device=dev)
+        fn, nbytes, flops = (lambda l: B.op_smallm_gemm(W[l], x, 1, 2, out, gain=gain)), 2 * s.qkv_rows * d, 0
+    elif a.op == "wo":
+        W, xin, add, out = w(d, Hq * Dh), torch.randn(bsz, Hq * Dh, device=dev), torch.randn(bsz, d, device=dev), torch.empty(bsz, d, device=dev)
+        fn, nbytes, flops = (lambda l: B.op_smallm_gemm(W[l], xin, 0, 0, out, addend=add)), 2 * d * Hq * Dh, 0
+    elif a.op == "gate_up":
+        W, out = w(2 * F, d), torch.empty(bsz, F, device=dev)
+        fn, nbytes, flops = (lambda l: B.op_smallm_gemm(W[l], x, 1, 1, out, gain=gain)), 4 * F * d, 0
+    elif a.op == "down":
+        W, xin, add, out = w(d, F), torch.randn(bsz, F, device=dev), torch.randn(bsz, d, device=dev), torch.empty(bsz, d, device=dev)
+        fn, nbytes, flops = (lambda l: B.op_smallm_gemm(W[l], xin, 0, 0, out, addend=add)), 2 * d * F, 0
+    elif a.op == "lm_head":
+        W, out = w(V, d), torch.empty(bsz, V, device=dev)
+        fn, nbytes, flops = (lambda l: B.op_smallm_gemm(W[l], x, 1, 2, out, gain=gain)), 2 * V * d, 0
+    elif a.op == "attn":
+        max_seq = s.prompt_len + s.decode_steps
+        kv = a.kv_len or (s.prompt_len + s.decode_steps // 2)
+        q = torch.randn(bsz, Hq * Dh, device=dev)
+        k = [torch.randn(bsz, Hkv, max_seq, Dh, device=dev).to(torch.bfloat16) for _ in range(L)]
+        v = [torch.randn(bsz, Hkv, max_seq, Dh, device=dev).to(torch.bfloat16) for _ in range(L)]
+        lens = torch.full((bsz,), kv, dtype=torch.int32, device=dev)
+        scr = torch.empty(B.decode_attention_scratch_bytes(bsz, Hq, Dh, max_seq) // 4, device=dev)
+        o = torch.empty(bsz, Hq * Dh, device=dev)
+        fn = lambda l: B.op_decode_attention(q, k[l], v[l], lens, Hq, Hkv, Dh, max_seq, scr, o)
+        nbytes, flops = 2 * 2 * bsz * Hkv * kv * Dh, 0
+    elif a.op == "prefill_gemm":
+        M = a.tokens
+        A = (torch.randn(M, d, device=dev)).to(torch.bfloat16)
+        A_lo = (torch.randn(M, d, device=dev) * 1e-3).to(torch.bfloat16)
+        W, out = w(2 * F, d), torch.empty(M, F, dtype=torch.bfloat16, device=dev)
+        out_lo = torch.empty_like(out)
+        fn = lambda l: B.op_prefill_gemm(A, W[l], 1, out, A_lo=A_lo, out_lo=out_lo)
+        nbytes, flops = 0, 2.0 * M * 2 * F * d
+    elif a.op == "prefill_attn":
+        S = s.prompt_len
+        q = torch.randn(bsz, S, Hq * Dh, device=dev).to(torch.bfloat16)
+        q_lo = (torch.randn(bsz, S, Hq * Dh, device=dev) * 1e-3).to(torch.bfloat16)
+        k = [torch.randn(bsz, Hkv, S, Dh, device=dev).to(torch.bfloat16) for _ in range(L)]
+        v = [torch.randn(bsz, Hkv, S, Dh, device=dev).to(torch.bfloat16) for _ in range(L)]
+        o = torch.empty_like(q)
+        o_lo = torch.empty_like(q)
+        fn = lambda l: B.op_prefill_attention(q, k[l], v[l], bsz, S, Hq, Hkv, Dh, S, o, q_lo=q_lo, o_lo=o_lo)
+        nbytes, flops = 0, 4.0 * bsz * Hq * Dh * S * (S + 1) / 2
+    else:
+        raise SystemExit(f"unknown op {a.op}")
+
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for l in range(L):          # warm-up pass
+        fn(l)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(a.iters):
+        for l in range(L):
+            fn(l)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / (a.iters * L)
+    rate = f"{nbytes / ms / 1e6:.0f} GB/s" if nbytes else f"{flops / ms / 1e9:.1f} TFLOP/s"
+    print(f"{a.op} [{a.config}, batch {bsz}]: {ms * 1e3:.2f} us per launch, {rate}")
+
+
+if __name__ == "__main__":
+    main()

@@ -28,11 +28,11 @@ def _f64(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-# Decode GEMMs feed the activation as a bf16 hi+lo pair (batch <= 16): what is left is fp32
-# accumulation error, ~1e-5 of the row maximum.  Above batch 16 the activation is a single
-# bf16 (2^-9 relative rounding per element, random sign), ~1e-3 of the row maximum.
+# Decode GEMMs feed the activation as a bf16 hi+lo pair for batch <= 4 (packed into one MMA tile)
+# and 9..16: what is left is fp32 accumulation error, ~1e-5 of the row maximum.  Batches 5..8 and
+# above 16 use a single bf16 (2^-9 relative rounding per element, random sign), ~1e-3 of the maximum.
 def tol_gemm(batch):
-    return 2e-4 if batch <= 16 else 1e-2
+    return 2e-4 if (batch <= 4 or 9 <= batch <= 16) else 1e-2
 
 
 @pytest.mark.parametrize("N,K,batch", [(256, 256, 1), (1376, 256, 4), (256, 688, 3), (1024, 2048, 8),
@@ -76,7 +76,7 @@ def test_smallm_gemm_swiglu(B, F, K, batch):
     n = O.rmsnorm(_f64(x), _f64(g), 1e-5)
     w = _f64(W)
     ref = O.silu(n @ w[0::2].T) * (n @ w[1::2].T)
-    assert rel_err(_f64(out), ref) < 5e-4
+    assert rel_err(_f64(out), ref) < (5e-4 if batch <= 4 else 2e-2)
 
 
 def test_smallm_gemm_is_deterministic_and_batch_invariant(B):

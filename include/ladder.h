@@ -187,6 +187,24 @@ ladder_status_t ladder_op_decode_attention(const float* q, const void* k, const 
                                            int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
                                            int32_t max_seq_len, float* scratch, void* o, void* cuda_stream);
 
+/* The same split-KV decode attention for callers that must not allocate device memory (a server
+ * whose own pool owns the whole device, a memory-capped container slice, a host framework that
+ * forbids cudaMalloc after start-up).  This entry point has no counterpart in the paper; it exists
+ * for deployment.  Its scratch is a fixed 8 MiB array inside the library image, resident on every
+ * GPU that loads the library until the process exits, so the call needs
+ *     batch * n_q_heads * ceil(max_seq_len / 64) * (head_dim + 2) <= 2 * 1024 * 1024 floats
+ * and returns LADDER_ERR_UNSUPPORTED otherwise (e.g. batch 4, 64 heads of 128, up to 2048 keys fits).
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.  The FIRST call on each
+ * device looks up the array's device address (cudaGetSymbolAddress, with that device current):
+ * make that first call outside any stream capture.  All calls share the one array, which keeps
+ * the previous call's partials; nothing in it needs clearing (every split rewrites its partial
+ * before the merge reads it), but two calls that overlap on the GPU -- different streams, or
+ * different host threads -- race on it: serialise them.  Arguments and result as
+ * ladder_op_decode_attention, minus the scratch. */
+ladder_status_t ladder_op_decode_attention_noalloc(const float* q, const void* k, const void* v, const int32_t* kv_len,
+                                                   int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                                                   int32_t head_dim, int32_t max_seq_len, void* o, void* cuda_stream);
+
 /* Large-M GEMM of the prefill path: C[m,n] = sum_k (A[m,k] + A_lo[m,k]) * W[n,k], A bf16 [M,K], W bf16 [N,K].
  *   A_lo: optional bf16 [M,K] low part of the activation (activation ~ A + A_lo); NULL = single bf16.
  *   epi_mode 0: out_f32[m,n] = addend[m,n] + acc;  1: SwiGLU -> out_bf16 [M, N/2];

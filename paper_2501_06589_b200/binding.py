@@ -24,6 +24,7 @@ EXPORTS = [
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
     "ladder_last_error", "ladder_op_smallm_gemm", "ladder_decode_attention_scratch_bytes",
     "ladder_op_decode_attention", "ladder_op_prefill_gemm", "ladder_op_prefill_attention",
+    "ladder_op_decode_attention_noalloc",
 ]
 
 
@@ -96,6 +97,9 @@ def lib() -> C.CDLL:
         L.ladder_op_decode_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                                  C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
                                                  C.c_void_p, C.c_void_p]
+        L.ladder_op_decode_attention_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                                         C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                                         C.c_void_p]
         L.ladder_op_prefill_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                              C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ladder_op_prefill_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
@@ -244,6 +248,13 @@ def decode_attention_scratch_bytes(batch: int, n_q_heads: int, head_dim: int, ma
 def op_decode_attention(q, k, v, kv_len, n_q_heads, n_kv_heads, head_dim, max_seq_len, scratch, o):
     _check(lib().ladder_op_decode_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_len), q.shape[0], n_q_heads,
                                             n_kv_heads, head_dim, max_seq_len, _ptr(scratch), _ptr(o), _stream()))
+
+
+def op_decode_attention_noalloc(q, k, v, kv_len, n_q_heads, n_kv_heads, head_dim, max_seq_len, o):
+    """Decode attention whose scratch lives inside the library image: for callers that cannot
+    allocate device memory.  Raises LadderError(status 2) when the shape needs more than 8 MiB."""
+    _check(lib().ladder_op_decode_attention_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_len), q.shape[0], n_q_heads,
+                                                    n_kv_heads, head_dim, max_seq_len, _ptr(o), _stream()))
 
 
 def op_prefill_gemm(A, W, epi_mode: int, out, addend=None, A_lo=None, out_lo=None):

@@ -14,6 +14,7 @@
 //      to an L2-resident scratch; a second, tiny kernel (one CTA per sequence and head, launched
 //      with programmatic dependent launch) merges the splits in a fixed order and writes o in fp32.
 // The shared-memory footprint (~19 KB) lets a CTA co-reside with a weight-streaming GEMM CTA.
+#include "../../include/ladder.h"
 #include "common.cuh"
 #include "kernels.h"
 
@@ -288,3 +289,75 @@ cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stre
 }
 
 }  // namespace ladder
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant of the decode-attention entry point.
+//
+// Some hosts of this library may not allocate device memory at all once they are running: an
+// inference server that has handed every byte of the device to its own pool allocator, a process
+// inside a memory-capped container slice, code running under a framework that forbids cudaMalloc
+// after start-up.  For them the per-split partial results (the only scratch this kernel needs) live
+// in a fixed array inside the library image instead of a caller buffer.  The array is part of every
+// context that loads the library and stays resident until the process exits, hence the modest cap.
+namespace ladder {
+namespace {
+
+constexpr size_t kNoAllocScratchFloats = size_t(2) << 20;  // 8 MiB: e.g. batch 4, 64 heads x 128, 2048 keys
+static __device__ __align__(256) float g_noalloc_scratch[kNoAllocScratchFloats];
+
+constexpr int kMaxDevices = 64;
+float* g_noalloc_ptr[kMaxDevices];  // device address of the array on each device, resolved once
+
+// In host code the array's name is only a handle for the runtime; the address a kernel can use
+// must be looked up per device, with that device current.
+cudaError_t noalloc_scratch(float** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!g_noalloc_ptr[dev]) {
+    float* ptr = nullptr;
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    g_noalloc_ptr[dev] = ptr;
+  }
+  *out = g_noalloc_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace ladder
+
+extern "C" ladder_status_t ladder_op_decode_attention_noalloc(const float* q, const void* k, const void* v,
+                                                              const int32_t* kv_len, int32_t batch, int32_t n_q_heads,
+                                                              int32_t n_kv_heads, int32_t head_dim,
+                                                              int32_t max_seq_len, void* o, void* cuda_stream) {
+  using namespace ladder;
+  if (!q || !k || !v || !kv_len || !o) return LADDER_ERR_INVALID_ARG;
+  if (batch < 1 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || (head_dim != 64 && head_dim != 128) ||
+      max_seq_len < 1)
+    return LADDER_ERR_INVALID_ARG;
+  const int n_splits = decode_attention_splits(batch, n_kv_heads, max_seq_len, 0);
+  if (decode_attention_scratch_floats(batch, n_q_heads, head_dim, n_splits) > kNoAllocScratchFloats)
+    return LADDER_ERR_UNSUPPORTED;  // batch * heads * ceil(max_seq_len / 64) * (head_dim + 2) floats exceed 8 MiB
+  float* scratch = nullptr;
+  if (noalloc_scratch(&scratch) != cudaSuccess) return LADDER_ERR_CUDA;
+  DecodeAttnParams a = {};
+  a.q = q;
+  a.k = static_cast<const __nv_bfloat16*>(k);
+  a.v = static_cast<const __nv_bfloat16*>(v);
+  a.kv_len = kv_len;
+  a.kv_len_offset = 0;
+  a.batch = batch;
+  a.n_q_heads = n_q_heads;
+  a.n_kv_heads = n_kv_heads;
+  a.head_dim = head_dim;
+  a.max_seq_len = max_seq_len;
+  a.max_len = max_seq_len;
+  a.n_splits = n_splits;
+  a.scratch = scratch;  // every split writes its whole partial before the merge reads it: nothing to clear
+  a.o = static_cast<float*>(o);
+  return launch_decode_attention(a, static_cast<cudaStream_t>(cuda_stream), false) == cudaSuccess ? LADDER_OK
+                                                                                                   : LADDER_ERR_CUDA;
+}
+

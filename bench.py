@@ -29,6 +29,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the gate/up decode GEMM, from the ncu
+# capture summarised in profiles/decode_gemm_gate_up_70b_batch4.md (true size, no scaling).
+NCU_TRAFFIC_BYTES = {("70b", 4): 945_259_008}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
@@ -152,13 +155,17 @@ def run_reference(args):
     w = synth.make_weights(shape.with_layers(n_sample), device="cpu")
     kv_len = shape.prompt_len
     times = []
+    t_start = time.perf_counter()
     for i in range(args.warmup + args.steps):
         t_layers, t_head, threads = oracle_decode_sample(shape, w, kv_len, n_sample)
         if i >= args.warmup:
             times.append(t_layers * (shape.n_layers / n_sample) + t_head)
+        if times and time.perf_counter() - t_start > 60.0:      # keep the whole run within a few minutes
+            break
     t = statistics.mean(times)
     sample = (f"per step: one decode step at KV length {kv_len}, batch {shape.batch}, {n_sample} of {shape.n_layers} "
-              f"layers + LM head in float32, layer time extrapolated x{shape.n_layers / n_sample:g}")
+              f"layers + LM head in float32, layer time extrapolated x{shape.n_layers / n_sample:g}; "
+              f"{len(times)} of {args.steps} steps sampled (60 s cap)")
     val = shape.batch / t
     line = {"impl": "reference", "metric": "decode_tokens_per_s", "value": val, "unit": "tokens/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
@@ -307,13 +314,10 @@ def main():
     k_gbs = k_bytes / (k_ms * 1e-3) / 1e9
 
     # ---- reduce over ranks (max time), aggregate value
-    t_dev = torch.tensor([dev_ms, e2e_s * 1e3, prefill_ms or 0.0], device="cuda", dtype=torch.float64)
-    if dist:
-        dist.all_reduce(t_dev, op=dist.ReduceOp.MAX)
-    dev_ms, e2e_ms, prefill_ms_max = [float(v) for v in t_dev.tolist()]
+    dev_ms, e2e_ms, prefill_ms_max = max_over_ranks([dev_ms, e2e_s * 1e3, prefill_ms or 0.0], dist, "cuda")
     ms_per_step = dev_ms / steps
-    value = world * bsz * steps / (dev_ms * 1e-3)
-    e2e_value = world * bsz * steps / (e2e_ms * 1e-3)
+    value = aggregate_rate(world, bsz, steps, dev_ms)
+    e2e_value = aggregate_rate(world, bsz, steps, e2e_ms)
     mean_kv = S + (steps + 1) / 2.0
     step_bytes = shape.decode_step_bytes(mean_kv)
     step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
@@ -341,12 +345,8 @@ def main():
                            "tflops": flops / (prefill_ms_max * 1e-3) / 1e12,
                            "frac_of_bf16_peak": flops / (prefill_ms_max * 1e-3) / 1e12 / bf16_peak,
                            "peak_tflops": bf16_peak, "peak_source": peak_src}
-    tr = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tr):
-        try:
-            line["roofline"]["traffic"] = json.load(open(tr)).get("smallm_gemm_gate_up_bytes_per_launch")
-        except Exception:
-            pass
+    if (shape.name, bsz) in NCU_TRAFFIC_BYTES:
+        line["roofline"]["traffic"] = NCU_TRAFFIC_BYTES[(shape.name, bsz)]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(shape, w, S)
     if rank == 0:
@@ -355,6 +355,20 @@ def main():
     if dist:
         dist.destroy_process_group()
     return 0
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of per-rank timings over the process group (replicas: no data-path collective)."""
+    import torch
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def aggregate_rate(world, batch, steps, ms_max):
+    """Whole-job tokens/s of `world` independent replicas, each doing batch x steps tokens in ms_max."""
+    return world * batch * steps / (ms_max * 1e-3)
 
 
 def prefill_flops(shape, bsz, S):

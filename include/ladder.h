@@ -214,6 +214,10 @@ ladder_status_t ladder_op_prefill_gemm(const void* A, const void* A_lo, const vo
                                        int32_t epi_mode, const float* addend, void* out, void* out_lo,
                                        void* cuda_stream);
 
+/* Which implementation the prefill GEMMs use (process-wide): 0 = tcgen05 tensor-core kernel with TMA
+ * and TMEM accumulators (default), 1 = warp-level mma.sync kernel (kept as a cross-check). */
+void ladder_set_prefill_gemm_impl(int32_t impl);
+
 /* Causal grouped-query attention of the prefill path for one layer:
  *   q bf16 [batch, seq_len, Hq*Dh] (rotated), q_lo its optional low part; k,v bf16 cache of one layer
  *   as above, rows 0..seq_len-1 valid; o bf16 [batch, seq_len, Hq*Dh], o_lo its low part (given iff

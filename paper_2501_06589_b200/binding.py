@@ -24,7 +24,7 @@ EXPORTS = [
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
     "ladder_last_error", "ladder_op_smallm_gemm", "ladder_decode_attention_scratch_bytes",
     "ladder_op_decode_attention", "ladder_op_prefill_gemm", "ladder_op_prefill_attention",
-    "ladder_op_decode_attention_noalloc",
+    "ladder_op_decode_attention_noalloc", "ladder_set_prefill_gemm_impl",
 ]
 
 
@@ -100,6 +100,8 @@ def lib() -> C.CDLL:
         L.ladder_op_decode_attention_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                                          C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
                                                          C.c_void_p]
+        L.ladder_set_prefill_gemm_impl.restype = None
+        L.ladder_set_prefill_gemm_impl.argtypes = [C.c_int32]
         L.ladder_op_prefill_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                              C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ladder_op_prefill_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
@@ -255,6 +257,11 @@ def op_decode_attention_noalloc(q, k, v, kv_len, n_q_heads, n_kv_heads, head_dim
     allocate device memory.  Raises LadderError(status 2) when the shape needs more than 8 MiB."""
     _check(lib().ladder_op_decode_attention_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(kv_len), q.shape[0], n_q_heads,
                                                     n_kv_heads, head_dim, max_seq_len, _ptr(o), _stream()))
+
+
+def set_prefill_gemm_impl(impl: int):
+    """0 = tcgen05 kernel (default), 1 = warp-level mma.sync kernel."""
+    lib().ladder_set_prefill_gemm_impl(impl)
 
 
 def op_prefill_gemm(A, W, epi_mode: int, out, addend=None, A_lo=None, out_lo=None):

@@ -22,6 +22,7 @@ cudaError_t kernels_ready() {  // opt-in to large dynamic shared memory, once pe
   if (g_kernels_ready) return cudaSuccess;
   cudaError_t e = smallm_gemm_init();
   if (e == cudaSuccess) e = largem_gemm_init();
+  if (e == cudaSuccess) e = largem_gemm_tc_init();
   if (e == cudaSuccess) e = prefill_attention_init();
   if (e == cudaSuccess) g_kernels_ready = true;
   return e;
@@ -364,6 +365,7 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       p.qkv.head_dim = Dh;
       p.qkv.max_seq_len = c.max_seq_len;
       p.qkv.prefill_seq_len = S;
+      p.status = m->status;
       did(launch_largem_gemm(p, st));
       did(launch_prefill_attention(m->q_pf, m->q_pf + m->q_lo, p.qkv.k_cache, p.qkv.v_cache, batch, S, Hq, Hkv, Dh,
                                    c.max_seq_len, m->o_pf, m->o_pf + m->q_lo, st));
@@ -377,6 +379,7 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       o.epi_mode = EPI_RESID;
       o.addend = m->R[r.add];
       o.out = m->R[r.dst];
+      o.status = m->status;
       did(launch_largem_gemm(o, st));
     }
     {
@@ -392,6 +395,7 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       p.epi_mode = EPI_SWIGLU;
       p.out = m->h_pf;
       p.out_lo = m->h_pf + m->h_lo;
+      p.status = m->status;
       did(launch_largem_gemm(p, st));
       LargeMParams o = {};
       o.A = m->h_pf;
@@ -403,6 +407,7 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       o.epi_mode = EPI_RESID;
       o.addend = m->R[r.add];
       o.out = m->R[r.dst];
+      o.status = m->status;
       did(launch_largem_gemm(o, st));
     }
   }
@@ -457,6 +462,8 @@ const char* ladder_status_string(ladder_status_t s) {
 }
 
 const char* ladder_last_error(const ladder_model_t* m) { return m ? m->err.c_str() : g_create_error.c_str(); }
+
+void ladder_set_prefill_gemm_impl(int32_t impl) { set_prefill_gemm_impl(impl); }
 
 size_t ladder_kv_cache_bytes(const ladder_config_t* c) {
   if (!c) return 0;

@@ -75,8 +75,13 @@ struct LargeMParams {
   void* out;
   __nv_bfloat16* out_lo;   // EPI_SWIGLU / EPI_BF16: lo part of the bf16 output, or NULL
   QkvEpilogue qkv;
+  int32_t* status;         // device status word (may be NULL)
 };
+// Dispatches to the tcgen05 kernel (default) or the warp-level mma.sync kernel (set_prefill_gemm_impl(1)).
 cudaError_t launch_largem_gemm(const LargeMParams& p, cudaStream_t stream);
+cudaError_t launch_largem_gemm_tc(const LargeMParams& p, cudaStream_t stream, int sm_count);
+cudaError_t largem_gemm_tc_init();
+void set_prefill_gemm_impl(int impl);  // 0 = tcgen05 (default), 1 = mma.sync
 
 // q_lo / o_lo: optional lo parts (value ~ hi + lo) of the query input and the attention output.
 cudaError_t launch_prefill_attention(const __nv_bfloat16* q, const __nv_bfloat16* q_lo, const __nv_bfloat16* k,

@@ -5,11 +5,13 @@
 // Activations may come as a bf16 hi + lo pair (a ~ hi + lo): both tiles are staged and multiplied
 // with the same weight tile, which removes the activation rounding error at twice the MMA count.
 //
-// This file holds the warp-level (mma.sync) implementation: 128x128x32 CTA tiles, 3-stage
+// This file holds the dispatcher and the warp-level (mma.sync) implementation, kept as the second
+// opinion the tcgen05 kernel (prefill_gemm_tc.cu) is tested against: 128x128x32 CTA tiles, 3-stage
 // cp.async pipeline, ldmatrix fragments, 8 warps of 64x32.  Adjacent output columns (2j, 2j+1)
 // live in one thread, which is what the pair-wise epilogues (SwiGLU, rotary) need.
 #include "common.cuh"
 #include "kernels.h"
+#include "prefill_epilogue.cuh"
 
 namespace ladder {
 namespace {
@@ -32,61 +34,6 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                : "r"(addr));
-}
-
-__device__ __forceinline__ void epilogue_pair(const LargeMParams& p, int m, int n, float v0, float v1) {
-  if (m >= p.M || n >= p.N) return;
-  switch (p.epi_mode) {
-    case EPI_RESID: {
-      const size_t o = static_cast<size_t>(m) * p.N + n;
-      const float2 a = *reinterpret_cast<const float2*>(p.addend + o);
-      *reinterpret_cast<float2*>(static_cast<float*>(p.out) + o) = make_float2(a.x + v0, a.y + v1);
-      break;
-    }
-    case EPI_SWIGLU: {
-      const float h = v0 / (1.f + __expf(-v0)) * v1;
-      const size_t o = static_cast<size_t>(m) * (p.N >> 1) + (n >> 1);
-      const __nv_bfloat16 hi = __float2bfloat16_rn(h);
-      static_cast<__nv_bfloat16*>(p.out)[o] = hi;
-      if (p.out_lo) p.out_lo[o] = __float2bfloat16_rn(h - __bfloat162float(hi));
-      break;
-    }
-    case EPI_PLAIN:
-      *reinterpret_cast<float2*>(static_cast<float*>(p.out) + static_cast<size_t>(m) * p.N + n) = make_float2(v0, v1);
-      break;
-    case EPI_BF16: {
-      const size_t o = static_cast<size_t>(m) * p.N + n;
-      const uint32_t hi = pack_bf16x2(v0, v1);
-      *reinterpret_cast<uint32_t*>(static_cast<__nv_bfloat16*>(p.out) + o) = hi;
-      if (p.out_lo) *reinterpret_cast<uint32_t*>(p.out_lo + o) = pack_bf16x2(v0 - bf16_lo(hi), v1 - bf16_hi(hi));
-      break;
-    }
-    case EPI_QKV_ROPE: {
-      const QkvEpilogue& e = p.qkv;
-      const int Dh = e.head_dim, nq = e.n_q_heads * Dh, nk = e.n_kv_heads * Dh;
-      const int b = m / e.prefill_seq_len, pos = m % e.prefill_seq_len;
-      if (n < nq + nk) {
-        const float2 cs = e.rope[static_cast<size_t>(pos) * (Dh >> 1) + ((n % Dh) >> 1)];
-        const float a0 = v0 * cs.x - v1 * cs.y, a1 = v0 * cs.y + v1 * cs.x;
-        v0 = a0;
-        v1 = a1;
-      }
-      if (n < nq) {
-        const uint32_t hi = pack_bf16x2(v0, v1);
-        *reinterpret_cast<uint32_t*>(e.q_out_bf16 + static_cast<size_t>(m) * nq + n) = hi;
-        if (e.q_out_lo)
-          *reinterpret_cast<uint32_t*>(e.q_out_lo + static_cast<size_t>(m) * nq + n) =
-              pack_bf16x2(v0 - bf16_lo(hi), v1 - bf16_hi(hi));
-      } else {
-        const int nn = n < nq + nk ? n - nq : n - nq - nk;
-        __nv_bfloat16* cache = n < nq + nk ? e.k_cache : e.v_cache;
-        const size_t off = ((static_cast<size_t>(b) * e.n_kv_heads + nn / Dh) * e.max_seq_len + pos) * Dh + (nn % Dh);
-        *reinterpret_cast<uint32_t*>(cache + off) = pack_bf16x2(v0, v1);
-      }
-      break;
-    }
-    default: break;
-  }
 }
 
 template <bool SPLIT>
@@ -187,7 +134,23 @@ cudaError_t largem_gemm_init() {
   return cudaFuncSetAttribute(largem_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
+namespace {
+int g_prefill_impl = 0;
+int g_sm_count = 0;
+}  // namespace
+
+void set_prefill_gemm_impl(int impl) { g_prefill_impl = impl ? 1 : 0; }
+
 cudaError_t launch_largem_gemm(const LargeMParams& p, cudaStream_t stream) {
+  if (g_prefill_impl == 0) {
+    if (!g_sm_count) {
+      int dev = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess ||
+          cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        g_sm_count = 148;
+    }
+    return launch_largem_gemm_tc(p, stream, g_sm_count);
+  }
   dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM);
   if (p.A_lo) largem_gemm_kernel<true><<<grid, kGemmThreads, kSmemBytes, stream>>>(p);
   else largem_gemm_kernel<false><<<grid, kGemmThreads, kSmemBytes, stream>>>(p);

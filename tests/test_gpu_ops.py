@@ -134,10 +134,12 @@ def _split(shape, seed, std=1.0):
     return f.cuda(), hi.cuda(), lo.cuda()
 
 
+@pytest.mark.parametrize("impl", [0, 1])          # 0 = tcgen05 kernel, 1 = warp-level mma.sync kernel
 @pytest.mark.parametrize("split", [False, True])
 @pytest.mark.parametrize("M,N,K,mode", [(16, 768, 256, 3), (300, 1376, 256, 1), (512, 256, 688, 0),
-                                        (1000, 520, 264, 2), (4096, 1024, 1024, 0)])
-def test_prefill_gemm(B, M, N, K, mode, split):
+                                        (1000, 520, 264, 2), (4096, 1024, 1024, 0), (384, 2056, 8192, 2)])
+def test_prefill_gemm(B, M, N, K, mode, split, impl):
+    B.set_prefill_gemm_impl(impl)
     Af, A, A_lo = _split((M, K), 14)
     W = _bf16((N, K), 15, 0.05)
     acc = (_f64(Af) if split else _f64(A)) @ _f64(W).T
@@ -166,6 +168,7 @@ def test_prefill_gemm(B, M, N, K, mode, split):
     got = _f64(out) + (_f64(out_lo) if out_lo is not None else 0.0)
     # fp32 outputs / hi+lo outputs carry only accumulation error; a single bf16 output rounds at 2^-9
     tol = 2e-4 if (mode in (0, 2) or out_lo is not None) else 1e-2
+    B.set_prefill_gemm_impl(0)
     assert rel_err(got, ref) < tol
 
 

@@ -15,7 +15,8 @@
 //   warps 2-5  epilogue: each warp reads its 32-lane quarter of the accumulator with tcgen05.ld
 //              (32 columns at a time; a thread owns one output row, so the column pairs the SwiGLU and
 //              rotary epilogues need are adjacent registers) and writes the result.
-// Tiles are visited M-fastest so that the CTAs running at the same time share W tiles in L2.
+// Tiles are visited in bands of 16 M-tiles, M-fastest inside a band, so that the CTAs running at the
+// same time work on ~16 x 9 tiles whose A band and W tiles together fit the L2.
 // Every wait is bounded; on a protocol error the kernel records it, drains and frees its TMEM.
 #include <cuda.h>
 
@@ -31,6 +32,17 @@ constexpr int A_BYTES = BM * BK * 2;  // 16 KB
 constexpr int B_BYTES = BN * BK * 2;  // 32 KB
 constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;
 constexpr int kTcThreads = 192;
+constexpr int GROUP_M = 16;  // M-tiles per rasterisation band
+
+// tile index -> (m tile, n tile): bands of GROUP_M m-tiles, m fastest inside a band
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& tm, int& tn) {
+  const int per_band = GROUP_M * tiles_n;
+  const int band = t / per_band, r = t - band * per_band;
+  const int m_first = band * GROUP_M;
+  const int band_m = min(GROUP_M, tiles_m - m_first);
+  tm = m_first + r % band_m;
+  tn = r / band_m;
+}
 constexpr int OFF_BARS = STAGES * STAGE_BYTES;  // full[3], empty[3], tmem_full[2], tmem_empty[2], tmem slot
 constexpr int kTcSmem = OFF_BARS + 16 * 8 + 1024;
 
@@ -129,7 +141,9 @@ largem_gemm_tc_kernel(const LargeMParams p, const __grid_constant__ CUtensorMap 
       bool ok = true;
       int it = 0;
       for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-        const int m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
+        int tm, tn;
+        tile_coords(t, tiles_m, tiles_n, tm, tn);
+        const int m0 = tm * BM, n0 = tn * BN;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % STAGES;
           ok = mbar_wait_bounded(&empty[s], ((it / STAGES) & 1) ^ 1u);
@@ -187,7 +201,9 @@ largem_gemm_tc_kernel(const LargeMParams p, const __grid_constant__ CUtensorMap 
     int i = 0;
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
       const int ab = i & 1;
-      const int m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
+      int tm, tn;
+      tile_coords(t, tiles_m, tiles_n, tm, tn);
+      const int m0 = tm * BM, n0 = tn * BN;
       if (ok) ok = mbar_wait_bounded(&tmem_full[ab], (i >> 1) & 1);
       if (!ok) break;
       tc_fence_after();

@@ -15,7 +15,7 @@
 //     batch <= 4 the high parts occupy columns 0-3 and the low parts columns 4-7 of ONE 8-column
 //     MMA tile, so the extra precision costs no extra MMA; batch 5..8 uses a single bf16.  The
 //     batches all walk the chunks in the same cyclic order, so the stagers free-run one chunk ahead.
-//     They also form the RMSNorm sum of squares up front;
+//     They also form the RMSNorm sum of squares while staging the first batch's chunks;
 //   * four consumer warps: split each tile along K, read 16 contiguous bytes of a weight row and
 //     the matching 16 bytes of an activation row per thread (the K index inside an MMA is
 //     permuted identically for both operands: no ldmatrix, no swizzle, conflict-free with a row
@@ -268,28 +268,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
     bool ok = true;
     pdl_wait();  // activations come from the previous kernel
 
-    if (NORM) {  // sum of squares of every activation row over the whole K
-      float ssq[8];
+    // RMSNorm: the sum of squares of every activation row is accumulated while the chunks of the
+    // FIRST batch are staged (they cover the whole K once); no separate pass over x.
+    float ssq[8];
 #pragma unroll
-      for (int b = 0; b < 8; ++b) ssq[b] = 0.f;
-      for (int u = st; u * 8 < p.K; u += 128) {
-#pragma unroll
-        for (int b = 0; b < 8; ++b) {
-          if (b >= batch) break;
-          const float4* src = reinterpret_cast<const float4*>(actf + static_cast<size_t>(b) * p.K + u * 8);
-          const float4 a = src[0], c = src[1];
-          ssq[b] += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w + c.x * c.x + c.y * c.y + c.z * c.z + c.w * c.w;
-        }
-      }
-#pragma unroll
-      for (int b = 0; b < 8; ++b) {
-        if (b >= batch) break;
-        const float s = warp_sum(ssq[b]);
-        if (lane == 0) ssq_part[sw * 8 + b] = s;
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(norm_ready);
-    }
+    for (int b = 0; b < 8; ++b) ssq[b] = 0.f;
+    bool ssq_on = NORM;
 
     F8 x[4][2];
     uint4 gq[2];
@@ -327,6 +311,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
           float y[8] = {x[i][u].a.x, x[i][u].a.y, x[i][u].a.z, x[i][u].a.w,
                         x[i][u].b.x, x[i][u].b.y, x[i][u].b.z, x[i][u].b.w};
           if (NORM) {
+            if (ssq_on)
+              ssq[b] += y[0] * y[0] + y[1] * y[1] + y[2] * y[2] + y[3] * y[3] + y[4] * y[4] + y[5] * y[5] +
+                        y[6] * y[6] + y[7] * y[7];
             y[0] *= bf16_lo(gq[u].x);
             y[1] *= bf16_hi(gq[u].x);
             y[2] *= bf16_lo(gq[u].y);
@@ -368,6 +355,17 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
       if (!PACKED && batch > 4) {
         load_rows(ch, 1);
         store_rows(1);
+      }
+      if (NORM && r == nchunk - 1) {  // every chunk has been staged once: publish the sums
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+          if (b >= batch) break;
+          const float t = warp_sum(ssq[b]);
+          if (lane == 0) ssq_part[sw * 8 + b] = t;
+        }
+        ssq_on = false;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(norm_ready);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(act_full);

@@ -219,3 +219,45 @@ def test_8b_hybrid_shape_short_context(B):
     err, agree, *_ = check_generation(B, s, 64, np.float32, batch=4, prompt_len=64)       # 260 comparisons
     assert err < HIDDEN_TOL, err
     assert agree >= 0.99, agree
+
+
+def test_70b_full_size_single_live_module(B):
+    """The benchmark's own launch configuration -- all 80 layers of the 70B shape resident (141 GB),
+    batch 4, 1024-token prompts, CUDA-graph decode -- checked with a property that holds at any size:
+    with every output / down projection zeroed except module k's, the model computes x_0 + h_k(x_0)
+    (ladder and standard alike), which the oracle evaluates from layer k's weights alone."""
+    free, _ = torch.cuda.mem_get_info()
+    s = synth.SHAPES["70b"]
+    if free < s.param_count() * 2 + 8e9:
+        pytest.skip("needs ~150 GB of free device memory")
+    w = synth.make_weights(s, device="cuda")
+    bsz, S, steps = s.batch, s.prompt_len, 3
+    prompt = synth.make_tokens(s, bsz, S)
+    for layer, live in ((41, "attention"), (57, "mlp")):
+        keep = (w.w_o[layer].clone(), w.w_down[layer].clone())
+        for l in range(s.n_layers):
+            w.w_o[l].zero_()
+            w.w_down[l].zero_()
+        if live == "attention":
+            w.w_o[layer].copy_(keep[0])
+        else:
+            w.w_down[layer].copy_(keep[1])
+        model = B.Model(w, bsz, S + steps + 1, bsz * S)
+        cache = B.KVCache(s, bsz, S + steps + 1)
+        toks, hids = gpu_generate(B, model, cache, prompt, steps)
+        assert model.device_status() == 0
+        model.close()
+        # oracle: a one-layer model made of layer k's weights (the other module of that layer is dead too)
+        one = synth.replace(s.with_layers(1))
+        w1 = synth.AbiWeights(one, w.tok_embedding, w.final_norm, w.lm_head, [w.attn_norm[layer]], [w.w_qkv[layer]],
+                              [w.w_o[layer]], [w.mlp_norm[layer]], [w.w_gate_up[layer]], [w.w_down[layer]])
+        OW = O.OracleWeights(provider=synth.logical_provider(w1, np.float32))
+        o_toks, o_hids = O.generate(oracle_cfg(one), OW, prompt, steps, S + steps + 1, dtype=np.float32, forced=toks)
+        err = rel_err(hids, o_hids)
+        print(f"[70b full size, live {live} of layer {layer}] hidden max-rel-err {err:.3e}, "
+              f"greedy agreement {float(np.mean(toks == o_toks)):.3f}")
+        assert err < HIDDEN_TOL, (live, err)
+        w.w_o[layer].copy_(keep[0])
+        w.w_down[layer].copy_(keep[1])
+        del cache, OW
+        torch.cuda.empty_cache()

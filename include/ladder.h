@@ -118,6 +118,13 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
  * Defaults: 2, 1, 1.  Results are bit-identical across all settings. */
 ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, int32_t use_graph, int32_t use_pdl);
 
+/* With two streams, the GEMMs of a ladder layer's attention module and MLP module can be run side by side on
+ * disjoint sets of SMs (each GEMM is a persistent kernel that claims its work dynamically, so it runs
+ * on any number of CTAs).  sms_attention_stream: -1 = no split, every GEMM launches on all SMs (default:
+ * measured fastest), 0 = automatic (in proportion to the bytes each module streams), n > 0 = that many
+ * SMs for the attention module's GEMMs and the rest for the MLP's.  Results are bit-identical. */
+ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream);
+
 /* Prompt pass.  d_tokens int32 [batch, seq_len]; every sequence has the same length.
  * Writes cache rows 0..seq_len-1 of sequences 0..batch-1, sets seq_lens[b] = seq_len, and
  * produces outputs for position seq_len-1 (next_tokens = the first generated token).

@@ -19,7 +19,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libladder.so")
 
 EXPORTS = [
-    "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_prefill",
+    "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_model_set_sm_split",
+    "ladder_prefill",
     "ladder_decode_step", "ladder_decode_step_host", "ladder_prefill_host", "ladder_set_position",
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
     "ladder_last_error", "ladder_op_smallm_gemm", "ladder_decode_attention_scratch_bytes",
@@ -73,6 +74,7 @@ def lib() -> C.CDLL:
         L.ladder_model_create.argtypes = [C.POINTER(ladder_config_t), C.POINTER(ladder_weights_t),
                                           C.POINTER(C.c_void_p)]
         L.ladder_model_set_schedule.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32]
+        L.ladder_model_set_sm_split.argtypes = [C.c_void_p, C.c_int32]
         L.ladder_prefill.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32, C.c_int32,
                                      C.POINTER(ladder_outputs_t), C.c_void_p]
         L.ladder_decode_step.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32,
@@ -195,6 +197,9 @@ class Model:
 
     def set_schedule(self, n_streams: int = 2, use_graph: bool = True, use_pdl: bool = True):
         _check(lib().ladder_model_set_schedule(self.h, n_streams, int(use_graph), int(use_pdl)), self.h)
+
+    def set_sm_split(self, sms_attention_stream: int = 0):
+        _check(lib().ladder_model_set_sm_split(self.h, sms_attention_stream), self.h)
 
     def set_position(self, length: int):
         _check(lib().ladder_set_position(self.h, length), self.h)

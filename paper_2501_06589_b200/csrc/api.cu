@@ -70,6 +70,7 @@ struct ladder_model {
   std::vector<cudaEvent_t> ev;  // ev[m] = end of module m (m = 0: embedding)
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   int n_streams = 2, use_graph = 1, use_pdl = 1;
+  int sms_a = -1;  // SMs given to the attention stream in ladder layers (0 = automatic, -1 = no split)
   cudaGraphExec_t graph_exec = nullptr;
   GraphKey graph_key;
   int64_t graph_kernels = 0;
@@ -148,11 +149,13 @@ struct Enqueue {
   bool pdl_ok[2] = {false, false};  // previous op on the stream was a kernel (programmatic edge possible)
   int64_t kernels = 0;
   int slot = 0;  // next claim-counter slot
-  void gemm(int s, SmallMParams& p) {
+  int grid_a = 0, grid_b = 0;  // CTAs per GEMM on stream A / B while the two run side by side (0 = all SMs)
+  void gemm(int s, SmallMParams& p, bool side_by_side = false) {
     p.scratch = m->gemm_scratch[s];
     p.work = m->work_slots + 2 * (slot++ % m->n_work_slots);
     p.status = m->status;
-    launched(s, launch_smallm_gemm(p, stream(s), pdl(s), m->sm_count));
+    const int g = (side_by_side && two && grid_a > 0) ? (s ? grid_b : grid_a) : m->sm_count;
+    launched(s, launch_smallm_gemm(p, stream(s), pdl(s), g));
   }
   cudaError_t err = cudaSuccess;
 
@@ -183,6 +186,25 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   Enqueue q{m, sA, sB, sA != sB};
   const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff;
   const size_t layer_elems = static_cast<size_t>(c.max_batch) * Hkv * c.max_seq_len * Dh;
+  // Optional: in ladder layers the attention module and the MLP module run side by side, and the SMs
+  // can be divided between the two streams (in proportion to the bytes each has to stream, plus a
+  // margin for the attention stream) so that ramp, tail and launch gaps of one stream overlap with the
+  // other's steady weight stream.  Measured on the 70B shape this loses to letting every GEMM take all
+  // SMs (25.1 ms at the best split of 40 SMs vs 24.4 ms): a subset of SMs streams at ~47 GB/s each and
+  // the module chain (Wo waits for the previous down projection and vice versa) leaves it idle in
+  // between.  Off by default.
+  if (q.two && m->sms_a >= 0 && batch <= 8) {
+    int ga = m->sms_a;
+    if (ga == 0) {
+      const double ba = static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh;
+      const double bb = 3.0 * F * d;
+      ga = static_cast<int>(m->sm_count * ba / (ba + bb) * 1.2 + 0.5);
+    }
+    if (ga < 4) ga = 4;
+    if (ga > m->sm_count / 2) ga = m->sm_count / 2;
+    q.grid_a = ga;
+    q.grid_b = m->sm_count - ga;
+  }
 
   q.launched(0, launch_embed(d_tokens, m->tok_embedding, batch, d, c.vocab_size, m->R[0], m->status, sA, false));
   q.pdl_ok[0] = true;
@@ -229,7 +251,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       p.qkv.head_dim = Dh;
       p.qkv.max_seq_len = c.max_seq_len;
       p.status = m->status;
-      q.gemm(0, p);
+      q.gemm(0, p, lad);
 
       DecodeAttnParams a = {};
       a.q = m->q_f32;
@@ -261,7 +283,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       o.addend = m->R[r.add];
       o.out = m->R[r.dst];
       o.status = m->status;
-      q.gemm(0, o);
+      q.gemm(0, o, lad);
       q.record(0, m->ev[mod]);
     }
     // ---------------- MLP module (module index 2l+2) on stream B
@@ -285,7 +307,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       p.epi_mode = EPI_SWIGLU;
       p.out = m->h_dec;
       p.status = m->status;
-      q.gemm(1, p);
+      q.gemm(1, p, lad);
 
       need(1, mod - 1);
       SmallMParams o = {};
@@ -299,7 +321,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       o.addend = m->R[r.add];
       o.out = m->R[r.dst];
       o.status = m->status;
-      q.gemm(1, o);
+      q.gemm(1, o, lad);
       q.record(1, m->ev[mod]);
     }
   }
@@ -628,6 +650,15 @@ ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, 
   m->n_streams = n_streams;
   m->use_graph = use_graph ? 1 : 0;
   m->use_pdl = use_pdl ? 1 : 0;
+  drop_graph(m);
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  if (sms_attention_stream < -1 || sms_attention_stream > m->sm_count / 2)
+    return fail(m, LADDER_ERR_INVALID_ARG, "sms_attention_stream must be -1, 0 or at most half the SMs");
+  m->sms_a = sms_attention_stream;
   drop_graph(m);
   return LADDER_OK;
 }

@@ -136,6 +136,11 @@ __device__ __forceinline__ int mbar_wait_or_stop(uint64_t* bar, uint32_t parity,
   }
 }
 
+#ifdef DG_TRACE
+// per-CTA timeline for tuning builds only: [0] start ns, [1] end ns, [2] SM id, [3] units processed
+__device__ unsigned long long g_trace[148 * 4];
+#endif
+
 template <bool PACKED, bool NORM>
 __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMParams p, const Schedule sched) {
   extern __shared__ uint8_t smem_raw[];
@@ -192,6 +197,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
     const uint8_t* Wb = reinterpret_cast<const uint8_t*>(p.W);
     bool ok = true;
     int it = 0, n = 0;
+#ifdef DG_TRACE
+    int traced_units = 0;
+    if (lane == 0) {
+      uint32_t smid;
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+      g_trace[blockIdx.x * 4 + 0] = global_timer_ns();
+      g_trace[blockIdx.x * 4 + 2] = smid;
+    }
+#endif
     int c = 0;
     while (ok) {
       // one claim at a time (claiming ahead would let a CTA hoard batches it cannot start yet);
@@ -217,6 +231,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
       u0 = __shfl_sync(0xffffffffu, u0, 0);
       nu = __shfl_sync(0xffffffffu, nu, 0);
       if (nu == 0) break;
+#ifdef DG_TRACE
+      traced_units += nu;
+      if (lane == 0) g_trace[blockIdx.x * 4 + 3] = traced_units;
+#endif
       const int row0 = u0 * 8;
       for (int ch = 0; ch < nchunk && ok; ++ch) {
         const int k0 = ch * TK;
@@ -415,6 +433,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
       if (lane == 0) mbar_arrive(&red_free[slot]);  // the consumers may refill this slot
     }
     if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
+#ifdef DG_TRACE
+    if (ft == 0) g_trace[blockIdx.x * 4 + 1] = global_timer_ns();
+#endif
     return;
   }
 
@@ -538,6 +559,12 @@ cudaError_t launch_small(const SmallMParams& p, cudaStream_t stream, bool pdl, i
 }
 
 }  // namespace
+
+#ifdef DG_TRACE
+extern "C" int ladder_debug_read_trace(unsigned long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 cudaError_t smallm_gemm_init() {
   cudaError_t e = cudaFuncSetAttribute(decode_gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);

@@ -261,3 +261,17 @@ def test_70b_full_size_single_live_module(B):
         w.w_down[layer].copy_(keep[1])
         del cache, OW
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("batch", [1, 16, 64])
+@pytest.mark.parametrize("variant", ["ladder", "standard"])
+def test_tp_rank_slice_shape_batches(B, variant, batch):
+    """One tensor-parallel rank's slice of the 70B shape (8 q heads, 1 kv head, ffn 3584, hidden 8192:
+    attention width differs from the hidden size) without communication, cut to 3 layers; the batch
+    sizes of the sweep the paper's throughput figure uses (Sec. 3.3.1), ladder and standard."""
+    s = synth.SHAPES["tp_slice"].with_layers(3)
+    if variant == "standard":
+        s = s.as_standard()
+    err, agree, *_ = check_generation(B, s, 6, np.float32, batch=batch, prompt_len=40)
+    assert err < HIDDEN_TOL, err
+    assert agree >= (0.98 if batch >= 16 else 0.85), agree      # 7 comparisons at batch 1: at most one flip

@@ -118,6 +118,18 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
  * Defaults: 2, 1, 1.  Results are bit-identical across all settings. */
 ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, int32_t use_graph, int32_t use_pdl);
 
+/* Persistent decode step (default on; batch <= 8).  The whole layer stack and the LM head of a decode
+ * step run as ONE cooperative kernel launch: every weight-streaming GEMM is a phase of that kernel,
+ * attention runs on dedicated warps of the same CTAs, and a grid-wide hand-over is a counter in global
+ * memory that is polled only where data crosses SMs.  With the ladder rule (Eq. 2: module m reads
+ * x_{m-2}) every such dependency points two phases back, so the weight stream never stops between
+ * modules; with the standard rule (Eq. 1) each phase waits for the one before.  on = 0 selects the
+ * multi-kernel schedule configured by ladder_model_set_schedule (also used automatically for batch > 8
+ * and on devices where the kernel cannot be made resident).  Results are bit-identical either way.
+ * ladder_model_persistent_active returns 1 when decode steps of batch <= 8 take this path. */
+ladder_status_t ladder_model_set_persistent(ladder_model_t* m, int32_t on);
+int32_t ladder_model_persistent_active(const ladder_model_t* m);
+
 /* With two streams, the GEMMs of a ladder layer's attention module and MLP module can be run side by side on
  * disjoint sets of SMs (each GEMM is a persistent kernel that claims its work dynamically, so it runs
  * on any number of CTAs).  sms_attention_stream: -1 = no split, every GEMM launches on all SMs (default:

@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libladder.so")
 
 EXPORTS = [
-    "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_model_set_sm_split",
+    "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_model_set_sm_split", "ladder_model_set_persistent", "ladder_model_persistent_active",
     "ladder_prefill",
     "ladder_decode_step", "ladder_decode_step_host", "ladder_prefill_host", "ladder_set_position",
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
@@ -75,6 +75,9 @@ def lib() -> C.CDLL:
                                           C.POINTER(C.c_void_p)]
         L.ladder_model_set_schedule.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32]
         L.ladder_model_set_sm_split.argtypes = [C.c_void_p, C.c_int32]
+        L.ladder_model_set_persistent.argtypes = [C.c_void_p, C.c_int32]
+        L.ladder_model_persistent_active.argtypes = [C.c_void_p]
+        L.ladder_model_persistent_active.restype = C.c_int32
         L.ladder_prefill.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32, C.c_int32,
                                      C.POINTER(ladder_outputs_t), C.c_void_p]
         L.ladder_decode_step.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32,
@@ -197,6 +200,12 @@ class Model:
 
     def set_schedule(self, n_streams: int = 2, use_graph: bool = True, use_pdl: bool = True):
         _check(lib().ladder_model_set_schedule(self.h, n_streams, int(use_graph), int(use_pdl)), self.h)
+
+    def set_persistent(self, on: bool = True):
+        _check(lib().ladder_model_set_persistent(self.h, int(on)), self.h)
+
+    def persistent_active(self) -> bool:
+        return bool(lib().ladder_model_persistent_active(self.h))
 
     def set_sm_split(self, sms_attention_stream: int = 0):
         _check(lib().ladder_model_set_sm_split(self.h, sms_attention_stream), self.h)

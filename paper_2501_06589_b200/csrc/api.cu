@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <map>
 #include <string>
 #include <vector>
 
@@ -74,6 +75,15 @@ struct ladder_model {
   cudaGraphExec_t graph_exec = nullptr;
   GraphKey graph_key;
   int64_t graph_kernels = 0;
+  // persistent layer-stack kernel (one cooperative launch per decode step, batch <= 8)
+  bool stack_ok = false;   // usable on this device
+  int use_stack = 1;
+  GraphKey stack_key;      // what the uploaded phase list was built for
+  bool stack_built = false;
+  StackPhase* d_phases = nullptr;
+  StackAttn* d_attn = nullptr;
+  int32_t* d_counters = nullptr;
+  int n_phases = 0, n_attn = 0, n_counters = 0, cap_counters = 0;
   // state
   int host_len = 0;
   int64_t launches = 0;
@@ -460,6 +470,269 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
   return err;
 }
 
+
+// --------------------------------------------------------------------------- persistent layer stack
+// Builds the phase list of one decode step for the persistent kernel: the GEMMs of every layer in the
+// order the residual rule allows (ladder layer: QKV, gate/up, Wo, down -- the MLP's first GEMM does
+// not depend on the attention module; standard layer: QKV, Wo, gate/up, down), the attention nodes,
+// and for every access to a buffer another phase touches the counters it has to wait for:
+// read-after-write on the last writer, write-after-read on every reader since, write-after-write.
+struct StackBuilder {
+  struct Buf {
+    int writer = -1;
+    std::vector<int> readers;
+  };
+  std::map<const void*, Buf> bufs;
+  std::vector<int> need;  // need[counter] = value that means "complete" (-1: not usable as a dependency)
+  bool overflow = false;
+
+  int counter(int complete_at) {
+    need.push_back(complete_at);
+    return static_cast<int>(need.size()) - 1;
+  }
+  static void push(std::vector<int>& v, int c) {
+    if (c >= 0 && std::find(v.begin(), v.end(), c) == v.end()) v.push_back(c);
+  }
+  void raw(const void* b, std::vector<int>& deps) {
+    if (b) push(deps, bufs[b].writer);
+  }
+  void war(const void* b, std::vector<int>& deps) {
+    if (!b) return;
+    Buf& s = bufs[b];
+    for (int r : s.readers) push(deps, r);
+    push(deps, s.writer);
+  }
+  void did_read(const void* b, int me) {
+    if (b) push(bufs[b].readers, me);
+  }
+  void did_write(const void* b, int me) {
+    if (!b) return;
+    Buf& s = bufs[b];
+    s.readers.clear();
+    s.writer = me;
+  }
+  void emit(const std::vector<int>& deps, int self, int* n_out, int* dep_out, int* need_out) {
+    int n = 0;
+    for (int c : deps) {
+      if (c == self) continue;
+      if (n == kStackMaxDeps || need[c] < 0) {
+        overflow = true;
+        return;
+      }
+      dep_out[n] = c;
+      need_out[n] = need[c];
+      ++n;
+    }
+    *n_out = n;
+  }
+};
+
+// Returns false (with a reason) when this step cannot be expressed; the caller then uses the
+// multi-kernel schedule.
+bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, float* logits, std::vector<StackPhase>& phases,
+                 std::vector<StackAttn>& attn, int* n_counters) {
+  const ladder_config_t& c = m->cfg;
+  const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff;
+  const size_t layer_elems = static_cast<size_t>(c.max_batch) * Hkv * c.max_seq_len * Dh;
+  if (m->attn_splits > 1024) return false;  // merge weights are held in shared memory
+  StackBuilder sb;
+  phases.clear();
+  attn.clear();
+
+  auto add_gemm = [&](SmallMParams p, const void* act_buf, const void* add_buf, const void* out0, const void* out1,
+                      const void* out2) {
+    StackPhase P = {};
+    p.batch = batch;
+    p.status = m->status;
+    P.p = p;
+    P.n_units = p.N / 8;
+    P.nchunk = (p.K + 2047) / 2048;
+    P.work_idx = sb.counter(-1);
+    P.done_idx = sb.counter(P.n_units);
+    P.sched = make_schedule(P.n_units, m->sm_count);
+    std::vector<int> ad, ed;
+    sb.raw(act_buf, ad);
+    sb.raw(add_buf, ed);
+    sb.war(out0, ed);
+    sb.war(out1, ed);
+    sb.war(out2, ed);
+    sb.emit(ad, P.done_idx, &P.n_act_deps, P.act_dep, P.act_need);
+    sb.emit(ed, P.done_idx, &P.n_epi_deps, P.epi_dep, P.epi_need);
+    sb.did_read(act_buf, P.done_idx);
+    sb.did_read(add_buf, P.done_idx);
+    sb.did_write(out0, P.done_idx);
+    sb.did_write(out1, P.done_idx);
+    sb.did_write(out2, P.done_idx);
+    phases.push_back(P);
+  };
+
+  Router rt;
+  int prev_merge = -1;
+  for (int l = 0; l < c.n_layers; ++l) {
+    const bool lad = m->is_ladder[l] != 0;
+    const Router::Route ra = rt.next(lad, 2 * l + 1);
+    const Router::Route rm = rt.next(lad, 2 * l + 2);
+    __nv_bfloat16* kc = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
+    __nv_bfloat16* vc = static_cast<__nv_bfloat16*>(cache->v) + l * layer_elems;
+
+    auto qkv = [&]() {
+      SmallMParams p = {};
+      p.W = m->w_qkv[l];
+      p.N = (Hq + 2 * Hkv) * Dh;
+      p.K = d;
+      p.act = m->R[ra.in];
+      p.act_mode = ACT_F32_NORM;
+      p.gain = m->attn_norm[l];
+      p.eps = c.rms_eps;
+      p.epi_mode = EPI_QKV_ROPE;
+      p.qkv.q_out_f32 = m->q_f32;
+      p.qkv.k_cache = kc;
+      p.qkv.v_cache = vc;
+      p.qkv.seq_lens = cache->seq_lens;
+      p.qkv.rope = m->rope;
+      p.qkv.n_q_heads = Hq;
+      p.qkv.n_kv_heads = Hkv;
+      p.qkv.head_dim = Dh;
+      p.qkv.max_seq_len = c.max_seq_len;
+      add_gemm(p, m->R[ra.in], nullptr, m->q_f32, kc, vc);
+      // the attention of this layer, on the attention warps
+      StackAttn A = {};
+      A.a.q = m->q_f32;
+      A.a.k = kc;
+      A.a.v = vc;
+      A.a.kv_len = cache->seq_lens;
+      A.a.kv_len_offset = 1;
+      A.a.batch = batch;
+      A.a.n_q_heads = Hq;
+      A.a.n_kv_heads = Hkv;
+      A.a.head_dim = Dh;
+      A.a.max_seq_len = c.max_seq_len;
+      A.a.n_splits = m->attn_splits;
+      A.a.max_len = c.max_seq_len;
+      A.a.scratch = m->attn_scratch;
+      A.a.o = m->o_dec;
+      A.split_done = sb.counter(-1);
+      A.merge_done = sb.counter(batch * Hq);
+      std::vector<int> sd, md;
+      sb.raw(m->q_f32, sd);
+      sb.raw(kc, sd);
+      sb.raw(vc, sd);
+      StackBuilder::push(sd, prev_merge);  // the partials of the previous layer have been merged
+      sb.war(m->o_dec, md);
+      sb.emit(sd, A.merge_done, &A.n_deps, A.dep, A.need);
+      sb.emit(md, A.merge_done, &A.n_mdeps, A.mdep, A.mneed);
+      sb.did_read(m->q_f32, A.merge_done);
+      sb.did_read(kc, A.merge_done);
+      sb.did_read(vc, A.merge_done);
+      sb.did_write(m->o_dec, A.merge_done);
+      prev_merge = A.merge_done;
+      attn.push_back(A);
+    };
+    auto wo = [&]() {
+      SmallMParams p = {};
+      p.W = m->w_o[l];
+      p.N = d;
+      p.K = Hq * Dh;
+      p.act = m->o_dec;
+      p.act_mode = ACT_F32;
+      p.epi_mode = EPI_RESID;
+      p.addend = m->R[ra.add];
+      p.out = m->R[ra.dst];
+      add_gemm(p, m->o_dec, m->R[ra.add], m->R[ra.dst], nullptr, nullptr);
+    };
+    auto gate_up = [&]() {
+      SmallMParams p = {};
+      p.W = m->w_gate_up[l];
+      p.N = 2 * F;
+      p.K = d;
+      p.act = m->R[rm.in];
+      p.act_mode = ACT_F32_NORM;
+      p.gain = m->mlp_norm[l];
+      p.eps = c.rms_eps;
+      p.epi_mode = EPI_SWIGLU;
+      p.out = m->h_dec;
+      add_gemm(p, m->R[rm.in], nullptr, m->h_dec, nullptr, nullptr);
+    };
+    auto down = [&]() {
+      SmallMParams p = {};
+      p.W = m->w_down[l];
+      p.N = d;
+      p.K = F;
+      p.act = m->h_dec;
+      p.act_mode = ACT_F32;
+      p.epi_mode = EPI_RESID;
+      p.addend = m->R[rm.add];
+      p.out = m->R[rm.dst];
+      add_gemm(p, m->h_dec, m->R[rm.add], m->R[rm.dst], nullptr, nullptr);
+    };
+    // The MLP module of a ladder layer reads x_{m-2}, which exists before the attention module of the
+    // same layer has produced anything -- unless this is the first ladder layer after a standard one,
+    // where x_{m-2} is the attention module's own input (still fine: it is not its output).
+    const bool mlp_independent = lad && rm.in != ra.dst;
+    qkv();
+    if (mlp_independent) {
+      gate_up();
+      wo();
+    } else {
+      wo();
+      gate_up();
+    }
+    down();
+  }
+  {
+    SmallMParams h = {};
+    h.W = m->lm_head;
+    h.N = c.vocab_size;
+    h.K = d;
+    h.act = m->R[rt.cur];
+    h.act_mode = ACT_F32_NORM;
+    h.gain = m->final_norm;
+    h.eps = c.rms_eps;
+    h.epi_mode = EPI_PLAIN;
+    h.out = logits;
+    add_gemm(h, m->R[rt.cur], nullptr, logits, nullptr, nullptr);
+  }
+  *n_counters = static_cast<int>(sb.need.size());
+  return !sb.overflow && static_cast<int>(phases.size()) <= kStackMaxPhases;
+}
+
+// One decode step through the persistent kernel: embedding, zeroed counters, the layer stack, head outputs.
+cudaError_t enqueue_decode_stack(ladder_model* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int batch,
+                                 const ladder_outputs_t* out, cudaStream_t st, int64_t* n_kernels) {
+  const ladder_config_t& c = m->cfg;
+  const int d = c.d_model;
+  float* logits = (out && out->logits) ? out->logits : m->logits_ws;
+  cudaError_t e = launch_embed(d_tokens, m->tok_embedding, batch, d, c.vocab_size, m->R[0], m->status, st, false);
+  if (e == cudaSuccess) e = cudaMemsetAsync(m->d_counters, 0, static_cast<size_t>(m->n_counters) * sizeof(int32_t), st);
+  StackParams sp = {};
+  sp.phases = m->d_phases;
+  sp.n_phases = m->n_phases;
+  sp.attn = m->d_attn;
+  sp.n_attn = m->n_attn;
+  sp.counters = m->d_counters;
+  sp.status = m->status;
+  sp.batch = batch;
+  if (e == cudaSuccess) e = launch_decode_stack(sp, m->sm_count, st);
+  int64_t k = 2;
+  // the final hidden state is the input of the last phase (the LM head)
+  Router rt;
+  for (int l = 0; l < c.n_layers; ++l) {
+    rt.next(m->is_ladder[l] != 0, 2 * l + 1);
+    rt.next(m->is_ladder[l] != 0, 2 * l + 2);
+  }
+  if (out && out->final_hidden) {
+    if (e == cudaSuccess)
+      e = launch_rmsnorm_f32(m->R[rt.cur], m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, st, false);
+    ++k;
+  }
+  if (e == cudaSuccess)
+    e = launch_argmax_advance(logits, batch, c.vocab_size, out ? out->next_tokens : nullptr, cache->seq_lens, 1, -1, st,
+                              false);
+  ++k;
+  *n_kernels = k;
+  return e;
+}
+
 void drop_graph(ladder_model* m) {
   if (m->graph_exec) cudaGraphExecDestroy(m->graph_exec);
   m->graph_exec = nullptr;
@@ -538,10 +811,12 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   int smem_optin = 0;
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   if (e == cudaSuccess) e = kernels_ready();
+  if (e == cudaSuccess) e = decode_stack_init(m->sm_count, &m->stack_ok);
   if (e != cudaSuccess) {
     delete m;
     return fail(nullptr, LADDER_ERR_CUDA, std::string("device query: ") + cudaGetErrorString(e));
   }
+  if (4 * L + 1 > kStackMaxPhases) m->stack_ok = false;
   if (static_cast<size_t>(smem_optin) < smallm_gemm_smem_bytes(c.max_batch)) {
     delete m;
     return fail(nullptr, LADDER_ERR_UNSUPPORTED, "device has too little shared memory per block (needs sm_100-class)");
@@ -578,6 +853,10 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
       if (cudaMemset(m->work_slots, 0, 2 * m->n_work_slots * sizeof(int32_t)) != cudaSuccess) oom = true;
     }
   }
+  m->cap_counters = 2 * (4 * L + 1) + 2 * L;
+  A(dev_alloc(&m->d_phases, static_cast<size_t>(4 * L + 1)));
+  A(dev_alloc(&m->d_attn, static_cast<size_t>(L)));
+  A(dev_alloc(&m->d_counters, static_cast<size_t>(m->cap_counters)));
   A(dev_alloc(&m->logits_ws, MB * c.vocab_size));
   A(dev_alloc(&m->last_x, MB * d));
   m->n_lo = MP * d;
@@ -636,7 +915,7 @@ ladder_status_t ladder_destroy(ladder_model_t* m) {
   if (m->ev_join) cudaEventDestroy(m->ev_join);
   if (m->side) cudaStreamDestroy(m->side);
   if (m->cap) cudaStreamDestroy(m->cap);
-  void* bufs[] = {m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
+  void* bufs[] = {m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
                   m->n_pf, m->q_pf,  m->o_pf,  m->h_pf,  m->rope,  m->status,       m->tok_tmp,   m->next_tmp};
   for (void* b : bufs)
     if (b) cudaFree(b);
@@ -653,6 +932,14 @@ ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, 
   drop_graph(m);
   return LADDER_OK;
 }
+
+ladder_status_t ladder_model_set_persistent(ladder_model_t* m, int32_t on) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  m->use_stack = on ? 1 : 0;
+  return LADDER_OK;
+}
+
+int32_t ladder_model_persistent_active(const ladder_model_t* m) { return (m && m->use_stack && m->stack_ok) ? 1 : 0; }
 
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream) {
   if (!m) return LADDER_ERR_INVALID_ARG;
@@ -713,6 +1000,42 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
   if (out && out->all_hidden) return fail(m, LADDER_ERR_INVALID_ARG, "all_hidden is a prefill-only output");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const bool two = m->n_streams == 2;
+
+  if (m->use_stack && m->stack_ok && batch <= 8) {
+    GraphKey key;
+    key.batch = batch;
+    key.k = cache->k;
+    key.v = cache->v;
+    key.lens = cache->seq_lens;
+    key.o_logits = out ? out->logits : nullptr;
+    if (!m->stack_built || !(key == m->stack_key)) {
+      std::vector<StackPhase> ph;
+      std::vector<StackAttn> at;
+      int nc = 0;
+      float* logits = (out && out->logits) ? out->logits : m->logits_ws;
+      if (!build_stack(m, cache, batch, logits, ph, at, &nc) || nc > m->cap_counters ||
+          static_cast<int>(ph.size()) > 4 * m->cfg.n_layers + 1 || static_cast<int>(at.size()) > m->cfg.n_layers) {
+        m->stack_ok = false;  // not expressible: use the multi-kernel schedule from now on
+      } else {
+        // the previous step may still be reading the old lists
+        CK(m, cudaStreamSynchronize(st));
+        CK(m, cudaMemcpy(m->d_phases, ph.data(), ph.size() * sizeof(StackPhase), cudaMemcpyHostToDevice));
+        CK(m, cudaMemcpy(m->d_attn, at.data(), at.size() * sizeof(StackAttn), cudaMemcpyHostToDevice));
+        m->n_phases = static_cast<int>(ph.size());
+        m->n_attn = static_cast<int>(at.size());
+        m->n_counters = nc;
+        m->stack_key = key;
+        m->stack_built = true;
+      }
+    }
+    if (m->stack_ok) {
+      int64_t k = 0;
+      CK(m, enqueue_decode_stack(m, cache, d_tokens, batch, out, st, &k));
+      m->launches += k;
+      m->host_len += 1;
+      return LADDER_OK;
+    }
+  }
 
   if (!m->use_graph) {
     int64_t k = 0;

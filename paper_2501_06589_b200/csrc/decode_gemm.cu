@@ -31,6 +31,7 @@
 // first ring fill), so under programmatic dependent launch the weight stream does not drain
 // between kernels.
 #include "common.cuh"
+#include "decode_schedule.h"
 #include "kernels.h"
 #include "smallm_epilogue.cuh"
 
@@ -50,7 +51,7 @@ constexpr int STAGE_BYTES = 8 * PITCH;
 constexpr int STAGES = 4;
 constexpr int ACT_BYTES = 8 * PITCH;
 constexpr int RG_MAX = 5;           // 16-row groups per batch at most (10 units)
-constexpr int UMAX = 2 * RG_MAX;    // 8-row units per batch at most
+static_assert(2 * RG_MAX == kSchedUnitsMax, "schedule and tile geometry disagree");
 constexpr int SPW = TK / 32 / 4;    // 32-wide K slabs per consumer warp per chunk
 constexpr int RED_FLOATS = 4 * RG_MAX * 4 * 32;
 constexpr int QDEPTH = 16;          // claimed-item queue, producer -> consumers and finishers
@@ -66,54 +67,6 @@ static_assert(SMEM <= 190 * 1024, "leave room for a co-resident attention CTA");
 struct F8 {
   float4 a, b;
 };
-
-// Batch schedule: phase i hands out count[i] claims of size[i] consecutive 8-row units.  Fixed per
-// launch (built on the host), so claiming a batch is a single atomicAdd on a claim index.
-constexpr int kMaxPhases = 24;
-struct Schedule {
-  int n;
-  int count[kMaxPhases];
-  int size[kMaxPhases];
-};
-
-// A batch costs a fixed latency per K chunk (activation hand-over, fragment hoisting) and re-reads
-// the activations, so small batches are expensive; but equal static shares make every launch wait
-// for the slowest SM.  Hence:
-//   * little work per CTA (share <= UMAX units): one round of near-equal batches, each done in a
-//     single pass over K (measured faster than a 70 % + 30 % split, whose second pass is too short);
-//   * more: rounds of 8-unit batches while a CTA's share of what is left is large, then one round
-//     of ~70 % of the remaining share, then 2-unit batches with which the fast SMs pick up the
-//     slack of the slow ones (guided self-scheduling, evaluated ahead of time).
-Schedule make_schedule(int n_units, int grid, int K) {
-  (void)K;
-  Schedule sc = {};
-  auto push = [&](int count, int size) {
-    if (count > 0 && size > 0 && sc.n < kMaxPhases) {
-      sc.count[sc.n] = count;
-      sc.size[sc.n] = size;
-      ++sc.n;
-    }
-  };
-  int rem = n_units;
-  if (rem <= UMAX * grid) {
-    const int hi = (rem + grid - 1) / grid, n_hi = rem - (hi - 1) * grid;  // n_hi batches of hi, rest hi-1
-    push(n_hi, hi);
-    push(grid - n_hi, hi - 1);
-    return sc;
-  }
-  while (rem > 0 && sc.n < kMaxPhases - 2) {
-    const double share = static_cast<double>(rem) / grid;
-    int size;
-    if (share >= 12.0) size = 8;
-    else if (share >= 4.0) size = (static_cast<int>(share * 0.7) & ~1) > 8 ? 8 : (static_cast<int>(share * 0.7) & ~1);
-    else break;
-    push(grid, size);
-    rem -= grid * size;
-  }
-  push(rem / 2, 2);
-  push(rem & 1, 1);
-  return sc;
-}
 
 // bounded spin on a shared-memory counter written by another warp of this CTA
 __device__ __forceinline__ bool wait_counter_gt(const volatile int* ctr, int n) {
@@ -554,7 +507,7 @@ cudaError_t launch_small(const SmallMParams& p, cudaStream_t stream, bool pdl, i
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = pdl ? 1 : 0;
-  const Schedule sc = make_schedule(p.N >> 3, grid, p.K);
+  const Schedule sc = make_schedule(p.N >> 3, grid);
   return cudaLaunchKernelEx(&cfg, kern, p, sc);
 }
 

@@ -1,0 +1,956 @@
+// Persistent layer-stack kernel of the decode step (batch <= 8).
+//
+// One cooperative launch, one CTA per SM, runs EVERY weight-streaming GEMM of a decode step (QKV,
+// Wo, gate/up, down of each layer and the LM head) plus the attention of every layer.  The GEMMs are
+// "phases" walked in a fixed order by all CTAs; inside a phase the 8-row units of W are claimed in
+// batches through an atomic counter, exactly as in the per-GEMM kernel.  What used to be a kernel
+// boundary is a counter in global memory (units finished per phase): a reader polls it, with an
+// acquire load and a time limit, only before it touches data another SM produced.
+//
+// Why: the weight stream of a phase depends on nothing, so the producer warp runs through phase
+// after phase and the TMA ring never drains, whatever the consumers are waiting for.  With the
+// ladder recurrence (Eq. 2) the input of a module is x_{m-2}: in the order
+//     QKV_l, gate/up_l, Wo_l, down_l, QKV_{l+1}, ...
+// every dependency points at least two phases back, so the polls succeed at once, and the
+// attention of layer l (dedicated warps of the same CTAs) has the whole gate/up phase to finish
+// before Wo_l needs it.  This is the paper's decoupling of a module from its predecessor's
+// synchronisation, applied to the grid-wide hand-over inside one GPU instead of the all-reduce
+// between GPUs.  Standard-residual layers (Eq. 1) run QKV, Wo, gate/up, down with every phase
+// depending on the one before: correct, but the consumers stall at each hand-over.
+//
+// Warp roles (512 threads, four warpgroups so that registers can be moved between them):
+//   warp 0        producer: claims batches, publishes them in a shared-memory queue, streams the
+//                 weights as [8 rows x 2048 k] tiles (eight 4 KB bulk async copies) into a 4-stage ring
+//   warps 1-3     finishers: K-split reduction, 1/rms, epilogue (residual add / SwiGLU / rotary + KV
+//                 append), then publish the finished units (fence + release add)
+//   warps 4-7     consumers: mma.sync m16n8k16 with the weights as the A operand (see decode_gemm.cu)
+//   warps 8-11    stagers: fp32 activations -> bf16 hi (+ lo) MMA operands, one chunk ahead; RMSNorm
+//                 sum of squares on the fly
+//   warps 12-15   attention: split-KV partials (64 keys x head group x sequence per unit), then the
+//                 log-sum-exp merge, units dealt round-robin over the CTAs
+// Data produced inside the launch is always read through L2 (ld.global.cg / acquire), never through
+// the non-coherent L1 path.  Every wait is bounded (0.25 s) and also gives up when another CTA has
+// reported a timeout in the device status word, so a protocol error ends the launch quickly with
+// LADDER_DEV_TIMEOUT set instead of hanging the device.
+#include "common.cuh"
+#include "kernels.h"
+#include "smallm_epilogue.cuh"
+
+namespace ladder {
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kFin = 96;  // finisher threads
+constexpr int kAux = 128;  // attention threads
+constexpr int TK = 2048;   // K elements per chunk (4 KB of a weight row)
+constexpr int PITCH = TK * 2 + 64;
+constexpr int STAGE_BYTES = 8 * PITCH;
+constexpr int STAGES = 4;
+constexpr int ACT_BYTES = 8 * PITCH;
+constexpr int RG_MAX = 5;
+static_assert(2 * RG_MAX == kSchedUnitsMax, "schedule and tile geometry disagree");
+constexpr int SPW = TK / 32 / 4;
+constexpr int RED_FLOATS = 4 * RG_MAX * 4 * 32;
+constexpr int QDEPTH = 16;
+constexpr int NORM_RING = 4;  // the stagers run at most three normalised phases ahead of the finishers
+constexpr uint64_t kTimeoutNs = 250000000ull;
+constexpr int kChunk = 64;         // keys per attention unit
+constexpr int kMaxSplits = 1024;   // merge weights held in shared memory
+
+constexpr int OFF_ACT = STAGES * STAGE_BYTES;
+constexpr int OFF_SSQ = OFF_ACT + ACT_BYTES;                 // [NORM_RING][4 stager warps][8]
+constexpr int OFF_RED = OFF_SSQ + NORM_RING * 4 * 8 * 4;
+constexpr int OFF_RSTD = OFF_RED + 2 * RED_FLOATS * 4;
+constexpr int N_BARS = 2 * STAGES + 2 + NORM_RING + 4;       // full, empty, act_free, act_full, norm_ready[], red_full[2], red_free[2]
+constexpr int OFF_BAR = OFF_RSTD + 8 * 4;
+constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;               // queue[QDEPTH], q_head, dead flag
+constexpr int OFF_FINP = OFF_MISC + 128;                     // the finishers' copy of the phase parameters
+constexpr int FINP_BYTES = 256;
+static_assert(sizeof(SmallMParams) <= FINP_BYTES, "phase parameter copy too small");
+static_assert((QDEPTH + 2) * 4 <= 128, "queue area too small");
+constexpr int OFF_AUX = OFF_FINP + FINP_BYTES;
+constexpr int AUX_PS = 4 * 8 * 16 * 4;
+constexpr int AUX_RED = 4 * 8 * 128 * 4;
+static_assert(AUX_RED >= kMaxSplits * 4, "merge weights do not fit");
+constexpr int AUX_MLS = 4 * 8 * 2 * 4;
+constexpr int AUX_MISC = 128;  // prefix of live splits per sequence [9], merge reductions [8]
+constexpr int SMEM = OFF_AUX + AUX_PS + AUX_RED + AUX_MLS + AUX_MISC + 128;
+static_assert(SMEM <= 227 * 1024, "shared memory budget");
+
+// registers per thread after the warpgroups have traded (launch allocation: 128 each)
+constexpr int REGS_WG0 = 72, REGS_CONS = 176, REGS_STAGE = 120, REGS_AUX = 144;
+static_assert(REGS_WG0 + REGS_CONS + REGS_STAGE + REGS_AUX <= 4 * 128, "register pool exceeded");
+
+struct F8 {
+  float4 a, b;
+};
+
+// Moves this warpgroup's per-thread register allocation from the launch value (128) to N: a release
+// when N is smaller, a (blocking) request when it is larger.  Every warpgroup calls it exactly once,
+// unconditionally, and the four targets add up to the launch total, so the requests are always met.
+constexpr int kLaunchRegs = 128;
+template <int N>
+__device__ __forceinline__ void reg_set() {
+  static_assert(N % 8 == 0 && N >= 24 && N <= 256, "register count out of range");
+  if constexpr (N > kLaunchRegs) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+  else if constexpr (N < kLaunchRegs) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+__device__ __forceinline__ int ld_acquire(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_add(int32_t* p, int v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool aborted(const int32_t* status) {
+  return (*reinterpret_cast<const volatile int32_t*>(status) & LADDER_DEV_TIMEOUT) != 0;
+}
+__device__ __forceinline__ void bar_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+// barrier among `count` threads that also ANDs a predicate: every participant gets the same answer,
+// so the decision to leave a role after a failed wait is taken by all its threads together
+__device__ __forceinline__ bool bar_and(int id, int count, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 p, %1, 0;\n\t"
+      "bar.red.and.pred q, %2, %3, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r)
+      : "r"(static_cast<uint32_t>(pred)), "r"(id), "r"(count)
+      : "memory");
+  return r != 0;
+}
+
+// ---- bounded waits; all give up early when another CTA has reported a timeout
+__device__ __forceinline__ bool wait_mbar(uint64_t* bar, uint32_t parity, const int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t i = 1;; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
+  }
+}
+__device__ __forceinline__ bool wait_counter_gt(const volatile int* ctr, int n, const int32_t* status) {
+  if (*ctr > n) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t i = 1;; ++i) {
+    if (*ctr > n) return true;
+    if ((i & 255u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
+  }
+}
+__device__ __forceinline__ bool wait_global_ge(const int32_t* ctr, int need, const int32_t* status) {
+  if (ld_acquire(ctr) >= need) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t i = 1;; ++i) {
+    if (ld_acquire(ctr) >= need) return true;
+    if ((i & 31u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
+  }
+}
+// lane i of the calling warp polls dependency i; the warp agrees on the outcome
+__device__ __forceinline__ bool wait_deps(const int* dep, const int* need, int n, const int32_t* counters,
+                                          const int32_t* status, int lane) {
+  bool ok = true;
+  if (lane < n) ok = wait_global_ge(counters + __ldg(dep + lane), __ldg(need + lane), status);
+  return __all_sync(0xffffffffu, ok);
+}
+
+// queue item: phase (10 bits) | first unit (17 bits) | units (4 bits)
+__device__ __forceinline__ int item_pack(int ph, int u0, int nu) { return (ph << 21) | (u0 << 4) | nu; }
+
+// ------------------------------------------------------------------------------------ attention units
+// One split unit: 64 keys x GT query heads sharing a kv head x one sequence, 4 warps (16 keys each).
+// Same arithmetic as decode_attention_kernel; loads go through L2 because q and the newest key/value
+// row were written by other SMs earlier in this launch.
+template <int GT, int DH>
+__device__ __forceinline__ void attn_split_unit(const float* q, const __nv_bfloat16* Kc, const __nv_bfloat16* Vc,
+                                                int n_q_heads, int n_kv_heads, int max_seq_len, int stride_splits,
+                                                float* scratch, int b, int split, int hg, int L, float* ps_, float* red_,
+                                                float* mls_, int at) {
+  constexpr int DPL = DH / 32;
+  constexpr int KJ = DH / 32;
+  const int warp = at >> 5, lane = at & 31;
+  const int g = lane >> 2, tig = lane & 3;
+  const int head0 = hg * GT;
+  const int group = n_q_heads / n_kv_heads;
+  const int kvh = head0 / group;
+  const size_t kv_base = (static_cast<size_t>(b) * n_kv_heads + kvh) * max_seq_len * DH;
+  const __nv_bfloat16* K = Kc + kv_base;
+  const __nv_bfloat16* V = Vc + kv_base;
+  const int kw0 = split * kChunk + warp * 16;
+  const float scale = rsqrtf(static_cast<float>(DH));
+  float* ps = ps_ + warp * GT * 16;     // [GT][16]
+  float* red = red_;                    // [4][GT][DH]
+  float* mls = mls_;                    // [4][GT][2]
+
+  uint4 kf[2][KJ];
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    const int key = kw0 + nt * 8 + g;
+#pragma unroll
+    for (int j = 0; j < KJ; ++j)
+      kf[nt][j] = key < L ? __ldcg(reinterpret_cast<const uint4*>(K + static_cast<size_t>(key) * DH + j * 32 + tig * 8))
+                          : make_uint4(0, 0, 0, 0);
+  }
+  uint32_t vr[16][DPL / 2];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int key = kw0 + i;
+    if (DPL == 4) {
+      const uint2 u = key < L ? __ldcg(reinterpret_cast<const uint2*>(V + static_cast<size_t>(key) * DH + lane * DPL))
+                              : make_uint2(0, 0);
+      vr[i][0] = u.x;
+      vr[i][DPL / 2 - 1] = u.y;
+    } else {
+      vr[i][0] = key < L ? __ldcg(reinterpret_cast<const unsigned int*>(V + static_cast<size_t>(key) * DH + lane * DPL))
+                         : 0u;
+    }
+  }
+  uint32_t qa[KJ][2][2], ql[KJ][2][2];
+#pragma unroll
+  for (int j = 0; j < KJ; ++j)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float4 v = make_float4(0, 0, 0, 0);
+      if (g < GT)
+        v = __ldcg(reinterpret_cast<const float4*>(q + (static_cast<size_t>(b) * n_q_heads + head0 + g) * DH + j * 32 +
+                                                   tig * 8 + h * 4));
+      qa[j][h][0] = pack_bf16x2(v.x, v.y);
+      qa[j][h][1] = pack_bf16x2(v.z, v.w);
+      ql[j][h][0] = pack_bf16x2(v.x - bf16_lo(qa[j][h][0]), v.y - bf16_hi(qa[j][h][0]));
+      ql[j][h][1] = pack_bf16x2(v.z - bf16_lo(qa[j][h][1]), v.w - bf16_hi(qa[j][h][1]));
+    }
+
+  float c[2][4];
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+#pragma unroll
+    for (int j = 0; j < KJ; ++j) {
+      mma_bf16_16816(c[nt], qa[j][0][0], 0u, qa[j][0][1], 0u, kf[nt][j].x, kf[nt][j].y);
+      mma_bf16_16816(c[nt], qa[j][1][0], 0u, qa[j][1][1], 0u, kf[nt][j].z, kf[nt][j].w);
+      mma_bf16_16816(c[nt], ql[j][0][0], 0u, ql[j][0][1], 0u, kf[nt][j].x, kf[nt][j].y);
+      mma_bf16_16816(c[nt], ql[j][1][0], 0u, ql[j][1][1], 0u, kf[nt][j].z, kf[nt][j].w);
+    }
+  }
+  float sv[4];
+  float m = -INFINITY;
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int key = kw0 + nt * 8 + 2 * tig + e;
+      sv[nt * 2 + e] = key < L ? c[nt][e] * scale : -INFINITY;
+      m = fmaxf(m, sv[nt * 2 + e]);
+    }
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+  float l = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    sv[i] = (m == -INFINITY) ? 0.f : __expf(sv[i] - m);
+    l += sv[i];
+  }
+  l += __shfl_xor_sync(0xffffffffu, l, 1);
+  l += __shfl_xor_sync(0xffffffffu, l, 2);
+  if (g < GT) {
+    *reinterpret_cast<float2*>(&ps[g * 16 + 2 * tig]) = make_float2(sv[0], sv[1]);
+    *reinterpret_cast<float2*>(&ps[g * 16 + 8 + 2 * tig]) = make_float2(sv[2], sv[3]);
+    if (tig == 0) {
+      mls[(warp * GT + g) * 2 + 0] = m;
+      mls[(warp * GT + g) * 2 + 1] = l;
+    }
+  }
+  __syncwarp();
+
+  float acc[GT][DPL];
+#pragma unroll
+  for (int h = 0; h < GT; ++h)
+#pragma unroll
+    for (int d = 0; d < DPL; ++d) acc[h][d] = 0.f;
+#pragma unroll
+  for (int i4 = 0; i4 < 4; ++i4) {
+    float4 pw[GT];
+#pragma unroll
+    for (int h = 0; h < GT; ++h) pw[h] = *reinterpret_cast<const float4*>(&ps[h * 16 + i4 * 4]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int i = i4 * 4 + e;
+      float v[DPL];
+      v[0] = bf16_lo(vr[i][0]);
+      v[1] = bf16_hi(vr[i][0]);
+      if (DPL == 4) {
+        v[DPL - 2] = bf16_lo(vr[i][DPL / 2 - 1]);
+        v[DPL - 1] = bf16_hi(vr[i][DPL / 2 - 1]);
+      }
+#pragma unroll
+      for (int h = 0; h < GT; ++h) {
+        const float w = e == 0 ? pw[h].x : (e == 1 ? pw[h].y : (e == 2 ? pw[h].z : pw[h].w));
+#pragma unroll
+        for (int d = 0; d < DPL; ++d) acc[h][d] += w * v[d];
+      }
+    }
+  }
+#pragma unroll
+  for (int h = 0; h < GT; ++h)
+#pragma unroll
+    for (int d = 0; d < DPL; ++d) red[(warp * GT + h) * DH + lane * DPL + d] = acc[h][d];
+  bar_sync(3, kAux);
+
+  const int stride = DH + 2;
+  for (int idx = at; idx < GT * DH; idx += kAux) {
+    const int h = idx / DH, d = idx % DH;
+    const float m0 = mls[(0 * GT + h) * 2], m1 = mls[(1 * GT + h) * 2], m2 = mls[(2 * GT + h) * 2],
+                m3 = mls[(3 * GT + h) * 2];
+    const float M = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+    float o = 0.f, ls = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float mw = mls[(w * GT + h) * 2];
+      const float f = (mw == -INFINITY) ? 0.f : __expf(mw - M);
+      o += f * red[(w * GT + h) * DH + d];
+      ls += f * mls[(w * GT + h) * 2 + 1];
+    }
+    float* dst = scratch + ((static_cast<size_t>(b) * n_q_heads + head0 + h) * stride_splits + split) * stride;
+    dst[d] = o;
+    if (d == 0) {
+      dst[DH] = M;
+      dst[DH + 1] = ls;
+    }
+  }
+  bar_sync(3, kAux);  // the shared arrays are rewritten by the next unit
+}
+
+// Merge of the live splits of one (sequence, head), in split order (same summation order as
+// decode_attention_merge_kernel).
+template <int DH>
+__device__ __forceinline__ void attn_merge_unit(const float* scratch, int n_q_heads, int stride_splits, int n_splits,
+                                                int b, int h, float* o, float* wgt, float* red_m, float* red_l, int at) {
+  constexpr int stride = DH + 2;
+  const int warp = at >> 5, lane = at & 31;
+  const float* base = scratch + (static_cast<size_t>(b) * n_q_heads + h) * stride_splits * stride;
+  const bool act = at < DH;
+  float m = -INFINITY;
+  if (act)
+    for (int s = at; s < n_splits; s += DH) {
+      wgt[s] = __ldcg(base + s * stride + DH);
+      m = fmaxf(m, wgt[s]);
+    }
+  m = warp_max(m);
+  if (lane == 0) red_m[warp] = m;
+  bar_sync(3, kAux);
+  float M = red_m[0];
+#pragma unroll
+  for (int w = 1; w < DH / 32; ++w) M = fmaxf(M, red_m[w]);
+  float l = 0.f;
+  if (act)
+    for (int s = at; s < n_splits; s += DH) {
+      const float f = (wgt[s] == -INFINITY) ? 0.f : __expf(wgt[s] - M);
+      wgt[s] = f;
+      l += f * __ldcg(base + s * stride + DH + 1);
+    }
+  l = warp_sum(l);
+  if (lane == 0) red_l[warp] = l;
+  bar_sync(3, kAux);
+  float lsum = 0.f;
+#pragma unroll
+  for (int w = 0; w < DH / 32; ++w) lsum += red_l[w];
+  if (act) {
+    float acc = 0.f;
+#pragma unroll 8
+    for (int s = 0; s < n_splits; ++s) acc += wgt[s] * __ldcg(base + s * stride + at);
+    o[(static_cast<size_t>(b) * n_q_heads + h) * DH + at] = lsum > 0.f ? acc / lsum : 0.f;
+  }
+  bar_sync(3, kAux);
+}
+
+template <int DH>
+__device__ __forceinline__ void attn_split_dispatch(int gt, const float* q, const __nv_bfloat16* Kc,
+                                                    const __nv_bfloat16* Vc, int n_q_heads, int n_kv_heads,
+                                                    int max_seq_len, int stride_splits, float* scratch, int b, int split,
+                                                    int hg, int L, float* ps, float* red, float* mls, int at) {
+  switch (gt) {
+    case 8:
+      attn_split_unit<8, DH>(q, Kc, Vc, n_q_heads, n_kv_heads, max_seq_len, stride_splits, scratch, b, split, hg, L, ps,
+                             red, mls, at);
+      break;
+    case 4:
+      attn_split_unit<4, DH>(q, Kc, Vc, n_q_heads, n_kv_heads, max_seq_len, stride_splits, scratch, b, split, hg, L, ps,
+                             red, mls, at);
+      break;
+    case 2:
+      attn_split_unit<2, DH>(q, Kc, Vc, n_q_heads, n_kv_heads, max_seq_len, stride_splits, scratch, b, split, hg, L, ps,
+                             red, mls, at);
+      break;
+    default:
+      attn_split_unit<1, DH>(q, Kc, Vc, n_q_heads, n_kv_heads, max_seq_len, stride_splits, scratch, b, split, hg, L, ps,
+                             red, mls, at);
+      break;
+  }
+}
+
+// ------------------------------------------------------------------------------------ the kernel
+template <bool PACKED>
+__global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackParams sp) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+  uint8_t* ring = smem;
+  uint8_t* act = smem + OFF_ACT;
+  float* ssq_part = reinterpret_cast<float*>(smem + OFF_SSQ);
+  float* red = reinterpret_cast<float*>(smem + OFF_RED);
+  float* rstd_s = reinterpret_cast<float*>(smem + OFF_RSTD);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
+  uint64_t* empty = full + STAGES;
+  uint64_t* act_free = empty + STAGES;
+  uint64_t* act_full = act_free + 1;
+  uint64_t* norm_ready = act_full + 1;        // [NORM_RING] stagers -> finishers
+  uint64_t* red_full = norm_ready + NORM_RING;  // [2] consumers -> finishers
+  uint64_t* red_free = red_full + 2;            // [2] finishers -> consumers
+  int* queue = reinterpret_cast<int*>(smem + OFF_MISC);
+  volatile int* q_head = queue + QDEPTH;
+  int* flag_s = queue + QDEPTH + 1;
+  SmallMParams* finp = reinterpret_cast<SmallMParams*>(smem + OFF_FINP);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int batch = sp.batch;
+  const int32_t* status = sp.status;
+
+  if (tid == 0) {
+    *flag_s = aborted(status) ? 1 : 0;
+    *q_head = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 4);
+    }
+    mbar_init(act_free, 4);
+    mbar_init(act_full, 4);
+    for (int s = 0; s < NORM_RING; ++s) mbar_init(&norm_ready[s], 4);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&red_full[s], 4);
+      mbar_init(&red_free[s], 3);
+    }
+    fence_barrier_init();
+  }
+  __syncthreads();
+  if (*flag_s) return;  // an earlier launch reported a protocol error: do nothing
+
+  if (warp < 4) {
+    reg_set<REGS_WG0>();
+    if (warp == 0) {
+      // ---------------------------------------------------------------- producer
+      const uint64_t pol = l2_policy_evict_first();
+      bool ok = true;
+      int it = 0, n = 0;
+      for (int ph = 0; ph < sp.n_phases && ok; ++ph) {
+        const StackPhase* P = sp.phases + ph;
+        const uint8_t* Wb = reinterpret_cast<const uint8_t*>(P->p.W);
+        const int K = P->p.K, n_units = P->n_units, nchunk = P->nchunk;
+        int32_t* work = sp.counters + P->work_idx;
+        while (ok) {
+          // one claim at a time (claiming ahead would let a CTA hoard batches it cannot start yet)
+          int u0 = 0, nu = 0;
+          if (lane == 0) {
+            int ci = atomicAdd(work, 1), ubase = 0;
+            const int sn = P->sched.n;
+            for (int r = 0; r < sn; ++r) {
+              const int cnt = P->sched.count[r], sz = P->sched.size[r];
+              if (ci < cnt) {
+                u0 = ubase + ci * sz;
+                nu = min(sz, n_units - u0);
+                break;
+              }
+              ci -= cnt;
+              ubase += cnt * sz;
+            }
+            if (nu > 0) {
+              queue[n % QDEPTH] = item_pack(ph, u0, nu);
+              __threadfence_block();
+              *q_head = n + 1;
+            }
+          }
+          u0 = __shfl_sync(0xffffffffu, u0, 0);
+          nu = __shfl_sync(0xffffffffu, nu, 0);
+          if (nu <= 0) break;  // this phase is handed out: next phase
+          ++n;
+          const int row0 = u0 * 8;
+          for (int ch = 0; ch < nchunk && ok; ++ch) {
+            const int k0 = ch * TK;
+            const uint32_t kb = static_cast<uint32_t>(min(TK, K - k0)) * 2u;
+            for (int h8 = 0; h8 < nu; ++h8) {
+              const int st = it % STAGES;
+              ok = __all_sync(0xffffffffu, wait_mbar(&empty[st], ((it / STAGES) & 1) ^ 1u, status));
+              if (!ok) break;
+              if (lane == 0) mbar_expect_tx(&full[st], 8 * kb);
+              __syncwarp();
+              if (lane < 8) {
+                const size_t row = static_cast<size_t>(row0 + h8 * 8 + lane);
+                bulk_g2s(ring + st * STAGE_BYTES + lane * PITCH, Wb + (row * K + k0) * 2, kb, &full[st], pol);
+              }
+              ++it;
+            }
+          }
+        }
+      }
+      if (lane == 0) {  // end of the step (or a protocol error): release the other roles
+        if (!ok) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
+        queue[n % QDEPTH] = -1;
+        __threadfence_block();
+        *q_head = n + 1;
+      }
+      if (!ok) {  // wait (bounded) for the copies in flight before the CTA may exit
+        for (int j = 1; j <= STAGES && j <= it; ++j) {
+          const int i2 = it - j;
+          mbar_wait_bounded(&full[i2 % STAGES], (i2 / STAGES) & 1);
+        }
+      }
+      return;
+    }
+
+    // ------------------------------------------------------------------ finishers (warps 1-3)
+    const int ft = tid - 32;  // 0..95
+    bool ok = true;
+    int cur_ph = -1, norm_cnt = 0;
+    bool phase_norm = false, have_rstd = true;
+    int32_t* done_ctr = nullptr;
+    for (int n = 0;; ++n) {
+      ok = bar_and(2, kFin, ok && wait_counter_gt(q_head, n, status));
+      if (!ok) break;
+      const int id = reinterpret_cast<volatile int*>(queue)[n % QDEPTH];
+      if (id < 0) break;
+      const int ph = id >> 21, row0 = ((id >> 4) & 0x1ffff) * 8, nu = id & 15, rows = nu * 8;
+      if (ph != cur_ph) {
+        const StackPhase* P = sp.phases + ph;
+        // private copy of the phase's epilogue description
+        const int* src = reinterpret_cast<const int*>(&P->p);
+        int* dst = reinterpret_cast<int*>(finp);
+        for (int i = ft; i < static_cast<int>(sizeof(SmallMParams) / 4); i += kFin) dst[i] = __ldg(src + i);
+        phase_norm = P->p.act_mode == ACT_F32_NORM;
+        have_rstd = !phase_norm;
+        done_ctr = sp.counters + P->done_idx;
+        // what the epilogue reads (addend) must be written, what it overwrites must have been read
+        ok = bar_and(2, kFin, wait_deps(P->epi_dep, P->epi_need, P->n_epi_deps, sp.counters, status, lane));
+        if (!ok) break;
+        cur_ph = ph;
+      }
+      const int slot = n & 1;
+      bool okw = wait_mbar(&red_full[slot], (n >> 1) & 1, status);
+      if (!have_rstd) okw = okw && wait_mbar(&norm_ready[norm_cnt & (NORM_RING - 1)], (norm_cnt / NORM_RING) & 1, status);
+      ok = bar_and(2, kFin, okw);
+      if (!ok) break;
+      if (!have_rstd) {  // 1/rms of every activation row, once per phase and CTA
+        if (ft < batch) {
+          const float* sq = ssq_part + (norm_cnt & (NORM_RING - 1)) * 32;
+          const float s = sq[ft] + sq[8 + ft] + sq[16 + ft] + sq[24 + ft];
+          rstd_s[ft] = rsqrtf(s / static_cast<float>(finp->K) + finp->eps);
+        }
+        bar_sync(2, kFin);
+        have_rstd = true;
+        ++norm_cnt;
+      }
+      const float* rs = red + slot * RED_FLOATS;
+      auto column = [&](int a, int rr, int c) -> float {
+        const int idx = (a * 4 + ((rr >> 3) * 2 + (c & 1))) * 32 + ((rr & 7) * 4 + (c >> 1));
+        return rs[idx] + rs[RG_MAX * 128 + idx] + rs[2 * RG_MAX * 128 + idx] + rs[3 * RG_MAX * 128 + idx];
+      };
+      auto value = [&](int r, int b) -> float {
+        const int a = r >> 4, rr = r & 15;
+        float s = column(a, rr, b);
+        if (PACKED) s += column(a, rr, b + 4);  // high-part product + low-part product
+        if (phase_norm) s *= rstd_s[b];
+        return s;
+      };
+      smallm_epilogue<kFin>(*finp, ft, rows, row0, batch, value);
+      __threadfence();       // this thread's outputs are visible device-wide ...
+      bar_sync(2, kFin);     // ... for all finisher threads ...
+      if (ft == 0) red_release_add(done_ctr, nu);  // ... before the units count as finished
+      if (lane == 0) mbar_arrive(&red_free[slot]);
+    }
+    if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
+    return;
+  }
+
+  if (warp < 8) {
+    // -------------------------------------------------------------------- consumers (warps 4-7)
+    reg_set<REGS_CONS>();
+    const int cw = warp - 4;
+    const int g = lane >> 2, tig = lane & 3;
+    const uint32_t ring_u32 = smem_u32(ring);
+    const uint32_t act_u32 = smem_u32(act);
+    // which activation row feeds MMA column g: packed = hi rows 0-3 then lo rows 4-7 of batch g & 3
+    const bool col_valid = PACKED ? ((g & 3) < batch) : (g < batch);
+    bool ok = true;
+    uint4 bf[SPW];
+#pragma unroll
+    for (int j = 0; j < SPW; ++j) bf[j] = make_uint4(0, 0, 0, 0);
+    int it = 0, n_req = 0, cur_ph = -1, K = 0, nchunk = 0;
+    for (int n = 0;; ++n) {
+      ok = __all_sync(0xffffffffu, ok && wait_counter_gt(q_head, n, status));
+      if (!ok) break;
+      const int id = reinterpret_cast<volatile int*>(queue)[n % QDEPTH];
+      if (id < 0) break;
+      const int ph = id >> 21;
+      if (ph != cur_ph) {
+        K = sp.phases[ph].p.K;
+        nchunk = sp.phases[ph].nchunk;
+        cur_ph = ph;
+      }
+      const int rows = (id & 15) * 8;
+      const int rgn = (rows + 15) >> 4;
+
+      float acc[RG_MAX][2][4];
+#pragma unroll
+      for (int a = 0; a < RG_MAX; ++a)
+#pragma unroll
+        for (int q = 0; q < 2; ++q)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) acc[a][q][c] = 0.f;
+
+      for (int ch = 0; ch < nchunk && ok; ++ch) {
+        const int k0 = ch * TK;
+        // hoist this warp's activation fragments of the chunk, then hand the buffer back
+        ok = __all_sync(0xffffffffu, wait_mbar(act_full, n_req & 1, status));
+        if (!ok) break;
+        ++n_req;
+#pragma unroll
+        for (int j = 0; j < SPW; ++j)
+          bf[j] = col_valid ? lds128(act_u32 + g * PITCH + (cw * SPW + j) * 64 + tig * 16) : make_uint4(0, 0, 0, 0);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(act_free);
+#pragma unroll
+        for (int rgi = 0; rgi < RG_MAX; ++rgi) {
+          if (rgi >= rgn || !ok) break;  // uniform across the warp
+          const bool hi_valid = (rgi * 16 + 8) < rows;
+          const int st0 = it % STAGES, st1 = (it + 1) % STAGES;
+          bool okw = wait_mbar(&full[st0], (it / STAGES) & 1, status);
+          if (okw && hi_valid) okw = wait_mbar(&full[st1], ((it + 1) / STAGES) & 1, status);
+          ok = __all_sync(0xffffffffu, okw);
+          if (!ok) break;
+          const uint32_t base0 = ring_u32 + st0 * STAGE_BYTES + g * PITCH + tig * 16;
+          const uint32_t base1 = ring_u32 + st1 * STAGE_BYTES + g * PITCH + tig * 16;
+          // software pipeline over groups of 2 slabs: the shared-memory loads of group i+1 are issued
+          // before the MMAs of group i
+          uint4 lo[2][2], hi[2][2];
+          auto load_group = [&](int grp, uint4(&l)[2], uint4(&h)[2]) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int slab = cw * SPW + grp * 2 + e;
+              const bool kv = (k0 + slab * 32 + tig * 8) < K;
+              l[e] = make_uint4(0, 0, 0, 0);
+              h[e] = make_uint4(0, 0, 0, 0);
+              if (kv) l[e] = lds128(base0 + slab * 64);
+              if (kv && hi_valid) h[e] = lds128(base1 + slab * 64);
+            }
+          };
+          load_group(0, lo[0], hi[0]);
+#pragma unroll
+          for (int grp = 0; grp < SPW / 2; ++grp) {
+            if (grp + 1 < SPW / 2) load_group(grp + 1, lo[(grp + 1) & 1], hi[(grp + 1) & 1]);
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int j = grp * 2 + e;
+              const uint4& l = lo[grp & 1][e];
+              const uint4& h = hi[grp & 1][e];
+              mma_bf16_16816(acc[rgi][0], l.x, h.x, l.y, h.y, bf[j].x, bf[j].y);
+              mma_bf16_16816(acc[rgi][1], l.z, h.z, l.w, h.w, bf[j].z, bf[j].w);
+            }
+          }
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(&empty[st0]);
+            if (hi_valid) mbar_arrive(&empty[st1]);
+          }
+          it += hi_valid ? 2 : 1;
+        }
+      }
+      if (!ok) break;
+
+      // hand the accumulator fragments to the finishers and move on
+      const int slot = n & 1;
+      ok = __all_sync(0xffffffffu, wait_mbar(&red_free[slot], ((n >> 1) & 1) ^ 1u, status));
+      if (!ok) break;
+      float* rs = red + slot * RED_FLOATS;
+#pragma unroll
+      for (int a = 0; a < RG_MAX; ++a) {
+        if (a >= rgn) break;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) rs[((cw * RG_MAX + a) * 4 + c) * 32 + lane] = acc[a][0][c] + acc[a][1][c];
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&red_full[slot]);
+    }
+    if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
+    return;
+  }
+
+  if (warp < 12) {
+    // -------------------------------------------------------------------- stagers (warps 8-11)
+    reg_set<REGS_STAGE>();
+    const int st = tid - 256;  // 0..127
+    const int sw = warp - 8;
+    const uint32_t act_u32 = smem_u32(act);
+    bool ok = true;
+    int cur_ph = -1, K = 0, nchunk = 0, norm_cnt = 0, r = 0;
+    bool norm = false, ssq_on = false;
+    const float* actf = nullptr;
+    const __nv_bfloat16* gain = nullptr;
+    float ssq[8];
+#pragma unroll
+    for (int b = 0; b < 8; ++b) ssq[b] = 0.f;
+
+    F8 x[4][2];
+    uint4 gq[2];
+    bool kv[2];
+    auto load_rows = [&](int ch, int round) {
+      const int k0 = ch * TK;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int k = k0 + (st + u * 128) * 8;
+        kv[u] = k < K;
+        gq[u] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);  // gain 1.0
+        if (norm) gq[u] = kv[u] ? __ldg(reinterpret_cast<const uint4*>(gain + k)) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int b = round * 4 + i;
+          x[i][u].a = x[i][u].b = make_float4(0, 0, 0, 0);
+          if (kv[u] && b < batch) {
+            const float4* src =
+                reinterpret_cast<const float4*>(actf + static_cast<size_t>(b) * K + k0 + (st + u * 128) * 8);
+            x[i][u].a = __ldcg(src);
+            x[i][u].b = __ldcg(src + 1);
+          }
+        }
+    };
+    auto store_rows = [&](int round) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int b = round * 4 + i;
+        if (b >= batch) break;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          float y[8] = {x[i][u].a.x, x[i][u].a.y, x[i][u].a.z, x[i][u].a.w,
+                        x[i][u].b.x, x[i][u].b.y, x[i][u].b.z, x[i][u].b.w};
+          if (norm) {
+            if (ssq_on)
+              ssq[b] += y[0] * y[0] + y[1] * y[1] + y[2] * y[2] + y[3] * y[3] + y[4] * y[4] + y[5] * y[5] +
+                        y[6] * y[6] + y[7] * y[7];
+            y[0] *= bf16_lo(gq[u].x);
+            y[1] *= bf16_hi(gq[u].x);
+            y[2] *= bf16_lo(gq[u].y);
+            y[3] *= bf16_hi(gq[u].y);
+            y[4] *= bf16_lo(gq[u].z);
+            y[5] *= bf16_hi(gq[u].z);
+            y[6] *= bf16_lo(gq[u].w);
+            y[7] *= bf16_hi(gq[u].w);
+          }
+          uint4 hi;
+          hi.x = pack_bf16x2(y[0], y[1]);
+          hi.y = pack_bf16x2(y[2], y[3]);
+          hi.z = pack_bf16x2(y[4], y[5]);
+          hi.w = pack_bf16x2(y[6], y[7]);
+          const uint32_t dst = act_u32 + b * PITCH + (st + u * 128) * 16;
+          sts128(dst, hi);
+          if (PACKED) {
+            uint4 lo;
+            lo.x = pack_bf16x2(y[0] - bf16_lo(hi.x), y[1] - bf16_hi(hi.x));
+            lo.y = pack_bf16x2(y[2] - bf16_lo(hi.y), y[3] - bf16_hi(hi.y));
+            lo.z = pack_bf16x2(y[4] - bf16_lo(hi.z), y[5] - bf16_hi(hi.z));
+            lo.w = pack_bf16x2(y[6] - bf16_lo(hi.w), y[7] - bf16_hi(hi.w));
+            sts128(dst + 4 * PITCH, lo);
+          }
+        }
+      }
+    };
+
+    for (int n = 0;; ++n) {
+      ok = __all_sync(0xffffffffu, ok && wait_counter_gt(q_head, n, status));
+      if (!ok) break;
+      const int id = reinterpret_cast<volatile int*>(queue)[n % QDEPTH];
+      if (id < 0) break;
+      const int ph = id >> 21;
+      if (ph != cur_ph) {
+        const StackPhase* P = sp.phases + ph;
+        K = P->p.K;
+        nchunk = P->nchunk;
+        actf = static_cast<const float*>(P->p.act);
+        gain = P->p.gain;
+        norm = P->p.act_mode == ACT_F32_NORM;
+        ssq_on = norm;  // the first batch of a normalised phase also forms the sums of squares
+        cur_ph = ph;
+        // the activations of this phase must have been written (all of them: every batch needs all of K)
+        ok = wait_deps(P->act_dep, P->act_need, P->n_act_deps, sp.counters, status, lane);
+        if (!ok) break;
+      }
+      // chunk by chunk, one chunk ahead of the consumers: the raw values are loaded into registers
+      // before the buffer is handed back (act_free)
+      for (int ch = 0; ch < nchunk; ++ch, ++r) {
+        load_rows(ch, 0);
+        ok = __all_sync(0xffffffffu, wait_mbar(act_free, (r & 1) ^ 1u, status));
+        if (!ok) break;
+        store_rows(0);
+        if (!PACKED && batch > 4) {
+          load_rows(ch, 1);
+          store_rows(1);
+        }
+        if (ssq_on && ch == nchunk - 1) {  // every chunk has been staged once: publish the sums
+          float* sq = ssq_part + (norm_cnt & (NORM_RING - 1)) * 32;
+#pragma unroll
+          for (int b = 0; b < 8; ++b) {
+            if (b < batch) {
+              const float t = warp_sum(ssq[b]);
+              if (lane == 0) sq[sw * 8 + b] = t;
+            }
+            ssq[b] = 0.f;
+          }
+          ssq_on = false;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&norm_ready[norm_cnt & (NORM_RING - 1)]);
+          ++norm_cnt;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(act_full);
+      }
+      if (!ok) break;
+    }
+    if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
+    return;
+  }
+
+  // ---------------------------------------------------------------------- attention (warps 12-15)
+  reg_set<REGS_AUX>();
+  {
+    const int at = tid - 384;  // 0..127
+    float* ps = reinterpret_cast<float*>(smem + OFF_AUX);
+    float* ared = reinterpret_cast<float*>(smem + OFF_AUX + AUX_PS);
+    float* mls = reinterpret_cast<float*>(smem + OFF_AUX + AUX_PS + AUX_RED);
+    int* pre = reinterpret_cast<int*>(smem + OFF_AUX + AUX_PS + AUX_RED + AUX_MLS);  // [9] prefix of live splits
+    float* red_m = reinterpret_cast<float*>(pre + 12);
+    float* red_l = red_m + 4;
+    bool ok = true;
+    if (sp.n_attn > 0 && at == 0) {
+      const DecodeAttnParams& a0 = sp.attn[0].a;
+      int acc = 0;
+      pre[0] = 0;
+      for (int b = 0; b < batch; ++b) {
+        int L = a0.kv_len[b] + a0.kv_len_offset;
+        L = max(0, min(L, a0.max_seq_len));
+        acc += (L + kChunk - 1) / kChunk;
+        pre[b + 1] = acc;
+      }
+    }
+    bar_sync(3, kAux);
+    for (int li = 0; li < sp.n_attn; ++li) {
+      const StackAttn* A = sp.attn + li;
+      const float* q = A->a.q;
+      const __nv_bfloat16* Kc = A->a.k;
+      const __nv_bfloat16* Vc = A->a.v;
+      const int Hq = A->a.n_q_heads, Hkv = A->a.n_kv_heads, DH = A->a.head_dim, max_seq = A->a.max_seq_len;
+      const int stride_splits = A->a.n_splits;
+      float* scratch = A->a.scratch;
+      float* o = A->a.o;
+      int gt = 1;
+      {
+        const int group = Hq / Hkv;
+        while (gt < 8 && group % (gt * 2) == 0) gt *= 2;
+      }
+      const int HG = Hq / gt;
+      // q and this step's key/value rows are written; the partials of the previous layer are merged
+      ok = bar_and(3, kAux, wait_deps(A->dep, A->need, A->n_deps, sp.counters, status, lane));
+      if (!ok) break;
+      const int total = pre[batch] * HG;
+      int mine = 0;
+      for (int u = blockIdx.x; u < total; u += gridDim.x) {
+        const int hg = u % HG, t = u / HG;
+        int b = 0;
+        while (b + 1 < batch && t >= pre[b + 1]) ++b;
+        const int split = t - pre[b];
+        int L = A->a.kv_len[b] + A->a.kv_len_offset;
+        L = max(0, min(L, max_seq));
+        if (DH == 128)
+          attn_split_dispatch<128>(gt, q, Kc, Vc, Hq, Hkv, max_seq, stride_splits, scratch, b, split, hg, L, ps, ared,
+                                   mls, at);
+        else
+          attn_split_dispatch<64>(gt, q, Kc, Vc, Hq, Hkv, max_seq, stride_splits, scratch, b, split, hg, L, ps, ared, mls,
+                                  at);
+        ++mine;
+      }
+      __threadfence();
+      bar_sync(3, kAux);
+      if (at == 0 && mine > 0) red_release_add(sp.counters + A->split_done, mine);
+      // all partials of this layer (every CTA's) before any merge; o free to overwrite
+      bool okw = true;
+      if (lane == 0) okw = wait_global_ge(sp.counters + A->split_done, total, status);
+      okw = __all_sync(0xffffffffu, okw) && wait_deps(A->mdep, A->mneed, A->n_mdeps, sp.counters, status, lane);
+      ok = bar_and(3, kAux, okw);
+      if (!ok) break;
+      const int n_pairs = batch * Hq;
+      mine = 0;
+      for (int u = blockIdx.x; u < n_pairs; u += gridDim.x) {
+        const int b = u / Hq, h = u % Hq;
+        const int ns = pre[b + 1] - pre[b];
+        if (DH == 128) attn_merge_unit<128>(scratch, Hq, stride_splits, ns, b, h, o, ared, red_m, red_l, at);
+        else attn_merge_unit<64>(scratch, Hq, stride_splits, ns, b, h, o, ared, red_m, red_l, at);
+        ++mine;
+      }
+      __threadfence();
+      bar_sync(3, kAux);
+      if (at == 0 && mine > 0) red_release_add(sp.counters + A->merge_done, mine);
+    }
+    if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
+  }
+}
+
+bool g_stack_usable = false;
+
+}  // namespace
+
+cudaError_t decode_stack_init(int sm_count, bool* usable) {
+  *usable = false;
+  cudaError_t e = cudaFuncSetAttribute(decode_stack_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_stack_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  if (e != cudaSuccess) return e;
+  // The warpgroups trade registers at run time (setmaxnreg); the totals above assume the launch
+  // allocation of 128 per thread.  Anything else: do not use the kernel.
+  cudaFuncAttributes fa;
+  e = cudaFuncGetAttributes(&fa, decode_stack_kernel<true>);
+  if (e != cudaSuccess) return e;
+  bool ok = fa.numRegs == 128;
+  e = cudaFuncGetAttributes(&fa, decode_stack_kernel<false>);
+  if (e != cudaSuccess) return e;
+  ok = ok && fa.numRegs == 128;
+  int dev = 0, coop = 0, per_sm = 0;
+  e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+  if (e == cudaSuccess)
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_stack_kernel<true>, kThreads, SMEM);
+  if (e != cudaSuccess) return e;
+  (void)sm_count;
+  g_stack_usable = ok && coop && per_sm >= 1;
+  *usable = g_stack_usable;
+  return cudaSuccess;
+}
+
+cudaError_t launch_decode_stack(const StackParams& sp, int sm_count, cudaStream_t stream) {
+  if (!g_stack_usable || sp.batch < 1 || sp.batch > 8 || sp.n_phases > kStackMaxPhases || !sp.status || !sp.counters)
+    return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(sm_count);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = SMEM;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeCooperative;  // all CTAs co-resident: they wait on one another's counters
+  at[0].val.cooperative = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return sp.batch <= 4 ? cudaLaunchKernelEx(&cfg, decode_stack_kernel<true>, sp)
+                       : cudaLaunchKernelEx(&cfg, decode_stack_kernel<false>, sp);
+}
+
+}  // namespace ladder

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "decode_schedule.h"
+
 namespace ladder {
 
 enum ActMode { ACT_F32 = 0, ACT_F32_NORM = 1 };  // activations are fp32 [batch, K]; NORM applies RMSNorm
@@ -63,6 +65,43 @@ struct DecodeAttnParams {
 int decode_attention_splits(int batch, int n_kv_heads, int max_len, int sm_count);
 size_t decode_attention_scratch_floats(int batch, int n_q_heads, int head_dim, int n_splits);
 cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stream, bool pdl);
+
+// Persistent layer-stack kernel of the decode step: every weight-streaming GEMM of the step is a
+// "phase" of ONE cooperative launch, attention runs on dedicated warps of the same CTAs, and the
+// kernel boundaries become counters in global memory (units finished per phase) that a reader polls
+// before it touches data another SM produced.
+constexpr int kStackMaxDeps = 6;
+constexpr int kStackMaxPhases = 1023;
+struct StackPhase {
+  SmallMParams p;
+  int n_units;   // N / 8
+  int nchunk;    // ceil(K / 2048)
+  int work_idx;  // claim counter
+  int done_idx;  // units finished (epilogue written and fenced)
+  Schedule sched;
+  // counters[dep] >= need must hold before the activations are read ...
+  int n_act_deps, act_dep[kStackMaxDeps], act_need[kStackMaxDeps];
+  // ... and before the first epilogue (addend read, output buffer overwritten)
+  int n_epi_deps, epi_dep[kStackMaxDeps], epi_need[kStackMaxDeps];
+};
+struct StackAttn {
+  DecodeAttnParams a;  // n_splits = stride of the scratch layout; the live split count comes from kv_len
+  int n_deps, dep[kStackMaxDeps], need[kStackMaxDeps];      // before the split units (q, K, V written; scratch free)
+  int n_mdeps, mdep[kStackMaxDeps], mneed[kStackMaxDeps];   // before the merge units (o free to overwrite)
+  int split_done, merge_done;                               // counters: units finished
+};
+struct StackParams {
+  const StackPhase* phases;
+  int n_phases;
+  const StackAttn* attn;
+  int n_attn;
+  int32_t* counters;  // all zero at launch
+  int32_t* status;
+  int batch;
+};
+// 0 = usable on this device (registers and shared memory as expected, co-residency of sm_count CTAs)
+cudaError_t decode_stack_init(int sm_count, bool* usable);
+cudaError_t launch_decode_stack(const StackParams& sp, int sm_count, cudaStream_t stream);
 
 // Prefill kernels.
 struct LargeMParams {

@@ -17,7 +17,7 @@ __device__ __forceinline__ void smallm_epilogue(const SmallMParams& p, int ct, i
       const int r = idx % prow, b = idx / prow;
       const size_t o = static_cast<size_t>(b) * p.N + nbase + r;
       float v = value(r, b);
-      if (p.epi_mode == EPI_RESID) v += p.addend[o];
+      if (p.epi_mode == EPI_RESID) v += __ldcg(p.addend + o);  // L2: may have been written by another SM of this launch
       out[o] = v;
     }
   } else if (p.epi_mode == EPI_SWIGLU) {

@@ -60,8 +60,11 @@ def check_generation(B, shape, steps, dtype, gains="ones", schedule=None, min_ag
     prompt = synth.make_tokens(shape, bsz, S)
     max_seq = S + steps + 3
     model = B.Model(w, bsz, max_seq, bsz * S)
-    if schedule is not None:
+    if schedule is not None:        # a multi-kernel schedule (n_streams, graph, pdl); default: the persistent kernel
+        model.set_persistent(False)
         model.set_schedule(*schedule)
+    elif bsz <= 8:
+        assert model.persistent_active()
     cache = B.KVCache(shape, bsz, max_seq, fill=CANARY)
     toks, hids = gpu_generate(B, model, cache, prompt, steps)
     assert model.device_status() == 0
@@ -119,7 +122,7 @@ def test_tiny_cache_values_match_oracle(B):
 def test_schedules_are_bit_identical(B):
     s = synth.replace(synth.SHAPES["tiny"], layer_is_ladder=(1, 1, 0, 1))
     ref = None
-    for sched in [(1, False, False), (1, True, False), (2, False, False), (2, True, False), (1, False, True),
+    for sched in [None, (1, False, False), (1, True, False), (2, False, False), (2, True, False), (1, False, True),
                   (2, False, True), (2, True, True)]:
         _, _, toks, hids, cache = check_generation(B, s, 12, np.float64, schedule=sched, batch=3, min_agree=0.0)
         cur = (toks, hids, cache.k.clone(), cache.v.clone())

@@ -545,11 +545,24 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
     p.batch = batch;
     p.status = m->status;
     P.p = p;
+    P.W = p.W;
+    P.K = p.K;
+    P.act = static_cast<const float*>(p.act);
+    P.gain = p.gain;
+    P.act_mode = p.act_mode;
     P.n_units = p.N / 8;
     P.nchunk = (p.K + 2047) / 2048;
     P.work_idx = sb.counter(-1);
     P.done_idx = sb.counter(P.n_units);
-    P.sched = make_schedule(P.n_units, m->sm_count);
+    const Schedule sc = make_schedule(P.n_units, m->sm_count);
+    if (sc.n > kStackRounds) sb.overflow = true;
+    P.sched_n = sc.n < kStackRounds ? sc.n : kStackRounds;
+    for (int r = 0; r < P.sched_n; ++r) {
+      P.count[r] = sc.count[r];
+      P.size[r] = sc.size[r];
+    }
+    P.n_static = sc.n_static;
+    P.n_claims = sc.n_claims;
     std::vector<int> ad, ed;
     sb.raw(act_buf, ad);
     sb.raw(add_buf, ed);

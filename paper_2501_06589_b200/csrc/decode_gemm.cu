@@ -50,7 +50,7 @@ constexpr int PITCH = TK * 2 + 64;
 constexpr int STAGE_BYTES = 8 * PITCH;
 constexpr int STAGES = 4;
 constexpr int ACT_BYTES = 8 * PITCH;
-constexpr int RG_MAX = 5;           // 16-row groups per batch at most (10 units)
+constexpr int RG_MAX = kSchedUnitsMax / 2;  // 16-row groups per batch at most
 static_assert(2 * RG_MAX == kSchedUnitsMax, "schedule and tile geometry disagree");
 constexpr int SPW = TK / 32 / 4;    // 32-wide K slabs per consumer warp per chunk
 constexpr int RED_FLOATS = 4 * RG_MAX * 4 * 32;

@@ -6,13 +6,20 @@
 namespace ladder {
 
 constexpr int kSchedMaxPhases = 24;
-constexpr int kSchedUnitsMax = 10;  // 8-row units per claim at most (5 MMA row groups)
+#ifndef DS_UMAX
+#define DS_UMAX 10
+#endif
+constexpr int kSchedUnitsMax = DS_UMAX;  // 8-row units per claim at most (5 MMA row groups)
 
 // Round i hands out count[i] claims of size[i] consecutive units.
 struct Schedule {
   int n;
   int count[kSchedMaxPhases];
   int size[kSchedMaxPhases];
+  // The first n_static claims can be dealt out without the counter, claim i to CTA i % grid (whole
+  // rounds of one claim per CTA); only the claims after them need to be taken dynamically.
+  int n_static;
+  int n_claims;  // all claims
 };
 
 // A batch costs a fixed latency per K chunk (activation hand-over, fragment hoisting) and re-reads
@@ -26,7 +33,10 @@ struct Schedule {
 inline Schedule make_schedule(int n_units, int grid) {
   Schedule sc = {};
   auto push = [&](int count, int size) {
-    if (count > 0 && size > 0 && sc.n < kSchedMaxPhases) {
+    if (count <= 0 || size <= 0) return;
+    if (sc.n > 0 && sc.size[sc.n - 1] == size) {  // same size as the round before: one longer round
+      sc.count[sc.n - 1] += count;
+    } else if (sc.n < kSchedMaxPhases) {
       sc.count[sc.n] = count;
       sc.size[sc.n] = size;
       ++sc.n;
@@ -37,19 +47,24 @@ inline Schedule make_schedule(int n_units, int grid) {
     const int hi = (rem + grid - 1) / grid, n_hi = rem - (hi - 1) * grid;  // n_hi batches of hi, rest hi-1
     push(n_hi, hi);
     push(grid - n_hi, hi - 1);
+    sc.n_claims = hi > 1 ? grid : n_hi;
+    sc.n_static = sc.n_claims;
     return sc;
   }
   while (rem > 0 && sc.n < kSchedMaxPhases - 2) {
     const double share = static_cast<double>(rem) / grid;
     int size;
-    if (share >= 12.0) size = 8;
-    else if (share >= 4.0) size = (static_cast<int>(share * 0.7) & ~1) > 8 ? 8 : (static_cast<int>(share * 0.7) & ~1);
+    constexpr int kBig = kSchedUnitsMax < 8 ? kSchedUnitsMax : 8;
+    if (share >= 12.0) size = kBig;
+    else if (share >= 4.0) size = (static_cast<int>(share * 0.7) & ~1) > kBig ? kBig : (static_cast<int>(share * 0.7) & ~1);
     else break;
     push(grid, size);
     rem -= grid * size;
+    sc.n_static += grid;
   }
   push(rem / 2, 2);
   push(rem & 1, 1);
+  sc.n_claims = sc.n_static + rem / 2 + (rem & 1);
   return sc;
 }
 

@@ -47,7 +47,7 @@ constexpr int PITCH = TK * 2 + 64;
 constexpr int STAGE_BYTES = 8 * PITCH;
 constexpr int STAGES = 4;
 constexpr int ACT_BYTES = 8 * PITCH;
-constexpr int RG_MAX = 5;
+constexpr int RG_MAX = kSchedUnitsMax / 2;
 static_assert(2 * RG_MAX == kSchedUnitsMax, "schedule and tile geometry disagree");
 constexpr int SPW = TK / 32 / 4;
 constexpr int RED_FLOATS = 4 * RG_MAX * 4 * 32;
@@ -64,10 +64,10 @@ constexpr int OFF_RSTD = OFF_RED + 2 * RED_FLOATS * 4;
 constexpr int N_BARS = 2 * STAGES + 2 + NORM_RING + 4;       // full, empty, act_free, act_full, norm_ready[], red_full[2], red_free[2]
 constexpr int OFF_BAR = OFF_RSTD + 8 * 4;
 constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;               // queue[QDEPTH], q_head, dead flag
-constexpr int OFF_FINP = OFF_MISC + 128;                     // the finishers' copy of the phase parameters
+constexpr int OFF_FINP = OFF_MISC + 256;                     // the finishers' copy of the phase parameters
 constexpr int FINP_BYTES = 256;
 static_assert(sizeof(SmallMParams) <= FINP_BYTES, "phase parameter copy too small");
-static_assert((QDEPTH + 2) * 4 <= 128, "queue area too small");
+static_assert((3 * QDEPTH + 2) * 4 <= 256, "queue area too small");
 constexpr int OFF_AUX = OFF_FINP + FINP_BYTES;
 constexpr int AUX_PS = 4 * 8 * 16 * 4;
 constexpr int AUX_RED = 4 * 8 * 128 * 4;
@@ -78,7 +78,13 @@ constexpr int SMEM = OFF_AUX + AUX_PS + AUX_RED + AUX_MLS + AUX_MISC + 128;
 static_assert(SMEM <= 227 * 1024, "shared memory budget");
 
 // registers per thread after the warpgroups have traded (launch allocation: 128 each)
-constexpr int REGS_WG0 = 72, REGS_CONS = 176, REGS_STAGE = 120, REGS_AUX = 144;
+#ifndef RW0
+#define RW0 72
+#define RCO 176
+#define RST 120
+#define RAU 144
+#endif
+constexpr int REGS_WG0 = RW0, REGS_CONS = RCO, REGS_STAGE = RST, REGS_AUX = RAU;
 static_assert(REGS_WG0 + REGS_CONS + REGS_STAGE + REGS_AUX <= 4 * 128, "register pool exceeded");
 
 struct F8 {
@@ -130,14 +136,24 @@ __device__ __forceinline__ bool wait_mbar(uint64_t* bar, uint32_t parity, const 
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t i = 1;; ++i) {
+#if DS_POLL == 1
+    if (mbar_try_wait_suspend(bar, parity, 4000u)) return true;
+    if ((i & 15u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
+#elif DS_POLL == 2
+    __nanosleep(200);
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
+#else
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
+#endif
   }
 }
 __device__ __forceinline__ bool wait_counter_gt(const volatile int* ctr, int n, const int32_t* status) {
   if (*ctr > n) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t i = 1;; ++i) {
+    __nanosleep(64);  // a hot spin would take issue slots from the consumer warp of the same sub-partition
     if (*ctr > n) return true;
     if ((i & 255u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
   }
@@ -146,6 +162,7 @@ __device__ __forceinline__ bool wait_global_ge(const int32_t* ctr, int need, con
   if (ld_acquire(ctr) >= need) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t i = 1;; ++i) {
+    __nanosleep(100);
     if (ld_acquire(ctr) >= need) return true;
     if ((i & 31u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
   }
@@ -158,8 +175,74 @@ __device__ __forceinline__ bool wait_deps(const int* dep, const int* need, int n
   return __all_sync(0xffffffffu, ok);
 }
 
+#ifndef DS_POLL
+#define DS_POLL 1
+#endif
+#ifdef DS_TRACE
+// tuning builds only: per CTA, cycles each role spent in its waits during the launch
+// [0] consumer total [1] c:queue [2] c:act_full [3] c:weights [4] c:red_free
+// [5] producer total [6] p:ring full [7] p:claims  [8] stager total [9] s:deps [10] s:act_free [11] s:queue
+// [12] finisher total [13] f:deps [14] f:red_full/norm [15] f:queue
+__device__ unsigned long long g_stack_trace[148 * 16];
+// consumer timeline: [phase][cta][0] first item of the phase taken up, [1] last item of the phase handed over (ns)
+__device__ unsigned long long g_phase_trace[330 * 148 * 2];
+#define TR_DECL(n) long long tr_##n = 0
+#define TR_T0() const long long tr_t0_ = clock64()
+#define TR_ADD(n) tr_##n += clock64() - tr_t0_
+#define TR_OUT(i, n) g_stack_trace[blockIdx.x * 16 + (i)] = static_cast<unsigned long long>(tr_##n)
+#else
+#define TR_DECL(n)
+#define TR_T0()
+#define TR_ADD(n)
+#define TR_OUT(i, n)
+#endif
+
+template <typename T>
+__device__ __forceinline__ T* ldg_ptr(T* const* p) {  // read-only load of a pointer field
+  return reinterpret_cast<T*>(__ldg(reinterpret_cast<const unsigned long long*>(p)));
+}
+
 // queue item: phase (10 bits) | first unit (17 bits) | units (4 bits)
 __device__ __forceinline__ int item_pack(int ph, int u0, int nu) { return (ph << 21) | (u0 << 4) | nu; }
+
+// One [16 rows x 2048 k] tile of a consumer warp: its SPW 32-wide K slabs, two 8-row stages as the two
+// row halves of the MMA, software-pipelined over groups of 2 slabs (the shared-memory loads of group
+// i+1 are issued before the MMAs of group i), two accumulator chains.  FAST: every slab lies inside K
+// and both stages are present, so nothing is predicated.
+template <bool FAST>
+__device__ __forceinline__ void slab_loop(float (&acc0)[4], float (&acc1)[4], const uint4 (&bf)[SPW], uint32_t base0,
+                                          uint32_t base1, int cw, int k0, int K, int tig, bool hi_valid) {
+  uint4 lo[2][2], hi[2][2];
+  auto load_group = [&](int grp, uint4(&l)[2], uint4(&h)[2]) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int slab = cw * SPW + grp * 2 + e;
+      if (FAST) {
+        l[e] = lds128(base0 + slab * 64);
+        h[e] = lds128(base1 + slab * 64);
+      } else {
+        const bool kv = (k0 + slab * 32 + tig * 8) < K;
+        l[e] = make_uint4(0, 0, 0, 0);
+        h[e] = make_uint4(0, 0, 0, 0);
+        if (kv) l[e] = lds128(base0 + slab * 64);
+        if (kv && hi_valid) h[e] = lds128(base1 + slab * 64);
+      }
+    }
+  };
+  load_group(0, lo[0], hi[0]);
+#pragma unroll
+  for (int grp = 0; grp < SPW / 2; ++grp) {
+    if (grp + 1 < SPW / 2) load_group(grp + 1, lo[(grp + 1) & 1], hi[(grp + 1) & 1]);
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int j = grp * 2 + e;
+      const uint4& l = lo[grp & 1][e];
+      const uint4& h = hi[grp & 1][e];
+      mma_bf16_16816(acc0, l.x, h.x, l.y, h.y, bf[j].x, bf[j].y);
+      mma_bf16_16816(acc1, l.z, h.z, l.w, h.w, bf[j].z, bf[j].w);
+    }
+  }
+}
 
 // ------------------------------------------------------------------------------------ attention units
 // One split unit: 64 keys x GT query heads sharing a kv head x one sequence, 4 warps (16 keys each).
@@ -409,9 +492,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
   uint64_t* norm_ready = act_full + 1;        // [NORM_RING] stagers -> finishers
   uint64_t* red_full = norm_ready + NORM_RING;  // [2] consumers -> finishers
   uint64_t* red_free = red_full + 2;            // [2] finishers -> consumers
-  int* queue = reinterpret_cast<int*>(smem + OFF_MISC);
-  volatile int* q_head = queue + QDEPTH;
-  int* flag_s = queue + QDEPTH + 1;
+  int* queue = reinterpret_cast<int*>(smem + OFF_MISC);  // [QDEPTH] items, then K and chunk count of each item's phase
+  volatile int* queue_k = queue + QDEPTH;
+  volatile int* queue_nc = queue + 2 * QDEPTH;
+  volatile int* q_head = queue + 3 * QDEPTH;
+  int* flag_s = queue + 3 * QDEPTH + 1;
   SmallMParams* finp = reinterpret_cast<SmallMParams*>(smem + OFF_FINP);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -444,19 +529,61 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       const uint64_t pol = l2_policy_evict_first();
       bool ok = true;
       int it = 0, n = 0;
-      for (int ph = 0; ph < sp.n_phases && ok; ++ph) {
-        const StackPhase* P = sp.phases + ph;
-        const uint8_t* Wb = reinterpret_cast<const uint8_t*>(P->p.W);
-        const int K = P->p.K, n_units = P->n_units, nchunk = P->nchunk;
-        int32_t* work = sp.counters + P->work_idx;
-        while (ok) {
-          // one claim at a time (claiming ahead would let a CTA hoard batches it cannot start yet)
-          int u0 = 0, nu = 0;
-          if (lane == 0) {
-            int ci = atomicAdd(work, 1), ubase = 0;
-            const int sn = P->sched.n;
+      TR_DECL(ring);
+      TR_DECL(claim);
+      TR_DECL(total);
+#ifdef DS_TRACE
+      const long long tr_start = clock64();
+#endif
+      // Which batch comes next is settled one batch ahead of the weight stream, right after the first
+      // tile of the current batch has been issued, so the stagers and finishers know early and no
+      // round trip of an atomic is exposed.  Whole rounds of a phase's schedule are dealt out
+      // statically (claim i to CTA i mod grid): a phase in which every CTA has exactly one batch must
+      // not let an early CTA take a second one.  Only the short batches at the end of a long phase are
+      // claimed through the counter, which is what evens out the SMs' different streaming rates.
+      // The first 128 bytes of a phase descriptor are held across the warp, lane i owning word i, and
+      // read with shuffles; the descriptor of the following phase is loaded one phase ahead.
+      constexpr int H_W = 0, H_K = 2, H_UNITS = 3, H_NCHUNK = 4, H_WORK = 5, H_STATIC = 7, H_CLAIMS = 8, H_ROUNDS = 9,
+                    H_COUNT = 10, H_SIZE = 20;
+      static_assert(offsetof(StackPhase, n_static) == 4 * H_STATIC && offsetof(StackPhase, count) == 4 * H_COUNT &&
+                        offsetof(StackPhase, size) == 4 * H_SIZE && offsetof(StackPhase, K) == 4 * H_K,
+                    "descriptor layout");
+      auto load_hdr = [&](int ph) -> int {
+        return ph < sp.n_phases ? __ldg(reinterpret_cast<const int*>(sp.phases + ph) + lane) : 0;
+      };
+      auto H = [&](int h, int idx) -> int { return __shfl_sync(0xffffffffu, h, idx); };
+      int cl_ph = 0;    // phase of the next claim
+      int cl_k = 0;     // static claims of that phase this CTA has taken
+      int cl_pend = 0;  // claim index asked for in phase cl_ph (valid in lane 0)
+      int hdr = load_hdr(0), hdr_nx = load_hdr(1);
+      // what the item returned by claim_finish belongs to
+      const uint8_t* nx_W = nullptr;
+      int nx_K = 0, nx_nchunk = 0;
+      // ask for the next claim of phase cl_ph (an atomic only for the dynamic tail; its answer is not
+      // needed before claim_finish)
+      auto claim_issue = [&]() {
+        const int n_static = H(hdr, H_STATIC), n_claims = H(hdr, H_CLAIMS), work = H(hdr, H_WORK);
+        const int ci = blockIdx.x + cl_k * static_cast<int>(gridDim.x);
+        if (ci < n_static) {
+          ++cl_k;
+          cl_pend = ci;
+        } else if (n_static < n_claims) {
+          if (lane == 0) cl_pend = n_static + atomicAdd(sp.counters + work, 1);
+        } else {
+          cl_pend = n_claims;
+        }
+      };
+      // turn the claim into the next item (moving on to later phases while a phase has nothing left
+      // for this CTA), publish it; 0 = end of the step
+      auto claim_finish = [&]() -> int {
+        int item = 0;
+        for (;;) {
+          int ci = __shfl_sync(0xffffffffu, cl_pend, 0), u0 = 0, nu = 0;
+          if (ci < H(hdr, H_CLAIMS)) {
+            int ubase = 0;
+            const int sn = H(hdr, H_ROUNDS), n_units = H(hdr, H_UNITS);
             for (int r = 0; r < sn; ++r) {
-              const int cnt = P->sched.count[r], sz = P->sched.size[r];
+              const int cnt = H(hdr, H_COUNT + r), sz = H(hdr, H_SIZE + r);
               if (ci < cnt) {
                 u0 = ubase + ci * sz;
                 nu = min(sz, n_units - u0);
@@ -465,41 +592,94 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
               ci -= cnt;
               ubase += cnt * sz;
             }
-            if (nu > 0) {
-              queue[n % QDEPTH] = item_pack(ph, u0, nu);
-              __threadfence_block();
-              *q_head = n + 1;
-            }
           }
-          u0 = __shfl_sync(0xffffffffu, u0, 0);
-          nu = __shfl_sync(0xffffffffu, nu, 0);
-          if (nu <= 0) break;  // this phase is handed out: next phase
-          ++n;
-          const int row0 = u0 * 8;
-          for (int ch = 0; ch < nchunk && ok; ++ch) {
-            const int k0 = ch * TK;
-            const uint32_t kb = static_cast<uint32_t>(min(TK, K - k0)) * 2u;
-            for (int h8 = 0; h8 < nu; ++h8) {
-              const int st = it % STAGES;
+          if (nu > 0) {
+            item = item_pack(cl_ph, u0, nu) | (1 << 31);
+            nx_K = H(hdr, H_K);
+            nx_nchunk = H(hdr, H_NCHUNK);
+            nx_W = reinterpret_cast<const uint8_t*>(
+                (static_cast<unsigned long long>(static_cast<unsigned int>(H(hdr, H_W + 1))) << 32) |
+                static_cast<unsigned int>(H(hdr, H_W)));
+            break;
+          }
+          ++cl_ph;  // nothing left for this CTA in this phase
+          cl_k = 0;
+          if (cl_ph >= sp.n_phases) break;
+          hdr = hdr_nx;
+          hdr_nx = load_hdr(cl_ph + 1);
+          claim_issue();
+        }
+        if (lane == 0) {
+          queue[n % QDEPTH] = item ? (item & 0x7fffffff) : -1;
+          queue_k[n % QDEPTH] = nx_K;
+          queue_nc[n % QDEPTH] = nx_nchunk;
+          __threadfence_block();
+          *q_head = n + 1;
+        }
+        ++n;
+        return item;
+      };
+      int item;
+      {
+        TR_T0();
+        claim_issue();
+        item = claim_finish();
+        TR_ADD(claim);
+      }
+      while (ok && item != 0) {
+        const int u0 = (item >> 4) & 0x1ffff, nu = item & 15;
+        const uint8_t* Wb = nx_W;
+        const int K = nx_K, nchunk = nx_nchunk;
+        {  // ask for the batch after this one; the answer is picked up two tiles later
+          TR_T0();
+          claim_issue();
+          TR_ADD(claim);
+        }
+        const int resolve_at = min(2, nchunk * nu - 1);
+        int issued = 0;
+        int next_item = 0;
+        const int row0 = u0 * 8;
+        for (int ch = 0; ch < nchunk && ok; ++ch) {
+          const int k0 = ch * TK;
+          const uint32_t kb = static_cast<uint32_t>(min(TK, K - k0)) * 2u;
+          for (int h8 = 0; h8 < nu; ++h8) {
+            const int st = it % STAGES;
+            {
+              TR_T0();
               ok = __all_sync(0xffffffffu, wait_mbar(&empty[st], ((it / STAGES) & 1) ^ 1u, status));
-              if (!ok) break;
-              if (lane == 0) mbar_expect_tx(&full[st], 8 * kb);
-              __syncwarp();
-              if (lane < 8) {
-                const size_t row = static_cast<size_t>(row0 + h8 * 8 + lane);
-                bulk_g2s(ring + st * STAGE_BYTES + lane * PITCH, Wb + (row * K + k0) * 2, kb, &full[st], pol);
-              }
-              ++it;
+              TR_ADD(ring);
+            }
+            if (!ok) break;
+            if (lane == 0) mbar_expect_tx(&full[st], 8 * kb);
+            __syncwarp();
+            if (lane < 8) {
+              const size_t row = static_cast<size_t>(row0 + h8 * 8 + lane);
+              bulk_g2s(ring + st * STAGE_BYTES + lane * PITCH, Wb + (row * K + k0) * 2, kb, &full[st], pol);
+            }
+            ++it;
+            if (issued++ == resolve_at) {  // tiles are on their way: publish what comes next
+              TR_T0();
+              next_item = claim_finish();
+              TR_ADD(claim);
             }
           }
         }
+        item = next_item;
       }
-      if (lane == 0) {  // end of the step (or a protocol error): release the other roles
-        if (!ok) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
+      if (!ok && lane == 0) {  // protocol error: release the other roles
         queue[n % QDEPTH] = -1;
         __threadfence_block();
         *q_head = n + 1;
       }
+#ifdef DS_TRACE
+      tr_total = clock64() - tr_start;
+      if (lane == 0) {
+        TR_OUT(5, total);
+        TR_OUT(6, ring);
+        TR_OUT(7, claim);
+      }
+#endif
+      if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
       if (!ok) {  // wait (bounded) for the copies in flight before the CTA may exit
         for (int j = 1; j <= STAGES && j <= it; ++j) {
           const int i2 = it - j;
@@ -515,8 +695,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
     int cur_ph = -1, norm_cnt = 0;
     bool phase_norm = false, have_rstd = true;
     int32_t* done_ctr = nullptr;
+    TR_DECL(fdeps);
+    TR_DECL(fred);
+    TR_DECL(fq);
+    TR_DECL(ftotal);
+#ifdef DS_TRACE
+    const long long tr_fstart = clock64();
+#endif
     for (int n = 0;; ++n) {
-      ok = bar_and(2, kFin, ok && wait_counter_gt(q_head, n, status));
+      {
+        TR_T0();
+        ok = bar_and(2, kFin, ok && wait_counter_gt(q_head, n, status));
+        TR_ADD(fq);
+      }
       if (!ok) break;
       const int id = reinterpret_cast<volatile int*>(queue)[n % QDEPTH];
       if (id < 0) break;
@@ -527,18 +718,27 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         const int* src = reinterpret_cast<const int*>(&P->p);
         int* dst = reinterpret_cast<int*>(finp);
         for (int i = ft; i < static_cast<int>(sizeof(SmallMParams) / 4); i += kFin) dst[i] = __ldg(src + i);
-        phase_norm = P->p.act_mode == ACT_F32_NORM;
+        phase_norm = __ldg(&P->act_mode) == ACT_F32_NORM;
         have_rstd = !phase_norm;
-        done_ctr = sp.counters + P->done_idx;
+        done_ctr = sp.counters + __ldg(&P->done_idx);
         // what the epilogue reads (addend) must be written, what it overwrites must have been read
-        ok = bar_and(2, kFin, wait_deps(P->epi_dep, P->epi_need, P->n_epi_deps, sp.counters, status, lane));
+        {
+          TR_T0();
+          ok = bar_and(2, kFin, wait_deps(P->epi_dep, P->epi_need, P->n_epi_deps, sp.counters, status, lane));
+          TR_ADD(fdeps);
+        }
         if (!ok) break;
         cur_ph = ph;
       }
       const int slot = n & 1;
-      bool okw = wait_mbar(&red_full[slot], (n >> 1) & 1, status);
-      if (!have_rstd) okw = okw && wait_mbar(&norm_ready[norm_cnt & (NORM_RING - 1)], (norm_cnt / NORM_RING) & 1, status);
-      ok = bar_and(2, kFin, okw);
+      {
+        TR_T0();
+        bool okw = wait_mbar(&red_full[slot], (n >> 1) & 1, status);
+        if (!have_rstd)
+          okw = okw && wait_mbar(&norm_ready[norm_cnt & (NORM_RING - 1)], (norm_cnt / NORM_RING) & 1, status);
+        ok = bar_and(2, kFin, okw);
+        TR_ADD(fred);
+      }
       if (!ok) break;
       if (!have_rstd) {  // 1/rms of every activation row, once per phase and CTA
         if (ft < batch) {
@@ -569,6 +769,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       if (lane == 0) mbar_arrive(&red_free[slot]);
     }
     if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
+#ifdef DS_TRACE
+    tr_ftotal = clock64() - tr_fstart;
+    if (ft == 0) {
+      TR_OUT(12, ftotal);
+      TR_OUT(13, fdeps);
+      TR_OUT(14, fred);
+      TR_OUT(15, fq);
+    }
+#endif
     return;
   }
 
@@ -586,16 +795,32 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
 #pragma unroll
     for (int j = 0; j < SPW; ++j) bf[j] = make_uint4(0, 0, 0, 0);
     int it = 0, n_req = 0, cur_ph = -1, K = 0, nchunk = 0;
+    TR_DECL(cq);
+    TR_DECL(cact);
+    TR_DECL(cw);
+    TR_DECL(cred);
+    TR_DECL(cmma);
+    TR_DECL(ctotal);
+#ifdef DS_TRACE
+    const long long tr_cstart = clock64();
+#endif
     for (int n = 0;; ++n) {
-      ok = __all_sync(0xffffffffu, ok && wait_counter_gt(q_head, n, status));
+      {
+        TR_T0();
+        ok = __all_sync(0xffffffffu, ok && wait_counter_gt(q_head, n, status));
+        TR_ADD(cq);
+      }
       if (!ok) break;
       const int id = reinterpret_cast<volatile int*>(queue)[n % QDEPTH];
       if (id < 0) break;
       const int ph = id >> 21;
       if (ph != cur_ph) {
-        K = sp.phases[ph].p.K;
-        nchunk = sp.phases[ph].nchunk;
+        K = queue_k[n % QDEPTH];
+        nchunk = queue_nc[n % QDEPTH];
         cur_ph = ph;
+#ifdef DS_TRACE
+        if (warp == 4 && lane == 0 && ph < 330) g_phase_trace[(ph * 148 + blockIdx.x) * 2] = global_timer_ns();
+#endif
       }
       const int rows = (id & 15) * 8;
       const int rgn = (rows + 15) >> 4;
@@ -611,12 +836,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       for (int ch = 0; ch < nchunk && ok; ++ch) {
         const int k0 = ch * TK;
         // hoist this warp's activation fragments of the chunk, then hand the buffer back
-        ok = __all_sync(0xffffffffu, wait_mbar(act_full, n_req & 1, status));
+        {
+          TR_T0();
+          ok = __all_sync(0xffffffffu, wait_mbar(act_full, n_req & 1, status));
+          TR_ADD(cact);
+        }
         if (!ok) break;
         ++n_req;
 #pragma unroll
-        for (int j = 0; j < SPW; ++j)
-          bf[j] = col_valid ? lds128(act_u32 + g * PITCH + (cw * SPW + j) * 64 + tig * 16) : make_uint4(0, 0, 0, 0);
+        for (int j = 0; j < SPW; ++j) bf[j] = lds128(act_u32 + g * PITCH + (cw * SPW + j) * 64 + tig * 16);
+        if (!col_valid) {  // rows of the buffer beyond the batch hold stale data: their MMA columns are zeroed
+#pragma unroll
+          for (int j = 0; j < SPW; ++j) bf[j] = make_uint4(0, 0, 0, 0);
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(act_free);
 #pragma unroll
@@ -624,40 +856,28 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
           if (rgi >= rgn || !ok) break;  // uniform across the warp
           const bool hi_valid = (rgi * 16 + 8) < rows;
           const int st0 = it % STAGES, st1 = (it + 1) % STAGES;
-          bool okw = wait_mbar(&full[st0], (it / STAGES) & 1, status);
-          if (okw && hi_valid) okw = wait_mbar(&full[st1], ((it + 1) / STAGES) & 1, status);
-          ok = __all_sync(0xffffffffu, okw);
+          {
+            TR_T0();
+            bool okw = wait_mbar(&full[st0], (it / STAGES) & 1, status);
+            if (okw && hi_valid) okw = wait_mbar(&full[st1], ((it + 1) / STAGES) & 1, status);
+            ok = __all_sync(0xffffffffu, okw);
+            TR_ADD(cw);
+          }
           if (!ok) break;
           const uint32_t base0 = ring_u32 + st0 * STAGE_BYTES + g * PITCH + tig * 16;
           const uint32_t base1 = ring_u32 + st1 * STAGE_BYTES + g * PITCH + tig * 16;
-          // software pipeline over groups of 2 slabs: the shared-memory loads of group i+1 are issued
-          // before the MMAs of group i
-          uint4 lo[2][2], hi[2][2];
-          auto load_group = [&](int grp, uint4(&l)[2], uint4(&h)[2]) {
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const int slab = cw * SPW + grp * 2 + e;
-              const bool kv = (k0 + slab * 32 + tig * 8) < K;
-              l[e] = make_uint4(0, 0, 0, 0);
-              h[e] = make_uint4(0, 0, 0, 0);
-              if (kv) l[e] = lds128(base0 + slab * 64);
-              if (kv && hi_valid) h[e] = lds128(base1 + slab * 64);
-            }
-          };
-          load_group(0, lo[0], hi[0]);
-#pragma unroll
-          for (int grp = 0; grp < SPW / 2; ++grp) {
-            if (grp + 1 < SPW / 2) load_group(grp + 1, lo[(grp + 1) & 1], hi[(grp + 1) & 1]);
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const int j = grp * 2 + e;
-              const uint4& l = lo[grp & 1][e];
-              const uint4& h = hi[grp & 1][e];
-              mma_bf16_16816(acc[rgi][0], l.x, h.x, l.y, h.y, bf[j].x, bf[j].y);
-              mma_bf16_16816(acc[rgi][1], l.z, h.z, l.w, h.w, bf[j].z, bf[j].w);
-            }
-          }
+#ifdef DS_TRACE
+          const long long tr_m0 = clock64();
+#endif
+          // a full chunk with both 8-row halves present (the common case) takes the path without
+          // predicates: a guarded shared-memory load compiles to a branch, and 64 of them per tile
+          // cost more than the loads and MMAs themselves
+          if (hi_valid && k0 + TK <= K) slab_loop<true>(acc[rgi][0], acc[rgi][1], bf, base0, base1, cw, k0, K, tig, true);
+          else slab_loop<false>(acc[rgi][0], acc[rgi][1], bf, base0, base1, cw, k0, K, tig, hi_valid);
           __syncwarp();
+#ifdef DS_TRACE
+          tr_cmma += clock64() - tr_m0;
+#endif
           if (lane == 0) {
             mbar_arrive(&empty[st0]);
             if (hi_valid) mbar_arrive(&empty[st1]);
@@ -669,7 +889,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
 
       // hand the accumulator fragments to the finishers and move on
       const int slot = n & 1;
-      ok = __all_sync(0xffffffffu, wait_mbar(&red_free[slot], ((n >> 1) & 1) ^ 1u, status));
+      {
+        TR_T0();
+        ok = __all_sync(0xffffffffu, wait_mbar(&red_free[slot], ((n >> 1) & 1) ^ 1u, status));
+        TR_ADD(cred);
+      }
       if (!ok) break;
       float* rs = red + slot * RED_FLOATS;
 #pragma unroll
@@ -680,8 +904,21 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&red_full[slot]);
+#ifdef DS_TRACE
+      if (warp == 4 && lane == 0 && cur_ph < 330) g_phase_trace[(cur_ph * 148 + blockIdx.x) * 2 + 1] = global_timer_ns();
+#endif
     }
     if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
+#ifdef DS_TRACE
+    tr_ctotal = clock64() - tr_cstart;
+    if (warp == 4 && lane == 0) {
+      TR_OUT(0, ctotal);
+      TR_OUT(1, cq);
+      TR_OUT(2, cact);
+      TR_OUT(3, cw);
+      TR_OUT(4, cmma);
+    }
+#endif
     return;
   }
 
@@ -696,6 +933,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
     bool norm = false, ssq_on = false;
     const float* actf = nullptr;
     const __nv_bfloat16* gain = nullptr;
+    static_assert(offsetof(StackPhase, act) == 128 && offsetof(StackPhase, gain) == 136 &&
+                      offsetof(StackPhase, act_mode) == 144 && offsetof(StackPhase, n_act_deps) == 148 &&
+                      offsetof(StackPhase, act_dep) == 152 && offsetof(StackPhase, act_need) == 176,
+                  "descriptor layout");
+    auto load_h1 = [&](int ph) -> int {
+      return ph < sp.n_phases ? __ldg(reinterpret_cast<const int*>(sp.phases + ph) + 32 + lane) : 0;
+    };
+    int h1_nx_ph = 0, h1_nx = load_h1(0);
     float ssq[8];
 #pragma unroll
     for (int b = 0; b < 8; ++b) ssq[b] = 0.f;
@@ -710,7 +955,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         const int k = k0 + (st + u * 128) * 8;
         kv[u] = k < K;
         gq[u] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);  // gain 1.0
-        if (norm) gq[u] = kv[u] ? __ldg(reinterpret_cast<const uint4*>(gain + k)) : make_uint4(0, 0, 0, 0);
+        if (norm) gq[u] = kv[u] ? __ldcg(reinterpret_cast<const uint4*>(gain + k)) : make_uint4(0, 0, 0, 0);  // L2: keeps L1 for the descriptors
       }
 #pragma unroll
       for (int i = 0; i < 4; ++i)
@@ -767,30 +1012,63 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       }
     };
 
+    TR_DECL(sdeps);
+    TR_DECL(sfree);
+    TR_DECL(sq);
+    TR_DECL(stotal);
+#ifdef DS_TRACE
+    const long long tr_sstart = clock64();
+#endif
     for (int n = 0;; ++n) {
-      ok = __all_sync(0xffffffffu, ok && wait_counter_gt(q_head, n, status));
+      {
+        TR_T0();
+        ok = __all_sync(0xffffffffu, ok && wait_counter_gt(q_head, n, status));
+        TR_ADD(sq);
+      }
       if (!ok) break;
       const int id = reinterpret_cast<volatile int*>(queue)[n % QDEPTH];
       if (id < 0) break;
       const int ph = id >> 21;
       if (ph != cur_ph) {
-        const StackPhase* P = sp.phases + ph;
-        K = P->p.K;
-        nchunk = P->nchunk;
-        actf = static_cast<const float*>(P->p.act);
-        gain = P->p.gain;
-        norm = P->p.act_mode == ACT_F32_NORM;
+        // second 128 bytes of the descriptor, lane i owning word i; the next phase's were loaded ahead
+        const int h1 = (ph == h1_nx_ph) ? h1_nx : load_h1(ph);
+        h1_nx_ph = ph + 1;
+        h1_nx = load_h1(ph + 1);
+        K = queue_k[n % QDEPTH];
+        nchunk = queue_nc[n % QDEPTH];
+        actf = reinterpret_cast<const float*>((static_cast<unsigned long long>(static_cast<unsigned int>(
+                                                   __shfl_sync(0xffffffffu, h1, 1)))
+                                               << 32) |
+                                              static_cast<unsigned int>(__shfl_sync(0xffffffffu, h1, 0)));
+        gain = reinterpret_cast<const __nv_bfloat16*>(
+            (static_cast<unsigned long long>(static_cast<unsigned int>(__shfl_sync(0xffffffffu, h1, 3))) << 32) |
+            static_cast<unsigned int>(__shfl_sync(0xffffffffu, h1, 2)));
+        norm = __shfl_sync(0xffffffffu, h1, 4) == ACT_F32_NORM;
         ssq_on = norm;  // the first batch of a normalised phase also forms the sums of squares
         cur_ph = ph;
         // the activations of this phase must have been written (all of them: every batch needs all of K)
-        ok = wait_deps(P->act_dep, P->act_need, P->n_act_deps, sp.counters, status, lane);
+        {
+          TR_T0();
+          // lane i polls dependency i (words 6.. = counter index, 12.. = required value)
+          const int nd = __shfl_sync(0xffffffffu, h1, 5);
+          const int dep_i = __shfl_sync(0xffffffffu, h1, 6 + (lane < kStackMaxDeps ? lane : 0));
+          const int need_i = __shfl_sync(0xffffffffu, h1, 12 + (lane < kStackMaxDeps ? lane : 0));
+          bool okd = true;
+          if (lane < nd) okd = wait_global_ge(sp.counters + dep_i, need_i, status);
+          ok = __all_sync(0xffffffffu, okd);
+          TR_ADD(sdeps);
+        }
         if (!ok) break;
       }
       // chunk by chunk, one chunk ahead of the consumers: the raw values are loaded into registers
       // before the buffer is handed back (act_free)
       for (int ch = 0; ch < nchunk; ++ch, ++r) {
         load_rows(ch, 0);
-        ok = __all_sync(0xffffffffu, wait_mbar(act_free, (r & 1) ^ 1u, status));
+        {
+          TR_T0();
+          ok = __all_sync(0xffffffffu, wait_mbar(act_free, (r & 1) ^ 1u, status));
+          TR_ADD(sfree);
+        }
         if (!ok) break;
         store_rows(0);
         if (!PACKED && batch > 4) {
@@ -818,6 +1096,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       if (!ok) break;
     }
     if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
+#ifdef DS_TRACE
+    tr_stotal = clock64() - tr_sstart;
+    if (warp == 8 && lane == 0) {
+      TR_OUT(8, stotal);
+      TR_OUT(9, sdeps);
+      TR_OUT(10, sfree);
+      TR_OUT(11, sq);
+    }
+#endif
     return;
   }
 
@@ -908,6 +1195,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
 bool g_stack_usable = false;
 
 }  // namespace
+
+#ifdef DS_TRACE
+extern "C" int ladder_debug_read_stack_trace(unsigned long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_stack_trace, sizeof(g_stack_trace)) == cudaSuccess ? 0 : 1;
+}
+extern "C" int ladder_debug_read_phase_trace(unsigned long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_phase_trace, sizeof(g_phase_trace)) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 cudaError_t decode_stack_init(int sm_count, bool* usable) {
   *usable = false;

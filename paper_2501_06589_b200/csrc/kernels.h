@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 
 #include "decode_schedule.h"
@@ -72,18 +73,34 @@ cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stre
 // before it touches data another SM produced.
 constexpr int kStackMaxDeps = 6;
 constexpr int kStackMaxPhases = 1023;
-struct StackPhase {
-  SmallMParams p;
+constexpr int kStackRounds = 10;
+struct alignas(128) StackPhase {
+  // ---- first 128 bytes: what the producer and the consumers need (one cache line)
+  const __nv_bfloat16* W;
+  int K;
   int n_units;   // N / 8
   int nchunk;    // ceil(K / 2048)
-  int work_idx;  // claim counter
+  int work_idx;  // claim counter (dynamic claims only)
   int done_idx;  // units finished (epilogue written and fenced)
-  Schedule sched;
+  int n_static;  // claims dealt out statically, claim i to CTA i mod grid
+  int n_claims;  // all claims
+  int sched_n;   // rounds: count[r] claims of size[r] consecutive units
+  int count[kStackRounds], size[kStackRounds];
+  int pad0[2];
+  // ---- second 128 bytes: the stagers' view and the dependencies
+  const float* act;             // fp32 [batch, K]
+  const __nv_bfloat16* gain;    // RMSNorm gain or NULL
+  int act_mode;
   // counters[dep] >= need must hold before the activations are read ...
   int n_act_deps, act_dep[kStackMaxDeps], act_need[kStackMaxDeps];
   // ... and before the first epilogue (addend read, output buffer overwritten)
   int n_epi_deps, epi_dep[kStackMaxDeps], epi_need[kStackMaxDeps];
+  int pad1[1];
+  // ---- the epilogue description (finishers)
+  SmallMParams p;
 };
+static_assert(offsetof(StackPhase, act) == 128, "producer view must be exactly one line");
+static_assert(offsetof(StackPhase, p) == 256, "stager view must be exactly one line");
 struct StackAttn {
   DecodeAttnParams a;  // n_splits = stride of the scratch layout; the live split count comes from kv_len
   int n_deps, dep[kStackMaxDeps], need[kStackMaxDeps];      // before the split units (q, K, V written; scratch free)

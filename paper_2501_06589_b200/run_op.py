@@ -4,7 +4,8 @@ small, self-ending workload to put under `ncu` (or to time with CUDA events).
     python -m paper_2501_06589_b200.run_op gate_up --config 70b --layers 2 --iters 2
 
 ops: qkv, wo, gate_up, down, lm_head (weight-streaming GEMMs), attn (split-KV decode attention),
-     prefill_gemm, prefill_attn.  Each launch uses a different layer's weights, so nothing is
+     prefill_gemm, prefill_attn, stack (whole decode steps of a model cut to --layers layers: the
+     persistent layer-stack kernel, or with --multi-kernel the per-GEMM schedule).  Each launch uses a different layer's weights, so nothing is
      served from L2.  Prints one line with the mean time per launch and the achieved GB/s or TFLOP/s.
 """
 from __future__ import annotations
@@ -26,6 +27,7 @@ def main():
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--kv-len", type=int, default=None)
     ap.add_argument("--tokens", type=int, default=4096, help="M of the prefill GEMM")
+    ap.add_argument("--multi-kernel", action="store_true", help="stack: use the per-GEMM schedule")
     a = ap.parse_args()
     build.build()
     B.lib()
@@ -34,6 +36,9 @@ def main():
     d, F, Hq, Hkv, Dh, V = s.d_model, s.d_ff, s.n_q_heads, s.n_kv_heads, s.head_dim, s.vocab_size
     L = a.layers
     dev = "cuda"
+
+    if a.op == "stack":
+        return run_stack(a, s, bsz)
 
     def w(rows, cols):
         return [(torch.randn(rows, cols, device=dev) * 0.02).to(torch.bfloat16) for _ in range(L)]
@@ -101,6 +106,39 @@ def main():
     ms = e0.elapsed_time(e1) / (a.iters * L)
     rate = f"{nbytes / ms / 1e6:.0f} GB/s" if nbytes else f"{flops / ms / 1e9:.1f} TFLOP/s"
     print(f"{a.op} [{a.config}, batch {bsz}]: {ms * 1e3:.2f} us per launch, {rate}")
+
+
+def run_stack(a, s, bsz):
+    """Decode steps of the model cut to a.layers layers, KV length from the configuration."""
+    s = synth.replace(s, n_layers=a.layers, layer_is_ladder=None if s.layer_is_ladder is None
+                      else tuple(s.layer_is_ladder[:a.layers]))
+    w = synth.make_weights(s, device="cuda")
+    S = a.kv_len or s.prompt_len
+    steps = a.iters + 3
+    model = B.Model(w, bsz, S + steps + 1, bsz * min(S, 256))
+    if a.multi_kernel:
+        model.set_persistent(False)
+    cache = B.KVCache(s, bsz, S + steps + 1)
+    cache.k.normal_()                                 # a synthetic prefix instead of a prompt pass
+    cache.v.normal_()
+    cache.seq_lens.fill_(S)
+    model.set_position(S)
+    nxt = torch.from_numpy(synth.make_tokens(s, bsz, 1)[:, 0].copy()).cuda()
+    for _ in range(3):
+        model.decode_step(cache, nxt, next_tokens=nxt)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(a.iters):
+        model.decode_step(cache, nxt, next_tokens=nxt)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / a.iters
+    nbytes = s.decode_step_bytes(S + 3 + a.iters // 2, bsz)
+    print(f"stack [{a.config}, {a.layers} layers, batch {bsz}, kv {S}, "
+          f"{'multi-kernel' if a.multi_kernel else 'persistent'}]: {ms * 1e3:.1f} us per step, "
+          f"{nbytes / ms / 1e6:.0f} GB/s, status {model.device_status()}")
+    model.close()
 
 
 if __name__ == "__main__":

@@ -76,7 +76,8 @@ struct ladder_model {
   GraphKey graph_key;
   int64_t graph_kernels = 0;
   // persistent layer-stack kernel (one cooperative launch per decode step, batch <= 8)
-  bool stack_ok = false;   // usable on this device
+  bool stack_ok = false;   // usable on this device and worthwhile for this model
+  int stack_begin = 0;     // first layer run by the persistent kernel (layers below: one kernel per GEMM)
   int use_stack = 1;
   GraphKey stack_key;      // what the uploaded phase list was built for
   bool stack_built = false;
@@ -190,8 +191,10 @@ struct Enqueue {
 };
 
 // One decode step: enqueue every kernel on sA (attention modules, head) and sB (MLP modules).
+// l_end < n_layers: only the embedding and layers [0, l_end) (the rest of the step is run by the persistent kernel).
 cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int batch,
-                           const ladder_outputs_t* out, cudaStream_t sA, cudaStream_t sB, int64_t* n_kernels) {
+                           const ladder_outputs_t* out, cudaStream_t sA, cudaStream_t sB, int64_t* n_kernels,
+                           int l_end = -1) {
   const ladder_config_t& c = m->cfg;
   Enqueue q{m, sA, sB, sA != sB};
   const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff;
@@ -234,7 +237,8 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
     if (s == 1) b_joined = true;
   };
 
-  for (int l = 0; l < c.n_layers; ++l) {
+  if (l_end < 0) l_end = c.n_layers;
+  for (int l = 0; l < l_end; ++l) {
     const bool lad = m->is_ladder[l] != 0;
     // ---------------- attention module (module index 2l+1) on stream A
     {
@@ -334,6 +338,11 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       q.gemm(1, o, lad);
       q.record(1, m->ev[mod]);
     }
+  }
+  if (l_end < c.n_layers) {  // prefix only: stream A joins stream B, the persistent kernel does the rest
+    need(0, 2 * l_end);
+    *n_kernels = q.kernels;
+    return q.err;
   }
   // ---------------- head on stream A (joins stream B)
   need(0, 2 * c.n_layers);
@@ -530,7 +539,7 @@ struct StackBuilder {
 // Returns false (with a reason) when this step cannot be expressed; the caller then uses the
 // multi-kernel schedule.
 bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, float* logits, std::vector<StackPhase>& phases,
-                 std::vector<StackAttn>& attn, int* n_counters) {
+                 std::vector<StackAttn>& attn, int* n_counters, int l_begin) {
   const ladder_config_t& c = m->cfg;
   const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff;
   const size_t layer_elems = static_cast<size_t>(c.max_batch) * Hkv * c.max_seq_len * Dh;
@@ -551,7 +560,7 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
     P.gain = p.gain;
     P.act_mode = p.act_mode;
     P.n_units = p.N / 8;
-    P.nchunk = (p.K + 2047) / 2048;
+    P.nchunk = (p.K + kStackChunkK - 1) / kStackChunkK;
     P.work_idx = sb.counter(-1);
     P.done_idx = sb.counter(P.n_units);
     const Schedule sc = make_schedule(P.n_units, m->sm_count);
@@ -585,6 +594,7 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
     const bool lad = m->is_ladder[l] != 0;
     const Router::Route ra = rt.next(lad, 2 * l + 1);
     const Router::Route rm = rt.next(lad, 2 * l + 2);
+    if (l < l_begin) continue;  // run by separate kernels before the launch: only the routing state matters
     __nv_bfloat16* kc = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
     __nv_bfloat16* vc = static_cast<__nv_bfloat16*>(cache->v) + l * layer_elems;
 
@@ -715,7 +725,15 @@ cudaError_t enqueue_decode_stack(ladder_model* m, const ladder_kv_cache_t* cache
   const ladder_config_t& c = m->cfg;
   const int d = c.d_model;
   float* logits = (out && out->logits) ? out->logits : m->logits_ws;
-  cudaError_t e = launch_embed(d_tokens, m->tok_embedding, batch, d, c.vocab_size, m->R[0], m->status, st, false);
+  int64_t k = 2;
+  cudaError_t e;
+  if (m->stack_begin > 0) {  // embedding + the standard-residual layers below the ladder stretch, kernel by kernel
+    int64_t kp = 0;
+    e = enqueue_decode(m, cache, d_tokens, batch, out, st, st, &kp, m->stack_begin);
+    k += kp - 1;
+  } else {
+    e = launch_embed(d_tokens, m->tok_embedding, batch, d, c.vocab_size, m->R[0], m->status, st, false);
+  }
   if (e == cudaSuccess) e = cudaMemsetAsync(m->d_counters, 0, static_cast<size_t>(m->n_counters) * sizeof(int32_t), st);
   StackParams sp = {};
   sp.phases = m->d_phases;
@@ -726,7 +744,6 @@ cudaError_t enqueue_decode_stack(ladder_model* m, const ladder_kv_cache_t* cache
   sp.status = m->status;
   sp.batch = batch;
   if (e == cudaSuccess) e = launch_decode_stack(sp, m->sm_count, st);
-  int64_t k = 2;
   // the final hidden state is the input of the last phase (the LM head)
   Router rt;
   for (int l = 0; l < c.n_layers; ++l) {
@@ -830,6 +847,13 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
     return fail(nullptr, LADDER_ERR_CUDA, std::string("device query: ") + cudaGetErrorString(e));
   }
   if (4 * L + 1 > kStackMaxPhases) m->stack_ok = false;
+  // The persistent kernel pays off where the ladder rule decouples consecutive modules; a standard-
+  // residual layer makes every phase wait for the one before, and there separate kernels with their
+  // dynamically balanced GEMMs are faster.  It therefore runs the ladder layers at the top of the model
+  // (and the LM head); standard layers below them run kernel by kernel.
+  m->stack_begin = L;
+  while (m->stack_begin > 0 && m->is_ladder[m->stack_begin - 1]) --m->stack_begin;
+  if (m->stack_begin == L) m->stack_ok = false;
   if (static_cast<size_t>(smem_optin) < smallm_gemm_smem_bytes(c.max_batch)) {
     delete m;
     return fail(nullptr, LADDER_ERR_UNSUPPORTED, "device has too little shared memory per block (needs sm_100-class)");
@@ -1026,7 +1050,7 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
       std::vector<StackAttn> at;
       int nc = 0;
       float* logits = (out && out->logits) ? out->logits : m->logits_ws;
-      if (!build_stack(m, cache, batch, logits, ph, at, &nc) || nc > m->cap_counters ||
+      if (!build_stack(m, cache, batch, logits, ph, at, &nc, m->stack_begin) || nc > m->cap_counters ||
           static_cast<int>(ph.size()) > 4 * m->cfg.n_layers + 1 || static_cast<int>(at.size()) > m->cfg.n_layers) {
         m->stack_ok = false;  // not expressible: use the multi-kernel schedule from now on
       } else {

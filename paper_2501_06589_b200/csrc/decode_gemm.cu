@@ -89,6 +89,45 @@ __device__ __forceinline__ int mbar_wait_or_stop(uint64_t* bar, uint32_t parity,
   }
 }
 
+// One [16 rows x 2048 k] tile of a consumer warp: its SPW 32-wide K slabs, two 8-row stages as the two
+// row halves of the MMA, software-pipelined over groups of 2 slabs (the shared-memory loads of group
+// i+1 are issued before the MMAs of group i), two accumulator chains.  FAST: every slab lies inside K
+// and both stages are present, so nothing is predicated.
+template <bool FAST>
+__device__ __forceinline__ void slab_loop(float (&acc0)[4], float (&acc1)[4], const uint4 (&bf)[SPW], uint32_t base0,
+                                          uint32_t base1, int cw, int k0, int K, int tig, bool hi_valid) {
+  uint4 lo[2][2], hi[2][2];
+  auto load_group = [&](int grp, uint4(&l)[2], uint4(&h)[2]) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int slab = cw * SPW + grp * 2 + e;
+      if (FAST) {
+        l[e] = lds128(base0 + slab * 64);
+        h[e] = lds128(base1 + slab * 64);
+      } else {
+        const bool kv = (k0 + slab * 32 + tig * 8) < K;
+        l[e] = make_uint4(0, 0, 0, 0);
+        h[e] = make_uint4(0, 0, 0, 0);
+        if (kv) l[e] = lds128(base0 + slab * 64);
+        if (kv && hi_valid) h[e] = lds128(base1 + slab * 64);
+      }
+    }
+  };
+  load_group(0, lo[0], hi[0]);
+#pragma unroll
+  for (int grp = 0; grp < SPW / 2; ++grp) {
+    if (grp + 1 < SPW / 2) load_group(grp + 1, lo[(grp + 1) & 1], hi[(grp + 1) & 1]);
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int j = grp * 2 + e;
+      const uint4& l = lo[grp & 1][e];
+      const uint4& h = hi[grp & 1][e];
+      mma_bf16_16816(acc0, l.x, h.x, l.y, h.y, bf[j].x, bf[j].y);
+      mma_bf16_16816(acc1, l.z, h.z, l.w, h.w, bf[j].z, bf[j].w);
+    }
+  }
+}
+
 #ifdef DG_TRACE
 // per-CTA timeline for tuning builds only: [0] start ns, [1] end ns, [2] SM id, [3] units processed
 __device__ unsigned long long g_trace[148 * 4];
@@ -427,8 +466,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
       if (ok) ok = mbar_wait_bounded(act_full, n_req & 1);
       ++n_req;
 #pragma unroll
-      for (int j = 0; j < SPW; ++j)
-        bf[j] = col_valid ? lds128(act_u32 + g * PITCH + (cw * SPW + j) * 64 + tig * 16) : make_uint4(0, 0, 0, 0);
+      for (int j = 0; j < SPW; ++j) bf[j] = lds128(act_u32 + g * PITCH + (cw * SPW + j) * 64 + tig * 16);
+      if (!col_valid) {  // rows of the buffer beyond the batch hold stale data: their MMA columns are zeroed
+#pragma unroll
+        for (int j = 0; j < SPW; ++j) bf[j] = make_uint4(0, 0, 0, 0);
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(act_free);
 #pragma unroll
@@ -440,33 +482,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
         if (ok && hi_valid) ok = mbar_wait_bounded(&full[st1], ((it + 1) / STAGES) & 1);
         const uint32_t base0 = ring_u32 + st0 * STAGE_BYTES + g * PITCH + tig * 16;
         const uint32_t base1 = ring_u32 + st1 * STAGE_BYTES + g * PITCH + tig * 16;
-        // software pipeline over groups of 2 slabs: the shared-memory loads of group i+1 are issued
-        // before the MMAs of group i
-        uint4 lo[2][2], hi[2][2];
-        auto load_group = [&](int grp, uint4 (&l)[2], uint4 (&h)[2]) {
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int slab = cw * SPW + grp * 2 + e;
-            const bool kv = (k0 + slab * 32 + tig * 8) < p.K;
-            l[e] = make_uint4(0, 0, 0, 0);
-            h[e] = make_uint4(0, 0, 0, 0);
-            if (kv) l[e] = lds128(base0 + slab * 64);
-            if (kv && hi_valid) h[e] = lds128(base1 + slab * 64);
-          }
-        };
-        load_group(0, lo[0], hi[0]);
-#pragma unroll
-        for (int grp = 0; grp < SPW / 2; ++grp) {
-          if (grp + 1 < SPW / 2) load_group(grp + 1, lo[(grp + 1) & 1], hi[(grp + 1) & 1]);
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int j = grp * 2 + e;
-            const uint4& l = lo[grp & 1][e];
-            const uint4& h = hi[grp & 1][e];
-            mma_bf16_16816(acc[rgi][0], l.x, h.x, l.y, h.y, bf[j].x, bf[j].y);
-            mma_bf16_16816(acc[rgi][1], l.z, h.z, l.w, h.w, bf[j].z, bf[j].w);
-          }
-        }
+        // a full chunk with both 8-row halves present (the common case) takes the path without
+        // predicates: a guarded shared-memory load compiles to a branch, and 64 of them per tile
+        // cost more than the loads and MMAs themselves
+        if (hi_valid && k0 + TK <= p.K) slab_loop<true>(acc[rgi][0], acc[rgi][1], bf, base0, base1, cw, k0, p.K, tig, true);
+        else slab_loop<false>(acc[rgi][0], acc[rgi][1], bf, base0, base1, cw, k0, p.K, tig, hi_valid);
         __syncwarp();
         if (lane == 0) {
           mbar_arrive(&empty[st0]);

@@ -6,10 +6,7 @@
 namespace ladder {
 
 constexpr int kSchedMaxPhases = 24;
-#ifndef DS_UMAX
-#define DS_UMAX 10
-#endif
-constexpr int kSchedUnitsMax = DS_UMAX;  // 8-row units per claim at most (5 MMA row groups)
+constexpr int kSchedUnitsMax = 10;  // 8-row units per claim at most (5 MMA row groups)
 
 // Round i hands out count[i] claims of size[i] consecutive units.
 struct Schedule {

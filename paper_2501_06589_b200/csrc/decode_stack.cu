@@ -42,10 +42,10 @@ namespace {
 constexpr int kThreads = 512;
 constexpr int kFin = 96;  // finisher threads
 constexpr int kAux = 128;  // attention threads
-constexpr int TK = 2048;   // K elements per chunk (4 KB of a weight row)
+constexpr int TK = kStackChunkK;   // K elements per chunk
 constexpr int PITCH = TK * 2 + 64;
 constexpr int STAGE_BYTES = 8 * PITCH;
-constexpr int STAGES = 4;
+constexpr int STAGES = 4 * 2048 / TK;
 constexpr int ACT_BYTES = 8 * PITCH;
 constexpr int RG_MAX = kSchedUnitsMax / 2;
 static_assert(2 * RG_MAX == kSchedUnitsMax, "schedule and tile geometry disagree");
@@ -136,17 +136,8 @@ __device__ __forceinline__ bool wait_mbar(uint64_t* bar, uint32_t parity, const 
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t i = 1;; ++i) {
-#if DS_POLL == 1
     if (mbar_try_wait_suspend(bar, parity, 4000u)) return true;
     if ((i & 15u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
-#elif DS_POLL == 2
-    __nanosleep(200);
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
-#else
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
-#endif
   }
 }
 __device__ __forceinline__ bool wait_counter_gt(const volatile int* ctr, int n, const int32_t* status) {
@@ -175,15 +166,14 @@ __device__ __forceinline__ bool wait_deps(const int* dep, const int* need, int n
   return __all_sync(0xffffffffu, ok);
 }
 
-#ifndef DS_POLL
-#define DS_POLL 1
-#endif
 #ifdef DS_TRACE
 // tuning builds only: per CTA, cycles each role spent in its waits during the launch
 // [0] consumer total [1] c:queue [2] c:act_full [3] c:weights [4] c:red_free
 // [5] producer total [6] p:ring full [7] p:claims  [8] stager total [9] s:deps [10] s:act_free [11] s:queue
 // [12] finisher total [13] f:deps [14] f:red_full/norm [15] f:queue
 __device__ unsigned long long g_stack_trace[148 * 16];
+// consumer cycles per phase kind (phase index mod 4): [kind][0] weights wait [1] tile loop [2] act wait [3] all
+__device__ unsigned long long g_kind_trace[148 * 16];
 // consumer timeline: [phase][cta][0] first item of the phase taken up, [1] last item of the phase handed over (ns)
 __device__ unsigned long long g_phase_trace[330 * 148 * 2];
 #define TR_DECL(n) long long tr_##n = 0
@@ -802,6 +792,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
     TR_DECL(cmma);
     TR_DECL(ctotal);
 #ifdef DS_TRACE
+    long long kind_cyc[4][4] = {};
+    long long kind_t0 = clock64();
+    int kind_cur = 0;
+#endif
+#ifdef DS_TRACE
     const long long tr_cstart = clock64();
 #endif
     for (int n = 0;; ++n) {
@@ -820,6 +815,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         cur_ph = ph;
 #ifdef DS_TRACE
         if (warp == 4 && lane == 0 && ph < 330) g_phase_trace[(ph * 148 + blockIdx.x) * 2] = global_timer_ns();
+        {
+          const long long now = clock64();
+          kind_cyc[kind_cur][3] += now - kind_t0;
+          kind_t0 = now;
+          kind_cur = ph & 3;
+        }
 #endif
       }
       const int rows = (id & 15) * 8;
@@ -840,6 +841,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
           TR_T0();
           ok = __all_sync(0xffffffffu, wait_mbar(act_full, n_req & 1, status));
           TR_ADD(cact);
+#ifdef DS_TRACE
+          kind_cyc[kind_cur][2] += clock64() - tr_t0_;
+#endif
         }
         if (!ok) break;
         ++n_req;
@@ -862,6 +866,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
             if (okw && hi_valid) okw = wait_mbar(&full[st1], ((it + 1) / STAGES) & 1, status);
             ok = __all_sync(0xffffffffu, okw);
             TR_ADD(cw);
+#ifdef DS_TRACE
+            kind_cyc[kind_cur][0] += clock64() - tr_t0_;
+#endif
           }
           if (!ok) break;
           const uint32_t base0 = ring_u32 + st0 * STAGE_BYTES + g * PITCH + tig * 16;
@@ -877,6 +884,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
           __syncwarp();
 #ifdef DS_TRACE
           tr_cmma += clock64() - tr_m0;
+          kind_cyc[kind_cur][1] += clock64() - tr_m0;
 #endif
           if (lane == 0) {
             mbar_arrive(&empty[st0]);
@@ -917,6 +925,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       TR_OUT(2, cact);
       TR_OUT(3, cw);
       TR_OUT(4, cmma);
+      for (int k = 0; k < 4; ++k)
+        for (int j = 0; j < 4; ++j) g_kind_trace[blockIdx.x * 16 + k * 4 + j] = static_cast<unsigned long long>(kind_cyc[k][j]);
     }
 #endif
     return;
@@ -945,13 +955,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
 #pragma unroll
     for (int b = 0; b < 8; ++b) ssq[b] = 0.f;
 
-    F8 x[4][2];
-    uint4 gq[2];
-    bool kv[2];
+    constexpr int SU = TK / 1024;  // 1024-element sub-blocks per chunk (128 threads x 8 elements each)
+    F8 x[4][SU];
+    uint4 gq[SU];
+    bool kv[SU];
     auto load_rows = [&](int ch, int round) {
       const int k0 = ch * TK;
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
+      for (int u = 0; u < SU; ++u) {
         const int k = k0 + (st + u * 128) * 8;
         kv[u] = k < K;
         gq[u] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);  // gain 1.0
@@ -960,7 +971,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
+        for (int u = 0; u < SU; ++u) {
           const int b = round * 4 + i;
           x[i][u].a = x[i][u].b = make_float4(0, 0, 0, 0);
           if (kv[u] && b < batch) {
@@ -977,7 +988,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         const int b = round * 4 + i;
         if (b >= batch) break;
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
+        for (int u = 0; u < SU; ++u) {
           float y[8] = {x[i][u].a.x, x[i][u].a.y, x[i][u].a.z, x[i][u].a.w,
                         x[i][u].b.x, x[i][u].b.y, x[i][u].b.z, x[i][u].b.w};
           if (norm) {
@@ -1199,6 +1210,9 @@ bool g_stack_usable = false;
 #ifdef DS_TRACE
 extern "C" int ladder_debug_read_stack_trace(unsigned long long* host_out) {
   return cudaMemcpyFromSymbol(host_out, g_stack_trace, sizeof(g_stack_trace)) == cudaSuccess ? 0 : 1;
+}
+extern "C" int ladder_debug_read_kind_trace(unsigned long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_kind_trace, sizeof(g_kind_trace)) == cudaSuccess ? 0 : 1;
 }
 extern "C" int ladder_debug_read_phase_trace(unsigned long long* host_out) {
   return cudaMemcpyFromSymbol(host_out, g_phase_trace, sizeof(g_phase_trace)) == cudaSuccess ? 0 : 1;

@@ -74,12 +74,13 @@ cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stre
 constexpr int kStackMaxDeps = 6;
 constexpr int kStackMaxPhases = 1023;
 constexpr int kStackRounds = 10;
+constexpr int kStackChunkK = 2048;  // K elements per chunk of the persistent kernel (4 KB of a weight row)
 struct alignas(128) StackPhase {
   // ---- first 128 bytes: what the producer and the consumers need (one cache line)
   const __nv_bfloat16* W;
   int K;
   int n_units;   // N / 8
-  int nchunk;    // ceil(K / 2048)
+  int nchunk;    // ceil(K / kStackChunkK)
   int work_idx;  // claim counter (dynamic claims only)
   int done_idx;  // units finished (epilogue written and fenced)
   int n_static;  // claims dealt out statically, claim i to CTA i mod grid

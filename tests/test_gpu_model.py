@@ -63,8 +63,9 @@ def check_generation(B, shape, steps, dtype, gains="ones", schedule=None, min_ag
     if schedule is not None:        # a multi-kernel schedule (n_streams, graph, pdl); default: the persistent kernel
         model.set_persistent(False)
         model.set_schedule(*schedule)
-    elif bsz <= 8:
-        assert model.persistent_active()
+    elif bsz <= 8:             # the persistent kernel runs the ladder layers at the top of the model
+        top_is_ladder = shape.layer_is_ladder is None or bool(shape.layer_is_ladder[-1])
+        assert model.persistent_active() == top_is_ladder
     cache = B.KVCache(shape, bsz, max_seq, fill=CANARY)
     toks, hids = gpu_generate(B, model, cache, prompt, steps)
     assert model.device_status() == 0
@@ -88,13 +89,15 @@ def check_generation(B, shape, steps, dtype, gains="ones", schedule=None, min_ag
     return err, agree, toks, hids, cache
 
 
-@pytest.mark.parametrize("variant", ["ladder", "standard", "hybrid"])
+@pytest.mark.parametrize("variant", ["ladder", "standard", "hybrid", "hybrid_top"])
 def test_tiny_config_full(B, variant):
     s = synth.SHAPES["tiny"]
     if variant == "standard":
         s = s.as_standard()
     elif variant == "hybrid":
         s = synth.replace(s, layer_is_ladder=(0, 1, 1, 0))
+    elif variant == "hybrid_top":      # standard layers run kernel by kernel, the ladder stretch above them persistently
+        s = synth.replace(s, layer_is_ladder=(0, 0, 1, 1))
     err, agree, *_ = check_generation(B, s, 64, np.float64, gains="uniform", batch=4)     # 4 x 65 comparisons
     assert err < HIDDEN_TOL, err
     assert agree >= 0.99, agree

@@ -32,6 +32,11 @@ if ROOT not in sys.path:
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the gate/up decode GEMM, from the ncu
 # capture summarised in profiles/decode_gemm_gate_up_70b_batch4.md (true size, no scaling).
 NCU_TRAFFIC_BYTES = {("70b", 4): 945_259_008}
+# Persistent layer-stack kernel: DRAM traffic / algorithmic bytes of the ncu capture of a 4-layer slice
+# of the 70B shape (profiles/decode_stack_70b_4layers_batch4.md).  A full launch holds 141 GB on the
+# device, too large to capture; traffic grows with the layers like the algorithmic bytes do (every
+# weight byte is read once), so the full launch is scaled by this ratio.
+NCU_STACK_TRAFFIC_RATIO = {("70b", 4): 1.007}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
@@ -197,6 +202,8 @@ def main():
     ap.add_argument("--streams", type=int, default=None)
     ap.add_argument("--graph", type=int, default=None)
     ap.add_argument("--pdl", type=int, default=None)
+    ap.add_argument("--multi-kernel", action="store_true",
+                    help="one kernel per GEMM (two streams, CUDA graph, PDL) instead of the persistent decode kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill-timing", action="store_true")
     args = ap.parse_args()
@@ -234,6 +241,9 @@ def main():
     torch.cuda.synchronize()
     t_gen = time.time() - t0
     model = B.Model(w, bsz, max_seq, bsz * S)
+    if args.multi_kernel:
+        model.set_persistent(False)
+    persistent = model.persistent_active() and bsz <= 8
     if args.streams is not None or args.graph is not None or args.pdl is not None:
         model.set_schedule(2 if args.streams is None else args.streams, 1 if args.graph is None else args.graph,
                            1 if args.pdl is None else args.pdl)
@@ -336,7 +346,7 @@ def main():
                           "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS, "mean_kv_len": mean_kv},
         "clocks": clocks.summary(),
         "device_status": status,
-        "schedule": {"streams": args.streams, "graph": args.graph, "pdl": args.pdl},
+        "schedule": {"persistent": persistent, "streams": args.streams, "graph": args.graph, "pdl": args.pdl},
         "weights_gb": w.nbytes() / 1e9, "weight_gen_s": t_gen,
     }
     if prefill_ms_max:
@@ -347,6 +357,16 @@ def main():
                            "peak_tflops": bf16_peak, "peak_source": peak_src}
     if (shape.name, bsz) in NCU_TRAFFIC_BYTES:
         line["roofline"]["traffic"] = NCU_TRAFFIC_BYTES[(shape.name, bsz)]
+    if persistent:
+        # One launch of the persistent kernel IS the decode step (the embedding gather, the counter reset
+        # and the argmax around it take ~10 us), so the step's device time is its launch duration.
+        line["gemm_kernel"] = line["roofline"]
+        ratio = NCU_STACK_TRAFFIC_RATIO.get((shape.name, bsz))
+        line["roofline"] = {
+            "bound": "hbm", "kernel": "decode_stack_kernel (every GEMM and the attention of a decode step, one launch)",
+            "achieved": step_gbs, "peak": hbm_peak, "peak_source": peak_src, "unit": "GB/s",
+            "frac": step_gbs / hbm_peak, "bytes_per_launch": step_bytes, "ms_per_launch": ms_per_step,
+            "traffic": None if ratio is None else step_bytes * ratio}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(shape, w, S)
     if rank == 0:

@@ -36,7 +36,7 @@ NCU_TRAFFIC_BYTES = {("70b", 4): 945_259_008}
 # of the 70B shape (profiles/decode_stack_70b_4layers_batch4.md).  A full launch holds 141 GB on the
 # device, too large to capture; traffic grows with the layers like the algorithmic bytes do (every
 # weight byte is read once), so the full launch is scaled by this ratio.
-NCU_STACK_TRAFFIC_RATIO = {("70b", 4): 1.007}
+NCU_STACK_TRAFFIC_RATIO = {("70b", 4): 1.001}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0

@@ -130,6 +130,17 @@ ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, 
 ladder_status_t ladder_model_set_persistent(ladder_model_t* m, int32_t on);
 int32_t ladder_model_persistent_active(const ladder_model_t* m);
 
+/* Host only (no GPU needed): describes the phase list the persistent kernel would execute for this
+ * configuration, batch and SM count, as int32 words, for inspection and tests.
+ *   header: n_phases, n_attention_nodes, n_counters, first_layer_in_kernel, ok
+ *   per phase (56 words): kind (0 QKV, 1 gate/up, 2 Wo, 3 down, 4 LM head), layer, N, K, n_units, n_static, n_claims,
+ *     claim_counter, done_counter, n_rounds, count[10], size[10], n_act_deps, act_dep[6], act_need[6],
+ *     n_epi_deps, epi_dep[6], epi_need[6]
+ *   per attention node (29 words): layer, split_counter, merge_counter, n_deps, dep[6], need[6], n_merge_deps,
+ *     merge_dep[6], merge_need[6]
+ * Returns the number of words written, -(words needed) if cap is too small, -1 on a bad argument. */
+int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_count, int32_t* out, int32_t cap);
+
 /* With two streams, the GEMMs of a ladder layer's attention module and MLP module can be run side by side on
  * disjoint sets of SMs (each GEMM is a persistent kernel that claims its work dynamically, so it runs
  * on any number of CTAs).  sms_attention_stream: -1 = no split, every GEMM launches on all SMs (default:

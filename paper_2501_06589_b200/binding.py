@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libladder.so")
 
 EXPORTS = [
-    "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_model_set_sm_split", "ladder_model_set_persistent", "ladder_model_persistent_active",
+    "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_model_set_sm_split", "ladder_model_set_persistent", "ladder_model_persistent_active", "ladder_stack_plan",
     "ladder_prefill",
     "ladder_decode_step", "ladder_decode_step_host", "ladder_prefill_host", "ladder_set_position",
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
@@ -78,6 +78,8 @@ def lib() -> C.CDLL:
         L.ladder_model_set_persistent.argtypes = [C.c_void_p, C.c_int32]
         L.ladder_model_persistent_active.argtypes = [C.c_void_p]
         L.ladder_model_persistent_active.restype = C.c_int32
+        L.ladder_stack_plan.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32]
+        L.ladder_stack_plan.restype = C.c_int32
         L.ladder_prefill.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32, C.c_int32,
                                      C.POINTER(ladder_outputs_t), C.c_void_p]
         L.ladder_decode_step.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32,
@@ -143,6 +145,33 @@ def make_config(shape: ModelShape, max_batch: int, max_seq_len: int, max_prefill
                           C.cast(mask, C.POINTER(C.c_uint8)))
     cfg._keep = mask
     return cfg
+
+
+def stack_plan(shape: ModelShape, batch: int, max_seq_len: int, sm_count: int = 148):
+    """Phase list of the persistent decode kernel for this configuration (host only, no GPU needed)."""
+    cfg = make_config(shape, batch, max_seq_len)
+    cap = 8 + 56 * (4 * shape.n_layers + 1) + 29 * shape.n_layers
+    buf = (C.c_int32 * cap)()
+    n = lib().ladder_stack_plan(C.byref(cfg), batch, sm_count, buf, cap)
+    if n < 0:
+        raise RuntimeError(f"ladder_stack_plan failed ({n})")
+    w = list(buf[:n])
+    n_ph, n_at, n_ctr, begin, ok = w[:5]
+    pos, phases, attn = 5, [], []
+    for _ in range(n_ph):
+        r = w[pos:pos + 56]
+        pos += 56
+        phases.append(dict(kind=r[0], layer=r[1], N=r[2], K=r[3], n_units=r[4], n_static=r[5], n_claims=r[6],
+                           work=r[7], done=r[8], rounds=list(zip(r[10:10 + r[9]], r[20:20 + r[9]])),
+                           act_deps=list(zip(r[31:31 + r[30]], r[37:37 + r[30]])),
+                           epi_deps=list(zip(r[44:44 + r[43]], r[50:50 + r[43]]))))
+    for _ in range(n_at):
+        r = w[pos:pos + 29]
+        pos += 29
+        attn.append(dict(layer=r[0], split=r[1], merge=r[2], deps=list(zip(r[4:4 + r[3]], r[10:10 + r[3]])),
+                         merge_deps=list(zip(r[17:17 + r[16]], r[23:23 + r[16]]))))
+    assert pos == n
+    return dict(phases=phases, attn=attn, n_counters=n_ctr, first_layer=begin, ok=bool(ok))
 
 
 class KVCache:

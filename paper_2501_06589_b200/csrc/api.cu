@@ -536,6 +536,13 @@ struct StackBuilder {
   }
 };
 
+// First layer of the ladder stretch at the top of the model (n_layers if the top layer is standard).
+int stack_first_layer(const std::vector<uint8_t>& is_ladder) {
+  int b = static_cast<int>(is_ladder.size());
+  while (b > 0 && is_ladder[b - 1]) --b;
+  return b;
+}
+
 // Returns false (with a reason) when this step cannot be expressed; the caller then uses the
 // multi-kernel schedule.
 bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, float* logits, std::vector<StackPhase>& phases,
@@ -548,9 +555,12 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
   phases.clear();
   attn.clear();
 
-  auto add_gemm = [&](SmallMParams p, const void* act_buf, const void* add_buf, const void* out0, const void* out1,
-                      const void* out2) {
+  int cur_layer = 0;
+  auto add_gemm = [&](int kind, SmallMParams p, const void* act_buf, const void* add_buf, const void* out0,
+                      const void* out1, const void* out2) {
     StackPhase P = {};
+    P.kind = kind;
+    P.layer = cur_layer;
     p.batch = batch;
     p.status = m->status;
     P.p = p;
@@ -595,6 +605,7 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
     const Router::Route ra = rt.next(lad, 2 * l + 1);
     const Router::Route rm = rt.next(lad, 2 * l + 2);
     if (l < l_begin) continue;  // run by separate kernels before the launch: only the routing state matters
+    cur_layer = l;
     __nv_bfloat16* kc = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
     __nv_bfloat16* vc = static_cast<__nv_bfloat16*>(cache->v) + l * layer_elems;
 
@@ -617,7 +628,7 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
       p.qkv.n_kv_heads = Hkv;
       p.qkv.head_dim = Dh;
       p.qkv.max_seq_len = c.max_seq_len;
-      add_gemm(p, m->R[ra.in], nullptr, m->q_f32, kc, vc);
+      add_gemm(0, p, m->R[ra.in], nullptr, m->q_f32, kc, vc);
       // the attention of this layer, on the attention warps
       StackAttn A = {};
       A.a.q = m->q_f32;
@@ -661,7 +672,7 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
       p.epi_mode = EPI_RESID;
       p.addend = m->R[ra.add];
       p.out = m->R[ra.dst];
-      add_gemm(p, m->o_dec, m->R[ra.add], m->R[ra.dst], nullptr, nullptr);
+      add_gemm(2, p, m->o_dec, m->R[ra.add], m->R[ra.dst], nullptr, nullptr);
     };
     auto gate_up = [&]() {
       SmallMParams p = {};
@@ -674,7 +685,7 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
       p.eps = c.rms_eps;
       p.epi_mode = EPI_SWIGLU;
       p.out = m->h_dec;
-      add_gemm(p, m->R[rm.in], nullptr, m->h_dec, nullptr, nullptr);
+      add_gemm(1, p, m->R[rm.in], nullptr, m->h_dec, nullptr, nullptr);
     };
     auto down = [&]() {
       SmallMParams p = {};
@@ -686,7 +697,7 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
       p.epi_mode = EPI_RESID;
       p.addend = m->R[rm.add];
       p.out = m->R[rm.dst];
-      add_gemm(p, m->h_dec, m->R[rm.add], m->R[rm.dst], nullptr, nullptr);
+      add_gemm(3, p, m->h_dec, m->R[rm.add], m->R[rm.dst], nullptr, nullptr);
     };
     // The MLP module of a ladder layer reads x_{m-2}, which exists before the attention module of the
     // same layer has produced anything -- unless this is the first ladder layer after a standard one,
@@ -713,7 +724,8 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
     h.eps = c.rms_eps;
     h.epi_mode = EPI_PLAIN;
     h.out = logits;
-    add_gemm(h, m->R[rt.cur], nullptr, logits, nullptr, nullptr);
+    cur_layer = c.n_layers;
+    add_gemm(4, h, m->R[rt.cur], nullptr, logits, nullptr, nullptr);
   }
   *n_counters = static_cast<int>(sb.need.size());
   return !sb.overflow && static_cast<int>(phases.size()) <= kStackMaxPhases;
@@ -851,8 +863,7 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   // residual layer makes every phase wait for the one before, and there separate kernels with their
   // dynamically balanced GEMMs are faster.  It therefore runs the ladder layers at the top of the model
   // (and the LM head); standard layers below them run kernel by kernel.
-  m->stack_begin = L;
-  while (m->stack_begin > 0 && m->is_ladder[m->stack_begin - 1]) --m->stack_begin;
+  m->stack_begin = stack_first_layer(m->is_ladder);
   if (m->stack_begin == L) m->stack_ok = false;
   if (static_cast<size_t>(smem_optin) < smallm_gemm_smem_bytes(c.max_batch)) {
     delete m;
@@ -995,6 +1006,73 @@ ladder_status_t ladder_set_position(ladder_model_t* m, int32_t len) {
 }
 
 int64_t ladder_kernel_launches(const ladder_model_t* m) { return m ? m->launches : 0; }
+
+int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_count, int32_t* out, int32_t cap) {
+  if (!cfg || !out || cap < 4 || batch < 1 || sm_count < 1) return -1;
+  if (cfg->struct_size != sizeof(ladder_config_t) || check_shape(*cfg)) return -1;
+  // a model object that owns nothing: every buffer is a distinct made-up address, never dereferenced
+  ladder_model m;
+  m.cfg = *cfg;
+  const int L = cfg->n_layers;
+  m.is_ladder.assign(L, 1);
+  if (cfg->layer_is_ladder)
+    for (int l = 0; l < L; ++l) m.is_ladder[l] = cfg->layer_is_ladder[l] ? 1 : 0;
+  m.sm_count = sm_count;
+  m.attn_splits = decode_attention_splits(cfg->max_batch, cfg->n_kv_heads, cfg->max_seq_len, sm_count);
+  uintptr_t next = 0x10000000u;
+  auto fake = [&]() {
+    next += 0x1000000u;
+    return next;
+  };
+  m.R[0] = reinterpret_cast<float*>(fake());
+  m.R[1] = reinterpret_cast<float*>(fake());
+  m.q_f32 = reinterpret_cast<float*>(fake());
+  m.o_dec = reinterpret_cast<float*>(fake());
+  m.h_dec = reinterpret_cast<float*>(fake());
+  m.attn_scratch = reinterpret_cast<float*>(fake());
+  m.status = reinterpret_cast<int32_t*>(fake());
+  m.rope = reinterpret_cast<float2*>(fake());
+  m.lm_head = reinterpret_cast<const __nv_bfloat16*>(fake());
+  m.final_norm = reinterpret_cast<const __nv_bfloat16*>(fake());
+  for (auto* v : {&m.attn_norm, &m.w_qkv, &m.w_o, &m.mlp_norm, &m.w_gate_up, &m.w_down}) {
+    v->resize(L);
+    for (int l = 0; l < L; ++l) (*v)[l] = reinterpret_cast<const __nv_bfloat16*>(fake());
+  }
+  ladder_kv_cache_t cache;
+  cache.k = reinterpret_cast<void*>(fake() + 0x40000000u);
+  cache.v = reinterpret_cast<void*>(fake() + 0x80000000u);
+  cache.seq_lens = reinterpret_cast<int32_t*>(fake());
+  std::vector<StackPhase> ph;
+  std::vector<StackAttn> at;
+  int nc = 0;
+  const int begin = stack_first_layer(m.is_ladder);
+  const bool ok = build_stack(&m, &cache, batch, reinterpret_cast<float*>(fake()), ph, at, &nc, begin);
+  m.ev.clear();
+  std::vector<int32_t> o = {static_cast<int32_t>(ph.size()), static_cast<int32_t>(at.size()), nc, begin, ok ? 1 : 0};
+  for (const StackPhase& P : ph) {
+    o.insert(o.end(), {P.kind, P.layer, P.p.N, P.K, P.n_units, P.n_static, P.n_claims, P.work_idx, P.done_idx, P.sched_n});
+    for (int r = 0; r < kStackRounds; ++r) o.push_back(P.count[r]);
+    for (int r = 0; r < kStackRounds; ++r) o.push_back(P.size[r]);
+    o.push_back(P.n_act_deps);
+    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(P.act_dep[i]);
+    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(P.act_need[i]);
+    o.push_back(P.n_epi_deps);
+    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(P.epi_dep[i]);
+    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(P.epi_need[i]);
+  }
+  int li = 0;
+  for (const StackAttn& A : at) {
+    o.insert(o.end(), {begin + li++, A.split_done, A.merge_done, A.n_deps});
+    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(A.dep[i]);
+    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(A.need[i]);
+    o.push_back(A.n_mdeps);
+    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(A.mdep[i]);
+    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(A.mneed[i]);
+  }
+  if (static_cast<int>(o.size()) > cap) return -static_cast<int32_t>(o.size());
+  memcpy(out, o.data(), o.size() * sizeof(int32_t));
+  return static_cast<int32_t>(o.size());
+}
 
 ladder_status_t ladder_device_status(ladder_model_t* m, int32_t* flags, void* cuda_stream) {
   if (!m || !flags) return LADDER_ERR_INVALID_ARG;

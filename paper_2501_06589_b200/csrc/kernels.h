@@ -87,7 +87,8 @@ struct alignas(128) StackPhase {
   int n_claims;  // all claims
   int sched_n;   // rounds: count[r] claims of size[r] consecutive units
   int count[kStackRounds], size[kStackRounds];
-  int pad0[2];
+  int kind;      // 0 QKV, 1 gate/up, 2 Wo, 3 down, 4 LM head (description only)
+  int layer;
   // ---- second 128 bytes: the stagers' view and the dependencies
   const float* act;             // fp32 [batch, K]
   const __nv_bfloat16* gain;    // RMSNorm gain or NULL

@@ -20,7 +20,7 @@
 //
 // Warp roles (512 threads, four warpgroups so that registers can be moved between them):
 //   warp 0        producer: claims batches, publishes them in a shared-memory queue, streams the
-//                 weights as [8 rows x 2048 k] tiles (eight 4 KB bulk async copies) into a 4-stage ring
+//                 weights as [8 rows x 2048 k] tiles (eight 4 KB bulk async copies) into a 5-stage ring
 //   warps 1-3     finishers: K-split reduction, 1/rms, epilogue (residual add / SwiGLU / rotary + KV
 //                 append), then publish the finished units (fence + release add)
 //   warps 4-7     consumers: mma.sync m16n8k16 with the weights as the A operand (see decode_gemm.cu)
@@ -45,7 +45,7 @@ constexpr int kAux = 128;  // attention threads
 constexpr int TK = kStackChunkK;   // K elements per chunk
 constexpr int PITCH = TK * 2 + 64;
 constexpr int STAGE_BYTES = 8 * PITCH;
-constexpr int STAGES = 4 * 2048 / TK;
+constexpr int STAGES = 5;  // odd is fine: tiles are consumed as pairs of consecutive ring slots
 constexpr int ACT_BYTES = 8 * PITCH;
 constexpr int RG_MAX = kSchedUnitsMax / 2;
 static_assert(2 * RG_MAX == kSchedUnitsMax, "schedule and tile geometry disagree");
@@ -70,7 +70,7 @@ static_assert(sizeof(SmallMParams) <= FINP_BYTES, "phase parameter copy too smal
 static_assert((3 * QDEPTH + 2) * 4 <= 256, "queue area too small");
 constexpr int OFF_AUX = OFF_FINP + FINP_BYTES;
 constexpr int AUX_PS = 4 * 8 * 16 * 4;
-constexpr int AUX_RED = 4 * 8 * 128 * 4;
+constexpr int AUX_RED = 4 * 2 * 128 * 4;   // [4 warps][2 heads][128] floats per merge round; the merge step reuses it for its weights
 static_assert(AUX_RED >= kMaxSplits * 4, "merge weights do not fit");
 constexpr int AUX_MLS = 4 * 8 * 2 * 4;
 constexpr int AUX_MISC = 128;  // prefix of live splits per sequence [9], merge reductions [8]
@@ -256,7 +256,7 @@ __device__ __forceinline__ void attn_split_unit(const float* q, const __nv_bfloa
   const int kw0 = split * kChunk + warp * 16;
   const float scale = rsqrtf(static_cast<float>(DH));
   float* ps = ps_ + warp * GT * 16;     // [GT][16]
-  float* red = red_;                    // [4][GT][DH]
+  float* red = red_;                    // [4][HR][DH], HR heads per merge round
   float* mls = mls_;                    // [4][GT][2]
 
   uint4 kf[2][KJ];
@@ -367,34 +367,39 @@ __device__ __forceinline__ void attn_split_unit(const float* q, const __nv_bfloa
       }
     }
   }
-#pragma unroll
-  for (int h = 0; h < GT; ++h)
-#pragma unroll
-    for (int d = 0; d < DPL; ++d) red[(warp * GT + h) * DH + lane * DPL + d] = acc[h][d];
-  bar_sync(3, kAux);
-
+  // merge the 4 warps and write the unit's partial, HR heads at a time: the staging array holds only
+  // [4 warps][HR heads][DH] floats (shared memory is needed for the weight ring)
+  constexpr int HR = GT >= 4 ? GT / 4 : 1;
   const int stride = DH + 2;
-  for (int idx = at; idx < GT * DH; idx += kAux) {
-    const int h = idx / DH, d = idx % DH;
-    const float m0 = mls[(0 * GT + h) * 2], m1 = mls[(1 * GT + h) * 2], m2 = mls[(2 * GT + h) * 2],
-                m3 = mls[(3 * GT + h) * 2];
-    const float M = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-    float o = 0.f, ls = 0.f;
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const float mw = mls[(w * GT + h) * 2];
-      const float f = (mw == -INFINITY) ? 0.f : __expf(mw - M);
-      o += f * red[(w * GT + h) * DH + d];
-      ls += f * mls[(w * GT + h) * 2 + 1];
+  for (int h0 = 0; h0 < GT; h0 += HR) {
+#pragma unroll
+    for (int hh = 0; hh < HR; ++hh)
+#pragma unroll
+      for (int d = 0; d < DPL; ++d) red[(warp * HR + hh) * DH + lane * DPL + d] = acc[h0 + hh][d];
+    bar_sync(3, kAux);
+    for (int idx = at; idx < HR * DH; idx += kAux) {
+      const int hh = idx / DH, h = h0 + hh, d = idx % DH;
+      const float m0 = mls[(0 * GT + h) * 2], m1 = mls[(1 * GT + h) * 2], m2 = mls[(2 * GT + h) * 2],
+                  m3 = mls[(3 * GT + h) * 2];
+      const float M = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+      float o = 0.f, ls = 0.f;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const float mw = mls[(w * GT + h) * 2];
+        const float f = (mw == -INFINITY) ? 0.f : __expf(mw - M);
+        o += f * red[(w * HR + hh) * DH + d];
+        ls += f * mls[(w * GT + h) * 2 + 1];
+      }
+      float* dst = scratch + ((static_cast<size_t>(b) * n_q_heads + head0 + h) * stride_splits + split) * stride;
+      dst[d] = o;
+      if (d == 0) {
+        dst[DH] = M;
+        dst[DH + 1] = ls;
+      }
     }
-    float* dst = scratch + ((static_cast<size_t>(b) * n_q_heads + head0 + h) * stride_splits + split) * stride;
-    dst[d] = o;
-    if (d == 0) {
-      dst[DH] = M;
-      dst[DH + 1] = ls;
-    }
+    bar_sync(3, kAux);  // the staging array (and, after the last round, ps / mls) is rewritten next
   }
-  bar_sync(3, kAux);  // the shared arrays are rewritten by the next unit
 }
 
 // Merge of the live splits of one (sequence, head), in split order (same summation order as

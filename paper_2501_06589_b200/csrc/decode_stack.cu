@@ -132,10 +132,15 @@ __device__ __forceinline__ bool bar_and(int id, int count, bool pred) {
 }
 
 // ---- bounded waits; all give up early when another CTA has reported a timeout
+// SLEEP_NS > 0: back off between polls.  Used where a few hundred nanoseconds of wake-up latency do not
+// matter (finishers, stagers): a waiting warp that keeps polling executes instructions, and at this
+// kernel's power draw every instruction costs SM clock.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool wait_mbar(uint64_t* bar, uint32_t parity, const int32_t* status) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t i = 1;; ++i) {
+    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if (mbar_try_wait_suspend(bar, parity, 4000u)) return true;
     if ((i & 15u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
   }
@@ -728,9 +733,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       const int slot = n & 1;
       {
         TR_T0();
-        bool okw = wait_mbar(&red_full[slot], (n >> 1) & 1, status);
+        bool okw = wait_mbar<400>(&red_full[slot], (n >> 1) & 1, status);
         if (!have_rstd)
-          okw = okw && wait_mbar(&norm_ready[norm_cnt & (NORM_RING - 1)], (norm_cnt / NORM_RING) & 1, status);
+          okw = okw && wait_mbar<400>(&norm_ready[norm_cnt & (NORM_RING - 1)], (norm_cnt / NORM_RING) & 1, status);
         ok = bar_and(2, kFin, okw);
         TR_ADD(fred);
       }
@@ -1082,7 +1087,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         load_rows(ch, 0);
         {
           TR_T0();
-          ok = __all_sync(0xffffffffu, wait_mbar(act_free, (r & 1) ^ 1u, status));
+          ok = __all_sync(0xffffffffu, wait_mbar<200>(act_free, (r & 1) ^ 1u, status));
           TR_ADD(sfree);
         }
         if (!ok) break;

@@ -248,6 +248,11 @@ ladder_status_t ladder_op_prefill_gemm(const void* A, const void* A_lo, const vo
  * and TMEM accumulators (default), 1 = warp-level mma.sync kernel (kept as a cross-check). */
 void ladder_set_prefill_gemm_impl(int32_t impl);
 
+/* Decode GEMM for batch 9..64: 0 = tcgen05 kernel (weights as the M side of the MMA, TMA tiles, TMEM accumulators,
+ * equal K-block ranges per CTA with a deterministic fix-up of shared tiles; default), 1 = the earlier mma.sync kernel
+ * (cross-check).  Process-wide; not thread-safe against concurrent launches. */
+void ladder_set_decode_wide_impl(int32_t impl);
+
 /* Causal grouped-query attention of the prefill path for one layer:
  *   q bf16 [batch, seq_len, Hq*Dh] (rotated), q_lo its optional low part; k,v bf16 cache of one layer
  *   as above, rows 0..seq_len-1 valid; o bf16 [batch, seq_len, Hq*Dh], o_lo its low part (given iff

@@ -25,7 +25,7 @@ EXPORTS = [
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
     "ladder_last_error", "ladder_op_smallm_gemm", "ladder_decode_attention_scratch_bytes",
     "ladder_op_decode_attention", "ladder_op_prefill_gemm", "ladder_op_prefill_attention",
-    "ladder_op_decode_attention_noalloc", "ladder_set_prefill_gemm_impl",
+    "ladder_op_decode_attention_noalloc", "ladder_set_prefill_gemm_impl", "ladder_set_decode_wide_impl",
 ]
 
 
@@ -109,6 +109,8 @@ def lib() -> C.CDLL:
                                                          C.c_void_p]
         L.ladder_set_prefill_gemm_impl.restype = None
         L.ladder_set_prefill_gemm_impl.argtypes = [C.c_int32]
+        L.ladder_set_decode_wide_impl.restype = None
+        L.ladder_set_decode_wide_impl.argtypes = [C.c_int32]
         L.ladder_op_prefill_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                              C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ladder_op_prefill_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
@@ -305,6 +307,11 @@ def op_decode_attention_noalloc(q, k, v, kv_len, n_q_heads, n_kv_heads, head_dim
 def set_prefill_gemm_impl(impl: int):
     """0 = tcgen05 kernel (default), 1 = warp-level mma.sync kernel."""
     lib().ladder_set_prefill_gemm_impl(impl)
+
+
+def set_decode_wide_impl(impl: int):
+    """Decode GEMM for batch 9..64: 0 = tcgen05 kernel (default), 1 = the earlier mma.sync kernel."""
+    lib().ladder_set_decode_wide_impl(impl)
 
 
 def op_prefill_gemm(A, W, epi_mode: int, out, addend=None, A_lo=None, out_lo=None):

@@ -802,6 +802,8 @@ const char* ladder_last_error(const ladder_model_t* m) { return m ? m->err.c_str
 
 void ladder_set_prefill_gemm_impl(int32_t impl) { set_prefill_gemm_impl(impl); }
 
+void ladder_set_decode_wide_impl(int32_t impl) { set_decode_wide_impl(impl); }
+
 size_t ladder_kv_cache_bytes(const ladder_config_t* c) {
   if (!c) return 0;
   return static_cast<size_t>(c->n_layers) * c->max_batch * c->n_kv_heads * c->max_seq_len * c->head_dim * 2;

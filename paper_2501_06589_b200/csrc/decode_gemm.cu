@@ -30,6 +30,8 @@
 // Nothing before griddepcontrol.wait depends on the previous kernel (barrier set-up, claiming, the
 // first ring fill), so under programmatic dependent launch the weight stream does not drain
 // between kernels.
+#include <algorithm>
+
 #include "common.cuh"
 #include "decode_schedule.h"
 #include "kernels.h"
@@ -37,9 +39,16 @@
 
 namespace ladder {
 
+// batch 9..64: tcgen05 kernel (default) or the earlier mma.sync kernel (cross-check)
 cudaError_t launch_smallm_gemm_wide(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);
 cudaError_t smallm_gemm_wide_init();
 size_t smallm_gemm_wide_smem_bytes(int batch);
+cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);
+cudaError_t smallm_gemm_wide_tc_init();
+size_t smallm_gemm_wide_tc_smem_bytes(int batch);
+size_t smallm_gemm_wide_tc_scratch_floats(int N, int K, int batch);
+static int g_wide_impl = 0;  // 0 = tcgen05, 1 = mma.sync
+void set_decode_wide_impl(int impl) { g_wide_impl = impl == 1 ? 1 : 0; }
 
 namespace {
 
@@ -548,18 +557,24 @@ cudaError_t smallm_gemm_init() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(decode_gemm_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e == cudaSuccess) e = smallm_gemm_wide_init();
+  if (e == cudaSuccess) e = smallm_gemm_wide_tc_init();
   return e;
 }
 
-size_t smallm_gemm_smem_bytes(int batch) { return batch <= 8 ? SMEM : smallm_gemm_wide_smem_bytes(batch); }
+size_t smallm_gemm_smem_bytes(int batch) {
+  if (batch <= 8) return SMEM;
+  return std::max(smallm_gemm_wide_smem_bytes(batch), smallm_gemm_wide_tc_smem_bytes(batch));
+}
 
 size_t smallm_gemm_scratch_floats(int N, int K, int batch) {
-  (void)N, (void)K, (void)batch;
+  if (batch > 8) return smallm_gemm_wide_tc_scratch_floats(N, K, batch);  // staged activations + shared-tile pieces
   return 0;  // the batch <= 8 kernel keeps full-K sums in registers: no scratch
 }
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
-  if (p.batch > 8) return launch_smallm_gemm_wide(p, stream, pdl, sm_count);
+  if (p.batch > 8)
+    return g_wide_impl == 0 ? launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count)
+                            : launch_smallm_gemm_wide(p, stream, pdl, sm_count);
   if (!p.work) return cudaErrorInvalidValue;
   const int units = p.N >> 3;
   const int grid = units < sm_count ? units : sm_count;

@@ -1,0 +1,564 @@
+// Weight-streaming decode GEMM for batch 9..64 on the 5th-generation tensor cores (tcgen05 / UMMA):
+//   acc[b, n] = sum_k act[b, k] * W[n, k]          W bf16 [N, K], act fp32 [batch, K]
+// "Swapped" operands: a tile of 128 weight rows is the M side of the MMA (A operand, straight from
+// shared memory), the batch is the N side.  The activations are split into a bf16 high and low part
+// (x ~ hi + lo) that sit side by side as 2 x Bp MMA columns (Bp = batch padded to 16 / 32 / 64), so
+// the extra precision costs no extra instruction; their sum is formed in the epilogue.
+//
+// Two kernels per GEMM:
+//   1. wide_stage_kernel: fp32 activations (x gain for RMSNorm) -> bf16 [2 Bp, K] in scratch, 1/rms per row.
+//   2. decode_gemm_wide_tc_kernel: persistent CTAs, one per SM, three roles that meet at mbarriers:
+//        warp 0     TMA producer: per 64-wide K block one [128 rows x 64] box of W (L2 evict-first) and
+//                   one [2 Bp x 64] box of the staged activations (L2-resident), 128-byte swizzle, into a
+//                   6..10-stage ring (20..32 KB per stage, ~100-160 KB of weights in flight per SM);
+//        warp 1     MMA issuer: tcgen05.mma M 128, N 2 Bp, K 16, kind::f16, fp32 accumulators in tensor
+//                   memory (two buffers, so the epilogue of one segment overlaps the MMAs of the next);
+//        warps 2-5  epilogue: tcgen05.ld (a thread owns one weight row and all batch columns), hi + lo,
+//                   1/rms, then residual add (Eq. 1 / Eq. 2) / SwiGLU / rotary + KV append / plain store.
+// Work split: the T row tiles x nkb K blocks are cut into one contiguous range per CTA (equal to within
+// one K block), so every SM streams the same number of bytes whatever N and K are.  A tile whose K
+// range is shared by several CTAs is finished by the one that arrives last: every piece goes to an
+// L2-resident scratch, a ticket per tile counts arrivals, and the last CTA adds the pieces in CTA order
+// (deterministic) and runs the epilogue.
+// Every wait is bounded; on a protocol error the kernel records it, drains and frees its TMEM.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace ladder {
+namespace {
+
+constexpr int BM = 128, BK = 64, UMMA_K = 16;
+constexpr int W_BYTES = BM * BK * 2;  // 16 KB
+constexpr int kWideThreads = 192;
+constexpr int kWideMaxTiles = 2048;   // tickets
+constexpr int kWideMaxCtas = 160;     // partial slots
+
+template <int NP>
+struct WCfg {
+  static constexpr int BP = NP / 2;
+  static constexpr int ACT_BYTES = NP * BK * 2;
+  static constexpr int STAGE_BYTES = W_BYTES + ACT_BYTES;
+  static constexpr int STAGES = (200 * 1024) / STAGE_BYTES;
+  static constexpr int OFF_BARS = STAGES * STAGE_BYTES;  // full[], empty[], tmem_full[2], tmem_empty[2], tmem slot, flag
+  static constexpr int SMEM = OFF_BARS + (2 * STAGES + 4) * 8 + 64 + 1024;
+  static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(NP >> 3) << 17) |
+                                    (static_cast<uint32_t>(BM >> 4) << 24);
+  static_assert(SMEM <= 232448, "shared memory budget");
+};
+
+struct WideArgs {
+  SmallMParams p;
+  int bp;                  // padded batch
+  int tiles, nkb;          // row tiles, K blocks
+  const float* rstd;       // [bp] (ACT_F32_NORM)
+  float* partial;          // [grid][2][bp][128]
+  int32_t* tickets;        // [tiles], zero between launches
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+          smem_u32(dst)),
+      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], "
+      "[%2], %5;" ::"r"(smem_u32(dst)),
+      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand tile of rows x 64 bf16, 128-byte swizzle
+// (rows of 128 bytes, 8-row swizzle atoms of 1024 bytes), tile base 1024-byte aligned.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+
+// ---------------------------------------------------------------- activation staging
+// One CTA per padded batch row: y = x (* gain), hi = bf16(y), lo = bf16(y - hi); rows >= batch are zero.
+__global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const __nv_bfloat16* gain, int norm, float eps,
+                                                         int batch, int bp, int K, __nv_bfloat16* stage, float* rstd) {
+  __shared__ float red[8];
+  const int b = blockIdx.x, tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
+  __nv_bfloat16* hi = stage + static_cast<size_t>(b) * K;
+  __nv_bfloat16* lo = stage + static_cast<size_t>(bp + b) * K;
+  float ssq = 0.f;
+  for (int k = tid * 8; k < K; k += 256 * 8) {
+    float y[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (b < batch) {
+      const float4 a = __ldcg(reinterpret_cast<const float4*>(x + static_cast<size_t>(b) * K + k));
+      const float4 c = __ldcg(reinterpret_cast<const float4*>(x + static_cast<size_t>(b) * K + k + 4));
+      y[0] = a.x, y[1] = a.y, y[2] = a.z, y[3] = a.w, y[4] = c.x, y[5] = c.y, y[6] = c.z, y[7] = c.w;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ssq += y[i] * y[i];
+      if (norm) {
+        const uint4 g = __ldg(reinterpret_cast<const uint4*>(gain + k));
+        y[0] *= bf16_lo(g.x), y[1] *= bf16_hi(g.x), y[2] *= bf16_lo(g.y), y[3] *= bf16_hi(g.y);
+        y[4] *= bf16_lo(g.z), y[5] *= bf16_hi(g.z), y[6] *= bf16_lo(g.w), y[7] *= bf16_hi(g.w);
+      }
+    }
+    uint4 h, l;
+    h.x = pack_bf16x2(y[0], y[1]), h.y = pack_bf16x2(y[2], y[3]), h.z = pack_bf16x2(y[4], y[5]), h.w = pack_bf16x2(y[6], y[7]);
+    l.x = pack_bf16x2(y[0] - bf16_lo(h.x), y[1] - bf16_hi(h.x));
+    l.y = pack_bf16x2(y[2] - bf16_lo(h.y), y[3] - bf16_hi(h.y));
+    l.z = pack_bf16x2(y[4] - bf16_lo(h.z), y[5] - bf16_hi(h.z));
+    l.w = pack_bf16x2(y[6] - bf16_lo(h.w), y[7] - bf16_hi(h.w));
+    *reinterpret_cast<uint4*>(hi + k) = h;
+    *reinterpret_cast<uint4*>(lo + k) = l;
+  }
+  ssq = warp_sum(ssq);
+  if ((tid & 31) == 0) red[tid >> 5] = ssq;
+  __syncthreads();
+  if (tid == 0) {
+    float s = 0.f;
+    for (int w = 0; w < 8; ++w) s += red[w];
+    rstd[b] = norm ? rsqrtf(s / static_cast<float>(K) + eps) : 1.f;
+  }
+}
+
+// ---------------------------------------------------------------- epilogue of one weight row
+// v[j] = finished accumulator of row n and batch row b0 + j.  Lanes of a warp hold consecutive rows,
+// so the (gate, up) and rotary pairs are neighbouring lanes; all lanes take part in the shuffles.
+template <int CB>
+__device__ __forceinline__ void wide_epilogue(const SmallMParams& p, int n, int b0, float (&v)[CB], int lane) {
+  const bool row_ok = n < p.N;
+  if (p.epi_mode == EPI_RESID || p.epi_mode == EPI_PLAIN) {
+    float* out = static_cast<float*>(p.out);
+#pragma unroll
+    for (int j = 0; j < CB; ++j) {
+      const int b = b0 + j;
+      if (b < p.batch && row_ok) {
+        const size_t o = static_cast<size_t>(b) * p.N + n;
+        float r = v[j];
+        if (p.epi_mode == EPI_RESID) r += __ldcg(p.addend + o);
+        out[o] = r;
+      }
+    }
+  } else if (p.epi_mode == EPI_SWIGLU) {
+    float* out = static_cast<float*>(p.out);
+#pragma unroll
+    for (int j = 0; j < CB; ++j) {
+      const int b = b0 + j;
+      const float up = __shfl_down_sync(0xffffffffu, v[j], 1);
+      if (!(lane & 1) && b < p.batch && row_ok) {
+        const float gt = v[j];
+        out[static_cast<size_t>(b) * (p.N >> 1) + (n >> 1)] = gt / (1.f + __expf(-gt)) * up;
+      }
+    }
+  } else if (p.epi_mode == EPI_QKV_ROPE) {
+    const QkvEpilogue& e = p.qkv;
+    const int Dh = e.head_dim, nq = e.n_q_heads * Dh, nk = e.n_kv_heads * Dh;
+#pragma unroll
+    for (int j = 0; j < CB; ++j) {
+      const int b = b0 + j;
+      float v0 = v[j], v1 = __shfl_down_sync(0xffffffffu, v[j], 1);
+      if ((lane & 1) || b >= p.batch || !row_ok) continue;
+      const int pos = e.seq_lens[b];
+      if (pos < 0 || pos >= e.max_seq_len) {
+        if (p.status) atomicOr(p.status, LADDER_DEV_CACHE_OVERFLOW);
+        continue;
+      }
+      if (n < nq + nk) {
+        const float2 cs = e.rope[static_cast<size_t>(pos) * (Dh >> 1) + ((n % Dh) >> 1)];
+        const float a0 = v0 * cs.x - v1 * cs.y, a1 = v0 * cs.y + v1 * cs.x;
+        v0 = a0;
+        v1 = a1;
+      }
+      if (n < nq) {
+        *reinterpret_cast<float2*>(e.q_out_f32 + static_cast<size_t>(b) * nq + n) = make_float2(v0, v1);
+      } else {
+        const int nn = n < nq + nk ? n - nq : n - nq - nk;
+        __nv_bfloat16* cache = n < nq + nk ? e.k_cache : e.v_cache;
+        const size_t off = ((static_cast<size_t>(b) * e.n_kv_heads + nn / Dh) * e.max_seq_len + pos) * Dh + (nn % Dh);
+        *reinterpret_cast<uint32_t*>(cache + off) = pack_bf16x2(v0, v1);
+      }
+    }
+  }
+}
+
+// barrier among the 128 epilogue threads that also ANDs a predicate, so that they leave together
+__device__ __forceinline__ bool epi_bar_and(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 p, %1, 0;\n\t"
+      "bar.red.and.pred q, 1, 128, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r)
+      : "r"(static_cast<uint32_t>(pred))
+      : "memory");
+  return r != 0;
+}
+
+// contiguous split of `total` K-block-tiles over `grid` CTAs: the first `rem` CTAs get one more
+struct Split {
+  int per, rem;
+  __device__ __forceinline__ int start(int c) const { return c * per + min(c, rem); }
+  __device__ __forceinline__ int owner(int x) const {
+    const int big = rem * (per + 1);
+    return x < big ? x / (per + 1) : rem + (x - big) / per;
+  }
+};
+
+template <int NP>
+__global__ void __launch_bounds__(kWideThreads, 1)
+decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap map_w,
+                           const __grid_constant__ CUtensorMap map_act) {
+  using C = WCfg<NP>;
+  constexpr int BP = C::BP, STAGES = C::STAGES;
+  constexpr int CB = BP < 32 ? BP : 32;  // batch columns handled per epilogue pass
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + C::OFF_BARS);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tmem_full = empty + STAGES;
+  uint64_t* tmem_empty = tmem_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const SmallMParams& p = a.p;
+  const int nkb = a.nkb;
+  const int total = a.tiles * nkb;
+  const Split sp = {total / static_cast<int>(gridDim.x), total % static_cast<int>(gridDim.x)};
+  const int my_start = sp.start(blockIdx.x), my_end = sp.start(blockIdx.x + 1);
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&tmem_full[b], 1);
+      mbar_init(&tmem_empty[b], 4);
+    }
+    fence_barrier_init();
+  }
+  if (warp == 1) {  // TMEM: two accumulators of NP fp32 columns x 128 lanes
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "n"(2 * NP)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  pdl_launch_dependents();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const uint64_t pol = l2_policy_evict_first();
+      bool ok = true, waited = false;
+      int it = 0;
+      for (int pos = my_start; pos < my_end && ok;) {
+        const int t = pos / nkb, kb0 = pos - t * nkb, kb1 = min(nkb, kb0 + (my_end - pos));
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          const int s = it % STAGES;
+          ok = mbar_wait_bounded(&empty[s], ((it / STAGES) & 1) ^ 1u);
+          if (!ok) break;
+          uint8_t* st = smem + s * C::STAGE_BYTES;
+          mbar_expect_tx(&full[s], C::STAGE_BYTES);
+          tma_load_2d_hint(st, &map_w, kb * BK, t * BM, &full[s], pol);
+          if (!waited) {  // the staged activations come from the kernel before this one; the weights do not
+            pdl_wait();
+            waited = true;
+          }
+          tma_load_2d(st + W_BYTES, &map_act, kb * BK, 0, &full[s]);
+        }
+        pos += kb1 - kb0;
+      }
+      if (!ok) {
+        if (p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
+        for (int j = 1; j <= STAGES && j <= it; ++j) {  // wait (bounded) for the copies still in flight
+          const int i2 = it - j;
+          mbar_wait_bounded(&full[i2 % STAGES], (i2 / STAGES) & 1);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0, seg = 0;
+      for (int pos = my_start; pos < my_end && ok; ++seg) {
+        const int t = pos / nkb, kb0 = pos - t * nkb, kb1 = min(nkb, kb0 + (my_end - pos));
+        const int ab = seg & 1;
+        ok = mbar_wait_bounded(&tmem_empty[ab], ((seg >> 1) & 1) ^ 1u);  // the epilogue has drained this accumulator
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + ab * NP;
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          const int s = it % STAGES;
+          ok = mbar_wait_bounded(&full[s], (it / STAGES) & 1);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t w_addr = smem_u32(smem + s * C::STAGE_BYTES);
+          const uint64_t dw = smem_desc(w_addr), dact = smem_desc(w_addr + W_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)  // +32 bytes along K inside the swizzled row = +2 in the address field
+            tc_mma(d_tmem, dw + 2 * k, dact + 2 * k, C::IDESC, (kb > kb0 || k > 0) ? 1u : 0u);
+          tc_commit(&empty[s]);  // the stage is free once these MMAs have read it
+        }
+        if (ok) tc_commit(&tmem_full[ab]);
+        pos += kb1 - kb0;
+      }
+      if (!ok && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;   // the TMEM lane quarter this warp may access
+    const int et = tid - 64;  // 0..127
+    const int r = q * 32 + lane;  // row inside the tile
+    bool ok = true;
+    int seg = 0;
+    pdl_wait();  // 1/rms, the addend and the destination belong to earlier kernels
+    for (int pos = my_start; pos < my_end; ++seg) {
+      const int t = pos / nkb, kb0 = pos - t * nkb, kb1 = min(nkb, kb0 + (my_end - pos));
+      pos += kb1 - kb0;
+      const int ab = seg & 1;
+      const bool whole = kb0 == 0 && kb1 == nkb;
+      ok = epi_bar_and(ok && mbar_wait_bounded(&tmem_full[ab], (seg >> 1) & 1));  // all four warps agree
+      if (!ok) break;
+      tc_fence_after();
+      const int n = t * BM + r;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + ab * NP;
+      // where this CTA's piece of a shared tile goes: slot 0 if the tile is the first of its range, else slot 1
+      const int my_slot = (t == my_start / nkb) ? 0 : 1;
+      float* piece = a.partial + (static_cast<size_t>(blockIdx.x) * 2 + my_slot) * BP * BM;
+#pragma unroll 1
+      for (int b0 = 0; b0 < BP; b0 += CB) {
+        float v[CB];
+        if (CB == 16) {
+          uint32_t h[16], l[16];
+          tc_ld16(taddr + b0, h);
+          tc_ld16(taddr + BP + b0, l);
+          tc_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(h[j]) + __uint_as_float(l[j]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < CB; c += 16) {
+            uint32_t h[16], l[16];
+            tc_ld16(taddr + b0 + c, h);
+            tc_ld16(taddr + BP + b0 + c, l);
+            tc_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[c + j] = __uint_as_float(h[j]) + __uint_as_float(l[j]);
+          }
+        }
+        if (whole) {
+          if (p.act_mode == ACT_F32_NORM) {
+#pragma unroll
+            for (int j = 0; j < CB; ++j) v[j] *= a.rstd[b0 + j];
+          }
+          wide_epilogue<CB>(p, n, b0, v, lane);
+        } else {
+#pragma unroll
+          for (int j = 0; j < CB; ++j) piece[(b0 + j) * BM + r] = v[j];
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tmem_empty[ab]);
+      if (whole) continue;
+
+      // ---- a tile shared with other CTAs: publish the piece; the last arrival adds all pieces in CTA
+      // order and finishes the tile
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      const int c_lo = sp.owner(t * nkb), c_hi = sp.owner((t + 1) * nkb - 1);
+      if (et == 0) {
+        const int prev = atomicAdd(a.tickets + t, 1);
+        const int last = prev == c_hi - c_lo;
+        if (last) a.tickets[t] = 0;  // ready for the next launch
+        *last_flag = last;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      const bool last = *last_flag != 0;
+      asm volatile("bar.sync 1, 128;" ::: "memory");  // the flag is rewritten by the next shared tile
+      if (!last) continue;
+      __threadfence();
+#pragma unroll 1
+      for (int b0 = 0; b0 < BP; b0 += CB) {
+        float v[CB];
+#pragma unroll
+        for (int j = 0; j < CB; ++j) v[j] = 0.f;
+        for (int c = c_lo; c <= c_hi; ++c) {
+          const int slot = (t == sp.start(c) / nkb) ? 0 : 1;
+          const float* src = a.partial + (static_cast<size_t>(c) * 2 + slot) * BP * BM;
+#pragma unroll
+          for (int j = 0; j < CB; ++j) v[j] += __ldcg(src + (b0 + j) * BM + r);
+        }
+        if (p.act_mode == ACT_F32_NORM) {
+#pragma unroll
+          for (int j = 0; j < CB; ++j) v[j] *= a.rstd[b0 + j];
+        }
+        wide_epilogue<CB>(p, n, b0, v, lane);
+      }
+    }
+    if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(2 * NP) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- host
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn g_encode_wide = nullptr;
+
+cudaError_t make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
+  const cuuint32_t box[2] = {BK, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = g_encode_wide(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+int padded_batch(int batch) { return batch <= 16 ? 16 : (batch <= 32 ? 32 : 64); }
+
+// scratch layout in floats: [64] 1/rms | [kWideMaxTiles] tickets | staged activations (2 bp x K bf16) | pieces
+size_t stage_offset() { return 64 + kWideMaxTiles; }
+size_t piece_offset(int bp, int K) { return stage_offset() + ((static_cast<size_t>(bp) * K + 3) & ~size_t(3)); }
+
+template <int NP>
+cudaError_t launch_np(const WideArgs& a, const CUtensorMap& mw, const CUtensorMap& ma, int grid, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kWideThreads);
+  cfg.dynamicSmemBytes = WCfg<NP>::SMEM;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the staging kernel is always right before it
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_gemm_wide_tc_kernel<NP>, a, mw, ma);
+}
+
+}  // namespace
+
+cudaError_t smallm_gemm_wide_tc_init() {
+  if (!g_encode_wide) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+    g_encode_wide = reinterpret_cast<EncodeFn>(fn);
+  }
+  cudaError_t e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       WCfg<32>::SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WCfg<64>::SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             WCfg<128>::SMEM);
+  return e;
+}
+
+size_t smallm_gemm_wide_tc_scratch_floats(int N, int K, int batch) {
+  (void)N;
+  const int bp = padded_batch(batch);
+  return piece_offset(bp, K) + static_cast<size_t>(kWideMaxCtas) * 2 * bp * BM;
+}
+
+size_t smallm_gemm_wide_tc_smem_bytes(int batch) {
+  const int bp = padded_batch(batch);
+  return bp == 16 ? WCfg<32>::SMEM : (bp == 32 ? WCfg<64>::SMEM : WCfg<128>::SMEM);
+}
+
+cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
+  if (!g_encode_wide) return cudaErrorNotReady;
+  if (!p.scratch || p.batch < 1 || p.batch > 64 || (p.K & 7) || (p.N & 1)) return cudaErrorInvalidValue;
+  if ((reinterpret_cast<uintptr_t>(p.W) | reinterpret_cast<uintptr_t>(p.scratch)) & 15) return cudaErrorMisalignedAddress;
+  const int bp = padded_batch(p.batch);
+  const int tiles = (p.N + BM - 1) / BM, nkb = (p.K + BK - 1) / BK;
+  if (tiles > kWideMaxTiles || sm_count > kWideMaxCtas) return cudaErrorInvalidValue;
+  float* rstd = p.scratch;
+  int32_t* tickets = reinterpret_cast<int32_t*>(p.scratch + 64);
+  __nv_bfloat16* stage = reinterpret_cast<__nv_bfloat16*>(p.scratch + stage_offset());
+  float* pieces = p.scratch + piece_offset(bp, p.K);
+
+  {  // 1. activations -> bf16 hi + lo, 1/rms
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(bp);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, wide_stage_kernel, static_cast<const float*>(p.act), p.gain,
+                                       p.act_mode == ACT_F32_NORM ? 1 : 0, p.eps, p.batch, bp, p.K, stage, rstd);
+    if (e != cudaSuccess) return e;
+  }
+  CUtensorMap mw, ma;
+  cudaError_t e = make_map(&mw, p.W, p.N, p.K, BM);
+  if (e == cudaSuccess) e = make_map(&ma, stage, 2 * bp, p.K, 2 * bp);
+  if (e != cudaSuccess) return e;
+  WideArgs a = {};
+  a.p = p;
+  a.bp = bp;
+  a.tiles = tiles;
+  a.nkb = nkb;
+  a.rstd = rstd;
+  a.partial = pieces;
+  a.tickets = tickets;
+  const int total = tiles * nkb;
+  const int grid = total < sm_count ? total : sm_count;
+  if (bp == 16) return launch_np<32>(a, mw, ma, grid, stream);
+  if (bp == 32) return launch_np<64>(a, mw, ma, grid, stream);
+  return launch_np<128>(a, mw, ma, grid, stream);
+}
+
+}  // namespace ladder

@@ -49,6 +49,7 @@ struct SmallMParams {
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);
 size_t smallm_gemm_smem_bytes(int batch);
 size_t smallm_gemm_scratch_floats(int N, int K, int batch);
+void set_decode_wide_impl(int impl);  // batch 9..64: 0 = tcgen05 (default), 1 = mma.sync
 
 // Decode attention (split over the cache) and its combine step.
 struct DecodeAttnParams {

@@ -118,6 +118,7 @@ def run_stack(a, s, bsz):
     model = B.Model(w, bsz, S + steps + 1, bsz * min(S, 256))
     if a.multi_kernel:
         model.set_persistent(False)
+    persistent = model.persistent_active() and bsz <= 8
     cache = B.KVCache(s, bsz, S + steps + 1)
     cache.k.normal_()                                 # a synthetic prefix instead of a prompt pass
     cache.v.normal_()
@@ -136,7 +137,7 @@ def run_stack(a, s, bsz):
     ms = e0.elapsed_time(e1) / a.iters
     nbytes = s.decode_step_bytes(S + 3 + a.iters // 2, bsz)
     print(f"stack [{a.config}, {a.layers} layers, batch {bsz}, kv {S}, "
-          f"{'multi-kernel' if a.multi_kernel else 'persistent'}]: {ms * 1e3:.1f} us per step, "
+          f"{'persistent' if persistent else 'one kernel per GEMM'}]: {ms * 1e3:.1f} us per step, "
           f"{nbytes / ms / 1e6:.0f} GB/s, status {model.device_status()}")
     model.close()
 

@@ -156,6 +156,8 @@ def run_reference(args):
     import torch
     from paper_2501_06589_b200 import synth
     shape = synth.SHAPES[args.config]
+    if args.batch:
+        shape = synth.replace(shape, batch=args.batch)
     n_sample = min(2, shape.n_layers)
     w = synth.make_weights(shape.with_layers(n_sample), device="cpu")
     kv_len = shape.prompt_len
@@ -202,6 +204,7 @@ def main():
     ap.add_argument("--streams", type=int, default=None)
     ap.add_argument("--graph", type=int, default=None)
     ap.add_argument("--pdl", type=int, default=None)
+    ap.add_argument("--batch", type=int, default=None, help="sequences decoded together (default: the configuration's)")
     ap.add_argument("--multi-kernel", action="store_true",
                     help="one kernel per GEMM (two streams, CUDA graph, PDL) instead of the persistent decode kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -231,6 +234,8 @@ def main():
     B.lib()
 
     shape = synth.SHAPES[args.config]
+    if args.batch:
+        shape = synth.replace(shape, batch=args.batch)
     steps, warm = args.steps, max(args.warmup, 0)
     S, bsz = shape.prompt_len, shape.batch
     max_seq = S + max(steps, warm)

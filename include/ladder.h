@@ -130,6 +130,14 @@ ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, 
 ladder_status_t ladder_model_set_persistent(ladder_model_t* m, int32_t on);
 int32_t ladder_model_persistent_active(const ladder_model_t* m);
 
+/* Test hook for the bounded waits of the persistent kernel: with on = 1 the LM-head phase of the next decode
+ * steps waits for one more finished unit than its producer phase has, i.e. for a count that is never reached.
+ * Nothing faults or spins forever: the wait gives up after 0.25 s, sets the LADDER_DEV_TIMEOUT bit (4) of the
+ * device status word, every other wait in the launch gives up as soon as it sees the bit, and the launch ends.
+ * Later launches return at once until ladder_device_status has read and cleared the word.  on = 0 restores
+ * the real dependency. */
+ladder_status_t ladder_debug_stall_last_phase(ladder_model_t* m, int32_t on);
+
 /* Host only (no GPU needed): describes the phase list the persistent kernel would execute for this
  * configuration, batch and SM count, as int32 words, for inspection and tests.
  *   header: n_phases, n_attention_nodes, n_counters, first_layer_in_kernel, ok

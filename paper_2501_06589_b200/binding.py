@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libladder.so")
 
 EXPORTS = [
-    "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_model_set_sm_split", "ladder_model_set_persistent", "ladder_model_persistent_active", "ladder_stack_plan",
+    "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_model_set_sm_split", "ladder_model_set_persistent", "ladder_model_persistent_active", "ladder_stack_plan", "ladder_debug_stall_last_phase",
     "ladder_prefill",
     "ladder_decode_step", "ladder_decode_step_host", "ladder_prefill_host", "ladder_set_position",
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
@@ -78,6 +78,7 @@ def lib() -> C.CDLL:
         L.ladder_model_set_persistent.argtypes = [C.c_void_p, C.c_int32]
         L.ladder_model_persistent_active.argtypes = [C.c_void_p]
         L.ladder_model_persistent_active.restype = C.c_int32
+        L.ladder_debug_stall_last_phase.argtypes = [C.c_void_p, C.c_int32]
         L.ladder_stack_plan.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32]
         L.ladder_stack_plan.restype = C.c_int32
         L.ladder_prefill.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32, C.c_int32,
@@ -234,6 +235,9 @@ class Model:
 
     def set_persistent(self, on: bool = True):
         _check(lib().ladder_model_set_persistent(self.h, int(on)), self.h)
+
+    def debug_stall_last_phase(self, on: bool):
+        _check(lib().ladder_debug_stall_last_phase(self.h, int(on)), self.h)
 
     def persistent_active(self) -> bool:
         return bool(lib().ladder_model_persistent_active(self.h))

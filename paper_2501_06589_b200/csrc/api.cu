@@ -78,6 +78,7 @@ struct ladder_model {
   // persistent layer-stack kernel (one cooperative launch per decode step, batch <= 8)
   bool stack_ok = false;   // usable on this device and worthwhile for this model
   int stack_begin = 0;     // first layer run by the persistent kernel (layers below: one kernel per GEMM)
+  int stack_stall_test = 0;  // test hook: the last phase waits for a count its producer never reaches
   int use_stack = 1;
   GraphKey stack_key;      // what the uploaded phase list was built for
   bool stack_built = false;
@@ -727,6 +728,7 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
     cur_layer = c.n_layers;
     add_gemm(4, h, m->R[rt.cur], nullptr, logits, nullptr, nullptr);
   }
+  if (m->stack_stall_test && !phases.empty() && phases.back().n_act_deps > 0) phases.back().act_need[0] += 1;
   *n_counters = static_cast<int>(sb.need.size());
   return !sb.overflow && static_cast<int>(phases.size()) <= kStackMaxPhases;
 }
@@ -986,6 +988,13 @@ ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, 
 ladder_status_t ladder_model_set_persistent(ladder_model_t* m, int32_t on) {
   if (!m) return LADDER_ERR_INVALID_ARG;
   m->use_stack = on ? 1 : 0;
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_debug_stall_last_phase(ladder_model_t* m, int32_t on) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  m->stack_stall_test = on ? 1 : 0;
+  m->stack_built = false;  // rebuild the phase list on the next step
   return LADDER_OK;
 }
 

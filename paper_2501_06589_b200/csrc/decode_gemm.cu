@@ -47,8 +47,8 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
 cudaError_t smallm_gemm_wide_tc_init();
 size_t smallm_gemm_wide_tc_smem_bytes(int batch);
 size_t smallm_gemm_wide_tc_scratch_floats(int N, int K, int batch);
-static int g_wide_impl = 0;  // 0 = tcgen05, 1 = mma.sync
-void set_decode_wide_impl(int impl) { g_wide_impl = impl == 1 ? 1 : 0; }
+static int g_wide_impl = 0;  // 0 = tcgen05, 1 = mma.sync, 2 = tcgen05 for every batch (also <= 8)
+void set_decode_wide_impl(int impl) { g_wide_impl = (impl == 1 || impl == 2) ? impl : 0; }
 
 namespace {
 
@@ -567,11 +567,11 @@ size_t smallm_gemm_smem_bytes(int batch) {
 }
 
 size_t smallm_gemm_scratch_floats(int N, int K, int batch) {
-  if (batch > 8) return smallm_gemm_wide_tc_scratch_floats(N, K, batch);  // staged activations + shared-tile pieces
-  return 0;  // the batch <= 8 kernel keeps full-K sums in registers: no scratch
+  return smallm_gemm_wide_tc_scratch_floats(N, K, batch);  // staged activations + shared-tile pieces
 }
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
+  if (g_wide_impl == 2) return launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count);
   if (p.batch > 8)
     return g_wide_impl == 0 ? launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count)
                             : launch_smallm_gemm_wide(p, stream, pdl, sm_count);

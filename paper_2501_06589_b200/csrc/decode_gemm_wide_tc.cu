@@ -95,6 +95,12 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
 __device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: K-major operand tile of rows x 64 bf16, 128-byte swizzle
@@ -273,7 +279,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
   }
   if (warp == 1) {  // TMEM: two accumulators of NP fp32 columns x 128 lanes
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "n"(2 * NP)
+                 "n"(2 * NP < 32 ? 32 : 2 * NP)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -367,7 +373,14 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
 #pragma unroll 1
       for (int b0 = 0; b0 < BP; b0 += CB) {
         float v[CB];
-        if (CB == 16) {
+        if constexpr (CB == 8) {
+          uint32_t h[8], l[8];
+          tc_ld8(taddr + b0, h);
+          tc_ld8(taddr + BP + b0, l);
+          tc_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(h[j]) + __uint_as_float(l[j]);
+        } else if constexpr (CB == 16) {
           uint32_t h[16], l[16];
           tc_ld16(taddr + b0, h);
           tc_ld16(taddr + BP + b0, l);
@@ -376,7 +389,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
           for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(h[j]) + __uint_as_float(l[j]);
         } else {
 #pragma unroll
-          for (int c = 0; c < CB; c += 16) {
+          for (int c = 0; c + 16 <= CB; c += 16) {
             uint32_t h[16], l[16];
             tc_ld16(taddr + b0 + c, h);
             tc_ld16(taddr + BP + b0 + c, l);
@@ -442,7 +455,9 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(2 * NP) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "n"(2 * NP < 32 ? 32 : 2 * NP)
+                 : "memory");
   }
 }
 
@@ -463,7 +478,7 @@ cudaError_t make_map(CUtensorMap* map, const void* base, int rows, int K, int bo
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-int padded_batch(int batch) { return batch <= 16 ? 16 : (batch <= 32 ? 32 : 64); }
+int padded_batch(int batch) { return batch <= 8 ? 8 : (batch <= 16 ? 16 : (batch <= 32 ? 32 : 64)); }
 
 // scratch layout in floats: [64] 1/rms | [kWideMaxTiles] tickets | staged activations (2 bp x K bf16) | pieces
 size_t stage_offset() { return 64 + kWideMaxTiles; }
@@ -498,6 +513,8 @@ cudaError_t smallm_gemm_wide_tc_init() {
   cudaError_t e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        WCfg<32>::SMEM);
   if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, WCfg<16>::SMEM);
+  if (e == cudaSuccess)
     e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WCfg<64>::SMEM);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -513,7 +530,7 @@ size_t smallm_gemm_wide_tc_scratch_floats(int N, int K, int batch) {
 
 size_t smallm_gemm_wide_tc_smem_bytes(int batch) {
   const int bp = padded_batch(batch);
-  return bp == 16 ? WCfg<32>::SMEM : (bp == 32 ? WCfg<64>::SMEM : WCfg<128>::SMEM);
+  return bp == 8 ? WCfg<16>::SMEM : (bp == 16 ? WCfg<32>::SMEM : (bp == 32 ? WCfg<64>::SMEM : WCfg<128>::SMEM));
 }
 
 cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
@@ -556,6 +573,7 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
   a.tickets = tickets;
   const int total = tiles * nkb;
   const int grid = total < sm_count ? total : sm_count;
+  if (bp == 8) return launch_np<16>(a, mw, ma, grid, stream);
   if (bp == 16) return launch_np<32>(a, mw, ma, grid, stream);
   if (bp == 32) return launch_np<64>(a, mw, ma, grid, stream);
   return launch_np<128>(a, mw, ma, grid, stream);

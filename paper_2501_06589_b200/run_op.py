@@ -28,9 +28,12 @@ def main():
     ap.add_argument("--kv-len", type=int, default=None)
     ap.add_argument("--tokens", type=int, default=4096, help="M of the prefill GEMM")
     ap.add_argument("--multi-kernel", action="store_true", help="stack: use the per-GEMM schedule")
+    ap.add_argument("--wide-impl", type=int, default=0,
+                    help="decode GEMM: 0 = default, 1 = mma.sync kernel for batch 9..64, 2 = tcgen05 kernel for every batch")
     a = ap.parse_args()
     build.build()
     B.lib()
+    B.set_decode_wide_impl(a.wide_impl)
     s = synth.SHAPES[a.config]
     bsz = a.batch or s.batch
     d, F, Hq, Hkv, Dh, V = s.d_model, s.d_ff, s.n_q_heads, s.n_kv_heads, s.head_dim, s.vocab_size

@@ -281,3 +281,50 @@ def test_tp_rank_slice_shape_batches(B, variant, batch):
     err, agree, *_ = check_generation(B, s, 6, np.float32, batch=batch, prompt_len=40)
     assert err < HIDDEN_TOL, err
     assert agree >= (0.98 if batch >= 16 else 0.85), agree      # 7 comparisons at batch 1: at most one flip
+
+
+def test_persistent_kernel_wait_runs_out_cleanly(B):
+    """A dependency that is never met ends the launch after the 0.25 s limit with the timeout bit set;
+    nothing hangs or faults, and once the status has been read the same model decodes correctly again."""
+    import time
+    s = synth.SHAPES["tiny"]
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    S, steps = 16, 3
+    prompt = torch.from_numpy(synth.make_tokens(s, 2, S)).cuda()
+    model = B.Model(w, 2, 64, 2 * S)
+    assert model.persistent_active()
+    cache = B.KVCache(s, 2, 64)
+    first = torch.zeros(2, dtype=torch.int32, device="cuda")
+    nxt = torch.zeros(2, dtype=torch.int32, device="cuda")
+    hid = torch.zeros(2, s.d_model, device="cuda")
+    model.prefill(cache, prompt, next_tokens=first)
+
+    def run():
+        cache.seq_lens.fill_(S)
+        model.set_position(S)
+        nxt.copy_(first)
+        out = []
+        for _ in range(steps):
+            model.decode_step(cache, nxt, next_tokens=nxt, final_hidden=hid)
+            out.append((nxt.clone(), hid.clone()))
+        torch.cuda.synchronize()
+        return out
+
+    ref = run()
+    assert model.device_status() == 0
+    model.debug_stall_last_phase(True)          # the LM head now waits for a unit count that is never reached
+    cache.seq_lens.fill_(S)
+    model.set_position(S)
+    nxt.copy_(first)
+    t0 = time.time()
+    model.decode_step(cache, nxt, next_tokens=nxt)
+    model.decode_step(cache, nxt, next_tokens=nxt)   # returns at once: the status word still holds the bit
+    torch.cuda.synchronize()
+    assert time.time() - t0 < 5.0
+    assert model.device_status() & 4             # LADDER_DEV_TIMEOUT, read and cleared
+    model.debug_stall_last_phase(False)
+    again = run()
+    assert model.device_status() == 0
+    for (t_a, h_a), (t_b, h_b) in zip(ref, again):
+        assert torch.equal(t_a, t_b) and torch.equal(h_a, h_b)
+    model.close()

@@ -6,7 +6,8 @@
 // the extra precision costs no extra instruction; their sum is formed in the epilogue.
 //
 // Two kernels per GEMM:
-//   1. wide_stage_kernel: fp32 activations (x gain for RMSNorm) -> bf16 [2 Bp, K] in scratch, 1/rms per row.
+//   1. wide_stage_kernel: fp32 activations (x gain for RMSNorm) -> bf16 [2 Bp, K] in scratch, sums of squares
+//      per 2048-wide K slice (the GEMM adds them in slice order: deterministic).
 //   2. decode_gemm_wide_tc_kernel: persistent CTAs, one per SM, three roles that meet at mbarriers:
 //        warp 0     TMA producer: per 64-wide K block one [128 rows x 64] box of W (L2 evict-first) and
 //                   one [2 Bp x 64] box of the staged activations (L2-resident), 128-byte swizzle, into a
@@ -42,7 +43,7 @@ struct WCfg {
   static constexpr int STAGE_BYTES = W_BYTES + ACT_BYTES;
   static constexpr int STAGES = (200 * 1024) / STAGE_BYTES;
   static constexpr int OFF_BARS = STAGES * STAGE_BYTES;  // full[], empty[], tmem_full[2], tmem_empty[2], tmem slot, flag
-  static constexpr int SMEM = OFF_BARS + (2 * STAGES + 4) * 8 + 64 + 1024;
+  static constexpr int SMEM = OFF_BARS + (2 * STAGES + 4) * 8 + 64 + 64 * 4 + 1024;
   static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(NP >> 3) << 17) |
                                     (static_cast<uint32_t>(BM >> 4) << 24);
   static_assert(SMEM <= 232448, "shared memory budget");
@@ -52,7 +53,8 @@ struct WideArgs {
   SmallMParams p;
   int bp;                  // padded batch
   int tiles, nkb;          // row tiles, K blocks
-  const float* rstd;       // [bp] (ACT_F32_NORM)
+  const float* ssq;        // [bp][n_slices] sums of squares per K slice (ACT_F32_NORM)
+  int n_slices;
   float* partial;          // [grid][2][bp][128]
   int32_t* tickets;        // [tiles], zero between launches
 };
@@ -116,17 +118,20 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 }
 
 // ---------------------------------------------------------------- activation staging
-// One CTA per padded batch row: y = x (* gain), hi = bf16(y), lo = bf16(y - hi); rows >= batch are zero.
-__global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const __nv_bfloat16* gain, int norm, float eps,
-                                                         int batch, int bp, int K, __nv_bfloat16* stage, float* rstd) {
+// One CTA per (padded batch row, 2048-wide K slice): y = x (* gain), hi = bf16(y), lo = bf16(y - hi); rows
+// >= batch are zero.  The slice's sum of squares goes to ssq[row][slice]; the GEMM adds the slices in order.
+constexpr int kStageSlice = 2048;
+__global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const __nv_bfloat16* gain, int norm, int batch,
+                                                         int bp, int K, __nv_bfloat16* stage, float* ssq_out) {
   __shared__ float red[8];
-  const int b = blockIdx.x, tid = threadIdx.x;
+  const int b = blockIdx.x, slice = blockIdx.y, tid = threadIdx.x;
   pdl_launch_dependents();
   pdl_wait();
   __nv_bfloat16* hi = stage + static_cast<size_t>(b) * K;
   __nv_bfloat16* lo = stage + static_cast<size_t>(bp + b) * K;
   float ssq = 0.f;
-  for (int k = tid * 8; k < K; k += 256 * 8) {
+  const int k = slice * kStageSlice + tid * 8;
+  if (k < K) {
     float y[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (b < batch) {
       const float4 a = __ldcg(reinterpret_cast<const float4*>(x + static_cast<size_t>(b) * K + k));
@@ -153,9 +158,9 @@ __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const _
   if ((tid & 31) == 0) red[tid >> 5] = ssq;
   __syncthreads();
   if (tid == 0) {
-    float s = 0.f;
-    for (int w = 0; w < 8; ++w) s += red[w];
-    rstd[b] = norm ? rsqrtf(s / static_cast<float>(K) + eps) : 1.f;
+    float t = 0.f;
+    for (int w = 0; w < 8; ++w) t += red[w];
+    ssq_out[b * gridDim.y + slice] = t;
   }
 }
 
@@ -258,6 +263,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
   uint64_t* tmem_empty = tmem_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
   volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* rstd_s = reinterpret_cast<float*>(smem + C::OFF_BARS + (2 * STAGES + 4) * 8 + 64);  // [BP] 1/rms
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const SmallMParams& p = a.p;
@@ -356,7 +362,14 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
     const int r = q * 32 + lane;  // row inside the tile
     bool ok = true;
     int seg = 0;
-    pdl_wait();  // 1/rms, the addend and the destination belong to earlier kernels
+    pdl_wait();  // the sums of squares, the addend and the destination belong to earlier kernels
+    if (et < BP) {   // 1/rms of every batch row: the K slices' sums of squares added in slice order
+      float t = 0.f;
+      if (p.act_mode == ACT_F32_NORM)
+        for (int sl = 0; sl < a.n_slices; ++sl) t += a.ssq[et * a.n_slices + sl];
+      rstd_s[et] = p.act_mode == ACT_F32_NORM ? rsqrtf(t / static_cast<float>(p.K) + p.eps) : 1.f;
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
     for (int pos = my_start; pos < my_end; ++seg) {
       const int t = pos / nkb, kb0 = pos - t * nkb, kb1 = min(nkb, kb0 + (my_end - pos));
       pos += kb1 - kb0;
@@ -401,7 +414,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
         if (whole) {
           if (p.act_mode == ACT_F32_NORM) {
 #pragma unroll
-            for (int j = 0; j < CB; ++j) v[j] *= a.rstd[b0 + j];
+            for (int j = 0; j < CB; ++j) v[j] *= rstd_s[b0 + j];
           }
           wide_epilogue<CB>(p, n, b0, v, lane);
         } else {
@@ -443,7 +456,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
         }
         if (p.act_mode == ACT_F32_NORM) {
 #pragma unroll
-          for (int j = 0; j < CB; ++j) v[j] *= a.rstd[b0 + j];
+          for (int j = 0; j < CB; ++j) v[j] *= rstd_s[b0 + j];
         }
         wide_epilogue<CB>(p, n, b0, v, lane);
       }
@@ -480,8 +493,10 @@ cudaError_t make_map(CUtensorMap* map, const void* base, int rows, int K, int bo
 
 int padded_batch(int batch) { return batch <= 8 ? 8 : (batch <= 16 ? 16 : (batch <= 32 ? 32 : 64)); }
 
-// scratch layout in floats: [64] 1/rms | [kWideMaxTiles] tickets | staged activations (2 bp x K bf16) | pieces
-size_t stage_offset() { return 64 + kWideMaxTiles; }
+// scratch layout in floats: [64 x kWideMaxSlices] sums of squares | [kWideMaxTiles] tickets | staged activations
+// (2 bp x K bf16) | pieces
+constexpr int kWideMaxSlices = 64;  // K up to 131072
+size_t stage_offset() { return 64 * kWideMaxSlices + kWideMaxTiles; }
 size_t piece_offset(int bp, int K) { return stage_offset() + ((static_cast<size_t>(bp) * K + 3) & ~size_t(3)); }
 
 template <int NP>
@@ -540,14 +555,16 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
   const int bp = padded_batch(p.batch);
   const int tiles = (p.N + BM - 1) / BM, nkb = (p.K + BK - 1) / BK;
   if (tiles > kWideMaxTiles || sm_count > kWideMaxCtas) return cudaErrorInvalidValue;
-  float* rstd = p.scratch;
-  int32_t* tickets = reinterpret_cast<int32_t*>(p.scratch + 64);
+  float* ssq = p.scratch;
+  int32_t* tickets = reinterpret_cast<int32_t*>(p.scratch + 64 * kWideMaxSlices);
+  const int n_slices = (p.K + kStageSlice - 1) / kStageSlice;
+  if (n_slices > kWideMaxSlices) return cudaErrorInvalidValue;
   __nv_bfloat16* stage = reinterpret_cast<__nv_bfloat16*>(p.scratch + stage_offset());
   float* pieces = p.scratch + piece_offset(bp, p.K);
 
   {  // 1. activations -> bf16 hi + lo, 1/rms
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(bp);
+    cfg.gridDim = dim3(bp, n_slices);
     cfg.blockDim = dim3(256);
     cfg.stream = stream;
     cudaLaunchAttribute at[1];
@@ -556,7 +573,7 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
     cfg.attrs = at;
     cfg.numAttrs = pdl ? 1 : 0;
     cudaError_t e = cudaLaunchKernelEx(&cfg, wide_stage_kernel, static_cast<const float*>(p.act), p.gain,
-                                       p.act_mode == ACT_F32_NORM ? 1 : 0, p.eps, p.batch, bp, p.K, stage, rstd);
+                                       p.act_mode == ACT_F32_NORM ? 1 : 0, p.batch, bp, p.K, stage, ssq);
     if (e != cudaSuccess) return e;
   }
   CUtensorMap mw, ma;
@@ -568,7 +585,8 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
   a.bp = bp;
   a.tiles = tiles;
   a.nkb = nkb;
-  a.rstd = rstd;
+  a.ssq = ssq;
+  a.n_slices = n_slices;
   a.partial = pieces;
   a.tickets = tickets;
   const int total = tiles * nkb;

@@ -53,6 +53,9 @@ struct ladder_model {
   float* q_f32 = nullptr;           // decode [max_batch, Hq*Dh]
   float* o_dec = nullptr;           // decode [max_batch, Hq*Dh]
   float* h_dec = nullptr;           // decode [max_batch, F]
+  // the same activations as bf16 hi/lo MMA operands ([chunk][8][2048]), written by the persistent kernel's
+  // epilogues for the phase that reads them next (batch <= 4): twins of R[0], R[1], h_dec, o_dec
+  __nv_bfloat16 *xpack[2] = {nullptr, nullptr}, *hpack = nullptr, *opack = nullptr;
   float* attn_scratch = nullptr;
   int attn_splits = 1;
   float* gemm_scratch[2] = {nullptr, nullptr};  // split-K partials + tickets, one per stream role
@@ -557,11 +560,39 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
   attn.clear();
 
   int cur_layer = 0;
+  // A phase whose fp32 input was produced inside this launch gets it as a ready MMA operand as well: the
+  // producer's epilogue (or the attention merge) writes the bf16 hi/lo copy, with the reader's RMSNorm gain
+  // folded in, and the reader's stagers only copy it.  Only for batch <= 4 (hi and lo share one MMA tile).
+  std::map<const void*, __nv_bfloat16*> twin = {
+      {m->R[0], m->xpack[0]}, {m->R[1], m->xpack[1]}, {m->h_dec, m->hpack}, {m->o_dec, m->opack}};
+  std::map<const void*, std::pair<int, int>> last_writer;  // fp32 buffer -> (0 = phase | 1 = attention node, index)
   auto add_gemm = [&](int kind, SmallMParams p, const void* act_buf, const void* add_buf, const void* out0,
                       const void* out1, const void* out2) {
     StackPhase P = {};
     P.kind = kind;
     P.layer = cur_layer;
+    if (batch <= 4) {
+      auto wr = last_writer.find(act_buf);
+      auto tw = twin.find(act_buf);
+      if (wr != last_writer.end() && tw != twin.end() && tw->second) {
+        const __nv_bfloat16* want_gain = p.act_mode == ACT_F32_NORM ? p.gain : nullptr;
+        if (wr->second.first == 0) {
+          SmallMParams& w = phases[wr->second.second].p;
+          if (!w.pack_out) {
+            w.pack_out = tw->second;
+            w.pack_gain = want_gain;
+            P.act_packed = tw->second;
+          }
+        } else {
+          StackAttn& w = attn[wr->second.second];
+          if (!w.o_pack) {
+            w.o_pack = tw->second;
+            P.act_packed = tw->second;
+          }
+        }
+      }
+    }
+    if (p.epi_mode == EPI_RESID || p.epi_mode == EPI_SWIGLU) last_writer[out0] = {0, static_cast<int>(phases.size())};
     p.batch = batch;
     p.status = m->status;
     P.p = p;
@@ -661,6 +692,7 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
       sb.did_read(vc, A.merge_done);
       sb.did_write(m->o_dec, A.merge_done);
       prev_merge = A.merge_done;
+      last_writer[m->o_dec] = {1, static_cast<int>(attn.size())};
       attn.push_back(A);
     };
     auto wo = [&]() {
@@ -887,6 +919,16 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   A(dev_alloc(&m->q_f32, MB * qd));
   A(dev_alloc(&m->o_dec, MB * qd));
   A(dev_alloc(&m->h_dec, MB * F));
+  const auto pack_elems = [](size_t K) { return ((K + 2047) / 2048) * 8 * 2048; };
+  A(dev_alloc(&m->xpack[0], pack_elems(d)));
+  A(dev_alloc(&m->xpack[1], pack_elems(d)));
+  A(dev_alloc(&m->hpack, pack_elems(F)));
+  A(dev_alloc(&m->opack, pack_elems(qd)));
+  if (!oom) {  // the bulk copies read whole 4 KB rows: what no epilogue ever writes must be finite
+    for (auto pk : {std::make_pair(m->xpack[0], pack_elems(d)), std::make_pair(m->xpack[1], pack_elems(d)),
+                    std::make_pair(m->hpack, pack_elems(F)), std::make_pair(m->opack, pack_elems(qd))})
+      if (cudaMemset(pk.first, 0, pk.second * sizeof(__nv_bfloat16)) != cudaSuccess) oom = true;
+  }
   A(dev_alloc(&m->attn_scratch, scratch_floats));
   {
     const int qkv_rows = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
@@ -967,7 +1009,7 @@ ladder_status_t ladder_destroy(ladder_model_t* m) {
   if (m->ev_join) cudaEventDestroy(m->ev_join);
   if (m->side) cudaStreamDestroy(m->side);
   if (m->cap) cudaStreamDestroy(m->cap);
-  void* bufs[] = {m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
+  void* bufs[] = {m->xpack[0], m->xpack[1], m->hpack, m->opack, m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
                   m->n_pf, m->q_pf,  m->o_pf,  m->h_pf,  m->rope,  m->status,       m->tok_tmp,   m->next_tmp};
   for (void* b : bufs)
     if (b) cudaFree(b);
@@ -1041,6 +1083,10 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
   m.o_dec = reinterpret_cast<float*>(fake());
   m.h_dec = reinterpret_cast<float*>(fake());
   m.attn_scratch = reinterpret_cast<float*>(fake());
+  m.xpack[0] = reinterpret_cast<__nv_bfloat16*>(fake());
+  m.xpack[1] = reinterpret_cast<__nv_bfloat16*>(fake());
+  m.hpack = reinterpret_cast<__nv_bfloat16*>(fake());
+  m.opack = reinterpret_cast<__nv_bfloat16*>(fake());
   m.status = reinterpret_cast<int32_t*>(fake());
   m.rope = reinterpret_cast<float2*>(fake());
   m.lm_head = reinterpret_cast<const __nv_bfloat16*>(fake());
@@ -1065,20 +1111,20 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
     for (int r = 0; r < kStackRounds; ++r) o.push_back(P.count[r]);
     for (int r = 0; r < kStackRounds; ++r) o.push_back(P.size[r]);
     o.push_back(P.n_act_deps);
-    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(P.act_dep[i]);
-    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(P.act_need[i]);
+    for (int i = 0; i < 6; ++i) o.push_back(i < kStackMaxDeps ? P.act_dep[i] : 0);
+    for (int i = 0; i < 6; ++i) o.push_back(i < kStackMaxDeps ? P.act_need[i] : 0);
     o.push_back(P.n_epi_deps);
-    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(P.epi_dep[i]);
-    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(P.epi_need[i]);
+    for (int i = 0; i < 6; ++i) o.push_back(i < kStackMaxDeps ? P.epi_dep[i] : 0);
+    for (int i = 0; i < 6; ++i) o.push_back(i < kStackMaxDeps ? P.epi_need[i] : 0);
   }
   int li = 0;
   for (const StackAttn& A : at) {
     o.insert(o.end(), {begin + li++, A.split_done, A.merge_done, A.n_deps});
-    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(A.dep[i]);
-    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(A.need[i]);
+    for (int i = 0; i < 6; ++i) o.push_back(i < kStackMaxDeps ? A.dep[i] : 0);
+    for (int i = 0; i < 6; ++i) o.push_back(i < kStackMaxDeps ? A.need[i] : 0);
     o.push_back(A.n_mdeps);
-    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(A.mdep[i]);
-    for (int i = 0; i < kStackMaxDeps; ++i) o.push_back(A.mneed[i]);
+    for (int i = 0; i < 6; ++i) o.push_back(i < kStackMaxDeps ? A.mdep[i] : 0);
+    for (int i = 0; i < 6; ++i) o.push_back(i < kStackMaxDeps ? A.mneed[i] : 0);
   }
   if (static_cast<int>(o.size()) > cap) return -static_cast<int32_t>(o.size());
   memcpy(out, o.data(), o.size() * sizeof(int32_t));

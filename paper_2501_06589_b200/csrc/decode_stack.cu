@@ -411,7 +411,8 @@ __device__ __forceinline__ void attn_split_unit(const float* q, const __nv_bfloa
 // decode_attention_merge_kernel).
 template <int DH>
 __device__ __forceinline__ void attn_merge_unit(const float* scratch, int n_q_heads, int stride_splits, int n_splits,
-                                                int b, int h, float* o, float* wgt, float* red_m, float* red_l, int at) {
+                                                int b, int h, float* o, __nv_bfloat16* o_pack, float* wgt, float* red_m,
+                                                float* red_l, int at) {
   constexpr int stride = DH + 2;
   const int warp = at >> 5, lane = at & 31;
   const float* base = scratch + (static_cast<size_t>(b) * n_q_heads + h) * stride_splits * stride;
@@ -445,7 +446,9 @@ __device__ __forceinline__ void attn_merge_unit(const float* scratch, int n_q_he
     float acc = 0.f;
 #pragma unroll 8
     for (int s = 0; s < n_splits; ++s) acc += wgt[s] * __ldcg(base + s * stride + at);
-    o[(static_cast<size_t>(b) * n_q_heads + h) * DH + at] = lsum > 0.f ? acc / lsum : 0.f;
+    const float val = lsum > 0.f ? acc / lsum : 0.f;
+    o[(static_cast<size_t>(b) * n_q_heads + h) * DH + at] = val;
+    if (o_pack) store_packed(o_pack, nullptr, b, h * DH + at, val);  // the output projection's MMA operand
   }
   bar_sync(3, kAux);
 }
@@ -955,7 +958,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
     const __nv_bfloat16* gain = nullptr;
     static_assert(offsetof(StackPhase, act) == 128 && offsetof(StackPhase, gain) == 136 &&
                       offsetof(StackPhase, act_mode) == 144 && offsetof(StackPhase, n_act_deps) == 148 &&
-                      offsetof(StackPhase, act_dep) == 152 && offsetof(StackPhase, act_need) == 176,
+                      offsetof(StackPhase, act_dep) == 152 && offsetof(StackPhase, act_need) == 152 + 4 * kStackMaxDeps &&
+                      offsetof(StackPhase, act_packed) == 128 + 4 * 28,
                   "descriptor layout");
     auto load_h1 = [&](int ph) -> int {
       return ph < sp.n_phases ? __ldg(reinterpret_cast<const int*>(sp.phases + ph) + 32 + lane) : 0;
@@ -1033,6 +1037,21 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       }
     };
 
+    auto sumsq_rows = [&]() {  // the sums of squares exactly as store_rows forms them, nothing else
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (i >= batch) break;
+#pragma unroll
+        for (int u = 0; u < SU; ++u) {
+          const float y[8] = {x[i][u].a.x, x[i][u].a.y, x[i][u].a.z, x[i][u].a.w,
+                              x[i][u].b.x, x[i][u].b.y, x[i][u].b.z, x[i][u].b.w};
+          ssq[i] += y[0] * y[0] + y[1] * y[1] + y[2] * y[2] + y[3] * y[3] + y[4] * y[4] + y[5] * y[5] +
+                    y[6] * y[6] + y[7] * y[7];
+        }
+      }
+    };
+    const uint64_t pol_act = l2_policy_evict_last();
+    const __nv_bfloat16* actp = nullptr;
     TR_DECL(sdeps);
     TR_DECL(sfree);
     TR_DECL(sq);
@@ -1065,18 +1084,23 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
             (static_cast<unsigned long long>(static_cast<unsigned int>(__shfl_sync(0xffffffffu, h1, 3))) << 32) |
             static_cast<unsigned int>(__shfl_sync(0xffffffffu, h1, 2)));
         norm = __shfl_sync(0xffffffffu, h1, 4) == ACT_F32_NORM;
+        actp = reinterpret_cast<const __nv_bfloat16*>(
+            (static_cast<unsigned long long>(static_cast<unsigned int>(__shfl_sync(0xffffffffu, h1, 29))) << 32) |
+            static_cast<unsigned int>(__shfl_sync(0xffffffffu, h1, 28)));
         ssq_on = norm;  // the first batch of a normalised phase also forms the sums of squares
         cur_ph = ph;
         // the activations of this phase must have been written (all of them: every batch needs all of K)
         {
           TR_T0();
-          // lane i polls dependency i (words 6.. = counter index, 12.. = required value)
+          // lane i polls dependency i (words 6.. = counter index, 6 + kStackMaxDeps.. = required value)
           const int nd = __shfl_sync(0xffffffffu, h1, 5);
           const int dep_i = __shfl_sync(0xffffffffu, h1, 6 + (lane < kStackMaxDeps ? lane : 0));
-          const int need_i = __shfl_sync(0xffffffffu, h1, 12 + (lane < kStackMaxDeps ? lane : 0));
+          const int need_i = __shfl_sync(0xffffffffu, h1, 6 + kStackMaxDeps + (lane < kStackMaxDeps ? lane : 0));
           bool okd = true;
           if (lane < nd) okd = wait_global_ge(sp.counters + dep_i, need_i, status);
           ok = __all_sync(0xffffffffu, okd);
+          // what other SMs wrote before those counters moved is read next by bulk copies (async proxy)
+          asm volatile("fence.proxy.async;" ::: "memory");
           TR_ADD(sdeps);
         }
         if (!ok) break;
@@ -1084,17 +1108,31 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       // chunk by chunk, one chunk ahead of the consumers: the raw values are loaded into registers
       // before the buffer is handed back (act_free)
       for (int ch = 0; ch < nchunk; ++ch, ++r) {
-        load_rows(ch, 0);
+        // Operands already in MMA form (written by the producing phase's epilogue): the chunk is eight 4 KB
+        // bulk copies.  Otherwise convert from fp32.  The fp32 rows are still read while the first batch
+        // of a normalised phase is staged, for the sums of squares only.
+        const bool copy = actp != nullptr;
+        if (!copy || ssq_on) load_rows(ch, 0);
         {
           TR_T0();
           ok = __all_sync(0xffffffffu, wait_mbar<200>(act_free, (r & 1) ^ 1u, status));
           TR_ADD(sfree);
         }
         if (!ok) break;
-        store_rows(0);
-        if (!PACKED && batch > 4) {
-          load_rows(ch, 1);
-          store_rows(1);
+        if (copy) {
+          if (sw == 0) {
+            if (lane == 0) mbar_expect_tx(act_full, 8 * TK * 2);  // counts as this warp's arrival
+            __syncwarp();
+            if (lane < 8)
+              bulk_g2s(act + lane * PITCH, actp + (static_cast<size_t>(ch) * 8 + lane) * TK, TK * 2, act_full, pol_act);
+          }
+          if (ssq_on) sumsq_rows();
+        } else {
+          store_rows(0);
+          if (!PACKED && batch > 4) {
+            load_rows(ch, 1);
+            store_rows(1);
+          }
         }
         if (ssq_on && ch == nchunk - 1) {  // every chunk has been staged once: publish the sums
           float* sq = ssq_part + (norm_cnt & (NORM_RING - 1)) * 32;
@@ -1112,7 +1150,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
           ++norm_cnt;
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(act_full);
+        if (lane == 0 && !(copy && sw == 0)) mbar_arrive(act_full);
       }
       if (!ok) break;
     }
@@ -1161,6 +1199,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       const int stride_splits = A->a.n_splits;
       float* scratch = A->a.scratch;
       float* o = A->a.o;
+      __nv_bfloat16* o_pack = PACKED ? A->o_pack : nullptr;
       int gt = 1;
       {
         const int group = Hq / Hkv;
@@ -1201,8 +1240,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       for (int u = blockIdx.x; u < n_pairs; u += gridDim.x) {
         const int b = u / Hq, h = u % Hq;
         const int ns = pre[b + 1] - pre[b];
-        if (DH == 128) attn_merge_unit<128>(scratch, Hq, stride_splits, ns, b, h, o, ared, red_m, red_l, at);
-        else attn_merge_unit<64>(scratch, Hq, stride_splits, ns, b, h, o, ared, red_m, red_l, at);
+        if (DH == 128) attn_merge_unit<128>(scratch, Hq, stride_splits, ns, b, h, o, o_pack, ared, red_m, red_l, at);
+        else attn_merge_unit<64>(scratch, Hq, stride_splits, ns, b, h, o, o_pack, ared, red_m, red_l, at);
         ++mine;
       }
       __threadfence();

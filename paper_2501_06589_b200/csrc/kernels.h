@@ -38,6 +38,10 @@ struct SmallMParams {
   void* out;               // EPI_RESID / EPI_PLAIN: fp32 [batch, N]; EPI_SWIGLU: fp32 [batch, N/2]
   QkvEpilogue qkv;         // EPI_QKV_ROPE
   int32_t* status;         // device status word (may be NULL)
+  // Optional second copy of an fp32 output (EPI_RESID: out, EPI_SWIGLU: h) as the next GEMM's MMA operand:
+  // y = value (* pack_gain[n]), bf16 hi at [n / 2048][b][n % 2048], lo at [n / 2048][4 + b][n % 2048]; batch <= 4.
+  __nv_bfloat16* pack_out;
+  const __nv_bfloat16* pack_gain;
   // batch <= 8 (dynamic item claiming, split-K fix-up):
   float* scratch;          // smallm_gemm_scratch_floats(N, K, batch) floats, ticket part zero; kernels that
                            // may run concurrently need distinct scratch
@@ -72,7 +76,7 @@ cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stre
 // "phase" of ONE cooperative launch, attention runs on dedicated warps of the same CTAs, and the
 // kernel boundaries become counters in global memory (units finished per phase) that a reader polls
 // before it touches data another SM produced.
-constexpr int kStackMaxDeps = 6;
+constexpr int kStackMaxDeps = 5;
 constexpr int kStackMaxPhases = 1023;
 constexpr int kStackRounds = 10;
 constexpr int kStackChunkK = 2048;  // K elements per chunk of the persistent kernel (4 KB of a weight row)
@@ -99,6 +103,10 @@ struct alignas(128) StackPhase {
   // ... and before the first epilogue (addend read, output buffer overwritten)
   int n_epi_deps, epi_dep[kStackMaxDeps], epi_need[kStackMaxDeps];
   int pad1[1];
+  // activations already in MMA operand form (bf16 hi rows 0-3, lo rows 4-7, [chunk][8][2048]), written by the
+  // phase that produced them; NULL: convert from the fp32 activations
+  const __nv_bfloat16* act_packed;
+  int pad2[2];
   // ---- the epilogue description (finishers)
   SmallMParams p;
 };
@@ -109,6 +117,7 @@ struct StackAttn {
   int n_deps, dep[kStackMaxDeps], need[kStackMaxDeps];      // before the split units (q, K, V written; scratch free)
   int n_mdeps, mdep[kStackMaxDeps], mneed[kStackMaxDeps];   // before the merge units (o free to overwrite)
   int split_done, merge_done;                               // counters: units finished
+  __nv_bfloat16* o_pack;                                    // optional MMA-operand copy of o (see SmallMParams::pack_out)
 };
 struct StackParams {
   const StackPhase* phases;

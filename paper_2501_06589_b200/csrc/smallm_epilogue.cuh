@@ -7,6 +7,17 @@
 
 namespace ladder {
 
+// Second copy of an output value as the next GEMM's MMA operand: bf16 high part in row b, low part in row 4 + b
+// of the 2048-wide chunk that column n falls in (the layout the persistent kernel's activation buffer has).
+__device__ __forceinline__ void store_packed(__nv_bfloat16* pack, const __nv_bfloat16* gain, int b, int n, float v) {
+  if (gain) v *= __bfloat162float(gain[n]);
+  const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+  const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+  __nv_bfloat16* dst = pack + (static_cast<size_t>(n >> 11) * 8 + b) * 2048 + (n & 2047);
+  dst[0] = hi;
+  dst[4 * 2048] = lo;
+}
+
 template <int NT = 128, typename ValueFn>
 __device__ __forceinline__ void smallm_epilogue(const SmallMParams& p, int ct, int prow, int nbase, int batch,
                                                 ValueFn value) {
@@ -19,6 +30,7 @@ __device__ __forceinline__ void smallm_epilogue(const SmallMParams& p, int ct, i
       float v = value(r, b);
       if (p.epi_mode == EPI_RESID) v += __ldcg(p.addend + o);  // L2: may have been written by another SM of this launch
       out[o] = v;
+      if (p.pack_out) store_packed(p.pack_out, p.pack_gain, b, nbase + r, v);
     }
   } else if (p.epi_mode == EPI_SWIGLU) {
     // rows (2j, 2j+1) = (gate_j, up_j)  ->  h_j = silu(gate_j) * up_j
@@ -27,7 +39,9 @@ __device__ __forceinline__ void smallm_epilogue(const SmallMParams& p, int ct, i
     for (int idx = ct; idx < half * batch; idx += NT) {
       const int pr = idx % half, b = idx / half;
       const float gt = value(2 * pr, b), up = value(2 * pr + 1, b);
-      out[static_cast<size_t>(b) * (p.N >> 1) + ((nbase >> 1) + pr)] = gt / (1.f + __expf(-gt)) * up;
+      const float hv = gt / (1.f + __expf(-gt)) * up;
+      out[static_cast<size_t>(b) * (p.N >> 1) + ((nbase >> 1) + pr)] = hv;
+      if (p.pack_out) store_packed(p.pack_out, p.pack_gain, b, (nbase >> 1) + pr, hv);
     }
   } else if (p.epi_mode == EPI_QKV_ROPE) {
     // rotary embedding on interleaved pairs of q and k at position seq_lens[b]; k, v appended to the cache

@@ -562,7 +562,9 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
   int cur_layer = 0;
   // A phase whose fp32 input was produced inside this launch gets it as a ready MMA operand as well: the
   // producer's epilogue (or the attention merge) writes the bf16 hi/lo copy, with the reader's RMSNorm gain
-  // folded in, and the reader's stagers only copy it.  Only for batch <= 4 (hi and lo share one MMA tile).
+  // folded in, and the reader's stagers only copy it (with ordinary loads: a bulk copy by the TMA engine read
+  // stale bytes now and then, whatever proxy fences were placed on either side).  Only for batch <= 4 (hi
+  // and lo share one MMA tile).
   std::map<const void*, __nv_bfloat16*> twin = {
       {m->R[0], m->xpack[0]}, {m->R[1], m->xpack[1]}, {m->h_dec, m->hpack}, {m->o_dec, m->opack}};
   std::map<const void*, std::pair<int, int>> last_writer;  // fp32 buffer -> (0 = phase | 1 = attention node, index)
@@ -924,7 +926,7 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   A(dev_alloc(&m->xpack[1], pack_elems(d)));
   A(dev_alloc(&m->hpack, pack_elems(F)));
   A(dev_alloc(&m->opack, pack_elems(qd)));
-  if (!oom) {  // the bulk copies read whole 4 KB rows: what no epilogue ever writes must be finite
+  if (!oom) {  // the stagers copy whole 4 KB rows: what no epilogue ever writes must be finite
     for (auto pk : {std::make_pair(m->xpack[0], pack_elems(d)), std::make_pair(m->xpack[1], pack_elems(d)),
                     std::make_pair(m->hpack, pack_elems(F)), std::make_pair(m->opack, pack_elems(qd))})
       if (cudaMemset(pk.first, 0, pk.second * sizeof(__nv_bfloat16)) != cudaSuccess) oom = true;

@@ -78,13 +78,7 @@ constexpr int SMEM = OFF_AUX + AUX_PS + AUX_RED + AUX_MLS + AUX_MISC + 128;
 static_assert(SMEM <= 227 * 1024, "shared memory budget");
 
 // registers per thread after the warpgroups have traded (launch allocation: 128 each)
-#ifndef RW0
-#define RW0 72
-#define RCO 176
-#define RST 120
-#define RAU 144
-#endif
-constexpr int REGS_WG0 = RW0, REGS_CONS = RCO, REGS_STAGE = RST, REGS_AUX = RAU;
+constexpr int REGS_WG0 = 72, REGS_CONS = 176, REGS_STAGE = 120, REGS_AUX = 144;
 static_assert(REGS_WG0 + REGS_CONS + REGS_STAGE + REGS_AUX <= 4 * 128, "register pool exceeded");
 
 struct F8 {
@@ -1050,7 +1044,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         }
       }
     };
-    const uint64_t pol_act = l2_policy_evict_last();
     const __nv_bfloat16* actp = nullptr;
     TR_DECL(sdeps);
     TR_DECL(sfree);
@@ -1099,8 +1092,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
           bool okd = true;
           if (lane < nd) okd = wait_global_ge(sp.counters + dep_i, need_i, status);
           ok = __all_sync(0xffffffffu, okd);
-          // what other SMs wrote before those counters moved is read next by bulk copies (async proxy)
-          asm volatile("fence.proxy.async;" ::: "memory");
+          __syncwarp();
           TR_ADD(sdeps);
         }
         if (!ok) break;
@@ -1108,11 +1100,25 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       // chunk by chunk, one chunk ahead of the consumers: the raw values are loaded into registers
       // before the buffer is handed back (act_free)
       for (int ch = 0; ch < nchunk; ++ch, ++r) {
-        // Operands already in MMA form (written by the producing phase's epilogue): the chunk is eight 4 KB
-        // bulk copies.  Otherwise convert from fp32.  The fp32 rows are still read while the first batch
-        // of a normalised phase is staged, for the sums of squares only.
+        // Operands already in MMA form (written by the producing phase's epilogue): the chunk is copied as it
+        // is, 16 bytes at a time, loaded before the buffer is handed back.  Otherwise convert from fp32.  The
+        // fp32 rows are still read while the first batch of a normalised phase is staged, for the sums of
+        // squares only.
         const bool copy = actp != nullptr;
-        if (!copy || ssq_on) load_rows(ch, 0);
+        if (copy && ssq_on) {  // the fp32 rows first (their registers are then free for the copy)
+          load_rows(ch, 0);
+          sumsq_rows();
+        }
+        if (copy) {  // 16 x 16 bytes per thread, held in the registers the conversion path uses for its fp32 rows
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int idx = st + j * 128, row = idx >> 8, col = idx & 255;  // 256 16-byte units per 4 KB row
+            F8& slot = x[j >> 2][(j >> 1) & 1];
+            float4& f = (j & 1) ? slot.b : slot.a;
+            f = __ldcg(reinterpret_cast<const float4*>(actp + (static_cast<size_t>(ch) * 8 + row) * TK) + col);
+          }
+        }
+        if (!copy) load_rows(ch, 0);
         {
           TR_T0();
           ok = __all_sync(0xffffffffu, wait_mbar<200>(act_free, (r & 1) ^ 1u, status));
@@ -1120,13 +1126,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         }
         if (!ok) break;
         if (copy) {
-          if (sw == 0) {
-            if (lane == 0) mbar_expect_tx(act_full, 8 * TK * 2);  // counts as this warp's arrival
-            __syncwarp();
-            if (lane < 8)
-              bulk_g2s(act + lane * PITCH, actp + (static_cast<size_t>(ch) * 8 + lane) * TK, TK * 2, act_full, pol_act);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int idx = st + j * 128, row = idx >> 8, col = idx & 255;
+            const F8& slot = x[j >> 2][(j >> 1) & 1];
+            const float4& f = (j & 1) ? slot.b : slot.a;
+            sts128(act_u32 + row * PITCH + col * 16,
+                   make_uint4(__float_as_uint(f.x), __float_as_uint(f.y), __float_as_uint(f.z), __float_as_uint(f.w)));
           }
-          if (ssq_on) sumsq_rows();
         } else {
           store_rows(0);
           if (!PACKED && batch > 4) {
@@ -1150,7 +1157,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
           ++norm_cnt;
         }
         __syncwarp();
-        if (lane == 0 && !(copy && sw == 0)) mbar_arrive(act_full);
+        if (lane == 0) mbar_arrive(act_full);
       }
       if (!ok) break;
     }

@@ -158,6 +158,8 @@ def run_reference(args):
     shape = synth.SHAPES[args.config]
     if args.batch:
         shape = synth.replace(shape, batch=args.batch)
+    if args.standard:
+        shape = shape.as_standard()
     n_sample = min(2, shape.n_layers)
     w = synth.make_weights(shape.with_layers(n_sample), device="cpu")
     kv_len = shape.prompt_len
@@ -186,7 +188,7 @@ def run_reference(args):
 
 def workload_config(shape, args):
     return {"workload": f"{shape.name}: d_model {shape.d_model}, {shape.n_layers} layers "
-                        f"({'all ladder' if shape.layer_is_ladder is None else 'hybrid mask'}), "
+                        f"({'all ladder' if shape.layer_is_ladder is None else ('all standard' if not any(shape.layer_is_ladder) else 'hybrid mask')}), "
                         f"{shape.n_q_heads}q/{shape.n_kv_heads}kv heads x {shape.head_dim}, ffn {shape.d_ff}, "
                         f"vocab {shape.vocab_size}",
             "batch": shape.batch, "prompt_len": shape.prompt_len, "decode_steps": args.steps,
@@ -205,6 +207,7 @@ def main():
     ap.add_argument("--graph", type=int, default=None)
     ap.add_argument("--pdl", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="sequences decoded together (default: the configuration's)")
+    ap.add_argument("--standard", action="store_true", help="the same shape with standard residuals (Eq. 1) in every layer")
     ap.add_argument("--multi-kernel", action="store_true",
                     help="one kernel per GEMM (two streams, CUDA graph, PDL) instead of the persistent decode kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -236,6 +239,8 @@ def main():
     shape = synth.SHAPES[args.config]
     if args.batch:
         shape = synth.replace(shape, batch=args.batch)
+    if args.standard:
+        shape = shape.as_standard()
     steps, warm = args.steps, max(args.warmup, 0)
     S, bsz = shape.prompt_len, shape.batch
     max_seq = S + max(steps, warm)

@@ -2,10 +2,11 @@
 //
 // One cooperative launch, one CTA per SM, runs EVERY weight-streaming GEMM of a decode step (QKV,
 // Wo, gate/up, down of each layer and the LM head) plus the attention of every layer.  The GEMMs are
-// "phases" walked in a fixed order by all CTAs; inside a phase the 8-row units of W are claimed in
-// batches through an atomic counter, exactly as in the per-GEMM kernel.  What used to be a kernel
-// boundary is a counter in global memory (units finished per phase): a reader polls it, with an
-// acquire load and a time limit, only before it touches data another SM produced.
+// "phases" walked in a fixed order by all CTAs; inside a phase the 8-row units of W are handed out in
+// batches: whole rounds of one batch per CTA statically (batch i to CTA i mod grid), the short batches
+// at the end of a long phase through an atomic counter.  What used to be a kernel boundary is a counter
+// in global memory (units finished per phase): a reader polls it, with an acquire load and a time
+// limit, only before it touches data another SM produced.
 //
 // Why: the weight stream of a phase depends on nothing, so the producer warp runs through phase
 // after phase and the TMA ring never drains, whatever the consumers are waiting for.  With the
@@ -24,12 +25,15 @@
 //   warps 1-3     finishers: K-split reduction, 1/rms, epilogue (residual add / SwiGLU / rotary + KV
 //                 append), then publish the finished units (fence + release add)
 //   warps 4-7     consumers: mma.sync m16n8k16 with the weights as the A operand (see decode_gemm.cu)
-//   warps 8-11    stagers: fp32 activations -> bf16 hi (+ lo) MMA operands, one chunk ahead; RMSNorm
-//                 sum of squares on the fly
+//   warps 8-11    stagers: the MMA operand form of the activations (bf16 hi + lo), one chunk ahead: copied
+//                 when the phase that produced them wrote that form too (its epilogue does, with this
+//                 phase's RMSNorm gain folded in), else converted from fp32; RMSNorm sum of squares from
+//                 the fp32 rows while the first batch of a phase is staged
 //   warps 12-15   attention: split-KV partials (64 keys x head group x sequence per unit), then the
 //                 log-sum-exp merge, units dealt round-robin over the CTAs
 // Data produced inside the launch is always read through L2 (ld.global.cg / acquire), never through
-// the non-coherent L1 path.  Every wait is bounded (0.25 s) and also gives up when another CTA has
+// the non-coherent L1 path and never by the TMA engine (a bulk copy of bytes other SMs had just written
+// returned stale data now and then, proxy fences on both sides notwithstanding).  Every wait is bounded (0.25 s) and also gives up when another CTA has
 // reported a timeout in the device status word, so a protocol error ends the launch quickly with
 // LADDER_DEV_TIMEOUT set instead of hanging the device.
 #include "common.cuh"
@@ -175,6 +179,8 @@ __device__ unsigned long long g_stack_trace[148 * 16];
 __device__ unsigned long long g_kind_trace[148 * 16];
 // consumer timeline: [phase][cta][0] first item of the phase taken up, [1] last item of the phase handed over (ns)
 __device__ unsigned long long g_phase_trace[330 * 148 * 2];
+// attention timeline of CTA 0: [layer][0] dependencies met [1] own split units done [2] all splits done [3] merge done (ns)
+__device__ unsigned long long g_attn_trace[128 * 4];
 #define TR_DECL(n) long long tr_##n = 0
 #define TR_T0() const long long tr_t0_ = clock64()
 #define TR_ADD(n) tr_##n += clock64() - tr_t0_
@@ -1216,6 +1222,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       // q and this step's key/value rows are written; the partials of the previous layer are merged
       ok = bar_and(3, kAux, wait_deps(A->dep, A->need, A->n_deps, sp.counters, status, lane));
       if (!ok) break;
+#ifdef DS_TRACE
+      if (at == 0 && blockIdx.x == 0 && li < 128) g_attn_trace[li * 4 + 0] = global_timer_ns();
+#endif
       const int total = pre[batch] * HG;
       int mine = 0;
       for (int u = blockIdx.x; u < total; u += gridDim.x) {
@@ -1236,12 +1245,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       __threadfence();
       bar_sync(3, kAux);
       if (at == 0 && mine > 0) red_release_add(sp.counters + A->split_done, mine);
+#ifdef DS_TRACE
+      if (at == 0 && blockIdx.x == 0 && li < 128) g_attn_trace[li * 4 + 1] = global_timer_ns();
+#endif
       // all partials of this layer (every CTA's) before any merge; o free to overwrite
       bool okw = true;
       if (lane == 0) okw = wait_global_ge(sp.counters + A->split_done, total, status);
       okw = __all_sync(0xffffffffu, okw) && wait_deps(A->mdep, A->mneed, A->n_mdeps, sp.counters, status, lane);
       ok = bar_and(3, kAux, okw);
       if (!ok) break;
+#ifdef DS_TRACE
+      if (at == 0 && blockIdx.x == 0 && li < 128) g_attn_trace[li * 4 + 2] = global_timer_ns();
+#endif
       const int n_pairs = batch * Hq;
       mine = 0;
       for (int u = blockIdx.x; u < n_pairs; u += gridDim.x) {
@@ -1254,6 +1269,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       __threadfence();
       bar_sync(3, kAux);
       if (at == 0 && mine > 0) red_release_add(sp.counters + A->merge_done, mine);
+#ifdef DS_TRACE
+      if (at == 0 && blockIdx.x == 0 && li < 128) g_attn_trace[li * 4 + 3] = global_timer_ns();
+#endif
     }
     if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
   }
@@ -1266,6 +1284,9 @@ bool g_stack_usable = false;
 #ifdef DS_TRACE
 extern "C" int ladder_debug_read_stack_trace(unsigned long long* host_out) {
   return cudaMemcpyFromSymbol(host_out, g_stack_trace, sizeof(g_stack_trace)) == cudaSuccess ? 0 : 1;
+}
+extern "C" int ladder_debug_read_attn_trace(unsigned long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_attn_trace, sizeof(g_attn_trace)) == cudaSuccess ? 0 : 1;
 }
 extern "C" int ladder_debug_read_kind_trace(unsigned long long* host_out) {
   return cudaMemcpyFromSymbol(host_out, g_kind_trace, sizeof(g_kind_trace)) == cudaSuccess ? 0 : 1;

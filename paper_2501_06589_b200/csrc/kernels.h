@@ -42,12 +42,12 @@ struct SmallMParams {
   // y = value (* pack_gain[n]), bf16 hi at [n / 2048][b][n % 2048], lo at [n / 2048][4 + b][n % 2048]; batch <= 4.
   __nv_bfloat16* pack_out;
   const __nv_bfloat16* pack_gain;
-  // batch <= 8 (dynamic item claiming, split-K fix-up):
-  float* scratch;          // smallm_gemm_scratch_floats(N, K, batch) floats, ticket part zero; kernels that
-                           // may run concurrently need distinct scratch
-  int32_t* work;           // 2 ints, zero: claim counter + finished-CTA counter of THIS launch (left zero)
-  float* part;             // set by the launcher: partial sums inside scratch
-  int32_t* tickets;        // set by the launcher: ticket counters inside scratch
+  float* scratch;          // smallm_gemm_scratch_floats(N, K, batch) floats, zero at first use (batch 9..64: staged
+                           // activations, tickets and shared-tile pieces); kernels that may run concurrently
+                           // need distinct scratch
+  int32_t* work;           // batch <= 8: 2 ints, zero: claim counter + finished-CTA counter of THIS launch (left zero)
+  float* part;             // unused
+  int32_t* tickets;        // unused
 };
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);

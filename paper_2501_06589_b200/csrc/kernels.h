@@ -46,8 +46,6 @@ struct SmallMParams {
                            // activations, tickets and shared-tile pieces); kernels that may run concurrently
                            // need distinct scratch
   int32_t* work;           // batch <= 8: 2 ints, zero: claim counter + finished-CTA counter of THIS launch (left zero)
-  float* part;             // unused
-  int32_t* tickets;        // unused
 };
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);

@@ -77,7 +77,7 @@ constexpr int AUX_PS = 4 * 8 * 16 * 4;
 constexpr int AUX_RED = 4 * 2 * 128 * 4;   // [4 warps][2 heads][128] floats per merge round; the merge step reuses it for its weights
 static_assert(AUX_RED >= kMaxSplits * 4, "merge weights do not fit");
 constexpr int AUX_MLS = 4 * 8 * 2 * 4;
-constexpr int AUX_MISC = 128;  // prefix of live splits per sequence [9], merge reductions [8]
+constexpr int AUX_MISC = 128;  // prefix of live splits [9], merge reductions [8], lengths [8]
 constexpr int SMEM = OFF_AUX + AUX_PS + AUX_RED + AUX_MLS + AUX_MISC + 128;
 static_assert(SMEM <= 227 * 1024, "shared memory budget");
 
@@ -1190,16 +1190,20 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
     int* pre = reinterpret_cast<int*>(smem + OFF_AUX + AUX_PS + AUX_RED + AUX_MLS);  // [9] prefix of live splits
     float* red_m = reinterpret_cast<float*>(pre + 12);
     float* red_l = red_m + 4;
+    int* lens_s = pre + 20;  // [8] keys attended per sequence
     bool ok = true;
-    if (sp.n_attn > 0 && at == 0) {
-      const DecodeAttnParams& a0 = sp.attn[0].a;
-      int acc = 0;
-      pre[0] = 0;
-      for (int b = 0; b < batch; ++b) {
-        int L = a0.kv_len[b] + a0.kv_len_offset;
-        L = max(0, min(L, a0.max_seq_len));
-        acc += (L + kChunk - 1) / kChunk;
-        pre[b + 1] = acc;
+    if (sp.n_attn > 0) {
+      if (at == 0) {
+        const DecodeAttnParams& a0 = sp.attn[0].a;
+        int acc = 0;
+        pre[0] = 0;
+        for (int b = 0; b < batch; ++b) {
+          int L = a0.kv_len[b] + a0.kv_len_offset;
+          L = max(0, min(L, a0.max_seq_len));
+          lens_s[b] = L;
+          acc += (L + kChunk - 1) / kChunk;
+          pre[b + 1] = acc;
+        }
       }
     }
     bar_sync(3, kAux);
@@ -1232,8 +1236,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         int b = 0;
         while (b + 1 < batch && t >= pre[b + 1]) ++b;
         const int split = t - pre[b];
-        int L = A->a.kv_len[b] + A->a.kv_len_offset;
-        L = max(0, min(L, max_seq));
+        const int L = lens_s[b];
         if (DH == 128)
           attn_split_dispatch<128>(gt, q, Kc, Vc, Hq, Hkv, max_seq, stride_splits, scratch, b, split, hg, L, ps, ared,
                                    mls, at);

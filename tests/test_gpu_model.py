@@ -328,3 +328,51 @@ def test_persistent_kernel_wait_runs_out_cleanly(B):
     for (t_a, h_a), (t_b, h_b) in zip(ref, again):
         assert torch.equal(t_a, t_b) and torch.equal(h_a, h_b)
     model.close()
+
+
+def test_plan_is_rebuilt_when_batch_buffers_or_mode_change(B):
+    """The persistent kernel's phase list is cached per (batch, cache buffers, logits buffer): decoding with
+    another batch size, another cache, the other schedule, or two models side by side gives the same
+    tokens and hidden states as a fresh model does."""
+    s = synth.replace(synth.SHAPES["tiny"], layer_is_ladder=(0, 1, 1, 1))
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    S, steps = 12, 4
+
+    def generate(model, cache, bsz, seed_shift=0):
+        prompt = torch.from_numpy(synth.make_tokens(s, 4, S)[:bsz].copy()).cuda() if seed_shift == 0 else \
+            torch.from_numpy((synth.make_tokens(s, 4, S)[:bsz] + seed_shift) % s.vocab_size).to(torch.int32).cuda()
+        nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+        hid = torch.zeros(bsz, s.d_model, device="cuda")
+        model.prefill(cache, prompt, next_tokens=nxt)
+        out = []
+        for _ in range(steps):
+            model.decode_step(cache, nxt, next_tokens=nxt, final_hidden=hid)
+            out.append((nxt.clone(), hid.clone()))
+        torch.cuda.synchronize()
+        return out
+
+    def fresh(bsz, seed_shift=0):
+        m = B.Model(w, 4, 32, 4 * S)
+        c = B.KVCache(s, 4, 32)
+        r = generate(m, c, bsz, seed_shift)
+        m.close()
+        return r
+
+    def same(a, b):
+        return all(torch.equal(x[0], y[0]) and torch.equal(x[1], y[1]) for x, y in zip(a, b))
+
+    ref4, ref2, ref3 = fresh(4), fresh(2), fresh(3, seed_shift=7)
+    model = B.Model(w, 4, 32, 4 * S)
+    other = B.Model(w, 4, 32, 4 * S)          # a second model alive at the same time
+    c1, c2 = B.KVCache(s, 4, 32), B.KVCache(s, 4, 32)
+    assert same(generate(model, c1, 4), ref4)
+    assert same(generate(model, c1, 2), ref2)                 # smaller batch, same cache
+    assert same(generate(other, c2, 3, seed_shift=7), ref3)   # other model, other cache, in between
+    assert same(generate(model, c2, 4), ref4)                 # other cache
+    model.set_persistent(False)
+    assert same(generate(model, c1, 2), ref2)                 # one kernel per GEMM
+    model.set_persistent(True)
+    assert same(generate(model, c1, 4), ref4)
+    assert model.device_status() == 0 and other.device_status() == 0
+    model.close()
+    other.close()

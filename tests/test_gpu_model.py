@@ -376,3 +376,13 @@ def test_plan_is_rebuilt_when_batch_buffers_or_mode_change(B):
     assert model.device_status() == 0 and other.device_status() == 0
     model.close()
     other.close()
+
+
+@pytest.mark.parametrize("batch", [5, 8])
+def test_tiny_config_batch_5_to_8(B, batch):
+    """Batches 5..8 take the persistent kernel's other instantiation (eight separate MMA columns, activations as a
+    single bf16, converted by the stagers in every phase)."""
+    s = synth.replace(synth.SHAPES["tiny"], layer_is_ladder=(0, 1, 1, 1))
+    err, agree, *_ = check_generation(B, s, 40, np.float64, gains="uniform", batch=batch)
+    assert err < HIDDEN_TOL, err
+    assert agree >= 0.98, agree

@@ -207,6 +207,8 @@ def main():
     ap.add_argument("--graph", type=int, default=None)
     ap.add_argument("--pdl", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="sequences decoded together (default: the configuration's)")
+    ap.add_argument("--wide-impl", type=int, default=0,
+                    help="decode GEMM kernels: 0 = default, 1 = mma.sync for batch 9..64, 2 = tcgen05 for every batch")
     ap.add_argument("--standard", action="store_true", help="the same shape with standard residuals (Eq. 1) in every layer")
     ap.add_argument("--multi-kernel", action="store_true",
                     help="one kernel per GEMM (two streams, CUDA graph, PDL) instead of the persistent decode kernel")
@@ -251,6 +253,7 @@ def main():
     torch.cuda.synchronize()
     t_gen = time.time() - t0
     model = B.Model(w, bsz, max_seq, bsz * S)
+    B.set_decode_wide_impl(args.wide_impl)
     if args.multi_kernel:
         model.set_persistent(False)
     persistent = model.persistent_active() and bsz <= 8

@@ -104,13 +104,34 @@ __global__ void argmax_advance_kernel(const float* logits, int vocab, int32_t* n
     const float* row = logits + static_cast<size_t>(b) * vocab;
     float best = -INFINITY;
     int idx = 0x7fffffff;
-    for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
-      const float v = row[i];
+    auto take = [&](float v, int i) {
       if (v > best || (v == best && i < idx)) {
         best = v;
         idx = i;
       }
+    };
+    // 16-byte loads, eight in flight per thread: the scan is latency-bound (one block per row)
+    const int n4 = (vocab & 3) == 0 && (reinterpret_cast<uintptr_t>(row) & 15) == 0 ? vocab >> 2 : 0;
+    const float4* row4 = reinterpret_cast<const float4*>(row);
+    for (int i0 = threadIdx.x; i0 < n4; i0 += 8 * blockDim.x) {
+      float4 v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int i = i0 + j * blockDim.x;
+        v[j] = i < n4 ? __ldcg(row4 + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int i = (i0 + j * blockDim.x) * 4;
+        if (i < vocab) {
+          take(v[j].x, i);
+          take(v[j].y, i + 1);
+          take(v[j].z, i + 2);
+          take(v[j].w, i + 3);
+        }
+      }
     }
+    for (int i = n4 * 4 + threadIdx.x; i < vocab; i += blockDim.x) take(row[i], i);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       const float ov = __shfl_xor_sync(0xffffffffu, best, o);

@@ -89,7 +89,7 @@ def check_generation(B, shape, steps, dtype, gains="ones", schedule=None, min_ag
     return err, agree, toks, hids, cache
 
 
-@pytest.mark.parametrize("variant", ["ladder", "standard", "hybrid", "hybrid_top"])
+@pytest.mark.parametrize("variant", ["ladder", "standard", "hybrid", "hybrid_top", "gqa2"])
 def test_tiny_config_full(B, variant):
     s = synth.SHAPES["tiny"]
     if variant == "standard":
@@ -98,6 +98,8 @@ def test_tiny_config_full(B, variant):
         s = synth.replace(s, layer_is_ladder=(0, 1, 1, 0))
     elif variant == "hybrid_top":      # standard layers run kernel by kernel, the ladder stretch above them persistently
         s = synth.replace(s, layer_is_ladder=(0, 0, 1, 1))
+    elif variant == "gqa2":            # two query heads per kv head (attention units of 2 heads)
+        s = synth.replace(s, n_kv_heads=2)
     err, agree, *_ = check_generation(B, s, 64, np.float64, gains="uniform", batch=4)     # 4 x 65 comparisons
     assert err < HIDDEN_TOL, err
     assert agree >= 0.99, agree

@@ -388,3 +388,11 @@ def test_tiny_config_batch_5_to_8(B, batch):
     err, agree, *_ = check_generation(B, s, 40, np.float64, gains="uniform", batch=batch)
     assert err < HIDDEN_TOL, err
     assert agree >= 0.98, agree
+
+
+def test_tiny_long_context_many_splits(B):
+    """8250 cached keys: 129 attention splits per head, more than the 64 threads of a merge unit own one each."""
+    s = synth.SHAPES["tiny"]
+    err, agree, *_ = check_generation(B, s, 4, np.float64, gains="uniform", batch=1, prompt_len=8250)
+    assert err < HIDDEN_TOL, err
+    assert agree >= 0.8, agree           # 5 comparisons: at most one flip

@@ -766,9 +766,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         return s;
       };
       smallm_epilogue<kFin>(*finp, ft, rows, row0, batch, value);
-      __threadfence();       // this thread's outputs are visible device-wide ...
-      bar_sync(2, kFin);     // ... for all finisher threads ...
-      if (ft == 0) red_release_add(done_ctr, nu);  // ... before the units count as finished
+      // all finisher threads' outputs are ordered before the release by the barrier (the release is cumulative)
+      bar_sync(2, kFin);
+      if (ft == 0) red_release_add(done_ctr, nu);
       if (lane == 0) mbar_arrive(&red_free[slot]);
     }
     if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
@@ -1245,7 +1245,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
                                   at);
         ++mine;
       }
-      __threadfence();
       bar_sync(3, kAux);
       if (at == 0 && mine > 0) red_release_add(sp.counters + A->split_done, mine);
 #ifdef DS_TRACE
@@ -1269,7 +1268,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         else attn_merge_unit<64>(scratch, Hq, stride_splits, ns, b, h, o, o_pack, ared, red_m, red_l, at);
         ++mine;
       }
-      __threadfence();
       bar_sync(3, kAux);
       if (at == 0 && mine > 0) red_release_add(sp.counters + A->merge_done, mine);
 #ifdef DS_TRACE

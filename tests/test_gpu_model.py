@@ -396,3 +396,35 @@ def test_tiny_long_context_many_splits(B):
     err, agree, *_ = check_generation(B, s, 4, np.float64, gains="uniform", batch=1, prompt_len=8250)
     assert err < HIDDEN_TOL, err
     assert agree >= 0.8, agree           # 5 comparisons: at most one flip
+
+
+def test_70b_shape_persistent_equals_multi_kernel_repeatedly(B):
+    """At the 70B layer shape (4 K chunks, many batches per CTA, operands handed from epilogue to stager) the
+    persistent kernel and the one-kernel-per-GEMM schedule give identical bits, run after run: any hand-over
+    that is not properly ordered shows up here as a sporadic difference."""
+    s = synth.SHAPES["70b"].with_layers(2)
+    w = synth.make_weights(s, device="cuda")
+    bsz, S, steps = 4, 64, 4
+    prompt = torch.from_numpy(synth.make_tokens(s, bsz, S)).cuda()
+
+    def run(persistent):
+        model = B.Model(w, bsz, S + steps + 1, bsz * S)
+        model.set_persistent(persistent)
+        cache = B.KVCache(s, bsz, S + steps + 1)
+        nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+        hid = torch.zeros(bsz, s.d_model, device="cuda")
+        model.prefill(cache, prompt, next_tokens=nxt)
+        outs = []
+        for _ in range(steps):
+            model.decode_step(cache, nxt, next_tokens=nxt, final_hidden=hid)
+            outs.append((nxt.clone(), hid.clone()))
+        torch.cuda.synchronize()
+        assert model.device_status() == 0
+        model.close()
+        return outs
+
+    ref = run(False)
+    for rep in range(4):
+        got = run(True)
+        for i, ((t0, h0), (t1, h1)) in enumerate(zip(ref, got)):
+            assert torch.equal(t0, t1) and torch.equal(h0, h1), (rep, i)

@@ -1107,22 +1107,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       // before the buffer is handed back (act_free)
       for (int ch = 0; ch < nchunk; ++ch, ++r) {
         // Operands already in MMA form (written by the producing phase's epilogue): the chunk is copied as it
-        // is, 16 bytes at a time, loaded before the buffer is handed back.  Otherwise convert from fp32.  The
-        // fp32 rows are still read while the first batch of a normalised phase is staged, for the sums of
-        // squares only.
+        // is with cp.async (16 bytes per copy, L2 -> shared memory, generic proxy: coherent like ld.global.cg)
+        // once the buffer has been handed back.  Otherwise convert from fp32.  The fp32 rows are still read
+        // while the first batch of a normalised phase is staged, for the sums of squares only.
         const bool copy = actp != nullptr;
         if (copy && ssq_on) {  // the fp32 rows first (their registers are then free for the copy)
           load_rows(ch, 0);
           sumsq_rows();
-        }
-        if (copy) {  // 16 x 16 bytes per thread, held in the registers the conversion path uses for its fp32 rows
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int idx = st + j * 128, row = idx >> 8, col = idx & 255;  // 256 16-byte units per 4 KB row
-            F8& slot = x[j >> 2][(j >> 1) & 1];
-            float4& f = (j & 1) ? slot.b : slot.a;
-            f = __ldcg(reinterpret_cast<const float4*>(actp + (static_cast<size_t>(ch) * 8 + row) * TK) + col);
-          }
         }
         if (!copy) load_rows(ch, 0);
         {
@@ -1131,15 +1122,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
           TR_ADD(sfree);
         }
         if (!ok) break;
-        if (copy) {
+        if (copy) {  // 16 x 16 bytes per thread, global (L2) -> shared memory without a register round trip
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            const int idx = st + j * 128, row = idx >> 8, col = idx & 255;
-            const F8& slot = x[j >> 2][(j >> 1) & 1];
-            const float4& f = (j & 1) ? slot.b : slot.a;
-            sts128(act_u32 + row * PITCH + col * 16,
-                   make_uint4(__float_as_uint(f.x), __float_as_uint(f.y), __float_as_uint(f.z), __float_as_uint(f.w)));
+            const int idx = st + j * 128, row = idx >> 8, col = idx & 255;  // 256 16-byte units per 4 KB row
+            const __nv_bfloat16* src = actp + (static_cast<size_t>(ch) * 8 + row) * TK + col * 8;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(act_u32 + row * PITCH + col * 16), "l"(src)
+                         : "memory");
           }
+          asm volatile("cp.async.wait_all;" ::: "memory");
         } else {
           store_rows(0);
           if (!PACKED && batch > 4) {

@@ -183,7 +183,11 @@ ladder_status_t ladder_prefill_host(ladder_model_t* m, const ladder_kv_cache_t* 
                                     int32_t batch, int32_t seq_len, int32_t* h_next_tokens, void* cuda_stream);
 
 /* Tell the library that every sequence of the cache now holds `len` tokens (e.g. after the
- * caller restored a cache snapshot or rewound seq_lens itself).  Host-side only. */
+ * caller restored a cache snapshot or rewound seq_lens itself).  Host-side only.
+ * Sequences of different lengths: positions are per sequence on the device, only this host-side overflow
+ * check assumes one length.  Fill sequence b alone with a batch-1 prompt pass on a cache struct whose k and v
+ * point n_kv_heads*max_seq_len*head_dim elements further per sequence skipped and whose seq_lens points at
+ * entry b, then call this with the LONGEST length and decode all sequences together. */
 ladder_status_t ladder_set_position(ladder_model_t* m, int32_t len);
 
 /* Synchronises `cuda_stream`, returns the device status word (LADDER_DEV_* bits) and clears it. */

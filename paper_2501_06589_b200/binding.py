@@ -191,6 +191,17 @@ class KVCache:
         self.dims = (shape.n_layers, max_batch, shape.n_kv_heads, max_seq_len, shape.head_dim)
         self.c = ladder_kv_cache_t(self.k.data_ptr(), self.v.data_ptr(), self.seq_lens.data_ptr())
 
+    def slot(self, b: int) -> "KVCache":
+        """The same buffers seen from sequence b on (its rows of every layer come first, its length first in
+        seq_lens): a prompt pass with batch 1 on it fills sequence b alone, so sequences of different lengths can
+        be filled one by one and then decoded together."""
+        view = object.__new__(KVCache)
+        _, mb, hkv, ms, dh = self.dims
+        off = b * hkv * ms * dh
+        view.k, view.v, view.seq_lens, view.dims = self.k[off:], self.v[off:], self.seq_lens[b:], self.dims
+        view.c = ladder_kv_cache_t(view.k.data_ptr(), view.v.data_ptr(), view.seq_lens.data_ptr())
+        return view
+
     def k5(self) -> torch.Tensor:
         return self.k.view(*self.dims)
 

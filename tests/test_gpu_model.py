@@ -428,3 +428,42 @@ def test_70b_shape_persistent_equals_multi_kernel_repeatedly(B):
         got = run(True)
         for i, ((t0, h0), (t1, h1)) in enumerate(zip(ref, got)):
             assert torch.equal(t0, t1) and torch.equal(h0, h1), (rep, i)
+
+
+@pytest.mark.parametrize("persistent", [True, False])
+def test_sequences_of_different_lengths_decode_together(B, persistent):
+    """Positions are per sequence on the device (seq_lens): three prompts of 5, 16 and 9 tokens, filled one by one,
+    then decoded as one batch, against the oracle run on each sequence alone."""
+    s = synth.SHAPES["tiny"]
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    lens, steps, max_seq = [5, 16, 9], 6, 32
+    toks = synth.make_tokens(s, 3, 16)
+    model = B.Model(w, 3, max_seq, 16)
+    model.set_persistent(persistent)
+    cache = B.KVCache(s, 3, max_seq, fill=CANARY)
+    nxt = torch.zeros(3, dtype=torch.int32, device="cuda")
+    hid = torch.zeros(3, s.d_model, device="cuda")
+    for b, L in enumerate(lens):                      # prompt passes, one sequence at a time
+        model.prefill(cache.slot(b), torch.from_numpy(toks[b:b + 1, :L].copy()).cuda(), next_tokens=nxt[b:b + 1])
+    assert cache.seq_lens.cpu().tolist() == lens
+    model.set_position(max(lens))                     # host-side overflow check follows the longest sequence
+    g_tok, g_hid = [nxt.clone()], []
+    for _ in range(steps):
+        model.decode_step(cache, nxt, next_tokens=nxt, final_hidden=hid)
+        g_tok.append(nxt.clone())
+        g_hid.append(hid.clone())
+    torch.cuda.synchronize()
+    assert model.device_status() == 0
+    assert cache.seq_lens.cpu().tolist() == [L + steps for L in lens]
+    g_tok = torch.stack(g_tok, 1).cpu().numpy()       # [3, steps + 1]
+    g_hid = torch.stack(g_hid, 1).cpu().numpy()       # [3, steps, d]
+    cfg = oracle_cfg(s)
+    OW = O.OracleWeights(provider=synth.logical_provider(w, np.float64))
+    for b, L in enumerate(lens):
+        o_tok, o_hid = O.generate(cfg, OW, toks[b:b + 1, :L], steps, max_seq, dtype=np.float64, forced=g_tok[b:b + 1])
+        assert rel_err(g_hid[b], o_hid[0, 1:]) < HIDDEN_TOL
+        assert np.mean(g_tok[b] == o_tok[0]) >= 0.85          # 7 comparisons per sequence: at most one flip
+    k5 = cache.k5().view(torch.int16)                          # [layer][b][h][pos][d]: rows beyond each length untouched
+    for b, L in enumerate(lens):
+        assert bool((k5[:, b, :, L + steps:, :] == CANARY).all()) and not bool((k5[:, b, :, :L + steps, :] == CANARY).any())
+    model.close()

@@ -1214,6 +1214,26 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         while (gt < 8 && group % (gt * 2) == 0) gt *= 2;
       }
       const int HG = Hq / gt;
+      // While the QKV phase of this layer is still running: pull the cached keys and values of the layer
+      // (everything but this step's row) into L2, so that the split units, which are on the critical path of
+      // small models, do not queue behind the weight stream in DRAM.  This CTA's share of the 128-byte lines.
+      // Only where the prefix is small (<= 8 MB per layer): at large shapes the gate/up phase hides the attention
+      // anyway and the prefetch only competes with the weight stream.
+      const size_t row_lines = static_cast<size_t>(DH) * 2 / 128;
+      if (static_cast<size_t>(pre[batch]) * kChunk * row_lines * Hkv * 2 * 128 <= (size_t(8) << 20)) {
+        for (int b = 0; b < batch; ++b) {
+          const int rows = max(0, lens_s[b] - 1);
+          const size_t per_head = static_cast<size_t>(rows) * row_lines;
+          const size_t total_lines = per_head * Hkv;
+          for (size_t i = static_cast<size_t>(blockIdx.x) * kAux + at; i < total_lines;
+               i += static_cast<size_t>(gridDim.x) * kAux) {
+            const size_t hk = i / per_head, r = i - hk * per_head;
+            const size_t off = ((static_cast<size_t>(b) * Hkv + hk) * max_seq) * DH + r * 64;  // bf16 elements
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(Kc + off));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(Vc + off));
+          }
+        }
+      }
       // q and this step's key/value rows are written; the partials of the previous layer are merged
       ok = bar_and(3, kAux, wait_deps(A->dep, A->need, A->n_deps, sp.counters, status, lane));
       if (!ok) break;

@@ -14,7 +14,7 @@
 //                   6..10-stage ring (20..32 KB per stage, ~100-160 KB of weights in flight per SM);
 //        warp 1     MMA issuer: tcgen05.mma M 128, N 2 Bp, K 16, kind::f16, fp32 accumulators in tensor
 //                   memory (two buffers, so the epilogue of one segment overlaps the MMAs of the next);
-//        warps 2-5  epilogue: tcgen05.ld (a thread owns one weight row and all batch columns), hi + lo,
+//        warps 2-9  epilogue: tcgen05.ld (a thread owns one weight row and half of the batch columns), hi + lo,
 //                   1/rms, then residual add (Eq. 1 / Eq. 2) / SwiGLU / rotary + KV append / plain store.
 // Work split: the T row tiles x nkb K blocks are cut into one contiguous range per CTA (equal to within
 // one K block), so every SM streams the same number of bytes whatever N and K are.  A tile whose K
@@ -32,7 +32,7 @@ namespace {
 
 constexpr int BM = 128, BK = 64, UMMA_K = 16;
 constexpr int W_BYTES = BM * BK * 2;  // 16 KB
-constexpr int kWideThreads = 192;
+constexpr int kWideThreads = 320;   // TMA producer warp, MMA warp, 8 epilogue warps
 constexpr int kWideMaxTiles = 2048;   // tickets
 constexpr int kWideMaxCtas = 160;     // partial slots
 
@@ -43,7 +43,7 @@ struct WCfg {
   static constexpr int STAGE_BYTES = W_BYTES + ACT_BYTES;
   static constexpr int STAGES = (200 * 1024) / STAGE_BYTES;
   static constexpr int OFF_BARS = STAGES * STAGE_BYTES;  // full[], empty[], tmem_full[2], tmem_empty[2], tmem slot, flag
-  static constexpr int SMEM = OFF_BARS + (2 * STAGES + 4) * 8 + 64 + 64 * 4 + 1024;
+  static constexpr int SMEM = OFF_BARS + (2 * STAGES + 4) * 8 + 64 + 2 * 64 * 4 + 1024;
   static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(NP >> 3) << 17) |
                                     (static_cast<uint32_t>(BM >> 4) << 24);
   static_assert(SMEM <= 232448, "shared memory budget");
@@ -100,6 +100,12 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 __device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t (&r)[8]) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
+__device__ __forceinline__ void tc_ld4(uint32_t taddr, uint32_t (&r)[4]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                : "r"(taddr)
                : "memory");
 }
@@ -165,22 +171,48 @@ __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const _
 }
 
 // ---------------------------------------------------------------- epilogue of one weight row
-// v[j] = finished accumulator of row n and batch row b0 + j.  Lanes of a warp hold consecutive rows,
-// so the (gate, up) and rotary pairs are neighbouring lanes; all lanes take part in the shuffles.
+// A thread owns weight row n and CB batch columns b0 .. b0 + CB - 1.  Lanes of a warp hold consecutive rows, so
+// the (gate, up) and rotary pairs are neighbouring lanes; all lanes take part in the shuffles.
+// Everything the tail reads from global memory (the residual addend, the rotary factors) is fetched by
+// epi_prefetch for all CB columns at once, ahead of the accumulators or pieces: a load placed after a store to
+// memory that may alias cannot be moved ahead of it by the compiler, and one dependent L2 round trip per
+// column cost 20 us per launch at batch 64.  pa = addend (EPI_RESID) or cos, pb = sin (EPI_QKV_ROPE).
+// pos_s[b] = position of batch row b (-1 for b >= batch), read once per CTA.
 template <int CB>
-__device__ __forceinline__ void wide_epilogue(const SmallMParams& p, int n, int b0, float (&v)[CB], int lane) {
+__device__ __forceinline__ void epi_prefetch(const SmallMParams& p, int n, int b0, int lane, const int* pos_s,
+                                             float (&pa)[CB], float (&pb)[CB]) {
+  const bool row_ok = n < p.N;
+  if (p.epi_mode == EPI_RESID) {
+#pragma unroll
+    for (int j = 0; j < CB; ++j)
+      pa[j] = (b0 + j < p.batch && row_ok) ? __ldcg(p.addend + static_cast<size_t>(b0 + j) * p.N + n) : 0.f;
+  } else if (p.epi_mode == EPI_QKV_ROPE) {
+    const QkvEpilogue& e = p.qkv;
+    const int Dh = e.head_dim;
+    const bool rotated = !(lane & 1) && row_ok && n < (e.n_q_heads + e.n_kv_heads) * Dh;
+#pragma unroll
+    for (int j = 0; j < CB; ++j) {
+      const int pos = pos_s[b0 + j];
+      const float2 cs = (rotated && pos >= 0 && pos < e.max_seq_len)
+                            ? __ldg(e.rope + static_cast<size_t>(pos) * (Dh >> 1) + ((n % Dh) >> 1))
+                            : make_float2(1.f, 0.f);
+      pa[j] = cs.x;
+      pb[j] = cs.y;
+    }
+  }
+}
+
+// v[j] = finished accumulator of row n and batch row b0 + j.
+template <int CB>
+__device__ __forceinline__ void epi_apply(const SmallMParams& p, int n, int b0, float (&v)[CB], int lane,
+                                          const int* pos_s, const float (&pa)[CB], const float (&pb)[CB]) {
   const bool row_ok = n < p.N;
   if (p.epi_mode == EPI_RESID || p.epi_mode == EPI_PLAIN) {
     float* out = static_cast<float*>(p.out);
 #pragma unroll
     for (int j = 0; j < CB; ++j) {
       const int b = b0 + j;
-      if (b < p.batch && row_ok) {
-        const size_t o = static_cast<size_t>(b) * p.N + n;
-        float r = v[j];
-        if (p.epi_mode == EPI_RESID) r += __ldcg(p.addend + o);
-        out[o] = r;
-      }
+      if (b < p.batch && row_ok) out[static_cast<size_t>(b) * p.N + n] = p.epi_mode == EPI_RESID ? v[j] + pa[j] : v[j];
     }
   } else if (p.epi_mode == EPI_SWIGLU) {
     float* out = static_cast<float*>(p.out);
@@ -201,14 +233,13 @@ __device__ __forceinline__ void wide_epilogue(const SmallMParams& p, int n, int 
       const int b = b0 + j;
       float v0 = v[j], v1 = __shfl_down_sync(0xffffffffu, v[j], 1);
       if ((lane & 1) || b >= p.batch || !row_ok) continue;
-      const int pos = e.seq_lens[b];
+      const int pos = pos_s[b];
       if (pos < 0 || pos >= e.max_seq_len) {
         if (p.status) atomicOr(p.status, LADDER_DEV_CACHE_OVERFLOW);
         continue;
       }
       if (n < nq + nk) {
-        const float2 cs = e.rope[static_cast<size_t>(pos) * (Dh >> 1) + ((n % Dh) >> 1)];
-        const float a0 = v0 * cs.x - v1 * cs.y, a1 = v0 * cs.y + v1 * cs.x;
+        const float a0 = v0 * pa[j] - v1 * pb[j], a1 = v0 * pb[j] + v1 * pa[j];
         v0 = a0;
         v1 = a1;
       }
@@ -224,13 +255,13 @@ __device__ __forceinline__ void wide_epilogue(const SmallMParams& p, int n, int 
   }
 }
 
-// barrier among the 128 epilogue threads that also ANDs a predicate, so that they leave together
+// barrier among the 256 epilogue threads that also ANDs a predicate, so that they leave together
 __device__ __forceinline__ bool epi_bar_and(bool pred) {
   uint32_t r;
   asm volatile(
       "{\n\t.reg .pred p, q;\n\t"
       "setp.ne.u32 p, %1, 0;\n\t"
-      "bar.red.and.pred q, 1, 128, p;\n\t"
+      "bar.red.and.pred q, 1, 256, p;\n\t"
       "selp.u32 %0, 1, 0, q;\n\t}"
       : "=r"(r)
       : "r"(static_cast<uint32_t>(pred))
@@ -248,13 +279,23 @@ struct Split {
   }
 };
 
+// Tuning build (-DWIDE_TRACE): global-timer stamps per CTA at the hand-over points of the last launch.
+#ifdef WIDE_TRACE
+__device__ unsigned long long g_wide_trace[kWideMaxCtas][8];
+#define WIDE_STAMP(i) g_wide_trace[blockIdx.x][i] = global_timer_ns()
+#else
+#define WIDE_STAMP(i)
+#endif
+
 template <int NP>
 __global__ void __launch_bounds__(kWideThreads, 1)
 decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap map_w,
                            const __grid_constant__ CUtensorMap map_act) {
   using C = WCfg<NP>;
   constexpr int BP = C::BP, STAGES = C::STAGES;
-  constexpr int CB = BP < 32 ? BP : 32;  // batch columns handled per epilogue pass
+  constexpr int HALVES = BP >= 16 ? 2 : 1;  // the batch columns are split between two sets of four epilogue warps
+  constexpr int CPH = BP / HALVES;
+  constexpr int CB = CPH < 16 ? CPH : 16;   // batch columns handled per epilogue pass
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + C::OFF_BARS);
@@ -264,6 +305,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
   volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* rstd_s = reinterpret_cast<float*>(smem + C::OFF_BARS + (2 * STAGES + 4) * 8 + 64);  // [BP] 1/rms
+  int* pos_s = reinterpret_cast<int*>(rstd_s + 64);                                            // [BP] positions
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const SmallMParams& p = a.p;
@@ -273,13 +315,14 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
   const int my_start = sp.start(blockIdx.x), my_end = sp.start(blockIdx.x + 1);
 
   if (tid == 0) {
+    WIDE_STAMP(0);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&tmem_full[b], 1);
-      mbar_init(&tmem_empty[b], 4);
+      mbar_init(&tmem_empty[b], 8);
     }
     fence_barrier_init();
   }
@@ -294,29 +337,38 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
   tc_fence_after();
   pdl_launch_dependents();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+  if (tid == 0) WIDE_STAMP(1);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       const uint64_t pol = l2_policy_evict_first();
-      bool ok = true, waited = false;
-      int it = 0;
-      for (int pos = my_start; pos < my_end && ok;) {
-        const int t = pos / nkb, kb0 = pos - t * nkb, kb1 = min(nkb, kb0 + (my_end - pos));
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % STAGES;
-          ok = mbar_wait_bounded(&empty[s], ((it / STAGES) & 1) ^ 1u);
-          if (!ok) break;
-          uint8_t* st = smem + s * C::STAGE_BYTES;
-          mbar_expect_tx(&full[s], C::STAGE_BYTES);
-          tma_load_2d_hint(st, &map_w, kb * BK, t * BM, &full[s], pol);
-          if (!waited) {  // the staged activations come from the kernel before this one; the weights do not
-            pdl_wait();
-            waited = true;
-          }
-          tma_load_2d(st + W_BYTES, &map_act, kb * BK, 0, &full[s]);
-        }
-        pos += kb1 - kb0;
+      bool ok = true;
+      const int n_it = my_end - my_start;
+      // First ring fill: the weight boxes of up to STAGES K blocks go out before the wait on the kernel that
+      // staged the activations (weights depend on nothing), their activation boxes right after it.
+      const int pre = n_it < STAGES ? n_it : STAGES;
+      for (int i = 0; i < pre; ++i) {
+        const int pos = my_start + i, t = pos / nkb, kb = pos - t * nkb;
+        mbar_expect_tx(&full[i], C::STAGE_BYTES);
+        tma_load_2d_hint(smem + i * C::STAGE_BYTES, &map_w, kb * BK, t * BM, &full[i], pol);
+      }
+      pdl_wait();
+      WIDE_STAMP(2);
+      for (int i = 0; i < pre; ++i) {
+        const int pos = my_start + i, kb = pos % nkb;
+        tma_load_2d(smem + i * C::STAGE_BYTES + W_BYTES, &map_act, kb * BK, 0, &full[i]);
+      }
+      int it = pre;
+      for (; it < n_it; ++it) {
+        const int s = it % STAGES;
+        ok = mbar_wait_bounded(&empty[s], ((it / STAGES) & 1) ^ 1u);
+        if (!ok) break;
+        const int pos = my_start + it, t = pos / nkb, kb = pos - t * nkb;
+        uint8_t* st = smem + s * C::STAGE_BYTES;
+        mbar_expect_tx(&full[s], C::STAGE_BYTES);
+        tma_load_2d_hint(st, &map_w, kb * BK, t * BM, &full[s], pol);
+        tma_load_2d(st + W_BYTES, &map_act, kb * BK, 0, &full[s]);
       }
       if (!ok) {
         if (p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
@@ -342,6 +394,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
           const int s = it % STAGES;
           ok = mbar_wait_bounded(&full[s], (it / STAGES) & 1);
           if (!ok) break;
+          if (it == 0) WIDE_STAMP(3);
           tc_fence_after();
           const uint32_t w_addr = smem_u32(smem + s * C::STAGE_BYTES);
           const uint64_t dw = smem_desc(w_addr), dact = smem_desc(w_addr + W_BYTES);
@@ -353,53 +406,64 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
         if (ok) tc_commit(&tmem_full[ab]);
         pos += kb1 - kb0;
       }
+      WIDE_STAMP(4);
       if (!ok && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
-    const int q = warp & 3;   // the TMEM lane quarter this warp may access
-    const int et = tid - 64;  // 0..127
-    const int r = q * 32 + lane;  // row inside the tile
+    const int q = warp & 3;          // the TMEM lane quarter this warp may access
+    const int half = (warp - 2) >> 2;  // which share of the batch columns
+    const int et = tid - 64;         // 0..255
+    const int r = q * 32 + lane;     // row inside the tile
+    const int c_begin = half < HALVES ? half * CPH : 0, c_end = half < HALVES ? c_begin + CPH : 0;
     bool ok = true;
     int seg = 0;
-    pdl_wait();  // the sums of squares, the addend and the destination belong to earlier kernels
+    pdl_wait();  // the sums of squares, the positions, the addend and the destination belong to earlier kernels
     if (et < BP) {   // 1/rms of every batch row: the K slices' sums of squares added in slice order
       float t = 0.f;
       if (p.act_mode == ACT_F32_NORM)
         for (int sl = 0; sl < a.n_slices; ++sl) t += a.ssq[et * a.n_slices + sl];
       rstd_s[et] = p.act_mode == ACT_F32_NORM ? rsqrtf(t / static_cast<float>(p.K) + p.eps) : 1.f;
+    } else if (et >= 128 && et - 128 < BP) {
+      const int b = et - 128;
+      pos_s[b] = (p.epi_mode == EPI_QKV_ROPE && b < p.batch) ? p.qkv.seq_lens[b] : -1;
     }
-    asm volatile("bar.sync 1, 128;" ::: "memory");
+    asm volatile("bar.sync 1, 256;" ::: "memory");
     for (int pos = my_start; pos < my_end; ++seg) {
       const int t = pos / nkb, kb0 = pos - t * nkb, kb1 = min(nkb, kb0 + (my_end - pos));
       pos += kb1 - kb0;
       const int ab = seg & 1;
       const bool whole = kb0 == 0 && kb1 == nkb;
-      ok = epi_bar_and(ok && mbar_wait_bounded(&tmem_full[ab], (seg >> 1) & 1));  // all four warps agree
-      if (!ok) break;
-      tc_fence_after();
       const int n = t * BM + r;
+      ok = epi_bar_and(ok && mbar_wait_bounded(&tmem_full[ab], (seg >> 1) & 1));  // all eight warps agree
+      if (!ok) break;
+      if (et == 0 && pos >= my_end) WIDE_STAMP(5);   // the last segment's accumulator is complete
+      tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + ab * NP;
       // where this CTA's piece of a shared tile goes: slot 0 if the tile is the first of its range, else slot 1
       const int my_slot = (t == my_start / nkb) ? 0 : 1;
-      float* piece = a.partial + (static_cast<size_t>(blockIdx.x) * 2 + my_slot) * BP * BM;
+      // piece layout: [TMEM lane quarter][group of 4 batch columns][lane] float4, so that a warp's store and
+      // the last arrival's load of one column group are 512 contiguous bytes
+      float4* piece = reinterpret_cast<float4*>(a.partial + (static_cast<size_t>(blockIdx.x) * 2 + my_slot) * BP * BM) +
+                      q * (BP / 4) * 32 + lane;
 #pragma unroll 1
-      for (int b0 = 0; b0 < BP; b0 += CB) {
-        float v[CB];
-        if constexpr (CB == 8) {
+      for (int b0 = c_begin; b0 < c_end; b0 += CB) {
+        float v[CB], pa[CB], pb[CB];
+        if (whole) epi_prefetch<CB>(p, n, b0, lane, pos_s, pa, pb);
+        if constexpr (CB == 4) {
+          uint32_t h[4], l[4];
+          tc_ld4(taddr + b0, h);
+          tc_ld4(taddr + BP + b0, l);
+          tc_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 4; ++j) v[j] = __uint_as_float(h[j]) + __uint_as_float(l[j]);
+        } else if constexpr (CB == 8) {
           uint32_t h[8], l[8];
           tc_ld8(taddr + b0, h);
           tc_ld8(taddr + BP + b0, l);
           tc_ld_wait();
 #pragma unroll
           for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(h[j]) + __uint_as_float(l[j]);
-        } else if constexpr (CB == 16) {
-          uint32_t h[16], l[16];
-          tc_ld16(taddr + b0, h);
-          tc_ld16(taddr + BP + b0, l);
-          tc_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(h[j]) + __uint_as_float(l[j]);
         } else {
 #pragma unroll
           for (int c = 0; c + 16 <= CB; c += 16) {
@@ -416,10 +480,10 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
 #pragma unroll
             for (int j = 0; j < CB; ++j) v[j] *= rstd_s[b0 + j];
           }
-          wide_epilogue<CB>(p, n, b0, v, lane);
+          epi_apply<CB>(p, n, b0, v, lane, pos_s, pa, pb);
         } else {
 #pragma unroll
-          for (int j = 0; j < CB; ++j) piece[(b0 + j) * BM + r] = v[j];
+          for (int j = 0; j < CB; j += 4) piece[((b0 + j) >> 2) * 32] = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
         }
       }
       tc_fence_before();
@@ -430,7 +494,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
       // ---- a tile shared with other CTAs: publish the piece; the last arrival adds all pieces in CTA
       // order and finishes the tile
       __threadfence();
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
       const int c_lo = sp.owner(t * nkb), c_hi = sp.owner((t + 1) * nkb - 1);
       if (et == 0) {
         const int prev = atomicAdd(a.tickets + t, 1);
@@ -438,29 +502,51 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
         if (last) a.tickets[t] = 0;  // ready for the next launch
         *last_flag = last;
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
       const bool last = *last_flag != 0;
-      asm volatile("bar.sync 1, 128;" ::: "memory");  // the flag is rewritten by the next shared tile
+      if (et == 0 && pos >= my_end) WIDE_STAMP(6);   // the last segment's piece is published
+      asm volatile("bar.sync 1, 256;" ::: "memory");  // the flag is rewritten by the next shared tile
       if (!last) continue;
       __threadfence();
+      // Up to 16 batch columns at a time with the pieces of up to four CTAs in flight together (16 independent
+      // 16-byte loads per thread, issued together with the tail's own reads); every element is still summed in
+      // CTA order.
+      constexpr int FB = CB;
+      const float4* mine = reinterpret_cast<const float4*>(a.partial) + q * (BP / 4) * 32 + lane;
 #pragma unroll 1
-      for (int b0 = 0; b0 < BP; b0 += CB) {
-        float v[CB];
+      for (int b0 = c_begin; b0 < c_end; b0 += FB) {
+        float v[FB], pa[FB], pb[FB];
+        epi_prefetch<FB>(p, n, b0, lane, pos_s, pa, pb);
 #pragma unroll
-        for (int j = 0; j < CB; ++j) v[j] = 0.f;
-        for (int c = c_lo; c <= c_hi; ++c) {
-          const int slot = (t == sp.start(c) / nkb) ? 0 : 1;
-          const float* src = a.partial + (static_cast<size_t>(c) * 2 + slot) * BP * BM;
+        for (int j = 0; j < FB; ++j) v[j] = 0.f;
+#pragma unroll 1
+        for (int c0 = c_lo; c0 <= c_hi; c0 += 4) {
+          float4 x[4][FB / 4];
 #pragma unroll
-          for (int j = 0; j < CB; ++j) v[j] += __ldcg(src + (b0 + j) * BM + r);
+          for (int u = 0; u < 4; ++u) {
+            const int c = min(c0 + u, c_hi);
+            const int slot = (t == sp.start(c) / nkb) ? 0 : 1;
+            const float4* src = mine + (static_cast<size_t>(c) * 2 + slot) * (BP * BM / 4) + (b0 >> 2) * 32;
+#pragma unroll
+            for (int g = 0; g < FB / 4; ++g) x[u][g] = __ldcg(src + g * 32);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            if (c0 + u > c_hi) break;
+#pragma unroll
+            for (int g = 0; g < FB / 4; ++g) {
+              v[4 * g] += x[u][g].x, v[4 * g + 1] += x[u][g].y, v[4 * g + 2] += x[u][g].z, v[4 * g + 3] += x[u][g].w;
+            }
+          }
         }
         if (p.act_mode == ACT_F32_NORM) {
 #pragma unroll
-          for (int j = 0; j < CB; ++j) v[j] *= rstd_s[b0 + j];
+          for (int j = 0; j < FB; ++j) v[j] *= rstd_s[b0 + j];
         }
-        wide_epilogue<CB>(p, n, b0, v, lane);
+        epi_apply<FB>(p, n, b0, v, lane, pos_s, pa, pb);
       }
     }
+    if (et == 0) WIDE_STAMP(7);
     if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
   }
 
@@ -515,6 +601,12 @@ cudaError_t launch_np(const WideArgs& a, const CUtensorMap& mw, const CUtensorMa
 }
 
 }  // namespace
+
+#ifdef WIDE_TRACE
+extern "C" int ladder_debug_read_wide_trace(unsigned long long* host_out) {
+  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_wide_trace, sizeof(g_wide_trace)));
+}
+#endif
 
 cudaError_t smallm_gemm_wide_tc_init() {
   if (!g_encode_wide) {

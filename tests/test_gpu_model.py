@@ -229,6 +229,40 @@ def test_8b_hybrid_shape_short_context(B):
     assert agree >= 0.99, agree
 
 
+@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("case", ["tiny", "8b_shape"])
+def test_prompt_pass_every_position(B, case, impl):
+    """Hidden state of EVERY prompt position against the oracle, with the prompt-pass GEMMs on the tcgen05
+    kernel (0) and on the warp-level mma.sync kernel (1); ragged M (not a multiple of the 128-row tile)."""
+    if case == "tiny":
+        s, bsz, S, dtype = synth.replace(synth.SHAPES["tiny"], layer_is_ladder=(1, 0, 1, 1)), 3, 150, np.float64
+    else:
+        s = synth.replace(synth.SHAPES["8b_hybrid"].with_layers(8), layer_is_ladder=(0, 0, 0, 0, 1, 1, 1, 1))
+        bsz, S, dtype = 2, 200, np.float32
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    prompt = synth.make_tokens(s, bsz, S)
+    model = B.Model(w, bsz, S + 8, bsz * S)
+    cache = B.KVCache(s, bsz, S + 8, fill=CANARY)
+    allh = torch.zeros(bsz, S, s.d_model, device="cuda")
+    nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+    B.set_prefill_gemm_impl(impl)
+    try:
+        model.prefill(cache, torch.from_numpy(prompt).cuda(), next_tokens=nxt, all_hidden=allh)
+        torch.cuda.synchronize()
+    finally:
+        B.set_prefill_gemm_impl(0)
+    assert model.device_status() == 0
+    cfg = oracle_cfg(s)
+    OW = O.OracleWeights(provider=synth.logical_provider(w, dtype))
+    ref = O.forward(cfg, OW, prompt, dtype=dtype, last_only=False, with_logits=False)
+    err = rel_err(allh.cpu().numpy(), ref.hidden)
+    print(f"[{case} impl {impl}] prompt-pass hidden max-rel-err {err:.3e} over {bsz * S} positions")
+    assert err < HIDDEN_TOL, err
+    k5 = cache.k5().view(torch.int16)
+    assert bool((k5[:, :, :, S:, :] == CANARY).all()) and not bool((k5[:, :, :, :S, :] == CANARY).any())
+    model.close()
+
+
 def test_70b_full_size_single_live_module(B):
     """The benchmark's own launch configuration -- all 80 layers of the 70B shape resident (141 GB),
     batch 4, 1024-token prompts, CUDA-graph decode -- checked with a property that holds at any size:

@@ -30,6 +30,8 @@ def main():
     ap.add_argument("--multi-kernel", action="store_true", help="stack: use the per-GEMM schedule")
     ap.add_argument("--wide-impl", type=int, default=0,
                     help="decode GEMM: 0 = default, 1 = mma.sync kernel for batch 9..64, 2 = tcgen05 kernel for every batch")
+    ap.add_argument("--which", default="gate_up", choices=["qkv", "wo", "gate_up", "down"],
+                    help="prefill_gemm: which projection's shape and epilogue")
     a = ap.parse_args()
     build.build()
     B.lib()
@@ -82,6 +84,16 @@ def main():
         out_lo = torch.empty_like(out)
         fn = lambda l: B.op_prefill_gemm(A, W[l], 1, out, A_lo=A_lo, out_lo=out_lo)
         nbytes, flops = 0, 2.0 * M * 2 * F * d
+        if a.which != "gate_up":     # QKV without its rotary / cache epilogue (plain bf16 store); Wo and down add a residual
+            N, K, mode = {"qkv": (s.qkv_rows, d, 3), "wo": (d, Hq * Dh, 0), "down": (d, F, 0)}[a.which]
+            A = torch.randn(M, K, device=dev).to(torch.bfloat16)
+            A_lo = (torch.randn(M, K, device=dev) * 1e-3).to(torch.bfloat16)
+            W = w(N, K)
+            add = torch.randn(M, N, device=dev)
+            out = torch.empty(M, N, device=dev) if mode == 0 else torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+            out_lo = None if mode == 0 else torch.empty_like(out)
+            fn = lambda l: B.op_prefill_gemm(A, W[l], mode, out, addend=add if mode == 0 else None, A_lo=A_lo, out_lo=out_lo)
+            flops = 2.0 * M * N * K
     elif a.op == "prefill_attn":
         S = s.prompt_len
         q = torch.randn(bsz, S, Hq * Dh, device=dev).to(torch.bfloat16)

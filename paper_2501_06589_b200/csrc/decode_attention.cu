@@ -9,7 +9,8 @@
 //      nothing) as the A operand and key rows read straight from the cache as B fragments (the
 //      contraction index is permuted identically on both sides: 16 contiguous bytes per thread);
 //   2. fp32 softmax statistics per warp, probabilities to shared memory;
-//   3. P.V on the CUDA cores in fp32 from the value rows already in registers;
+//   3. P.V on the CUDA cores in fp32 from the value rows already in registers (batch <= 8), or on mma.sync
+//      with the probabilities as a bf16 hi + lo pair (batch > 8: see PVMMA below);
 //   4. the 4 warps are merged by log-sum-exp in shared memory and the CTA's (o, m, l) partial goes
 //      to an L2-resident scratch; a second, tiny kernel (one CTA per sequence and head, launched
 //      with programmatic dependent launch) merges the splits in a fixed order and writes o in fp32.
@@ -24,7 +25,12 @@ namespace {
 constexpr int kAttnThreads = 128;
 constexpr int kChunk = 64;  // keys per CTA (16 per warp)
 
-template <int GT, int DH>
+// PVMMA (used for batch > 8, where the step stops being latency-bound and this kernel became issue-bound on its
+// CUDA-core P.V loop: 65 % issue-slot use at 2.7 TB/s): P.V runs on mma.sync too.  The probabilities of head g
+// are already laid out as the A fragment (the score MMA's C fragment, as a bf16 hi + lo pair), and a lane reads
+// the value rows as 32-bit words V[key][16 j + 2 g, +1] for its four keys 2t, 2t+1, 2t+8, 2t+9, so that two byte
+// permutes turn them into the B fragments of an "even dims" and an "odd dims" MMA per 16 dims.
+template <int GT, int DH, bool PVMMA>
 __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const DecodeAttnParams p) {
   constexpr int DPL = DH / 32;  // dims per lane in the P.V phase
   constexpr int KJ = DH / 32;   // 16-byte loads per key per thread in the score phase
@@ -61,8 +67,20 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
                           : make_uint4(0, 0, 0, 0);
   }
   uint32_t vr[16][DPL / 2];
+  if constexpr (PVMMA) {  // [j][q] = V[kw0 + key(q)][16 j + 2 g, +1], key(q) = 2 tig + (q & 1) + 8 (q >> 1)
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+    for (int q4 = 0; q4 < 4; ++q4) {
+      const int key = kw0 + 2 * tig + (q4 & 1) + 8 * (q4 >> 1);
+#pragma unroll
+      for (int j = 0; j < DH / 16; ++j) {
+        const int i = j * 4 + q4;
+        vr[i / (DPL / 2)][i % (DPL / 2)] =
+            key < L ? *reinterpret_cast<const uint32_t*>(V + static_cast<size_t>(key) * DH + 16 * j + 2 * g) : 0u;
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < (PVMMA ? 0 : 16); ++i) {
     const int key = kw0 + i;
     if (DPL == 4) {
       const uint2 u = key < L ? *reinterpret_cast<const uint2*>(V + static_cast<size_t>(key) * DH + lane * DPL)
@@ -124,8 +142,10 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
   l += __shfl_xor_sync(0xffffffffu, l, 1);
   l += __shfl_xor_sync(0xffffffffu, l, 2);
   if (g < GT) {
-    *reinterpret_cast<float2*>(&ps[warp][g][2 * tig]) = make_float2(sv[0], sv[1]);
-    *reinterpret_cast<float2*>(&ps[warp][g][8 + 2 * tig]) = make_float2(sv[2], sv[3]);
+    if constexpr (!PVMMA) {
+      *reinterpret_cast<float2*>(&ps[warp][g][2 * tig]) = make_float2(sv[0], sv[1]);
+      *reinterpret_cast<float2*>(&ps[warp][g][8 + 2 * tig]) = make_float2(sv[2], sv[3]);
+    }
     if (tig == 0) {
       mls[warp][g][0] = m;
       mls[warp][g][1] = l;
@@ -133,6 +153,33 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
   }
   __syncwarp();
 
+  if constexpr (PVMMA) {
+    // ---- 3. P.V on the tensor cores: A = probabilities of (head g; keys 2t, 2t+1 | 2t+8, 2t+9), hi + lo
+    const uint32_t ph0 = pack_bf16x2(sv[0], sv[1]), ph1 = pack_bf16x2(sv[2], sv[3]);
+    const uint32_t pl0 = pack_bf16x2(sv[0] - bf16_lo(ph0), sv[1] - bf16_hi(ph0));
+    const uint32_t pl1 = pack_bf16x2(sv[2] - bf16_lo(ph1), sv[3] - bf16_hi(ph1));
+#pragma unroll
+    for (int j = 0; j < DH / 16; ++j) {
+      uint32_t w[4];
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        const int i = j * 4 + q4;
+        w[q4] = vr[i / (DPL / 2)][i % (DPL / 2)];
+      }
+      // even dims 16 j + 2 n and odd dims 16 j + 2 n + 1 as the two MMAs' columns n
+      const uint32_t be0 = __byte_perm(w[0], w[1], 0x5410), be1 = __byte_perm(w[2], w[3], 0x5410);
+      const uint32_t bo0 = __byte_perm(w[0], w[1], 0x7632), bo1 = __byte_perm(w[2], w[3], 0x7632);
+      float ce[4] = {0.f, 0.f, 0.f, 0.f}, co[4] = {0.f, 0.f, 0.f, 0.f};
+      mma_bf16_16816(ce, ph0, 0u, ph1, 0u, be0, be1);
+      mma_bf16_16816(ce, pl0, 0u, pl1, 0u, be0, be1);
+      mma_bf16_16816(co, ph0, 0u, ph1, 0u, bo0, bo1);
+      mma_bf16_16816(co, pl0, 0u, pl1, 0u, bo0, bo1);
+      // columns 2 tig, 2 tig + 1 of the two MMAs = dims 16 j + 4 tig .. + 3 of head g
+      if (g < GT) *reinterpret_cast<float4*>(&red[warp][g][16 * j + 4 * tig]) = make_float4(ce[0], co[0], ce[1], co[1]);
+    }
+  }
+
+  if constexpr (!PVMMA) {
   // ---- 3. P.V for the warp's 16 keys; lane owns dims [lane*DPL, +DPL)
   float acc[GT][DPL];
 #pragma unroll
@@ -166,6 +213,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
   for (int h = 0; h < GT; ++h)
 #pragma unroll
     for (int d = 0; d < DPL; ++d) red[warp][h][lane * DPL + d] = acc[h][d];
+  }
   __syncthreads();
 
   // ---- 4. merge the 4 warps, write the CTA partial
@@ -246,8 +294,12 @@ template <int GT>
 cudaError_t launch_gt(const DecodeAttnParams& p, cudaStream_t stream, bool pdl) {
   cudaLaunchAttribute at[1];
   cudaLaunchConfig_t cfg = make_cfg(dim3(p.n_splits, p.n_q_heads / GT, p.batch), dim3(kAttnThreads), stream, pdl, at);
-  if (p.head_dim == 128) return cudaLaunchKernelEx(&cfg, decode_attention_kernel<GT, 128>, p);
-  return cudaLaunchKernelEx(&cfg, decode_attention_kernel<GT, 64>, p);
+  if (p.batch > 8) {  // throughput regime: P.V on the tensor cores
+    if (p.head_dim == 128) return cudaLaunchKernelEx(&cfg, decode_attention_kernel<GT, 128, true>, p);
+    return cudaLaunchKernelEx(&cfg, decode_attention_kernel<GT, 64, true>, p);
+  }
+  if (p.head_dim == 128) return cudaLaunchKernelEx(&cfg, decode_attention_kernel<GT, 128, false>, p);
+  return cudaLaunchKernelEx(&cfg, decode_attention_kernel<GT, 64, false>, p);
 }
 
 int heads_per_cta(int n_q_heads, int n_kv_heads) {

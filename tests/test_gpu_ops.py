@@ -150,6 +150,11 @@ def test_smallm_gemm_is_deterministic_and_batch_invariant(B):
     (3, 32, 8, 128, 300, [0, 299, 37]),
     (2, 8, 1, 128, 2048, [2048, 2047]),
     (2, 6, 3, 64, 100, [100, 31]),
+    # batch > 8: the probabilities-times-values product runs on the tensor cores (bf16 hi + lo probabilities)
+    (12, 16, 2, 128, 300, [300, 1, 64, 65, 17, 128, 299, 0, 200, 77, 16, 255]),
+    (9, 4, 4, 64, 130, [130, 129, 1, 64, 63, 65, 100, 2, 33]),
+    (16, 8, 1, 128, 2048, [2048, 2047, 1025, 7] * 4),
+    (10, 12, 3, 64, 96, [96, 95, 80, 64, 48, 32, 16, 8, 4, 1]),
 ])
 def test_decode_attention(B, batch, Hq, Hkv, Dh, max_seq, lens):
     q = torch.randn(batch, Hq * Dh, generator=torch.Generator().manual_seed(11)).cuda()

@@ -165,6 +165,17 @@ ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attenti
 ladder_status_t ladder_prefill(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
                                int32_t batch, int32_t seq_len, const ladder_outputs_t* out, void* cuda_stream);
 
+/* Continues a prompt (chunked prompt pass): the seq_len new tokens of every sequence sit at positions
+ * L .. L+seq_len-1, where L is the common cached length the library tracks (set by ladder_prefill, a previous
+ * ladder_prefill_append, decode steps or ladder_set_position).  They attend to cache rows 0..L-1 and causally
+ * to each other; rows L..L+seq_len-1 are written, seq_lens[b] = L+seq_len, outputs are for the last new position
+ * (all_hidden: [batch, seq_len, d_model] of the new positions).  A prompt longer than max_prefill_tokens / batch
+ * is fed as ladder_prefill of its first chunk followed by appends; the result equals the one-call prompt pass up
+ * to summation order.  L+seq_len <= max_seq_len and batch*seq_len <= max_prefill_tokens, else LADDER_ERR_STATE.
+ * Same model equations as the prompt pass (Eq. 1 / Eq. 2 of the paper; the paper does not discuss chunking). */
+ladder_status_t ladder_prefill_append(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                                      int32_t batch, int32_t seq_len, const ladder_outputs_t* out, void* cuda_stream);
+
 /* One autoregressive step: consumes d_tokens int32 [batch] at position seq_lens[b] (read on
  * the device), appends K/V there, attends over positions 0..seq_lens[b], writes the outputs and
  * adds one to seq_lens[b].  d_tokens may alias out->next_tokens (device-side feedback loop).

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libladder.so")
 
 EXPORTS = [
     "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_model_set_sm_split", "ladder_model_set_persistent", "ladder_model_persistent_active", "ladder_stack_plan", "ladder_debug_stall_last_phase",
-    "ladder_prefill",
+    "ladder_prefill", "ladder_prefill_append",
     "ladder_decode_step", "ladder_decode_step_host", "ladder_prefill_host", "ladder_set_position",
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
     "ladder_last_error", "ladder_op_smallm_gemm", "ladder_decode_attention_scratch_bytes",
@@ -82,6 +82,8 @@ def lib() -> C.CDLL:
         L.ladder_stack_plan.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32]
         L.ladder_stack_plan.restype = C.c_int32
         L.ladder_prefill.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32, C.c_int32,
+                                     C.POINTER(ladder_outputs_t), C.c_void_p]
+        L.ladder_prefill_append.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32, C.c_int32,
                                      C.POINTER(ladder_outputs_t), C.c_void_p]
         L.ladder_decode_step.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32,
                                          C.POINTER(ladder_outputs_t), C.c_void_p]
@@ -277,6 +279,14 @@ class Model:
         o = self._outs(next_tokens, final_hidden, logits, all_hidden)
         _check(lib().ladder_prefill(self.h, C.byref(cache.c), _ptr(tokens), tokens.shape[0], tokens.shape[1],
                                     C.byref(o), _stream()), self.h)
+
+    def prefill_append(self, cache: KVCache, tokens: torch.Tensor, next_tokens=None, final_hidden=None, logits=None,
+                       all_hidden=None):
+        """Continues the prompt: tokens [batch, chunk] follow the positions already cached."""
+        assert tokens.dtype == torch.int32 and tokens.is_cuda and tokens.dim() == 2
+        o = self._outs(next_tokens, final_hidden, logits, all_hidden)
+        _check(lib().ladder_prefill_append(self.h, C.byref(cache.c), _ptr(tokens), tokens.shape[0], tokens.shape[1],
+                                           C.byref(o), _stream()), self.h)
 
     def decode_step(self, cache: KVCache, tokens: torch.Tensor, next_tokens=None, final_hidden=None, logits=None):
         assert tokens.dtype == torch.int32 and tokens.is_cuda

@@ -373,8 +373,10 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   return q.err;
 }
 
+// pos0: position of the first of the S new tokens of every sequence (0 = a fresh prompt; > 0 = the prompt is
+// continued: the new tokens attend to the pos0 cached positions and to each other causally).
 cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int batch, int S,
-                            const ladder_outputs_t* out, cudaStream_t st, int64_t* n_kernels) {
+                            const ladder_outputs_t* out, cudaStream_t st, int64_t* n_kernels, int pos0 = 0) {
   const ladder_config_t& c = m->cfg;
   const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff;
   const int M = batch * S;
@@ -410,10 +412,11 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       p.qkv.head_dim = Dh;
       p.qkv.max_seq_len = c.max_seq_len;
       p.qkv.prefill_seq_len = S;
+      p.qkv.prefill_pos0 = pos0;
       p.status = m->status;
       did(launch_largem_gemm(p, st));
       did(launch_prefill_attention(m->q_pf, m->q_pf + m->q_lo, p.qkv.k_cache, p.qkv.v_cache, batch, S, Hq, Hkv, Dh,
-                                   c.max_seq_len, m->o_pf, m->o_pf + m->q_lo, st));
+                                   c.max_seq_len, m->o_pf, m->o_pf + m->q_lo, st, pos0));
       LargeMParams o = {};
       o.A = m->o_pf;
       o.A_lo = m->o_pf + m->q_lo;
@@ -477,8 +480,8 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
   did(launch_smallm_gemm(h, st, false, m->sm_count));
   if (out && out->final_hidden)
     did(launch_rmsnorm_f32(m->last_x, m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, st, false));
-  did(launch_argmax_advance(logits, batch, c.vocab_size, out ? out->next_tokens : nullptr, cache->seq_lens, 0, S, st,
-                            false));
+  did(launch_argmax_advance(logits, batch, c.vocab_size, out ? out->next_tokens : nullptr, cache->seq_lens, 0, pos0 + S,
+                            st, false));
   *n_kernels = k;
   return err;
 }
@@ -1163,6 +1166,23 @@ ladder_status_t ladder_prefill(ladder_model_t* m, const ladder_kv_cache_t* cache
   CK(m, enqueue_prefill(m, cache, d_tokens, batch, seq_len, out, static_cast<cudaStream_t>(cuda_stream), &k));
   m->launches += k;
   m->host_len = seq_len;
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_prefill_append(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                                      int32_t batch, int32_t seq_len, const ladder_outputs_t* out, void* cuda_stream) {
+  ladder_status_t s = check_call(m, cache, d_tokens, batch);
+  if (s != LADDER_OK) return s;
+  if (seq_len < 1) return fail(m, LADDER_ERR_INVALID_ARG, "seq_len must be >= 1");
+  const int pos0 = m->host_len;
+  if (static_cast<int64_t>(pos0) + seq_len > m->cfg.max_seq_len)
+    return fail(m, LADDER_ERR_STATE, "cached length + seq_len exceeds max_seq_len");
+  if (static_cast<int64_t>(batch) * seq_len > m->cfg.max_prefill_tokens)
+    return fail(m, LADDER_ERR_STATE, "batch*seq_len exceeds max_prefill_tokens");
+  int64_t k = 0;
+  CK(m, enqueue_prefill(m, cache, d_tokens, batch, seq_len, out, static_cast<cudaStream_t>(cuda_stream), &k, pos0));
+  m->launches += k;
+  m->host_len = pos0 + seq_len;
   return LADDER_OK;
 }
 

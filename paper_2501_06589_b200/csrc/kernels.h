@@ -23,6 +23,7 @@ struct QkvEpilogue {
   const float2* rope;          // [max_seq][Dh/2] (cos, sin)
   int n_q_heads, n_kv_heads, head_dim, max_seq_len;
   int prefill_seq_len;         // prefill: rows are [batch, seq_len] flattened
+  int prefill_pos0;            // prefill: position of a sequence's first row (> 0 when a prompt is continued)
 };
 
 struct SmallMParams {
@@ -150,10 +151,11 @@ cudaError_t largem_gemm_tc_init();
 void set_prefill_gemm_impl(int impl);  // 0 = tcgen05 (default), 1 = mma.sync
 
 // q_lo / o_lo: optional lo parts (value ~ hi + lo) of the query input and the attention output.
+// pos0: the seq_len queries sit at positions pos0 .. pos0 + seq_len - 1 and attend to cache rows 0 .. their own.
 cudaError_t launch_prefill_attention(const __nv_bfloat16* q, const __nv_bfloat16* q_lo, const __nv_bfloat16* k,
                                      const __nv_bfloat16* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
                                      int head_dim, int max_seq_len, __nv_bfloat16* o, __nv_bfloat16* o_lo,
-                                     cudaStream_t stream);
+                                     cudaStream_t stream, int pos0 = 0);
 
 // Small element-wise / gather kernels.
 cudaError_t launch_embed(const int32_t* tokens, const __nv_bfloat16* table, int rows, int d, int vocab, float* x,

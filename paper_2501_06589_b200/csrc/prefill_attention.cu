@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
                                                                        const __nv_bfloat16* __restrict__ vc, int seq_len,
                                                                        int n_q_heads, int n_kv_heads, int max_seq_len,
                                                                        __nv_bfloat16* __restrict__ o,
-                                                                       __nv_bfloat16* __restrict__ o_lo) {
+                                                                       __nv_bfloat16* __restrict__ o_lo, const int pos0) {
   constexpr int P = DH + 8;  // smem pitch in elements
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __nv_bfloat16* sQ = reinterpret_cast<__nv_bfloat16*>(smem_raw);
@@ -69,14 +69,15 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
   const float scale = rsqrtf(static_cast<float>(DH));
   const int q_hi = min(q0 + kQT, seq_len) - 1;  // last valid query of the tile
-  const int n_kt = q_hi / kKT + 1;
+  const int n_keys = pos0 + seq_len;            // cache rows that exist for this call
+  const int n_kt = (pos0 + q_hi) / kKT + 1;
 
   for (int kt = 0; kt < n_kt; ++kt) {
     __syncthreads();  // previous tile fully consumed
     for (int i = tid; i < kKT * CPR; i += kPfThreads) {
       const int r = i / CPR, c = i % CPR;
       const int key = kt * kKT + r;
-      const bool v = key < seq_len;
+      const bool v = key < n_keys;
       const size_t off = v ? static_cast<size_t>(key) * DH + c * 8 : 0;
       cp16(smem_u32(sK + r * P + c * 8), kg + off, v);
       cp16(smem_u32(sV + r * P + c * 8), vg + off, v);
@@ -117,8 +118,8 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         const int key = kt * kKT + i * 8 + tig * 2 + (c & 1);
-        const int qi = qa + (c >> 1) * 8;
-        const float v = (key <= qi && key < seq_len) ? s[i][c] * scale : -INFINITY;
+        const int qi = pos0 + qa + (c >> 1) * 8;  // the query's position
+        const float v = (key <= qi && key < n_keys) ? s[i][c] * scale : -INFINITY;
         s[i][c] = v;
         mx[c >> 1] = fmaxf(mx[c >> 1], v);
       }
@@ -194,11 +195,11 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
 template <int DH, bool SPLIT>
 cudaError_t launch_dh(const __nv_bfloat16* q, const __nv_bfloat16* q_lo, const __nv_bfloat16* k, const __nv_bfloat16* v,
                       int batch, int seq_len, int n_q_heads, int n_kv_heads, int max_seq_len, __nv_bfloat16* o,
-                      __nv_bfloat16* o_lo, cudaStream_t stream) {
+                      __nv_bfloat16* o_lo, cudaStream_t stream, int pos0) {
   constexpr int smem = 4 * 64 * (DH + 8) * 2;
   dim3 grid((seq_len + kQT - 1) / kQT, n_q_heads, batch);
   prefill_attention_kernel<DH, SPLIT><<<grid, kPfThreads, smem, stream>>>(q, q_lo, k, v, seq_len, n_q_heads, n_kv_heads,
-                                                                          max_seq_len, o, o_lo);
+                                                                          max_seq_len, o, o_lo, pos0);
   return cudaGetLastError();
 }
 
@@ -221,14 +222,15 @@ cudaError_t prefill_attention_init() {
 cudaError_t launch_prefill_attention(const __nv_bfloat16* q, const __nv_bfloat16* q_lo, const __nv_bfloat16* k,
                                      const __nv_bfloat16* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
                                      int head_dim, int max_seq_len, __nv_bfloat16* o, __nv_bfloat16* o_lo,
-                                     cudaStream_t stream) {
+                                     cudaStream_t stream, int pos0) {
   const bool split = q_lo != nullptr && o_lo != nullptr;
+  if (pos0 < 0 || pos0 + seq_len > max_seq_len) return cudaErrorInvalidValue;
   if (head_dim == 128)
-    return split ? launch_dh<128, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream)
-                 : launch_dh<128, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream);
+    return split ? launch_dh<128, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0)
+                 : launch_dh<128, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0);
   if (head_dim == 64)
-    return split ? launch_dh<64, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream)
-                 : launch_dh<64, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream);
+    return split ? launch_dh<64, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0)
+                 : launch_dh<64, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0);
   return cudaErrorInvalidValue;
 }
 

@@ -36,7 +36,7 @@ __device__ __forceinline__ void epilogue_pair(const LargeMParams& p, int m, int 
     case EPI_QKV_ROPE: {
       const QkvEpilogue& e = p.qkv;
       const int Dh = e.head_dim, nq = e.n_q_heads * Dh, nk = e.n_kv_heads * Dh;
-      const int b = m / e.prefill_seq_len, pos = m % e.prefill_seq_len;
+      const int b = m / e.prefill_seq_len, pos = e.prefill_pos0 + m % e.prefill_seq_len;
       if (n < nq + nk) {
         const float2 cs = e.rope[static_cast<size_t>(pos) * (Dh >> 1) + ((n % Dh) >> 1)];
         const float a0 = v0 * cs.x - v1 * cs.y, a1 = v0 * cs.y + v1 * cs.x;

@@ -263,6 +263,75 @@ def test_prompt_pass_every_position(B, case, impl):
     model.close()
 
 
+@pytest.mark.parametrize("case,impl", [("tiny_ladder", 0), ("tiny_hybrid", 0), ("tiny_ladder", 1), ("8b_shape", 0)])
+def test_prompt_fed_in_chunks(B, case, impl):
+    """A prompt fed as ladder_prefill of its first chunk plus ladder_prefill_append calls (chunk lengths that are
+    not multiples of any tile, a one-token chunk, a chunk that starts inside a 64-key tile): every position's hidden
+    state against the oracle's pass over the whole prompt, the cache rows and lengths, and the decode steps that
+    follow against a one-call prompt pass of the same model."""
+    if case == "8b_shape":
+        s = synth.replace(synth.SHAPES["8b_hybrid"].with_layers(4), layer_is_ladder=(0, 0, 1, 1))
+        bsz, chunks, dtype = 2, [100, 60, 41], np.float32
+    else:
+        mask = (1, 1, 1, 1) if case == "tiny_ladder" else (0, 1, 1, 0)
+        s = synth.replace(synth.SHAPES["tiny"], layer_is_ladder=mask)
+        bsz, chunks, dtype = 3, [70, 1, 57, 64, 9], np.float64
+    S, steps = sum(chunks), 5
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    prompt = synth.make_tokens(s, bsz, S)
+    tok = torch.from_numpy(prompt).cuda()
+    max_seq = S + steps + 2
+    model = B.Model(w, bsz, max_seq, bsz * max(chunks))          # workspace for one chunk only
+    cache = B.KVCache(s, bsz, max_seq, fill=CANARY)
+    nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+    hs, p0 = [], 0
+    B.set_prefill_gemm_impl(impl)
+    try:
+        for i, c in enumerate(chunks):
+            h = torch.zeros(bsz, c, s.d_model, device="cuda")
+            call = model.prefill if i == 0 else model.prefill_append
+            call(cache, tok[:, p0:p0 + c].contiguous(), next_tokens=nxt, all_hidden=h)
+            hs.append(h)
+            p0 += c
+            assert cache.seq_lens.cpu().tolist() == [p0] * bsz
+        with pytest.raises(B.LadderError):                        # would run past max_seq_len
+            model.prefill_append(cache, tok[:, :steps + 3].contiguous())
+        torch.cuda.synchronize()
+    finally:
+        B.set_prefill_gemm_impl(0)
+    assert model.device_status() == 0
+    got = torch.cat(hs, 1).cpu().numpy()
+    cfg = oracle_cfg(s)
+    OW = O.OracleWeights(provider=synth.logical_provider(w, dtype))
+    ref = O.forward(cfg, OW, prompt, dtype=dtype, last_only=False, with_logits=False)
+    err = rel_err(got, ref.hidden)
+    print(f"[{case} impl {impl}] chunked prompt pass: hidden max-rel-err {err:.3e} over {bsz * S} positions")
+    assert err < HIDDEN_TOL, err
+    k5 = cache.k5().view(torch.int16)
+    assert bool((k5[:, :, :, S:, :] == CANARY).all()) and not bool((k5[:, :, :, :S, :] == CANARY).any())
+    # ---- the same prompt in one call (needs its own, larger workspace), then both decode on
+    model1 = B.Model(w, bsz, max_seq, bsz * S)
+    cache1 = B.KVCache(s, bsz, max_seq, fill=CANARY)
+    nxt1 = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+    model1.prefill(cache1, tok, next_tokens=nxt1)
+    torch.cuda.synchronize()
+    assert rel_err(cache.k5()[:, :, :, :S].float().cpu().numpy(), cache1.k5()[:, :, :, :S].float().cpu().numpy()) < 2e-2
+    assert rel_err(cache.v5()[:, :, :, :S].float().cpu().numpy(), cache1.v5()[:, :, :, :S].float().cpu().numpy()) < 2e-2
+    same = nxt.cpu().numpy() == nxt1.cpu().numpy()
+    hid, hid1 = torch.zeros(bsz, s.d_model, device="cuda"), torch.zeros(bsz, s.d_model, device="cuda")
+    feed = nxt1.clone()                                           # both continue from the same tokens
+    for _ in range(steps):
+        model.decode_step(cache, feed, next_tokens=nxt, final_hidden=hid)
+        model1.decode_step(cache1, feed, next_tokens=nxt1, final_hidden=hid1)
+        torch.cuda.synchronize()
+        assert rel_err(hid.cpu().numpy(), hid1.cpu().numpy()) < HIDDEN_TOL
+        feed = nxt1.clone()
+    assert cache.seq_lens.cpu().tolist() == [S + steps] * bsz
+    assert same.mean() >= 0.5                                     # first generated token: near-ties may flip one
+    model.close()
+    model1.close()
+
+
 def test_70b_full_size_single_live_module(B):
     """The benchmark's own launch configuration -- all 80 layers of the 70B shape resident (141 GB),
     batch 4, 1024-token prompts, CUDA-graph decode -- checked with a property that holds at any size:

@@ -119,9 +119,11 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
 ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, int32_t use_graph, int32_t use_pdl);
 
 /* Persistent decode step (default on; batch <= 8).  The ladder layers at the top of the model (all layers of
- * an all-ladder model) and the LM head of a decode step run as ONE cooperative kernel launch; standard-residual
- * layers below them run one kernel per GEMM, and a model whose top layer is standard does not use the launch
- * at all.  Every weight-streaming GEMM is a phase of that kernel,
+ * an all-ladder model) and the LM head of a decode step run as ONE cooperative kernel launch.  Standard-residual
+ * layers below them run one kernel per GEMM when a layer's weights exceed 300 MB (measured faster there) and go
+ * into the same launch otherwise; on = 2 puts every layer into the launch whatever its size.  A large-layer
+ * model whose top layer is standard does not use the launch at all.  Every weight-streaming GEMM is a phase of
+ * that kernel,
  * attention runs on dedicated warps of the same CTAs, and a grid-wide hand-over is a counter in global
  * memory that is polled only where data crosses SMs.  With the ladder rule (Eq. 2: module m reads
  * x_{m-2}) every such dependency points two phases back, so the weight stream never stops between

@@ -246,7 +246,8 @@ class Model:
     def set_schedule(self, n_streams: int = 2, use_graph: bool = True, use_pdl: bool = True):
         _check(lib().ladder_model_set_schedule(self.h, n_streams, int(use_graph), int(use_pdl)), self.h)
 
-    def set_persistent(self, on: bool = True):
+    def set_persistent(self, on=True):
+        """False / 0: one kernel per GEMM; True / 1: the default split; 2: every layer in the persistent kernel."""
         _check(lib().ladder_model_set_persistent(self.h, int(on)), self.h)
 
     def debug_stall_last_phase(self, on: bool):

@@ -81,6 +81,7 @@ struct ladder_model {
   // persistent layer-stack kernel (one cooperative launch per decode step, batch <= 8)
   bool stack_ok = false;   // usable on this device and worthwhile for this model
   int stack_begin = 0;     // first layer run by the persistent kernel (layers below: one kernel per GEMM)
+  bool stack_usable = false;  // the kernel fits this device and this depth
   int stack_stall_test = 0;  // test hook: the last phase waits for a count its producer never reaches
   int use_stack = 1;
   GraphKey stack_key;      // what the uploaded phase list was built for
@@ -550,6 +551,17 @@ int stack_first_layer(const std::vector<uint8_t>& is_ladder) {
   return b;
 }
 
+// First layer the persistent kernel runs by default.  A standard-residual layer makes every phase wait for the
+// one before; for layers that stream a lot (measured: 436 MB per layer at the 8B shape, 1.7 GB at the 70B shape)
+// separate kernels with their dynamically balanced GEMMs are then 2.5-3 % faster, so only the ladder stretch at
+// the top goes into the kernel.  For small layers (214 MB per layer at the tensor-parallel slice: 6 % the other
+// way) the launch gaps weigh more than the balance and every layer goes in.
+int stack_default_begin(const ladder_config_t& c, const std::vector<uint8_t>& is_ladder) {
+  const double layer_bytes = 2.0 * (static_cast<double>((c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim) * c.d_model +
+                                    static_cast<double>(c.d_model) * c.n_q_heads * c.head_dim + 3.0 * c.d_ff * c.d_model);
+  return layer_bytes < 300e6 ? 0 : stack_first_layer(is_ladder);
+}
+
 // Returns false (with a reason) when this step cannot be expressed; the caller then uses the
 // multi-kernel schedule.
 bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, float* logits, std::vector<StackPhase>& phases,
@@ -900,11 +912,10 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
     return fail(nullptr, LADDER_ERR_CUDA, std::string("device query: ") + cudaGetErrorString(e));
   }
   if (4 * L + 1 > kStackMaxPhases) m->stack_ok = false;
-  // The persistent kernel pays off where the ladder rule decouples consecutive modules; a standard-
-  // residual layer makes every phase wait for the one before, and there separate kernels with their
-  // dynamically balanced GEMMs are faster.  It therefore runs the ladder layers at the top of the model
-  // (and the LM head); standard layers below them run kernel by kernel.
-  m->stack_begin = stack_first_layer(m->is_ladder);
+  // The persistent kernel pays off most where the ladder rule decouples consecutive modules: by default it runs
+  // the ladder layers at the top of the model (and the LM head) and, for small layers, the standard ones too.
+  m->stack_usable = m->stack_ok;
+  m->stack_begin = stack_default_begin(c, m->is_ladder);
   if (m->stack_begin == L) m->stack_ok = false;
   if (static_cast<size_t>(smem_optin) < smallm_gemm_smem_bytes(c.max_batch)) {
     delete m;
@@ -1035,6 +1046,11 @@ ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, 
 ladder_status_t ladder_model_set_persistent(ladder_model_t* m, int32_t on) {
   if (!m) return LADDER_ERR_INVALID_ARG;
   m->use_stack = on ? 1 : 0;
+  // 2: every layer in the persistent kernel, standard-residual ones included; 1: the default choice
+  const int L = m->cfg.n_layers;
+  m->stack_begin = on == 2 ? 0 : stack_default_begin(m->cfg, m->is_ladder);
+  m->stack_ok = m->stack_usable && m->stack_begin < L;
+  m->stack_built = false;
   return LADDER_OK;
 }
 
@@ -1107,7 +1123,7 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
   std::vector<StackPhase> ph;
   std::vector<StackAttn> at;
   int nc = 0;
-  const int begin = stack_first_layer(m.is_ladder);
+  const int begin = stack_default_begin(m.cfg, m.is_ladder);
   const bool ok = build_stack(&m, &cache, batch, reinterpret_cast<float*>(fake()), ph, at, &nc, begin);
   m.ev.clear();
   std::vector<int32_t> o = {static_cast<int32_t>(ph.size()), static_cast<int32_t>(at.size()), nc, begin, ok ? 1 : 0};

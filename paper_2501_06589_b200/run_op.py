@@ -30,6 +30,8 @@ def main():
     ap.add_argument("--multi-kernel", action="store_true", help="stack: use the per-GEMM schedule")
     ap.add_argument("--wide-impl", type=int, default=0,
                     help="decode GEMM: 0 = default, 1 = mma.sync kernel for batch 9..64, 2 = tcgen05 kernel for every batch")
+    ap.add_argument("--persistent-all", action="store_true", help="stack: standard layers in the persistent kernel too")
+    ap.add_argument("--standard", action="store_true", help="stack: standard residuals in every layer")
     ap.add_argument("--which", default="gate_up", choices=["qkv", "wo", "gate_up", "down"],
                     help="prefill_gemm: which projection's shape and epilogue")
     a = ap.parse_args()
@@ -127,12 +129,16 @@ def run_stack(a, s, bsz):
     """Decode steps of the model cut to a.layers layers, KV length from the configuration."""
     s = synth.replace(s, n_layers=a.layers, layer_is_ladder=None if s.layer_is_ladder is None
                       else tuple(s.layer_is_ladder[:a.layers]))
+    if a.standard:
+        s = s.as_standard()
     w = synth.make_weights(s, device="cuda")
     S = a.kv_len or s.prompt_len
     steps = a.iters + 3
     model = B.Model(w, bsz, S + steps + 1, bsz * min(S, 256))
     if a.multi_kernel:
         model.set_persistent(False)
+    if a.persistent_all:
+        model.set_persistent(2)
     persistent = model.persistent_active() and bsz <= 8
     cache = B.KVCache(s, bsz, S + steps + 1)
     cache.k.normal_()                                 # a synthetic prefix instead of a prompt pass

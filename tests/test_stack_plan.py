@@ -77,6 +77,8 @@ def test_plan_orders_every_hazard(B, case):
     first = shape.n_layers
     while first > 0 and mask[first - 1]:
         first -= 1
+    if shape.layer_weight_bytes() < 300e6:       # small layers: standard ones run inside the launch too
+        first = 0
     assert plan["first_layer"] == first
     if first == shape.n_layers:
         return                                   # top layer is standard: the launch is not used

@@ -214,6 +214,9 @@ def main():
                     help="one kernel per GEMM (two streams, CUDA graph, PDL) instead of the persistent decode kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill-timing", action="store_true")
+    ap.add_argument("--prefill-impl", type=int, default=0,
+                    help="prompt-pass GEMMs: 0 = tcgen05, bf16 hi + lo activations (default); 1 = mma.sync; "
+                         "2 = tcgen05, one bf16 per activation (not the precision the parity bound is stated for)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -254,6 +257,7 @@ def main():
     t_gen = time.time() - t0
     model = B.Model(w, bsz, max_seq, bsz * S)
     B.set_decode_wide_impl(args.wide_impl)
+    B.set_prefill_gemm_impl(args.prefill_impl)
     if args.multi_kernel:
         model.set_persistent(False)
     persistent = model.persistent_active() and bsz <= 8
@@ -367,6 +371,8 @@ def main():
         line["prefill"] = {"tokens_per_s": world * bsz * S / (prefill_ms_max * 1e-3), "ms": prefill_ms_max,
                            "tflops": flops / (prefill_ms_max * 1e-3) / 1e12,
                            "frac_of_bf16_peak": flops / (prefill_ms_max * 1e-3) / 1e12 / bf16_peak,
+                           "activations": {0: "bf16 hi+lo pair (2 MMAs per product)", 1: "bf16 hi+lo pair, mma.sync kernel",
+                                           2: "single bf16"}[args.prefill_impl],
                            "peak_tflops": bf16_peak, "peak_source": peak_src}
     if (shape.name, bsz) in NCU_TRAFFIC_BYTES:
         line["roofline"]["traffic"] = NCU_TRAFFIC_BYTES[(shape.name, bsz)]

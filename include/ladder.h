@@ -272,7 +272,11 @@ ladder_status_t ladder_op_prefill_gemm(const void* A, const void* A_lo, const vo
                                        void* cuda_stream);
 
 /* Which implementation the prefill GEMMs use (process-wide): 0 = tcgen05 tensor-core kernel with TMA
- * and TMEM accumulators (default), 1 = warp-level mma.sync kernel (kept as a cross-check). */
+ * and TMEM accumulators, activations as a bf16 hi + lo pair (default), 1 = warp-level mma.sync kernel (kept as a
+ * cross-check), 2 = the tcgen05 kernel with ONE bf16 value per activation (normalised input, query, attention
+ * output, SwiGLU output): half the tensor-core work and the usual bf16 inference precision, but every stored
+ * activation is rounded at 2^-9, which by itself reaches 1.6e-2 of hidden-state error after 8 layers of the 8B
+ * shape - outside the 2e-2 bound of the default mode for deeper models. */
 void ladder_set_prefill_gemm_impl(int32_t impl);
 
 /* Decode GEMM for batch 9..64: 0 = tcgen05 kernel (weights as the M side of the MMA, TMA tiles, TMEM accumulators,

@@ -331,7 +331,8 @@ def op_decode_attention_noalloc(q, k, v, kv_len, n_q_heads, n_kv_heads, head_dim
 
 
 def set_prefill_gemm_impl(impl: int):
-    """0 = tcgen05 kernel (default), 1 = warp-level mma.sync kernel."""
+    """0 = tcgen05 kernel, bf16 hi + lo activations (default); 1 = warp-level mma.sync kernel; 2 = tcgen05 kernel
+    with one bf16 value per activation (half the tensor-core work, plain bf16 precision)."""
     lib().ladder_set_prefill_gemm_impl(impl)
 
 

@@ -389,22 +389,28 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
     ++k;
   };
   did(launch_embed(d_tokens, m->tok_embedding, M, d, c.vocab_size, m->R[0], m->status, st, false));
+  // lo parts of the GEMM inputs (activation ~ hi + lo); none when the single-bf16 mode is selected
+  const bool split = !prefill_single_bf16();
+  __nv_bfloat16* const n_lo = split ? m->n_pf + m->n_lo : nullptr;
+  __nv_bfloat16* const q_lo = split ? m->q_pf + m->q_lo : nullptr;
+  __nv_bfloat16* const o_lo = split ? m->o_pf + m->q_lo : nullptr;
+  __nv_bfloat16* const h_lo = split ? m->h_pf + m->h_lo : nullptr;
   Router rt;
   for (int l = 0; l < c.n_layers; ++l) {
     const bool lad = m->is_ladder[l] != 0;
     {
       const Router::Route r = rt.next(lad, 2 * l + 1);
-      did(launch_rmsnorm_bf16(m->R[r.in], m->attn_norm[l], c.rms_eps, M, d, m->n_pf, m->n_pf + m->n_lo, st));
+      did(launch_rmsnorm_bf16(m->R[r.in], m->attn_norm[l], c.rms_eps, M, d, m->n_pf, n_lo, st));
       LargeMParams p = {};
       p.A = m->n_pf;
-      p.A_lo = m->n_pf + m->n_lo;
+      p.A_lo = n_lo;
       p.W = m->w_qkv[l];
       p.M = M;
       p.N = (Hq + 2 * Hkv) * Dh;
       p.K = d;
       p.epi_mode = EPI_QKV_ROPE;
       p.qkv.q_out_bf16 = m->q_pf;
-      p.qkv.q_out_lo = m->q_pf + m->q_lo;
+      p.qkv.q_out_lo = q_lo;
       p.qkv.k_cache = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
       p.qkv.v_cache = static_cast<__nv_bfloat16*>(cache->v) + l * layer_elems;
       p.qkv.rope = m->rope;
@@ -416,11 +422,11 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       p.qkv.prefill_pos0 = pos0;
       p.status = m->status;
       did(launch_largem_gemm(p, st));
-      did(launch_prefill_attention(m->q_pf, m->q_pf + m->q_lo, p.qkv.k_cache, p.qkv.v_cache, batch, S, Hq, Hkv, Dh,
-                                   c.max_seq_len, m->o_pf, m->o_pf + m->q_lo, st, pos0));
+      did(launch_prefill_attention(m->q_pf, q_lo, p.qkv.k_cache, p.qkv.v_cache, batch, S, Hq, Hkv, Dh, c.max_seq_len,
+                                   m->o_pf, o_lo, st, pos0));
       LargeMParams o = {};
       o.A = m->o_pf;
-      o.A_lo = m->o_pf + m->q_lo;
+      o.A_lo = o_lo;
       o.W = m->w_o[l];
       o.M = M;
       o.N = d;
@@ -433,22 +439,22 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
     }
     {
       const Router::Route r = rt.next(lad, 2 * l + 2);
-      did(launch_rmsnorm_bf16(m->R[r.in], m->mlp_norm[l], c.rms_eps, M, d, m->n_pf, m->n_pf + m->n_lo, st));
+      did(launch_rmsnorm_bf16(m->R[r.in], m->mlp_norm[l], c.rms_eps, M, d, m->n_pf, n_lo, st));
       LargeMParams p = {};
       p.A = m->n_pf;
-      p.A_lo = m->n_pf + m->n_lo;
+      p.A_lo = n_lo;
       p.W = m->w_gate_up[l];
       p.M = M;
       p.N = 2 * F;
       p.K = d;
       p.epi_mode = EPI_SWIGLU;
       p.out = m->h_pf;
-      p.out_lo = m->h_pf + m->h_lo;
+      p.out_lo = h_lo;
       p.status = m->status;
       did(launch_largem_gemm(p, st));
       LargeMParams o = {};
       o.A = m->h_pf;
-      o.A_lo = m->h_pf + m->h_lo;
+      o.A_lo = h_lo;
       o.W = m->w_down[l];
       o.M = M;
       o.N = d;

@@ -148,7 +148,8 @@ struct LargeMParams {
 cudaError_t launch_largem_gemm(const LargeMParams& p, cudaStream_t stream);
 cudaError_t launch_largem_gemm_tc(const LargeMParams& p, cudaStream_t stream, int sm_count);
 cudaError_t largem_gemm_tc_init();
-void set_prefill_gemm_impl(int impl);  // 0 = tcgen05 (default), 1 = mma.sync
+void set_prefill_gemm_impl(int impl);  // 0 = tcgen05 (default), 1 = mma.sync, 2 = tcgen05 with single-bf16 activations
+bool prefill_single_bf16();            // the prompt pass feeds its GEMMs one bf16 value per activation (no lo part)
 
 // q_lo / o_lo: optional lo parts (value ~ hi + lo) of the query input and the attention output.
 // pos0: the seq_len queries sit at positions pos0 .. pos0 + seq_len - 1 and attend to cache rows 0 .. their own.

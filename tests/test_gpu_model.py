@@ -229,11 +229,14 @@ def test_8b_hybrid_shape_short_context(B):
     assert agree >= 0.99, agree
 
 
-@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("impl", [0, 1, 2])
 @pytest.mark.parametrize("case", ["tiny", "8b_shape"])
 def test_prompt_pass_every_position(B, case, impl):
     """Hidden state of EVERY prompt position against the oracle, with the prompt-pass GEMMs on the tcgen05
-    kernel (0) and on the warp-level mma.sync kernel (1); ragged M (not a multiple of the 128-row tile)."""
+    kernel (0), on the warp-level mma.sync kernel (1) and on the tcgen05 kernel with one bf16 value per activation
+    (2: not the default: at 8 layers of the 8B shape it already measures 3.5e-2, outside the 2e-2 bound, which is
+    why the default keeps a hi + lo pair; checked against 6e-2 so that a real defect would still show);
+    ragged M (not a multiple of the 128-row tile)."""
     if case == "tiny":
         s, bsz, S, dtype = synth.replace(synth.SHAPES["tiny"], layer_is_ladder=(1, 0, 1, 1)), 3, 150, np.float64
     else:
@@ -257,7 +260,7 @@ def test_prompt_pass_every_position(B, case, impl):
     ref = O.forward(cfg, OW, prompt, dtype=dtype, last_only=False, with_logits=False)
     err = rel_err(allh.cpu().numpy(), ref.hidden)
     print(f"[{case} impl {impl}] prompt-pass hidden max-rel-err {err:.3e} over {bsz * S} positions")
-    assert err < HIDDEN_TOL, err
+    assert err < (HIDDEN_TOL if impl != 2 else 6e-2), err
     k5 = cache.k5().view(torch.int16)
     assert bool((k5[:, :, :, S:, :] == CANARY).all()) and not bool((k5[:, :, :, :S, :] == CANARY).any())
     model.close()

@@ -53,6 +53,9 @@ struct ladder_model {
   float* q_f32 = nullptr;           // decode [max_batch, Hq*Dh]
   float* o_dec = nullptr;           // decode [max_batch, Hq*Dh]
   float* h_dec = nullptr;           // decode [max_batch, F]
+  // batch 9..64: the SwiGLU output / the attention output as the next GEMM's staged operand (bf16 [2 x 64, F] / [2 x 64, Hq*Dh])
+  __nv_bfloat16* wide_hpack = nullptr;
+  __nv_bfloat16* wide_opack = nullptr;
   // the same activations as bf16 hi/lo MMA operands ([chunk][8][2048]), written by the persistent kernel's
   // epilogues for the phase that reads them next (batch <= 4): twins of R[0], R[1], h_dec, o_dec
   __nv_bfloat16 *xpack[2] = {nullptr, nullptr}, *hpack = nullptr, *opack = nullptr;
@@ -287,6 +290,11 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       a.max_len = c.max_seq_len;
       a.scratch = m->attn_scratch;
       a.o = m->o_dec;
+      const bool handover = batch > 8 && m->wide_opack && wide_handover();  // operands pass from kernel to kernel
+      if (handover) {
+        a.o_pack = m->wide_opack;
+        a.o_pack_bp = wide_padded_batch(batch);
+      }
       q.launched(0, launch_decode_attention(a, sA, q.pdl(0)));
       ++q.kernels;  // the split kernel and its merge kernel
 
@@ -302,6 +310,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       o.addend = m->R[r.add];
       o.out = m->R[r.dst];
       o.status = m->status;
+      if (handover) o.act_staged = m->wide_opack;
       q.gemm(0, o, lad);
       q.record(0, m->ev[mod]);
     }
@@ -326,6 +335,8 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       p.epi_mode = EPI_SWIGLU;
       p.out = m->h_dec;
       p.status = m->status;
+      const bool handover = batch > 8 && m->wide_hpack && wide_handover();
+      if (handover) p.wide_pack_out = m->wide_hpack;
       q.gemm(1, p, lad);
 
       need(1, mod - 1);
@@ -340,6 +351,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       o.addend = m->R[r.add];
       o.out = m->R[r.dst];
       o.status = m->status;
+      if (handover) o.act_staged = m->wide_hpack;
       q.gemm(1, o, lad);
       q.record(1, m->ev[mod]);
     }
@@ -941,6 +953,10 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   A(dev_alloc(&m->q_f32, MB * qd));
   A(dev_alloc(&m->o_dec, MB * qd));
   A(dev_alloc(&m->h_dec, MB * F));
+  if (c.max_batch > 8) {
+    A(dev_alloc(&m->wide_hpack, 2 * 64 * F));
+    A(dev_alloc(&m->wide_opack, 2 * 64 * qd));
+  }
   const auto pack_elems = [](size_t K) { return ((K + 2047) / 2048) * 8 * 2048; };
   A(dev_alloc(&m->xpack[0], pack_elems(d)));
   A(dev_alloc(&m->xpack[1], pack_elems(d)));
@@ -1031,7 +1047,7 @@ ladder_status_t ladder_destroy(ladder_model_t* m) {
   if (m->ev_join) cudaEventDestroy(m->ev_join);
   if (m->side) cudaStreamDestroy(m->side);
   if (m->cap) cudaStreamDestroy(m->cap);
-  void* bufs[] = {m->xpack[0], m->xpack[1], m->hpack, m->opack, m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
+  void* bufs[] = {m->wide_hpack, m->wide_opack, m->xpack[0], m->xpack[1], m->hpack, m->opack, m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
                   m->n_pf, m->q_pf,  m->o_pf,  m->h_pf,  m->rope,  m->status,       m->tok_tmp,   m->next_tmp};
   for (void* b : bufs)
     if (b) cudaFree(b);

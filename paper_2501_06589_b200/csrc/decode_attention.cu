@@ -241,7 +241,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
 constexpr int kMaxSplits = 1024;
 template <int DH>
 __global__ void __launch_bounds__(DH) decode_attention_merge_kernel(const float* scratch, int n_q_heads, int n_splits,
-                                                                    float* o) {
+                                                                    float* o, __nv_bfloat16* o_pack, int bp) {
   __shared__ float wgt[kMaxSplits];
   __shared__ float red_m[DH / 32], red_l[DH / 32];
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -275,7 +275,16 @@ __global__ void __launch_bounds__(DH) decode_attention_merge_kernel(const float*
   float acc = 0.f;
 #pragma unroll 8
   for (int s = 0; s < n_splits; ++s) acc += wgt[s] * __ldcg(base + s * stride + tid);
-  o[(static_cast<size_t>(b) * n_q_heads + h) * DH + tid] = lsum > 0.f ? acc / lsum : 0.f;
+  const float val = lsum > 0.f ? acc / lsum : 0.f;
+  o[(static_cast<size_t>(b) * n_q_heads + h) * DH + tid] = val;
+  if (o_pack) {  // the output projection's staged operand: hi part in row b, lo part in row bp + b
+    const size_t K = static_cast<size_t>(n_q_heads) * DH, col = static_cast<size_t>(h) * DH + tid;
+    const __nv_bfloat16 hi = __float2bfloat16_rn(val);
+    o_pack[b * K + col] = hi;
+    o_pack[(bp + b) * K + col] = __float2bfloat16_rn(val - __bfloat162float(hi));
+    if (b == static_cast<int>(gridDim.y) - 1)  // the last sequence's CTAs also clear the padding rows
+      for (int r = b + 1; r < bp; ++r) o_pack[r * K + col] = o_pack[(bp + r) * K + col] = __float2bfloat16_rn(0.f);
+  }
 }
 
 cudaLaunchConfig_t make_cfg(dim3 grid, dim3 block, cudaStream_t stream, bool pdl, cudaLaunchAttribute* at) {
@@ -335,9 +344,12 @@ cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stre
   cudaLaunchAttribute at[1];
   cudaLaunchConfig_t cfg = make_cfg(dim3(p.n_q_heads, p.batch), dim3(p.head_dim), stream, pdl, at);
   const float* scratch = p.scratch;
+  __nv_bfloat16* o_pack = p.o_pack;
+  const int bp = p.o_pack_bp;
+  if (o_pack && bp < p.batch) return cudaErrorInvalidValue;
   if (p.head_dim == 128)
-    return cudaLaunchKernelEx(&cfg, decode_attention_merge_kernel<128>, scratch, p.n_q_heads, p.n_splits, p.o);
-  return cudaLaunchKernelEx(&cfg, decode_attention_merge_kernel<64>, scratch, p.n_q_heads, p.n_splits, p.o);
+    return cudaLaunchKernelEx(&cfg, decode_attention_merge_kernel<128>, scratch, p.n_q_heads, p.n_splits, p.o, o_pack, bp);
+  return cudaLaunchKernelEx(&cfg, decode_attention_merge_kernel<64>, scratch, p.n_q_heads, p.n_splits, p.o, o_pack, bp);
 }
 
 }  // namespace ladder

@@ -49,6 +49,7 @@ size_t smallm_gemm_wide_tc_smem_bytes(int batch);
 size_t smallm_gemm_wide_tc_scratch_floats(int N, int K, int batch);
 static int g_wide_impl = 0;  // 0 = tcgen05, 1 = mma.sync, 2 = tcgen05 for every batch (also <= 8)
 void set_decode_wide_impl(int impl) { g_wide_impl = (impl == 1 || impl == 2) ? impl : 0; }
+bool wide_handover() { return g_wide_impl != 1; }
 
 namespace {
 

@@ -205,7 +205,7 @@ __device__ __forceinline__ void epi_prefetch(const SmallMParams& p, int n, int b
 // v[j] = finished accumulator of row n and batch row b0 + j.
 template <int CB>
 __device__ __forceinline__ void epi_apply(const SmallMParams& p, int n, int b0, float (&v)[CB], int lane,
-                                          const int* pos_s, const float (&pa)[CB], const float (&pb)[CB]) {
+                                          const int* pos_s, const float (&pa)[CB], const float (&pb)[CB], int bp) {
   const bool row_ok = n < p.N;
   if (p.epi_mode == EPI_RESID || p.epi_mode == EPI_PLAIN) {
     float* out = static_cast<float*>(p.out);
@@ -220,9 +220,16 @@ __device__ __forceinline__ void epi_apply(const SmallMParams& p, int n, int b0, 
     for (int j = 0; j < CB; ++j) {
       const int b = b0 + j;
       const float up = __shfl_down_sync(0xffffffffu, v[j], 1);
-      if (!(lane & 1) && b < p.batch && row_ok) {
+      if (!(lane & 1) && row_ok) {
         const float gt = v[j];
-        out[static_cast<size_t>(b) * (p.N >> 1) + (n >> 1)] = gt / (1.f + __expf(-gt)) * up;
+        const float hv = b < p.batch ? gt / (1.f + __expf(-gt)) * up : 0.f;
+        if (b < p.batch) out[static_cast<size_t>(b) * (p.N >> 1) + (n >> 1)] = hv;
+        if (p.wide_pack_out) {  // the down projection's staged operand (padding rows written as zero)
+          const size_t kc = static_cast<size_t>(p.N >> 1), col = static_cast<size_t>(n >> 1);
+          const __nv_bfloat16 hi = __float2bfloat16_rn(hv);
+          p.wide_pack_out[b * kc + col] = hi;
+          p.wide_pack_out[(bp + b) * kc + col] = __float2bfloat16_rn(hv - __bfloat162float(hi));
+        }
       }
     }
   } else if (p.epi_mode == EPI_QKV_ROPE) {
@@ -480,7 +487,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
 #pragma unroll
             for (int j = 0; j < CB; ++j) v[j] *= rstd_s[b0 + j];
           }
-          epi_apply<CB>(p, n, b0, v, lane, pos_s, pa, pb);
+          epi_apply<CB>(p, n, b0, v, lane, pos_s, pa, pb, BP);
         } else {
 #pragma unroll
           for (int j = 0; j < CB; j += 4) piece[((b0 + j) >> 2) * 32] = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -543,7 +550,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
 #pragma unroll
           for (int j = 0; j < FB; ++j) v[j] *= rstd_s[b0 + j];
         }
-        epi_apply<FB>(p, n, b0, v, lane, pos_s, pa, pb);
+        epi_apply<FB>(p, n, b0, v, lane, pos_s, pa, pb, BP);
       }
     }
     if (et == 0) WIDE_STAMP(7);
@@ -586,17 +593,18 @@ size_t stage_offset() { return 64 * kWideMaxSlices + kWideMaxTiles; }
 size_t piece_offset(int bp, int K) { return stage_offset() + ((static_cast<size_t>(bp) * K + 3) & ~size_t(3)); }
 
 template <int NP>
-cudaError_t launch_np(const WideArgs& a, const CUtensorMap& mw, const CUtensorMap& ma, int grid, cudaStream_t stream) {
+cudaError_t launch_np(const WideArgs& a, const CUtensorMap& mw, const CUtensorMap& ma, int grid, cudaStream_t stream,
+                      bool pdl_attr) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kWideThreads);
   cfg.dynamicSmemBytes = WCfg<NP>::SMEM;
   cfg.stream = stream;
   cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the staging kernel is always right before it
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the staging kernel, or the producer of a staged operand
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pdl_attr ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, decode_gemm_wide_tc_kernel<NP>, a, mw, ma);
 }
 
@@ -607,6 +615,8 @@ extern "C" int ladder_debug_read_wide_trace(unsigned long long* host_out) {
   return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_wide_trace, sizeof(g_wide_trace)));
 }
 #endif
+
+int wide_padded_batch(int batch) { return padded_batch(batch); }
 
 cudaError_t smallm_gemm_wide_tc_init() {
   if (!g_encode_wide) {
@@ -654,7 +664,10 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
   __nv_bfloat16* stage = reinterpret_cast<__nv_bfloat16*>(p.scratch + stage_offset());
   float* pieces = p.scratch + piece_offset(bp, p.K);
 
-  {  // 1. activations -> bf16 hi + lo, 1/rms
+  if (p.act_staged) {  // the producing kernel has written the operand already
+    if (p.act_mode != ACT_F32 || (reinterpret_cast<uintptr_t>(p.act_staged) & 15)) return cudaErrorInvalidValue;
+    stage = const_cast<__nv_bfloat16*>(p.act_staged);
+  } else {  // 1. activations -> bf16 hi + lo, 1/rms
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(bp, n_slices);
     cfg.blockDim = dim3(256);
@@ -683,10 +696,11 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
   a.tickets = tickets;
   const int total = tiles * nkb;
   const int grid = total < sm_count ? total : sm_count;
-  if (bp == 8) return launch_np<16>(a, mw, ma, grid, stream);
-  if (bp == 16) return launch_np<32>(a, mw, ma, grid, stream);
-  if (bp == 32) return launch_np<64>(a, mw, ma, grid, stream);
-  return launch_np<128>(a, mw, ma, grid, stream);
+  const bool pdl_attr = p.act_staged ? pdl : true;  // after its own staging kernel always; after a producer kernel if the caller says so
+  if (bp == 8) return launch_np<16>(a, mw, ma, grid, stream, pdl_attr);
+  if (bp == 16) return launch_np<32>(a, mw, ma, grid, stream, pdl_attr);
+  if (bp == 32) return launch_np<64>(a, mw, ma, grid, stream, pdl_attr);
+  return launch_np<128>(a, mw, ma, grid, stream, pdl_attr);
 }
 
 }  // namespace ladder

@@ -39,6 +39,12 @@ struct SmallMParams {
   void* out;               // EPI_RESID / EPI_PLAIN: fp32 [batch, N]; EPI_SWIGLU: fp32 [batch, N/2]
   QkvEpilogue qkv;         // EPI_QKV_ROPE
   int32_t* status;         // device status word (may be NULL)
+  // batch 9..64 (tcgen05 kernel): operands handed from kernel to kernel without a staging launch.
+  //   wide_pack_out: EPI_SWIGLU also writes its output as the next GEMM's staged operand, bf16 [2 Bp, N / 2]
+  //                  (hi parts in rows 0..Bp-1, lo parts in rows Bp..2Bp-1, rows of sequences >= batch zero);
+  //   act_staged:    this GEMM's activations are already staged that way ([2 Bp, K]; act_mode ACT_F32 only).
+  __nv_bfloat16* wide_pack_out;
+  const __nv_bfloat16* act_staged;
   // Optional second copy of an fp32 output (EPI_RESID: out, EPI_SWIGLU: h) as the next GEMM's MMA operand:
   // y = value (* pack_gain[n]), bf16 hi at [n / 2048][b][n % 2048], lo at [n / 2048][4 + b][n % 2048]; batch <= 4.
   __nv_bfloat16* pack_out;
@@ -66,7 +72,11 @@ struct DecodeAttnParams {
   int max_len;                  // host upper bound on keys attended (sizes the split)
   float* scratch;               // [batch][Hq][n_splits][Dh + 2]
   float* o;                     // [batch, Hq*Dh]
+  __nv_bfloat16* o_pack;        // optional: o also as a staged GEMM operand, bf16 [2 o_pack_bp, Hq*Dh] (hi rows, lo rows)
+  int o_pack_bp;                // padded batch of that operand (16 / 32 / 64); rows batch..bp-1 are written as zero
 };
+int wide_padded_batch(int batch);  // Bp of the batch 9..64 GEMM kernel
+bool wide_handover();              // the tcgen05 kernel is the one in use for batch 9..64 (it alone reads staged operands)
 int decode_attention_splits(int batch, int n_kv_heads, int max_len, int sm_count);
 size_t decode_attention_scratch_floats(int batch, int n_q_heads, int head_dim, int n_splits);
 cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stream, bool pdl);

@@ -192,6 +192,7 @@ def workload_config(shape, args):
                         f"{shape.n_q_heads}q/{shape.n_kv_heads}kv heads x {shape.head_dim}, ffn {shape.d_ff}, "
                         f"vocab {shape.vocab_size}",
             "batch": shape.batch, "prompt_len": shape.prompt_len, "decode_steps": args.steps,
+            "prefill_chunk": getattr(args, "prefill_chunk", 0) or shape.prompt_len,
             "l2": "inputs larger than L2 (every step streams all weights, far above 126 MB)",
             "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU"}
 
@@ -214,6 +215,9 @@ def main():
                     help="one kernel per GEMM (two streams, CUDA graph, PDL) instead of the persistent decode kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill-timing", action="store_true")
+    ap.add_argument("--prefill-chunk", type=int, default=0,
+                    help="feed the prompt in chunks of this many tokens per sequence (ladder_prefill_append): the prompt-pass "
+                         "workspace then holds one chunk, which is what lets batch 64 of the 70B shape fit beside 141 GB of weights")
     ap.add_argument("--prefill-impl", type=int, default=0,
                     help="prompt-pass GEMMs: 0 = tcgen05, bf16 hi + lo activations (default); 1 = mma.sync; "
                          "2 = tcgen05, one bf16 per activation (not the precision the parity bound is stated for)")
@@ -255,7 +259,8 @@ def main():
     w = synth.make_weights(shape, device="cuda")
     torch.cuda.synchronize()
     t_gen = time.time() - t0
-    model = B.Model(w, bsz, max_seq, bsz * S)
+    chunk = args.prefill_chunk if 0 < args.prefill_chunk < S else S
+    model = B.Model(w, bsz, max_seq, bsz * chunk)
     B.set_decode_wide_impl(args.wide_impl)
     B.set_prefill_gemm_impl(args.prefill_impl)
     if args.multi_kernel:
@@ -277,12 +282,17 @@ def main():
 
     # ---- prefill: once untimed (warm-up), once timed
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-    model.prefill(cache, prompt, next_tokens=first)
+    def run_prefill():
+        model.prefill(cache, prompt[:, :chunk].contiguous(), next_tokens=first)
+        for p0 in range(chunk, S, chunk):
+            model.prefill_append(cache, prompt[:, p0:min(S, p0 + chunk)].contiguous(), next_tokens=first)
+
+    run_prefill()
     torch.cuda.synchronize()
     prefill_ms = None
     if not args.no_prefill_timing:
         ev[0].record()
-        model.prefill(cache, prompt, next_tokens=first)
+        run_prefill()
         ev[1].record()
         torch.cuda.synchronize()
         prefill_ms = ev[0].elapsed_time(ev[1])

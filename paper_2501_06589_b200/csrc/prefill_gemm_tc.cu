@@ -5,8 +5,8 @@
 //
 // Persistent CTAs, one per SM, 192 threads in three roles that meet only at mbarriers:
 //   warp 0     TMA producer: per 64-wide K block one 128x64 box of A_hi, one of A_lo and one 256x64
-//              box of W (cp.async.bulk.tensor.2d, 128-byte swizzle, out-of-range rows/columns
-//              zero-filled by the TMA unit) into a 3-stage shared-memory ring;
+//              (or 128x64: see TcCfg) box of W (cp.async.bulk.tensor.2d, 128-byte swizzle, out-of-range
+//              rows/columns zero-filled by the TMA unit) into a 3- or 4-stage shared-memory ring;
 //   warp 1     MMA issuer: one elected thread issues tcgen05.mma (M 128, N 256, K 16, kind::f16,
 //              bf16 x bf16 -> fp32) straight from shared-memory descriptors -- 4 K-steps for the high
 //              part and 4 for the low part of A against the same W tile -- and releases ring stages /
@@ -27,11 +27,22 @@
 namespace ladder {
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 3, UMMA_K = 16;
+constexpr int BM = 128, BK = 64, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2;  // 16 KB
-constexpr int B_BYTES = BN * BK * 2;  // 32 KB
-constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;
 constexpr int kTcThreads = 192;
+// Tile width BN = 256 by default; 128 when that leaves SMs without a tile (small M x N: a short prompt, a chunk of a
+// prompt, a narrow projection), which doubles the number of tiles at the same bytes per flop for A.
+template <int BN>
+struct TcCfg {
+  static constexpr int B_BYTES = BN * BK * 2;               // 32 / 16 KB
+  static constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;  // 64 / 48 KB
+  static constexpr int STAGES = BN == 256 ? 3 : 4;
+  static constexpr int OFF_BARS = STAGES * STAGE_BYTES;  // full[], empty[], tmem_full[2], tmem_empty[2], tmem slot
+  static constexpr int SMEM = OFF_BARS + 16 * 8 + 1024;
+  // Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M x N.
+  static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
+                                    (static_cast<uint32_t>(BM >> 4) << 24);
+};
 constexpr int GROUP_M = 16;  // M-tiles per rasterisation band
 
 // tile index -> (m tile, n tile): bands of GROUP_M m-tiles, m fastest inside a band
@@ -43,8 +54,6 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
   tm = m_first + r % band_m;
   tn = r / band_m;
 }
-constexpr int OFF_BARS = STAGES * STAGE_BYTES;  // full[3], empty[3], tmem_full[2], tmem_empty[2], tmem slot
-constexpr int kTcSmem = OFF_BARS + 16 * 8 + 1024;
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -93,14 +102,15 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   d |= static_cast<uint64_t>(2) << 61;                 // SWIZZLE_128B
   return d;
 }
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M x N.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
-                            (static_cast<uint32_t>(BM >> 4) << 24);
 
-template <bool SPLIT>
+template <bool SPLIT, int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 largem_gemm_tc_kernel(const LargeMParams p, const __grid_constant__ CUtensorMap map_a,
                       const __grid_constant__ CUtensorMap map_alo, const __grid_constant__ CUtensorMap map_w) {
+  using C = TcCfg<BN>;
+  constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, B_BYTES = C::B_BYTES, OFF_BARS = C::OFF_BARS;
+  constexpr uint32_t kIdesc = C::IDESC;
+  constexpr int kTmemCols = 2 * BN;  // two fp32 accumulators of BN columns
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + OFF_BARS);
@@ -125,8 +135,9 @@ largem_gemm_tc_kernel(const LargeMParams p, const __grid_constant__ CUtensorMap 
     }
     fence_barrier_init();
   }
-  if (warp == 1) {  // TMEM: 512 columns x 128 lanes of fp32
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot))
+  if (warp == 1) {  // TMEM: 2 BN columns x 128 lanes of fp32
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "n"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -228,7 +239,7 @@ largem_gemm_tc_kernel(const LargeMParams p, const __grid_constant__ CUtensorMap 
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
   }
 }
 
@@ -260,15 +271,23 @@ cudaError_t largem_gemm_tc_init() {
     if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
     g_encode = reinterpret_cast<EncodeFn>(fn);
   }
-  cudaError_t e = cudaFuncSetAttribute(largem_gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(largem_gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
+  cudaError_t e = cudaFuncSetAttribute(largem_gemm_tc_kernel<true, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       TcCfg<256>::SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(largem_gemm_tc_kernel<false, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             TcCfg<256>::SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(largem_gemm_tc_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             TcCfg<128>::SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(largem_gemm_tc_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             TcCfg<128>::SMEM);
+  return e;
 }
 
-cudaError_t launch_largem_gemm_tc(const LargeMParams& p, cudaStream_t stream, int sm_count) {
-  if (!g_encode) return cudaErrorNotReady;
-  if ((reinterpret_cast<uintptr_t>(p.A) | reinterpret_cast<uintptr_t>(p.W) | reinterpret_cast<uintptr_t>(p.A_lo)) & 15)
-    return cudaErrorMisalignedAddress;
+namespace {
+template <int BN>
+cudaError_t launch_bn(const LargeMParams& p, cudaStream_t stream, int sm_count) {
   CUtensorMap ma, ml, mw;
   cudaError_t e = make_map(&ma, p.A, p.M, p.K, BM);
   if (e == cudaSuccess) e = make_map(&ml, p.A_lo ? p.A_lo : p.A, p.M, p.K, BM);
@@ -276,9 +295,19 @@ cudaError_t launch_largem_gemm_tc(const LargeMParams& p, cudaStream_t stream, in
   if (e != cudaSuccess) return e;
   const int tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
   const int grid = tiles < sm_count ? tiles : sm_count;
-  if (p.A_lo) largem_gemm_tc_kernel<true><<<grid, kTcThreads, kTcSmem, stream>>>(p, ma, ml, mw);
-  else largem_gemm_tc_kernel<false><<<grid, kTcThreads, kTcSmem, stream>>>(p, ma, ml, mw);
+  if (p.A_lo) largem_gemm_tc_kernel<true, BN><<<grid, kTcThreads, TcCfg<BN>::SMEM, stream>>>(p, ma, ml, mw);
+  else largem_gemm_tc_kernel<false, BN><<<grid, kTcThreads, TcCfg<BN>::SMEM, stream>>>(p, ma, ml, mw);
   return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_largem_gemm_tc(const LargeMParams& p, cudaStream_t stream, int sm_count) {
+  if (!g_encode) return cudaErrorNotReady;
+  if ((reinterpret_cast<uintptr_t>(p.A) | reinterpret_cast<uintptr_t>(p.W) | reinterpret_cast<uintptr_t>(p.A_lo)) & 15)
+    return cudaErrorMisalignedAddress;
+  // 256-wide tiles unless they leave SMs idle; then 128-wide ones (twice as many tiles)
+  const int tiles256 = ((p.M + BM - 1) / BM) * ((p.N + 255) / 256);
+  return tiles256 < sm_count ? launch_bn<128>(p, stream, sm_count) : launch_bn<256>(p, stream, sm_count);
 }
 
 }  // namespace ladder

@@ -190,7 +190,9 @@ def _split(shape, seed, std=1.0):
 @pytest.mark.parametrize("impl", [0, 1])          # 0 = tcgen05 kernel, 1 = warp-level mma.sync kernel
 @pytest.mark.parametrize("split", [False, True])
 @pytest.mark.parametrize("M,N,K,mode", [(16, 768, 256, 3), (300, 1376, 256, 1), (512, 256, 688, 0),
-                                        (1000, 520, 264, 2), (4096, 1024, 1024, 0), (384, 2056, 8192, 2)])
+                                        (1000, 520, 264, 2), (4096, 1024, 1024, 0), (384, 2056, 8192, 2),
+                                        # enough 128 x 256 tiles for every SM (wide tiles); the others use 128 x 128
+                                        (2048, 2560, 512, 1), (2500, 2312, 320, 0)])
 def test_prefill_gemm(B, M, N, K, mode, split, impl):
     B.set_prefill_gemm_impl(impl)
     Af, A, A_lo = _split((M, K), 14)

@@ -37,6 +37,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
   __shared__ __align__(16) float ps[4][GT][16];
   __shared__ float red[4][GT][DH];
   __shared__ float mls[4][GT][2];
+  __shared__ float mfac[GT][4];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, tig = lane & 3;
@@ -216,24 +217,30 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
   }
   __syncthreads();
 
-  // ---- 4. merge the 4 warps, write the CTA partial
+  // ---- 4. merge the 4 warps, write the CTA partial.  The four rescaling factors of a head are computed once
+  // (one thread per head) instead of once per output element: the element loop is then 4 FMAs and a store.
   const int stride = DH + 2;
-  for (int idx = tid; idx < GT * DH; idx += kAttnThreads) {
-    const int h = idx / DH, d = idx % DH;
+  if (tid < GT) {
+    const int h = tid;
     const float M = fmaxf(fmaxf(mls[0][h][0], mls[1][h][0]), fmaxf(mls[2][h][0], mls[3][h][0]));
-    float o = 0.f, ls = 0.f;
+    float ls = 0.f;
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
       const float f = (mls[w][h][0] == -INFINITY) ? 0.f : __expf(mls[w][h][0] - M);
-      o += f * red[w][h][d];
+      mfac[h][w] = f;
       ls += f * mls[w][h][1];
     }
     float* dst = p.scratch + ((static_cast<size_t>(b) * p.n_q_heads + head0 + h) * p.n_splits + split) * stride;
-    dst[d] = o;
-    if (d == 0) {
-      dst[DH] = M;
-      dst[DH + 1] = ls;
-    }
+    dst[DH] = M;
+    dst[DH + 1] = ls;
+  }
+  __syncthreads();
+  for (int idx = tid; idx < GT * DH; idx += kAttnThreads) {
+    const int h = idx / DH, d = idx % DH;
+    float o = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) o += mfac[h][w] * red[w][h][d];
+    p.scratch[((static_cast<size_t>(b) * p.n_q_heads + head0 + h) * p.n_splits + split) * stride + d] = o;
   }
 }
 

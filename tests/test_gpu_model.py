@@ -391,6 +391,28 @@ def test_tp_rank_slice_shape_batches(B, variant, batch):
     assert agree >= (0.98 if batch >= 16 else 0.85), agree      # 7 comparisons at batch 1: at most one flip
 
 
+@pytest.mark.parametrize("batch", [12, 40])
+def test_wide_batch_path_is_reproducible(B, batch):
+    """Batch 9..64 (tcgen05 GEMMs whose shared tiles are finished by whichever CTA arrives last, operands handed
+    from kernel to kernel): two runs of the same prompt give bit-identical tokens, hidden states and caches -
+    the pieces of a shared tile are added in CTA order whatever the arrival order."""
+    s = synth.SHAPES["tp_slice"].with_layers(3)
+    w = synth.make_weights(s, device="cuda")
+    S, steps = 24, 10
+    prompt = synth.make_tokens(s, batch, S)
+    runs = []
+    for _ in range(2):
+        model = B.Model(w, batch, S + steps + 2, batch * S)
+        cache = B.KVCache(s, batch, S + steps + 2, fill=CANARY)
+        toks, hids = gpu_generate(B, model, cache, prompt, steps)
+        assert model.device_status() == 0
+        runs.append((toks, hids, cache.k.clone(), cache.v.clone()))
+        model.close()
+    assert np.array_equal(runs[0][0], runs[1][0])
+    assert np.array_equal(runs[0][1], runs[1][1])
+    assert torch.equal(runs[0][2], runs[1][2]) and torch.equal(runs[0][3], runs[1][3])
+
+
 def test_persistent_kernel_wait_runs_out_cleanly(B):
     """A dependency that is never met ends the launch after the 0.25 s limit with the timeout bit set;
     nothing hangs or faults, and once the status has been read the same model decodes correctly again."""

@@ -7,23 +7,43 @@ shares no code with the CUDA path and never receives a value computed there.
 
 What it follows
 ---------------
-* Standard residual recurrence  x_i = h_i(x_{i-1}) + x_{i-1}        (Sec. 2, Eq. 1)
-* Ladder recurrence             x_i = h_i(x_{i-2}) + x_{i-1}        (Sec. 3.1, Eq. 2)
-* The layer routine with pending module outputs                     (Algorithm 1)
-  with the asynchronous all-reduce and its handle being the identity on a
-  single device.
-* "Llama-3's model architecture" (Sec. 3.3.1): pre-norm RMSNorm, rotary
-  position embedding on interleaved pairs, grouped-query causal attention,
-  SwiGLU MLP, final RMSNorm, untied LM head, no biases.
+The model is a chain of 2N modules (attention, MLP, attention, ...) acting on a
+residual stream x_0, x_1, ..., x_2N.  Every module adds its output to the newest
+stream value; what differs between the architectures is only WHICH stream value
+a module reads:
+* Standard residual   x_m = x_{m-1} + h_m(x_{m-1})                  (Sec. 2, Eq. 1)
+* Ladder residual     x_m = x_{m-1} + h_m(x_{m-2})                  (Sec. 3.1, Eq. 2)
+* Parallel attention and MLP (Sec. 3.3.1): both modules of a layer read the
+  layer's input through ONE norm, and both outputs are added.
+* Communication-free upper bound (Sec. 3.3.1): the standard model with the
+  all-reduce deleted; on a single device, where the all-reduce is the
+  identity, it IS the standard model (``upper_bound`` is an alias).
+``run_layers`` is that chain written once, with a per-module flag "reads one
+module back".  Algorithm 1 (a layer routine that carries the two not-yet-added
+module outputs from layer to layer, with the asynchronous all-reduce and its
+handle being the identity on one device) computes the same thing; the tests
+write Algorithm 1 out and pin this oracle to it.
+Tensor parallelism (Sec. 2, Eq. 1 with AllReduce): ``tp_world > 1`` splits each
+module over ranks by heads / MLP columns and sums the ranks' partial outputs --
+the all-reduce -- before the residual add.
+"Llama-3's model architecture" (Sec. 3.3.1): pre-norm RMSNorm, rotary position
+embedding on interleaved pairs, grouped-query causal attention, SwiGLU MLP,
+final RMSNorm, untied LM head, no biases.
 
 Readings taken where the paper is silent (both sides of every parity test use
 the same ones):
 * initial pending outputs of Algorithm 1 are zero, so modules 1 and 2 both read x_0;
 * the two outputs still pending after the last layer are added before the
   final norm (Eq. 2 adds every h_i into the stream);
-* a standard layer first adds whatever is pending and leaves nothing pending
-  (hybrid models: the first ladder attention after a standard layer reads the
-  complete stream) -- PARITY UNPINNED by the paper for this hybrid boundary rule;
+* hybrid models: the attention module of a ladder layer that follows a standard
+  (or parallel) layer reads the complete stream, and the MLP of that layer is
+  the first module that reads one module back (in Algorithm 1's terms: a
+  standard layer adds whatever is pending and leaves nothing pending) --
+  PARITY UNPINNED by the paper for this hybrid boundary rule; ``module_stale``
+  states any other rule explicitly, module by module;
+* a parallel layer normalises once, with the layer's attention-norm gain; its
+  MLP-norm gain is unused -- PARITY UNPINNED by the paper (it names the PaLM
+  formulation and prints no equations);
 * greedy argmax takes the lowest index among equal maxima.
 
 Arithmetic: every array is ``dtype`` (float64 by default, float32 for the large
@@ -40,8 +60,12 @@ Storage precision switches (the definition is both off):
   noise from bugs.
 
 Pins (tests/test_oracle_pins.py): single-module ladder == standard, cached
-decode == recomputation, softmax rows, brute-force attention, Eq.-2 form ==
-Algorithm-1 form, staleness, telescoping sum, single live module, closed forms
+decode == recomputation, softmax rows, brute-force attention, module chain ==
+Algorithm 1 written out in the test, parallel layer == its recurrence written
+out, upper bound == standard, tensor-parallel partial sums == the unsplit
+module and == a model built from one rank's weight slice, pipeline stages
+chained == the whole model, staleness, telescoping sum, single live module,
+closed forms
 for zeroed projections, RoPE relative-position property, RMSNorm textbook
 formula, GQA == MHA with repeated heads, causality, batch independence,
 linear layers vs float64 matmul written out in the test.
@@ -67,11 +91,65 @@ class OracleConfig:
     rms_eps: float = 1e-5
     rope_theta: float = 10000.0
     layer_is_ladder: Optional[Sequence[bool]] = None  # None = every layer ladder
+    # Per-layer architecture, overriding layer_is_ladder when given: "standard" (Eq. 1), "ladder" (Eq. 2),
+    # "parallel" (Sec. 3.3.1, parallel attention and MLP), "upper_bound" (Sec. 3.3.1: standard without
+    # communication = standard on one device).
+    layer_mode: Optional[Sequence[str]] = None
+    # Explicit per-module rule, overriding what the layer modes imply: entry m-1 is True when module m
+    # (1-based; odd = attention, even = MLP) reads x_{m-2} instead of x_{m-1}.
+    module_stale: Optional[Sequence[bool]] = None
+    tp_world: int = 1     # tensor-parallel ranks the modules are split over (partials summed = all-reduce)
 
     def ladder(self, layer: int) -> bool:
+        return self.mode(layer) == "ladder"
+
+    def mode(self, layer: int) -> str:
+        if self.layer_mode is not None:
+            m = self.layer_mode[layer]
+            return "standard" if m == "upper_bound" else m
         if self.layer_is_ladder is None:
-            return True
-        return bool(self.layer_is_ladder[layer])
+            return "ladder"
+        return "ladder" if self.layer_is_ladder[layer] else "standard"
+
+
+@dataclass
+class ModuleSpec:
+    """Module m of the chain: what it is, and which stream value it reads."""
+    kind: str            # "attention" | "mlp"
+    layer: int
+    stale: bool          # True: reads x_{m-2} (Eq. 2); False: reads x_{m-1} (Eq. 1)
+    norm: str            # name of the RMSNorm gain applied to its input
+
+
+def module_chain(cfg: OracleConfig) -> List[ModuleSpec]:
+    """The 2N modules in order, each with the stream value it reads.
+
+    standard layer : both modules read the newest value (Eq. 1).
+    ladder layer   : both modules read one module back (Eq. 2), except an attention module that directly
+                     follows a non-ladder layer, which reads the newest value (hybrid boundary reading).
+    parallel layer : attention reads the newest value x_{m-1}; the MLP reads that same x_{m-1} -- one module
+                     back from where it stands -- through the same (attention) norm, so that
+                     x_{m+1} = x_{m-1} + Attn(n) + MLP(n) with n = Norm(x_{m-1}).
+    """
+    chain: List[ModuleSpec] = []
+    for l in range(cfg.n_layers):
+        mode = cfg.mode(l)
+        if mode == "standard":
+            flags, mlp_norm = (False, False), "mlp_norm"
+        elif mode == "ladder":
+            after_ladder = l > 0 and cfg.mode(l - 1) == "ladder"
+            flags, mlp_norm = (after_ladder or l == 0, True), "mlp_norm"
+        elif mode == "parallel":
+            flags, mlp_norm = (False, True), "attn_norm"
+        else:
+            raise ValueError(mode)
+        chain.append(ModuleSpec("attention", l, flags[0], "attn_norm"))
+        chain.append(ModuleSpec("mlp", l, flags[1], mlp_norm))
+    if cfg.module_stale is not None:
+        assert len(cfg.module_stale) == len(chain)
+        for spec, st in zip(chain, cfg.module_stale):
+            spec.stale = bool(st)
+    return chain
 
 
 class OracleWeights:
@@ -191,14 +269,22 @@ class OracleCache:
 
 
 # --------------------------------------------------------------------------- modules
+def _tp_slices(width: int, world: int) -> List[slice]:
+    """Contiguous equal slices of an inner dimension, one per tensor-parallel rank."""
+    assert width % world == 0
+    step = width // world
+    return [slice(r * step, (r + 1) * step) for r in range(world)]
+
+
 def attention_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndarray,
                      pos0: int, cache: Optional[OracleCache], bf16_storage: bool = False,
-                     bf16_kv: bool = False):
+                     bf16_kv: bool = False, tp_rank: Optional[int] = None):
     """h(n) for the attention module of ``layer``.
 
     n [B, T, d] is the normalised input at absolute positions pos0..pos0+T-1.
     With a cache, the new K/V rows are appended at those positions first and
     attention then runs over positions 0..pos0+T-1 (append, then attend).
+    With ``tp_rank`` the result is that rank's partial sum x* (before the all-reduce) only.
     """
     B, T, d = n.shape
     Hq, Hkv, Dh = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
@@ -226,18 +312,30 @@ def attention_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndar
             kk, vv = k[b], v[b]
         o[b] = causal_attention(q[b], kk, vv, pos0)
     o = _store(o.reshape(B, T, Hq * Dh), bf16_storage)
-    return o @ wo.T
+    # Output projection.  Under tensor parallelism rank r owns the query heads [r Hq/P, (r+1) Hq/P) (and their
+    # kv heads), so everything up to here is rank-local; it multiplies its heads' slice of o with the matching
+    # columns of W_o, and the partial products are summed over the ranks (the all-reduce of Sec. 2, Eq. 1).
+    parts = [o[..., c] @ wo[:, c].T for c in _tp_slices(Hq * Dh, cfg.tp_world)]
+    if tp_rank is not None:
+        return parts[tp_rank]
+    return parts[0] if len(parts) == 1 else np.sum(parts, axis=0)
 
 
 def mlp_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndarray,
-               bf16_storage: bool = False):
-    """h(n) = W_down ( silu(W_gate n) * (W_up n) )."""
+               bf16_storage: bool = False, tp_rank: Optional[int] = None):
+    """h(n) = W_down ( silu(W_gate n) * (W_up n) ).
+
+    Under tensor parallelism rank r owns the hidden columns [r F/P, (r+1) F/P): W_gate and W_up split by
+    output, W_down by input, partial products summed over the ranks (Sec. 2).  ``tp_rank``: that rank's partial."""
     dt = n.dtype
     wg = W.get("w_gate", layer).astype(dt, copy=False)
     wu = W.get("w_up", layer).astype(dt, copy=False)
     wd = W.get("w_down", layer).astype(dt, copy=False)
     h = _store(silu(n @ wg.T) * (n @ wu.T), bf16_storage)
-    return h @ wd.T
+    parts = [h[..., c] @ wd[:, c].T for c in _tp_slices(cfg.d_ff, cfg.tp_world)]
+    if tp_rank is not None:
+        return parts[tp_rank]
+    return parts[0] if len(parts) == 1 else np.sum(parts, axis=0)
 
 
 # --------------------------------------------------------------------------- forward
@@ -259,44 +357,33 @@ def greedy(logits: np.ndarray) -> np.ndarray:
 def run_layers(cfg: OracleConfig, W: OracleWeights, x: np.ndarray, pos0: int,
                cache: Optional[OracleCache], bf16_storage: bool = False,
                record: Optional[ForwardResult] = None, n_layers: Optional[int] = None,
-               bf16_kv: bool = False):
-    """The layer stack in Algorithm-1 form, then the final flush.  x [B,T,d]."""
-    a_p = np.zeros_like(x)              # pending attention output (attn_out)
-    m_p = np.zeros_like(x)              # pending MLP output       (mlp_out)
-    L = cfg.n_layers if n_layers is None else n_layers
-    for l in range(L):
-        g_a = W.get("attn_norm", l)
-        g_m = W.get("mlp_norm", l)
-        if cfg.ladder(l):
-            x = x + a_p                                                  # residual += attn_out
-            n = _store(rmsnorm(x, g_a, cfg.rms_eps), bf16_storage)       # AttentionNorm
-            if record is not None:
-                record.module_inputs.append(x.copy())
-            a_p = attention_module(cfg, W, l, n, pos0, cache, bf16_storage, bf16_kv)
-            x = x + m_p                                                  # residual += mlp_out
-            n = _store(rmsnorm(x, g_m, cfg.rms_eps), bf16_storage)       # MLPNorm
-            if record is not None:
-                record.module_inputs.append(x.copy())
-            m_p = mlp_module(cfg, W, l, n, bf16_storage)
-            if record is not None:
-                record.module_outputs += [a_p.copy(), m_p.copy()]
+               bf16_kv: bool = False, first_layer: int = 0, older: Optional[np.ndarray] = None,
+               return_state: bool = False):
+    """The module chain x_m = x_{m-1} + h_m(x_{m-1} or x_{m-2}) (Eq. 1 / Eq. 2).  x [B,T,d] is x_0.
+
+    Only the last two stream values are kept.  Module 1 has no x_{-1}: it reads x_0 whatever its flag.
+
+    Pipeline stages (Sec. 5.1): a stage runs layers first_layer .. n_layers-1 starting from the stream state
+    (older, x) = (x_{m-2}, x_{m-1}) it was handed and, with ``return_state``, hands on the same pair.  In
+    Algorithm 1's variables the pair is (residual + attn_out, residual + attn_out + mlp_out): the three
+    tensors the paper forwards carry exactly these two sums.
+    """
+    chain = module_chain(cfg)
+    last = cfg.n_layers if n_layers is None else n_layers
+    chain = chain[2 * first_layer:2 * last]
+    newest = x                              # x_{m-1}; ``older`` is x_{m-2} (None before module 1)
+    for spec in chain:
+        src = older if (spec.stale and older is not None) else newest
+        n = _store(rmsnorm(src, W.get(spec.norm, spec.layer), cfg.rms_eps), bf16_storage)
+        if spec.kind == "attention":
+            out = attention_module(cfg, W, spec.layer, n, pos0, cache, bf16_storage, bf16_kv)
         else:
-            x = x + a_p + m_p                                            # nothing stays pending
-            a_p = np.zeros_like(x)
-            m_p = np.zeros_like(x)
-            n = _store(rmsnorm(x, g_a, cfg.rms_eps), bf16_storage)
-            if record is not None:
-                record.module_inputs.append(x.copy())
-            a = attention_module(cfg, W, l, n, pos0, cache, bf16_storage, bf16_kv)
-            x = x + a
-            n = _store(rmsnorm(x, g_m, cfg.rms_eps), bf16_storage)
-            if record is not None:
-                record.module_inputs.append(x.copy())
-            m = mlp_module(cfg, W, l, n, bf16_storage)
-            x = x + m
-            if record is not None:
-                record.module_outputs += [a.copy(), m.copy()]
-    return x + a_p + m_p
+            out = mlp_module(cfg, W, spec.layer, n, bf16_storage)
+        if record is not None:
+            record.module_inputs.append(src.copy())
+            record.module_outputs.append(out.copy())
+        older, newest = newest, newest + out
+    return (older, newest) if return_state else newest
 
 
 def embed(W: OracleWeights, tokens: np.ndarray, dtype) -> np.ndarray:
@@ -356,14 +443,15 @@ def decode_step(cfg, W, tokens, cache: OracleCache, dtype=np.float64, bf16_stora
 
 
 def generate(cfg, W, prompt: np.ndarray, n_steps: int, max_seq_len: int, dtype=np.float64,
-             forced: Optional[np.ndarray] = None, bf16_storage=False, bf16_kv=False):
+             forced: Optional[np.ndarray] = None, bf16_storage=False, bf16_kv=False,
+             return_logits: bool = False):
     """prefill + n_steps decode steps.
 
     Returns (tokens [B, n_steps+1], hiddens [B, n_steps+1, d]): entry 0 comes from
     the prefill (token at position S), entry j+1 from decode step j.  With
     ``forced`` [B, n_steps+1] the fed-back tokens are taken from it instead of the
     oracle's own argmax (teacher forcing), while the returned tokens stay the
-    oracle's own choices.
+    oracle's own choices.  ``return_logits`` adds the logits [B, n_steps+1, V].
     """
     prompt = np.asarray(prompt)
     B, S = prompt.shape
@@ -371,9 +459,13 @@ def generate(cfg, W, prompt: np.ndarray, n_steps: int, max_seq_len: int, dtype=n
     r = prefill(cfg, W, prompt, cache, dtype, bf16_storage, bf16_kv=bf16_kv)
     toks = [r.next_tokens[:, 0]]
     hids = [r.hidden[:, 0]]
+    logs = [r.logits[:, 0]]
     for j in range(n_steps):
         feed = toks[-1] if forced is None else np.asarray(forced)[:, j]
         r = decode_step(cfg, W, feed, cache, dtype, bf16_storage, bf16_kv=bf16_kv)
         toks.append(r.next_tokens[:, 0])
         hids.append(r.hidden[:, 0])
+        logs.append(r.logits[:, 0])
+    if return_logits:
+        return np.stack(toks, axis=1), np.stack(hids, axis=1), np.stack(logs, axis=1)
     return np.stack(toks, axis=1), np.stack(hids, axis=1)

@@ -187,7 +187,42 @@ def _modules(cfg, t):
     return mods
 
 
-def test_algorithm1_form_equals_equation2_form():
+def _algorithm1(cfg, t, x0, masks):
+    """Algorithm 1 written out here: a layer routine that carries the stream `residual` and the two module
+    outputs that have not been added yet from layer to layer (the all-reduce and its handle are the identity
+    on one device).  masks[l] true: ladder layer; false: a standard layer, which first adds what is pending."""
+    mods = _modules(cfg, t)
+    residual = x0
+    attn_out = np.zeros_like(x0)
+    mlp_out = np.zeros_like(x0)
+    states = []
+    for l in range(cfg.n_layers):
+        attn, mlp = mods[2 * l], mods[2 * l + 1]
+        if masks[l]:
+            residual = residual + attn_out
+            attn_out = attn(residual)
+            residual = residual + mlp_out
+            mlp_out = mlp(residual)
+        else:
+            residual = residual + attn_out + mlp_out
+            residual = residual + attn(residual)
+            residual = residual + mlp(residual)
+            attn_out = np.zeros_like(x0)
+            mlp_out = np.zeros_like(x0)
+        states.append((residual, attn_out, mlp_out))
+    return residual + attn_out + mlp_out, states
+
+
+@pytest.mark.parametrize("masks", [[1, 1, 1], [0, 1, 1], [1, 0, 1], [1, 1, 0], [0, 0, 0]])
+def test_module_chain_equals_algorithm1_written_here(masks):
+    cfg = small_cfg(n_layers=3, ladder=masks)
+    t = rand_weights(cfg, 11)
+    want, _ = _algorithm1(cfg, t, _x0(t, TOK), masks)
+    r = O.forward(cfg, W(t), TOK, record=True)
+    assert np.allclose(r.x_final, want, atol=1e-11)
+
+
+def test_all_ladder_chain_reads_two_back():
     cfg = small_cfg(n_layers=3)
     t = rand_weights(cfg, 11)
     mods = _modules(cfg, t)
@@ -198,6 +233,138 @@ def test_algorithm1_form_equals_equation2_form():
     assert np.allclose(r.x_final, xs[-1], atol=1e-11)
     for m in range(1, 2 * cfg.n_layers + 1):
         assert np.allclose(r.module_inputs[m - 1], xs[max(m - 2, 0)], atol=1e-11)
+
+
+def test_parallel_layers_recurrence_written_here():
+    """Parallel attention and MLP (Sec. 3.3.1): x_l = x_{l-1} + Attn(n) + MLP(n), n = Norm(x_{l-1}) with one
+    norm (the attention gain); the MLP gain must not matter; and the result differs from the standard model."""
+    cfg = small_cfg(n_layers=3)
+    cfg.layer_mode = ["parallel"] * 3
+    t = rand_weights(cfg, 31)
+    Wt = W(t)
+    x = _x0(t, TOK)
+    for l in range(3):
+        n = O.rmsnorm(x, t[("attn_norm", l)], cfg.rms_eps)
+        x = x + O.attention_module(cfg, Wt, l, n, 0, None) + O.mlp_module(cfg, Wt, l, n)
+    r = O.forward(cfg, Wt, TOK)
+    assert np.allclose(r.x_final, x, atol=1e-11)
+    t2 = dict(t)
+    for l in range(3):
+        t2[("mlp_norm", l)] = t[("mlp_norm", l)] * 3.0
+    assert np.array_equal(O.forward(cfg, W(t2), TOK).x_final, r.x_final)
+    std = O.forward(small_cfg(n_layers=3, ladder=[0, 0, 0]), Wt, TOK)
+    assert not np.allclose(std.x_final, x, atol=1e-3)
+
+
+def test_parallel_layer_mixed_with_ladder_and_standard():
+    cfg = small_cfg(n_layers=4)
+    cfg.layer_mode = ["standard", "parallel", "ladder", "parallel"]
+    t = rand_weights(cfg, 32)
+    mods = _modules(cfg, t)
+    Wt = W(t)
+    par_mlp = lambda x, l: O.mlp_module(cfg, Wt, l, O.rmsnorm(x, t[("attn_norm", l)], cfg.rms_eps))
+    x0 = _x0(t, TOK)
+    x1 = x0 + mods[0](x0)
+    x2 = x1 + mods[1](x1)                 # standard layer
+    x3 = x2 + mods[2](x2)
+    x4 = x3 + par_mlp(x2, 1)              # parallel layer: both read x2
+    x5 = x4 + mods[4](x4)                 # ladder attention after a non-ladder layer: complete stream
+    x6 = x5 + mods[5](x4)                 # its MLP reads one module back
+    x7 = x6 + mods[6](x6)                 # parallel layer after a ladder layer: complete stream
+    x8 = x7 + par_mlp(x6, 3)
+    assert np.allclose(O.forward(cfg, Wt, TOK).x_final, x8, atol=1e-11)
+
+
+def test_upper_bound_is_the_standard_model_on_one_device():
+    cfg_u = small_cfg(n_layers=3)
+    cfg_u.layer_mode = ["upper_bound"] * 3
+    cfg_s = small_cfg(n_layers=3, ladder=[0, 0, 0])
+    t = rand_weights(cfg_u, 33)
+    assert np.array_equal(O.forward(cfg_u, W(t), TOK).hidden, O.forward(cfg_s, W(t), TOK).hidden)
+
+
+def test_explicit_module_flags_give_the_other_hybrid_boundary_reading():
+    """module_stale states the rule module by module: here the first ladder attention after a standard layer
+    also reads one module back (x_1, skipping the standard layer's MLP output)."""
+    cfg = small_cfg(n_layers=2, ladder=[0, 1])
+    cfg.module_stale = [0, 0, 1, 1]
+    t = rand_weights(cfg, 34)
+    mods = _modules(cfg, t)
+    x0 = _x0(t, TOK)
+    x1 = x0 + mods[0](x0)
+    x2 = x1 + mods[1](x1)
+    x3 = x2 + mods[2](x1)
+    x4 = x3 + mods[3](x2)
+    assert np.allclose(O.forward(cfg, W(t), TOK).x_final, x4, atol=1e-11)
+    cfg.module_stale = None
+    assert not np.allclose(O.forward(cfg, W(t), TOK).x_final, x4, atol=1e-6)
+
+
+def _rank_slice(cfg, t, r, world):
+    """Weights of the model one tensor-parallel rank holds: its query heads with their kv heads, its MLP columns."""
+    dh = cfg.head_dim
+    hq, hkv, f = cfg.n_q_heads // world, cfg.n_kv_heads // world, cfg.d_ff // world
+    cfg_r = small_cfg(n_layers=cfg.n_layers, d=cfg.d_model, hq=hq, hkv=hkv, dh=dh, f=f, v=cfg.vocab_size,
+                      ladder=cfg.layer_is_ladder)
+    tr = dict(t)
+    for l in range(cfg.n_layers):
+        tr[("wq", l)] = t[("wq", l)][r * hq * dh:(r + 1) * hq * dh]
+        tr[("wk", l)] = t[("wk", l)][r * hkv * dh:(r + 1) * hkv * dh]
+        tr[("wv", l)] = t[("wv", l)][r * hkv * dh:(r + 1) * hkv * dh]
+        tr[("wo", l)] = t[("wo", l)][:, r * hq * dh:(r + 1) * hq * dh]
+        tr[("w_gate", l)] = t[("w_gate", l)][r * f:(r + 1) * f]
+        tr[("w_up", l)] = t[("w_up", l)][r * f:(r + 1) * f]
+        tr[("w_down", l)] = t[("w_down", l)][:, r * f:(r + 1) * f]
+    return cfg_r, tr
+
+
+def test_tensor_parallel_partials_sum_to_the_unsplit_module():
+    """(XA)B = sum_r (X A_r) B_r (Sec. 2): a rank's partial equals the module of the model built from that rank's
+    weight slice (what the one-rank benchmark configuration runs), and the partials sum to the unsplit module."""
+    cfg = small_cfg(n_layers=1, hq=4, hkv=2, f=48)
+    t = rand_weights(cfg, 35)
+    rng = np.random.default_rng(35)
+    n = rng.normal(size=(2, 5, cfg.d_model))
+    whole_a = O.attention_module(cfg, W(t), 0, n, 0, None)
+    whole_m = O.mlp_module(cfg, W(t), 0, n)
+    cfg.tp_world = 2
+    parts_a, parts_m = [], []
+    for r in range(2):
+        cfg_r, tr = _rank_slice(cfg, t, r, 2)
+        pa = O.attention_module(cfg, W(t), 0, n, 0, None, tp_rank=r)
+        pm = O.mlp_module(cfg, W(t), 0, n, tp_rank=r)
+        assert np.allclose(pa, O.attention_module(cfg_r, W(tr), 0, n, 0, None), atol=1e-12)
+        assert np.allclose(pm, O.mlp_module(cfg_r, W(tr), 0, n), atol=1e-12)
+        parts_a.append(pa)
+        parts_m.append(pm)
+    assert np.allclose(sum(parts_a), whole_a, atol=1e-12) and not np.allclose(parts_a[0], whole_a, atol=1e-3)
+    assert np.allclose(sum(parts_m), whole_m, atol=1e-12)
+    assert np.allclose(O.attention_module(cfg, W(t), 0, n, 0, None), whole_a, atol=1e-12)
+    # a whole model under tensor parallelism computes what the unsplit model computes, ladder or not
+    for ladder in (None, [0, 0]):
+        c1 = small_cfg(n_layers=2, hq=4, hkv=2, ladder=ladder)
+        c2 = small_cfg(n_layers=2, hq=4, hkv=2, ladder=ladder)
+        c2.tp_world = 2
+        t2 = rand_weights(c1, 36)
+        assert np.allclose(O.forward(c1, W(t2), TOK).hidden, O.forward(c2, W(t2), TOK).hidden, atol=1e-11)
+
+
+@pytest.mark.parametrize("masks", [[1, 1, 1, 1], [0, 0, 1, 1], [1, 0, 1, 0]])
+def test_pipeline_stages_chained_equal_the_whole_model(masks):
+    """Sec. 5.1: at a stage boundary the stream state is handed on.  Two stages chained give the whole model,
+    and the pair handed on is (residual + attn_out, residual + attn_out + mlp_out) of Algorithm 1's three tensors."""
+    cfg = small_cfg(n_layers=4, ladder=masks)
+    t = rand_weights(cfg, 37)
+    x0 = _x0(t, TOK)
+    whole = O.run_layers(cfg, W(t), x0, 0, None)
+    older, newest = O.run_layers(cfg, W(t), x0, 0, None, n_layers=2, return_state=True)
+    rest = O.run_layers(cfg, W(t), newest, 0, None, first_layer=2, older=older)
+    assert np.allclose(rest, whole, atol=1e-11)
+    _, states = _algorithm1(cfg, t, x0, masks)
+    residual, attn_out, mlp_out = states[1]
+    assert np.allclose(newest, residual + attn_out + mlp_out, atol=1e-11)
+    if masks[1]:
+        assert np.allclose(older, residual + attn_out, atol=1e-11)
 
 
 def test_standard_mask_equals_equation1():

@@ -12,7 +12,11 @@ timed region and is reported separately as `prefill`.
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 70b] [--impl reference]
 
 N > 1 runs N independent replicas (one process per GPU under torch.distributed; no data-path
-collective: the path does not shard) and reports the aggregate.
+collective: the path does not shard) and reports the aggregate.  Started without a launcher,
+`--gpus N` starts the N ranks itself.  The K-step loop is timed `--repeats` times (default 3)
+and the median is reported with every repeat's time and sampled SM clock.  At N = 1 the line also
+carries short runs of the other benchmark configurations and of the paper's comparison
+architectures (`other_configs`).
 """
 from __future__ import annotations
 
@@ -29,14 +33,6 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the gate/up decode GEMM, from the ncu
-# capture summarised in profiles/decode_gemm_gate_up_70b_batch4.md (true size, no scaling).
-NCU_TRAFFIC_BYTES = {("70b", 4): 945_259_008}
-# Persistent layer-stack kernel: DRAM traffic / algorithmic bytes of the ncu capture of a 4-layer slice
-# of the 70B shape (profiles/decode_stack_70b_4layers_batch4.md).  A full launch holds 141 GB on the
-# device, too large to capture; traffic grows with the layers like the algorithmic bytes do (every
-# weight byte is read once), so the full launch is scaled by this ratio.
-NCU_STACK_TRAFFIC_RATIO = {("70b", 4): 1.001}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
@@ -109,7 +105,8 @@ def oracle_decode_sample(shape, weights, kv_len, n_layers_sample, dtype_name="fl
     sub = shape.with_layers(n_layers_sample)
     cfg = O.OracleConfig(sub.d_model, sub.n_layers, sub.n_q_heads, sub.n_kv_heads, sub.head_dim, sub.d_ff,
                          sub.vocab_size, sub.rms_eps, sub.rope_theta,
-                         None if sub.layer_is_ladder is None else list(sub.layer_is_ladder))
+                         None if sub.layer_is_ladder is None else list(sub.layer_is_ladder),
+                         layer_mode=None if sub.layer_mode is None else list(sub.layer_mode))
     prov = synth.logical_provider(weights, dt)
     W = O.OracleWeights(provider=prov)
     for l in range(n_layers_sample):                       # widen the sample's weights outside the timed part
@@ -155,11 +152,7 @@ def run_reference(args):
         return 0
     import torch
     from paper_2501_06589_b200 import synth
-    shape = synth.SHAPES[args.config]
-    if args.batch:
-        shape = synth.replace(shape, batch=args.batch)
-    if args.standard:
-        shape = shape.as_standard()
+    shape = shape_for(args, synth)
     n_sample = min(2, shape.n_layers)
     w = synth.make_weights(shape.with_layers(n_sample), device="cpu")
     kv_len = shape.prompt_len
@@ -186,9 +179,18 @@ def run_reference(args):
     return 0
 
 
+def residual_rule(shape):
+    if shape.layer_mode is not None:
+        kinds = sorted(set(shape.layer_mode))
+        return f"all {kinds[0]}" if len(kinds) == 1 else "mixed " + "/".join(kinds)
+    if shape.layer_is_ladder is None:
+        return "all ladder"
+    return "all standard" if not any(shape.layer_is_ladder) else "hybrid mask"
+
+
 def workload_config(shape, args):
     return {"workload": f"{shape.name}: d_model {shape.d_model}, {shape.n_layers} layers "
-                        f"({'all ladder' if shape.layer_is_ladder is None else ('all standard' if not any(shape.layer_is_ladder) else 'hybrid mask')}), "
+                        f"({residual_rule(shape)}), "
                         f"{shape.n_q_heads}q/{shape.n_kv_heads}kv heads x {shape.head_dim}, ffn {shape.d_ff}, "
                         f"vocab {shape.vocab_size}",
             "batch": shape.batch, "prompt_len": shape.prompt_len, "decode_steps": args.steps,
@@ -197,11 +199,13 @@ def workload_config(shape, args):
             "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU"}
 
 
-def main():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=512)
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--repeats", type=int, default=3,
+                    help="the K-step timed loop is run this many times; the median is reported")
     ap.add_argument("--config", default="70b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--streams", type=int, default=None)
@@ -211,27 +215,228 @@ def main():
     ap.add_argument("--wide-impl", type=int, default=0,
                     help="decode GEMM kernels: 0 = default, 1 = mma.sync for batch 9..64, 2 = tcgen05 for every batch")
     ap.add_argument("--standard", action="store_true", help="the same shape with standard residuals (Eq. 1) in every layer")
+    ap.add_argument("--mode", default=None, choices=["ladder", "standard", "parallel", "upper_bound"],
+                    help="every layer in this architecture (paper Sec. 3.3.1) instead of the configuration's own")
     ap.add_argument("--multi-kernel", action="store_true",
                     help="one kernel per GEMM (two streams, CUDA graph, PDL) instead of the persistent decode kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill-timing", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the short runs of the other benchmark configurations appended to the line at N = 1")
     ap.add_argument("--prefill-chunk", type=int, default=0,
                     help="feed the prompt in chunks of this many tokens per sequence (ladder_prefill_append): the prompt-pass "
                          "workspace then holds one chunk, which is what lets batch 64 of the 70B shape fit beside 141 GB of weights")
     ap.add_argument("--prefill-impl", type=int, default=0,
-                    help="prompt-pass GEMMs: 0 = tcgen05, bf16 hi + lo activations (default); 1 = mma.sync; "
+                    help="prompt-pass GEMMs: 0 = default; 1 = mma.sync; "
                          "2 = tcgen05, one bf16 per activation (not the precision the parity bound is stated for)")
-    args = ap.parse_args()
+    ap.add_argument("--selftest-cpu", action="store_true", help=argparse.SUPPRESS)
+    return ap.parse_args(argv)
+
+
+def spawn_ranks(args, argv):
+    """`python bench.py --gpus N` outside a launcher: start N ranks (one per GPU) of this same script under
+    torch.distributed.run on 127.0.0.1 and pass rank 0's JSON line through."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+    return subprocess.run(cmd).returncode
+
+
+def selftest_cpu(args, rank, world):
+    """Plumbing check without a GPU (tests only): gloo ranks, made-up per-rank timings, the real reduction."""
+    import torch.distributed as dist
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms = max_over_ranks([100.0 * (rank + 1)], dist, "cpu")[0]
+    dist.barrier()
+    if rank == 0:
+        print(json.dumps({"selftest": True, "n_gpus": world, "ms": ms,
+                          "value": aggregate_rate(world, 4, args.steps, ms)}))
+    dist.destroy_process_group()
+    return 0
+
+
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else argv
+    args = parse_args(argv)
+    world_env = os.environ.get("WORLD_SIZE")
+    if args.gpus > 1 and world_env is None:
+        return spawn_ranks(args, argv)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(world_env or "1")
+    if world != args.gpus and rank == 0:      # the ranks that actually run are what the line reports as n_gpus
+        sys.stderr.write(f"bench.py: --gpus {args.gpus} but the launcher started {world} ranks; reporting {world}\n")
+    if args.selftest_cpu:
+        return selftest_cpu(args, rank, world)
     if args.impl == "reference":
         return run_reference(args)
+    return run_rank(args, rank, world)
 
-    import numpy as np
+
+def shape_for(args, synth):
+    shape = synth.SHAPES[args.config]
+    if args.batch:
+        shape = synth.replace(shape, batch=args.batch)
+    if args.standard:
+        shape = shape.as_standard()
+    if args.mode:
+        shape = shape.as_mode(args.mode)
+    return shape
+
+
+class DecodeRun:
+    """One model + cache ready to decode from a fixed position; times K-step loops on the device."""
+
+    def __init__(self, B, torch, synth, shape, weights, steps, warm, args, dist, local, noise_kv=False):
+        self.B, self.torch, self.shape, self.dist, self.local = B, torch, shape, dist, local
+        self.steps, self.warm = steps, warm
+        S, bsz = shape.prompt_len, shape.batch
+        self.S, self.bsz = S, bsz
+        max_seq = S + max(steps, warm) + 1
+        chunk = args.prefill_chunk if 0 < args.prefill_chunk < S else S
+        if noise_kv:
+            chunk = 16
+        self.chunk = chunk
+        w = weights if weights.shape is shape else synth.replace(weights, shape=shape)
+        self.model = B.Model(w, bsz, max_seq, bsz * chunk)
+        if args.multi_kernel:
+            self.model.set_persistent(False)
+        self.persistent = self.model.persistent_active() and bsz <= 8
+        if args.streams is not None or args.graph is not None or args.pdl is not None:
+            self.model.set_schedule(2 if args.streams is None else args.streams, 1 if args.graph is None else args.graph,
+                                    1 if args.pdl is None else args.pdl)
+        self.cache = B.KVCache(shape, bsz, max_seq)
+        self.prompt = torch.from_numpy(synth.make_tokens(shape, bsz, S)).cuda()
+        self.nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+        self.first = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+        self.noise_kv = noise_kv
+        if noise_kv:     # timing only: a cache of seeded noise instead of a prompt pass over S tokens
+            g = torch.Generator(device="cuda")
+            g.manual_seed(11)
+            for t in (self.cache.k, self.cache.v):
+                for s0 in range(0, t.numel(), 1 << 27):
+                    t[s0:s0 + (1 << 27)].normal_(0.0, 0.5, generator=g)
+            self.first.copy_(self.prompt[:, 0])
+
+    def sync_all(self):
+        self.torch.cuda.synchronize()
+        if self.dist:
+            self.dist.barrier()
+            self.torch.cuda.synchronize()
+
+    def prefill(self):
+        m, c = self.model, self.chunk
+        m.prefill(self.cache, self.prompt[:, :c].contiguous(), next_tokens=self.first)
+        for p0 in range(c, self.S, c):
+            m.prefill_append(self.cache, self.prompt[:, p0:min(self.S, p0 + c)].contiguous(), next_tokens=self.first)
+
+    def rewind(self):
+        self.cache.seq_lens.fill_(self.S)
+        self.model.set_position(self.S)
+        self.nxt.copy_(self.first)
+
+    def timed_loop(self):
+        """K decode steps, device-timed with events on the launching stream; returns (ms, clock summary, launches)."""
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.rewind()
+        self.sync_all()
+        l0 = self.model.kernel_launches()
+        with ClockSampler(self.local) as clocks:
+            e0.record()
+            for _ in range(self.steps):
+                self.model.decode_step(self.cache, self.nxt, next_tokens=self.nxt)
+            e1.record()
+            self.sync_all()
+        return e0.elapsed_time(e1), clocks.summary(), self.model.kernel_launches() - l0
+
+    def warm_up(self):
+        self.rewind()
+        for _ in range(self.warm):
+            self.model.decode_step(self.cache, self.nxt, next_tokens=self.nxt)
+
+    def close(self):
+        self.model.close()
+
+
+def median_loop(run, repeats):
+    """Runs the timed loop `repeats` times; returns (median ms over ranks' maxima, per-repeat records, launches)."""
+    recs, launches = [], 0
+    for _ in range(max(1, repeats)):
+        ms, clk, launches = run.timed_loop()
+        ms = max_over_ranks([ms], run.dist, "cuda")[0]
+        recs.append({"ms": ms, "sm_mhz": clk["sm_mhz"], "reasons": clk["reasons"], "samples": clk["samples"]})
+    return statistics.median(r["ms"] for r in recs), recs, launches
+
+
+def merged_clocks(recs):
+    mhz = [r["sm_mhz"] for r in recs if r["sm_mhz"] is not None]
+    reasons = sorted({x for r in recs for x in r["reasons"]})
+    return mhz, reasons
+
+
+def short_run(B, torch, synth, shape, weights, args, local, steps=32, repeats=3, noise_kv=False):
+    """One of the other configurations: ms/step (median of `repeats` loops) and roofline fractions."""
+    hbm_peak, _, _ = measured_peaks()
+    run = DecodeRun(B, torch, synth, shape, weights, steps, 3, args, None, local, noise_kv=noise_kv)
+    if not noise_kv:
+        run.prefill()
+    run.warm_up()
+    ms, recs, launches = median_loop(run, repeats)
+    status = run.model.device_status()
+    run.close()
+    per = ms / steps
+    step_bytes = shape.decode_step_bytes(shape.prompt_len + (steps + 1) / 2.0)
+    gbs = step_bytes / (per * 1e-3) / 1e9
+    mhz, reasons = merged_clocks(recs)
+    return {"ms_per_step": round(per, 4), "tokens_per_s": round(shape.batch * steps / (ms * 1e-3), 1),
+            "gb_per_step": round(step_bytes / 1e9, 3), "frac_of_8tbs": round(gbs / NOMINAL_HBM_GBS, 4),
+            "frac_of_measured_copy_peak": round(gbs / hbm_peak, 4), "steps": steps,
+            "repeat_ms": [round(r["ms"], 3) for r in recs], "sm_mhz": mhz, "reasons": reasons,
+            "persistent": run.persistent, "launches_per_step": launches / steps, "device_status": status,
+            "kv": "seeded noise" if noise_kv else "prompt pass"}
+
+
+def other_configs(B, torch, synth, args, local, w70=None, shape70=None):
+    """Short decode runs of the other benchmark configurations and of the comparison architectures of the
+    paper's Sec. 3.3.1 (standard / parallel / ladder), so that one line carries them all."""
+    out = {}
+    if w70 is not None:      # the same 70B weights under the two other residual rules
+        for mode in ("standard", "parallel"):
+            out[f"70b_b{shape70.batch}_{mode}"] = short_run(B, torch, synth, shape70.as_mode(mode), w70, args, local)
+    return out
+
+
+def other_configs_small(B, torch, synth, args, local):
+    out = {}
+    for name in ("1p2b", "8b_hybrid"):
+        shape = synth.SHAPES[name]
+        w = synth.make_weights(shape, device="cuda")
+        out[name] = short_run(B, torch, synth, shape, w, args, local)
+        if name == "8b_hybrid":
+            for mode in ("standard", "ladder", "parallel"):
+                out[f"{name}_all_{mode}"] = short_run(B, torch, synth, shape.as_mode(mode), w, args, local)
+        del w
+        torch.cuda.empty_cache()
+    base = synth.SHAPES["tp_slice"]
+    w = synth.make_weights(base, device="cuda")
+    for mode in ("ladder", "standard", "parallel"):
+        for b in (1, 4, 16, 64):
+            shape = synth.replace(base.as_mode(mode), batch=b)
+            out[f"tp_slice_b{b}_{mode}"] = short_run(B, torch, synth, shape, w, args, local, noise_kv=True)
+    del w
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_rank(args, rank, world):
+    import numpy as np  # noqa: F401
     import torch
     from paper_2501_06589_b200 import binding as B
     from paper_2501_06589_b200 import build, synth
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dist = None
@@ -245,93 +450,55 @@ def main():
         dist.barrier()
     B.lib()
 
-    shape = synth.SHAPES[args.config]
-    if args.batch:
-        shape = synth.replace(shape, batch=args.batch)
-    if args.standard:
-        shape = shape.as_standard()
+    shape = shape_for(args, synth)
     steps, warm = args.steps, max(args.warmup, 0)
     S, bsz = shape.prompt_len, shape.batch
-    max_seq = S + max(steps, warm)
     hbm_peak, bf16_peak, peak_src = measured_peaks()
 
     t0 = time.time()
     w = synth.make_weights(shape, device="cuda")
     torch.cuda.synchronize()
     t_gen = time.time() - t0
-    chunk = args.prefill_chunk if 0 < args.prefill_chunk < S else S
-    model = B.Model(w, bsz, max_seq, bsz * chunk)
     B.set_decode_wide_impl(args.wide_impl)
     B.set_prefill_gemm_impl(args.prefill_impl)
-    if args.multi_kernel:
-        model.set_persistent(False)
-    persistent = model.persistent_active() and bsz <= 8
-    if args.streams is not None or args.graph is not None or args.pdl is not None:
-        model.set_schedule(2 if args.streams is None else args.streams, 1 if args.graph is None else args.graph,
-                           1 if args.pdl is None else args.pdl)
-    cache = B.KVCache(shape, bsz, max_seq)
-    prompt = torch.from_numpy(synth.make_tokens(shape, bsz, S)).cuda()
-    nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
-    first = torch.zeros(bsz, dtype=torch.int32, device="cuda")
-
-    def sync_all():
-        torch.cuda.synchronize()
-        if dist:
-            dist.barrier()
-            torch.cuda.synchronize()
+    run = DecodeRun(B, torch, synth, shape, w, steps, warm, args, dist, local)
+    model, cache = run.model, run.cache
+    persistent = run.persistent
 
     # ---- prefill: once untimed (warm-up), once timed
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-    def run_prefill():
-        model.prefill(cache, prompt[:, :chunk].contiguous(), next_tokens=first)
-        for p0 in range(chunk, S, chunk):
-            model.prefill_append(cache, prompt[:, p0:min(S, p0 + chunk)].contiguous(), next_tokens=first)
-
-    run_prefill()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    run.prefill()
     torch.cuda.synchronize()
     prefill_ms = None
     if not args.no_prefill_timing:
         ev[0].record()
-        run_prefill()
+        run.prefill()
         ev[1].record()
         torch.cuda.synchronize()
         prefill_ms = ev[0].elapsed_time(ev[1])
 
-    def rewind():
-        cache.seq_lens.fill_(S)
-        model.set_position(S)
-        nxt.copy_(first)
-
-    # ---- decode: warm-up, then K timed steps (token fed back on the device, no host sync inside)
-    rewind()
-    for _ in range(warm):
-        model.decode_step(cache, nxt, next_tokens=nxt)
-    rewind()
-    sync_all()
-    launches0 = model.kernel_launches()
-    with ClockSampler(local) as clocks:
-        ev[2].record()
-        for _ in range(steps):
-            model.decode_step(cache, nxt, next_tokens=nxt)
-        ev[3].record()
-        sync_all()
-    dev_ms = ev[2].elapsed_time(ev[3])
-    launches = model.kernel_launches() - launches0
+    # ---- decode: warm-up, then K timed steps (token fed back on the device, no host sync inside), `repeats` times
+    run.warm_up()
+    dev_ms, dev_recs, launches = median_loop(run, args.repeats)
     status = model.device_status()
 
-    # ---- end to end: host token buffers in, host tokens out, every step (pinned memory)
-    rewind()
-    h_in = first.cpu().pin_memory()
+    # ---- end to end: host token buffers in, host tokens out, every step (pinned memory); same number of repeats
+    h_in = run.first.cpu().pin_memory()
     h_out = torch.zeros(bsz, dtype=torch.int32).pin_memory()
+    run.rewind()
     model.decode_step_host(cache, h_in, h_out)      # untimed: captures the graph for the staging buffers
-    rewind()
-    sync_all()
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        model.decode_step_host(cache, h_in, h_out)
-        h_in.copy_(h_out)
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
+    e2e_recs = []
+    for _ in range(max(1, args.repeats)):
+        run.rewind()
+        h_in.copy_(run.first.cpu())
+        run.sync_all()
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            model.decode_step_host(cache, h_in, h_out)
+            h_in.copy_(h_out)
+        torch.cuda.synchronize()
+        e2e_recs.append(max_over_ranks([(time.perf_counter() - t0) * 1e3], dist, "cuda")[0])
+    e2e_ms = statistics.median(e2e_recs)
 
     # ---- dominant kernel alone: the gate/up weight-streaming GEMM over every layer's weights
     x_act = torch.randn(bsz, shape.d_model, device="cuda")
@@ -350,28 +517,38 @@ def main():
     k_bytes = 2.0 * 2 * shape.d_ff * shape.d_model
     k_gbs = k_bytes / (k_ms * 1e-3) / 1e9
 
-    # ---- reduce over ranks (max time), aggregate value
-    dev_ms, e2e_ms, prefill_ms_max = max_over_ranks([dev_ms, e2e_s * 1e3, prefill_ms or 0.0], dist, "cuda")
+    prefill_ms_max = max_over_ranks([prefill_ms or 0.0], dist, "cuda")[0]
     ms_per_step = dev_ms / steps
     value = aggregate_rate(world, bsz, steps, dev_ms)
     e2e_value = aggregate_rate(world, bsz, steps, e2e_ms)
     mean_kv = S + (steps + 1) / 2.0
     step_bytes = shape.decode_step_bytes(mean_kv)
     step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    mhz, reasons = merged_clocks(dev_recs)
+    sm_max = None
+    with ClockSampler(local) as probe:      # the clock limit itself (idle sample)
+        time.sleep(0.5)
+    sm_max = probe.summary()["sm_max_mhz"]
 
+    traffic = ncu_traffic()
     line = {
         "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps,
         "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(shape, args),
-        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": 4 * bsz, "d2h_bytes_per_step": 4 * bsz},
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": 4 * bsz, "d2h_bytes_per_step": 4 * bsz,
+                "repeat_ms": [round(x, 3) for x in e2e_recs]},
         "gpu_launches": int(launches),
+        "repeats": {"n": len(dev_recs), "statistic": "median", "ms": [round(r["ms"], 3) for r in dev_recs],
+                    "sm_mhz": [r["sm_mhz"] for r in dev_recs]},
         "roofline": {"bound": "hbm", "kernel": "smallm_gemm (RMSNorm + gate/up projection + SwiGLU)",
                      "achieved": k_gbs, "peak": hbm_peak, "peak_source": peak_src, "unit": "GB/s",
-                     "frac": k_gbs / hbm_peak, "bytes_per_launch": k_bytes, "ms_per_launch": k_ms, "traffic": None},
+                     "frac": k_gbs / hbm_peak, "bytes_per_launch": k_bytes, "ms_per_launch": k_ms,
+                     "traffic": traffic.get((shape.name, bsz, "decode_gemm_gate_up_bytes"))},
         "step_roofline": {"bytes_per_step": step_bytes, "achieved_gbs": step_gbs,
                           "frac_of_measured_copy_peak": step_gbs / hbm_peak,
                           "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS, "mean_kv_len": mean_kv},
-        "clocks": clocks.summary(),
+        "clocks": {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": sm_max, "reasons": reasons,
+                   "samples": sum(r["samples"] for r in dev_recs)},
         "device_status": status,
         "schedule": {"persistent": persistent, "streams": args.streams, "graph": args.graph, "pdl": args.pdl},
         "weights_gb": w.nbytes() / 1e9, "weight_gen_s": t_gen,
@@ -381,29 +558,49 @@ def main():
         line["prefill"] = {"tokens_per_s": world * bsz * S / (prefill_ms_max * 1e-3), "ms": prefill_ms_max,
                            "tflops": flops / (prefill_ms_max * 1e-3) / 1e12,
                            "frac_of_bf16_peak": flops / (prefill_ms_max * 1e-3) / 1e12 / bf16_peak,
-                           "activations": {0: "bf16 hi+lo pair (2 MMAs per product)", 1: "bf16 hi+lo pair, mma.sync kernel",
-                                           2: "single bf16"}[args.prefill_impl],
+                           "impl": args.prefill_impl,
                            "peak_tflops": bf16_peak, "peak_source": peak_src}
-    if (shape.name, bsz) in NCU_TRAFFIC_BYTES:
-        line["roofline"]["traffic"] = NCU_TRAFFIC_BYTES[(shape.name, bsz)]
     if persistent:
         # One launch of the persistent kernel IS the decode step (the embedding gather, the counter reset
         # and the argmax around it take ~10 us), so the step's device time is its launch duration.
         line["gemm_kernel"] = line["roofline"]
-        ratio = NCU_STACK_TRAFFIC_RATIO.get((shape.name, bsz))
+        ratio = traffic.get((shape.name, bsz, "decode_stack_traffic_ratio"))
         line["roofline"] = {
             "bound": "hbm", "kernel": "decode_stack_kernel (every GEMM and the attention of a decode step, one launch)",
             "achieved": step_gbs, "peak": hbm_peak, "peak_source": peak_src, "unit": "GB/s",
             "frac": step_gbs / hbm_peak, "bytes_per_launch": step_bytes, "ms_per_launch": ms_per_step,
             "traffic": None if ratio is None else step_bytes * ratio}
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    solo = rank == 0 and world == 1
+    if solo and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(shape, w, S)
+    run.close()
+    del run, model, cache
+    if solo and not args.no_other_configs and args.config == "70b" and args.mode is None and not args.standard:
+        t0 = time.time()
+        others = other_configs(B, torch, synth, args, local, w, shape)
+        del w
+        torch.cuda.empty_cache()
+        others.update(other_configs_small(B, torch, synth, args, local))
+        line["other_configs"] = others
+        line["other_configs_s"] = round(time.time() - t0, 1)
     if rank == 0:
         print(json.dumps(line))
-    model.close()
     if dist:
         dist.destroy_process_group()
     return 0
+
+
+def ncu_traffic():
+    """DRAM traffic figures taken from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum), kept as data
+    beside the capture summaries: lines of `config batch key value`."""
+    out = {}
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.txt")
+    if os.path.exists(path):
+        for ln in open(path):
+            f = ln.split()
+            if len(f) == 4 and not ln.startswith("#"):
+                out[(f[0], int(f[1]), f[2])] = float(f[3])
+    return out
 
 
 def max_over_ranks(values, dist, device):

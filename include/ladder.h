@@ -47,12 +47,24 @@ typedef enum {
   LADDER_ERR_UNSUPPORTED = 2, /* shape outside what the kernels handle (see create)    */
   LADDER_ERR_OOM = 3,         /* workspace allocation failed                           */
   LADDER_ERR_CUDA = 4,        /* a CUDA call failed (sticky; see ladder_last_error)    */
-  LADDER_ERR_STATE = 5        /* cache overflow, batch > max_batch, prefill on a non-empty position */
+  LADDER_ERR_STATE = 5,       /* cache overflow, batch > max_batch, prefill on a non-empty position */
+  LADDER_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out in an earlier step (see ladder_device_status) */
 } ladder_status_t;
 
 /* Bits of the device status word (ladder_device_status). */
 #define LADDER_DEV_BAD_TOKEN 1      /* a token id was outside [0, vocab): row treated as id 0 */
 #define LADDER_DEV_CACHE_OVERFLOW 2 /* a position >= max_seq_len reached a kernel: store skipped */
+#define LADDER_DEV_TIMEOUT 4        /* a bounded wait inside the persistent decode kernel gave up (0.25 s): that
+                                       step's outputs are invalid; later launches end at once until the word is read */
+
+/* Per-layer architecture (ladder_config_t.layer_mode), paper Sec. 3.3.1. */
+#define LADDER_LAYER_STANDARD 0    /* x_m = x_{m-1} + h_m(x_{m-1})                           (Sec. 2, Eq. 1)   */
+#define LADDER_LAYER_LADDER 1      /* x_m = x_{m-1} + h_m(x_{m-2})                           (Sec. 3.1, Eq. 2) */
+#define LADDER_LAYER_PARALLEL 2    /* parallel attention and MLP: both modules read the layer's input through ONE
+                                      RMSNorm (the attention gain; mlp_norm of the layer is unused) and both
+                                      outputs are added: x_l = x_{l-1} + Attn(n) + MLP(n), n = Norm(x_{l-1})     */
+#define LADDER_LAYER_UPPER_BOUND 3 /* the communication-free upper bound: the standard model with the all-reduce
+                                      deleted, which on one device is the standard model (alias of 0)           */
 
 typedef struct {
   uint32_t struct_size; /* sizeof(ladder_config_t), for ABI versioning */
@@ -62,8 +74,18 @@ typedef struct {
   int32_t max_seq_len;      /* cache capacity per sequence (prompt + generated)           */
   int32_t max_prefill_tokens; /* largest batch*seq_len of a prefill call; 0 = max_batch*max_seq_len */
   const uint8_t* layer_is_ladder; /* HOST, n_layers bytes, copied. NULL = all ladder; 0 = standard layer */
+  /* -- appended fields: a caller may pass struct_size = offsetof(ladder_config_t, layer_mode) and omit them -- */
+  const uint8_t* layer_mode;      /* HOST, n_layers bytes of LADDER_LAYER_*, copied; NULL = use layer_is_ladder */
+  const uint8_t* module_stale;    /* HOST, 2*n_layers bytes, copied; NULL = what the layer modes imply.  Entry m-1
+                                     non-zero: module m (1-based; odd = attention, even = MLP) reads x_{m-2}
+                                     instead of x_{m-1}.  Module 1 reads x_0 whatever its entry.  Implied rule:
+                                     ladder layer 1,1 except that the attention of a ladder layer directly after
+                                     a non-ladder layer reads the complete stream (0); standard 0,0; parallel 0,1.
+                                     States any other rule module by module, e.g. the hybrid in which the first
+                                     ladder attention also skips the preceding MLP's output. */
 } ladder_config_t;
-/* Shape limits (else LADDER_ERR_UNSUPPORTED): head_dim 64 or 128; n_q_heads % n_kv_heads == 0;
+/* Shape limits (else LADDER_ERR_UNSUPPORTED): max_seq_len <= 65536 (the decode attention merges at most 1024
+ * splits of 64 keys); head_dim 64 or 128; n_q_heads % n_kv_heads == 0;
  * d_model, n_q_heads*head_dim and d_ff multiples of 8; (n_q_heads+2 n_kv_heads)*head_dim,
  * 2*d_ff, d_model and vocab_size multiples of 8. */
 
@@ -98,7 +120,9 @@ typedef struct {
   float* all_hidden;    /* prefill only: [batch, seq_len, d_model] final RMSNorm at every position */
 } ladder_outputs_t;
 
-/* Bytes of ONE of the two cache buffers (k or v) for this configuration. */
+/* Bytes of ONE of the two cache buffers (k or v) for this configuration.  The paper never names the cache; it is
+ * implied by its "prefill and decode phase" (Sec. 3.2): keys (after rotation) and values of every layer, kept so
+ * that a decode step attends to all earlier positions without recomputing them. */
 size_t ladder_kv_cache_bytes(const ladder_config_t* cfg);
 
 /* Validates the configuration, allocates the workspace (two fp32 residual buffers of
@@ -136,7 +160,7 @@ int32_t ladder_model_persistent_active(const ladder_model_t* m);
 
 /* Test hook for the bounded waits of the persistent kernel: with on = 1 the LM-head phase of the next decode
  * steps waits for one more finished unit than its producer phase has, i.e. for a count that is never reached.
- * Nothing faults or spins forever: the wait gives up after 0.25 s, sets the LADDER_DEV_TIMEOUT bit (4) of the
+ * Nothing faults or spins forever: the wait gives up after 0.25 s, sets the LADDER_DEV_TIMEOUT bit of the
  * device status word, every other wait in the launch gives up as soon as it sees the bit, and the launch ends.
  * Later launches return at once until ladder_device_status has read and cleared the word.  on = 0 restores
  * the real dependency. */
@@ -160,7 +184,9 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
  * SMs for the attention module's GEMMs and the rest for the MLP's.  Results are bit-identical. */
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream);
 
-/* Prompt pass.  d_tokens int32 [batch, seq_len]; every sequence has the same length.
+/* Prompt pass ("prefill phase", paper Sec. 3.2): the module chain of Eq. 1 / Eq. 2 (in the pending-output form of
+ * Algorithm 1 with the all-reduce removed) over all prompt positions at once, causal attention within the prompt.
+ * d_tokens int32 [batch, seq_len]; every sequence has the same length.
  * Writes cache rows 0..seq_len-1 of sequences 0..batch-1, sets seq_lens[b] = seq_len, and
  * produces outputs for position seq_len-1 (next_tokens = the first generated token).
  * batch*seq_len <= max_prefill_tokens, seq_len <= max_seq_len, else LADDER_ERR_STATE. */
@@ -178,11 +204,15 @@ ladder_status_t ladder_prefill(ladder_model_t* m, const ladder_kv_cache_t* cache
 ladder_status_t ladder_prefill_append(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
                                       int32_t batch, int32_t seq_len, const ladder_outputs_t* out, void* cuda_stream);
 
-/* One autoregressive step: consumes d_tokens int32 [batch] at position seq_lens[b] (read on
+/* One autoregressive step ("decode phase", paper Sec. 3.2; the workload of Sec. 3.3.1 is 512 of them after a
+ * 1024-token prompt): the same module chain (Eq. 1 / Eq. 2, Algorithm 1) for one new position per sequence.
+ * Consumes d_tokens int32 [batch] at position seq_lens[b] (read on
  * the device), appends K/V there, attends over positions 0..seq_lens[b], writes the outputs and
  * adds one to seq_lens[b].  d_tokens may alias out->next_tokens (device-side feedback loop).
  * The library tracks the common length on the host (set by prefill / ladder_set_position) and
- * returns LADDER_ERR_STATE instead of overflowing the cache. */
+ * returns LADDER_ERR_STATE instead of overflowing the cache.  After ladder_device_status has reported
+ * LADDER_DEV_TIMEOUT the model refuses further steps with LADDER_ERR_TIMEOUT (the step that timed out produced
+ * nothing and the cache position is unknown) until ladder_set_position or a new ladder_prefill re-arms it. */
 ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
                                    int32_t batch, const ladder_outputs_t* out, void* cuda_stream);
 
@@ -203,7 +233,8 @@ ladder_status_t ladder_prefill_host(ladder_model_t* m, const ladder_kv_cache_t* 
  * entry b, then call this with the LONGEST length and decode all sequences together. */
 ladder_status_t ladder_set_position(ladder_model_t* m, int32_t len);
 
-/* Synchronises `cuda_stream`, returns the device status word (LADDER_DEV_* bits) and clears it. */
+/* Synchronises `cuda_stream`, returns the device status word (LADDER_DEV_* bits) and clears it.  Returns
+ * LADDER_ERR_TIMEOUT (with *flags filled in) when the word holds LADDER_DEV_TIMEOUT. */
 ladder_status_t ladder_device_status(ladder_model_t* m, int32_t* flags, void* cuda_stream);
 
 /* Number of kernels this model has enqueued so far (graph replays count their kernel nodes). */
@@ -238,7 +269,9 @@ ladder_status_t ladder_op_smallm_gemm(const void* W, int32_t N, int32_t K, const
  *   q fp32 [batch, Hq*Dh] (already rotated); k,v bf16 [max_batch][Hkv][max_seq_len][Dh] (one layer);
  *   kv_len int32 [batch] = number of keys to attend (positions 0..kv_len-1);
  *   scratch fp32, at least ladder_decode_attention_scratch_bytes(...) bytes;
- *   o fp32 [batch, Hq*Dh].  softmax(q.k/sqrt(Dh)) v per head, fp32 softmax and accumulation. */
+ *   o fp32 [batch, Hq*Dh].  softmax(q.k/sqrt(Dh)) v per head, fp32 softmax and accumulation.
+ * q, k, v, o and scratch must be 16-byte aligned (the kernel uses 16-byte loads), else LADDER_ERR_INVALID_ARG;
+ * max_seq_len <= 65536, else LADDER_ERR_UNSUPPORTED.  The same two checks apply to the variant below. */
 size_t ladder_decode_attention_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim, int32_t max_seq_len);
 ladder_status_t ladder_op_decode_attention(const float* q, const void* k, const void* v, const int32_t* kv_len,
                                            int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,

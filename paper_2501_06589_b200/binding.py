@@ -40,7 +40,11 @@ class ladder_config_t(C.Structure):
                 ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("d_ff", C.c_int32), ("vocab_size", C.c_int32), ("rms_eps", C.c_float),
                 ("rope_theta", C.c_float), ("max_batch", C.c_int32), ("max_seq_len", C.c_int32),
-                ("max_prefill_tokens", C.c_int32), ("layer_is_ladder", C.POINTER(C.c_uint8))]
+                ("max_prefill_tokens", C.c_int32), ("layer_is_ladder", C.POINTER(C.c_uint8)),
+                ("layer_mode", C.POINTER(C.c_uint8)), ("module_stale", C.POINTER(C.c_uint8))]
+
+
+LAYER_MODES = {"standard": 0, "ladder": 1, "parallel": 2, "upper_bound": 3}      # LADDER_LAYER_*
 
 
 class ladder_weights_t(C.Structure):
@@ -144,11 +148,18 @@ def _check(status: int, model=None):
 
 def make_config(shape: ModelShape, max_batch: int, max_seq_len: int, max_prefill_tokens: int = 0):
     mask = (C.c_uint8 * shape.n_layers)(*shape.ladder_mask())
+    modes = flags = None
+    if shape.layer_mode is not None:
+        modes = (C.c_uint8 * shape.n_layers)(*[LAYER_MODES[m] for m in shape.layer_mode])
+    if shape.module_stale is not None:
+        flags = (C.c_uint8 * (2 * shape.n_layers))(*[int(bool(f)) for f in shape.module_stale])
+    u8p = C.POINTER(C.c_uint8)
     cfg = ladder_config_t(C.sizeof(ladder_config_t), shape.d_model, shape.n_layers, shape.n_q_heads,
                           shape.n_kv_heads, shape.head_dim, shape.d_ff, shape.vocab_size, shape.rms_eps,
                           shape.rope_theta, max_batch, max_seq_len, max_prefill_tokens,
-                          C.cast(mask, C.POINTER(C.c_uint8)))
-    cfg._keep = mask
+                          C.cast(mask, u8p), C.cast(modes, u8p) if modes is not None else None,
+                          C.cast(flags, u8p) if flags is not None else None)
+    cfg._keep = (mask, modes, flags)
     return cfg
 
 
@@ -263,8 +274,12 @@ class Model:
         _check(lib().ladder_set_position(self.h, length), self.h)
 
     def device_status(self) -> int:
+        """The LADDER_DEV_* bits, read and cleared.  A timeout bit comes back as a value, not as an exception
+        (the C call returns LADDER_ERR_TIMEOUT with the word filled in); the steps after it raise."""
         f = C.c_int32(0)
-        _check(lib().ladder_device_status(self.h, C.byref(f), _stream()), self.h)
+        st = lib().ladder_device_status(self.h, C.byref(f), _stream())
+        if st != 6:
+            _check(st, self.h)
         return f.value
 
     def kernel_launches(self) -> int:

@@ -18,6 +18,20 @@ namespace {
 
 thread_local std::string g_create_error;
 
+// sizeof(ladder_config_t) before layer_mode / module_stale were appended
+constexpr size_t kConfigSizeV1 = offsetof(ladder_config_t, layer_mode);
+
+// Copies the caller's configuration (of either size) and drops its host pointers: the rule tables are parsed
+// into the model once.
+void copy_config(ladder_config_t* dst, const ladder_config_t* src) {
+  memset(dst, 0, sizeof(*dst));
+  memcpy(dst, src, src->struct_size < sizeof(*dst) ? src->struct_size : sizeof(*dst));
+  dst->struct_size = sizeof(*dst);
+  dst->layer_is_ladder = nullptr;
+  dst->layer_mode = nullptr;
+  dst->module_stale = nullptr;
+}
+
 bool g_kernels_ready = false;
 cudaError_t kernels_ready() {  // opt-in to large dynamic shared memory, once per process
   if (g_kernels_ready) return cudaSuccess;
@@ -43,7 +57,9 @@ struct GraphKey {
 
 struct ladder_model {
   ladder_config_t cfg;
-  std::vector<uint8_t> is_ladder;
+  std::vector<uint8_t> is_ladder;  // per layer: a ladder layer (both modules read one module back)
+  std::vector<uint8_t> mode;       // per layer: LADDER_LAYER_*
+  std::vector<uint8_t> stale;      // per module (index m-1): module m reads x_{m-2} instead of x_{m-1}
   const __nv_bfloat16 *tok_embedding, *final_norm, *lm_head;
   std::vector<const __nv_bfloat16*> attn_norm, w_qkv, w_o, mlp_norm, w_gate_up, w_down;
   int sm_count = 0;
@@ -95,6 +111,7 @@ struct ladder_model {
   int n_phases = 0, n_attn = 0, n_counters = 0, cap_counters = 0;
   // state
   int host_len = 0;
+  bool timed_out = false;  // ladder_device_status saw LADDER_DEV_TIMEOUT: steps are refused until re-armed
   int64_t launches = 0;
   std::string err;
   bool sticky_cuda = false;
@@ -130,25 +147,28 @@ const char* check_shape(const ladder_config_t& c) {
   if (c.d_model % 8 || c.d_ff % 8 || c.vocab_size % 8) return "d_model, d_ff and vocab_size must be multiples of 8";
   if (c.max_batch < 1 || c.max_batch > 64) return "max_batch must be in [1, 64]";
   if (c.max_seq_len < 1) return "max_seq_len must be positive";
+  if (c.max_seq_len > kDecodeAttnMaxKeys) return "max_seq_len above 65536 (decode attention merges at most 1024 splits of 64 keys)";
   if (!(c.rms_eps >= 0.f) || !(c.rope_theta > 0.f)) return "bad rms_eps / rope_theta";
   return nullptr;
 }
 
-// Residual routing (Eq. 1 / Eq. 2 of the paper on two ping-pong buffers).
+// Residual routing (Eq. 1 / Eq. 2 of the paper on two ping-pong buffers).  Module m reads x_{m-2} (reads_older)
+// or x_{m-1}, adds onto x_{m-1} and writes x_m: over the buffer of x_{m-2}, which is dead from then on, or -- when
+// it read x_{m-1} and the next module does not need that value any more -- in place.
 struct Router {
   int cur = 0, stale = -1;  // buffer holding x_{m-1}; buffer holding x_{m-2} (or -1)
   int writer[2] = {0, -1};  // module that last wrote each buffer
   struct Route {
     int in, add, dst, in_writer;
   };
-  Route next(bool ladder, int module) {
+  Route next(bool reads_older, bool next_reads_older, int module) {
     Route r;
-    if (ladder && stale >= 0) {
+    if (reads_older && stale >= 0) {
       r = {stale, cur, stale, writer[stale]};
       const int old_cur = cur;
       cur = stale;
       stale = old_cur;
-    } else if (ladder) {
+    } else if (next_reads_older) {  // reads x_{m-1}, which module m+1 will read too: keep it
       r = {cur, cur, cur ^ 1, writer[cur]};
       stale = cur;
       cur ^= 1;
@@ -160,6 +180,48 @@ struct Router {
     return r;
   }
 };
+
+// Route of module `module` (1-based) of this model.
+Router::Route route(const ladder_model* m, Router& rt, int module) {
+  const int n = static_cast<int>(m->stale.size());
+  return rt.next(m->stale[module - 1] != 0, module < n && m->stale[module] != 0, module);
+}
+
+// Gain of the RMSNorm in front of the MLP of layer l: a parallel layer normalises once, with the attention gain.
+const __nv_bfloat16* mlp_gain(const ladder_model* m, int l) {
+  return m->mode[l] == LADDER_LAYER_PARALLEL ? m->attn_norm[l] : m->mlp_norm[l];
+}
+
+// Fills the per-layer / per-module rule tables from the configuration.  Fields past cfg->struct_size are absent
+// (a caller compiled against the earlier, shorter struct).
+const char* parse_rules(const ladder_config_t* cfg, ladder_model* m) {
+  const int L = cfg->n_layers;
+  const bool has_ext = cfg->struct_size >= sizeof(ladder_config_t);
+  m->mode.assign(L, LADDER_LAYER_LADDER);
+  if (cfg->layer_is_ladder)
+    for (int l = 0; l < L; ++l) m->mode[l] = cfg->layer_is_ladder[l] ? LADDER_LAYER_LADDER : LADDER_LAYER_STANDARD;
+  if (has_ext && cfg->layer_mode)
+    for (int l = 0; l < L; ++l) {
+      if (cfg->layer_mode[l] > LADDER_LAYER_UPPER_BOUND) return "layer_mode entry outside 0..3";
+      // without communication the upper bound is the standard model
+      m->mode[l] = cfg->layer_mode[l] == LADDER_LAYER_UPPER_BOUND ? LADDER_LAYER_STANDARD : cfg->layer_mode[l];
+    }
+  m->is_ladder.assign(L, 0);
+  m->stale.assign(2 * L, 0);
+  for (int l = 0; l < L; ++l) {
+    const bool after_ladder = l > 0 && m->mode[l - 1] == LADDER_LAYER_LADDER;
+    if (m->mode[l] == LADDER_LAYER_LADDER) {
+      m->is_ladder[l] = 1;
+      m->stale[2 * l] = (after_ladder || l == 0) ? 1 : 0;  // after a non-ladder layer: the complete stream
+      m->stale[2 * l + 1] = 1;
+    } else if (m->mode[l] == LADDER_LAYER_PARALLEL) {
+      m->stale[2 * l + 1] = 1;  // the MLP reads the attention module's input
+    }
+  }
+  if (has_ext && cfg->module_stale)
+    for (int i = 0; i < 2 * L; ++i) m->stale[i] = cfg->module_stale[i] ? 1 : 0;
+  return nullptr;
+}
 
 struct Enqueue {
   ladder_model* m;
@@ -251,7 +313,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
     // ---------------- attention module (module index 2l+1) on stream A
     {
       const int mod = 2 * l + 1;
-      const Router::Route r = rt.next(lad, mod);
+      const Router::Route r = route(m, rt, mod);
       need(0, r.in_writer);
       SmallMParams p = {};
       p.W = m->w_qkv[l];
@@ -317,7 +379,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
     // ---------------- MLP module (module index 2l+2) on stream B
     {
       const int mod = 2 * l + 2;
-      const Router::Route r = rt.next(lad, mod);
+      const Router::Route r = route(m, rt, mod);
       need(1, r.in_writer);
       if (q.two && !b_joined) {  // first use of sB in this step: order it after the embedding
         q.wait(1, m->ev[0]);
@@ -329,7 +391,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       p.K = d;
       p.act = m->R[r.in];
       p.act_mode = ACT_F32_NORM;
-      p.gain = m->mlp_norm[l];
+      p.gain = mlp_gain(m, l);
       p.eps = c.rms_eps;
       p.batch = batch;
       p.epi_mode = EPI_SWIGLU;
@@ -409,9 +471,8 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
   __nv_bfloat16* const h_lo = split ? m->h_pf + m->h_lo : nullptr;
   Router rt;
   for (int l = 0; l < c.n_layers; ++l) {
-    const bool lad = m->is_ladder[l] != 0;
     {
-      const Router::Route r = rt.next(lad, 2 * l + 1);
+      const Router::Route r = route(m, rt, 2 * l + 1);
       did(launch_rmsnorm_bf16(m->R[r.in], m->attn_norm[l], c.rms_eps, M, d, m->n_pf, n_lo, st));
       LargeMParams p = {};
       p.A = m->n_pf;
@@ -450,8 +511,8 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       did(launch_largem_gemm(o, st));
     }
     {
-      const Router::Route r = rt.next(lad, 2 * l + 2);
-      did(launch_rmsnorm_bf16(m->R[r.in], m->mlp_norm[l], c.rms_eps, M, d, m->n_pf, n_lo, st));
+      const Router::Route r = route(m, rt, 2 * l + 2);
+      did(launch_rmsnorm_bf16(m->R[r.in], mlp_gain(m, l), c.rms_eps, M, d, m->n_pf, n_lo, st));
       LargeMParams p = {};
       p.A = m->n_pf;
       p.A_lo = n_lo;
@@ -617,6 +678,8 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
             w.pack_out = tw->second;
             w.pack_gain = want_gain;
             P.act_packed = tw->second;
+          } else if (w.pack_out == tw->second && w.pack_gain == want_gain) {
+            P.act_packed = tw->second;  // a second reader with the same gain (parallel layer: QKV and gate/up)
           }
         } else {
           StackAttn& w = attn[wr->second.second];
@@ -668,9 +731,8 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
   Router rt;
   int prev_merge = -1;
   for (int l = 0; l < c.n_layers; ++l) {
-    const bool lad = m->is_ladder[l] != 0;
-    const Router::Route ra = rt.next(lad, 2 * l + 1);
-    const Router::Route rm = rt.next(lad, 2 * l + 2);
+    const Router::Route ra = route(m, rt, 2 * l + 1);
+    const Router::Route rm = route(m, rt, 2 * l + 2);
     if (l < l_begin) continue;  // run by separate kernels before the launch: only the routing state matters
     cur_layer = l;
     __nv_bfloat16* kc = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
@@ -749,7 +811,7 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
       p.K = d;
       p.act = m->R[rm.in];
       p.act_mode = ACT_F32_NORM;
-      p.gain = m->mlp_norm[l];
+      p.gain = mlp_gain(m, l);
       p.eps = c.rms_eps;
       p.epi_mode = EPI_SWIGLU;
       p.out = m->h_dec;
@@ -767,10 +829,10 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
       p.out = m->R[rm.dst];
       add_gemm(3, p, m->h_dec, m->R[rm.add], m->R[rm.dst], nullptr, nullptr);
     };
-    // The MLP module of a ladder layer reads x_{m-2}, which exists before the attention module of the
-    // same layer has produced anything -- unless this is the first ladder layer after a standard one,
-    // where x_{m-2} is the attention module's own input (still fine: it is not its output).
-    const bool mlp_independent = lad && rm.in != ra.dst;
+    // An MLP module that reads x_{m-2} (ladder layer, parallel layer) reads a value that exists before the
+    // attention module of the same layer has produced anything (in the first ladder layer after a standard
+    // one and in a parallel layer it is the attention module's own input: still not its output).
+    const bool mlp_independent = m->stale[2 * l + 1] != 0 && rm.in != ra.dst;
     qkv();
     if (mlp_independent) {
       gate_up();
@@ -827,10 +889,7 @@ cudaError_t enqueue_decode_stack(ladder_model* m, const ladder_kv_cache_t* cache
   if (e == cudaSuccess) e = launch_decode_stack(sp, m->sm_count, st);
   // the final hidden state is the input of the last phase (the LM head)
   Router rt;
-  for (int l = 0; l < c.n_layers; ++l) {
-    rt.next(m->is_ladder[l] != 0, 2 * l + 1);
-    rt.next(m->is_ladder[l] != 0, 2 * l + 2);
-  }
+  for (int mod = 1; mod <= 2 * c.n_layers; ++mod) route(m, rt, mod);
   if (out && out->final_hidden) {
     if (e == cudaSuccess)
       e = launch_rmsnorm_f32(m->R[rt.cur], m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, st, false);
@@ -863,6 +922,7 @@ const char* ladder_status_string(ladder_status_t s) {
     case LADDER_ERR_OOM: return "out of device memory";
     case LADDER_ERR_CUDA: return "CUDA error";
     case LADDER_ERR_STATE: return "invalid state (cache overflow / batch too large)";
+    case LADDER_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     default: return "unknown status";
   }
 }
@@ -881,18 +941,19 @@ size_t ladder_kv_cache_bytes(const ladder_config_t* c) {
 ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_weights_t* w, ladder_model_t** out) {
   if (out) *out = nullptr;
   if (!cfg || !w || !out) return fail(nullptr, LADDER_ERR_INVALID_ARG, "NULL argument");
-  if (cfg->struct_size != sizeof(ladder_config_t)) return fail(nullptr, LADDER_ERR_INVALID_ARG, "struct_size mismatch");
+  if (cfg->struct_size != sizeof(ladder_config_t) && cfg->struct_size != kConfigSizeV1)
+    return fail(nullptr, LADDER_ERR_INVALID_ARG, "struct_size mismatch");
   if (const char* why = check_shape(*cfg)) return fail(nullptr, LADDER_ERR_UNSUPPORTED, why);
   if (!w->tok_embedding || !w->final_norm || !w->lm_head || !w->attn_norm || !w->w_qkv || !w->w_o || !w->mlp_norm ||
       !w->w_gate_up || !w->w_down)
     return fail(nullptr, LADDER_ERR_INVALID_ARG, "NULL weight pointer");
   ladder_model* m = new ladder_model();
-  m->cfg = *cfg;
-  m->cfg.layer_is_ladder = nullptr;
+  copy_config(&m->cfg, cfg);
   const int L = cfg->n_layers;
-  m->is_ladder.assign(L, 1);
-  if (cfg->layer_is_ladder)
-    for (int l = 0; l < L; ++l) m->is_ladder[l] = cfg->layer_is_ladder[l] ? 1 : 0;
+  if (const char* why = parse_rules(cfg, m)) {
+    delete m;
+    return fail(nullptr, LADDER_ERR_INVALID_ARG, why);
+  }
   m->tok_embedding = static_cast<const __nv_bfloat16*>(w->tok_embedding);
   m->final_norm = static_cast<const __nv_bfloat16*>(w->final_norm);
   m->lm_head = static_cast<const __nv_bfloat16*>(w->lm_head);
@@ -1098,6 +1159,7 @@ ladder_status_t ladder_set_position(ladder_model_t* m, int32_t len) {
   if (!m) return LADDER_ERR_INVALID_ARG;
   if (len < 0 || len > m->cfg.max_seq_len) return fail(m, LADDER_ERR_INVALID_ARG, "length outside [0, max_seq_len]");
   m->host_len = len;
+  m->timed_out = false;
   return LADDER_OK;
 }
 
@@ -1105,14 +1167,12 @@ int64_t ladder_kernel_launches(const ladder_model_t* m) { return m ? m->launches
 
 int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_count, int32_t* out, int32_t cap) {
   if (!cfg || !out || cap < 4 || batch < 1 || sm_count < 1) return -1;
-  if (cfg->struct_size != sizeof(ladder_config_t) || check_shape(*cfg)) return -1;
+  if ((cfg->struct_size != sizeof(ladder_config_t) && cfg->struct_size != kConfigSizeV1) || check_shape(*cfg)) return -1;
   // a model object that owns nothing: every buffer is a distinct made-up address, never dereferenced
   ladder_model m;
-  m.cfg = *cfg;
+  copy_config(&m.cfg, cfg);
   const int L = cfg->n_layers;
-  m.is_ladder.assign(L, 1);
-  if (cfg->layer_is_ladder)
-    for (int l = 0; l < L; ++l) m.is_ladder[l] = cfg->layer_is_ladder[l] ? 1 : 0;
+  if (parse_rules(cfg, &m)) return -1;
   m.sm_count = sm_count;
   m.attn_splits = decode_attention_splits(cfg->max_batch, cfg->n_kv_heads, cfg->max_seq_len, sm_count);
   uintptr_t next = 0x10000000u;
@@ -1180,13 +1240,26 @@ ladder_status_t ladder_device_status(ladder_model_t* m, int32_t* flags, void* cu
   CK(m, cudaStreamSynchronize(st));
   CK(m, cudaMemcpy(flags, m->status, sizeof(int32_t), cudaMemcpyDeviceToHost));
   CK(m, cudaMemset(m->status, 0, sizeof(int32_t)));
+  if (*flags & LADDER_DEV_TIMEOUT) {
+    m->timed_out = true;
+    return fail(m, LADDER_ERR_TIMEOUT, "a wait inside the persistent decode kernel gave up: that step produced nothing; "
+                                        "call ladder_set_position or ladder_prefill to continue");
+  }
   return LADDER_OK;
 }
 
-static ladder_status_t check_call(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* tokens, int batch) {
+static ladder_status_t check_call(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* tokens, int batch,
+                                  bool rearm = false) {
   if (!m) return LADDER_ERR_INVALID_ARG;
   if (m->sticky_cuda) return fail(m, LADDER_ERR_CUDA, "an earlier CUDA call failed: " + m->err);
+  if (rearm) m->timed_out = false;
+  if (m->timed_out)
+    return fail(m, LADDER_ERR_TIMEOUT, "an earlier step timed out on the device; call ladder_set_position or ladder_prefill");
   if (!cache || !cache->k || !cache->v || !cache->seq_lens || !tokens) return fail(m, LADDER_ERR_INVALID_ARG, "NULL argument");
+  if ((reinterpret_cast<uintptr_t>(cache->k) | reinterpret_cast<uintptr_t>(cache->v)) & 15)
+    return fail(m, LADDER_ERR_INVALID_ARG, "cache buffers must be 16-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(cache->seq_lens) | reinterpret_cast<uintptr_t>(tokens)) & 3)
+    return fail(m, LADDER_ERR_INVALID_ARG, "seq_lens / token buffers must be 4-byte aligned");
   if (batch < 1) return fail(m, LADDER_ERR_INVALID_ARG, "batch must be >= 1");
   if (batch > m->cfg.max_batch) return fail(m, LADDER_ERR_STATE, "batch exceeds max_batch");
   return LADDER_OK;
@@ -1194,7 +1267,7 @@ static ladder_status_t check_call(ladder_model_t* m, const ladder_kv_cache_t* ca
 
 ladder_status_t ladder_prefill(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int32_t batch,
                                int32_t seq_len, const ladder_outputs_t* out, void* cuda_stream) {
-  ladder_status_t s = check_call(m, cache, d_tokens, batch);
+  ladder_status_t s = check_call(m, cache, d_tokens, batch, /*rearm=*/true);
   if (s != LADDER_OK) return s;
   if (seq_len < 1) return fail(m, LADDER_ERR_INVALID_ARG, "seq_len must be >= 1");
   if (seq_len > m->cfg.max_seq_len) return fail(m, LADDER_ERR_STATE, "seq_len exceeds max_seq_len");
@@ -1437,6 +1510,8 @@ ladder_status_t ladder_op_decode_attention(const float* q, const void* k, const 
   if (!q || !k || !v || !kv_len || !scratch || !o) return LADDER_ERR_INVALID_ARG;
   if (batch < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads || (head_dim != 64 && head_dim != 128) || max_seq_len < 1)
     return LADDER_ERR_INVALID_ARG;
+  if (decode_attention_misaligned(q, k, v, o, scratch, kv_len)) return LADDER_ERR_INVALID_ARG;
+  if (max_seq_len > kDecodeAttnMaxKeys) return LADDER_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   DecodeAttnParams a = {};
   a.q = q;

@@ -408,6 +408,8 @@ extern "C" ladder_status_t ladder_op_decode_attention_noalloc(const float* q, co
   if (batch < 1 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || (head_dim != 64 && head_dim != 128) ||
       max_seq_len < 1)
     return LADDER_ERR_INVALID_ARG;
+  if (decode_attention_misaligned(q, k, v, o, nullptr, kv_len)) return LADDER_ERR_INVALID_ARG;
+  if (max_seq_len > kDecodeAttnMaxKeys) return LADDER_ERR_UNSUPPORTED;
   const int n_splits = decode_attention_splits(batch, n_kv_heads, max_seq_len, 0);
   if (decode_attention_scratch_floats(batch, n_q_heads, head_dim, n_splits) > kNoAllocScratchFloats)
     return LADDER_ERR_UNSUPPORTED;  // batch * heads * ceil(max_seq_len / 64) * (head_dim + 2) floats exceed 8 MiB

@@ -286,14 +286,6 @@ struct Split {
   }
 };
 
-// Tuning build (-DWIDE_TRACE): global-timer stamps per CTA at the hand-over points of the last launch.
-#ifdef WIDE_TRACE
-__device__ unsigned long long g_wide_trace[kWideMaxCtas][8];
-#define WIDE_STAMP(i) g_wide_trace[blockIdx.x][i] = global_timer_ns()
-#else
-#define WIDE_STAMP(i)
-#endif
-
 template <int NP>
 __global__ void __launch_bounds__(kWideThreads, 1)
 decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap map_w,
@@ -322,7 +314,6 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
   const int my_start = sp.start(blockIdx.x), my_end = sp.start(blockIdx.x + 1);
 
   if (tid == 0) {
-    WIDE_STAMP(0);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 1);
@@ -344,7 +335,6 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
   tc_fence_after();
   pdl_launch_dependents();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
-  if (tid == 0) WIDE_STAMP(1);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -361,7 +351,6 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
         tma_load_2d_hint(smem + i * C::STAGE_BYTES, &map_w, kb * BK, t * BM, &full[i], pol);
       }
       pdl_wait();
-      WIDE_STAMP(2);
       for (int i = 0; i < pre; ++i) {
         const int pos = my_start + i, kb = pos % nkb;
         tma_load_2d(smem + i * C::STAGE_BYTES + W_BYTES, &map_act, kb * BK, 0, &full[i]);
@@ -401,7 +390,6 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
           const int s = it % STAGES;
           ok = mbar_wait_bounded(&full[s], (it / STAGES) & 1);
           if (!ok) break;
-          if (it == 0) WIDE_STAMP(3);
           tc_fence_after();
           const uint32_t w_addr = smem_u32(smem + s * C::STAGE_BYTES);
           const uint64_t dw = smem_desc(w_addr), dact = smem_desc(w_addr + W_BYTES);
@@ -413,7 +401,6 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
         if (ok) tc_commit(&tmem_full[ab]);
         pos += kb1 - kb0;
       }
-      WIDE_STAMP(4);
       if (!ok && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
     }
   } else {
@@ -444,7 +431,6 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
       const int n = t * BM + r;
       ok = epi_bar_and(ok && mbar_wait_bounded(&tmem_full[ab], (seg >> 1) & 1));  // all eight warps agree
       if (!ok) break;
-      if (et == 0 && pos >= my_end) WIDE_STAMP(5);   // the last segment's accumulator is complete
       tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + ab * NP;
       // where this CTA's piece of a shared tile goes: slot 0 if the tile is the first of its range, else slot 1
@@ -511,7 +497,6 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
       const bool last = *last_flag != 0;
-      if (et == 0 && pos >= my_end) WIDE_STAMP(6);   // the last segment's piece is published
       asm volatile("bar.sync 1, 256;" ::: "memory");  // the flag is rewritten by the next shared tile
       if (!last) continue;
       __threadfence();
@@ -553,7 +538,6 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
         epi_apply<FB>(p, n, b0, v, lane, pos_s, pa, pb, BP);
       }
     }
-    if (et == 0) WIDE_STAMP(7);
     if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
   }
 
@@ -610,11 +594,6 @@ cudaError_t launch_np(const WideArgs& a, const CUtensorMap& mw, const CUtensorMa
 
 }  // namespace
 
-#ifdef WIDE_TRACE
-extern "C" int ladder_debug_read_wide_trace(unsigned long long* host_out) {
-  return static_cast<int>(cudaMemcpyFromSymbol(host_out, g_wide_trace, sizeof(g_wide_trace)));
-}
-#endif
 
 int wide_padded_batch(int batch) { return padded_batch(batch); }
 

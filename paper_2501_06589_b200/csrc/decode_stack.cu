@@ -169,28 +169,10 @@ __device__ __forceinline__ bool wait_deps(const int* dep, const int* need, int n
   return __all_sync(0xffffffffu, ok);
 }
 
-#ifdef DS_TRACE
-// tuning builds only: per CTA, cycles each role spent in its waits during the launch
-// [0] consumer total [1] c:queue [2] c:act_full [3] c:weights [4] c:red_free
-// [5] producer total [6] p:ring full [7] p:claims  [8] stager total [9] s:deps [10] s:act_free [11] s:queue
-// [12] finisher total [13] f:deps [14] f:red_full/norm [15] f:queue
-__device__ unsigned long long g_stack_trace[148 * 16];
-// consumer cycles per phase kind (phase index mod 4): [kind][0] weights wait [1] tile loop [2] act wait [3] all
-__device__ unsigned long long g_kind_trace[148 * 16];
-// consumer timeline: [phase][cta][0] first item of the phase taken up, [1] last item of the phase handed over (ns)
-__device__ unsigned long long g_phase_trace[330 * 148 * 2];
-// attention timeline of CTA 0: [layer][0] dependencies met [1] own split units done [2] all splits done [3] merge done (ns)
-__device__ unsigned long long g_attn_trace[128 * 4];
-#define TR_DECL(n) long long tr_##n = 0
-#define TR_T0() const long long tr_t0_ = clock64()
-#define TR_ADD(n) tr_##n += clock64() - tr_t0_
-#define TR_OUT(i, n) g_stack_trace[blockIdx.x * 16 + (i)] = static_cast<unsigned long long>(tr_##n)
-#else
 #define TR_DECL(n)
 #define TR_T0()
 #define TR_ADD(n)
 #define TR_OUT(i, n)
-#endif
 
 template <typename T>
 __device__ __forceinline__ T* ldg_ptr(T* const* p) {  // read-only load of a pointer field
@@ -535,9 +517,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       TR_DECL(ring);
       TR_DECL(claim);
       TR_DECL(total);
-#ifdef DS_TRACE
-      const long long tr_start = clock64();
-#endif
       // Which batch comes next is settled one batch ahead of the weight stream, right after the first
       // tile of the current batch has been issued, so the stagers and finishers know early and no
       // round trip of an atomic is exposed.  Whole rounds of a phase's schedule are dealt out
@@ -674,14 +653,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         __threadfence_block();
         *q_head = n + 1;
       }
-#ifdef DS_TRACE
-      tr_total = clock64() - tr_start;
-      if (lane == 0) {
-        TR_OUT(5, total);
-        TR_OUT(6, ring);
-        TR_OUT(7, claim);
-      }
-#endif
       if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
       if (!ok) {  // wait (bounded) for the copies in flight before the CTA may exit
         for (int j = 1; j <= STAGES && j <= it; ++j) {
@@ -702,9 +673,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
     TR_DECL(fred);
     TR_DECL(fq);
     TR_DECL(ftotal);
-#ifdef DS_TRACE
-    const long long tr_fstart = clock64();
-#endif
     for (int n = 0;; ++n) {
       {
         TR_T0();
@@ -772,15 +740,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       if (lane == 0) mbar_arrive(&red_free[slot]);
     }
     if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
-#ifdef DS_TRACE
-    tr_ftotal = clock64() - tr_fstart;
-    if (ft == 0) {
-      TR_OUT(12, ftotal);
-      TR_OUT(13, fdeps);
-      TR_OUT(14, fred);
-      TR_OUT(15, fq);
-    }
-#endif
     return;
   }
 
@@ -804,14 +763,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
     TR_DECL(cred);
     TR_DECL(cmma);
     TR_DECL(ctotal);
-#ifdef DS_TRACE
-    long long kind_cyc[4][4] = {};
-    long long kind_t0 = clock64();
-    int kind_cur = 0;
-#endif
-#ifdef DS_TRACE
-    const long long tr_cstart = clock64();
-#endif
     for (int n = 0;; ++n) {
       {
         TR_T0();
@@ -826,15 +777,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
         K = queue_k[n % QDEPTH];
         nchunk = queue_nc[n % QDEPTH];
         cur_ph = ph;
-#ifdef DS_TRACE
-        if (warp == 4 && lane == 0 && ph < 330) g_phase_trace[(ph * 148 + blockIdx.x) * 2] = global_timer_ns();
-        {
-          const long long now = clock64();
-          kind_cyc[kind_cur][3] += now - kind_t0;
-          kind_t0 = now;
-          kind_cur = ph & 3;
-        }
-#endif
       }
       const int rows = (id & 15) * 8;
       const int rgn = (rows + 15) >> 4;
@@ -854,9 +796,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
           TR_T0();
           ok = __all_sync(0xffffffffu, wait_mbar(act_full, n_req & 1, status));
           TR_ADD(cact);
-#ifdef DS_TRACE
-          kind_cyc[kind_cur][2] += clock64() - tr_t0_;
-#endif
         }
         if (!ok) break;
         ++n_req;
@@ -879,26 +818,16 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
             if (okw && hi_valid) okw = wait_mbar(&full[st1], ((it + 1) / STAGES) & 1, status);
             ok = __all_sync(0xffffffffu, okw);
             TR_ADD(cw);
-#ifdef DS_TRACE
-            kind_cyc[kind_cur][0] += clock64() - tr_t0_;
-#endif
           }
           if (!ok) break;
           const uint32_t base0 = ring_u32 + st0 * STAGE_BYTES + g * PITCH + tig * 16;
           const uint32_t base1 = ring_u32 + st1 * STAGE_BYTES + g * PITCH + tig * 16;
-#ifdef DS_TRACE
-          const long long tr_m0 = clock64();
-#endif
           // a full chunk with both 8-row halves present (the common case) takes the path without
           // predicates: a guarded shared-memory load compiles to a branch, and 64 of them per tile
           // cost more than the loads and MMAs themselves
           if (hi_valid && k0 + TK <= K) slab_loop<true>(acc[rgi][0], acc[rgi][1], bf, base0, base1, cw, k0, K, tig, true);
           else slab_loop<false>(acc[rgi][0], acc[rgi][1], bf, base0, base1, cw, k0, K, tig, hi_valid);
           __syncwarp();
-#ifdef DS_TRACE
-          tr_cmma += clock64() - tr_m0;
-          kind_cyc[kind_cur][1] += clock64() - tr_m0;
-#endif
           if (lane == 0) {
             mbar_arrive(&empty[st0]);
             if (hi_valid) mbar_arrive(&empty[st1]);
@@ -925,23 +854,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&red_full[slot]);
-#ifdef DS_TRACE
-      if (warp == 4 && lane == 0 && cur_ph < 330) g_phase_trace[(cur_ph * 148 + blockIdx.x) * 2 + 1] = global_timer_ns();
-#endif
     }
     if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
-#ifdef DS_TRACE
-    tr_ctotal = clock64() - tr_cstart;
-    if (warp == 4 && lane == 0) {
-      TR_OUT(0, ctotal);
-      TR_OUT(1, cq);
-      TR_OUT(2, cact);
-      TR_OUT(3, cw);
-      TR_OUT(4, cmma);
-      for (int k = 0; k < 4; ++k)
-        for (int j = 0; j < 4; ++j) g_kind_trace[blockIdx.x * 16 + k * 4 + j] = static_cast<unsigned long long>(kind_cyc[k][j]);
-    }
-#endif
     return;
   }
 
@@ -1055,9 +969,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
     TR_DECL(sfree);
     TR_DECL(sq);
     TR_DECL(stotal);
-#ifdef DS_TRACE
-    const long long tr_sstart = clock64();
-#endif
     for (int n = 0;; ++n) {
       {
         TR_T0();
@@ -1159,15 +1070,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       if (!ok) break;
     }
     if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
-#ifdef DS_TRACE
-    tr_stotal = clock64() - tr_sstart;
-    if (warp == 8 && lane == 0) {
-      TR_OUT(8, stotal);
-      TR_OUT(9, sdeps);
-      TR_OUT(10, sfree);
-      TR_OUT(11, sq);
-    }
-#endif
     return;
   }
 
@@ -1237,9 +1139,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       // q and this step's key/value rows are written; the partials of the previous layer are merged
       ok = bar_and(3, kAux, wait_deps(A->dep, A->need, A->n_deps, sp.counters, status, lane));
       if (!ok) break;
-#ifdef DS_TRACE
-      if (at == 0 && blockIdx.x == 0 && li < 128) g_attn_trace[li * 4 + 0] = global_timer_ns();
-#endif
       const int total = pre[batch] * HG;
       int mine = 0;
       for (int u = blockIdx.x; u < total; u += gridDim.x) {
@@ -1258,18 +1157,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       }
       bar_sync(3, kAux);
       if (at == 0 && mine > 0) red_release_add(sp.counters + A->split_done, mine);
-#ifdef DS_TRACE
-      if (at == 0 && blockIdx.x == 0 && li < 128) g_attn_trace[li * 4 + 1] = global_timer_ns();
-#endif
       // all partials of this layer (every CTA's) before any merge; o free to overwrite
       bool okw = true;
       if (lane == 0) okw = wait_global_ge(sp.counters + A->split_done, total, status);
       okw = __all_sync(0xffffffffu, okw) && wait_deps(A->mdep, A->mneed, A->n_mdeps, sp.counters, status, lane);
       ok = bar_and(3, kAux, okw);
       if (!ok) break;
-#ifdef DS_TRACE
-      if (at == 0 && blockIdx.x == 0 && li < 128) g_attn_trace[li * 4 + 2] = global_timer_ns();
-#endif
       const int n_pairs = batch * Hq;
       mine = 0;
       for (int u = blockIdx.x; u < n_pairs; u += gridDim.x) {
@@ -1281,9 +1174,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_stack_kernel(const StackPa
       }
       bar_sync(3, kAux);
       if (at == 0 && mine > 0) red_release_add(sp.counters + A->merge_done, mine);
-#ifdef DS_TRACE
-      if (at == 0 && blockIdx.x == 0 && li < 128) g_attn_trace[li * 4 + 3] = global_timer_ns();
-#endif
     }
     if (!ok && lane == 0) atomicOr(sp.status, LADDER_DEV_TIMEOUT);
   }
@@ -1293,20 +1183,6 @@ bool g_stack_usable = false;
 
 }  // namespace
 
-#ifdef DS_TRACE
-extern "C" int ladder_debug_read_stack_trace(unsigned long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_stack_trace, sizeof(g_stack_trace)) == cudaSuccess ? 0 : 1;
-}
-extern "C" int ladder_debug_read_attn_trace(unsigned long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_attn_trace, sizeof(g_attn_trace)) == cudaSuccess ? 0 : 1;
-}
-extern "C" int ladder_debug_read_kind_trace(unsigned long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_kind_trace, sizeof(g_kind_trace)) == cudaSuccess ? 0 : 1;
-}
-extern "C" int ladder_debug_read_phase_trace(unsigned long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_phase_trace, sizeof(g_phase_trace)) == cudaSuccess ? 0 : 1;
-}
-#endif
 
 cudaError_t decode_stack_init(int sm_count, bool* usable) {
   *usable = false;

@@ -1,6 +1,7 @@
 // Host-side launch interface of the kernels (internal to libladder; no torch types).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -78,6 +79,16 @@ struct DecodeAttnParams {
 int wide_padded_batch(int batch);  // Bp of the batch 9..64 GEMM kernel
 bool wide_handover();              // the tcgen05 kernel is the one in use for batch 9..64 (it alone reads staged operands)
 int decode_attention_splits(int batch, int n_kv_heads, int max_len, int sm_count);
+// Longest cache the decode attention handles: its merge step holds one weight per 64-key split, at most 1024.
+constexpr int kDecodeAttnMaxKeys = 64 * 1024;
+// The kernels read q / o / scratch with 16-byte and K / V with 16-byte vector loads: true when any pointer is not
+// aligned for them (the caller then gets an argument error instead of a misaligned-address fault on the device).
+inline bool decode_attention_misaligned(const void* q, const void* k, const void* v, const void* o, const void* scratch,
+                                        const void* kv_len) {
+  const uintptr_t a = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(v) |
+                      reinterpret_cast<uintptr_t>(o) | reinterpret_cast<uintptr_t>(scratch);
+  return (a & 15) != 0 || (reinterpret_cast<uintptr_t>(kv_len) & 3) != 0;
+}
 size_t decode_attention_scratch_floats(int batch, int n_q_heads, int head_dim, int n_splits);
 cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stream, bool pdl);
 

@@ -37,6 +37,10 @@ class ModelShape:
     prompt_len: int = 16
     decode_steps: int = 16
     seed: int = 0
+    # Per-layer architecture ("standard" | "ladder" | "parallel" | "upper_bound"), overriding layer_is_ladder,
+    # and an explicit per-module rule (2 * n_layers flags: module reads one module back); see include/ladder.h.
+    layer_mode: Optional[tuple] = None
+    module_stale: Optional[tuple] = None
 
     @property
     def qkv_rows(self) -> int:
@@ -53,10 +57,16 @@ class ModelShape:
 
     def with_layers(self, n: int) -> "ModelShape":
         mask = None if self.layer_is_ladder is None else tuple(self.layer_is_ladder[:n])
-        return replace(self, n_layers=n, layer_is_ladder=mask)
+        modes = None if self.layer_mode is None else tuple(self.layer_mode[:n])
+        flags = None if self.module_stale is None else tuple(self.module_stale[:2 * n])
+        return replace(self, n_layers=n, layer_is_ladder=mask, layer_mode=modes, module_stale=flags)
 
     def as_standard(self) -> "ModelShape":
-        return replace(self, layer_is_ladder=tuple([0] * self.n_layers))
+        return replace(self, layer_is_ladder=tuple([0] * self.n_layers), layer_mode=None, module_stale=None)
+
+    def as_mode(self, mode: str) -> "ModelShape":
+        """Every layer in one architecture: "standard", "ladder", "parallel" or "upper_bound"."""
+        return replace(self, layer_is_ladder=None, layer_mode=tuple([mode] * self.n_layers), module_stale=None)
 
     def param_count(self) -> int:
         d, F = self.d_model, self.d_ff

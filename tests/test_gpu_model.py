@@ -10,10 +10,15 @@ from tests.helpers import rel_err
 
 pytestmark = pytest.mark.gpu
 
-# Final hidden state: max_i |g_i - o_i| / max_i |o_i| per (sequence, position), bf16 path vs the exact
-# oracle.  Greedy tokens: teacher-forced (the oracle is fed the GPU's history) and, because floating
-# point decides an integer there, taken with both sides at the KV cache's bf16 storage precision.
+# Final hidden state: max_i |g_i - o_i| / max_i |o_i| per (sequence, position), bf16 path vs the exact oracle.
+# Greedy tokens: teacher-forced (the oracle is fed the GPU's history); the asserted figure is agreement with
+# the EXACT oracle's argmax, over at least 256 comparisons per claim.  Where the two disagree the step must be
+# a near-tie: the oracle's top-two logit margin at that step is below NEAR_TIE x the measured rms logit error
+# of the run.  A flip at a clear margin is a defect whatever the agreement rate.  The oracle with K/V rounded
+# to the cache's bf16 storage precision is run as a printed diagnostic only.
 HIDDEN_TOL = 2e-2
+MIN_AGREE = 0.99
+NEAR_TIE = 4.0
 CANARY = 0x7F7F            # bf16 bit pattern pre-filled into the cache (a huge finite value)
 
 
@@ -27,34 +32,102 @@ def B():
 
 def oracle_cfg(s: synth.ModelShape) -> O.OracleConfig:
     return O.OracleConfig(s.d_model, s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.vocab_size,
-                          s.rms_eps, s.rope_theta, None if s.layer_is_ladder is None else list(s.layer_is_ladder))
+                          s.rms_eps, s.rope_theta, None if s.layer_is_ladder is None else list(s.layer_is_ladder),
+                          layer_mode=None if s.layer_mode is None else list(s.layer_mode),
+                          module_stale=None if s.module_stale is None else list(s.module_stale))
 
 
-def gpu_generate(B, model, cache, prompt: np.ndarray, steps: int, want_hidden=True):
-    """prefill + `steps` greedy decode steps on the device. Returns tokens [B, steps+1], hiddens."""
+def gpu_generate(B, model, cache, prompt: np.ndarray, steps: int, want_hidden=True, want_logits=False):
+    """prefill + `steps` greedy decode steps on the device. Returns tokens [B, steps+1], hiddens (, logits)."""
     bsz = prompt.shape[0]
     d = model.shape.d_model
     tok = torch.from_numpy(prompt).cuda()
     nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
     hid = torch.zeros(bsz, d, device="cuda") if want_hidden else None
-    toks, hids = [], []
-    model.prefill(cache, tok, next_tokens=nxt, final_hidden=hid)
-    toks.append(nxt.clone())
-    if want_hidden:
-        hids.append(hid.clone())
-    for _ in range(steps):
-        model.decode_step(cache, nxt, next_tokens=nxt, final_hidden=hid)     # token feedback stays on the device
+    lg = torch.zeros(bsz, model.shape.vocab_size, device="cuda") if want_logits else None
+    toks, hids, logs = [], [], []
+
+    def keep():
         toks.append(nxt.clone())
         if want_hidden:
             hids.append(hid.clone())
+        if want_logits:
+            logs.append(lg.cpu())
+
+    model.prefill(cache, tok, next_tokens=nxt, final_hidden=hid, logits=lg)
+    keep()
+    for _ in range(steps):
+        model.decode_step(cache, nxt, next_tokens=nxt, final_hidden=hid, logits=lg)  # token feedback stays on the device
+        keep()
     torch.cuda.synchronize()
     toks = torch.stack(toks, 1).cpu().numpy()
     hids = torch.stack(hids, 1).cpu().numpy() if want_hidden else None
+    if want_logits:
+        return toks, hids, torch.stack(logs, 1).numpy()
     return toks, hids
 
 
-def check_generation(B, shape, steps, dtype, gains="ones", schedule=None, min_agree=0.99, batch=None, prompt_len=None):
-    w = synth.make_weights(shape, device="cuda", gains=gains)
+def oracle_teacher_forced(shape, w, prompt, toks, dtype, stream=False, bf16_kv=False):
+    """The oracle fed the GPU's token history: its own greedy choice, hidden state and logits at every step
+    [B, steps+1, ...].  stream=False: prompt pass + cached decode steps.  stream=True (models larger than host
+    memory): ONE pass over the whole token sequence without a cache -- the same function of the same tokens
+    (the oracle's cached decode equals full recomputation: tests/test_oracle_pins.py) -- so that every layer's
+    weights are fetched from the device exactly once."""
+    cfg = oracle_cfg(shape)
+    S, steps = prompt.shape[1], toks.shape[1] - 1
+    if not stream:
+        OW = O.OracleWeights(provider=synth.logical_provider(w, dtype))
+        return O.generate(cfg, OW, prompt, steps, S + steps + 1, dtype=dtype, forced=toks, bf16_kv=bf16_kv,
+                          return_logits=True)
+    OW = O.OracleWeights(provider=synth.logical_provider(w, dtype, keep=False))
+    seq = np.concatenate([prompt, toks[:, :-1]], axis=1)
+    r = O.forward(cfg, OW, seq, dtype=dtype, last_only=False, bf16_kv=bf16_kv)
+    return r.next_tokens[:, S - 1:], r.hidden[:, S - 1:], r.logits[:, S - 1:]
+
+
+class Parity:
+    """Outcome of one GPU-vs-oracle generation; `+` pools the greedy statistics of several runs into one claim."""
+
+    def __init__(self, err=0.0, n=0, flips=0, clear_flips=0, logit_rms=0.0, worst_clear=0.0, label=""):
+        self.err, self.n, self.flips, self.clear_flips = err, n, flips, clear_flips
+        self.logit_rms, self.worst_clear, self.label = logit_rms, worst_clear, label
+
+    @property
+    def agree(self) -> float:
+        return 1.0 - self.flips / max(self.n, 1)
+
+    def __add__(self, o):
+        return Parity(max(self.err, o.err), self.n + o.n, self.flips + o.flips, self.clear_flips + o.clear_flips,
+                      max(self.logit_rms, o.logit_rms), max(self.worst_clear, o.worst_clear), self.label or o.label)
+
+    def check(self, min_n=256):
+        print(f"[{self.label}] POOLED: hidden max-rel-err {self.err:.3e}; exact-oracle greedy agreement "
+              f"{self.agree:.4f} over {self.n} comparisons ({self.flips} flips, {self.clear_flips} at a clear margin)")
+        assert self.n >= min_n, f"{self.n} comparisons: too few for a claim"
+        assert self.err < HIDDEN_TOL, self.err
+        assert self.clear_flips == 0, f"{self.clear_flips} flips at a clear margin (worst {self.worst_clear:.3g} x rms)"
+        assert self.agree >= MIN_AGREE, self.agree
+
+
+def compare_with_oracle(label, toks, hids, logits, o_toks, o_hids, o_logits) -> Parity:
+    err = rel_err(hids, o_hids)
+    diff = logits.astype(np.float64) - o_logits
+    rms = float(np.sqrt(np.mean(diff * diff)))
+    top2 = np.partition(o_logits, -2, axis=-1)[..., -2:]
+    margin = top2[..., 1] - top2[..., 0]                       # oracle's top-two margin per step
+    flip = toks != o_toks
+    clear = flip & (margin >= NEAR_TIE * rms)
+    worst = float((margin[clear] / rms).max()) if clear.any() else 0.0
+    p = Parity(err, toks.size, int(flip.sum()), int(clear.sum()), rms, worst, label)
+    print(f"[{label}] hidden max-rel-err {err:.3e}; logit rms err {rms:.3e} (median oracle top-2 margin "
+          f"{float(np.median(margin)):.3e}); exact-oracle greedy agreement {p.agree:.4f} over {p.n} "
+          f"({p.flips} flips, {p.clear_flips} at a margin >= {NEAR_TIE:g} x rms)")
+    return p
+
+
+def check_generation(B, shape, steps, dtype, gains="ones", schedule=None, batch=None, prompt_len=None,
+                     stream=False, diagnostic=True, weights=None):
+    w = synth.make_weights(shape, device="cuda", gains=gains) if weights is None else weights
     bsz = shape.batch if batch is None else batch
     S = shape.prompt_len if prompt_len is None else prompt_len
     prompt = synth.make_tokens(shape, bsz, S)
@@ -63,22 +136,21 @@ def check_generation(B, shape, steps, dtype, gains="ones", schedule=None, min_ag
     if schedule is not None:        # a multi-kernel schedule (n_streams, graph, pdl); default: the persistent kernel
         model.set_persistent(False)
         model.set_schedule(*schedule)
-    elif bsz <= 8:             # the persistent kernel runs the ladder layers at the top of the model, every layer if small
+    elif bsz <= 8 and shape.layer_mode is None and shape.module_stale is None:
+        # the persistent kernel runs the ladder layers at the top of the model, every layer if small
         top_is_ladder = shape.layer_is_ladder is None or bool(shape.layer_is_ladder[-1])
         assert model.persistent_active() == (top_is_ladder or shape.layer_weight_bytes() < 300e6)
     cache = B.KVCache(shape, bsz, max_seq, fill=CANARY)
-    toks, hids = gpu_generate(B, model, cache, prompt, steps)
+    toks, hids, logits = gpu_generate(B, model, cache, prompt, steps, want_logits=True)
     assert model.device_status() == 0
-    # --- oracle, fed the GPU's token history (teacher forcing)
-    cfg = oracle_cfg(shape)
-    OW = O.OracleWeights(provider=synth.logical_provider(w, dtype))
-    o_toks, o_hids = O.generate(cfg, OW, prompt, steps, max_seq, dtype=dtype, forced=toks)
-    err = rel_err(hids, o_hids)
-    # the argmax decision is compared with both sides holding K/V at the cache's bf16 precision
-    k_toks, _ = O.generate(cfg, OW, prompt, steps, max_seq, dtype=dtype, forced=toks, bf16_kv=True)
-    agree = float(np.mean(toks == k_toks))
-    print(f"[{shape.name} L{shape.n_layers}] hidden max-rel-err {err:.3e}; greedy agreement {agree:.4f} "
-          f"(oracle with bf16 KV), {float(np.mean(toks == o_toks)):.4f} (exact oracle), {toks.size} comparisons")
+    # --- the exact oracle, fed the GPU's token history (teacher forcing)
+    label = f"{shape.name} L{shape.n_layers} B{bsz} S{S}"
+    o_toks, o_hids, o_logits = oracle_teacher_forced(shape, w, prompt, toks, dtype, stream)
+    par = compare_with_oracle(label, toks, hids, logits, o_toks, o_hids, o_logits)
+    if diagnostic:      # printed only: the same comparison with the oracle's K/V at the cache's bf16 precision
+        k_toks, k_hids, _ = oracle_teacher_forced(shape, w, prompt, toks, dtype, stream, bf16_kv=True)
+        print(f"[{label}] diagnostic, oracle holding bf16 K/V: agreement {float(np.mean(toks == k_toks)):.4f}, "
+              f"hidden max-rel-err {rel_err(hids, k_hids):.3e} (exact oracle vs that oracle: {rel_err(k_hids, o_hids):.3e})")
     # --- KV cache indexing
     used = S + steps
     assert cache.seq_lens.cpu().tolist() == [used] * bsz
@@ -86,23 +158,50 @@ def check_generation(B, shape, steps, dtype, gains="ones", schedule=None, min_ag
     assert bool((k5[:, :, :, used:, :] == CANARY).all()) and bool((v5[:, :, :, used:, :] == CANARY).all())
     assert not bool((k5[:, :, :, :used, :] == CANARY).any()) and not bool((v5[:, :, :, :used, :] == CANARY).any())
     model.close()
-    return err, agree, toks, hids, cache
+    return par, toks, hids, cache
 
 
-@pytest.mark.parametrize("variant", ["ladder", "standard", "hybrid", "hybrid_top", "gqa2"])
+@pytest.mark.parametrize("variant", ["ladder", "standard", "hybrid", "hybrid_top", "gqa2", "parallel", "parallel_mixed",
+                                     "explicit_flags"])
 def test_tiny_config_full(B, variant):
     s = synth.SHAPES["tiny"]
     if variant == "standard":
         s = s.as_standard()
+    elif variant == "parallel":        # parallel attention and MLP in every layer (paper Sec. 3.3.1)
+        s = s.as_mode("parallel")
+    elif variant == "parallel_mixed":
+        s = synth.replace(s, layer_mode=("standard", "parallel", "ladder", "parallel"))
+    elif variant == "explicit_flags":  # the rule stated module by module: the first ladder attention after the
+        s = synth.replace(s, layer_is_ladder=(0, 1, 1, 0), module_stale=(0, 0, 1, 1, 1, 1, 0, 0))   # standard layer is stale too
     elif variant == "hybrid":
         s = synth.replace(s, layer_is_ladder=(0, 1, 1, 0))
     elif variant == "hybrid_top":      # standard layers run kernel by kernel, the ladder stretch above them persistently
         s = synth.replace(s, layer_is_ladder=(0, 0, 1, 1))
     elif variant == "gqa2":            # two query heads per kv head (attention units of 2 heads)
         s = synth.replace(s, n_kv_heads=2)
-    err, agree, *_ = check_generation(B, s, 64, np.float64, gains="uniform", batch=4)     # 4 x 65 comparisons
-    assert err < HIDDEN_TOL, err
-    assert agree >= 0.99, agree
+    par, *_ = check_generation(B, s, 64, np.float64, gains="uniform", batch=4)     # 4 x 65 comparisons
+    par.check()
+
+
+def test_upper_bound_mode_is_bitwise_the_standard_model(B):
+    """The communication-free upper bound (paper Sec. 3.3.1) deletes the all-reduce of the standard model; on
+    one device there is none, so the mode must give the standard model's bits."""
+    base = synth.SHAPES["tiny"]
+    outs = []
+    for s in (base.as_standard(), base.as_mode("upper_bound")):
+        _, toks, hids, cache = check_generation(B, s, 12, np.float64, batch=3, diagnostic=False)
+        outs.append((toks, hids, cache.k.clone()))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    assert torch.equal(outs[0][2], outs[1][2])
+
+
+@pytest.mark.parametrize("schedule", [None, (2, True, True)])
+def test_8b_shape_parallel_layers(B, schedule):
+    """Eight parallel attention+MLP layers at the 8B shape (GQA 32/8): persistent kernel does not take them
+    (large layers that are not ladder), so this runs kernel by kernel; 260 comparisons."""
+    s = synth.SHAPES["8b_hybrid"].with_layers(8).as_mode("parallel")
+    par, *_ = check_generation(B, s, 64, np.float32, batch=4, prompt_len=64, schedule=schedule, diagnostic=False)
+    par.check()
 
 
 def test_tiny_cache_values_match_oracle(B):
@@ -129,7 +228,7 @@ def test_schedules_are_bit_identical(B):
     ref = None
     for sched in [None, (1, False, False), (1, True, False), (2, False, False), (2, True, False), (1, False, True),
                   (2, False, True), (2, True, True)]:
-        _, _, toks, hids, cache = check_generation(B, s, 12, np.float64, schedule=sched, batch=3, min_agree=0.0)
+        _, toks, hids, cache = check_generation(B, s, 12, np.float64, schedule=sched, batch=3, diagnostic=False)
         cur = (toks, hids, cache.k.clone(), cache.v.clone())
         if ref is None:
             ref = cur
@@ -206,27 +305,24 @@ def test_config_1p2b_full(B):
     oracle in float32.  Four sequences instead of the configuration's one, so that the agreement
     is a statistic over 260 comparisons rather than all-or-nothing over 65."""
     s = synth.SHAPES["1p2b"]
-    err, agree, *_ = check_generation(B, s, 64, np.float32, batch=4)
-    assert err < HIDDEN_TOL, err
-    assert agree >= 0.99, agree
+    par, *_ = check_generation(B, s, 64, np.float32, batch=4)
+    par.check()
 
 
 def test_70b_shape_shallow_full_context(B):
-    """First 2 layers of the 70B shape, batch 4, 1024-token prompts, 8 decode steps:
+    """First 2 layers of the 70B shape, batch 4, 1024-token prompts, 64 decode steps (260 comparisons):
     long-cache indexing, the split over the cache, M = 4096 prefill tiles."""
     s = synth.SHAPES["70b"].with_layers(2)
-    err, agree, *_ = check_generation(B, s, 8, np.float32)
-    assert err < HIDDEN_TOL, err
-    assert agree >= 0.97, agree          # 36 comparisons: at most one flip
+    par, *_ = check_generation(B, s, 64, np.float32, diagnostic=False)
+    par.check()
 
 
 def test_8b_hybrid_shape_short_context(B):
     """The 8B hybrid shape (GQA 32/8, theta 500000) cut to 4 standard + 4 ladder layers so the
     float32 oracle copy fits any host; 64-token prompts, 64 greedy steps."""
     s = synth.replace(synth.SHAPES["8b_hybrid"].with_layers(8), layer_is_ladder=(0, 0, 0, 0, 1, 1, 1, 1))
-    err, agree, *_ = check_generation(B, s, 64, np.float32, batch=4, prompt_len=64)       # 260 comparisons
-    assert err < HIDDEN_TOL, err
-    assert agree >= 0.99, agree
+    par, *_ = check_generation(B, s, 64, np.float32, batch=4, prompt_len=64)       # 260 comparisons
+    par.check()
 
 
 @pytest.mark.parametrize("impl", [0, 1, 2])
@@ -287,13 +383,14 @@ def test_prompt_fed_in_chunks(B, case, impl):
     model = B.Model(w, bsz, max_seq, bsz * max(chunks))          # workspace for one chunk only
     cache = B.KVCache(s, bsz, max_seq, fill=CANARY)
     nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+    lg = torch.zeros(bsz, s.vocab_size, device="cuda")
     hs, p0 = [], 0
     B.set_prefill_gemm_impl(impl)
     try:
         for i, c in enumerate(chunks):
             h = torch.zeros(bsz, c, s.d_model, device="cuda")
             call = model.prefill if i == 0 else model.prefill_append
-            call(cache, tok[:, p0:p0 + c].contiguous(), next_tokens=nxt, all_hidden=h)
+            call(cache, tok[:, p0:p0 + c].contiguous(), next_tokens=nxt, all_hidden=h, logits=lg)
             hs.append(h)
             p0 += c
             assert cache.seq_lens.cpu().tolist() == [p0] * bsz
@@ -310,17 +407,23 @@ def test_prompt_fed_in_chunks(B, case, impl):
     err = rel_err(got, ref.hidden)
     print(f"[{case} impl {impl}] chunked prompt pass: hidden max-rel-err {err:.3e} over {bsz * S} positions")
     assert err < HIDDEN_TOL, err
+    _, o_logits = O.head(cfg, OW, ref.x_final[:, -1:].astype(dtype))        # the oracle's logits at the last position
     k5 = cache.k5().view(torch.int16)
     assert bool((k5[:, :, :, S:, :] == CANARY).all()) and not bool((k5[:, :, :, :S, :] == CANARY).any())
     # ---- the same prompt in one call (needs its own, larger workspace), then both decode on
     model1 = B.Model(w, bsz, max_seq, bsz * S)
     cache1 = B.KVCache(s, bsz, max_seq, fill=CANARY)
     nxt1 = torch.zeros(bsz, dtype=torch.int32, device="cuda")
-    model1.prefill(cache1, tok, next_tokens=nxt1)
+    lg1 = torch.zeros(bsz, s.vocab_size, device="cuda")
+    model1.prefill(cache1, tok, next_tokens=nxt1, logits=lg1)
     torch.cuda.synchronize()
     assert rel_err(cache.k5()[:, :, :, :S].float().cpu().numpy(), cache1.k5()[:, :, :, :S].float().cpu().numpy()) < 2e-2
     assert rel_err(cache.v5()[:, :, :, :S].float().cpu().numpy(), cache1.v5()[:, :, :, :S].float().cpu().numpy()) < 2e-2
-    same = nxt.cpu().numpy() == nxt1.cpu().numpy()
+    # first generated token of either run: the oracle's choice, or a near-tie of the oracle's logits
+    for name, t, l in (("chunked", nxt, lg), ("one call", nxt1, lg1)):
+        p = compare_with_oracle(f"{case} {name}", t.cpu().numpy()[:, None], got[:, -1:], l.cpu().numpy()[:, None],
+                                O.greedy(o_logits), ref.hidden[:, -1:], o_logits)
+        assert p.clear_flips == 0, (name, p.worst_clear)
     hid, hid1 = torch.zeros(bsz, s.d_model, device="cuda"), torch.zeros(bsz, s.d_model, device="cuda")
     feed = nxt1.clone()                                           # both continue from the same tokens
     for _ in range(steps):
@@ -330,65 +433,26 @@ def test_prompt_fed_in_chunks(B, case, impl):
         assert rel_err(hid.cpu().numpy(), hid1.cpu().numpy()) < HIDDEN_TOL
         feed = nxt1.clone()
     assert cache.seq_lens.cpu().tolist() == [S + steps] * bsz
-    assert same.mean() >= 0.5                                     # first generated token: near-ties may flip one
     model.close()
     model1.close()
 
 
-def test_70b_full_size_single_live_module(B):
-    """The benchmark's own launch configuration -- all 80 layers of the 70B shape resident (141 GB),
-    batch 4, 1024-token prompts, CUDA-graph decode -- checked with a property that holds at any size:
-    with every output / down projection zeroed except module k's, the model computes x_0 + h_k(x_0)
-    (ladder and standard alike), which the oracle evaluates from layer k's weights alone."""
-    free, _ = torch.cuda.mem_get_info()
-    s = synth.SHAPES["70b"]
-    if free < s.param_count() * 2 + 8e9:
-        pytest.skip("needs ~150 GB of free device memory")
-    w = synth.make_weights(s, device="cuda")
-    bsz, S, steps = s.batch, s.prompt_len, 3
-    prompt = synth.make_tokens(s, bsz, S)
-    for layer, live in ((41, "attention"), (57, "mlp")):
-        keep = (w.w_o[layer].clone(), w.w_down[layer].clone())
-        for l in range(s.n_layers):
-            w.w_o[l].zero_()
-            w.w_down[l].zero_()
-        if live == "attention":
-            w.w_o[layer].copy_(keep[0])
-        else:
-            w.w_down[layer].copy_(keep[1])
-        model = B.Model(w, bsz, S + steps + 1, bsz * S)
-        cache = B.KVCache(s, bsz, S + steps + 1)
-        toks, hids = gpu_generate(B, model, cache, prompt, steps)
-        assert model.device_status() == 0
-        model.close()
-        # oracle: a one-layer model made of layer k's weights (the other module of that layer is dead too)
-        one = synth.replace(s.with_layers(1))
-        w1 = synth.AbiWeights(one, w.tok_embedding, w.final_norm, w.lm_head, [w.attn_norm[layer]], [w.w_qkv[layer]],
-                              [w.w_o[layer]], [w.mlp_norm[layer]], [w.w_gate_up[layer]], [w.w_down[layer]])
-        OW = O.OracleWeights(provider=synth.logical_provider(w1, np.float32))
-        o_toks, o_hids = O.generate(oracle_cfg(one), OW, prompt, steps, S + steps + 1, dtype=np.float32, forced=toks)
-        err = rel_err(hids, o_hids)
-        print(f"[70b full size, live {live} of layer {layer}] hidden max-rel-err {err:.3e}, "
-              f"greedy agreement {float(np.mean(toks == o_toks)):.3f}")
-        assert err < HIDDEN_TOL, (live, err)
-        w.w_o[layer].copy_(keep[0])
-        w.w_down[layer].copy_(keep[1])
-        del cache, OW
-        torch.cuda.empty_cache()
-
-
-@pytest.mark.parametrize("batch", [1, 16, 64])
 @pytest.mark.parametrize("variant", ["ladder", "standard"])
-def test_tp_rank_slice_shape_batches(B, variant, batch):
+def test_tp_rank_slice_shape_batches(B, variant):
     """One tensor-parallel rank's slice of the 70B shape (8 q heads, 1 kv head, ffn 3584, hidden 8192:
     attention width differs from the hidden size) without communication, cut to 3 layers; the batch
-    sizes of the sweep the paper's throughput figure uses (Sec. 3.3.1), ladder and standard."""
+    sizes of the sweep the paper's throughput figure uses (Sec. 3.3.1), ladder and standard.  The greedy
+    statistics of the four batch sizes are pooled into one claim (85 sequences x 13 steps)."""
     s = synth.SHAPES["tp_slice"].with_layers(3)
     if variant == "standard":
         s = s.as_standard()
-    err, agree, *_ = check_generation(B, s, 6, np.float32, batch=batch, prompt_len=40)
-    assert err < HIDDEN_TOL, err
-    assert agree >= (0.98 if batch >= 16 else 0.85), agree      # 7 comparisons at batch 1: at most one flip
+    w = synth.make_weights(s, device="cuda")
+    total = Parity()
+    for batch in (1, 4, 16, 64):
+        par, *_ = check_generation(B, s, 12, np.float32, batch=batch, prompt_len=40, weights=w, diagnostic=False)
+        assert par.err < HIDDEN_TOL, (batch, par.err)
+        total = total + par
+    total.check()
 
 
 @pytest.mark.parametrize("batch", [12, 40])
@@ -452,6 +516,9 @@ def test_persistent_kernel_wait_runs_out_cleanly(B):
     torch.cuda.synchronize()
     assert time.time() - t0 < 5.0
     assert model.device_status() & 4             # LADDER_DEV_TIMEOUT, read and cleared
+    with pytest.raises(B.LadderError) as e:      # the step that timed out produced nothing: further steps are
+        model.decode_step(cache, nxt, next_tokens=nxt)          # refused until the position is set again
+    assert e.value.status == 6                   # LADDER_ERR_TIMEOUT
     model.debug_stall_last_phase(False)
     again = run()
     assert model.device_status() == 0
@@ -513,17 +580,15 @@ def test_tiny_config_batch_5_to_8(B, batch):
     """Batches 5..8 take the persistent kernel's other instantiation (eight separate MMA columns, activations as a
     single bf16, converted by the stagers in every phase)."""
     s = synth.replace(synth.SHAPES["tiny"], layer_is_ladder=(0, 1, 1, 1))
-    err, agree, *_ = check_generation(B, s, 40, np.float64, gains="uniform", batch=batch)
-    assert err < HIDDEN_TOL, err
-    assert agree >= 0.98, agree
+    par, *_ = check_generation(B, s, 64, np.float64, gains="uniform", batch=batch)
+    par.check()
 
 
 def test_tiny_long_context_many_splits(B):
     """8250 cached keys: 129 attention splits per head, more than the 64 threads of a merge unit own one each."""
     s = synth.SHAPES["tiny"]
-    err, agree, *_ = check_generation(B, s, 4, np.float64, gains="uniform", batch=1, prompt_len=8250)
-    assert err < HIDDEN_TOL, err
-    assert agree >= 0.8, agree           # 5 comparisons: at most one flip
+    par, *_ = check_generation(B, s, 64, np.float64, gains="uniform", batch=4, prompt_len=8250, diagnostic=False)
+    par.check()
 
 
 def test_70b_shape_persistent_equals_multi_kernel_repeatedly(B):
@@ -564,7 +629,7 @@ def test_sequences_of_different_lengths_decode_together(B, persistent):
     then decoded as one batch, against the oracle run on each sequence alone."""
     s = synth.SHAPES["tiny"]
     w = synth.make_weights(s, device="cuda", gains="uniform")
-    lens, steps, max_seq = [5, 16, 9], 6, 32
+    lens, steps, max_seq = [5, 16, 9], 90, 112            # 3 x 91 comparisons
     toks = synth.make_tokens(s, 3, 16)
     model = B.Model(w, 3, max_seq, 16)
     model.set_persistent(persistent)
@@ -575,23 +640,127 @@ def test_sequences_of_different_lengths_decode_together(B, persistent):
         model.prefill(cache.slot(b), torch.from_numpy(toks[b:b + 1, :L].copy()).cuda(), next_tokens=nxt[b:b + 1])
     assert cache.seq_lens.cpu().tolist() == lens
     model.set_position(max(lens))                     # host-side overflow check follows the longest sequence
-    g_tok, g_hid = [nxt.clone()], []
+    lg = torch.zeros(3, s.vocab_size, device="cuda")
+    g_tok, g_hid, g_log = [nxt.clone()], [], []
     for _ in range(steps):
-        model.decode_step(cache, nxt, next_tokens=nxt, final_hidden=hid)
+        model.decode_step(cache, nxt, next_tokens=nxt, final_hidden=hid, logits=lg)
         g_tok.append(nxt.clone())
         g_hid.append(hid.clone())
+        g_log.append(lg.clone())
     torch.cuda.synchronize()
     assert model.device_status() == 0
     assert cache.seq_lens.cpu().tolist() == [L + steps for L in lens]
     g_tok = torch.stack(g_tok, 1).cpu().numpy()       # [3, steps + 1]
     g_hid = torch.stack(g_hid, 1).cpu().numpy()       # [3, steps, d]
+    g_log = torch.stack(g_log, 1).cpu().numpy()       # [3, steps, V]
     cfg = oracle_cfg(s)
     OW = O.OracleWeights(provider=synth.logical_provider(w, np.float64))
+    total = Parity()
     for b, L in enumerate(lens):
-        o_tok, o_hid = O.generate(cfg, OW, toks[b:b + 1, :L], steps, max_seq, dtype=np.float64, forced=g_tok[b:b + 1])
-        assert rel_err(g_hid[b], o_hid[0, 1:]) < HIDDEN_TOL
-        assert np.mean(g_tok[b] == o_tok[0]) >= 0.85          # 7 comparisons per sequence: at most one flip
+        o_tok, o_hid, o_log = O.generate(cfg, OW, toks[b:b + 1, :L], steps, max_seq, dtype=np.float64,
+                                         forced=g_tok[b:b + 1], return_logits=True)
+        total = total + compare_with_oracle(f"ragged seq {b} len {L}", g_tok[b:b + 1, 1:], g_hid[b:b + 1],
+                                            g_log[b:b + 1], o_tok[:, 1:], o_hid[:, 1:], o_log[:, 1:])
+    total.check()
     k5 = cache.k5().view(torch.int16)                          # [layer][b][h][pos][d]: rows beyond each length untouched
     for b, L in enumerate(lens):
         assert bool((k5[:, b, :, L + steps:, :] == CANARY).all()) and not bool((k5[:, b, :, :L + steps, :] == CANARY).any())
     model.close()
+
+
+# ----------------------------------------------------------------------------- full depth, every module live
+def truncated(w: synth.AbiWeights, shape: synth.ModelShape) -> synth.AbiWeights:
+    """The first shape.n_layers layers of w as a model of their own (same tensors, nothing copied)."""
+    n = shape.n_layers
+    return synth.AbiWeights(shape, w.tok_embedding, w.final_norm, w.lm_head, w.attn_norm[:n], w.w_qkv[:n], w.w_o[:n],
+                            w.mlp_norm[:n], w.w_gate_up[:n], w.w_down[:n])
+
+
+def test_8b_hybrid_full_depth_and_depth_sweep(B):
+    """The third benchmark configuration at its full depth with every module live: 32 layers, layers 0-15
+    standard (Eq. 1) and 16-31 ladder (Eq. 2), batch 4, 64-token prompts, 64 greedy steps, against the exact
+    float32 oracle streamed one layer at a time.  Shallower cuts of the same weights (half standard, half ladder)
+    show how the hidden-state error grows with depth."""
+    full = synth.SHAPES["8b_hybrid"]
+    w = synth.make_weights(full, device="cuda")
+    rows = []
+    for n in (8, 16, 32):
+        s = synth.replace(full.with_layers(n), layer_is_ladder=tuple([0] * (n // 2) + [1] * (n // 2)))
+        par, *_ = check_generation(B, s, 64, np.float32, batch=4, prompt_len=64, stream=True, diagnostic=True,
+                                   weights=truncated(w, s))
+        rows.append((n, par))
+    print("DEPTH SWEEP 8b_hybrid shape (layers, hidden max-rel-err, logit rms, agreement, flips): " +
+          "; ".join(f"{n}: {p.err:.3e} {p.logit_rms:.3e} {p.agree:.4f} {p.flips}" for n, p in rows))
+    for _, par in rows:
+        par.check()
+
+
+@pytest.fixture(scope="module")
+def weights_70b():
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    s = synth.SHAPES["70b"]
+    if free < s.param_count() * 2 + 10e9:
+        pytest.skip("needs ~152 GB of free device memory")
+    w = synth.make_weights(s, device="cuda")
+    yield w
+    del w
+    torch.cuda.empty_cache()
+
+
+def test_70b_full_depth_and_depth_sweep(B, weights_70b):
+    """The headline configuration with all 80 ladder layers resident and live (141 GB), batch 4, 16-token
+    prompts, 64 greedy steps, against the exact float32 oracle, which fetches each layer's weights from the
+    device once (one pass over prompt + generated tokens).  This is Eq. 2 applied 160 times: what the
+    benchmark times.  Cuts to 8, 16 and 32 layers of the same weights give the error growth with depth."""
+    full = synth.SHAPES["70b"]
+    rows = []
+    for n in (8, 16, 32, 80):
+        s = full.with_layers(n)
+        par, *_ = check_generation(B, s, 64, np.float32, batch=4, prompt_len=16, stream=True, diagnostic=(n < 80),
+                                   weights=truncated(weights_70b, s))
+        rows.append((n, par))
+        torch.cuda.empty_cache()
+    print("DEPTH SWEEP 70b shape (layers, hidden max-rel-err, logit rms, agreement, flips): " +
+          "; ".join(f"{n}: {p.err:.3e} {p.logit_rms:.3e} {p.agree:.4f} {p.flips}" for n, p in rows))
+    for _, par in rows:
+        par.check()
+
+
+def test_70b_full_size_single_live_module(B, weights_70b):
+    """The benchmark's own launch configuration -- all 80 layers of the 70B shape resident (141 GB),
+    batch 4, 1024-token prompts, CUDA-graph decode -- checked with a property that holds at any size:
+    with every output / down projection zeroed except module k's, the model computes x_0 + h_k(x_0)
+    (ladder and standard alike), which the oracle evaluates from layer k's weights alone."""
+    s = synth.SHAPES["70b"]
+    w = weights_70b          # NOTE: this test zeroes projections in place; it is the last user of the fixture
+    bsz, S, steps = s.batch, s.prompt_len, 3
+    prompt = synth.make_tokens(s, bsz, S)
+    for layer, live in ((41, "attention"), (57, "mlp")):
+        keep = (w.w_o[layer].clone(), w.w_down[layer].clone())
+        for l in range(s.n_layers):
+            w.w_o[l].zero_()
+            w.w_down[l].zero_()
+        if live == "attention":
+            w.w_o[layer].copy_(keep[0])
+        else:
+            w.w_down[layer].copy_(keep[1])
+        model = B.Model(w, bsz, S + steps + 1, bsz * S)
+        cache = B.KVCache(s, bsz, S + steps + 1)
+        toks, hids = gpu_generate(B, model, cache, prompt, steps)
+        assert model.device_status() == 0
+        model.close()
+        # oracle: a one-layer model made of layer k's weights (the other module of that layer is dead too)
+        one = synth.replace(s.with_layers(1))
+        w1 = synth.AbiWeights(one, w.tok_embedding, w.final_norm, w.lm_head, [w.attn_norm[layer]], [w.w_qkv[layer]],
+                              [w.w_o[layer]], [w.mlp_norm[layer]], [w.w_gate_up[layer]], [w.w_down[layer]])
+        OW = O.OracleWeights(provider=synth.logical_provider(w1, np.float32))
+        o_toks, o_hids = O.generate(oracle_cfg(one), OW, prompt, steps, S + steps + 1, dtype=np.float32, forced=toks)
+        err = rel_err(hids, o_hids)
+        print(f"[70b full size, live {live} of layer {layer}] hidden max-rel-err {err:.3e}, "
+              f"greedy agreement {float(np.mean(toks == o_toks)):.3f}")
+        assert err < HIDDEN_TOL, (live, err)
+        w.w_o[layer].copy_(keep[0])
+        w.w_down[layer].copy_(keep[1])
+        del cache, OW
+        torch.cuda.empty_cache()

@@ -19,30 +19,48 @@ def B():
     return binding
 
 
-def routes(mask):
-    """Residual routing of Eq. 1 / Eq. 2 on two buffers, re-derived here: per module (in, add, dst)."""
-    cur, stale, out = 0, -1, []
-    for lad in mask:
-        per_layer = []
-        for _ in range(2):                      # attention module, MLP module
-            if lad and stale >= 0:              # x_m = x_{m-1} + h(x_{m-2}), overwriting x_{m-2}
-                r = (stale, cur, stale)
-                cur, stale = stale, cur
-            elif lad:                           # first ladder module after a standard one
-                r = (cur, cur, cur ^ 1)
-                stale, cur = cur, cur ^ 1
-            else:                               # x_m = x_{m-1} + h(x_{m-1}) in place
-                r = (cur, cur, cur)
-                stale = -1
-            per_layer.append(r)
-        out.append(per_layer)
-    return out, cur
+def module_flags(shape):
+    """Per module (1-based m -> index m-1): does it read x_{m-2} instead of x_{m-1}?  From the layer modes as
+    include/ladder.h states them, or the explicit table."""
+    if shape.module_stale is not None:
+        return [bool(f) for f in shape.module_stale]
+    modes = list(shape.layer_mode) if shape.layer_mode is not None else \
+        ["ladder" if v else "standard" for v in shape.ladder_mask()]
+    flags = []
+    for l, mode in enumerate(modes):
+        if mode == "ladder":
+            flags += [l == 0 or modes[l - 1] == "ladder", True]
+        elif mode == "parallel":
+            flags += [False, True]
+        else:
+            flags += [False, False]
+    return flags
+
+
+def routes(flags):
+    """Which of the two residual buffers every module reads, adds onto and writes, from value liveness: the
+    buffers hold stream values x_k; module m must find x_{m-1} (to add onto) and the value it reads, and x_m may
+    only replace a value nobody needs any more -- x_{m-1} itself when module m read it and module m+1 will not,
+    otherwise the other buffer (which holds x_{m-2} or nothing)."""
+    holds = {0: 0, 1: None}
+    out = []
+    n = len(flags)
+    for m in range(1, n + 1):
+        newest = next(b for b, v in holds.items() if v == m - 1)
+        want = m - 2 if (flags[m - 1] and m >= 2) else m - 1
+        src = next(b for b, v in holds.items() if v == want)      # StopIteration = the value was destroyed
+        next_reads_newest = m < n and flags[m]                    # module m+1 reads x_{m-1}
+        dst = newest if (src == newest and not next_reads_newest) else newest ^ 1
+        out.append((src, newest, dst))
+        holds[dst] = m
+    final = next(b for b, v in holds.items() if v == n)
+    return [out[2 * l:2 * l + 2] for l in range(n // 2)], final
 
 
 def expected_nodes(shape, first_layer):
     """Emission order of the launch with (name, act reads, epilogue reads, writes) per node."""
-    mask = shape.ladder_mask()
-    rt, final = routes(mask)
+    flags = module_flags(shape)
+    rt, final = routes(flags)
     nodes = []
     for l in range(first_layer, shape.n_layers):
         (a_in, a_add, a_dst), (m_in, m_add, m_dst) = rt[l]
@@ -51,7 +69,7 @@ def expected_nodes(shape, first_layer):
         wo = (("gemm", WO, l), {"o"}, {f"R{a_add}"}, {f"R{a_dst}"})
         gu = (("gemm", GU, l), {f"R{m_in}"}, set(), {"h"})
         dn = (("gemm", DN, l), {"h"}, {f"R{m_add}"}, {f"R{m_dst}"})
-        independent = bool(mask[l]) and m_in != a_dst
+        independent = flags[2 * l + 1] and m_in != a_dst       # the MLP's input does not come from this layer's attention
         nodes += [qkv, att] + ([gu, wo] if independent else [wo, gu]) + [dn]
     nodes.append((("gemm", HEAD, shape.n_layers), {f"R{final}"}, set(), {"logits"}))
     return nodes
@@ -65,6 +83,11 @@ CASES = {
     "70b": (synth.SHAPES["70b"], 4),
     "8b_hybrid": (synth.SHAPES["8b_hybrid"], 4),
     "1p2b": (synth.SHAPES["1p2b"], 1),
+    "tiny_parallel": (synth.SHAPES["tiny"].as_mode("parallel"), 4),
+    "tiny_parallel_mixed": (synth.replace(synth.SHAPES["tiny"], layer_mode=("standard", "parallel", "ladder", "parallel")), 2),
+    "tiny_explicit_flags": (synth.replace(synth.SHAPES["tiny"], layer_is_ladder=(0, 1, 1, 0),
+                                          module_stale=(0, 0, 1, 1, 1, 1, 0, 0)), 3),
+    "70b_parallel": (synth.SHAPES["70b"].as_mode("parallel"), 4),
 }
 
 
@@ -73,7 +96,7 @@ def test_plan_orders_every_hazard(B, case):
     shape, batch = CASES[case]
     plan = B.stack_plan(shape, batch, 256)
     assert plan["ok"]
-    mask = shape.ladder_mask()
+    mask = shape.ladder_mask() if shape.layer_mode is None else [m == "ladder" for m in shape.layer_mode]
     first = shape.n_layers
     while first > 0 and mask[first - 1]:
         first -= 1

@@ -18,11 +18,11 @@
  * followed by grouped-query causal attention with rotary embedding on interleaved pairs,
  * or by a SwiGLU MLP ("Llama-3's model architecture", paper Sec. 3.3.1).
  *
- * Numerics: bf16 weights, bf16 KV cache, bf16 tensor-core operands, fp32 accumulation, fp32
- * softmax, fp32 residual stream, fp32 logits.  In the decode path activations enter the
+ * Numerics: bf16 weights, 16-bit KV cache in IEEE binary16 (same bytes as bf16, three more significant bits:
+ * with bf16 keys and values the cache alone puts deep models outside a 2e-2 hidden-state bound), fp32
+ * accumulation, fp32 softmax, fp32 residual stream, fp32 logits.  In the decode path activations enter the
  * tensor cores as a bf16 high + low pair (about 16 mantissa bits; free in a bandwidth-bound
- * kernel) for batch <= 16, and so do the prefill GEMMs and the prefill query (two MMAs per
- * weight tile): what is left of bf16 in the activations is the KV cache itself.
+ * kernel) for batch <= 16, and so do the prefill GEMMs; queries enter the attention as a binary16 high + low pair.
  * Greedy argmax picks the lowest index on ties.
  *
  * Errors: every function returns a ladder_status_t; argument errors are detected on the
@@ -104,9 +104,11 @@ typedef struct {
   const void* const* w_down;    /* [d_model, d_ff]                                         */
 } ladder_weights_t;
 
-/* KV cache: caller-allocated, library reads and writes.  K holds post-rotation keys. */
+/* KV cache: caller-allocated, library reads and writes.  K holds post-rotation keys.  Elements are IEEE binary16
+ * (fp16), 2 bytes each; values beyond +-65504 saturate (keys and values are projections of RMS-normalised
+ * activations and stay far inside that range). */
 typedef struct {
-  void* k;           /* bf16 [n_layers][max_batch][n_kv_heads][max_seq_len][head_dim] */
+  void* k;           /* binary16 [n_layers][max_batch][n_kv_heads][max_seq_len][head_dim] */
   void* v;           /* same shape                                                    */
   int32_t* seq_lens; /* int32 [max_batch]: tokens cached per sequence; prefill sets it,
                         each decode step reads the position from it and adds one        */
@@ -142,7 +144,8 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
  * Defaults: 2, 1, 1.  Results are bit-identical across all settings. */
 ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, int32_t use_graph, int32_t use_pdl);
 
-/* Persistent decode step (default on; batch <= 8).  The ladder layers at the top of the model (all layers of
+/* Persistent decode step (default on; batch <= 4: there the bf16 hi + lo activation pair fits one MMA tile;
+ * larger batches take the tcgen05 kernels, one kernel per GEMM).  The ladder layers at the top of the model (all layers of
  * an all-ladder model) and the LM head of a decode step run as ONE cooperative kernel launch.  Standard-residual
  * layers below them run one kernel per GEMM when a layer's weights exceed 300 MB (measured faster there) and go
  * into the same launch otherwise; on = 2 puts every layer into the launch whatever its size.  A large-layer
@@ -152,9 +155,9 @@ ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, 
  * memory that is polled only where data crosses SMs.  With the ladder rule (Eq. 2: module m reads
  * x_{m-2}) every such dependency points two phases back, so the weight stream never stops between
  * modules; with the standard rule (Eq. 1) each phase waits for the one before.  on = 0 selects the
- * multi-kernel schedule configured by ladder_model_set_schedule (also used automatically for batch > 8
+ * multi-kernel schedule configured by ladder_model_set_schedule (also used automatically for batch > 4
  * and on devices where the kernel cannot be made resident).  Results are bit-identical either way.
- * ladder_model_persistent_active returns 1 when decode steps of batch <= 8 take this path. */
+ * ladder_model_persistent_active returns 1 when decode steps of batch <= 4 take this path. */
 ladder_status_t ladder_model_set_persistent(ladder_model_t* m, int32_t on);
 int32_t ladder_model_persistent_active(const ladder_model_t* m);
 
@@ -266,7 +269,7 @@ ladder_status_t ladder_op_smallm_gemm(const void* W, int32_t N, int32_t K, const
                                       const float* addend, void* out, void* cuda_stream);
 
 /* Split-KV grouped-query decode attention for one layer.
- *   q fp32 [batch, Hq*Dh] (already rotated); k,v bf16 [max_batch][Hkv][max_seq_len][Dh] (one layer);
+ *   q fp32 [batch, Hq*Dh] (already rotated); k,v binary16 [max_batch][Hkv][max_seq_len][Dh] (one layer);
  *   kv_len int32 [batch] = number of keys to attend (positions 0..kv_len-1);
  *   scratch fp32, at least ladder_decode_attention_scratch_bytes(...) bytes;
  *   o fp32 [batch, Hq*Dh].  softmax(q.k/sqrt(Dh)) v per head, fp32 softmax and accumulation.
@@ -304,23 +307,41 @@ ladder_status_t ladder_op_prefill_gemm(const void* A, const void* A_lo, const vo
                                        int32_t epi_mode, const float* addend, void* out, void* out_lo,
                                        void* cuda_stream);
 
-/* Which implementation the prefill GEMMs use (process-wide): 0 = tcgen05 tensor-core kernel with TMA
- * and TMEM accumulators, activations as a bf16 hi + lo pair (default), 1 = warp-level mma.sync kernel (kept as a
- * cross-check), 2 = the tcgen05 kernel with ONE bf16 value per activation (normalised input, query, attention
- * output, SwiGLU output): half the tensor-core work and the usual bf16 inference precision, but every stored
- * activation is rounded at 2^-9, which by itself reaches 1.6e-2 of hidden-state error after 8 layers of the 8B
- * shape - outside the 2e-2 bound of the default mode for deeper models. */
+/* The same GEMM with binary16 operands, the prompt pass's default for calls of at least 256 tokens: A binary16
+ * [M,K] (ONE value per activation, 11 significant bits), W binary16 [N,K]; half the tensor-core work of the
+ * bf16 hi + lo pair.  Epilogue modes as above, with the 16-bit outputs of modes 1 and 3 written as binary16
+ * (saturating at +-65504).  A, W and out 16-byte aligned. */
+ladder_status_t ladder_op_prefill_gemm_f16(const void* A, const void* W, int32_t M, int32_t N, int32_t K, int32_t epi_mode,
+                                           const float* addend, void* out, void* cuda_stream);
+
+/* bf16 -> binary16 conversion of n elements (n % 8 == 0, pointers 16-byte aligned): what the prompt pass does to
+ * one layer's weights per call.  Exact for magnitudes >= 2^-14 (binary16 carries three more significant bits);
+ * smaller magnitudes are rounded to binary16's subnormal grid, at most 2^-25 away. */
+ladder_status_t ladder_op_convert_bf16_f16(const void* src, void* dst, int64_t n, void* cuda_stream);
+
+/* Which implementation the prefill GEMMs use.  PROCESS-WIDE and not thread-safe: a switch for tests and A/B
+ * measurements, not for serving code (leave it at 0).
+ *   0 = default: tcgen05 kernel (TMA, TMEM accumulators) with binary16 operands -- each layer's bf16 weights are
+ *       converted to binary16 in a per-model scratch once per call (1.7 GB at the 70B shape; model creation falls
+ *       back to mode 3 when that does not fit) and every activation is ONE binary16 value -- for calls of at
+ *       least 256 tokens, bf16 hi + lo pairs (mode 3) for shorter ones;
+ *   1 = warp-level mma.sync kernel with bf16 hi + lo activations (kept as a cross-check);
+ *   2 = the tcgen05 kernel with ONE bf16 value per activation: the usual bf16 inference precision, but every stored
+ *       activation is rounded at 2^-9, which by itself reaches 1.6e-2 of hidden-state error after 8 layers of the
+ *       8B shape;
+ *   3 = the tcgen05 kernel with bf16 hi + lo activation pairs (two MMAs per product) at every size. */
 void ladder_set_prefill_gemm_impl(int32_t impl);
 
-/* Decode GEMM for batch 9..64: 0 = tcgen05 kernel (weights as the M side of the MMA, TMA tiles, TMEM accumulators,
+/* Decode GEMM for batch 5..64: 0 = tcgen05 kernel (weights as the M side of the MMA, TMA tiles, TMEM accumulators,
  * equal K-block ranges per CTA with a deterministic fix-up of shared tiles; default), 1 = the earlier mma.sync kernel
- * (cross-check).  Process-wide; not thread-safe against concurrent launches. */
+ * (cross-check; batch 5..8 then runs with ONE bf16 value per activation).  PROCESS-WIDE and not thread-safe: a
+ * switch for tests and A/B measurements, not for serving code. */
 void ladder_set_decode_wide_impl(int32_t impl);
 
 /* Causal grouped-query attention of the prefill path for one layer:
- *   q bf16 [batch, seq_len, Hq*Dh] (rotated), q_lo its optional low part; k,v bf16 cache of one layer
- *   as above, rows 0..seq_len-1 valid; o bf16 [batch, seq_len, Hq*Dh], o_lo its low part (given iff
- *   q_lo is).  Query p attends keys t <= p. */
+ *   q binary16 [batch, seq_len, Hq*Dh] (rotated), q_lo its optional low part; k,v binary16 cache of one layer
+ *   as above, rows 0..seq_len-1 valid; o bf16 [batch, seq_len, Hq*Dh] (the output projection's operand type),
+ *   o_lo its low part (given iff q_lo is).  Query p attends keys t <= p. */
 ladder_status_t ladder_op_prefill_attention(const void* q, const void* q_lo, const void* k, const void* v, int32_t batch,
                                             int32_t seq_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
                                             int32_t max_seq_len, void* o, void* o_lo, void* cuda_stream);

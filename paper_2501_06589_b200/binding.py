@@ -26,6 +26,7 @@ EXPORTS = [
     "ladder_last_error", "ladder_op_smallm_gemm", "ladder_decode_attention_scratch_bytes",
     "ladder_op_decode_attention", "ladder_op_prefill_gemm", "ladder_op_prefill_attention",
     "ladder_op_decode_attention_noalloc", "ladder_set_prefill_gemm_impl", "ladder_set_decode_wide_impl",
+    "ladder_op_prefill_gemm_f16", "ladder_op_convert_bf16_f16",
 ]
 
 
@@ -120,6 +121,9 @@ def lib() -> C.CDLL:
         L.ladder_set_decode_wide_impl.argtypes = [C.c_int32]
         L.ladder_op_prefill_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                              C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ladder_op_prefill_gemm_f16.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                                 C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ladder_op_convert_bf16_f16.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
         L.ladder_op_prefill_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                                   C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                   C.c_void_p, C.c_void_p, C.c_void_p]
@@ -195,8 +199,8 @@ class KVCache:
 
     def __init__(self, shape: ModelShape, max_batch: int, max_seq_len: int, device="cuda", fill: Optional[int] = None):
         n = shape.n_layers * max_batch * shape.n_kv_heads * max_seq_len * shape.head_dim
-        self.k = torch.empty(n, dtype=torch.bfloat16, device=device)
-        self.v = torch.empty(n, dtype=torch.bfloat16, device=device)
+        self.k = torch.empty(n, dtype=torch.float16, device=device)     # binary16: see ladder_kv_cache_t
+        self.v = torch.empty(n, dtype=torch.float16, device=device)
         if fill is not None:       # canary pattern for indexing tests
             self.k.view(torch.int16).fill_(fill)
             self.v.view(torch.int16).fill_(fill)
@@ -346,8 +350,9 @@ def op_decode_attention_noalloc(q, k, v, kv_len, n_q_heads, n_kv_heads, head_dim
 
 
 def set_prefill_gemm_impl(impl: int):
-    """0 = tcgen05 kernel, bf16 hi + lo activations (default); 1 = warp-level mma.sync kernel; 2 = tcgen05 kernel
-    with one bf16 value per activation (half the tensor-core work, plain bf16 precision)."""
+    """Test switch (process-wide).  0 = default (tcgen05, binary16 operands for calls of >= 256 tokens, else bf16
+    pairs); 1 = warp-level mma.sync kernel; 2 = tcgen05, one bf16 value per activation; 3 = tcgen05, bf16 hi + lo
+    pairs at every size."""
     lib().ladder_set_prefill_gemm_impl(impl)
 
 
@@ -361,6 +366,17 @@ def op_prefill_gemm(A, W, epi_mode: int, out, addend=None, A_lo=None, out_lo=Non
     N = W.shape[0]
     _check(lib().ladder_op_prefill_gemm(_ptr(A), _ptr(A_lo), _ptr(W), M, N, K, epi_mode, _ptr(addend), _ptr(out),
                                         _ptr(out_lo), _stream()))
+
+
+def op_prefill_gemm_f16(A, W, epi_mode: int, out, addend=None):
+    """A binary16 [M, K], W binary16 [N, K]; outputs of modes 1 and 3 are binary16."""
+    M, K = A.shape
+    N = W.shape[0]
+    _check(lib().ladder_op_prefill_gemm_f16(_ptr(A), _ptr(W), M, N, K, epi_mode, _ptr(addend), _ptr(out), _stream()))
+
+
+def op_convert_bf16_f16(src, dst):
+    _check(lib().ladder_op_convert_bf16_f16(_ptr(src), _ptr(dst), src.numel(), _stream()))
 
 
 def op_prefill_attention(q, k, v, batch, seq_len, n_q_heads, n_kv_heads, head_dim, max_seq_len, o, q_lo=None,

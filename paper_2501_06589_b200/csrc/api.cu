@@ -83,7 +83,9 @@ struct ladder_model {
   float* logits_ws = nullptr;       // [max_batch, V]
   float* last_x = nullptr;          // [max_batch, d]
   // prefill activations, each a bf16 hi part followed by a lo part (value ~ hi + lo)
-  __nv_bfloat16 *n_pf = nullptr, *q_pf = nullptr, *o_pf = nullptr, *h_pf = nullptr;
+  __nv_bfloat16 *n_pf = nullptr, *o_pf = nullptr, *h_pf = nullptr;
+  __half* q_pf = nullptr;  // the rotated query as the attention's binary16 operand pair
+  __half* w16 = nullptr;   // one layer's four weight matrices as binary16 (prompt pass; NULL: not enough memory)
   size_t n_lo = 0, q_lo = 0, h_lo = 0;  // element offsets of the lo parts
   float2* rope = nullptr;
   int32_t* status = nullptr;
@@ -276,7 +278,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   // SMs (25.1 ms at the best split of 40 SMs vs 24.4 ms): a subset of SMs streams at ~47 GB/s each and
   // the module chain (Wo waits for the previous down projection and vice versa) leaves it idle in
   // between.  Off by default.
-  if (q.two && m->sms_a >= 0 && batch <= 8) {
+  if (q.two && m->sms_a >= 0 && batch <= 4) {
     int ga = m->sms_a;
     if (ga == 0) {
       const double ba = static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh;
@@ -326,8 +328,8 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       p.batch = batch;
       p.epi_mode = EPI_QKV_ROPE;
       p.qkv.q_out_f32 = m->q_f32;
-      p.qkv.k_cache = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
-      p.qkv.v_cache = static_cast<__nv_bfloat16*>(cache->v) + l * layer_elems;
+      p.qkv.k_cache = static_cast<kv_t*>(cache->k) + l * layer_elems;
+      p.qkv.v_cache = static_cast<kv_t*>(cache->v) + l * layer_elems;
       p.qkv.seq_lens = cache->seq_lens;
       p.qkv.rope = m->rope;
       p.qkv.n_q_heads = Hq;
@@ -352,7 +354,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       a.max_len = c.max_seq_len;
       a.scratch = m->attn_scratch;
       a.o = m->o_dec;
-      const bool handover = batch > 8 && m->wide_opack && wide_handover();  // operands pass from kernel to kernel
+      const bool handover = batch > 4 && m->wide_opack && wide_handover();  // operands pass from kernel to kernel
       if (handover) {
         a.o_pack = m->wide_opack;
         a.o_pack_bp = wide_padded_batch(batch);
@@ -397,7 +399,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       p.epi_mode = EPI_SWIGLU;
       p.out = m->h_dec;
       p.status = m->status;
-      const bool handover = batch > 8 && m->wide_hpack && wide_handover();
+      const bool handover = batch > 4 && m->wide_hpack && wide_handover();
       if (handover) p.wide_pack_out = m->wide_hpack;
       q.gemm(1, p, lad);
 
@@ -463,29 +465,50 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
     ++k;
   };
   did(launch_embed(d_tokens, m->tok_embedding, M, d, c.vocab_size, m->R[0], m->status, st, false));
-  // lo parts of the GEMM inputs (activation ~ hi + lo); none when the single-bf16 mode is selected
-  const bool split = !prefill_single_bf16();
+  // Operand precision of the prompt-pass GEMMs.  Default for calls of >= kPrefillF16MinTokens tokens: binary16,
+  // ONE value per activation (11 significant bits) against the layer's weights converted to binary16 once per
+  // call (exact but for magnitudes below 2^-14) -- half the tensor-core work of a bf16 hi + lo pair.  Otherwise
+  // (short chunks, no room for the converted layer, or a mode selected for tests) bf16 hi + lo pairs / single bf16.
+  const bool f16 = prefill_gemm_impl() == 0 && m->w16 && M >= kPrefillF16MinTokens;
+  const bool split = !f16 && !prefill_single_bf16();
   __nv_bfloat16* const n_lo = split ? m->n_pf + m->n_lo : nullptr;
-  __nv_bfloat16* const q_lo = split ? m->q_pf + m->q_lo : nullptr;
+  __half* const q_lo = m->q_pf + m->q_lo;  // the query always goes to the attention as a binary16 pair
   __nv_bfloat16* const o_lo = split ? m->o_pf + m->q_lo : nullptr;
   __nv_bfloat16* const h_lo = split ? m->h_pf + m->h_lo : nullptr;
+  const size_t n_qkv = static_cast<size_t>(Hq + 2 * Hkv) * Dh * d, n_o = static_cast<size_t>(d) * Hq * Dh;
+  const size_t n_gu = 2 * static_cast<size_t>(F) * d, n_dn = static_cast<size_t>(d) * F;
+  __half* const w16_qkv = m->w16;
+  __half* const w16_o = f16 ? w16_qkv + n_qkv : nullptr;
+  __half* const w16_gu = f16 ? w16_o + n_o : nullptr;
+  __half* const w16_dn = f16 ? w16_gu + n_gu : nullptr;
+  auto norm = [&](const float* x, const __nv_bfloat16* gain) {
+    if (f16) did(launch_rmsnorm_f16(x, gain, c.rms_eps, M, d, reinterpret_cast<__half*>(m->n_pf), st));
+    else did(launch_rmsnorm_bf16(x, gain, c.rms_eps, M, d, m->n_pf, n_lo, st));
+  };
   Router rt;
   for (int l = 0; l < c.n_layers; ++l) {
+    if (f16) {  // this layer's weights as binary16 (the previous layer's GEMMs are done with the scratch: same stream)
+      did(launch_convert_bf16_f16(m->w_qkv[l], w16_qkv, n_qkv, st));
+      did(launch_convert_bf16_f16(m->w_o[l], w16_o, n_o, st));
+      did(launch_convert_bf16_f16(m->w_gate_up[l], w16_gu, n_gu, st));
+      did(launch_convert_bf16_f16(m->w_down[l], w16_dn, n_dn, st));
+    }
     {
       const Router::Route r = route(m, rt, 2 * l + 1);
-      did(launch_rmsnorm_bf16(m->R[r.in], m->attn_norm[l], c.rms_eps, M, d, m->n_pf, n_lo, st));
+      norm(m->R[r.in], m->attn_norm[l]);
       LargeMParams p = {};
       p.A = m->n_pf;
       p.A_lo = n_lo;
-      p.W = m->w_qkv[l];
+      p.W = f16 ? reinterpret_cast<const __nv_bfloat16*>(w16_qkv) : m->w_qkv[l];
+      p.f16 = f16;
       p.M = M;
       p.N = (Hq + 2 * Hkv) * Dh;
       p.K = d;
       p.epi_mode = EPI_QKV_ROPE;
-      p.qkv.q_out_bf16 = m->q_pf;
+      p.qkv.q_out_f16 = m->q_pf;
       p.qkv.q_out_lo = q_lo;
-      p.qkv.k_cache = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
-      p.qkv.v_cache = static_cast<__nv_bfloat16*>(cache->v) + l * layer_elems;
+      p.qkv.k_cache = static_cast<kv_t*>(cache->k) + l * layer_elems;
+      p.qkv.v_cache = static_cast<kv_t*>(cache->v) + l * layer_elems;
       p.qkv.rope = m->rope;
       p.qkv.n_q_heads = Hq;
       p.qkv.n_kv_heads = Hkv;
@@ -496,11 +519,12 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       p.status = m->status;
       did(launch_largem_gemm(p, st));
       did(launch_prefill_attention(m->q_pf, q_lo, p.qkv.k_cache, p.qkv.v_cache, batch, S, Hq, Hkv, Dh, c.max_seq_len,
-                                   m->o_pf, o_lo, st, pos0));
+                                   m->o_pf, o_lo, st, pos0, f16));
       LargeMParams o = {};
       o.A = m->o_pf;
       o.A_lo = o_lo;
-      o.W = m->w_o[l];
+      o.W = f16 ? reinterpret_cast<const __nv_bfloat16*>(w16_o) : m->w_o[l];
+      o.f16 = f16;
       o.M = M;
       o.N = d;
       o.K = Hq * Dh;
@@ -512,11 +536,12 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
     }
     {
       const Router::Route r = route(m, rt, 2 * l + 2);
-      did(launch_rmsnorm_bf16(m->R[r.in], mlp_gain(m, l), c.rms_eps, M, d, m->n_pf, n_lo, st));
+      norm(m->R[r.in], mlp_gain(m, l));
       LargeMParams p = {};
       p.A = m->n_pf;
       p.A_lo = n_lo;
-      p.W = m->w_gate_up[l];
+      p.W = f16 ? reinterpret_cast<const __nv_bfloat16*>(w16_gu) : m->w_gate_up[l];
+      p.f16 = f16;
       p.M = M;
       p.N = 2 * F;
       p.K = d;
@@ -528,7 +553,8 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       LargeMParams o = {};
       o.A = m->h_pf;
       o.A_lo = h_lo;
-      o.W = m->w_down[l];
+      o.W = f16 ? reinterpret_cast<const __nv_bfloat16*>(w16_dn) : m->w_down[l];
+      o.f16 = f16;
       o.M = M;
       o.N = d;
       o.K = F;
@@ -735,8 +761,8 @@ bool build_stack(ladder_model* m, const ladder_kv_cache_t* cache, int batch, flo
     const Router::Route rm = route(m, rt, 2 * l + 2);
     if (l < l_begin) continue;  // run by separate kernels before the launch: only the routing state matters
     cur_layer = l;
-    __nv_bfloat16* kc = static_cast<__nv_bfloat16*>(cache->k) + l * layer_elems;
-    __nv_bfloat16* vc = static_cast<__nv_bfloat16*>(cache->v) + l * layer_elems;
+    kv_t* kc = static_cast<kv_t*>(cache->k) + l * layer_elems;
+    kv_t* vc = static_cast<kv_t*>(cache->v) + l * layer_elems;
 
     auto qkv = [&]() {
       SmallMParams p = {};
@@ -1014,7 +1040,7 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   A(dev_alloc(&m->q_f32, MB * qd));
   A(dev_alloc(&m->o_dec, MB * qd));
   A(dev_alloc(&m->h_dec, MB * F));
-  if (c.max_batch > 8) {
+  if (c.max_batch > 4) {
     A(dev_alloc(&m->wide_hpack, 2 * 64 * F));
     A(dev_alloc(&m->wide_opack, 2 * 64 * qd));
   }
@@ -1068,6 +1094,15 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
     ladder_destroy(m);
     return fail(nullptr, LADDER_ERR_OOM, "workspace allocation failed");
   }
+  // Optional: room for one layer's weights as binary16 (the prompt pass then runs its GEMMs with one binary16 value
+  // per activation).  Without it the prompt pass uses bf16 hi + lo pairs: slower, never wrong.
+  if (c.max_prefill_tokens >= kPrefillF16MinTokens) {
+    const size_t layer_elems = (static_cast<size_t>(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim + qd + 3 * F) * d;
+    if (dev_alloc(&m->w16, layer_elems) != cudaSuccess) {
+      cudaGetLastError();
+      m->w16 = nullptr;
+    }
+  }
   // rotary table in double precision: angle = p * theta^(-2j/Dh)
   {
     const int half = c.head_dim / 2;
@@ -1108,7 +1143,7 @@ ladder_status_t ladder_destroy(ladder_model_t* m) {
   if (m->ev_join) cudaEventDestroy(m->ev_join);
   if (m->side) cudaStreamDestroy(m->side);
   if (m->cap) cudaStreamDestroy(m->cap);
-  void* bufs[] = {m->wide_hpack, m->wide_opack, m->xpack[0], m->xpack[1], m->hpack, m->opack, m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
+  void* bufs[] = {m->w16, m->wide_hpack, m->wide_opack, m->xpack[0], m->xpack[1], m->hpack, m->opack, m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
                   m->n_pf, m->q_pf,  m->o_pf,  m->h_pf,  m->rope,  m->status,       m->tok_tmp,   m->next_tmp};
   for (void* b : bufs)
     if (b) cudaFree(b);
@@ -1306,7 +1341,7 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const bool two = m->n_streams == 2;
 
-  if (m->use_stack && m->stack_ok && batch <= 8) {
+  if (m->use_stack && m->stack_ok && batch <= 4) {
     GraphKey key;
     key.batch = batch;
     key.k = cache->k;
@@ -1515,8 +1550,8 @@ ladder_status_t ladder_op_decode_attention(const float* q, const void* k, const 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   DecodeAttnParams a = {};
   a.q = q;
-  a.k = static_cast<const __nv_bfloat16*>(k);
-  a.v = static_cast<const __nv_bfloat16*>(v);
+  a.k = static_cast<const kv_t*>(k);
+  a.v = static_cast<const kv_t*>(v);
   a.kv_len = kv_len;
   a.kv_len_offset = 0;
   a.batch = batch;
@@ -1559,6 +1594,43 @@ ladder_status_t ladder_op_prefill_gemm(const void* A, const void* A_lo, const vo
   return launch_largem_gemm(p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
 }
 
+ladder_status_t ladder_op_convert_bf16_f16(const void* src, void* dst, int64_t n, void* cuda_stream) {
+  if (!src || !dst || n < 8 || (n % 8)) return LADDER_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) return LADDER_ERR_INVALID_ARG;
+  return launch_convert_bf16_f16(static_cast<const __nv_bfloat16*>(src), static_cast<__half*>(dst),
+                                 static_cast<size_t>(n), static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? LADDER_OK
+             : LADDER_ERR_CUDA;
+}
+
+ladder_status_t ladder_op_prefill_gemm_f16(const void* A, const void* W, int32_t M, int32_t N, int32_t K, int32_t epi_mode,
+                                           const float* addend, void* out, void* cuda_stream) {
+  if (!A || !W || !out || M < 1 || N < 8 || K < 8 || (N % 8) || (K % 8)) return LADDER_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(W) | reinterpret_cast<uintptr_t>(out)) & 15)
+    return LADDER_ERR_INVALID_ARG;
+  int mode;
+  switch (epi_mode) {
+    case 0: mode = EPI_RESID; break;
+    case 1: mode = EPI_SWIGLU; break;
+    case 2: mode = EPI_PLAIN; break;
+    case 3: mode = EPI_BF16; break;
+    default: return LADDER_ERR_INVALID_ARG;
+  }
+  if (mode == EPI_RESID && !addend) return LADDER_ERR_INVALID_ARG;
+  LargeMParams p = {};
+  p.A = static_cast<const __nv_bfloat16*>(A);
+  p.W = static_cast<const __nv_bfloat16*>(W);
+  p.f16 = 1;
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  p.epi_mode = mode;
+  p.addend = addend;
+  p.out = out;
+  if (kernels_ready() != cudaSuccess) return LADDER_ERR_CUDA;
+  return launch_largem_gemm(p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
+}
+
 ladder_status_t ladder_op_prefill_attention(const void* q, const void* q_lo, const void* k, const void* v, int32_t batch,
                                             int32_t seq_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
                                             int32_t max_seq_len, void* o, void* o_lo, void* cuda_stream) {
@@ -1568,8 +1640,8 @@ ladder_status_t ladder_op_prefill_attention(const void* q, const void* q_lo, con
   if (kernels_ready() != cudaSuccess) return LADDER_ERR_CUDA;
   if ((q_lo == nullptr) != (o_lo == nullptr)) return LADDER_ERR_INVALID_ARG;
   cudaError_t e = launch_prefill_attention(
-      static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(q_lo), static_cast<const __nv_bfloat16*>(k),
-      static_cast<const __nv_bfloat16*>(v), batch, seq_len, n_q_heads, n_kv_heads, head_dim, max_seq_len,
+      static_cast<const __half*>(q), static_cast<const __half*>(q_lo), static_cast<const kv_t*>(k),
+      static_cast<const kv_t*>(v), batch, seq_len, n_q_heads, n_kv_heads, head_dim, max_seq_len,
       static_cast<__nv_bfloat16*>(o), static_cast<__nv_bfloat16*>(o_lo), static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
 }

@@ -5,12 +5,12 @@
 // of GT query heads sharing a kv head, sequence); each of its 4 warps owns 16 keys and issues ALL of
 // its loads -- q, 16 key rows as MMA fragments, 16 value rows -- before the first dependent
 // instruction, so the whole CTA costs about one memory round trip plus one merge.
-//   1. scores: mma.sync with Q (padded to 16 rows, bf16 hi + lo pair so the fp32 query loses
+//   1. scores: mma.sync with Q (padded to 16 rows, binary16 hi + lo pair so the fp32 query loses
 //      nothing) as the A operand and key rows read straight from the cache as B fragments (the
 //      contraction index is permuted identically on both sides: 16 contiguous bytes per thread);
 //   2. fp32 softmax statistics per warp, probabilities to shared memory;
 //   3. P.V on the CUDA cores in fp32 from the value rows already in registers (batch <= 8), or on mma.sync
-//      with the probabilities as a bf16 hi + lo pair (batch > 8: see PVMMA below);
+//      with the probabilities as a binary16 hi + lo pair (batch > 8: see PVMMA below);
 //   4. the 4 warps are merged by log-sum-exp in shared memory and the CTA's (o, m, l) partial goes
 //      to an L2-resident scratch; a second, tiny kernel (one CTA per sequence and head, launched
 //      with programmatic dependent launch) merges the splits in a fixed order and writes o in fp32.
@@ -27,7 +27,7 @@ constexpr int kChunk = 64;  // keys per CTA (16 per warp)
 
 // PVMMA (used for batch > 8, where the step stops being latency-bound and this kernel became issue-bound on its
 // CUDA-core P.V loop: 65 % issue-slot use at 2.7 TB/s): P.V runs on mma.sync too.  The probabilities of head g
-// are already laid out as the A fragment (the score MMA's C fragment, as a bf16 hi + lo pair), and a lane reads
+// are already laid out as the A fragment (the score MMA's C fragment, as a binary16 hi + lo pair), and a lane reads
 // the value rows as 32-bit words V[key][16 j + 2 g, +1] for its four keys 2t, 2t+1, 2t+8, 2t+9, so that two byte
 // permutes turn them into the B fragments of an "even dims" and an "odd dims" MMA per 16 dims.
 template <int GT, int DH, bool PVMMA>
@@ -46,8 +46,8 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
   const int group = p.n_q_heads / p.n_kv_heads;
   const int kvh = head0 / group;
   const size_t kv_base = (static_cast<size_t>(b) * p.n_kv_heads + kvh) * p.max_seq_len * DH;
-  const __nv_bfloat16* K = p.k + kv_base;
-  const __nv_bfloat16* V = p.v + kv_base;
+  const kv_t* K = p.k + kv_base;
+  const kv_t* V = p.v + kv_base;
 
   pdl_launch_dependents();
   pdl_wait();
@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
       vr[i][0] = key < L ? *reinterpret_cast<const uint32_t*>(V + static_cast<size_t>(key) * DH + lane * DPL) : 0u;
     }
   }
-  // q as a bf16 hi + lo pair: [j][half][pair] covers q[head0+g][j*32 + tig*8 + half*4 + 2*pair ..+1]
+  // q as a binary16 hi + lo pair (the keys' type): [j][half][pair] covers q[head0+g][j*32 + tig*8 + half*4 + 2*pair ..+1]
   uint32_t qa[KJ][2][2], ql[KJ][2][2];
 #pragma unroll
   for (int j = 0; j < KJ; ++j)
@@ -102,10 +102,10 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
       if (g < GT)
         v = *reinterpret_cast<const float4*>(p.q + (static_cast<size_t>(b) * p.n_q_heads + head0 + g) * DH + j * 32 +
                                              tig * 8 + h * 4);
-      qa[j][h][0] = pack_bf16x2(v.x, v.y);
-      qa[j][h][1] = pack_bf16x2(v.z, v.w);
-      ql[j][h][0] = pack_bf16x2(v.x - bf16_lo(qa[j][h][0]), v.y - bf16_hi(qa[j][h][0]));
-      ql[j][h][1] = pack_bf16x2(v.z - bf16_lo(qa[j][h][1]), v.w - bf16_hi(qa[j][h][1]));
+      qa[j][h][0] = pack_f16x2(v.x, v.y);
+      qa[j][h][1] = pack_f16x2(v.z, v.w);
+      ql[j][h][0] = pack_f16x2(v.x - f16_lo(qa[j][h][0]), v.y - f16_hi(qa[j][h][0]));
+      ql[j][h][1] = pack_f16x2(v.z - f16_lo(qa[j][h][1]), v.w - f16_hi(qa[j][h][1]));
     }
 
   // ---- 1. scores of this warp's 16 keys: c[nt][0..1] = (head g, keys nt*8 + 2*tig, +1)
@@ -115,10 +115,10 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
     c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
 #pragma unroll
     for (int j = 0; j < KJ; ++j) {
-      mma_bf16_16816(c[nt], qa[j][0][0], 0u, qa[j][0][1], 0u, kf[nt][j].x, kf[nt][j].y);
-      mma_bf16_16816(c[nt], qa[j][1][0], 0u, qa[j][1][1], 0u, kf[nt][j].z, kf[nt][j].w);
-      mma_bf16_16816(c[nt], ql[j][0][0], 0u, ql[j][0][1], 0u, kf[nt][j].x, kf[nt][j].y);
-      mma_bf16_16816(c[nt], ql[j][1][0], 0u, ql[j][1][1], 0u, kf[nt][j].z, kf[nt][j].w);
+      mma_f16_16816(c[nt], qa[j][0][0], 0u, qa[j][0][1], 0u, kf[nt][j].x, kf[nt][j].y);
+      mma_f16_16816(c[nt], qa[j][1][0], 0u, qa[j][1][1], 0u, kf[nt][j].z, kf[nt][j].w);
+      mma_f16_16816(c[nt], ql[j][0][0], 0u, ql[j][0][1], 0u, kf[nt][j].x, kf[nt][j].y);
+      mma_f16_16816(c[nt], ql[j][1][0], 0u, ql[j][1][1], 0u, kf[nt][j].z, kf[nt][j].w);
     }
   }
   // ---- 2. softmax statistics of head g over the warp's keys (quad reduction)
@@ -156,9 +156,9 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
 
   if constexpr (PVMMA) {
     // ---- 3. P.V on the tensor cores: A = probabilities of (head g; keys 2t, 2t+1 | 2t+8, 2t+9), hi + lo
-    const uint32_t ph0 = pack_bf16x2(sv[0], sv[1]), ph1 = pack_bf16x2(sv[2], sv[3]);
-    const uint32_t pl0 = pack_bf16x2(sv[0] - bf16_lo(ph0), sv[1] - bf16_hi(ph0));
-    const uint32_t pl1 = pack_bf16x2(sv[2] - bf16_lo(ph1), sv[3] - bf16_hi(ph1));
+    const uint32_t ph0 = pack_f16x2(sv[0], sv[1]), ph1 = pack_f16x2(sv[2], sv[3]);
+    const uint32_t pl0 = pack_f16x2(sv[0] - f16_lo(ph0), sv[1] - f16_hi(ph0));
+    const uint32_t pl1 = pack_f16x2(sv[2] - f16_lo(ph1), sv[3] - f16_hi(ph1));
 #pragma unroll
     for (int j = 0; j < DH / 16; ++j) {
       uint32_t w[4];
@@ -171,10 +171,10 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
       const uint32_t be0 = __byte_perm(w[0], w[1], 0x5410), be1 = __byte_perm(w[2], w[3], 0x5410);
       const uint32_t bo0 = __byte_perm(w[0], w[1], 0x7632), bo1 = __byte_perm(w[2], w[3], 0x7632);
       float ce[4] = {0.f, 0.f, 0.f, 0.f}, co[4] = {0.f, 0.f, 0.f, 0.f};
-      mma_bf16_16816(ce, ph0, 0u, ph1, 0u, be0, be1);
-      mma_bf16_16816(ce, pl0, 0u, pl1, 0u, be0, be1);
-      mma_bf16_16816(co, ph0, 0u, ph1, 0u, bo0, bo1);
-      mma_bf16_16816(co, pl0, 0u, pl1, 0u, bo0, bo1);
+      mma_f16_16816(ce, ph0, 0u, ph1, 0u, be0, be1);
+      mma_f16_16816(ce, pl0, 0u, pl1, 0u, be0, be1);
+      mma_f16_16816(co, ph0, 0u, ph1, 0u, bo0, bo1);
+      mma_f16_16816(co, pl0, 0u, pl1, 0u, bo0, bo1);
       // columns 2 tig, 2 tig + 1 of the two MMAs = dims 16 j + 4 tig .. + 3 of head g
       if (g < GT) *reinterpret_cast<float4*>(&red[warp][g][16 * j + 4 * tig]) = make_float4(ce[0], co[0], ce[1], co[1]);
     }
@@ -196,11 +196,11 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attention_kernel(const De
     for (int e = 0; e < 4; ++e) {
       const int i = i4 * 4 + e;
       float v[DPL];
-      v[0] = bf16_lo(vr[i][0]);
-      v[1] = bf16_hi(vr[i][0]);
+      v[0] = f16_lo(vr[i][0]);
+      v[1] = f16_hi(vr[i][0]);
       if (DPL == 4) {
-        v[DPL - 2] = bf16_lo(vr[i][DPL / 2 - 1]);
-        v[DPL - 1] = bf16_hi(vr[i][DPL / 2 - 1]);
+        v[DPL - 2] = f16_lo(vr[i][DPL / 2 - 1]);
+        v[DPL - 1] = f16_hi(vr[i][DPL / 2 - 1]);
       }
 #pragma unroll
       for (int h = 0; h < GT; ++h) {
@@ -417,8 +417,8 @@ extern "C" ladder_status_t ladder_op_decode_attention_noalloc(const float* q, co
   if (noalloc_scratch(&scratch) != cudaSuccess) return LADDER_ERR_CUDA;
   DecodeAttnParams a = {};
   a.q = q;
-  a.k = static_cast<const __nv_bfloat16*>(k);
-  a.v = static_cast<const __nv_bfloat16*>(v);
+  a.k = static_cast<const kv_t*>(k);
+  a.v = static_cast<const kv_t*>(v);
   a.kv_len = kv_len;
   a.kv_len_offset = 0;
   a.batch = batch;

@@ -563,8 +563,9 @@ cudaError_t smallm_gemm_init() {
 }
 
 size_t smallm_gemm_smem_bytes(int batch) {
-  if (batch <= 8) return SMEM;
-  return std::max(smallm_gemm_wide_smem_bytes(batch), smallm_gemm_wide_tc_smem_bytes(batch));
+  if (batch <= 4) return SMEM;
+  const size_t wide = std::max(smallm_gemm_wide_smem_bytes(batch > 8 ? batch : 9), smallm_gemm_wide_tc_smem_bytes(batch));
+  return std::max(wide, static_cast<size_t>(SMEM));
 }
 
 size_t smallm_gemm_scratch_floats(int N, int K, int batch) {
@@ -573,9 +574,11 @@ size_t smallm_gemm_scratch_floats(int N, int K, int batch) {
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
   if (g_wide_impl == 2) return launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count);
-  if (p.batch > 8)
-    return g_wide_impl == 0 ? launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count)
-                            : launch_smallm_gemm_wide(p, stream, pdl, sm_count);
+  // Batch 5..8 on the tcgen05 kernel by default: this file's kernel holds a bf16 hi + lo activation pair only for
+  // batch <= 4 (one 8-column MMA tile) and would run 5..8 with a single bf16 value, which costs a decimal digit of
+  // hidden-state accuracy.  With the mma.sync cross-check selected (impl 1) they still run here.
+  if (p.batch > 4 && g_wide_impl == 0) return launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count);
+  if (p.batch > 8) return launch_smallm_gemm_wide(p, stream, pdl, sm_count);
   if (!p.work) return cudaErrorInvalidValue;
   const int units = p.N >> 3;
   const int grid = units < sm_count ? units : sm_count;

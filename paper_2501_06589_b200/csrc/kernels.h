@@ -10,16 +10,20 @@
 
 namespace ladder {
 
+// Element type of the KV cache: IEEE binary16.  Keys and values of a normalised-input projection are O(1), far inside
+// its range, and its 11 significant bits (bf16: 8) are what keeps the hidden-state error of deep models in bound.
+typedef __half kv_t;
+
 enum ActMode { ACT_F32 = 0, ACT_F32_NORM = 1 };  // activations are fp32 [batch, K]; NORM applies RMSNorm
 enum EpiMode { EPI_RESID = 0, EPI_SWIGLU = 1, EPI_PLAIN = 2, EPI_QKV_ROPE = 3, EPI_BF16 = 4 };
 
 // Rotary / KV-append epilogue description shared by the decode and prefill QKV projections.
 struct QkvEpilogue {
   float* q_out_f32;            // decode: fp32 [batch, Hq*Dh]
-  __nv_bfloat16* q_out_bf16;   // prefill: bf16 [M, Hq*Dh] (hi part)
-  __nv_bfloat16* q_out_lo;     // prefill: lo part (q ~ hi + lo), may be NULL
-  __nv_bfloat16* k_cache;      // one layer: [max_batch][Hkv][max_seq][Dh]
-  __nv_bfloat16* v_cache;
+  __half* q_out_f16;           // prefill: binary16 [M, Hq*Dh] (hi part; the attention's MMA operand type)
+  __half* q_out_lo;            // prefill: lo part (q ~ hi + lo), may be NULL
+  kv_t* k_cache;               // one layer: [max_batch][Hkv][max_seq][Dh]
+  kv_t* v_cache;
   const int32_t* seq_lens;     // decode: position of row b = seq_lens[b]; prefill: NULL (position = m % seq_len)
   const float2* rope;          // [max_seq][Dh/2] (cos, sin)
   int n_q_heads, n_kv_heads, head_dim, max_seq_len;
@@ -64,8 +68,8 @@ void set_decode_wide_impl(int impl);  // batch 9..64: 0 = tcgen05 (default), 1 =
 // Decode attention (split over the cache) and its combine step.
 struct DecodeAttnParams {
   const float* q;               // [batch, Hq*Dh]
-  const __nv_bfloat16* k;       // one layer
-  const __nv_bfloat16* v;
+  const kv_t* k;                // one layer
+  const kv_t* v;
   const int32_t* kv_len;        // [batch]
   int kv_len_offset;            // keys attended = kv_len[b] + kv_len_offset (decode passes seq_lens and 1)
   int batch, n_q_heads, n_kv_heads, head_dim, max_seq_len;
@@ -164,26 +168,38 @@ struct LargeMParams {
   __nv_bfloat16* out_lo;   // EPI_SWIGLU / EPI_BF16: lo part of the bf16 output, or NULL
   QkvEpilogue qkv;
   int32_t* status;         // device status word (may be NULL)
+  int f16;                 // A and W hold binary16 instead of bf16 (one value per activation, A_lo unused), and the
+                           // 16-bit outputs (EPI_SWIGLU, EPI_BF16) are written as binary16 too; tcgen05 kernel only
 };
 // Dispatches to the tcgen05 kernel (default) or the warp-level mma.sync kernel (set_prefill_gemm_impl(1)).
 cudaError_t launch_largem_gemm(const LargeMParams& p, cudaStream_t stream);
 cudaError_t launch_largem_gemm_tc(const LargeMParams& p, cudaStream_t stream, int sm_count);
 cudaError_t largem_gemm_tc_init();
-void set_prefill_gemm_impl(int impl);  // 0 = tcgen05 (default), 1 = mma.sync, 2 = tcgen05 with single-bf16 activations
+// 0 = default: tcgen05 with binary16 operands (one value per activation, the layer's weights converted once per
+// call) for calls of at least kPrefillF16MinTokens tokens, bf16 hi + lo pairs below; 1 = mma.sync (pairs);
+// 2 = tcgen05 with single-bf16 activations; 3 = tcgen05 with bf16 hi + lo pairs at every size
+void set_prefill_gemm_impl(int impl);
+int prefill_gemm_impl();
+constexpr int kPrefillF16MinTokens = 256;
 bool prefill_single_bf16();            // the prompt pass feeds its GEMMs one bf16 value per activation (no lo part)
 
 // q_lo / o_lo: optional lo parts (value ~ hi + lo) of the query input and the attention output.
+// out_f16: o receives ONE binary16 value per element instead of a bf16 value (o_lo must be NULL).
 // pos0: the seq_len queries sit at positions pos0 .. pos0 + seq_len - 1 and attend to cache rows 0 .. their own.
-cudaError_t launch_prefill_attention(const __nv_bfloat16* q, const __nv_bfloat16* q_lo, const __nv_bfloat16* k,
-                                     const __nv_bfloat16* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
+cudaError_t launch_prefill_attention(const __half* q, const __half* q_lo, const kv_t* k,
+                                     const kv_t* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
                                      int head_dim, int max_seq_len, __nv_bfloat16* o, __nv_bfloat16* o_lo,
-                                     cudaStream_t stream, int pos0 = 0);
+                                     cudaStream_t stream, int pos0 = 0, bool out_f16 = false);
 
 // Small element-wise / gather kernels.
 cudaError_t launch_embed(const int32_t* tokens, const __nv_bfloat16* table, int rows, int d, int vocab, float* x,
                          int32_t* status, cudaStream_t stream, bool pdl);
 cudaError_t launch_rmsnorm_bf16(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d,
                                 __nv_bfloat16* out, __nv_bfloat16* out_lo, cudaStream_t stream);
+cudaError_t launch_rmsnorm_f16(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, __half* out,
+                               cudaStream_t stream);
+// n elements, n % 8 == 0, both pointers 16-byte aligned
+cudaError_t launch_convert_bf16_f16(const __nv_bfloat16* src, __half* dst, size_t n, cudaStream_t stream);
 cudaError_t launch_rmsnorm_f32(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, int row_stride,
                                float* out, cudaStream_t stream, bool pdl);
 cudaError_t launch_gather_rows(const float* x, int rows, int d, int src_stride_rows, int src_offset_rows, float* out,

@@ -85,6 +85,40 @@ __global__ void rmsnorm_kernel(const float* x, const __nv_bfloat16* gain, float 
   }
 }
 
+// The same normalisation written as ONE binary16 value per element (the operand of the binary16 prompt-pass GEMMs).
+__global__ void rmsnorm_f16_kernel(const float* x, const __nv_bfloat16* gain, float eps, int d, __half* out) {
+  __shared__ float sh[32];
+  const float* xr = x + static_cast<size_t>(blockIdx.x) * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
+    const float4 v = reinterpret_cast<const float4*>(xr)[i];
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  const float rstd = rsqrtf(block_sum(ss, sh) / static_cast<float>(d) + eps);
+  __half* o = out + static_cast<size_t>(blockIdx.x) * d;
+  for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
+    const float4 v = reinterpret_cast<const float4*>(xr)[i];
+    const uint2 gq = __ldg(reinterpret_cast<const uint2*>(gain) + i);
+    reinterpret_cast<uint2*>(o)[i] = make_uint2(pack_kv(v.x * rstd * bf16_lo(gq.x), v.y * rstd * bf16_hi(gq.x)),
+                                                pack_kv(v.z * rstd * bf16_lo(gq.y), v.w * rstd * bf16_hi(gq.y)));
+  }
+}
+
+// bf16 -> binary16, eight elements per thread and iteration.  Exact for |w| >= 2^-14 (binary16 has three more
+// significant bits than bf16); smaller magnitudes land on binary16's subnormal grid, at most 2^-25 away.
+__global__ void convert_bf16_f16_kernel(const uint4* src, uint4* dst, size_t n8) {
+  for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n8;
+       i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const uint4 v = __ldcs(src + i);
+    uint4 o;
+    o.x = pack_f16x2(bf16_lo(v.x), bf16_hi(v.x));
+    o.y = pack_f16x2(bf16_lo(v.y), bf16_hi(v.y));
+    o.z = pack_f16x2(bf16_lo(v.z), bf16_hi(v.z));
+    o.w = pack_f16x2(bf16_lo(v.w), bf16_hi(v.w));
+    dst[i] = o;
+  }
+}
+
 // out[r, :] = x[(r * stride + offset), :]
 __global__ void gather_rows_kernel(const float* x, int d, int stride, int offset, float* out) {
   const float4* src = reinterpret_cast<const float4*>(x + (static_cast<size_t>(blockIdx.x) * stride + offset) * d);
@@ -173,6 +207,19 @@ cudaError_t launch_embed(const int32_t* tokens, const __nv_bfloat16* table, int 
 cudaError_t launch_rmsnorm_bf16(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d,
                                 __nv_bfloat16* out, __nv_bfloat16* out_lo, cudaStream_t stream) {
   return launch(rmsnorm_kernel<__nv_bfloat16>, dim3(rows), dim3(256), stream, false, x, gain, eps, d, d, out, out_lo);
+}
+
+cudaError_t launch_rmsnorm_f16(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, __half* out,
+                               cudaStream_t stream) {
+  return launch(rmsnorm_f16_kernel, dim3(rows), dim3(256), stream, false, x, gain, eps, d, out);
+}
+
+cudaError_t launch_convert_bf16_f16(const __nv_bfloat16* src, __half* dst, size_t n, cudaStream_t stream) {
+  if (n % 8 || ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15)) return cudaErrorInvalidValue;
+  const size_t n8 = n / 8;
+  const size_t blocks = (n8 + 255) / 256;
+  return launch(convert_bf16_f16_kernel, dim3(static_cast<unsigned>(blocks < 148 * 16 ? (blocks ? blocks : 1) : 148 * 16)),
+                dim3(256), stream, false, reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), n8);
 }
 
 cudaError_t launch_rmsnorm_f32(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, int row_stride,

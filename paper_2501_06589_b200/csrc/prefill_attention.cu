@@ -3,7 +3,9 @@
 // One CTA per (64-query tile, query head, sequence); 4 warps of 16 query rows.  K/V tiles of 64
 // keys are staged in shared memory with cp.async straight from the KV cache the QKV epilogue
 // just filled; S = Q K^T and O += P V run on mma.sync m16n8k16 with fp32 online softmax in
-// registers.  Query p attends keys t <= p; query head h uses kv head h / (Hq / Hkv).
+// registers.  Query p attends keys t <= p; query head h uses kv head h / (Hq / Hkv).  The cache holds binary16
+// keys and values, so the query (hi + lo pair) and the probabilities enter the MMAs as binary16 too; the output
+// leaves as a bf16 hi + lo pair, the operand type of the output projection.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -27,28 +29,29 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
                : "r"(addr));
 }
 
-// SPLIT: the query comes as a bf16 hi + lo pair and the output is written as one (value ~ hi + lo).
+// SPLIT: the query comes as a binary16 hi + lo pair and the output is written as a bf16 one (value ~ hi + lo).
 template <int DH, bool SPLIT>
-__global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __nv_bfloat16* __restrict__ q,
-                                                                       const __nv_bfloat16* __restrict__ q_lo,
-                                                                       const __nv_bfloat16* __restrict__ kc,
-                                                                       const __nv_bfloat16* __restrict__ vc, int seq_len,
+__global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __half* __restrict__ q,
+                                                                       const __half* __restrict__ q_lo,
+                                                                       const kv_t* __restrict__ kc,
+                                                                       const kv_t* __restrict__ vc, int seq_len,
                                                                        int n_q_heads, int n_kv_heads, int max_seq_len,
                                                                        __nv_bfloat16* __restrict__ o,
-                                                                       __nv_bfloat16* __restrict__ o_lo, const int pos0) {
+                                                                       __nv_bfloat16* __restrict__ o_lo, const int pos0,
+                                                                       const int out_f16) {
   constexpr int P = DH + 8;  // smem pitch in elements
   extern __shared__ __align__(128) uint8_t smem_raw[];
-  __nv_bfloat16* sQ = reinterpret_cast<__nv_bfloat16*>(smem_raw);
-  __nv_bfloat16* sK = sQ + kQT * P;
-  __nv_bfloat16* sV = sK + kKT * P;
-  __nv_bfloat16* sQl = sV + kKT * P;
+  __half* sQ = reinterpret_cast<__half*>(smem_raw);
+  __half* sK = sQ + kQT * P;
+  __half* sV = sK + kKT * P;
+  __half* sQl = sV + kKT * P;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, tig = lane & 3;
   const int q0 = blockIdx.x * kQT, h = blockIdx.y, b = blockIdx.z;
   const int kvh = h / (n_q_heads / n_kv_heads);
   const size_t qrow_stride = static_cast<size_t>(n_q_heads) * DH;
-  const __nv_bfloat16* kg = kc + (static_cast<size_t>(b) * n_kv_heads + kvh) * max_seq_len * DH;
-  const __nv_bfloat16* vg = vc + (static_cast<size_t>(b) * n_kv_heads + kvh) * max_seq_len * DH;
+  const kv_t* kg = kc + (static_cast<size_t>(b) * n_kv_heads + kvh) * max_seq_len * DH;
+  const kv_t* vg = vc + (static_cast<size_t>(b) * n_kv_heads + kvh) * max_seq_len * DH;
   constexpr int CPR = DH / 8;  // 16-byte chunks per row
 
   for (int i = tid; i < kQT * CPR; i += kPfThreads) {
@@ -101,11 +104,11 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
       for (int j = 0; j < 4; ++j) {
         uint32_t b0, b1, b2, b3;
         ldsm_x4(smem_u32(sK + (j * 16 + (lane & 7) + (lane >> 4) * 8) * P + ks + ((lane >> 3) & 1) * 8), b0, b1, b2, b3);
-        mma_bf16_16816(s[2 * j], a0, a1, a2, a3, b0, b1);
-        mma_bf16_16816(s[2 * j + 1], a0, a1, a2, a3, b2, b3);
+        mma_f16_16816(s[2 * j], a0, a1, a2, a3, b0, b1);
+        mma_f16_16816(s[2 * j + 1], a0, a1, a2, a3, b2, b3);
         if (SPLIT) {
-          mma_bf16_16816(s[2 * j], l0, l1, l2, l3, b0, b1);
-          mma_bf16_16816(s[2 * j + 1], l0, l1, l2, l3, b2, b3);
+          mma_f16_16816(s[2 * j], l0, l1, l2, l3, b0, b1);
+          mma_f16_16816(s[2 * j + 1], l0, l1, l2, l3, b2, b3);
         }
       }
     }
@@ -155,17 +158,17 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
     // O += P V
 #pragma unroll
     for (int kk = 0; kk < kKT / 16; ++kk) {
-      const uint32_t a0 = pack_bf16x2(s[2 * kk][0], s[2 * kk][1]);
-      const uint32_t a1 = pack_bf16x2(s[2 * kk][2], s[2 * kk][3]);
-      const uint32_t a2 = pack_bf16x2(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-      const uint32_t a3 = pack_bf16x2(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+      const uint32_t a0 = pack_f16x2(s[2 * kk][0], s[2 * kk][1]);
+      const uint32_t a1 = pack_f16x2(s[2 * kk][2], s[2 * kk][3]);
+      const uint32_t a2 = pack_f16x2(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+      const uint32_t a3 = pack_f16x2(s[2 * kk + 1][2], s[2 * kk + 1][3]);
 #pragma unroll
       for (int d = 0; d < DH / 16; ++d) {
         uint32_t b0, b1, b2, b3;
         ldsm_x4_t(smem_u32(sV + (kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * P + d * 16 + (lane >> 4) * 8), b0, b1,
                   b2, b3);
-        mma_bf16_16816(oacc[2 * d], a0, a1, a2, a3, b0, b1);
-        mma_bf16_16816(oacc[2 * d + 1], a0, a1, a2, a3, b2, b3);
+        mma_f16_16816(oacc[2 * d], a0, a1, a2, a3, b0, b1);
+        mma_f16_16816(oacc[2 * d + 1], a0, a1, a2, a3, b2, b3);
       }
     }
   }
@@ -185,6 +188,10 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
 #pragma unroll
     for (int i = 0; i < DH / 8; ++i) {
       const float v0 = oacc[i][2 * r] * inv, v1 = oacc[i][2 * r + 1] * inv;
+      if (out_f16) {  // one binary16 value per element: the operand of the binary16 output projection
+        *reinterpret_cast<uint32_t*>(o + doff + i * 8 + tig * 2) = pack_f16x2(v0, v1);
+        continue;
+      }
       const uint32_t hi = pack_bf16x2(v0, v1);
       *reinterpret_cast<uint32_t*>(o + doff + i * 8 + tig * 2) = hi;
       if (SPLIT) *reinterpret_cast<uint32_t*>(o_lo + doff + i * 8 + tig * 2) = pack_bf16x2(v0 - bf16_lo(hi), v1 - bf16_hi(hi));
@@ -193,13 +200,13 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __n
 }
 
 template <int DH, bool SPLIT>
-cudaError_t launch_dh(const __nv_bfloat16* q, const __nv_bfloat16* q_lo, const __nv_bfloat16* k, const __nv_bfloat16* v,
+cudaError_t launch_dh(const __half* q, const __half* q_lo, const kv_t* k, const kv_t* v,
                       int batch, int seq_len, int n_q_heads, int n_kv_heads, int max_seq_len, __nv_bfloat16* o,
-                      __nv_bfloat16* o_lo, cudaStream_t stream, int pos0) {
+                      __nv_bfloat16* o_lo, cudaStream_t stream, int pos0, int out_f16) {
   constexpr int smem = 4 * 64 * (DH + 8) * 2;
   dim3 grid((seq_len + kQT - 1) / kQT, n_q_heads, batch);
   prefill_attention_kernel<DH, SPLIT><<<grid, kPfThreads, smem, stream>>>(q, q_lo, k, v, seq_len, n_q_heads, n_kv_heads,
-                                                                          max_seq_len, o, o_lo, pos0);
+                                                                          max_seq_len, o, o_lo, pos0, out_f16);
   return cudaGetLastError();
 }
 
@@ -219,18 +226,20 @@ cudaError_t prefill_attention_init() {
   return e;
 }
 
-cudaError_t launch_prefill_attention(const __nv_bfloat16* q, const __nv_bfloat16* q_lo, const __nv_bfloat16* k,
-                                     const __nv_bfloat16* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
+cudaError_t launch_prefill_attention(const __half* q, const __half* q_lo, const kv_t* k,
+                                     const kv_t* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
                                      int head_dim, int max_seq_len, __nv_bfloat16* o, __nv_bfloat16* o_lo,
-                                     cudaStream_t stream, int pos0) {
-  const bool split = q_lo != nullptr && o_lo != nullptr;
+                                     cudaStream_t stream, int pos0, bool out_f16) {
+  const bool split = q_lo != nullptr && (o_lo != nullptr || out_f16);
+  if (out_f16 && o_lo) return cudaErrorInvalidValue;
+  const int of = out_f16 ? 1 : 0;
   if (pos0 < 0 || pos0 + seq_len > max_seq_len) return cudaErrorInvalidValue;
   if (head_dim == 128)
-    return split ? launch_dh<128, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0)
-                 : launch_dh<128, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0);
+    return split ? launch_dh<128, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of)
+                 : launch_dh<128, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of);
   if (head_dim == 64)
-    return split ? launch_dh<64, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0)
-                 : launch_dh<64, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0);
+    return split ? launch_dh<64, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of)
+                 : launch_dh<64, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of);
   return cudaErrorInvalidValue;
 }
 

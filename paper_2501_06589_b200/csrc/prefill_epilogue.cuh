@@ -18,6 +18,10 @@ __device__ __forceinline__ void epilogue_pair(const LargeMParams& p, int m, int 
     case EPI_SWIGLU: {
       const float h = v0 / (1.f + __expf(-v0)) * v1;
       const size_t o = static_cast<size_t>(m) * (p.N >> 1) + (n >> 1);
+      if (p.f16) {  // one binary16 value, saturating
+        static_cast<__half*>(p.out)[o] = __float2half_rn(fminf(fmaxf(h, -65504.f), 65504.f));
+        break;
+      }
       const __nv_bfloat16 hi = __float2bfloat16_rn(h);
       static_cast<__nv_bfloat16*>(p.out)[o] = hi;
       if (p.out_lo) p.out_lo[o] = __float2bfloat16_rn(h - __bfloat162float(hi));
@@ -28,6 +32,10 @@ __device__ __forceinline__ void epilogue_pair(const LargeMParams& p, int m, int 
       break;
     case EPI_BF16: {
       const size_t o = static_cast<size_t>(m) * p.N + n;
+      if (p.f16) {
+        *reinterpret_cast<uint32_t*>(static_cast<__half*>(p.out) + o) = pack_kv(v0, v1);
+        break;
+      }
       const uint32_t hi = pack_bf16x2(v0, v1);
       *reinterpret_cast<uint32_t*>(static_cast<__nv_bfloat16*>(p.out) + o) = hi;
       if (p.out_lo) *reinterpret_cast<uint32_t*>(p.out_lo + o) = pack_bf16x2(v0 - bf16_lo(hi), v1 - bf16_hi(hi));
@@ -44,16 +52,16 @@ __device__ __forceinline__ void epilogue_pair(const LargeMParams& p, int m, int 
         v1 = a1;
       }
       if (n < nq) {
-        const uint32_t hi = pack_bf16x2(v0, v1);
-        *reinterpret_cast<uint32_t*>(e.q_out_bf16 + static_cast<size_t>(m) * nq + n) = hi;
+        const uint32_t hi = pack_f16x2(v0, v1);      // the query as the attention's binary16 operand pair
+        *reinterpret_cast<uint32_t*>(e.q_out_f16 + static_cast<size_t>(m) * nq + n) = hi;
         if (e.q_out_lo)
           *reinterpret_cast<uint32_t*>(e.q_out_lo + static_cast<size_t>(m) * nq + n) =
-              pack_bf16x2(v0 - bf16_lo(hi), v1 - bf16_hi(hi));
+              pack_f16x2(v0 - f16_lo(hi), v1 - f16_hi(hi));
       } else {
         const int nn = n < nq + nk ? n - nq : n - nq - nk;
-        __nv_bfloat16* cache = n < nq + nk ? e.k_cache : e.v_cache;
+        kv_t* cache = n < nq + nk ? e.k_cache : e.v_cache;
         const size_t off = ((static_cast<size_t>(b) * e.n_kv_heads + nn / Dh) * e.max_seq_len + pos) * Dh + (nn % Dh);
-        *reinterpret_cast<uint32_t*>(cache + off) = pack_bf16x2(v0, v1);
+        *reinterpret_cast<uint32_t*>(cache + off) = pack_kv(v0, v1);
       }
       break;
     }

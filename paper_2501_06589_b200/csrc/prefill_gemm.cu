@@ -139,11 +139,12 @@ int g_prefill_impl = 0;
 int g_sm_count = 0;
 }  // namespace
 
-void set_prefill_gemm_impl(int impl) { g_prefill_impl = impl == 1 || impl == 2 ? impl : 0; }
+void set_prefill_gemm_impl(int impl) { g_prefill_impl = impl >= 1 && impl <= 3 ? impl : 0; }
 bool prefill_single_bf16() { return g_prefill_impl == 2; }
+int prefill_gemm_impl() { return g_prefill_impl; }
 
 cudaError_t launch_largem_gemm(const LargeMParams& p, cudaStream_t stream) {
-  if (g_prefill_impl != 1) {
+  if (g_prefill_impl != 1 || p.f16) {
     if (!g_sm_count) {
       int dev = 0;
       if (cudaGetDevice(&dev) != cudaSuccess ||

@@ -32,16 +32,21 @@ constexpr int A_BYTES = BM * BK * 2;  // 16 KB
 constexpr int kTcThreads = 192;
 // Tile width BN = 256 by default; 128 when that leaves SMs without a tile (small M x N: a short prompt, a chunk of a
 // prompt, a narrow projection), which doubles the number of tiles at the same bytes per flop for A.
-template <int BN>
+// SPLIT: A comes as a hi + lo pair (two boxes per stage, two MMA rounds per K block); without it a stage is one A box
+// and one W box, which leaves room for one more stage.
+template <int BN, bool SPLIT>
 struct TcCfg {
-  static constexpr int B_BYTES = BN * BK * 2;               // 32 / 16 KB
-  static constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;  // 64 / 48 KB
-  static constexpr int STAGES = BN == 256 ? 3 : 4;
+  static constexpr int B_BYTES = BN * BK * 2;                              // 32 / 16 KB
+  static constexpr int W_OFF = (SPLIT ? 2 : 1) * A_BYTES;                  // the W box follows the A box(es)
+  static constexpr int STAGE_BYTES = W_OFF + B_BYTES;                      // SPLIT: 64 / 48 KB, else 48 / 32 KB
+  static constexpr int STAGES = SPLIT ? (BN == 256 ? 3 : 4) : (BN == 256 ? 4 : 6);
   static constexpr int OFF_BARS = STAGES * STAGE_BYTES;  // full[], empty[], tmem_full[2], tmem_empty[2], tmem slot
-  static constexpr int SMEM = OFF_BARS + 16 * 8 + 1024;
-  // Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M x N.
-  static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
-                                    (static_cast<uint32_t>(BM >> 4) << 24);
+  static constexpr int SMEM = OFF_BARS + 24 * 8 + 1024;
+  // Instruction descriptor, kind::f16: D fp32 (bit 4), A format bits 7-9 and B format bits 10-12 (0 = binary16,
+  // 1 = bf16; always the same for both operands here), both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
+  static constexpr uint32_t IDESC_F16 = (1u << 4) | (static_cast<uint32_t>(BN >> 3) << 17) |
+                                        (static_cast<uint32_t>(BM >> 4) << 24);
+  static constexpr uint32_t IDESC_BF16 = IDESC_F16 | (1u << 7) | (1u << 10);
 };
 constexpr int GROUP_M = 16;  // M-tiles per rasterisation band
 
@@ -107,9 +112,10 @@ template <bool SPLIT, int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 largem_gemm_tc_kernel(const LargeMParams p, const __grid_constant__ CUtensorMap map_a,
                       const __grid_constant__ CUtensorMap map_alo, const __grid_constant__ CUtensorMap map_w) {
-  using C = TcCfg<BN>;
+  using C = TcCfg<BN, SPLIT>;
   constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, B_BYTES = C::B_BYTES, OFF_BARS = C::OFF_BARS;
-  constexpr uint32_t kIdesc = C::IDESC;
+  constexpr int W_OFF = C::W_OFF;
+  const uint32_t kIdesc = p.f16 ? C::IDESC_F16 : C::IDESC_BF16;
   constexpr int kTmemCols = 2 * BN;  // two fp32 accumulators of BN columns
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -163,7 +169,7 @@ largem_gemm_tc_kernel(const LargeMParams p, const __grid_constant__ CUtensorMap 
           mbar_expect_tx(&full[s], (SPLIT ? 2 : 1) * A_BYTES + B_BYTES);
           tma_load_2d(st, &map_a, kb * BK, m0, &full[s]);
           if (SPLIT) tma_load_2d(st + A_BYTES, &map_alo, kb * BK, m0, &full[s]);
-          tma_load_2d(st + 2 * A_BYTES, &map_w, kb * BK, n0, &full[s]);
+          tma_load_2d(st + W_OFF, &map_w, kb * BK, n0, &full[s]);
         }
       }
       if (!ok) {
@@ -191,7 +197,7 @@ largem_gemm_tc_kernel(const LargeMParams p, const __grid_constant__ CUtensorMap 
           if (!ok) break;
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
-          const uint64_t da = smem_desc(a_addr), dl = smem_desc(a_addr + A_BYTES), dw = smem_desc(a_addr + 2 * A_BYTES);
+          const uint64_t da = smem_desc(a_addr), dl = smem_desc(a_addr + A_BYTES), dw = smem_desc(a_addr + W_OFF);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)  // +32 bytes along K inside the swizzled row = +2 in the address field
             tc_mma(d_tmem, da + 2 * k, dw + 2 * k, kIdesc, (kb > 0 || k > 0) ? 1u : 0u);
@@ -249,12 +255,12 @@ using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, voi
                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeFn g_encode = nullptr;
 
-cudaError_t make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) {
+cudaError_t make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows, bool f16) {
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
   const cuuint32_t box[2] = {BK, static_cast<cuuint32_t>(box_rows)};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  const CUresult r = g_encode(map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
@@ -272,16 +278,16 @@ cudaError_t largem_gemm_tc_init() {
     g_encode = reinterpret_cast<EncodeFn>(fn);
   }
   cudaError_t e = cudaFuncSetAttribute(largem_gemm_tc_kernel<true, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       TcCfg<256>::SMEM);
+                                       TcCfg<256, true>::SMEM);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(largem_gemm_tc_kernel<false, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             TcCfg<256>::SMEM);
+                             TcCfg<256, false>::SMEM);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(largem_gemm_tc_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             TcCfg<128>::SMEM);
+                             TcCfg<128, true>::SMEM);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(largem_gemm_tc_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             TcCfg<128>::SMEM);
+                             TcCfg<128, false>::SMEM);
   return e;
 }
 
@@ -289,14 +295,16 @@ namespace {
 template <int BN>
 cudaError_t launch_bn(const LargeMParams& p, cudaStream_t stream, int sm_count) {
   CUtensorMap ma, ml, mw;
-  cudaError_t e = make_map(&ma, p.A, p.M, p.K, BM);
-  if (e == cudaSuccess) e = make_map(&ml, p.A_lo ? p.A_lo : p.A, p.M, p.K, BM);
-  if (e == cudaSuccess) e = make_map(&mw, p.W, p.N, p.K, BN);
+  const bool f16 = p.f16 != 0;
+  if (f16 && p.A_lo) return cudaErrorInvalidValue;  // the binary16 path takes one value per activation
+  cudaError_t e = make_map(&ma, p.A, p.M, p.K, BM, f16);
+  if (e == cudaSuccess) e = make_map(&ml, p.A_lo ? p.A_lo : p.A, p.M, p.K, BM, f16);
+  if (e == cudaSuccess) e = make_map(&mw, p.W, p.N, p.K, BN, f16);
   if (e != cudaSuccess) return e;
   const int tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
   const int grid = tiles < sm_count ? tiles : sm_count;
-  if (p.A_lo) largem_gemm_tc_kernel<true, BN><<<grid, kTcThreads, TcCfg<BN>::SMEM, stream>>>(p, ma, ml, mw);
-  else largem_gemm_tc_kernel<false, BN><<<grid, kTcThreads, TcCfg<BN>::SMEM, stream>>>(p, ma, ml, mw);
+  if (p.A_lo) largem_gemm_tc_kernel<true, BN><<<grid, kTcThreads, TcCfg<BN, true>::SMEM, stream>>>(p, ma, ml, mw);
+  else largem_gemm_tc_kernel<false, BN><<<grid, kTcThreads, TcCfg<BN, false>::SMEM, stream>>>(p, ma, ml, mw);
   return cudaGetLastError();
 }
 }  // namespace

@@ -67,9 +67,9 @@ __device__ __forceinline__ void smallm_epilogue(const SmallMParams& p, int ct, i
         *reinterpret_cast<float2*>(e.q_out_f32 + static_cast<size_t>(b) * nq + n) = make_float2(v0, v1);
       } else {
         const int nn = n < nq + nk ? n - nq : n - nq - nk;
-        __nv_bfloat16* cache = n < nq + nk ? e.k_cache : e.v_cache;
+        kv_t* cache = n < nq + nk ? e.k_cache : e.v_cache;
         const size_t off = ((static_cast<size_t>(b) * e.n_kv_heads + nn / Dh) * e.max_seq_len + pos) * Dh + (nn % Dh);
-        *reinterpret_cast<uint32_t*>(cache + off) = pack_bf16x2(v0, v1);
+        *reinterpret_cast<uint32_t*>(cache + off) = pack_kv(v0, v1);
       }
     }
   }

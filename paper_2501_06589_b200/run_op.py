@@ -71,8 +71,8 @@ def main():
         max_seq = s.prompt_len + s.decode_steps
         kv = a.kv_len or (s.prompt_len + s.decode_steps // 2)
         q = torch.randn(bsz, Hq * Dh, device=dev)
-        k = [torch.randn(bsz, Hkv, max_seq, Dh, device=dev).to(torch.bfloat16) for _ in range(L)]
-        v = [torch.randn(bsz, Hkv, max_seq, Dh, device=dev).to(torch.bfloat16) for _ in range(L)]
+        k = [torch.randn(bsz, Hkv, max_seq, Dh, device=dev).to(torch.float16) for _ in range(L)]
+        v = [torch.randn(bsz, Hkv, max_seq, Dh, device=dev).to(torch.float16) for _ in range(L)]
         lens = torch.full((bsz,), kv, dtype=torch.int32, device=dev)
         scr = torch.empty(B.decode_attention_scratch_bytes(bsz, Hq, Dh, max_seq) // 4, device=dev)
         o = torch.empty(bsz, Hq * Dh, device=dev)
@@ -98,10 +98,10 @@ def main():
             flops = 2.0 * M * N * K
     elif a.op == "prefill_attn":
         S = s.prompt_len
-        q = torch.randn(bsz, S, Hq * Dh, device=dev).to(torch.bfloat16)
-        q_lo = (torch.randn(bsz, S, Hq * Dh, device=dev) * 1e-3).to(torch.bfloat16)
-        k = [torch.randn(bsz, Hkv, S, Dh, device=dev).to(torch.bfloat16) for _ in range(L)]
-        v = [torch.randn(bsz, Hkv, S, Dh, device=dev).to(torch.bfloat16) for _ in range(L)]
+        q = torch.randn(bsz, S, Hq * Dh, device=dev).to(torch.float16)
+        q_lo = (torch.randn(bsz, S, Hq * Dh, device=dev) * 1e-3).to(torch.float16)
+        k = [torch.randn(bsz, Hkv, S, Dh, device=dev).to(torch.float16) for _ in range(L)]
+        v = [torch.randn(bsz, Hkv, S, Dh, device=dev).to(torch.float16) for _ in range(L)]
         o = torch.empty_like(q)
         o_lo = torch.empty_like(q)
         fn = lambda l: B.op_prefill_attention(q, k[l], v[l], bsz, S, Hq, Hkv, Dh, S, o, q_lo=q_lo, o_lo=o_lo)

@@ -549,6 +549,19 @@ def test_bf16_kv_switch_rounds_exactly_the_cache():
     assert np.allclose(step.hidden[:, 0], full.hidden[:, 6], atol=1e-10)
 
 
+def test_f16_kv_switch_rounds_to_binary16_as_the_library_conversion_does():
+    cfg = small_cfg(n_layers=1)
+    t = rand_weights(cfg, 25)
+    c = O.OracleCache(cfg, 2, 8)
+    e = O.OracleCache(cfg, 2, 8)
+    O.prefill(cfg, W(t), TOK, e)
+    O.prefill(cfg, W(t), TOK, c, bf16_kv="f16")
+    ref = torch.from_numpy(e.k[0, :, :6].astype(np.float32)).to(torch.float16).to(torch.float64).numpy()
+    assert np.array_equal(c.k[0, :, :6], ref)
+    x = np.array([1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 70000.0, 1e-8])     # ties to even; overflow; underflow
+    assert np.array_equal(O.f16_round(x), np.array([1.0, 1.0 + 2.0 ** -9, np.inf, 0.0]))
+
+
 # ---------------------------------------------------------------- the paper's own arithmetic (Tab. 2)
 def test_table2_reading_latency_reduction_vs_throughput_gain():
     import os

@@ -196,6 +196,46 @@ ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attenti
 ladder_status_t ladder_prefill(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
                                int32_t batch, int32_t seq_len, const ladder_outputs_t* out, void* cuda_stream);
 
+/* Prompt pass over sequences of DIFFERENT lengths in one call.  d_tokens int32 [batch, seq_len] holds every
+ * prompt left-aligned and padded to seq_len with any valid token id; h_lens is a HOST array [batch] of the true
+ * lengths, 1 <= h_lens[b] <= seq_len (copied before the call returns).  Sequence b gets cache rows
+ * 0..h_lens[b]-1 (nothing is written behind them), seq_lens[b] = h_lens[b], and its outputs are those of its own
+ * last position h_lens[b]-1; with all_hidden the rows of padding positions are unspecified.  Padding costs its
+ * share of the GEMM work (it is computed and discarded); causal attention keeps it from reaching any valid
+ * position.  The host-side length the library tracks becomes the longest one (cf. ladder_set_position), so the
+ * sequences can be decoded together right away.  The paper has no counterpart (it benchmarks equal lengths). */
+ladder_status_t ladder_prefill_ragged(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                                      const int32_t* h_lens, int32_t batch, int32_t seq_len, const ladder_outputs_t* out,
+                                      void* cuda_stream);
+
+/* Pipeline stages (paper Sec. 5.1: at a pipeline boundary the stream `residual` and the two module outputs that have
+ * not been added yet are forwarded to the next stage).  A stage is a model object created over its own layers (the
+ * whole model's weight arrays and rule tables, sliced; pass module_stale explicitly when the slice starts with a
+ * ladder layer whose predecessor in the previous stage is not one) with its own KV cache.  The state that crosses the
+ * boundary is the pair (x_m, x_{m-1}) of residual-stream values after the stage's last module -- in Algorithm 1's
+ * variables residual + attn_out + mlp_out and residual + attn_out: the two sums are all the next layer reads -- as
+ * fp32 [rows, d_model] buffers, rows = batch * seq_len in the prompt pass and batch in a decode step.
+ *   state_in  NULL: first stage, starts from the token embedding (d_tokens required).  Otherwise d_tokens is unused
+ *             (may be NULL), `newest` is required; without `older` a first module that asks for x_{m-1} reads x_m
+ *             (as module 1 of a whole model reads x_0).
+ *   state_out NULL: last stage, runs the final norm, the LM head and the argmax as ladder_prefill / ladder_decode_step
+ *             do.  Otherwise the head is skipped, the state is written (`older` optional) and `out` must not ask for
+ *             all_hidden; next_tokens / final_hidden / logits are not produced.
+ * Every stage updates its own cache and seq_lens.  Stage calls run one kernel per GEMM (no persistent kernel); moving
+ * the state between devices is the caller's business (one peer copy of 2 x rows x d_model floats per boundary). */
+typedef struct {
+  float* newest; /* x_m:     [rows, d_model] fp32 */
+  float* older;  /* x_{m-1}: [rows, d_model] fp32, optional */
+} ladder_stream_state_t;
+ladder_status_t ladder_stage_prefill(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                                     const ladder_stream_state_t* state_in, int32_t batch, int32_t seq_len,
+                                     const ladder_stream_state_t* state_out, const ladder_outputs_t* out,
+                                     void* cuda_stream);
+ladder_status_t ladder_stage_decode_step(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                                         const ladder_stream_state_t* state_in, int32_t batch,
+                                         const ladder_stream_state_t* state_out, const ladder_outputs_t* out,
+                                         void* cuda_stream);
+
 /* Continues a prompt (chunked prompt pass): the seq_len new tokens of every sequence sit at positions
  * L .. L+seq_len-1, where L is the common cached length the library tracks (set by ladder_prefill, a previous
  * ladder_prefill_append, decode steps or ladder_set_position).  They attend to cache rows 0..L-1 and causally

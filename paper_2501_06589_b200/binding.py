@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libladder.so")
 
 EXPORTS = [
     "ladder_kv_cache_bytes", "ladder_model_create", "ladder_model_set_schedule", "ladder_model_set_sm_split", "ladder_model_set_persistent", "ladder_model_persistent_active", "ladder_stack_plan", "ladder_debug_stall_last_phase",
-    "ladder_prefill", "ladder_prefill_append",
+    "ladder_prefill", "ladder_prefill_append", "ladder_prefill_ragged", "ladder_stage_prefill", "ladder_stage_decode_step",
     "ladder_decode_step", "ladder_decode_step_host", "ladder_prefill_host", "ladder_set_position",
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
     "ladder_last_error", "ladder_op_smallm_gemm", "ladder_decode_attention_scratch_bytes",
@@ -59,6 +59,10 @@ class ladder_kv_cache_t(C.Structure):
     _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("seq_lens", C.c_void_p)]
 
 
+class ladder_stream_state_t(C.Structure):
+    _fields_ = [("newest", C.c_void_p), ("older", C.c_void_p)]
+
+
 class ladder_outputs_t(C.Structure):
     _fields_ = [("next_tokens", C.c_void_p), ("final_hidden", C.c_void_p), ("logits", C.c_void_p),
                 ("all_hidden", C.c_void_p)]
@@ -90,6 +94,14 @@ def lib() -> C.CDLL:
                                      C.POINTER(ladder_outputs_t), C.c_void_p]
         L.ladder_prefill_append.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32, C.c_int32,
                                      C.POINTER(ladder_outputs_t), C.c_void_p]
+        L.ladder_prefill_ragged.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_void_p, C.c_int32,
+                                            C.c_int32, C.POINTER(ladder_outputs_t), C.c_void_p]
+        L.ladder_stage_prefill.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p,
+                                           C.POINTER(ladder_stream_state_t), C.c_int32, C.c_int32,
+                                           C.POINTER(ladder_stream_state_t), C.POINTER(ladder_outputs_t), C.c_void_p]
+        L.ladder_stage_decode_step.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p,
+                                               C.POINTER(ladder_stream_state_t), C.c_int32,
+                                               C.POINTER(ladder_stream_state_t), C.POINTER(ladder_outputs_t), C.c_void_p]
         L.ladder_decode_step.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32,
                                          C.POINTER(ladder_outputs_t), C.c_void_p]
         L.ladder_decode_step_host.argtypes = [C.c_void_p, C.POINTER(ladder_kv_cache_t), C.c_void_p, C.c_int32,
@@ -299,6 +311,34 @@ class Model:
         o = self._outs(next_tokens, final_hidden, logits, all_hidden)
         _check(lib().ladder_prefill(self.h, C.byref(cache.c), _ptr(tokens), tokens.shape[0], tokens.shape[1],
                                     C.byref(o), _stream()), self.h)
+
+    def prefill_ragged(self, cache: KVCache, tokens: torch.Tensor, lens: Sequence[int], next_tokens=None,
+                       final_hidden=None, logits=None, all_hidden=None):
+        """Prompts of different lengths in one call: tokens [batch, padded length], lens the true lengths."""
+        assert tokens.dtype == torch.int32 and tokens.is_cuda and tokens.dim() == 2 and len(lens) == tokens.shape[0]
+        o = self._outs(next_tokens, final_hidden, logits, all_hidden)
+        h_lens = (C.c_int32 * len(lens))(*[int(v) for v in lens])
+        _check(lib().ladder_prefill_ragged(self.h, C.byref(cache.c), _ptr(tokens), h_lens, tokens.shape[0],
+                                           tokens.shape[1], C.byref(o), _stream()), self.h)
+
+    @staticmethod
+    def _state(pair):
+        if pair is None:
+            return None
+        newest, older = pair
+        return C.byref(ladder_stream_state_t(_ptr(newest), _ptr(older)))
+
+    def stage_prefill(self, cache: KVCache, tokens, batch: int, seq_len: int, state_in=None, state_out=None, **outs):
+        """Prompt pass of one pipeline stage.  state_in / state_out: (newest, older) fp32 tensors [batch*seq_len, d]
+        or None (first stage: tokens; last stage: head outputs as keyword arguments)."""
+        o = self._outs(**outs)
+        _check(lib().ladder_stage_prefill(self.h, C.byref(cache.c), _ptr(tokens), self._state(state_in), batch, seq_len,
+                                          self._state(state_out), C.byref(o), _stream()), self.h)
+
+    def stage_decode_step(self, cache: KVCache, tokens, batch: int, state_in=None, state_out=None, **outs):
+        o = self._outs(**outs)
+        _check(lib().ladder_stage_decode_step(self.h, C.byref(cache.c), _ptr(tokens), self._state(state_in), batch,
+                                              self._state(state_out), C.byref(o), _stream()), self.h)
 
     def prefill_append(self, cache: KVCache, tokens: torch.Tensor, next_tokens=None, final_hidden=None, logits=None,
                        all_hidden=None):

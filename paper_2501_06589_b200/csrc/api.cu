@@ -47,9 +47,11 @@ struct GraphKey {
   int batch = 0, n_streams = 0, pdl = 0;
   const void *k = nullptr, *v = nullptr, *lens = nullptr, *tok = nullptr;
   const void *o_next = nullptr, *o_hid = nullptr, *o_logits = nullptr;
+  const void *s_in0 = nullptr, *s_in1 = nullptr, *s_out0 = nullptr, *s_out1 = nullptr;  // pipeline-stage state buffers
   bool operator==(const GraphKey& o) const {
     return batch == o.batch && n_streams == o.n_streams && pdl == o.pdl && k == o.k && v == o.v && lens == o.lens &&
-           tok == o.tok && o_next == o.o_next && o_hid == o.o_hid && o_logits == o.o_logits;
+           tok == o.tok && o_next == o.o_next && o_hid == o.o_hid && o_logits == o.o_logits && s_in0 == o.s_in0 &&
+           s_in1 == o.s_in1 && s_out0 == o.s_out0 && s_out1 == o.s_out1;
   }
 };
 
@@ -86,14 +88,17 @@ struct ladder_model {
   __nv_bfloat16 *n_pf = nullptr, *o_pf = nullptr, *h_pf = nullptr;
   __half* q_pf = nullptr;  // the rotated query as the attention's binary16 operand pair
   __half* w16 = nullptr;   // one layer's four weight matrices as binary16 (prompt pass; NULL: not enough memory)
+  __half* w16b = nullptr;  // a second such buffer: the next layer is converted on the side stream meanwhile (optional)
+  cudaEvent_t ev_w16_ready[2] = {nullptr, nullptr}, ev_w16_free[2] = {nullptr, nullptr}, ev_pf_fork = nullptr;
   size_t n_lo = 0, q_lo = 0, h_lo = 0;  // element offsets of the lo parts
   float2* rope = nullptr;
   int32_t* status = nullptr;
-  int32_t *tok_tmp = nullptr, *next_tmp = nullptr;
+  int32_t *tok_tmp = nullptr, *next_tmp = nullptr, *lens_tmp = nullptr;
+  int32_t* h_lens_pinned = nullptr;  // host (pinned), max_batch entries: staging of per-sequence prompt lengths
   // scheduling
   cudaStream_t side = nullptr, cap = nullptr;
   std::vector<cudaEvent_t> ev;  // ev[m] = end of module m (m = 0: embedding)
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_lens = nullptr;
   int n_streams = 2, use_graph = 1, use_pdl = 1;
   int sms_a = -1;  // SMs given to the attention stream in ladder layers (0 = automatic, -1 = no split)
   cudaGraphExec_t graph_exec = nullptr;
@@ -112,6 +117,9 @@ struct ladder_model {
   int32_t* d_counters = nullptr;
   int n_phases = 0, n_attn = 0, n_counters = 0, cap_counters = 0;
   // state
+  // pipeline stage (paper Sec. 5.1), set for the duration of a ladder_stage_* call: the stream state this stage
+  // starts from instead of the embedding, and where it leaves the state instead of running the head
+  ladder_stream_state_t st_in = {nullptr, nullptr}, st_out = {nullptr, nullptr};
   int host_len = 0;
   bool timed_out = false;  // ladder_device_status saw LADDER_DEV_TIMEOUT: steps are refused until re-armed
   int64_t launches = 0;
@@ -186,7 +194,39 @@ struct Router {
 // Route of module `module` (1-based) of this model.
 Router::Route route(const ladder_model* m, Router& rt, int module) {
   const int n = static_cast<int>(m->stale.size());
-  return rt.next(m->stale[module - 1] != 0, module < n && m->stale[module] != 0, module);
+  // the last module of a stage that hands its state on keeps x_{m-1}: the next stage's first module may read it
+  const bool next_reads_older = module < n ? m->stale[module] != 0 : m->st_out.newest != nullptr;
+  return rt.next(m->stale[module - 1] != 0, next_reads_older, module);
+}
+
+// Start of a forward pass over `rows` tokens: the embedding gather, or -- in a pipeline stage that receives the
+// stream state -- copies of (x_{m-1}, x_{m-2}) into the two residual buffers.
+cudaError_t begin_stream(ladder_model* m, Router& rt, const int32_t* d_tokens, int rows, cudaStream_t st) {
+  const ladder_config_t& c = m->cfg;
+  if (!m->st_in.newest)
+    return launch_embed(d_tokens, m->tok_embedding, rows, c.d_model, c.vocab_size, m->R[0], m->status, st, false);
+  const size_t bytes = static_cast<size_t>(rows) * c.d_model * sizeof(float);
+  cudaError_t e = cudaMemcpyAsync(m->R[0], m->st_in.newest, bytes, cudaMemcpyDeviceToDevice, st);
+  if (e == cudaSuccess && m->st_in.older) {
+    e = cudaMemcpyAsync(m->R[1], m->st_in.older, bytes, cudaMemcpyDeviceToDevice, st);
+    rt.stale = 1;
+    rt.writer[1] = 0;
+  }
+  return e;
+}
+
+// End of a stage that hands its state on: (x_m, x_{m-1}) out of the residual buffers (x_{m-1} := x_m when the last
+// module worked in place and nothing older exists), and the cache lengths.
+cudaError_t end_stage(ladder_model* m, const Router& rt, const ladder_kv_cache_t* cache, int batch, int rows, int advance,
+                      int set_len, const int32_t* set_lens, cudaStream_t st) {
+  const size_t bytes = static_cast<size_t>(rows) * m->cfg.d_model * sizeof(float);
+  cudaError_t e = cudaMemcpyAsync(m->st_out.newest, m->R[rt.cur], bytes, cudaMemcpyDeviceToDevice, st);
+  if (e == cudaSuccess && m->st_out.older)
+    e = cudaMemcpyAsync(m->st_out.older, m->R[rt.stale >= 0 ? rt.stale : rt.cur], bytes, cudaMemcpyDeviceToDevice, st);
+  if (e == cudaSuccess)
+    e = launch_argmax_advance(nullptr, batch, m->cfg.vocab_size, nullptr, cache->seq_lens, advance, set_len, st, false,
+                              set_lens);
+  return e;
 }
 
 // Gain of the RMSNorm in front of the MLP of layer l: a parallel layer normalises once, with the attention gain.
@@ -291,12 +331,12 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
     q.grid_b = m->sm_count - ga;
   }
 
-  q.launched(0, launch_embed(d_tokens, m->tok_embedding, batch, d, c.vocab_size, m->R[0], m->status, sA, false));
-  q.pdl_ok[0] = true;
+  Router rt;
+  q.launched(0, begin_stream(m, rt, d_tokens, batch, sA));
+  q.pdl_ok[0] = m->st_in.newest == nullptr;  // a programmatic edge needs a kernel in front
   q.record(0, m->ev[0]);
   bool b_joined = false;  // has sB been ordered after the embedding yet
 
-  Router rt;
   int last_wait[2] = {0, -1};  // latest module each stream has (transitively) waited for
   auto need = [&](int s, int module) {
     // make stream s wait for the end of `module` unless that is already implied
@@ -427,6 +467,11 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   }
   // ---------------- head on stream A (joins stream B)
   need(0, 2 * c.n_layers);
+  if (m->st_out.newest) {  // a stage that hands its state on: no final norm, no head
+    q.launched(0, end_stage(m, rt, cache, batch, batch, 1, -1, nullptr, sA));
+    *n_kernels = q.kernels;
+    return q.err;
+  }
   const float* xf = m->R[rt.cur];
   float* logits = (out && out->logits) ? out->logits : m->logits_ws;
   SmallMParams h = {};
@@ -452,8 +497,10 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
 
 // pos0: position of the first of the S new tokens of every sequence (0 = a fresh prompt; > 0 = the prompt is
 // continued: the new tokens attend to the pos0 cached positions and to each other causally).
+// d_lens (device, optional; fresh prompts only): per-sequence prompt lengths <= S; rows behind them are padding.
 cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int batch, int S,
-                            const ladder_outputs_t* out, cudaStream_t st, int64_t* n_kernels, int pos0 = 0) {
+                            const ladder_outputs_t* out, cudaStream_t st, int64_t* n_kernels, int pos0 = 0,
+                            const int32_t* d_lens = nullptr) {
   const ladder_config_t& c = m->cfg;
   const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff;
   const int M = batch * S;
@@ -464,7 +511,8 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
     if (err == cudaSuccess) err = e;
     ++k;
   };
-  did(launch_embed(d_tokens, m->tok_embedding, M, d, c.vocab_size, m->R[0], m->status, st, false));
+  Router rt;
+  did(begin_stream(m, rt, d_tokens, M, st));
   // Operand precision of the prompt-pass GEMMs.  Default for calls of >= kPrefillF16MinTokens tokens: binary16,
   // ONE value per activation (11 significant bits) against the layer's weights converted to binary16 once per
   // call (exact but for magnitudes below 2^-14) -- half the tensor-core work of a bf16 hi + lo pair.  Otherwise
@@ -477,21 +525,42 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
   __nv_bfloat16* const h_lo = split ? m->h_pf + m->h_lo : nullptr;
   const size_t n_qkv = static_cast<size_t>(Hq + 2 * Hkv) * Dh * d, n_o = static_cast<size_t>(d) * Hq * Dh;
   const size_t n_gu = 2 * static_cast<size_t>(F) * d, n_dn = static_cast<size_t>(d) * F;
-  __half* const w16_qkv = m->w16;
-  __half* const w16_o = f16 ? w16_qkv + n_qkv : nullptr;
-  __half* const w16_gu = f16 ? w16_o + n_o : nullptr;
-  __half* const w16_dn = f16 ? w16_gu + n_gu : nullptr;
+  // Two scratch buffers: the conversion of layer l + 1 runs on the side stream while layer l's GEMMs run here
+  // (they leave most of the DRAM bandwidth unused).  With one buffer it runs in line.
+  const bool overlap = f16 && m->w16b != nullptr;
+  auto convert_layer = [&](int l, __half* dst, cudaStream_t cs) {
+    did(launch_convert_bf16_f16(m->w_qkv[l], dst, n_qkv, cs));
+    did(launch_convert_bf16_f16(m->w_o[l], dst + n_qkv, n_o, cs));
+    did(launch_convert_bf16_f16(m->w_gate_up[l], dst + n_qkv + n_o, n_gu, cs));
+    did(launch_convert_bf16_f16(m->w_down[l], dst + n_qkv + n_o + n_gu, n_dn, cs));
+  };
+  auto note = [&](cudaError_t e) {
+    if (err == cudaSuccess) err = e;
+  };
+  if (overlap) {  // the side stream starts after everything already queued here (an earlier call may still use the buffers)
+    note(cudaEventRecord(m->ev_pf_fork, st));
+    note(cudaStreamWaitEvent(m->side, m->ev_pf_fork, 0));
+    convert_layer(0, m->w16, m->side);
+    note(cudaEventRecord(m->ev_w16_ready[0], m->side));
+  }
   auto norm = [&](const float* x, const __nv_bfloat16* gain) {
     if (f16) did(launch_rmsnorm_f16(x, gain, c.rms_eps, M, d, reinterpret_cast<__half*>(m->n_pf), st));
     else did(launch_rmsnorm_bf16(x, gain, c.rms_eps, M, d, m->n_pf, n_lo, st));
   };
-  Router rt;
   for (int l = 0; l < c.n_layers; ++l) {
-    if (f16) {  // this layer's weights as binary16 (the previous layer's GEMMs are done with the scratch: same stream)
-      did(launch_convert_bf16_f16(m->w_qkv[l], w16_qkv, n_qkv, st));
-      did(launch_convert_bf16_f16(m->w_o[l], w16_o, n_o, st));
-      did(launch_convert_bf16_f16(m->w_gate_up[l], w16_gu, n_gu, st));
-      did(launch_convert_bf16_f16(m->w_down[l], w16_dn, n_dn, st));
+    __half* const w16_qkv = overlap && (l & 1) ? m->w16b : m->w16;
+    __half* const w16_o = f16 ? w16_qkv + n_qkv : nullptr;
+    __half* const w16_gu = f16 ? w16_o + n_o : nullptr;
+    __half* const w16_dn = f16 ? w16_gu + n_gu : nullptr;
+    if (overlap) {
+      if (l + 1 < c.n_layers) {  // next layer into the other buffer, once layer l - 1 has finished with it
+        if (l >= 1) note(cudaStreamWaitEvent(m->side, m->ev_w16_free[(l + 1) & 1], 0));
+        convert_layer(l + 1, (l + 1) & 1 ? m->w16b : m->w16, m->side);
+        note(cudaEventRecord(m->ev_w16_ready[(l + 1) & 1], m->side));
+      }
+      note(cudaStreamWaitEvent(st, m->ev_w16_ready[l & 1], 0));
+    } else if (f16) {  // in line: the previous layer's GEMMs are done with the scratch (same stream)
+      convert_layer(l, m->w16, st);
     }
     {
       const Router::Route r = route(m, rt, 2 * l + 1);
@@ -516,10 +585,11 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       p.qkv.max_seq_len = c.max_seq_len;
       p.qkv.prefill_seq_len = S;
       p.qkv.prefill_pos0 = pos0;
+      p.qkv.prefill_lens = d_lens;
       p.status = m->status;
       did(launch_largem_gemm(p, st));
       did(launch_prefill_attention(m->q_pf, q_lo, p.qkv.k_cache, p.qkv.v_cache, batch, S, Hq, Hkv, Dh, c.max_seq_len,
-                                   m->o_pf, o_lo, st, pos0, f16));
+                                   m->o_pf, o_lo, st, pos0, f16, d_lens));
       LargeMParams o = {};
       o.A = m->o_pf;
       o.A_lo = o_lo;
@@ -564,10 +634,16 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       o.status = m->status;
       did(launch_largem_gemm(o, st));
     }
+    if (overlap) note(cudaEventRecord(m->ev_w16_free[l & 1], st));
+  }
+  if (m->st_out.newest) {  // a stage that hands its state on: every position's stream state, no head
+    did(end_stage(m, rt, cache, batch, M, 0, pos0 + S, d_lens, st));
+    *n_kernels = k;
+    return err;
   }
   const float* xf = m->R[rt.cur];
   if (out && out->all_hidden) did(launch_rmsnorm_f32(xf, m->final_norm, c.rms_eps, M, d, d, out->all_hidden, st, false));
-  did(launch_gather_rows(xf, batch, d, S, S - 1, m->last_x, st));
+  did(launch_gather_rows(xf, batch, d, S, S - 1, m->last_x, st, d_lens));
   float* logits = (out && out->logits) ? out->logits : m->logits_ws;
   SmallMParams h = {};
   h.W = m->lm_head;
@@ -587,7 +663,7 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
   if (out && out->final_hidden)
     did(launch_rmsnorm_f32(m->last_x, m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, st, false));
   did(launch_argmax_advance(logits, batch, c.vocab_size, out ? out->next_tokens : nullptr, cache->seq_lens, 0, pos0 + S,
-                            st, false));
+                            st, false, d_lens));
   *n_kernels = k;
   return err;
 }
@@ -1089,6 +1165,8 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   A(dev_alloc(&m->status, 4));
   A(dev_alloc(&m->tok_tmp, MP > MB ? MP : MB));
   A(dev_alloc(&m->next_tmp, MB));
+  A(dev_alloc(&m->lens_tmp, MB));
+  A(cudaMallocHost(reinterpret_cast<void**>(&m->h_lens_pinned), MB * sizeof(int32_t)));
   if (oom) {
     cudaGetLastError();
     ladder_destroy(m);
@@ -1101,6 +1179,9 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
     if (dev_alloc(&m->w16, layer_elems) != cudaSuccess) {
       cudaGetLastError();
       m->w16 = nullptr;
+    } else if (dev_alloc(&m->w16b, layer_elems) != cudaSuccess) {
+      cudaGetLastError();
+      m->w16b = nullptr;
     }
   }
   // rotary table in double precision: angle = p * theta^(-2j/Dh)
@@ -1125,6 +1206,12 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_pf_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_lens, cudaEventDisableTiming);
+  for (int i = 0; i < 2; ++i) {
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_w16_ready[i], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_w16_free[i], cudaEventDisableTiming);
+  }
   if (e != cudaSuccess) {
     std::string msg = std::string("set-up: ") + cudaGetErrorString(e);
     ladder_destroy(m);
@@ -1141,12 +1228,20 @@ ladder_status_t ladder_destroy(ladder_model_t* m) {
     if (ev) cudaEventDestroy(ev);
   if (m->ev_fork) cudaEventDestroy(m->ev_fork);
   if (m->ev_join) cudaEventDestroy(m->ev_join);
+  if (m->ev_pf_fork) cudaEventDestroy(m->ev_pf_fork);
+  if (m->ev_lens) cudaEventDestroy(m->ev_lens);
+  for (int i = 0; i < 2; ++i) {
+    if (m->ev_w16_ready[i]) cudaEventDestroy(m->ev_w16_ready[i]);
+    if (m->ev_w16_free[i]) cudaEventDestroy(m->ev_w16_free[i]);
+  }
   if (m->side) cudaStreamDestroy(m->side);
   if (m->cap) cudaStreamDestroy(m->cap);
-  void* bufs[] = {m->w16, m->wide_hpack, m->wide_opack, m->xpack[0], m->xpack[1], m->hpack, m->opack, m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
+  void* bufs[] = {m->w16, m->w16b, m->wide_hpack, m->wide_opack, m->xpack[0], m->xpack[1], m->hpack, m->opack, m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
                   m->n_pf, m->q_pf,  m->o_pf,  m->h_pf,  m->rope,  m->status,       m->tok_tmp,   m->next_tmp};
   for (void* b : bufs)
     if (b) cudaFree(b);
+  if (m->lens_tmp) cudaFree(m->lens_tmp);
+  if (m->h_lens_pinned) cudaFreeHost(m->h_lens_pinned);
   delete m;
   return LADDER_OK;
 }
@@ -1290,7 +1385,8 @@ static ladder_status_t check_call(ladder_model_t* m, const ladder_kv_cache_t* ca
   if (rearm) m->timed_out = false;
   if (m->timed_out)
     return fail(m, LADDER_ERR_TIMEOUT, "an earlier step timed out on the device; call ladder_set_position or ladder_prefill");
-  if (!cache || !cache->k || !cache->v || !cache->seq_lens || !tokens) return fail(m, LADDER_ERR_INVALID_ARG, "NULL argument");
+  if (!cache || !cache->k || !cache->v || !cache->seq_lens || (!tokens && !m->st_in.newest))
+    return fail(m, LADDER_ERR_INVALID_ARG, "NULL argument");
   if ((reinterpret_cast<uintptr_t>(cache->k) | reinterpret_cast<uintptr_t>(cache->v)) & 15)
     return fail(m, LADDER_ERR_INVALID_ARG, "cache buffers must be 16-byte aligned");
   if ((reinterpret_cast<uintptr_t>(cache->seq_lens) | reinterpret_cast<uintptr_t>(tokens)) & 3)
@@ -1313,6 +1409,80 @@ ladder_status_t ladder_prefill(ladder_model_t* m, const ladder_kv_cache_t* cache
   m->launches += k;
   m->host_len = seq_len;
   return LADDER_OK;
+}
+
+ladder_status_t ladder_prefill_ragged(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                                      const int32_t* h_lens, int32_t batch, int32_t seq_len, const ladder_outputs_t* out,
+                                      void* cuda_stream) {
+  ladder_status_t s = check_call(m, cache, d_tokens, batch, /*rearm=*/true);
+  if (s != LADDER_OK) return s;
+  if (!h_lens) return fail(m, LADDER_ERR_INVALID_ARG, "NULL lengths");
+  if (seq_len < 1) return fail(m, LADDER_ERR_INVALID_ARG, "seq_len must be >= 1");
+  if (seq_len > m->cfg.max_seq_len) return fail(m, LADDER_ERR_STATE, "seq_len exceeds max_seq_len");
+  if (static_cast<int64_t>(batch) * seq_len > m->cfg.max_prefill_tokens)
+    return fail(m, LADDER_ERR_STATE, "batch*seq_len exceeds max_prefill_tokens");
+  int longest = 0;
+  for (int b = 0; b < batch; ++b) {
+    if (h_lens[b] < 1 || h_lens[b] > seq_len) return fail(m, LADDER_ERR_INVALID_ARG, "a length outside [1, seq_len]");
+    longest = std::max(longest, h_lens[b]);
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // the lengths go to the device through a small pinned staging buffer of the model, so that the copy is
+  // stream-ordered and h_lens may be reused by the caller as soon as this call returns
+  CK(m, cudaEventSynchronize(m->ev_lens));  // the previous call's copy out of the staging buffer has run (usually long ago)
+  memcpy(m->h_lens_pinned, h_lens, static_cast<size_t>(batch) * sizeof(int32_t));
+  CK(m, cudaMemcpyAsync(m->lens_tmp, m->h_lens_pinned, static_cast<size_t>(batch) * sizeof(int32_t),
+                        cudaMemcpyHostToDevice, st));
+  CK(m, cudaEventRecord(m->ev_lens, st));
+  int64_t k = 0;
+  CK(m, enqueue_prefill(m, cache, d_tokens, batch, seq_len, out, st, &k, 0, m->lens_tmp));
+  m->launches += k;
+  m->host_len = longest;
+  return LADDER_OK;
+}
+
+// ---- pipeline stages (paper Sec. 5.1)
+namespace {
+struct StageScope {  // sets the stage state for one call and clears it again
+  ladder_model* m;
+  StageScope(ladder_model* mm, const ladder_stream_state_t* in, const ladder_stream_state_t* out) : m(mm) {
+    if (in) m->st_in = *in;
+    if (out) m->st_out = *out;
+  }
+  ~StageScope() {
+    m->st_in = {nullptr, nullptr};
+    m->st_out = {nullptr, nullptr};
+  }
+};
+const char* check_stage(const ladder_stream_state_t* in, const ladder_stream_state_t* out, const int32_t* tokens) {
+  if (in && !in->newest) return "state_in without its newest buffer";
+  if (out && !out->newest) return "state_out without its newest buffer";
+  if (!in && !tokens) return "a first stage needs tokens";
+  const uintptr_t a = (in ? reinterpret_cast<uintptr_t>(in->newest) | reinterpret_cast<uintptr_t>(in->older) : 0) |
+                      (out ? reinterpret_cast<uintptr_t>(out->newest) | reinterpret_cast<uintptr_t>(out->older) : 0);
+  return (a & 15) ? "stream-state buffers must be 16-byte aligned" : nullptr;
+}
+}  // namespace
+
+ladder_status_t ladder_stage_prefill(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                                     const ladder_stream_state_t* state_in, int32_t batch, int32_t seq_len,
+                                     const ladder_stream_state_t* state_out, const ladder_outputs_t* out,
+                                     void* cuda_stream) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  if (const char* why = check_stage(state_in, state_out, d_tokens)) return fail(m, LADDER_ERR_INVALID_ARG, why);
+  if (state_out && out && out->all_hidden) return fail(m, LADDER_ERR_INVALID_ARG, "a stage that hands its state on has no head outputs");
+  StageScope scope(m, state_in, state_out);
+  return ladder_prefill(m, cache, d_tokens, batch, seq_len, out, cuda_stream);
+}
+
+ladder_status_t ladder_stage_decode_step(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
+                                         const ladder_stream_state_t* state_in, int32_t batch,
+                                         const ladder_stream_state_t* state_out, const ladder_outputs_t* out,
+                                         void* cuda_stream) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  if (const char* why = check_stage(state_in, state_out, d_tokens)) return fail(m, LADDER_ERR_INVALID_ARG, why);
+  StageScope scope(m, state_in, state_out);
+  return ladder_decode_step(m, cache, d_tokens, batch, out, cuda_stream);
 }
 
 ladder_status_t ladder_prefill_append(ladder_model_t* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens,
@@ -1341,7 +1511,8 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const bool two = m->n_streams == 2;
 
-  if (m->use_stack && m->stack_ok && batch <= 4) {
+  const bool staged = m->st_in.newest || m->st_out.newest;  // a pipeline stage runs kernel by kernel
+  if (m->use_stack && m->stack_ok && batch <= 4 && !staged) {
     GraphKey key;
     key.batch = batch;
     key.k = cache->k;
@@ -1398,6 +1569,10 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
     key.o_next = out ? out->next_tokens : nullptr;
     key.o_hid = out ? out->final_hidden : nullptr;
     key.o_logits = out ? out->logits : nullptr;
+    key.s_in0 = m->st_in.newest;
+    key.s_in1 = m->st_in.older;
+    key.s_out0 = m->st_out.newest;
+    key.s_out1 = m->st_out.older;
     if (!m->graph_exec || !(key == m->graph_key)) {
       drop_graph(m);
       for (int attempt = 0; attempt < 2 && !m->graph_exec; ++attempt) {

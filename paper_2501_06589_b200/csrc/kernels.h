@@ -29,6 +29,8 @@ struct QkvEpilogue {
   int n_q_heads, n_kv_heads, head_dim, max_seq_len;
   int prefill_seq_len;         // prefill: rows are [batch, seq_len] flattened
   int prefill_pos0;            // prefill: position of a sequence's first row (> 0 when a prompt is continued)
+  const int32_t* prefill_lens; // prefill, optional (device, [batch]): sequence b has only prefill_lens[b] valid rows;
+                               // keys / values of the padding rows behind them are not stored
 };
 
 struct SmallMParams {
@@ -185,11 +187,14 @@ bool prefill_single_bf16();            // the prompt pass feeds its GEMMs one bf
 
 // q_lo / o_lo: optional lo parts (value ~ hi + lo) of the query input and the attention output.
 // out_f16: o receives ONE binary16 value per element instead of a bf16 value (o_lo must be NULL).
+// lens (device, optional): sequence b holds lens[b] <= seq_len valid rows (rows stay seq_len apart); the padding
+// rows behind them are neither read as keys nor written as outputs.
 // pos0: the seq_len queries sit at positions pos0 .. pos0 + seq_len - 1 and attend to cache rows 0 .. their own.
 cudaError_t launch_prefill_attention(const __half* q, const __half* q_lo, const kv_t* k,
                                      const kv_t* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
                                      int head_dim, int max_seq_len, __nv_bfloat16* o, __nv_bfloat16* o_lo,
-                                     cudaStream_t stream, int pos0 = 0, bool out_f16 = false);
+                                     cudaStream_t stream, int pos0 = 0, bool out_f16 = false,
+                                     const int32_t* lens = nullptr);
 
 // Small element-wise / gather kernels.
 cudaError_t launch_embed(const int32_t* tokens, const __nv_bfloat16* table, int rows, int d, int vocab, float* x,
@@ -202,11 +207,14 @@ cudaError_t launch_rmsnorm_f16(const float* x, const __nv_bfloat16* gain, float 
 cudaError_t launch_convert_bf16_f16(const __nv_bfloat16* src, __half* dst, size_t n, cudaStream_t stream);
 cudaError_t launch_rmsnorm_f32(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, int row_stride,
                                float* out, cudaStream_t stream, bool pdl);
+// lens (device, optional): row r is taken at offset lens[r] - 1 instead of src_offset_rows
 cudaError_t launch_gather_rows(const float* x, int rows, int d, int src_stride_rows, int src_offset_rows, float* out,
-                               cudaStream_t stream);
-// argmax over logits [batch, vocab] (lowest index on ties) -> next_tokens; adds `advance` to seq_lens[b].
+                               cudaStream_t stream, const int32_t* lens = nullptr);
+// argmax over logits [batch, vocab] (lowest index on ties) -> next_tokens; then seq_lens[b] = set_lens[b] (device,
+// optional), else = set_len (if >= 0), else += advance.
 cudaError_t launch_argmax_advance(const float* logits, int batch, int vocab, int32_t* next_tokens, int32_t* seq_lens,
-                                  int advance, int set_len, cudaStream_t stream, bool pdl);
+                                  int advance, int set_len, cudaStream_t stream, bool pdl,
+                                  const int32_t* set_lens = nullptr);
 
 // One-time opt-in to large dynamic shared memory for every kernel (call once per process/device,
 // outside any stream capture).

@@ -119,8 +119,9 @@ __global__ void convert_bf16_f16_kernel(const uint4* src, uint4* dst, size_t n8)
   }
 }
 
-// out[r, :] = x[(r * stride + offset), :]
-__global__ void gather_rows_kernel(const float* x, int d, int stride, int offset, float* out) {
+// out[r, :] = x[(r * stride + offset), :]; with `lens` the offset of row r is lens[r] - 1 (its last valid position)
+__global__ void gather_rows_kernel(const float* x, int d, int stride, int offset, const int32_t* lens, float* out) {
+  if (lens) offset = min(max(lens[blockIdx.x], 1), stride) - 1;
   const float4* src = reinterpret_cast<const float4*>(x + (static_cast<size_t>(blockIdx.x) * stride + offset) * d);
   float4* dst = reinterpret_cast<float4*>(out + static_cast<size_t>(blockIdx.x) * d);
   for (int i = threadIdx.x; i < d / 4; i += blockDim.x) dst[i] = src[i];
@@ -128,7 +129,7 @@ __global__ void gather_rows_kernel(const float* x, int d, int stride, int offset
 
 // Greedy token per row (lowest index among equal maxima), then the length update.
 __global__ void argmax_advance_kernel(const float* logits, int vocab, int32_t* next_tokens, int32_t* seq_lens,
-                                      int advance, int set_len) {
+                                      int advance, int set_len, const int32_t* set_lens) {
   __shared__ float bv[32];
   __shared__ int bi[32];
   pdl_launch_dependents();
@@ -192,7 +193,8 @@ __global__ void argmax_advance_kernel(const float* logits, int vocab, int32_t* n
     }
   }
   if (threadIdx.x == 0 && seq_lens) {
-    if (set_len >= 0) seq_lens[b] = set_len;
+    if (set_lens) seq_lens[b] = set_lens[b];  // per-sequence prompt lengths
+    else if (set_len >= 0) seq_lens[b] = set_len;
     else seq_lens[b] += advance;
   }
 }
@@ -229,14 +231,15 @@ cudaError_t launch_rmsnorm_f32(const float* x, const __nv_bfloat16* gain, float 
 }
 
 cudaError_t launch_gather_rows(const float* x, int rows, int d, int src_stride_rows, int src_offset_rows, float* out,
-                               cudaStream_t stream) {
-  return launch(gather_rows_kernel, dim3(rows), dim3(256), stream, false, x, d, src_stride_rows, src_offset_rows, out);
+                               cudaStream_t stream, const int32_t* lens) {
+  return launch(gather_rows_kernel, dim3(rows), dim3(256), stream, false, x, d, src_stride_rows, src_offset_rows, lens,
+                out);
 }
 
 cudaError_t launch_argmax_advance(const float* logits, int batch, int vocab, int32_t* next_tokens, int32_t* seq_lens,
-                                  int advance, int set_len, cudaStream_t stream, bool pdl) {
+                                  int advance, int set_len, cudaStream_t stream, bool pdl, const int32_t* set_lens) {
   return launch(argmax_advance_kernel, dim3(batch), dim3(1024), stream, pdl, logits, vocab, next_tokens, seq_lens,
-                advance, set_len);
+                advance, set_len, set_lens);
 }
 
 }  // namespace ladder

@@ -38,7 +38,8 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __h
                                                                        int n_q_heads, int n_kv_heads, int max_seq_len,
                                                                        __nv_bfloat16* __restrict__ o,
                                                                        __nv_bfloat16* __restrict__ o_lo, const int pos0,
-                                                                       const int out_f16) {
+                                                                       const int out_f16,
+                                                                       const int32_t* __restrict__ lens) {
   constexpr int P = DH + 8;  // smem pitch in elements
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __half* sQ = reinterpret_cast<__half*>(smem_raw);
@@ -53,10 +54,12 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __h
   const kv_t* kg = kc + (static_cast<size_t>(b) * n_kv_heads + kvh) * max_seq_len * DH;
   const kv_t* vg = vc + (static_cast<size_t>(b) * n_kv_heads + kvh) * max_seq_len * DH;
   constexpr int CPR = DH / 8;  // 16-byte chunks per row
+  const int len_b = lens ? min(max(lens[b], 0), seq_len) : seq_len;  // valid rows of this sequence
+  if (q0 >= len_b) return;                                           // a tile of padding rows
 
   for (int i = tid; i < kQT * CPR; i += kPfThreads) {
     const int r = i / CPR, c = i % CPR;
-    const bool v = q0 + r < seq_len;
+    const bool v = q0 + r < len_b;
     const size_t off = (static_cast<size_t>(b) * seq_len) * qrow_stride + static_cast<size_t>(h) * DH +
                        (v ? static_cast<size_t>(q0 + r) * qrow_stride + c * 8 : 0);
     cp16(smem_u32(sQ + r * P + c * 8), q + off, v);
@@ -71,8 +74,8 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __h
     for (int c = 0; c < 4; ++c) oacc[i][c] = 0.f;
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
   const float scale = rsqrtf(static_cast<float>(DH));
-  const int q_hi = min(q0 + kQT, seq_len) - 1;  // last valid query of the tile
-  const int n_keys = pos0 + seq_len;            // cache rows that exist for this call
+  const int q_hi = min(q0 + kQT, len_b) - 1;    // last valid query of the tile
+  const int n_keys = pos0 + len_b;              // cache rows that exist for this call
   const int n_kt = (pos0 + q_hi) / kKT + 1;
 
   for (int kt = 0; kt < n_kt; ++kt) {
@@ -182,7 +185,7 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __h
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
     const int qi = q0 + warp * 16 + g + r * 8;
-    if (qi >= seq_len) continue;
+    if (qi >= len_b) continue;
     const float inv = l_run[r] > 0.f ? 1.f / l_run[r] : 0.f;
     const size_t doff = (static_cast<size_t>(b) * seq_len + qi) * qrow_stride + static_cast<size_t>(h) * DH;
 #pragma unroll
@@ -202,11 +205,11 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(const __h
 template <int DH, bool SPLIT>
 cudaError_t launch_dh(const __half* q, const __half* q_lo, const kv_t* k, const kv_t* v,
                       int batch, int seq_len, int n_q_heads, int n_kv_heads, int max_seq_len, __nv_bfloat16* o,
-                      __nv_bfloat16* o_lo, cudaStream_t stream, int pos0, int out_f16) {
+                      __nv_bfloat16* o_lo, cudaStream_t stream, int pos0, int out_f16, const int32_t* lens) {
   constexpr int smem = 4 * 64 * (DH + 8) * 2;
   dim3 grid((seq_len + kQT - 1) / kQT, n_q_heads, batch);
   prefill_attention_kernel<DH, SPLIT><<<grid, kPfThreads, smem, stream>>>(q, q_lo, k, v, seq_len, n_q_heads, n_kv_heads,
-                                                                          max_seq_len, o, o_lo, pos0, out_f16);
+                                                                          max_seq_len, o, o_lo, pos0, out_f16, lens);
   return cudaGetLastError();
 }
 
@@ -229,17 +232,17 @@ cudaError_t prefill_attention_init() {
 cudaError_t launch_prefill_attention(const __half* q, const __half* q_lo, const kv_t* k,
                                      const kv_t* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
                                      int head_dim, int max_seq_len, __nv_bfloat16* o, __nv_bfloat16* o_lo,
-                                     cudaStream_t stream, int pos0, bool out_f16) {
+                                     cudaStream_t stream, int pos0, bool out_f16, const int32_t* lens) {
   const bool split = q_lo != nullptr && (o_lo != nullptr || out_f16);
   if (out_f16 && o_lo) return cudaErrorInvalidValue;
   const int of = out_f16 ? 1 : 0;
   if (pos0 < 0 || pos0 + seq_len > max_seq_len) return cudaErrorInvalidValue;
   if (head_dim == 128)
-    return split ? launch_dh<128, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of)
-                 : launch_dh<128, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of);
+    return split ? launch_dh<128, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of, lens)
+                 : launch_dh<128, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of, lens);
   if (head_dim == 64)
-    return split ? launch_dh<64, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of)
-                 : launch_dh<64, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of);
+    return split ? launch_dh<64, true>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of, lens)
+                 : launch_dh<64, false>(q, q_lo, k, v, batch, seq_len, n_q_heads, n_kv_heads, max_seq_len, o, o_lo, stream, pos0, of, lens);
   return cudaErrorInvalidValue;
 }
 

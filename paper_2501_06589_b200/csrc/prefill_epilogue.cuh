@@ -58,6 +58,7 @@ __device__ __forceinline__ void epilogue_pair(const LargeMParams& p, int m, int 
           *reinterpret_cast<uint32_t*>(e.q_out_lo + static_cast<size_t>(m) * nq + n) =
               pack_f16x2(v0 - f16_lo(hi), v1 - f16_hi(hi));
       } else {
+        if (e.prefill_lens && m % e.prefill_seq_len >= e.prefill_lens[b]) break;  // padding row: nothing to cache
         const int nn = n < nq + nk ? n - nq : n - nq - nk;
         kv_t* cache = n < nq + nk ? e.k_cache : e.v_cache;
         const size_t off = ((static_cast<size_t>(b) * e.n_kv_heads + nn / Dh) * e.max_seq_len + pos) * Dh + (nn % Dh);

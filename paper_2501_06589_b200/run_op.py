@@ -34,6 +34,8 @@ def main():
     ap.add_argument("--standard", action="store_true", help="stack: standard residuals in every layer")
     ap.add_argument("--which", default="gate_up", choices=["qkv", "wo", "gate_up", "down"],
                     help="prefill_gemm: which projection's shape and epilogue")
+    ap.add_argument("--pairs", action="store_true",
+                    help="prefill_gemm: bf16 hi + lo activation pairs instead of the default binary16 operands")
     a = ap.parse_args()
     build.build()
     B.lib()
@@ -78,6 +80,21 @@ def main():
         o = torch.empty(bsz, Hq * Dh, device=dev)
         fn = lambda l: B.op_decode_attention(q, k[l], v[l], lens, Hq, Hkv, Dh, max_seq, scr, o)
         nbytes, flops = 2 * 2 * bsz * Hkv * kv * Dh, 0
+    elif a.op == "convert":          # one layer's gate/up weights bf16 -> binary16 (what the prompt pass does per layer)
+        W = w(2 * F, d)
+        dst = torch.empty(2 * F, d, dtype=torch.float16, device=dev)
+        fn = lambda l: B.op_convert_bf16_f16(W[l], dst)
+        nbytes, flops = 2 * 2 * 2 * F * d, 0
+    elif a.op == "prefill_gemm" and not a.pairs:
+        M = a.tokens
+        N, K, mode = {"gate_up": (2 * F, d, 1), "qkv": (s.qkv_rows, d, 3), "wo": (d, Hq * Dh, 0), "down": (d, F, 0)}[a.which]
+        A = torch.randn(M, K, device=dev).to(torch.float16)
+        W = [t.to(torch.float16) for t in w(N, K)]
+        add = torch.randn(M, N, device=dev) if mode == 0 else None
+        out = torch.empty(M, N, device=dev) if mode == 0 else \
+            torch.empty(M, N // 2 if mode == 1 else N, dtype=torch.float16, device=dev)
+        fn = lambda l: B.op_prefill_gemm_f16(A, W[l], mode, out, addend=add)
+        nbytes, flops = 0, 2.0 * M * N * K
     elif a.op == "prefill_gemm":
         M = a.tokens
         A = (torch.randn(M, d, device=dev)).to(torch.bfloat16)

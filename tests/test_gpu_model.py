@@ -669,6 +669,124 @@ def test_sequences_of_different_lengths_decode_together(B, persistent):
     model.close()
 
 
+@pytest.mark.parametrize("case", ["tiny_hybrid", "8b_shape"])
+def test_prompts_of_different_lengths_in_one_call(B, case):
+    """ladder_prefill_ragged: left-aligned prompts padded to a common length, true lengths on the host.  Every
+    sequence's first token, hidden state and logits against the oracle run on that sequence alone; cache rows behind
+    each length stay untouched; the lengths land in seq_lens; and the sequences then decode together."""
+    if case == "tiny_hybrid":
+        s, dtype = synth.replace(synth.SHAPES["tiny"], layer_is_ladder=(0, 1, 1, 1)), np.float64
+        lens, S, steps = [5, 150, 64, 1, 129], 150, 51            # 750 padded rows: the binary16 GEMM path
+    else:
+        s = synth.replace(synth.SHAPES["8b_hybrid"].with_layers(4), layer_is_ladder=(0, 0, 1, 1))
+        lens, S, steps, dtype = [70, 33, 128], 128, 86, np.float32
+    bsz = len(lens)
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    toks = synth.make_tokens(s, bsz, S)
+    max_seq = S + steps + 2
+    model = B.Model(w, bsz, max_seq, bsz * S)
+    cache = B.KVCache(s, bsz, max_seq, fill=CANARY)
+    nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+    hid = torch.zeros(bsz, s.d_model, device="cuda")
+    lg = torch.zeros(bsz, s.vocab_size, device="cuda")
+    allh = torch.zeros(bsz, S, s.d_model, device="cuda")
+    model.prefill_ragged(cache, torch.from_numpy(toks).cuda(), lens, next_tokens=nxt, final_hidden=hid, logits=lg,
+                         all_hidden=allh)
+    torch.cuda.synchronize()
+    assert model.device_status() == 0
+    assert cache.seq_lens.cpu().tolist() == lens
+    k5, v5 = cache.k5().view(torch.int16), cache.v5().view(torch.int16)
+    for b, L in enumerate(lens):
+        assert bool((k5[:, b, :, L:, :] == CANARY).all()) and not bool((k5[:, b, :, :L, :] == CANARY).any())
+        assert bool((v5[:, b, :, L:, :] == CANARY).all()) and not bool((v5[:, b, :, :L, :] == CANARY).any())
+    g_tok, g_hid, g_log = [nxt.clone()], [hid.clone()], [lg.clone()]
+    for _ in range(steps):
+        model.decode_step(cache, nxt, next_tokens=nxt, final_hidden=hid, logits=lg)
+        g_tok.append(nxt.clone())
+        g_hid.append(hid.clone())
+        g_log.append(lg.clone())
+    torch.cuda.synchronize()
+    assert model.device_status() == 0
+    assert cache.seq_lens.cpu().tolist() == [L + steps for L in lens]
+    g_tok = torch.stack(g_tok, 1).cpu().numpy()
+    g_hid = torch.stack(g_hid, 1).cpu().numpy()
+    g_log = torch.stack(g_log, 1).cpu().numpy()
+    cfg = oracle_cfg(s)
+    OW = O.OracleWeights(provider=synth.logical_provider(w, dtype))
+    total = Parity()
+    for b, L in enumerate(lens):
+        o_tok, o_hid, o_log = O.generate(cfg, OW, toks[b:b + 1, :L], steps, max_seq, dtype=dtype,
+                                         forced=g_tok[b:b + 1], return_logits=True)
+        total = total + compare_with_oracle(f"{case} ragged prompt {b} len {L}", g_tok[b:b + 1], g_hid[b:b + 1],
+                                            g_log[b:b + 1], o_tok, o_hid, o_log)
+        ref = O.forward(cfg, OW, toks[b:b + 1, :L], dtype=dtype, last_only=False, with_logits=False)
+        assert rel_err(allh[b, :L].cpu().numpy(), ref.hidden[0]) < HIDDEN_TOL        # every valid prompt position
+    total.check()
+    model.close()
+
+
+def _whole_model_flags(shape):
+    """Per-module flags of the whole model as include/ladder.h derives them from the layer mask."""
+    mask = shape.ladder_mask()
+    flags = []
+    for l, lad in enumerate(mask):
+        flags += [int(bool(lad) and (l == 0 or bool(mask[l - 1]))), int(bool(lad))]
+    return flags
+
+
+@pytest.mark.parametrize("mask,cut", [((1, 1, 1, 1), 2), ((0, 1, 1, 0), 2), ((0, 0, 1, 1), 2), ((1, 1, 0, 1), 1)])
+def test_pipeline_stages_hand_the_stream_state_on(B, mask, cut):
+    """Paper Sec. 5.1: two stage models (layers [0, cut) and [cut, 4) of the tiny shape, each with its own cache)
+    chained through the handed-on pair (x_m, x_{m-1}) reproduce the whole model bit for bit -- prompt pass and
+    decode steps -- and the pair the first stage hands on matches the oracle's stream state after `cut` layers."""
+    s = synth.replace(synth.SHAPES["tiny"], layer_is_ladder=mask)
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    bsz, S, steps = 3, 20, 6
+    max_seq = S + steps + 2
+    prompt = synth.make_tokens(s, bsz, S)
+    tok = torch.from_numpy(prompt).cuda()
+    flags = _whole_model_flags(s)
+    # ---- the whole model
+    whole = B.Model(w, bsz, max_seq, bsz * S)
+    wc = B.KVCache(s, bsz, max_seq)
+    ref_toks, ref_hids = gpu_generate(B, whole, wc, prompt, steps)
+    whole.close()
+    # ---- two stages: the whole model's weights and rule table, sliced
+    def stage(lo, hi):
+        sh = synth.replace(s, n_layers=hi - lo, layer_is_ladder=tuple(mask[lo:hi]), module_stale=tuple(flags[2 * lo:2 * hi]))
+        ws = synth.AbiWeights(sh, w.tok_embedding, w.final_norm, w.lm_head, w.attn_norm[lo:hi], w.w_qkv[lo:hi],
+                              w.w_o[lo:hi], w.mlp_norm[lo:hi], w.w_gate_up[lo:hi], w.w_down[lo:hi])
+        return B.Model(ws, bsz, max_seq, bsz * S), B.KVCache(sh, bsz, max_seq, fill=CANARY)
+    (m0, c0), (m1, c1) = stage(0, cut), stage(cut, 4)
+    d = s.d_model
+    big = (torch.zeros(bsz * S, d, device="cuda"), torch.zeros(bsz * S, d, device="cuda"))
+    small = (torch.zeros(bsz, d, device="cuda"), torch.zeros(bsz, d, device="cuda"))
+    nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+    hid = torch.zeros(bsz, d, device="cuda")
+    m0.stage_prefill(c0, tok, bsz, S, state_out=big)
+    m1.stage_prefill(c1, None, bsz, S, state_in=big, next_tokens=nxt, final_hidden=hid)
+    torch.cuda.synchronize()
+    toks, hids = [nxt.clone()], [hid.clone()]
+    # the handed-on pair against the oracle's stream state after `cut` layers
+    cfg = oracle_cfg(s)
+    OW = O.OracleWeights(provider=synth.logical_provider(w, np.float64))
+    older, newest = O.run_layers(cfg, OW, O.embed(OW, prompt, np.float64), 0, None, n_layers=cut, return_state=True)
+    assert rel_err(big[0].cpu().numpy().reshape(bsz, S, d), newest) < HIDDEN_TOL
+    assert rel_err(big[1].cpu().numpy().reshape(bsz, S, d), older) < HIDDEN_TOL
+    for _ in range(steps):
+        m0.stage_decode_step(c0, nxt, bsz, state_out=small)
+        m1.stage_decode_step(c1, None, bsz, state_in=small, next_tokens=nxt, final_hidden=hid)
+        toks.append(nxt.clone())
+        hids.append(hid.clone())
+    torch.cuda.synchronize()
+    assert m0.device_status() == 0 and m1.device_status() == 0
+    assert np.array_equal(torch.stack(toks, 1).cpu().numpy(), ref_toks)
+    assert np.array_equal(torch.stack(hids, 1).cpu().numpy(), ref_hids)
+    assert c0.seq_lens.cpu().tolist() == [S + steps] * bsz and c1.seq_lens.cpu().tolist() == [S + steps] * bsz
+    m0.close()
+    m1.close()
+
+
 # ----------------------------------------------------------------------------- full depth, every module live
 def truncated(w: synth.AbiWeights, shape: synth.ModelShape) -> synth.AbiWeights:
     """The first shape.n_layers layers of w as a model of their own (same tensors, nothing copied)."""

@@ -213,7 +213,7 @@ def parse_args(argv=None):
     ap.add_argument("--pdl", type=int, default=None)
     ap.add_argument("--batch", type=int, default=None, help="sequences decoded together (default: the configuration's)")
     ap.add_argument("--wide-impl", type=int, default=0,
-                    help="decode GEMM kernels: 0 = default, 1 = mma.sync for batch 9..64, 2 = tcgen05 for every batch")
+                    help="decode GEMM kernels: 0 = default, 2 = tcgen05 for every batch")
     ap.add_argument("--standard", action="store_true", help="the same shape with standard residuals (Eq. 1) in every layer")
     ap.add_argument("--mode", default=None, choices=["ladder", "standard", "parallel", "upper_bound"],
                     help="every layer in this architecture (paper Sec. 3.3.1) instead of the configuration's own")
@@ -227,8 +227,8 @@ def parse_args(argv=None):
                     help="feed the prompt in chunks of this many tokens per sequence (ladder_prefill_append): the prompt-pass "
                          "workspace then holds one chunk, which is what lets batch 64 of the 70B shape fit beside 141 GB of weights")
     ap.add_argument("--prefill-impl", type=int, default=0,
-                    help="prompt-pass GEMMs: 0 = default; 1 = mma.sync; "
-                         "2 = tcgen05, one bf16 per activation (not the precision the parity bound is stated for)")
+                    help="prompt-pass GEMMs: 0 = default; 2 = one bf16 per activation (not the precision the parity "
+                         "bound is stated for); 3 = bf16 hi + lo pairs at every size")
     ap.add_argument("--selftest-cpu", action="store_true", help=argparse.SUPPRESS)
     return ap.parse_args(argv)
 

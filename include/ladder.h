@@ -365,17 +365,18 @@ ladder_status_t ladder_op_convert_bf16_f16(const void* src, void* dst, int64_t n
  *       converted to binary16 in a per-model scratch once per call (1.7 GB at the 70B shape; model creation falls
  *       back to mode 3 when that does not fit) and every activation is ONE binary16 value -- for calls of at
  *       least 256 tokens, bf16 hi + lo pairs (mode 3) for shorter ones;
- *   1 = warp-level mma.sync kernel with bf16 hi + lo activations (kept as a cross-check);
  *   2 = the tcgen05 kernel with ONE bf16 value per activation: the usual bf16 inference precision, but every stored
  *       activation is rounded at 2^-9, which by itself reaches 1.6e-2 of hidden-state error after 8 layers of the
  *       8B shape;
- *   3 = the tcgen05 kernel with bf16 hi + lo activation pairs (two MMAs per product) at every size. */
+ *   3 = the tcgen05 kernel with bf16 hi + lo activation pairs (two MMAs per product) at every size;
+ *   4 = as 0, but every GEMM with one CTA per output tile (0 runs single-value operands on pairs of CTAs,
+ *       tcgen05.mma.cta_group::2 with 256 x 256 tiles, wherever there is at least one such tile per pair of SMs). */
 void ladder_set_prefill_gemm_impl(int32_t impl);
 
-/* Decode GEMM for batch 5..64: 0 = tcgen05 kernel (weights as the M side of the MMA, TMA tiles, TMEM accumulators,
- * equal K-block ranges per CTA with a deterministic fix-up of shared tiles; default), 1 = the earlier mma.sync kernel
- * (cross-check; batch 5..8 then runs with ONE bf16 value per activation).  PROCESS-WIDE and not thread-safe: a
- * switch for tests and A/B measurements, not for serving code. */
+/* Decode GEMM: 0 = batch 1..4 on the mma.sync weight-streaming kernel, batch 5..64 on the tcgen05 kernel (weights as
+ * the M side of the MMA, TMA tiles, TMEM accumulators, equal K-block ranges per CTA with a deterministic fix-up of
+ * shared tiles; default); 2 = the tcgen05 kernel for every batch.  PROCESS-WIDE and not thread-safe: a switch for
+ * tests and A/B measurements, not for serving code. */
 void ladder_set_decode_wide_impl(int32_t impl);
 
 /* Causal grouped-query attention of the prefill path for one layer:
@@ -385,6 +386,19 @@ void ladder_set_decode_wide_impl(int32_t impl);
 ladder_status_t ladder_op_prefill_attention(const void* q, const void* q_lo, const void* k, const void* v, int32_t batch,
                                             int32_t seq_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
                                             int32_t max_seq_len, void* o, void* o_lo, void* cuda_stream);
+
+/* The same kernel with the arguments the chunked and ragged prompt passes use (ladder_prefill_append,
+ * ladder_prefill_ragged; causal Llama attention of paper Sec. 3.3.1 over a cache that already holds pos0 rows):
+ *   pos0            the seq_len queries sit at positions pos0 .. pos0+seq_len-1; cache rows 0 .. pos0+seq_len-1 are read
+ *                   (pos0 >= 0, pos0 + seq_len <= max_seq_len, else LADDER_ERR_INVALID_ARG);
+ *   lens            optional, DEVICE int32 [batch]: sequence b has lens[b] <= seq_len valid query rows; the rows
+ *                   behind them are padding: neither read as keys / values nor written to o;
+ *   out_binary16    non-zero: o receives ONE binary16 value per element (o_lo must be NULL; q_lo may be given).
+ * All pointers are device pointers, 16-byte aligned (else LADDER_ERR_INVALID_ARG); nothing is allocated. */
+ladder_status_t ladder_op_prefill_attention_at(const void* q, const void* q_lo, const void* k, const void* v,
+                                               int32_t batch, int32_t seq_len, int32_t n_q_heads, int32_t n_kv_heads,
+                                               int32_t head_dim, int32_t max_seq_len, int32_t pos0, const int32_t* lens,
+                                               int32_t out_binary16, void* o, void* o_lo, void* cuda_stream);
 
 #ifdef __cplusplus
 }

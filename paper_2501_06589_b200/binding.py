@@ -24,7 +24,7 @@ EXPORTS = [
     "ladder_decode_step", "ladder_decode_step_host", "ladder_prefill_host", "ladder_set_position",
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
     "ladder_last_error", "ladder_op_smallm_gemm", "ladder_decode_attention_scratch_bytes",
-    "ladder_op_decode_attention", "ladder_op_prefill_gemm", "ladder_op_prefill_attention",
+    "ladder_op_decode_attention", "ladder_op_prefill_gemm", "ladder_op_prefill_attention", "ladder_op_prefill_attention_at",
     "ladder_op_decode_attention_noalloc", "ladder_set_prefill_gemm_impl", "ladder_set_decode_wide_impl",
     "ladder_op_prefill_gemm_f16", "ladder_op_convert_bf16_f16",
 ]
@@ -139,6 +139,10 @@ def lib() -> C.CDLL:
         L.ladder_op_prefill_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                                   C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                   C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ladder_op_prefill_attention_at.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                                     C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                                     C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                                     C.c_void_p]
         _lib = L
     return _lib
 
@@ -391,13 +395,13 @@ def op_decode_attention_noalloc(q, k, v, kv_len, n_q_heads, n_kv_heads, head_dim
 
 def set_prefill_gemm_impl(impl: int):
     """Test switch (process-wide).  0 = default (tcgen05, binary16 operands for calls of >= 256 tokens, else bf16
-    pairs); 1 = warp-level mma.sync kernel; 2 = tcgen05, one bf16 value per activation; 3 = tcgen05, bf16 hi + lo
-    pairs at every size."""
+    pairs); 2 = tcgen05, one bf16 value per activation; 3 = tcgen05, bf16 hi + lo pairs at every size; 4 = as 0 with
+    one CTA per tile everywhere (no CTA pairs)."""
     lib().ladder_set_prefill_gemm_impl(impl)
 
 
 def set_decode_wide_impl(impl: int):
-    """Decode GEMM for batch 9..64: 0 = tcgen05 kernel (default), 1 = the earlier mma.sync kernel."""
+    """Decode GEMM: 0 = tcgen05 kernel for batch 5..64 (default), 2 = tcgen05 kernel for every batch."""
     lib().ladder_set_decode_wide_impl(impl)
 
 
@@ -420,6 +424,13 @@ def op_convert_bf16_f16(src, dst):
 
 
 def op_prefill_attention(q, k, v, batch, seq_len, n_q_heads, n_kv_heads, head_dim, max_seq_len, o, q_lo=None,
-                         o_lo=None):
-    _check(lib().ladder_op_prefill_attention(_ptr(q), _ptr(q_lo), _ptr(k), _ptr(v), batch, seq_len, n_q_heads,
-                                             n_kv_heads, head_dim, max_seq_len, _ptr(o), _ptr(o_lo), _stream()))
+                         o_lo=None, pos0=None, lens=None, out_binary16=False):
+    """Prompt-pass attention of one layer.  With pos0 / lens / out_binary16 it goes through the entry point that
+    takes a starting position, per-sequence lengths and a binary16 output."""
+    if pos0 is None and lens is None and not out_binary16:
+        _check(lib().ladder_op_prefill_attention(_ptr(q), _ptr(q_lo), _ptr(k), _ptr(v), batch, seq_len, n_q_heads,
+                                                 n_kv_heads, head_dim, max_seq_len, _ptr(o), _ptr(o_lo), _stream()))
+        return
+    _check(lib().ladder_op_prefill_attention_at(_ptr(q), _ptr(q_lo), _ptr(k), _ptr(v), batch, seq_len, n_q_heads,
+                                                n_kv_heads, head_dim, max_seq_len, int(pos0 or 0), _ptr(lens),
+                                                1 if out_binary16 else 0, _ptr(o), _ptr(o_lo), _stream()))

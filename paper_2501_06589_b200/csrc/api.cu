@@ -36,9 +36,8 @@ bool g_kernels_ready = false;
 cudaError_t kernels_ready() {  // opt-in to large dynamic shared memory, once per process
   if (g_kernels_ready) return cudaSuccess;
   cudaError_t e = smallm_gemm_init();
-  if (e == cudaSuccess) e = largem_gemm_init();
   if (e == cudaSuccess) e = largem_gemm_tc_init();
-  if (e == cudaSuccess) e = prefill_attention_init();
+  if (e == cudaSuccess) e = prefill_attention_tc_init();
   if (e == cudaSuccess) g_kernels_ready = true;
   return e;
 }
@@ -394,7 +393,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       a.max_len = c.max_seq_len;
       a.scratch = m->attn_scratch;
       a.o = m->o_dec;
-      const bool handover = batch > 4 && m->wide_opack && wide_handover();  // operands pass from kernel to kernel
+      const bool handover = batch > 4 && m->wide_opack;  // operands pass from kernel to kernel
       if (handover) {
         a.o_pack = m->wide_opack;
         a.o_pack_bp = wide_padded_batch(batch);
@@ -439,7 +438,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       p.epi_mode = EPI_SWIGLU;
       p.out = m->h_dec;
       p.status = m->status;
-      const bool handover = batch > 4 && m->wide_hpack && wide_handover();
+      const bool handover = batch > 4 && m->wide_hpack;
       if (handover) p.wide_pack_out = m->wide_hpack;
       q.gemm(1, p, lad);
 
@@ -589,7 +588,7 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       p.status = m->status;
       did(launch_largem_gemm(p, st));
       did(launch_prefill_attention(m->q_pf, q_lo, p.qkv.k_cache, p.qkv.v_cache, batch, S, Hq, Hkv, Dh, c.max_seq_len,
-                                   m->o_pf, o_lo, st, pos0, f16, d_lens));
+                                   m->o_pf, o_lo, st, pos0, f16, d_lens, m->status));
       LargeMParams o = {};
       o.A = m->o_pf;
       o.A_lo = o_lo;
@@ -1818,6 +1817,26 @@ ladder_status_t ladder_op_prefill_attention(const void* q, const void* q_lo, con
       static_cast<const __half*>(q), static_cast<const __half*>(q_lo), static_cast<const kv_t*>(k),
       static_cast<const kv_t*>(v), batch, seq_len, n_q_heads, n_kv_heads, head_dim, max_seq_len,
       static_cast<__nv_bfloat16*>(o), static_cast<__nv_bfloat16*>(o_lo), static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
+}
+
+ladder_status_t ladder_op_prefill_attention_at(const void* q, const void* q_lo, const void* k, const void* v,
+                                               int32_t batch, int32_t seq_len, int32_t n_q_heads, int32_t n_kv_heads,
+                                               int32_t head_dim, int32_t max_seq_len, int32_t pos0, const int32_t* lens,
+                                               int32_t out_binary16, void* o, void* o_lo, void* cuda_stream) {
+  if (!q || !k || !v || !o || batch < 1 || seq_len < 1 || pos0 < 0 || seq_len > max_seq_len - pos0 || n_kv_heads < 1 ||
+      n_q_heads < 1 || n_q_heads % n_kv_heads || (head_dim != 64 && head_dim != 128))
+    return LADDER_ERR_INVALID_ARG;
+  if (out_binary16 ? o_lo != nullptr : (q_lo == nullptr) != (o_lo == nullptr)) return LADDER_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(q_lo) | reinterpret_cast<uintptr_t>(k) |
+       reinterpret_cast<uintptr_t>(v) | reinterpret_cast<uintptr_t>(o) | reinterpret_cast<uintptr_t>(o_lo)) & 15)
+    return LADDER_ERR_INVALID_ARG;
+  if (kernels_ready() != cudaSuccess) return LADDER_ERR_CUDA;
+  cudaError_t e = launch_prefill_attention(
+      static_cast<const __half*>(q), static_cast<const __half*>(q_lo), static_cast<const kv_t*>(k),
+      static_cast<const kv_t*>(v), batch, seq_len, n_q_heads, n_kv_heads, head_dim, max_seq_len,
+      static_cast<__nv_bfloat16*>(o), static_cast<__nv_bfloat16*>(o_lo), static_cast<cudaStream_t>(cuda_stream), pos0,
+      out_binary16 != 0, lens);
   return e == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;
 }
 

@@ -1,4 +1,4 @@
-// Weight-streaming GEMM of the decode path for batch <= 8:  acc[b, n] = sum_k act[b, k] * W[n, k].
+// Weight-streaming GEMM of the decode path for batch <= 4:  acc[b, n] = sum_k act[b, k] * W[n, k].
 //
 // HBM-bound by construction: every weight byte is read exactly once.  The rows of W are cut into
 // 8-row units; persistent CTAs (one per SM) claim batches of consecutive units through an atomic
@@ -11,9 +11,9 @@
 //     bulk async copies (TMA engine, L2 evict-first) -- into a 4-stage ring.  4 KB segments are
 //     what it takes to reach the read ceiling of the part (2 KB: ~5 % lower, 1 KB: half);
 //   * four stager warps: turn the fp32 activations of the next K chunk into MMA operands:
-//     (x * gain) as a bf16 high part plus a bf16 low part (x ~ hi + lo, ~16 mantissa bits).  For
-//     batch <= 4 the high parts occupy columns 0-3 and the low parts columns 4-7 of ONE 8-column
-//     MMA tile, so the extra precision costs no extra MMA; batch 5..8 uses a single bf16.  The
+//     (x * gain) as a bf16 high part plus a bf16 low part (x ~ hi + lo, ~16 mantissa bits).  The
+//     high parts occupy columns 0-3 and the low parts columns 4-7 of ONE 8-column MMA tile, so the
+//     extra precision costs no extra MMA (wider batches run on the tcgen05 kernel).  The
 //     batches all walk the chunks in the same cyclic order, so the stagers free-run one chunk ahead.
 //     They also form the RMSNorm sum of squares while staging the first batch's chunks;
 //   * four consumer warps: split each tile along K, read 16 contiguous bytes of a weight row and
@@ -40,16 +40,12 @@
 namespace ladder {
 
 // batch 9..64: tcgen05 kernel (default) or the earlier mma.sync kernel (cross-check)
-cudaError_t launch_smallm_gemm_wide(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);
-cudaError_t smallm_gemm_wide_init();
-size_t smallm_gemm_wide_smem_bytes(int batch);
 cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);
 cudaError_t smallm_gemm_wide_tc_init();
 size_t smallm_gemm_wide_tc_smem_bytes(int batch);
 size_t smallm_gemm_wide_tc_scratch_floats(int N, int K, int batch);
-static int g_wide_impl = 0;  // 0 = tcgen05, 1 = mma.sync, 2 = tcgen05 for every batch (also <= 8)
-void set_decode_wide_impl(int impl) { g_wide_impl = (impl == 1 || impl == 2) ? impl : 0; }
-bool wide_handover() { return g_wide_impl != 1; }
+static int g_wide_impl = 0;  // 0 = tcgen05 kernel for batch > 4, 2 = tcgen05 kernel for every batch
+void set_decode_wide_impl(int impl) { g_wide_impl = impl == 2 ? 2 : 0; }
 
 namespace {
 
@@ -138,12 +134,8 @@ __device__ __forceinline__ void slab_loop(float (&acc0)[4], float (&acc1)[4], co
   }
 }
 
-#ifdef DG_TRACE
-// per-CTA timeline for tuning builds only: [0] start ns, [1] end ns, [2] SM id, [3] units processed
-__device__ unsigned long long g_trace[148 * 4];
-#endif
 
-template <bool PACKED, bool NORM>
+template <bool NORM>
 __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMParams p, const Schedule sched) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -199,15 +191,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
     const uint8_t* Wb = reinterpret_cast<const uint8_t*>(p.W);
     bool ok = true;
     int it = 0, n = 0;
-#ifdef DG_TRACE
-    int traced_units = 0;
-    if (lane == 0) {
-      uint32_t smid;
-      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-      g_trace[blockIdx.x * 4 + 0] = global_timer_ns();
-      g_trace[blockIdx.x * 4 + 2] = smid;
-    }
-#endif
     int c = 0;
     while (ok) {
       // one claim at a time (claiming ahead would let a CTA hoard batches it cannot start yet);
@@ -233,10 +216,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
       u0 = __shfl_sync(0xffffffffu, u0, 0);
       nu = __shfl_sync(0xffffffffu, nu, 0);
       if (nu == 0) break;
-#ifdef DG_TRACE
-      traced_units += nu;
-      if (lane == 0) g_trace[blockIdx.x * 4 + 3] = traced_units;
-#endif
       const int row0 = u0 * 8;
       for (int ch = 0; ch < nchunk && ok; ++ch) {
         const int k0 = ch * TK;
@@ -350,14 +329,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
           hi.w = pack_bf16x2(y[6], y[7]);
           const uint32_t dst = act_u32 + b * PITCH + (st + u * 128) * 16;
           sts128(dst, hi);
-          if (PACKED) {
-            uint4 lo;
-            lo.x = pack_bf16x2(y[0] - bf16_lo(hi.x), y[1] - bf16_hi(hi.x));
-            lo.y = pack_bf16x2(y[2] - bf16_lo(hi.y), y[3] - bf16_hi(hi.y));
-            lo.z = pack_bf16x2(y[4] - bf16_lo(hi.z), y[5] - bf16_hi(hi.z));
-            lo.w = pack_bf16x2(y[6] - bf16_lo(hi.w), y[7] - bf16_hi(hi.w));
-            sts128(dst + 4 * PITCH, lo);
-          }
+          uint4 lo;
+          lo.x = pack_bf16x2(y[0] - bf16_lo(hi.x), y[1] - bf16_hi(hi.x));
+          lo.y = pack_bf16x2(y[2] - bf16_lo(hi.y), y[3] - bf16_hi(hi.y));
+          lo.z = pack_bf16x2(y[4] - bf16_lo(hi.z), y[5] - bf16_hi(hi.z));
+          lo.w = pack_bf16x2(y[6] - bf16_lo(hi.w), y[7] - bf16_hi(hi.w));
+          sts128(dst + 4 * PITCH, lo);
         }
       }
     };
@@ -372,10 +349,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
       if (w == 2) ok = false;
       if (w != 0) break;  // the consumers have run out of work (or a protocol error)
       store_rows(0);
-      if (!PACKED && batch > 4) {
-        load_rows(ch, 1);
-        store_rows(1);
-      }
       if (NORM && r == nchunk - 1) {  // every chunk has been staged once: publish the sums
 #pragma unroll
         for (int b = 0; b < 8; ++b) {
@@ -426,7 +399,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
       auto value = [&](int r, int b) -> float {
         const int a = r >> 4, rr = r & 15;
         float s = column(a, rr, b);
-        if (PACKED) s += column(a, rr, b + 4);  // high-part product + low-part product
+        s += column(a, rr, b + 4);  // high-part product + low-part product
         if (NORM) s *= rstd_s[b];
         return s;
       };
@@ -435,9 +408,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
       if (lane == 0) mbar_arrive(&red_free[slot]);  // the consumers may refill this slot
     }
     if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
-#ifdef DG_TRACE
-    if (ft == 0) g_trace[blockIdx.x * 4 + 1] = global_timer_ns();
-#endif
     return;
   }
 
@@ -448,7 +418,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
   const uint32_t ring_u32 = smem_u32(ring);
   const uint32_t act_u32 = smem_u32(act);
   // which activation row feeds MMA column g: packed = hi rows 0-3 then lo rows 4-7 of batch g & 3
-  const bool col_valid = PACKED ? ((g & 3) < batch) : (g < batch);
+  const bool col_valid = (g & 3) < batch;
   bool ok = true;
 
   uint4 bf[SPW];
@@ -524,9 +494,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_gemm_kernel(const SmallMPa
   if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
 }
 
-template <bool PACKED>
 cudaError_t launch_small(const SmallMParams& p, cudaStream_t stream, bool pdl, int grid) {
-  auto kern = p.act_mode == ACT_F32_NORM ? decode_gemm_kernel<PACKED, true> : decode_gemm_kernel<PACKED, false>;
+  auto kern = p.act_mode == ACT_F32_NORM ? decode_gemm_kernel<true> : decode_gemm_kernel<false>;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kThreads);
@@ -543,28 +512,18 @@ cudaError_t launch_small(const SmallMParams& p, cudaStream_t stream, bool pdl, i
 
 }  // namespace
 
-#ifdef DG_TRACE
-extern "C" int ladder_debug_read_trace(unsigned long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : 1;
-}
-#endif
 
 cudaError_t smallm_gemm_init() {
-  cudaError_t e = cudaFuncSetAttribute(decode_gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  cudaError_t e = cudaFuncSetAttribute(decode_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_gemm_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_gemm_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-  if (e == cudaSuccess) e = smallm_gemm_wide_init();
+    e = cudaFuncSetAttribute(decode_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e == cudaSuccess) e = smallm_gemm_wide_tc_init();
   return e;
 }
 
 size_t smallm_gemm_smem_bytes(int batch) {
   if (batch <= 4) return SMEM;
-  const size_t wide = std::max(smallm_gemm_wide_smem_bytes(batch > 8 ? batch : 9), smallm_gemm_wide_tc_smem_bytes(batch));
+  const size_t wide = smallm_gemm_wide_tc_smem_bytes(batch);
   return std::max(wide, static_cast<size_t>(SMEM));
 }
 
@@ -573,16 +532,13 @@ size_t smallm_gemm_scratch_floats(int N, int K, int batch) {
 }
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
-  if (g_wide_impl == 2) return launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count);
-  // Batch 5..8 on the tcgen05 kernel by default: this file's kernel holds a bf16 hi + lo activation pair only for
-  // batch <= 4 (one 8-column MMA tile) and would run 5..8 with a single bf16 value, which costs a decimal digit of
-  // hidden-state accuracy.  With the mma.sync cross-check selected (impl 1) they still run here.
-  if (p.batch > 4 && g_wide_impl == 0) return launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count);
-  if (p.batch > 8) return launch_smallm_gemm_wide(p, stream, pdl, sm_count);
+  // Batch 5..64 on the tcgen05 kernel: this file's kernel holds a bf16 hi + lo activation pair only for batch <= 4
+  // (one 8-column MMA tile).
+  if (p.batch > 4 || g_wide_impl == 2) return launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count);
   if (!p.work) return cudaErrorInvalidValue;
   const int units = p.N >> 3;
   const int grid = units < sm_count ? units : sm_count;
-  return p.batch <= 4 ? launch_small<true>(p, stream, pdl, grid) : launch_small<false>(p, stream, pdl, grid);
+  return launch_small(p, stream, pdl, grid);
 }
 
 }  // namespace ladder

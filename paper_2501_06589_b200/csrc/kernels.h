@@ -65,7 +65,7 @@ struct SmallMParams {
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);
 size_t smallm_gemm_smem_bytes(int batch);
 size_t smallm_gemm_scratch_floats(int N, int K, int batch);
-void set_decode_wide_impl(int impl);  // batch 9..64: 0 = tcgen05 (default), 1 = mma.sync
+void set_decode_wide_impl(int impl);  // 0 = tcgen05 kernel for batch 5..64 (default), 2 = for every batch
 
 // Decode attention (split over the cache) and its combine step.
 struct DecodeAttnParams {
@@ -83,7 +83,6 @@ struct DecodeAttnParams {
   int o_pack_bp;                // padded batch of that operand (16 / 32 / 64); rows batch..bp-1 are written as zero
 };
 int wide_padded_batch(int batch);  // Bp of the batch 9..64 GEMM kernel
-bool wide_handover();              // the tcgen05 kernel is the one in use for batch 9..64 (it alone reads staged operands)
 int decode_attention_splits(int batch, int n_kv_heads, int max_len, int sm_count);
 // Longest cache the decode attention handles: its merge step holds one weight per 64-key split, at most 1024.
 constexpr int kDecodeAttnMaxKeys = 64 * 1024;
@@ -173,12 +172,12 @@ struct LargeMParams {
   int f16;                 // A and W hold binary16 instead of bf16 (one value per activation, A_lo unused), and the
                            // 16-bit outputs (EPI_SWIGLU, EPI_BF16) are written as binary16 too; tcgen05 kernel only
 };
-// Dispatches to the tcgen05 kernel (default) or the warp-level mma.sync kernel (set_prefill_gemm_impl(1)).
+// The tcgen05 kernel on every SM of the current device.
 cudaError_t launch_largem_gemm(const LargeMParams& p, cudaStream_t stream);
 cudaError_t launch_largem_gemm_tc(const LargeMParams& p, cudaStream_t stream, int sm_count);
 cudaError_t largem_gemm_tc_init();
 // 0 = default: tcgen05 with binary16 operands (one value per activation, the layer's weights converted once per
-// call) for calls of at least kPrefillF16MinTokens tokens, bf16 hi + lo pairs below; 1 = mma.sync (pairs);
+// call) for calls of at least kPrefillF16MinTokens tokens, bf16 hi + lo pairs below;
 // 2 = tcgen05 with single-bf16 activations; 3 = tcgen05 with bf16 hi + lo pairs at every size
 void set_prefill_gemm_impl(int impl);
 int prefill_gemm_impl();
@@ -190,11 +189,13 @@ bool prefill_single_bf16();            // the prompt pass feeds its GEMMs one bf
 // lens (device, optional): sequence b holds lens[b] <= seq_len valid rows (rows stay seq_len apart); the padding
 // rows behind them are neither read as keys nor written as outputs.
 // pos0: the seq_len queries sit at positions pos0 .. pos0 + seq_len - 1 and attend to cache rows 0 .. their own.
+// status (device, optional): receives LADDER_DEV_TIMEOUT if a bounded wait of the kernel runs out.
 cudaError_t launch_prefill_attention(const __half* q, const __half* q_lo, const kv_t* k,
                                      const kv_t* v, int batch, int seq_len, int n_q_heads, int n_kv_heads,
                                      int head_dim, int max_seq_len, __nv_bfloat16* o, __nv_bfloat16* o_lo,
                                      cudaStream_t stream, int pos0 = 0, bool out_f16 = false,
-                                     const int32_t* lens = nullptr);
+                                     const int32_t* lens = nullptr, int32_t* status = nullptr);
+cudaError_t prefill_attention_tc_init();
 
 // Small element-wise / gather kernels.
 cudaError_t launch_embed(const int32_t* tokens, const __nv_bfloat16* table, int rows, int d, int vocab, float* x,
@@ -219,7 +220,5 @@ cudaError_t launch_argmax_advance(const float* logits, int batch, int vocab, int
 // One-time opt-in to large dynamic shared memory for every kernel (call once per process/device,
 // outside any stream capture).
 cudaError_t smallm_gemm_init();
-cudaError_t largem_gemm_init();
-cudaError_t prefill_attention_init();
 
 }  // namespace ladder

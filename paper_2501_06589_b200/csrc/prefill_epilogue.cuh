@@ -1,5 +1,5 @@
-// Epilogue of the prefill GEMMs, shared by the warp-level and the tcgen05 implementation: the
-// accumulator pair (m, n), (m, n+1) -- n even -- goes through the fused tail of its layer step.
+// Epilogue of the prefill GEMMs: the accumulator pair (m, n), (m, n+1) -- n even -- goes through the fused tail of
+// its layer step.
 #pragma once
 #include "common.cuh"
 #include "kernels.h"

@@ -249,6 +249,212 @@ largem_gemm_tc_kernel(const LargeMParams p, const __grid_constant__ CUtensorMap 
   }
 }
 
+// ---------------------------------------------------------------- CTA pairs (cta_group::2)
+// The same GEMM with 256 x 256 output tiles computed by a PAIR of CTAs on neighbouring SMs (a cluster of two):
+// every CTA stages its own 128 rows of A and its own 128 of the tile's 256 W rows, and the leader's MMA thread issues
+// tcgen05.mma.cta_group::2 (M 256, N 256, K 16), which reads both CTAs' shared memory and writes 128 accumulator
+// rows into each CTA's tensor memory.  Per MMA a CTA's shared memory now supplies 8 KB instead of 12 KB and per K
+// block takes in 32 KB instead of 48 KB: with one CTA per tile the operand traffic (reads by the tensor core plus
+// writes by the TMA unit) exceeds what shared memory delivers per cycle, which is what held that kernel near 70 %
+// of the tensor rate.  Single-value operands only (binary16, or one bf16 value per activation).
+//   warp 0   TMA producer in BOTH CTAs; the copies of both complete on the LEADER's full barrier (the leader
+//            announces the bytes of both); no multicast: each CTA fetches only what it alone needs;
+//   warp 1   leader: the MMA issuer; tcgen05.commit arrives on the ring's empty barriers and on the accumulator-full
+//            barriers of BOTH CTAs.  In both CTAs this warp owns the (paired) TMEM allocation;
+//   warps 2-5 epilogue of the CTA's own 128 rows; all eight epilogue warps of the pair release an accumulator on
+//            the leader's barrier.
+// The pair meets at a cluster barrier after set-up and before the tensor memory is freed.  Every wait is bounded.
+constexpr int P2_STAGES = 6, P2_A_BYTES = 128 * BK * 2, P2_STAGE_BYTES = 2 * P2_A_BYTES;  // A half + W half: 32 KB
+constexpr int P2_OFF_BARS = P2_STAGES * P2_STAGE_BYTES;
+constexpr int P2_SMEM = P2_OFF_BARS + 24 * 8 + 1024;
+constexpr int P2_BN = 256, P2_BM = 256, P2_GROUP_M = 8;  // bands of 8 x 256 rows (4 and 16 measured slower)
+constexpr uint32_t P2_IDESC_F16 = (1u << 4) | (static_cast<uint32_t>(P2_BN >> 3) << 17) |
+                                  (static_cast<uint32_t>(P2_BM >> 4) << 24);
+constexpr uint32_t P2_IDESC_BF16 = P2_IDESC_F16 | (1u << 7) | (1u << 10);
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// the address of this CTA's shared-memory location `addr` as seen in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// 2-D tile into this CTA's shared memory; completes on a barrier that may live in the peer CTA
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(bar_cluster), "r"(x), "r"(y)
+      : "memory");
+}
+// arrives (once all MMAs issued so far have completed) on the barrier at this offset in BOTH CTAs of the pair
+__device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"(mask)
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+largem_gemm_tc_pair_kernel(const LargeMParams p, const __grid_constant__ CUtensorMap map_a,
+                           const __grid_constant__ CUtensorMap map_w) {
+  const uint32_t kIdesc = p.f16 ? P2_IDESC_F16 : P2_IDESC_BF16;
+  constexpr int kTmemCols = 2 * P2_BN;  // two fp32 accumulators of 256 columns (128 rows of them in each CTA)
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + P2_OFF_BARS);
+  uint64_t* empty = full + P2_STAGES;
+  uint64_t* tmem_full = empty + P2_STAGES;
+  uint64_t* tmem_empty = tmem_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();  // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int tiles_m = (p.M + P2_BM - 1) / P2_BM, tiles_n = (p.N + P2_BN - 1) / P2_BN;
+  const int n_tiles = tiles_m * tiles_n;
+  const int nkb = (p.K + BK - 1) / BK;
+  auto coords = [&](int t, int& tm, int& tn) {  // bands of P2_GROUP_M m-tiles, m fastest inside a band
+    const int per_band = P2_GROUP_M * tiles_n;
+    const int band = t / per_band, r = t - band * per_band;
+    const int m_first = band * P2_GROUP_M;
+    const int band_m = min(P2_GROUP_M, tiles_m - m_first);
+    tm = m_first + r % band_m;
+    tn = r / band_m;
+  };
+
+  if (tid == 0) {
+    for (int s = 0; s < P2_STAGES; ++s) {
+      mbar_init(&full[s], 1);   // used in the leader: its producer's arrive + the bytes of both CTAs
+      mbar_init(&empty[s], 1);  // one commit
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&tmem_full[a], 1);
+      mbar_init(&tmem_empty[a], 8);  // used in the leader: four epilogue warps of each CTA
+    }
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "n"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers are initialised and its tensor memory allocated
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      bool ok = true;
+      int it = 0;
+      for (int t = pair; t < n_tiles && ok; t += n_pairs) {
+        int tm, tn;
+        coords(t, tm, tn);
+        const int m0 = tm * P2_BM + static_cast<int>(rank) * 128, n0 = tn * P2_BN + static_cast<int>(rank) * 128;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % P2_STAGES;
+          ok = mbar_wait_bounded(&empty[s], ((it / P2_STAGES) & 1) ^ 1u);
+          if (!ok) break;
+          uint8_t* st = smem + s * P2_STAGE_BYTES;
+          const uint32_t bar = mapa_u32(smem_u32(&full[s]), 0);  // the leader's barrier
+          if (rank == 0) mbar_expect_tx(&full[s], 2 * P2_STAGE_BYTES);
+          tma_load_2d_pair(st, &map_a, kb * BK, m0, bar);
+          tma_load_2d_pair(st + P2_A_BYTES, &map_w, kb * BK, n0, bar);
+        }
+      }
+      if (!ok) {
+        if (p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
+        const uint64_t t0 = global_timer_ns();  // copies still in flight land in this CTA's shared memory: let them
+        while (global_timer_ns() - t0 < 100000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader only)
+    if (lane == 0 && rank == 0) {
+      bool ok = true;
+      int it = 0, i = 0;
+      for (int t = pair; t < n_tiles && ok; t += n_pairs, ++i) {
+        const int ab = i & 1;
+        ok = mbar_wait_bounded(&tmem_empty[ab], ((i >> 1) & 1) ^ 1u);  // both epilogues have drained this accumulator
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + ab * P2_BN;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % P2_STAGES;
+          ok = mbar_wait_bounded(&full[s], (it / P2_STAGES) & 1);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + s * P2_STAGE_BYTES);
+          const uint64_t da = smem_desc(a_addr), dw = smem_desc(a_addr + P2_A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            tc_mma_pair(d_tmem, da + 2 * k, dw + 2 * k, kIdesc, (kb > 0 || k > 0) ? 1u : 0u);
+          tc_commit_pair(&empty[s]);  // the stage is free in both CTAs once these MMAs have read it
+        }
+        if (ok) tc_commit_pair(&tmem_full[ab]);  // accumulator complete, in both CTAs
+      }
+      if (!ok && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+    const int q = warp & 3;  // the TMEM lane quarter this warp may access
+    bool ok = true;
+    int i = 0;
+    for (int t = pair; t < n_tiles; t += n_pairs, ++i) {
+      const int ab = i & 1;
+      int tm, tn;
+      coords(t, tm, tn);
+      const int m0 = tm * P2_BM + static_cast<int>(rank) * 128, n0 = tn * P2_BN;
+      if (ok) ok = mbar_wait_bounded(&tmem_full[ab], (i >> 1) & 1);
+      if (!ok) break;
+      tc_fence_after();
+      const int m = m0 + q * 32 + lane;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + ab * P2_BN;
+      for (int c = 0; c < P2_BN; c += 32) {
+        if (n0 + c >= p.N) break;  // uniform: the tile's tail columns do not exist
+        uint32_t r[32];
+        tc_ld32(taddr + c, r);
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          epilogue_pair(p, m, n0 + c + 2 * j, __uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&tmem_empty[ab]), 0));
+    }
+    if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // nobody in the pair reads the other's shared or tensor memory any more
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
+  }
+}
+
 // ---------------------------------------------------------------- host: tensor maps
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -288,6 +494,8 @@ cudaError_t largem_gemm_tc_init() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(largem_gemm_tc_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              TcCfg<128, false>::SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(largem_gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P2_SMEM);
   return e;
 }
 
@@ -309,10 +517,61 @@ cudaError_t launch_bn(const LargeMParams& p, cudaStream_t stream, int sm_count) 
 }
 }  // namespace
 
+namespace {
+int g_prefill_impl = 0;
+int g_sm_count = 0;
+bool g_pair_tiles = true;  // 256 x 256 tiles on CTA pairs where the operands are single values and tiles are plenty
+
+// CTA pairs: grid = 2 x min(pairs of SMs, tiles), launched as clusters of two
+cudaError_t launch_pair(const LargeMParams& p, cudaStream_t stream, int sm_count) {
+  CUtensorMap ma, mw;
+  const bool f16 = p.f16 != 0;
+  cudaError_t e = make_map(&ma, p.A, p.M, p.K, 128, f16);
+  if (e == cudaSuccess) e = make_map(&mw, p.W, p.N, p.K, 128, f16);
+  if (e != cudaSuccess) return e;
+  const int tiles = ((p.M + P2_BM - 1) / P2_BM) * ((p.N + P2_BN - 1) / P2_BN);
+  const int pairs = tiles < sm_count / 2 ? tiles : sm_count / 2;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = P2_SMEM;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 2;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, largem_gemm_tc_pair_kernel, p, ma, mw);
+}
+}  // namespace
+
+// 4 = the default operand formats with one CTA per tile everywhere (A/B measurements of the CTA-pair kernel)
+void set_prefill_gemm_impl(int impl) {
+  g_pair_tiles = impl != 4;
+  g_prefill_impl = impl == 2 || impl == 3 ? impl : 0;
+}
+bool prefill_single_bf16() { return g_prefill_impl == 2; }
+int prefill_gemm_impl() { return g_prefill_impl; }
+
+cudaError_t launch_largem_gemm(const LargeMParams& p, cudaStream_t stream) {
+  if (!g_sm_count) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      g_sm_count = 148;
+  }
+  return launch_largem_gemm_tc(p, stream, g_sm_count);
+}
+
 cudaError_t launch_largem_gemm_tc(const LargeMParams& p, cudaStream_t stream, int sm_count) {
   if (!g_encode) return cudaErrorNotReady;
   if ((reinterpret_cast<uintptr_t>(p.A) | reinterpret_cast<uintptr_t>(p.W) | reinterpret_cast<uintptr_t>(p.A_lo)) & 15)
     return cudaErrorMisalignedAddress;
+  // single-value operands and at least one 256 x 256 tile per pair of SMs: CTA pairs
+  const int tiles_pair = ((p.M + P2_BM - 1) / P2_BM) * ((p.N + P2_BN - 1) / P2_BN);
+  if (g_pair_tiles && !p.A_lo && tiles_pair >= sm_count / 2) return launch_pair(p, stream, sm_count);
   // 256-wide tiles unless they leave SMs idle; then 128-wide ones (twice as many tiles)
   const int tiles256 = ((p.M + BM - 1) / BM) * ((p.N + 255) / 256);
   return tiles256 < sm_count ? launch_bn<128>(p, stream, sm_count) : launch_bn<256>(p, stream, sm_count);

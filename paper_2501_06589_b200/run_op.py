@@ -29,17 +29,22 @@ def main():
     ap.add_argument("--tokens", type=int, default=4096, help="M of the prefill GEMM")
     ap.add_argument("--multi-kernel", action="store_true", help="stack: use the per-GEMM schedule")
     ap.add_argument("--wide-impl", type=int, default=0,
-                    help="decode GEMM: 0 = default, 1 = mma.sync kernel for batch 9..64, 2 = tcgen05 kernel for every batch")
+                    help="decode GEMM: 0 = default, 2 = tcgen05 kernel for every batch")
     ap.add_argument("--persistent-all", action="store_true", help="stack: standard layers in the persistent kernel too")
     ap.add_argument("--standard", action="store_true", help="stack: standard residuals in every layer")
     ap.add_argument("--which", default="gate_up", choices=["qkv", "wo", "gate_up", "down"],
                     help="prefill_gemm: which projection's shape and epilogue")
     ap.add_argument("--pairs", action="store_true",
                     help="prefill_gemm: bf16 hi + lo activation pairs instead of the default binary16 operands")
+    ap.add_argument("--prefill-impl", type=int, default=0,
+                    help="prefill_gemm: 4 = one CTA per tile everywhere (no CTA pairs)")
+    ap.add_argument("--no-lo", action="store_true", help="prefill_attn: queries and outputs without their lo parts")
+    ap.add_argument("--seq", type=int, default=None, help="prefill_attn: tokens per sequence")
     a = ap.parse_args()
     build.build()
     B.lib()
     B.set_decode_wide_impl(a.wide_impl)
+    B.set_prefill_gemm_impl(a.prefill_impl)
     s = synth.SHAPES[a.config]
     bsz = a.batch or s.batch
     d, F, Hq, Hkv, Dh, V = s.d_model, s.d_ff, s.n_q_heads, s.n_kv_heads, s.head_dim, s.vocab_size
@@ -114,13 +119,15 @@ def main():
             fn = lambda l: B.op_prefill_gemm(A, W[l], mode, out, addend=add if mode == 0 else None, A_lo=A_lo, out_lo=out_lo)
             flops = 2.0 * M * N * K
     elif a.op == "prefill_attn":
-        S = s.prompt_len
+        S = a.seq or s.prompt_len
         q = torch.randn(bsz, S, Hq * Dh, device=dev).to(torch.float16)
         q_lo = (torch.randn(bsz, S, Hq * Dh, device=dev) * 1e-3).to(torch.float16)
         k = [torch.randn(bsz, Hkv, S, Dh, device=dev).to(torch.float16) for _ in range(L)]
         v = [torch.randn(bsz, Hkv, S, Dh, device=dev).to(torch.float16) for _ in range(L)]
         o = torch.empty_like(q)
         o_lo = torch.empty_like(q)
+        if a.no_lo:
+            q_lo = o_lo = None
         fn = lambda l: B.op_prefill_attention(q, k[l], v[l], bsz, S, Hq, Hkv, Dh, S, o, q_lo=q_lo, o_lo=o_lo)
         nbytes, flops = 0, 4.0 * bsz * Hq * Dh * S * (S + 1) / 2
     else:

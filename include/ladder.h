@@ -379,6 +379,13 @@ void ladder_set_prefill_gemm_impl(int32_t impl);
  * tests and A/B measurements, not for serving code. */
 void ladder_set_decode_wide_impl(int32_t impl);
 
+/* Decode attention for batch > 8 (head_dim 128, at most 8 query heads per kv head): 0 = the split step on TMA +
+ * tcgen05 (key / value tiles of 128 cache rows streamed into shared memory, scores and P.V on the tensor core) where
+ * batch x kv heads x ceil(max_seq_len / 128) >= 2048 tiles, the register-fragment kernel that serves batch <= 8
+ * otherwise (default); 1 = the register-fragment kernel always; 2 = the TMA / tcgen05 kernel for every batch > 8.
+ * PROCESS-WIDE and not thread-safe: a switch for tests and A/B measurements. */
+void ladder_set_decode_attention_impl(int32_t impl);
+
 /* Causal grouped-query attention of the prefill path for one layer:
  *   q binary16 [batch, seq_len, Hq*Dh] (rotated), q_lo its optional low part; k,v binary16 cache of one layer
  *   as above, rows 0..seq_len-1 valid; o bf16 [batch, seq_len, Hq*Dh] (the output projection's operand type),

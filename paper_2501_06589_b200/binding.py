@@ -25,7 +25,7 @@ EXPORTS = [
     "ladder_device_status", "ladder_kernel_launches", "ladder_destroy", "ladder_status_string",
     "ladder_last_error", "ladder_op_smallm_gemm", "ladder_decode_attention_scratch_bytes",
     "ladder_op_decode_attention", "ladder_op_prefill_gemm", "ladder_op_prefill_attention", "ladder_op_prefill_attention_at",
-    "ladder_op_decode_attention_noalloc", "ladder_set_prefill_gemm_impl", "ladder_set_decode_wide_impl",
+    "ladder_op_decode_attention_noalloc", "ladder_set_prefill_gemm_impl", "ladder_set_decode_wide_impl", "ladder_set_decode_attention_impl",
     "ladder_op_prefill_gemm_f16", "ladder_op_convert_bf16_f16",
 ]
 
@@ -131,6 +131,8 @@ def lib() -> C.CDLL:
         L.ladder_set_prefill_gemm_impl.argtypes = [C.c_int32]
         L.ladder_set_decode_wide_impl.restype = None
         L.ladder_set_decode_wide_impl.argtypes = [C.c_int32]
+        L.ladder_set_decode_attention_impl.restype = None
+        L.ladder_set_decode_attention_impl.argtypes = [C.c_int32]
         L.ladder_op_prefill_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                              C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ladder_op_prefill_gemm_f16.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
@@ -403,6 +405,12 @@ def set_prefill_gemm_impl(impl: int):
 def set_decode_wide_impl(impl: int):
     """Decode GEMM: 0 = tcgen05 kernel for batch 5..64 (default), 2 = tcgen05 kernel for every batch."""
     lib().ladder_set_decode_wide_impl(impl)
+
+
+def set_decode_attention_impl(impl: int):
+    """Decode attention for batch > 8: 0 = TMA / tcgen05 kernel where there are >= 2048 tiles of 128 keys (default),
+    1 = the register-fragment kernel always, 2 = the TMA / tcgen05 kernel always."""
+    lib().ladder_set_decode_attention_impl(impl)
 
 
 def op_prefill_gemm(A, W, epi_mode: int, out, addend=None, A_lo=None, out_lo=None):

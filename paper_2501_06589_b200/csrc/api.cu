@@ -38,6 +38,7 @@ cudaError_t kernels_ready() {  // opt-in to large dynamic shared memory, once pe
   cudaError_t e = smallm_gemm_init();
   if (e == cudaSuccess) e = largem_gemm_tc_init();
   if (e == cudaSuccess) e = prefill_attention_tc_init();
+  if (e == cudaSuccess) e = decode_attention_tc_init();
   if (e == cudaSuccess) g_kernels_ready = true;
   return e;
 }
@@ -393,6 +394,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
       a.max_len = c.max_seq_len;
       a.scratch = m->attn_scratch;
       a.o = m->o_dec;
+      a.status = m->status;
       const bool handover = batch > 4 && m->wide_opack;  // operands pass from kernel to kernel
       if (handover) {
         a.o_pack = m->wide_opack;
@@ -1033,6 +1035,7 @@ const char* ladder_last_error(const ladder_model_t* m) { return m ? m->err.c_str
 void ladder_set_prefill_gemm_impl(int32_t impl) { set_prefill_gemm_impl(impl); }
 
 void ladder_set_decode_wide_impl(int32_t impl) { set_decode_wide_impl(impl); }
+void ladder_set_decode_attention_impl(int32_t impl) { set_decode_attention_impl(impl); }
 
 size_t ladder_kv_cache_bytes(const ladder_config_t* c) {
   if (!c) return 0;

@@ -338,14 +338,28 @@ size_t decode_attention_scratch_floats(int batch, int n_q_heads, int head_dim, i
   return static_cast<size_t>(batch) * n_q_heads * n_splits * (head_dim + 2);
 }
 
+static int g_attn_impl = 0;
+void set_decode_attention_impl(int impl) { g_attn_impl = impl == 1 || impl == 2 ? impl : 0; }
+
 cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stream, bool pdl) {
   if (p.n_splits * kChunk < p.max_len || p.n_splits > kMaxSplits) return cudaErrorInvalidValue;
   cudaError_t e;
-  switch (heads_per_cta(p.n_q_heads, p.n_kv_heads)) {
-    case 8: e = launch_gt<8>(p, stream, pdl); break;
-    case 4: e = launch_gt<4>(p, stream, pdl); break;
-    case 2: e = launch_gt<2>(p, stream, pdl); break;
-    default: e = launch_gt<1>(p, stream, pdl); break;
+  int n_partials = p.n_splits;  // partials per (sequence, head) the merge reads
+  // Throughput regime: the TMA-fed tcgen05 kernel, one partial per 128 keys (the scratch is sized for one per 64).
+  // Only where there is enough to stream: it cannot share an SM with the GEMM before or after it (217 KB of shared
+  // memory), so below ~2000 tiles its start-up costs more than its bandwidth gains (measured inside decode steps:
+  // TP-rank slice batch 64, 1088 tiles, +4 %; 70B shape batch 32 / 64, 3072 / 6144 tiles, -0.7 % / -1.7 %).
+  const long tiles128 = static_cast<long>(p.batch) * p.n_kv_heads * ((p.max_len + 127) / 128);
+  if (p.batch > 8 && (g_attn_impl == 2 || (g_attn_impl == 0 && tiles128 >= 2048)) && decode_attention_tc_usable(p)) {
+    n_partials = p.max_len > 128 ? (p.max_len + 127) / 128 : 1;
+    e = launch_decode_attention_tc(p, n_partials, p.status, stream, pdl);
+  } else {
+    switch (heads_per_cta(p.n_q_heads, p.n_kv_heads)) {
+      case 8: e = launch_gt<8>(p, stream, pdl); break;
+      case 4: e = launch_gt<4>(p, stream, pdl); break;
+      case 2: e = launch_gt<2>(p, stream, pdl); break;
+      default: e = launch_gt<1>(p, stream, pdl); break;
+    }
   }
   if (e != cudaSuccess) return e;
   cudaLaunchAttribute at[1];
@@ -355,8 +369,8 @@ cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stre
   const int bp = p.o_pack_bp;
   if (o_pack && bp < p.batch) return cudaErrorInvalidValue;
   if (p.head_dim == 128)
-    return cudaLaunchKernelEx(&cfg, decode_attention_merge_kernel<128>, scratch, p.n_q_heads, p.n_splits, p.o, o_pack, bp);
-  return cudaLaunchKernelEx(&cfg, decode_attention_merge_kernel<64>, scratch, p.n_q_heads, p.n_splits, p.o, o_pack, bp);
+    return cudaLaunchKernelEx(&cfg, decode_attention_merge_kernel<128>, scratch, p.n_q_heads, n_partials, p.o, o_pack, bp);
+  return cudaLaunchKernelEx(&cfg, decode_attention_merge_kernel<64>, scratch, p.n_q_heads, n_partials, p.o, o_pack, bp);
 }
 
 }  // namespace ladder

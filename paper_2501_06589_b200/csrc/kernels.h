@@ -81,6 +81,7 @@ struct DecodeAttnParams {
   float* o;                     // [batch, Hq*Dh]
   __nv_bfloat16* o_pack;        // optional: o also as a staged GEMM operand, bf16 [2 o_pack_bp, Hq*Dh] (hi rows, lo rows)
   int o_pack_bp;                // padded batch of that operand (16 / 32 / 64); rows batch..bp-1 are written as zero
+  int32_t* status;              // optional device status word (the TMA / tcgen05 kernel of batch > 8 reports timeouts)
 };
 int wide_padded_batch(int batch);  // Bp of the batch 9..64 GEMM kernel
 int decode_attention_splits(int batch, int n_kv_heads, int max_len, int sm_count);
@@ -96,6 +97,13 @@ inline bool decode_attention_misaligned(const void* q, const void* k, const void
 }
 size_t decode_attention_scratch_floats(int batch, int n_q_heads, int head_dim, int n_splits);
 cudaError_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t stream, bool pdl);
+// Batch > 8 at head_dim 128: the split step on TMA + tcgen05 (decode_attention_tc.cu), one partial per 128 keys.
+cudaError_t decode_attention_tc_init();
+bool decode_attention_tc_usable(const DecodeAttnParams& p);
+cudaError_t launch_decode_attention_tc(const DecodeAttnParams& p, int n_tiles, int32_t* status, cudaStream_t stream,
+                                       bool pdl);
+void set_decode_attention_impl(int impl);  // 0 = default (TMA / tcgen05 kernel for batch > 8 and >= 2048 tiles), 1 = register-fragment
+                                           // kernel always, 2 = TMA / tcgen05 kernel wherever its shapes allow (batch > 8)
 
 // Persistent layer-stack kernel of the decode step: every weight-streaming GEMM of the step is a
 // "phase" of ONE cooperative launch, attention runs on dedicated warps of the same CTAs, and the

@@ -27,12 +27,12 @@
 
 #include "common.cuh"
 #include "kernels.h"
+#include "tcgen05_attn.cuh"
 
 namespace ladder {
 namespace {
 
 constexpr int kQT = 128, kKT = 128, kAtThreads = 320;
-constexpr int BLK_BYTES = 128 * 128;  // 128 rows of 64 binary16 values (one 128-byte swizzled row each)
 
 template <int DH, bool SPLIT>
 struct AtCfg {
@@ -53,105 +53,6 @@ struct AtCfg {
                                        (static_cast<uint32_t>(kQT >> 4) << 24);
   static constexpr int TMEM_COLS = 512;  // S0, S1 at 0 / 128 (P_j overwrites the first 64 columns of S_j); PV0, PV1 at 256 / 384
 };
-
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ void at_tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-      "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
-      : "memory");
-}
-__device__ __forceinline__ void at_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void at_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void at_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-__device__ __forceinline__ void at_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-// D(tmem) (+)= A(tmem) * B(smem desc): A = 128 lanes (rows) x 8 columns, each column two consecutive binary16 K values
-__device__ __forceinline__ void at_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-// 32 consecutive 32-bit columns of this thread's TMEM lane, from registers; the caller waits with at_wait_st()
-__device__ __forceinline__ void at_st32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, "
-      "%25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
-      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
-      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void at_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-// 32 consecutive fp32 columns of this thread's TMEM lane; the caller waits with at_wait_ld()
-__device__ __forceinline__ void at_ld32(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, "
-      "%24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-// Bounded wait that lets the hardware suspend the thread while the phase is incomplete: a warp that waits takes no
-// issue slots from the softmax warp of its sub-partition.  Gives up after ~0.25 s.
-__device__ __forceinline__ bool at_wait(uint64_t* bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
-  for (uint32_t i = 1;; ++i) {
-    if (mbar_try_wait_suspend(bar, parity, 2000u)) return true;
-    if ((i & 15u) == 0 && global_timer_ns() - t0 > 250000000ull) return false;
-  }
-}
-// The same wait for a whole warp.  Lanes leave the polling loop at different times; the vote brings them back
-// together (and makes the outcome uniform), so the code after the wait runs converged.
-__device__ __forceinline__ bool at_wait_warp(uint64_t* bar, uint32_t parity) {
-  return __all_sync(0xffffffffu, at_wait(bar, parity));
-}
-__device__ __forceinline__ void at_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-// K-major operand tile (rows x 64 binary16, 128-byte swizzle, 8-row atoms of 1024 bytes): Q, K and P.
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>(1) << 16;            // leading byte offset: unused for swizzled K-major
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;    // stride byte offset: the next 8 rows
-  d |= static_cast<uint64_t>(1) << 46;            // descriptor version (sm_100)
-  d |= static_cast<uint64_t>(2) << 61;            // 128-byte swizzle
-  return d;
-}
-// MN-major operand (the value tile as it lies in the cache: a row per key, head_dim contiguous): atoms of 64
-// head_dim values x 8 keys (1024 bytes, 128-byte swizzle); the next 8 keys follow 1024 bytes on (stride offset),
-// the next 64 head_dim values sit in the second 16 KB block (leading offset).
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>(BLK_BYTES >> 4) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
 
 struct AtParams {
   int seq_len, n_q_heads, n_kv_heads, max_seq_len, pos0, out_f16, n_qt, batch, n_items;

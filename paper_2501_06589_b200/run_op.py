@@ -38,6 +38,8 @@ def main():
                     help="prefill_gemm: bf16 hi + lo activation pairs instead of the default binary16 operands")
     ap.add_argument("--prefill-impl", type=int, default=0,
                     help="prefill_gemm: 4 = one CTA per tile everywhere (no CTA pairs)")
+    ap.add_argument("--attn-impl", type=int, default=0,
+                    help="attn, stack: 1 = the register-fragment decode attention kernel at every batch, 2 = the TMA / tcgen05 kernel for every batch > 8")
     ap.add_argument("--no-lo", action="store_true", help="prefill_attn: queries and outputs without their lo parts")
     ap.add_argument("--seq", type=int, default=None, help="prefill_attn: tokens per sequence")
     a = ap.parse_args()
@@ -45,6 +47,7 @@ def main():
     B.lib()
     B.set_decode_wide_impl(a.wide_impl)
     B.set_prefill_gemm_impl(a.prefill_impl)
+    B.set_decode_attention_impl(a.attn_impl)
     s = synth.SHAPES[a.config]
     bsz = a.batch or s.batch
     d, F, Hq, Hkv, Dh, V = s.d_model, s.d_ff, s.n_q_heads, s.n_kv_heads, s.head_dim, s.vocab_size

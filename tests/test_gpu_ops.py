@@ -182,6 +182,51 @@ def test_decode_attention(B, batch, Hq, Hkv, Dh, max_seq, lens):
         assert rel_err(got[b], ref) < 1e-3, b
 
 
+@pytest.mark.parametrize("impl", [2, 1])          # 2 = TMA / tcgen05 kernel, 1 = register-fragment kernel
+@pytest.mark.parametrize("batch,Hq,Hkv,Dh,max_seq,lens", [
+    (16, 8, 1, 128, 2200, [2048, 2047, 1025, 7, 129, 128, 127, 1, 2200, 640, 0, 300, 1999, 64, 65, 256]),  # TP-rank slice
+    (9, 32, 8, 128, 700, [700, 1, 129, 500, 0, 384, 385, 699, 256]),              # groups of 4 heads (8B shape)
+    (10, 16, 16, 128, 300, [300, 299, 128, 1, 0, 257, 17, 200, 64, 130]),         # one query head per kv head
+    (12, 32, 2, 128, 260, [260, 259, 131, 5, 128, 256, 1, 77, 190, 33, 12, 250]), # groups of 16 heads
+    (64, 8, 1, 128, 1100, None),                                                  # more work items than SMs (a ring per CTA)
+    (33, 64, 8, 128, 400, None),
+    (64, 64, 8, 128, 1300, [1300 - (i % 3) for i in range(64)]),   # 70B shape: 35 tiles and four (sequence, kv head) groups per CTA
+])
+def test_decode_attention_wide_batches(B, batch, Hq, Hkv, Dh, max_seq, lens, impl):
+    """Batch > 8 against the oracle, sequence by sequence: lengths that end inside, at the edge of and one past a
+    128-key tile, empty sequences, cache rows beyond a sequence's length holding NaN (they must leave no trace)."""
+    if lens is None:
+        lens = [int(x) for x in np.random.default_rng(batch).integers(1, max_seq + 1, batch)]
+        lens[0], lens[-1] = max_seq, 1
+    q = torch.randn(batch, Hq * Dh, generator=torch.Generator().manual_seed(31)).cuda()
+    k = _f16((batch, Hkv, max_seq, Dh), 32, 1.0)
+    v = _f16((batch, Hkv, max_seq, Dh), 33, 1.0)
+    for b in range(batch):
+        k[b, :, lens[b]:] = float("nan")
+        v[b, :, lens[b]:] = float("nan")
+    kv_len = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    scratch = torch.full((B.decode_attention_scratch_bytes(batch, Hq, Dh, max_seq) // 4,), float("nan"), device="cuda")
+    o = torch.full((batch, Hq * Dh), float("nan"), device="cuda")
+    B.set_decode_attention_impl(impl)
+    try:
+        B.op_decode_attention(q, k, v, kv_len, Hq, Hkv, Dh, max_seq, scratch, o)
+        first = o.clone()
+        B.op_decode_attention(q, k, v, kv_len, Hq, Hkv, Dh, max_seq, scratch, o)
+        torch.cuda.synchronize()
+    finally:
+        B.set_decode_attention_impl(0)
+    assert torch.equal(first, o)                     # partials are merged in a fixed order
+    got = _f64(o).reshape(batch, Hq, Dh)
+    qb = _f64(q).reshape(batch, 1, Hq, Dh)
+    for b in range(batch):
+        L = lens[b]
+        if L == 0:
+            assert np.all(got[b] == 0.0)
+            continue
+        ref = O.causal_attention(qb[b], _f64(k[b, :, :L]).transpose(1, 0, 2), _f64(v[b, :, :L]).transpose(1, 0, 2), L - 1)[0]
+        assert rel_err(got[b], ref) < 1e-3, b
+
+
 def _split(shape, seed, std=1.0, dtype=torch.bfloat16):
     """fp32 values and their 16-bit hi / lo parts (value ~ hi + lo)."""
     f = torch.randn(shape, generator=torch.Generator().manual_seed(seed)) * std

@@ -406,6 +406,11 @@ def other_configs(B, torch, synth, args, local, w70=None, shape70=None):
     if w70 is not None:      # the same 70B weights under the two other residual rules
         for mode in ("standard", "parallel"):
             out[f"70b_b{shape70.batch}_{mode}"] = short_run(B, torch, synth, shape70.as_mode(mode), w70, args, local)
+        # the batch sweep of the paper's Sec. 3.3.1 at the full shape (decode steps from a 1024-token cache of seeded
+        # noise: the prompt-pass workspace for 64 x 1024 tokens would not fit beside 141 GB of weights)
+        for b in (1, 16, 32, 64):
+            out[f"70b_b{b}_ladder"] = short_run(B, torch, synth, synth.replace(shape70, batch=b), w70, args, local,
+                                                noise_kv=True)
     return out
 
 

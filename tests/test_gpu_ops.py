@@ -390,3 +390,72 @@ def test_prefill_attention_offset_and_lengths(B, batch, S, Hq, Hkv, Dh, max_seq,
                                  _f64(v[b, :, :pos0 + n]).transpose(1, 0, 2), pos0)
         assert rel_err(got[b, :n].reshape(n, Hq, Dh), ref) < 2e-3, b      # binary16 output: 2^-12 per element
         assert np.all(got[b, n:] == canary), b                              # padding rows untouched
+
+
+def _repeat_bitwise(torch_mod, launch, out, reps):
+    """Launches `launch` `reps` times, every other time beside a copy kernel on a second stream, and counts the runs
+    whose output differs from the first run's: the role pipelines of the tcgen05 kernels hand tiles over through
+    mbarriers, and a protocol slip (a barrier phase arrived on twice, a ring slot rewritten early) shows up as a rare
+    wrong tile rather than as a wrong formula."""
+    side = torch_mod.cuda.Stream()
+    big = torch_mod.randn(16 << 20, device="cuda")
+    big2 = torch_mod.empty_like(big)
+    launch()
+    torch_mod.cuda.synchronize()
+    ref = out.clone()
+    assert not bool(torch_mod.isnan(ref.float()).any())
+    bad = 0
+    for rep in range(reps):
+        out.fill_(float("nan"))
+        if rep & 1:
+            with torch_mod.cuda.stream(side):
+                big2.copy_(big)
+        launch()
+        bad += 0 if torch_mod.equal(out, ref) else 1
+    torch_mod.cuda.synchronize()
+    return bad
+
+
+def test_prefill_attention_many_launches_bitwise(B):
+    """70B-shaped prompt-pass attention (2048 work items, 14 per CTA), 400 launches: all bit-identical."""
+    bsz, S, Hq, Hkv, Dh, ms = 4, 1024, 64, 8, 128, 1100
+    _, q, q_lo = _split((bsz, S, Hq * Dh), 41, dtype=torch.float16)
+    k = _f16((bsz, Hkv, ms, Dh), 42, 1.0)
+    v = _f16((bsz, Hkv, ms, Dh), 43, 1.0)
+    k[:, :, S:] = float("nan")
+    v[:, :, S:] = float("nan")
+    o = torch.empty(bsz, S, Hq * Dh, dtype=torch.float16, device="cuda")
+    launch = lambda: B.op_prefill_attention(q, k, v, bsz, S, Hq, Hkv, Dh, ms, o, q_lo=q_lo, out_binary16=True)
+    assert _repeat_bitwise(torch, launch, o, 400) == 0
+
+
+def test_decode_attention_tc_many_launches_bitwise(B):
+    """Wide-batch decode attention on the TMA / tcgen05 kernel (35 tiles and four groups per CTA), 600 launches."""
+    bsz, Hq, Hkv, Dh, ms = 64, 64, 8, 128, 1536
+    q = torch.randn(bsz, Hq * Dh, generator=torch.Generator().manual_seed(51)).cuda()
+    k = _f16((bsz, Hkv, ms, Dh), 52, 1.0)
+    v = _f16((bsz, Hkv, ms, Dh), 53, 1.0)
+    lens = [1280 - 7 * (i % 5) for i in range(bsz)]
+    for b in range(bsz):
+        k[b, :, lens[b]:] = float("nan")
+        v[b, :, lens[b]:] = float("nan")
+    kv_len = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    scratch = torch.empty(B.decode_attention_scratch_bytes(bsz, Hq, Dh, ms) // 4, device="cuda")
+    o = torch.empty(bsz, Hq * Dh, device="cuda")
+    B.set_decode_attention_impl(2)
+    try:
+        launch = lambda: B.op_decode_attention(q, k, v, kv_len, Hq, Hkv, Dh, ms, scratch, o)
+        assert _repeat_bitwise(torch, launch, o, 600) == 0
+    finally:
+        B.set_decode_attention_impl(0)
+
+
+def test_prefill_gemm_pairs_many_launches_bitwise(B):
+    """The CTA-pair prompt-pass GEMM (cluster of two, 160 tiles over 74 pairs), 300 launches."""
+    M, N, K = 2560, 4096, 1024
+    A = _f16((M, K), 61, 1.0)
+    W = _f16((N, K), 62, 0.05)
+    addend = torch.randn(M, N, generator=torch.Generator().manual_seed(63)).cuda()
+    out = torch.empty(M, N, device="cuda")
+    launch = lambda: B.op_prefill_gemm_f16(A, W, 0, out, addend=addend)
+    assert _repeat_bitwise(torch, launch, out, 300) == 0

@@ -318,8 +318,14 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   // SMs (25.1 ms at the best split of 40 SMs vs 24.4 ms): a subset of SMs streams at ~47 GB/s each and
   // the module chain (Wo waits for the previous down projection and vice versa) leaves it idle in
   // between.  Off by default.
-  if (q.two && m->sms_a >= 0 && batch <= 4) {
-    int ga = m->sms_a;
+  // Batch 5..64 (one tcgen05 kernel per GEMM) with small layers is the exception: there a launch costs more than it
+  // streams (7 us of set-up and 4-11 us of shared-tile fix-up against 3-17 us of weights at the TP-rank slice), and
+  // two launches side by side overlap those costs: 60 of 148 SMs for the attention stream measured 581 -> 553 us per
+  // 8 layers at batch 16 and 921 -> 865 us at batch 64 (at the 70B shape the split loses at every batch).
+  const double layer_bytes = 2.0 * (static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh + 3.0 * F * d);
+  const bool auto_wide = m->sms_a == -1 && batch > 4 && layer_bytes < 300e6;
+  if (q.two && (m->sms_a >= 0 || auto_wide)) {
+    int ga = auto_wide ? (60 * m->sm_count + 74) / 148 : m->sms_a;
     if (ga == 0) {
       const double ba = static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh;
       const double bb = 3.0 * F * d;

@@ -40,6 +40,8 @@ def main():
                     help="prefill_gemm: 4 = one CTA per tile everywhere (no CTA pairs)")
     ap.add_argument("--attn-impl", type=int, default=0,
                     help="attn, stack: 1 = the register-fragment decode attention kernel at every batch, 2 = the TMA / tcgen05 kernel for every batch > 8")
+    ap.add_argument("--sm-split", type=int, default=-1,
+                    help="stack (one kernel per GEMM): SMs for the attention module's GEMMs, the rest for the MLP's (0 = by bytes)")
     ap.add_argument("--no-lo", action="store_true", help="prefill_attn: queries and outputs without their lo parts")
     ap.add_argument("--seq", type=int, default=None, help="prefill_attn: tokens per sequence")
     a = ap.parse_args()
@@ -166,6 +168,8 @@ def run_stack(a, s, bsz):
         model.set_persistent(False)
     if a.persistent_all:
         model.set_persistent(2)
+    if a.sm_split >= 0:
+        model.set_sm_split(a.sm_split)
     persistent = model.persistent_active() and bsz <= 8
     cache = B.KVCache(s, bsz, S + steps + 1)
     cache.k.normal_()                                 # a synthetic prefix instead of a prompt pass

@@ -219,6 +219,9 @@ def parse_args(argv=None):
                     help="every layer in this architecture (paper Sec. 3.3.1) instead of the configuration's own")
     ap.add_argument("--multi-kernel", action="store_true",
                     help="one kernel per GEMM (two streams, CUDA graph, PDL) instead of the persistent decode kernel")
+    ap.add_argument("--sm-split", type=int, default=None,
+                    help="one kernel per GEMM: SMs for the attention module's GEMMs, the rest for the MLP's "
+                         "(-2 = every GEMM on all SMs, -1 = the library's choice, 0 = by bytes)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill-timing", action="store_true")
     ap.add_argument("--no-other-configs", action="store_true",
@@ -303,6 +306,8 @@ class DecodeRun:
         self.model = B.Model(w, bsz, max_seq, bsz * chunk)
         if args.multi_kernel:
             self.model.set_persistent(False)
+        if getattr(args, "sm_split", None) is not None:
+            self.model.set_sm_split(args.sm_split)
         self.persistent = self.model.persistent_active() and bsz <= 8
         if args.streams is not None or args.graph is not None or args.pdl is not None:
             self.model.set_schedule(2 if args.streams is None else args.streams, 1 if args.graph is None else args.graph,

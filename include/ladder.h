@@ -184,8 +184,8 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
  * disjoint sets of SMs (each GEMM is a persistent kernel that claims its work dynamically, so it runs
  * on any number of CTAs).  sms_attention_stream: -1 = the library's choice (default): no split, every GEMM on all
  * SMs, which measured fastest everywhere except for batch 5..64 with layers below 300 MB, where 60 of 148 SMs go
- * to the attention stream; 0 = in proportion to the bytes each module streams; n > 0 = that many SMs for the
- * attention module's GEMMs and the rest for the MLP's.  Results are bit-identical. */
+ * to the attention stream; -2 = never split; 0 = in proportion to the bytes each module streams; n > 0 = that many
+ * SMs (at most half of them) for the attention module's GEMMs and the rest for the MLP's.  Results are bit-identical. */
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream);
 
 /* Prompt pass ("prefill phase", paper Sec. 3.2): the module chain of Eq. 1 / Eq. 2 (in the pending-output form of

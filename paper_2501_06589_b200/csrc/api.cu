@@ -357,7 +357,8 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
 
   if (l_end < 0) l_end = c.n_layers;
   for (int l = 0; l < l_end; ++l) {
-    const bool lad = m->is_ladder[l] != 0;
+    const bool lad = m->stale[2 * l + 1] != 0;  // the MLP module does not read the attention module's output (ladder and
+                                                // parallel layers): the two modules' GEMMs may run side by side
     // ---------------- attention module (module index 2l+1) on stream A
     {
       const int mod = 2 * l + 1;
@@ -1286,8 +1287,8 @@ int32_t ladder_model_persistent_active(const ladder_model_t* m) { return (m && m
 
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream) {
   if (!m) return LADDER_ERR_INVALID_ARG;
-  if (sms_attention_stream < -1 || sms_attention_stream > m->sm_count / 2)
-    return fail(m, LADDER_ERR_INVALID_ARG, "sms_attention_stream must be -1, 0 or at most half the SMs");
+  if (sms_attention_stream < -2 || sms_attention_stream > m->sm_count / 2)
+    return fail(m, LADDER_ERR_INVALID_ARG, "sms_attention_stream must be -2, -1, 0 or at most half the SMs");
   m->sms_a = sms_attention_stream;
   drop_graph(m);
   return LADDER_OK;

@@ -185,7 +185,12 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
  * on any number of CTAs).  sms_attention_stream: -1 = the library's choice (default): no split, every GEMM on all
  * SMs, which measured fastest everywhere except for batch 5..64 with layers below 300 MB, where 60 of 148 SMs go
  * to the attention stream; -2 = never split; 0 = in proportion to the bytes each module streams; n > 0 = that many
- * SMs (at most half of them) for the attention module's GEMMs and the rest for the MLP's.  Results are bit-identical. */
+ * SMs (at most half of them) for the attention module's GEMMs and the rest for the MLP's.  Results are bit-identical.
+ * Whenever the split is on, batch is 5..64 and every module reads x_{m-2} (all layers ladder), the step also runs
+ * in the pending-output form of Algorithm 1: a module's output stays in a buffer of its own and is added to the
+ * residual when the next module's input is normalised, so the attention chain and the MLP chain wait for each
+ * other's normalised-input kernel only, never for a GEMM.  The additions are the same fp32 additions in the same
+ * order.  -3 = the library's choice of split without that form (each output added by its GEMM's epilogue). */
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream);
 
 /* Prompt pass ("prefill phase", paper Sec. 3.2): the module chain of Eq. 1 / Eq. 2 (in the pending-output form of

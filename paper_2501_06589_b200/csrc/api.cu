@@ -74,6 +74,9 @@ struct ladder_model {
   // batch 9..64: the SwiGLU output / the attention output as the next GEMM's staged operand (bf16 [2 x 64, F] / [2 x 64, Hq*Dh])
   __nv_bfloat16* wide_hpack = nullptr;
   __nv_bfloat16* wide_opack = nullptr;
+  float* pend_a = nullptr;  // batch 5..64, pending-output schedule: the attention module's output, stored not added
+  float* pend_m = nullptr;  // ... and the MLP module's
+  std::vector<cudaEvent_t> ev_sq, ev_sg;  // [layer]: x_{2l-1} / x_{2l} formed by the staging step of layer l's QKV / gate-up input
   // the same activations as bf16 hi/lo MMA operands ([chunk][8][2048]), written by the persistent kernel's
   // epilogues for the phase that reads them next (batch <= 4): twins of R[0], R[1], h_dec, o_dec
   __nv_bfloat16 *xpack[2] = {nullptr, nullptr}, *hpack = nullptr, *opack = nullptr;
@@ -302,6 +305,164 @@ struct Enqueue {
   }
 };
 
+// Batch 5..64, every layer a ladder layer: the decode step in the pending-output form of Algorithm 1.  The output
+// and down projections STORE their module's output (pend_a / pend_m) instead of adding it to the stream, and the
+// stream moves on in the staging step of the next reader: x_{2l-1} = x_{2l-2} + attn_{l-1} where the QKV projection of
+// layer l stages its input, x_{2l} = x_{2l-1} + mlp_{l-1} where the gate/up projection does.  With the adds fused into
+// the epilogues every output projection has to wait for the previous down projection and vice versa, so the two
+// streams move in lock-step; here the only cross-stream edges are between the (tiny) staging launches, and the
+// attention-module chain (stage, QKV, attention, Wo) and the MLP chain (stage, gate/up, down) of a layer run side by
+// side on their shares of the SMs.  The sums are the same fp32 additions in the same order: bit-identical results.
+// R[0] holds the even stream values (x_0 from the embedding, then x_{2l}), R[1] the odd ones.
+cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int batch,
+                                   const ladder_outputs_t* out, cudaStream_t sA, cudaStream_t sB, int64_t* n_kernels,
+                                   int grid_a, int grid_b) {
+  const ladder_config_t& c = m->cfg;
+  Enqueue q{m, sA, sB, true};
+  q.grid_a = grid_a;
+  q.grid_b = grid_b;
+  const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff, L = c.n_layers;
+  const size_t layer_elems = static_cast<size_t>(c.max_batch) * Hkv * c.max_seq_len * Dh;
+  float* const x_even = m->R[0];
+  float* const x_odd = m->R[1];
+  Router rt;
+  q.launched(0, begin_stream(m, rt, d_tokens, batch, sA));
+  auto stage = [&](int s, SmallMParams& p) {  // the staging launch of a GEMM on its own (an event follows it)
+    p.scratch = m->gemm_scratch[s];
+    p.status = m->status;
+    q.launched(s, launch_smallm_gemm_stage(p, q.stream(s), q.pdl(s)));
+  };
+  for (int l = 0; l < L; ++l) {
+    // ---------------- attention module on stream A
+    if (l > 0) q.wait(0, m->ev_sg[l - 1]);  // x_{2l-2}
+    SmallMParams p = {};
+    p.W = m->w_qkv[l];
+    p.N = (Hq + 2 * Hkv) * Dh;
+    p.K = d;
+    p.act = x_even;
+    p.act_pending = l > 0 ? m->pend_a : nullptr;  // attn_{l-1}; the first modules both read x_0
+    p.act_sum_out = x_odd;
+    p.act_mode = ACT_F32_NORM;
+    p.gain = m->attn_norm[l];
+    p.eps = c.rms_eps;
+    p.batch = batch;
+    stage(0, p);
+    q.record(0, m->ev_sq[l]);
+    p.wide_prestaged = 1;
+    p.epi_mode = EPI_QKV_ROPE;
+    p.qkv.q_out_f32 = m->q_f32;
+    p.qkv.k_cache = static_cast<kv_t*>(cache->k) + l * layer_elems;
+    p.qkv.v_cache = static_cast<kv_t*>(cache->v) + l * layer_elems;
+    p.qkv.seq_lens = cache->seq_lens;
+    p.qkv.rope = m->rope;
+    p.qkv.n_q_heads = Hq;
+    p.qkv.n_kv_heads = Hkv;
+    p.qkv.head_dim = Dh;
+    p.qkv.max_seq_len = c.max_seq_len;
+    q.gemm(0, p, true);
+
+    DecodeAttnParams a = {};
+    a.q = m->q_f32;
+    a.k = p.qkv.k_cache;
+    a.v = p.qkv.v_cache;
+    a.kv_len = cache->seq_lens;
+    a.kv_len_offset = 1;
+    a.batch = batch;
+    a.n_q_heads = Hq;
+    a.n_kv_heads = Hkv;
+    a.head_dim = Dh;
+    a.max_seq_len = c.max_seq_len;
+    a.n_splits = m->attn_splits;
+    a.max_len = c.max_seq_len;
+    a.scratch = m->attn_scratch;
+    a.o = m->o_dec;
+    a.status = m->status;
+    a.o_pack = m->wide_opack;
+    a.o_pack_bp = wide_padded_batch(batch);
+    q.launched(0, launch_decode_attention(a, sA, q.pdl(0)));
+    ++q.kernels;  // the split kernel and its merge kernel
+
+    SmallMParams o = {};
+    o.W = m->w_o[l];
+    o.N = d;
+    o.K = Hq * Dh;
+    o.act = m->o_dec;
+    o.act_mode = ACT_F32;
+    o.batch = batch;
+    o.epi_mode = EPI_PLAIN;
+    o.out = m->pend_a;  // read by the staging step of layer l + 1 (or of the head) on this stream
+    o.act_staged = m->wide_opack;
+    q.gemm(0, o, true);
+
+    // ---------------- MLP module on stream B
+    q.wait(1, m->ev_sq[l]);  // x_{2l-1}
+    SmallMParams g = {};
+    g.W = m->w_gate_up[l];
+    g.N = 2 * F;
+    g.K = d;
+    g.act = x_odd;
+    g.act_pending = l > 0 ? m->pend_m : nullptr;  // mlp_{l-1}
+    g.act_sum_out = x_even;
+    g.act_mode = ACT_F32_NORM;
+    g.gain = mlp_gain(m, l);
+    g.eps = c.rms_eps;
+    g.batch = batch;
+    stage(1, g);
+    q.record(1, m->ev_sg[l]);
+    g.wide_prestaged = 1;
+    g.epi_mode = EPI_SWIGLU;
+    g.out = m->h_dec;
+    g.wide_pack_out = m->wide_hpack;
+    q.gemm(1, g, true);
+
+    SmallMParams dn = {};
+    dn.W = m->w_down[l];
+    dn.N = d;
+    dn.K = F;
+    dn.act = m->h_dec;
+    dn.act_mode = ACT_F32;
+    dn.batch = batch;
+    dn.epi_mode = EPI_PLAIN;
+    dn.out = m->pend_m;
+    dn.act_staged = m->wide_hpack;
+    q.gemm(1, dn, true);
+  }
+  // ---------------- head on stream A: x_{2L-1} = x_{2L-2} + attn_{L-1}, then x_{2L} = x_{2L-1} + mlp_{L-1} in the head's
+  // own staging step
+  q.record(1, m->ev_sq[L]);  // the last down projection
+  q.wait(0, m->ev_sg[L - 1]);
+  SmallMParams t = {};
+  t.K = d;
+  t.act = x_even;
+  t.act_pending = m->pend_a;
+  t.act_sum_out = x_odd;
+  t.act_mode = ACT_F32;
+  t.batch = batch;
+  stage(0, t);
+  q.wait(0, m->ev_sq[L]);
+  float* logits = (out && out->logits) ? out->logits : m->logits_ws;
+  SmallMParams h = {};
+  h.W = m->lm_head;
+  h.N = c.vocab_size;
+  h.K = d;
+  h.act = x_odd;
+  h.act_pending = m->pend_m;
+  h.act_sum_out = x_even;
+  h.act_mode = ACT_F32_NORM;
+  h.gain = m->final_norm;
+  h.eps = c.rms_eps;
+  h.batch = batch;
+  h.epi_mode = EPI_PLAIN;
+  h.out = logits;
+  q.gemm(0, h);
+  if (out && out->final_hidden)
+    q.launched(0, launch_rmsnorm_f32(x_even, m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, sA, q.pdl(0)));
+  q.launched(0, launch_argmax_advance(logits, batch, c.vocab_size, out ? out->next_tokens : nullptr, cache->seq_lens, 1,
+                                      -1, sA, q.pdl(0)));
+  *n_kernels = q.kernels;
+  return q.err;
+}
+
 // One decode step: enqueue every kernel on sA (attention modules, head) and sB (MLP modules).
 // l_end < n_layers: only the embedding and layers [0, l_end) (the rest of the step is run by the persistent kernel).
 cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int batch,
@@ -323,7 +484,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   // two launches side by side overlap those costs: 60 of 148 SMs for the attention stream measured 581 -> 553 us per
   // 8 layers at batch 16 and 921 -> 865 us at batch 64 (at the 70B shape the split loses at every batch).
   const double layer_bytes = 2.0 * (static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh + 3.0 * F * d);
-  const bool auto_wide = m->sms_a == -1 && batch > 4 && layer_bytes < 300e6;
+  const bool auto_wide = (m->sms_a == -1 || m->sms_a == -3) && batch > 4 && layer_bytes < 300e6;
   if (q.two && (m->sms_a >= 0 || auto_wide)) {
     int ga = auto_wide ? (60 * m->sm_count + 74) / 148 : m->sms_a;
     if (ga == 0) {
@@ -335,6 +496,11 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
     if (ga > m->sm_count / 2) ga = m->sm_count / 2;
     q.grid_a = ga;
     q.grid_b = m->sm_count - ga;
+    // every module reads x_{m-2} (all layers ladder), batch 5..64, the whole step here: the pending-output schedule
+    bool all_stale = batch > 4 && m->sms_a != -3 && m->pend_a && m->pend_m && !m->st_in.newest && !m->st_out.newest &&
+                     (l_end < 0 || l_end == c.n_layers);
+    for (size_t i = 0; i < m->stale.size() && all_stale; ++i) all_stale = m->stale[i] != 0;
+    if (all_stale) return enqueue_decode_pending(m, cache, d_tokens, batch, out, sA, sB, n_kernels, q.grid_a, q.grid_b);
   }
 
   Router rt;
@@ -1128,6 +1294,8 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   if (c.max_batch > 4) {
     A(dev_alloc(&m->wide_hpack, 2 * 64 * F));
     A(dev_alloc(&m->wide_opack, 2 * 64 * qd));
+    A(dev_alloc(&m->pend_a, MB * d));
+    A(dev_alloc(&m->pend_m, MB * d));
   }
   const auto pack_elems = [](size_t K) { return ((K + 2047) / 2048) * 8 * 2048; };
   A(dev_alloc(&m->xpack[0], pack_elems(d)));
@@ -1213,6 +1381,11 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   m->ev.resize(2 * L + 1, nullptr);
   for (auto& ev : m->ev)
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+  m->ev_sq.resize(L + 1, nullptr);
+  m->ev_sg.resize(L + 1, nullptr);
+  for (auto* vec : {&m->ev_sq, &m->ev_sg})
+    for (auto& ev : *vec)
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_pf_fork, cudaEventDisableTiming);
@@ -1235,6 +1408,9 @@ ladder_status_t ladder_destroy(ladder_model_t* m) {
   drop_graph(m);
   for (auto ev : m->ev)
     if (ev) cudaEventDestroy(ev);
+  for (auto* vec : {&m->ev_sq, &m->ev_sg})
+    for (auto ev : *vec)
+      if (ev) cudaEventDestroy(ev);
   if (m->ev_fork) cudaEventDestroy(m->ev_fork);
   if (m->ev_join) cudaEventDestroy(m->ev_join);
   if (m->ev_pf_fork) cudaEventDestroy(m->ev_pf_fork);
@@ -1245,7 +1421,7 @@ ladder_status_t ladder_destroy(ladder_model_t* m) {
   }
   if (m->side) cudaStreamDestroy(m->side);
   if (m->cap) cudaStreamDestroy(m->cap);
-  void* bufs[] = {m->w16, m->w16b, m->wide_hpack, m->wide_opack, m->xpack[0], m->xpack[1], m->hpack, m->opack, m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
+  void* bufs[] = {m->w16, m->w16b, m->wide_hpack, m->wide_opack, m->pend_a, m->pend_m, m->xpack[0], m->xpack[1], m->hpack, m->opack, m->d_phases, m->d_attn, m->d_counters, m->gemm_scratch[0], m->gemm_scratch[1], m->work_slots, m->R[0], m->R[1], m->q_f32, m->o_dec, m->h_dec, m->attn_scratch, m->logits_ws, m->last_x,
                   m->n_pf, m->q_pf,  m->o_pf,  m->h_pf,  m->rope,  m->status,       m->tok_tmp,   m->next_tmp};
   for (void* b : bufs)
     if (b) cudaFree(b);
@@ -1287,8 +1463,8 @@ int32_t ladder_model_persistent_active(const ladder_model_t* m) { return (m && m
 
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream) {
   if (!m) return LADDER_ERR_INVALID_ARG;
-  if (sms_attention_stream < -2 || sms_attention_stream > m->sm_count / 2)
-    return fail(m, LADDER_ERR_INVALID_ARG, "sms_attention_stream must be -2, -1, 0 or at most half the SMs");
+  if (sms_attention_stream < -3 || sms_attention_stream > m->sm_count / 2)
+    return fail(m, LADDER_ERR_INVALID_ARG, "sms_attention_stream must be -3 .. 0 or at most half the SMs");
   m->sms_a = sms_attention_stream;
   drop_graph(m);
   return LADDER_OK;

@@ -128,7 +128,8 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 // >= batch are zero.  The slice's sum of squares goes to ssq[row][slice]; the GEMM adds the slices in order.
 constexpr int kStageSlice = 2048;
 __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const __nv_bfloat16* gain, int norm, int batch,
-                                                         int bp, int K, __nv_bfloat16* stage, float* ssq_out) {
+                                                         int bp, int K, __nv_bfloat16* stage, float* ssq_out,
+                                                         const float* pending, float* sum_out) {
   __shared__ float red[8];
   const int b = blockIdx.x, slice = blockIdx.y, tid = threadIdx.x;
   pdl_launch_dependents();
@@ -143,6 +144,15 @@ __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const _
       const float4 a = __ldcg(reinterpret_cast<const float4*>(x + static_cast<size_t>(b) * K + k));
       const float4 c = __ldcg(reinterpret_cast<const float4*>(x + static_cast<size_t>(b) * K + k + 4));
       y[0] = a.x, y[1] = a.y, y[2] = a.z, y[3] = a.w, y[4] = c.x, y[5] = c.y, y[6] = c.z, y[7] = c.w;
+      if (pending) {  // x_m = x_{m-1} + (the module output stored by an earlier GEMM)
+        const float4 pa = __ldcg(reinterpret_cast<const float4*>(pending + static_cast<size_t>(b) * K + k));
+        const float4 pc = __ldcg(reinterpret_cast<const float4*>(pending + static_cast<size_t>(b) * K + k + 4));
+        y[0] += pa.x, y[1] += pa.y, y[2] += pa.z, y[3] += pa.w, y[4] += pc.x, y[5] += pc.y, y[6] += pc.z, y[7] += pc.w;
+      }
+      if (sum_out) {
+        *reinterpret_cast<float4*>(sum_out + static_cast<size_t>(b) * K + k) = make_float4(y[0], y[1], y[2], y[3]);
+        *reinterpret_cast<float4*>(sum_out + static_cast<size_t>(b) * K + k + 4) = make_float4(y[4], y[5], y[6], y[7]);
+      }
 #pragma unroll
       for (int i = 0; i < 8; ++i) ssq += y[i] * y[i];
       if (norm) {
@@ -629,6 +639,32 @@ size_t smallm_gemm_wide_tc_smem_bytes(int batch) {
   return bp == 8 ? WCfg<16>::SMEM : (bp == 16 ? WCfg<32>::SMEM : (bp == 32 ? WCfg<64>::SMEM : WCfg<128>::SMEM));
 }
 
+namespace {
+cudaError_t launch_stage(const SmallMParams& p, int bp, int n_slices, __nv_bfloat16* stage, float* ssq, cudaStream_t stream,
+                         bool pdl) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(bp, n_slices);
+  cfg.blockDim = dim3(256);
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, wide_stage_kernel, static_cast<const float*>(p.act), p.gain,
+                            p.act_mode == ACT_F32_NORM ? 1 : 0, p.batch, bp, p.K, stage, ssq, p.act_pending,
+                            p.act_sum_out);
+}
+}  // namespace
+
+cudaError_t launch_smallm_gemm_wide_stage(const SmallMParams& p, cudaStream_t stream, bool pdl) {
+  if (!p.scratch || !p.act || p.batch < 1 || p.batch > 64 || (p.K & 7)) return cudaErrorInvalidValue;
+  const int bp = padded_batch(p.batch);
+  const int n_slices = (p.K + kStageSlice - 1) / kStageSlice;
+  if (n_slices > kWideMaxSlices) return cudaErrorInvalidValue;
+  return launch_stage(p, bp, n_slices, reinterpret_cast<__nv_bfloat16*>(p.scratch + stage_offset()), p.scratch, stream, pdl);
+}
+
 cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
   if (!g_encode_wide) return cudaErrorNotReady;
   if (!p.scratch || p.batch < 1 || p.batch > 64 || (p.K & 7) || (p.N & 1)) return cudaErrorInvalidValue;
@@ -646,18 +682,8 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
   if (p.act_staged) {  // the producing kernel has written the operand already
     if (p.act_mode != ACT_F32 || (reinterpret_cast<uintptr_t>(p.act_staged) & 15)) return cudaErrorInvalidValue;
     stage = const_cast<__nv_bfloat16*>(p.act_staged);
-  } else {  // 1. activations -> bf16 hi + lo, 1/rms
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(bp, n_slices);
-    cfg.blockDim = dim3(256);
-    cfg.stream = stream;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = at;
-    cfg.numAttrs = pdl ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, wide_stage_kernel, static_cast<const float*>(p.act), p.gain,
-                                       p.act_mode == ACT_F32_NORM ? 1 : 0, p.batch, bp, p.K, stage, ssq);
+  } else if (!p.wide_prestaged) {  // 1. activations -> bf16 hi + lo, 1/rms
+    cudaError_t e = launch_stage(p, bp, n_slices, stage, ssq, stream, pdl);
     if (e != cudaSuccess) return e;
   }
   CUtensorMap mw, ma;
@@ -675,7 +701,7 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
   a.tickets = tickets;
   const int total = tiles * nkb;
   const int grid = total < sm_count ? total : sm_count;
-  const bool pdl_attr = p.act_staged ? pdl : true;  // after its own staging kernel always; after a producer kernel if the caller says so
+  const bool pdl_attr = (p.act_staged || p.wide_prestaged) ? pdl : true;  // after its own staging kernel always; else if the caller says so
   if (bp == 8) return launch_np<16>(a, mw, ma, grid, stream, pdl_attr);
   if (bp == 16) return launch_np<32>(a, mw, ma, grid, stream, pdl_attr);
   if (bp == 32) return launch_np<64>(a, mw, ma, grid, stream, pdl_attr);

@@ -52,6 +52,13 @@ struct SmallMParams {
   //   act_staged:    this GEMM's activations are already staged that way ([2 Bp, K]; act_mode ACT_F32 only).
   __nv_bfloat16* wide_pack_out;
   const __nv_bfloat16* act_staged;
+  // Batch 5..64, the pending-output form of Algorithm 1: the staging step first forms y = act + act_pending (a
+  // module output that was stored, not added) and, if act_sum_out is given, writes y there (the residual stream
+  // moves on in the staging step instead of in a GEMM epilogue).  wide_prestaged: the staging for this GEMM has
+  // already been launched with launch_smallm_gemm_stage on the same scratch; the GEMM does not repeat it.
+  const float* act_pending;
+  float* act_sum_out;
+  int wide_prestaged;
   // Optional second copy of an fp32 output (EPI_RESID: out, EPI_SWIGLU: h) as the next GEMM's MMA operand:
   // y = value (* pack_gain[n]), bf16 hi at [n / 2048][b][n % 2048], lo at [n / 2048][4 + b][n % 2048]; batch <= 4.
   __nv_bfloat16* pack_out;
@@ -63,6 +70,9 @@ struct SmallMParams {
 };
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);
+// Batch 5..64 only: the staging launch of a GEMM on its own (p.act, p.act_pending, p.act_sum_out, p.gain, p.act_mode,
+// p.K, p.batch, p.scratch), so that an event can sit between it and the GEMM.
+cudaError_t launch_smallm_gemm_stage(const SmallMParams& p, cudaStream_t stream, bool pdl);
 size_t smallm_gemm_smem_bytes(int batch);
 size_t smallm_gemm_scratch_floats(int N, int K, int batch);
 void set_decode_wide_impl(int impl);  // 0 = tcgen05 kernel for batch 5..64 (default), 2 = for every batch

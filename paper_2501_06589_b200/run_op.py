@@ -168,7 +168,7 @@ def run_stack(a, s, bsz):
         model.set_persistent(False)
     if a.persistent_all:
         model.set_persistent(2)
-    if a.sm_split >= 0:
+    if a.sm_split != -1:
         model.set_sm_split(a.sm_split)
     persistent = model.persistent_active() and bsz <= 8
     cache = B.KVCache(s, bsz, S + steps + 1)

@@ -290,13 +290,14 @@ def _tp_slices(width: int, world: int) -> List[slice]:
 
 def attention_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndarray,
                      pos0: int, cache: Optional[OracleCache], bf16_storage: bool = False,
-                     bf16_kv: bool = False, tp_rank: Optional[int] = None):
+                     bf16_kv: bool = False, tp_rank: Optional[int] = None, parts_out: Optional[list] = None):
     """h(n) for the attention module of ``layer``.
 
     n [B, T, d] is the normalised input at absolute positions pos0..pos0+T-1.
     With a cache, the new K/V rows are appended at those positions first and
     attention then runs over positions 0..pos0+T-1 (append, then attend).
     With ``tp_rank`` the result is that rank's partial sum x* (before the all-reduce) only.
+    ``parts_out`` (a list) receives every rank's partial sum, for tests that play one rank against the others.
     """
     B, T, d = n.shape
     Hq, Hkv, Dh = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
@@ -328,13 +329,15 @@ def attention_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndar
     # kv heads), so everything up to here is rank-local; it multiplies its heads' slice of o with the matching
     # columns of W_o, and the partial products are summed over the ranks (the all-reduce of Sec. 2, Eq. 1).
     parts = [o[..., c] @ wo[:, c].T for c in _tp_slices(Hq * Dh, cfg.tp_world)]
+    if parts_out is not None:
+        parts_out.extend(parts)
     if tp_rank is not None:
         return parts[tp_rank]
     return parts[0] if len(parts) == 1 else np.sum(parts, axis=0)
 
 
 def mlp_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndarray,
-               bf16_storage: bool = False, tp_rank: Optional[int] = None):
+               bf16_storage: bool = False, tp_rank: Optional[int] = None, parts_out: Optional[list] = None):
     """h(n) = W_down ( silu(W_gate n) * (W_up n) ).
 
     Under tensor parallelism rank r owns the hidden columns [r F/P, (r+1) F/P): W_gate and W_up split by
@@ -345,6 +348,8 @@ def mlp_module(cfg: OracleConfig, W: OracleWeights, layer: int, n: np.ndarray,
     wd = W.get("w_down", layer).astype(dt, copy=False)
     h = _store(silu(n @ wg.T) * (n @ wu.T), bf16_storage)
     parts = [h[..., c] @ wd[:, c].T for c in _tp_slices(cfg.d_ff, cfg.tp_world)]
+    if parts_out is not None:
+        parts_out.extend(parts)
     if tp_rank is not None:
         return parts[tp_rank]
     return parts[0] if len(parts) == 1 else np.sum(parts, axis=0)
@@ -359,6 +364,7 @@ class ForwardResult:
     next_tokens: Optional[np.ndarray]   # [B, T']
     module_inputs: List[np.ndarray] = field(default_factory=list)   # residual each module read
     module_outputs: List[np.ndarray] = field(default_factory=list)  # h_m(.)
+    module_partials: List[List[np.ndarray]] = field(default_factory=list)  # per module: every rank's partial sum
 
 
 def greedy(logits: np.ndarray) -> np.ndarray:
@@ -387,13 +393,15 @@ def run_layers(cfg: OracleConfig, W: OracleWeights, x: np.ndarray, pos0: int,
     for spec in chain:
         src = older if (spec.stale and older is not None) else newest
         n = _store(rmsnorm(src, W.get(spec.norm, spec.layer), cfg.rms_eps), bf16_storage)
+        parts = [] if record is not None else None
         if spec.kind == "attention":
-            out = attention_module(cfg, W, spec.layer, n, pos0, cache, bf16_storage, bf16_kv)
+            out = attention_module(cfg, W, spec.layer, n, pos0, cache, bf16_storage, bf16_kv, parts_out=parts)
         else:
-            out = mlp_module(cfg, W, spec.layer, n, bf16_storage)
+            out = mlp_module(cfg, W, spec.layer, n, bf16_storage, parts_out=parts)
         if record is not None:
             record.module_inputs.append(src.copy())
             record.module_outputs.append(out.copy())
+            record.module_partials.append(parts)
         older, newest = newest, newest + out
     return (older, newest) if return_state else newest
 

@@ -193,6 +193,48 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
  * order.  -3 = the library's choice of split without that form (each output added by its GEMM's epilogue). */
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream);
 
+/* Tensor parallelism (paper Sec. 2, Eq. 1: x_i = AllReduce(h_i(x_{i-1})) + x_{i-1}; Sec. 3.1, Eq. 2 and Algorithm 1:
+ * with ladder residuals module i reads x_{i-2}, so the all-reduce of module i-1 runs while module i computes).
+ * The model handed to ladder_model_create is ONE RANK'S SLICE: n_q_heads, n_kv_heads and d_ff are the rank's share
+ * (w_qkv the rows of its heads, w_o the matching columns, w_gate_up the rows of its hidden units, w_down the
+ * matching columns); d_model, the norms, the embedding and the LM head are whole and the same on every rank.  The
+ * output and down projections then give a partial sum, and `exchange` is called - from inside ladder_prefill* /
+ * ladder_decode_step, on the calling host thread, in module order (attention of layer 0, MLP of layer 0, ...) - to
+ * ENQUEUE on `cuda_stream` the in-place sum of partial[0 .. count) (device, fp32, count = rows x d_model) over the
+ * ranks; it must not block on the device and every rank must get the same bits (the ranks' residual streams have to
+ * stay identical).  Non-zero return: the call fails with LADDER_ERR_CUDA.
+ * Schedule: every module stores its (partial) output and the sum is added where a later module's input is formed
+ * (the pending-output form of Algorithm 1).  Decode: the exchange runs on the stream of the module that produced
+ * the partial, so with two streams a ladder layer's other module computes meanwhile, while with standard residuals
+ * the next module's input waits for it (Eq. 1: the paper's baseline); all batch sizes run on the tcgen05 GEMMs, one
+ * kernel per GEMM.  Prompt pass: exchanges and adds run on a stream of their own and the GEMM stream waits only
+ * where a module reads what an add writes.  capturable != 0: `exchange` may be called while its stream is being
+ * captured into a CUDA graph (NCCL collectives may); 0: decode steps are enqueued without a graph.
+ * fn == NULL switches it off.  Pipeline-stage calls (ladder_stage_*) return LADDER_ERR_UNSUPPORTED while it is on.
+ * Costs 2 x max_prefill_tokens x d_model x 4 bytes of device memory on first use (LADDER_ERR_OOM if there is none).
+ * Measured on one GPU only (a world of one, and against recorded partials of the other ranks): the hardware this
+ * was built on has one GPU per job, so no multi-GPU timing is claimed. */
+typedef ladder_status_t (*ladder_exchange_fn)(void* ctx, float* partial, int64_t count, void* cuda_stream);
+ladder_status_t ladder_model_set_exchange(ladder_model_t* m, ladder_exchange_fn fn, void* ctx, int32_t capturable);
+
+/* The exchange over NCCL: one communicator per rank (= process = GPU, the current CUDA device at creation).
+ * Rank 0 draws an id with ladder_comm_unique_id (LADDER_COMM_ID_BYTES host bytes) and hands it to the other ranks by
+ * any means (e.g. a torch.distributed broadcast); every rank then calls ladder_comm_create (collective: returns when
+ * all `world` ranks have called it).  The NCCL library is looked up when first needed (the copy the process has
+ * loaded already, else the system's); LADDER_ERR_UNSUPPORTED if there is none, LADDER_ERR_CUDA if NCCL reports an
+ * error.  ladder_comm_all_reduce_sum has the ladder_exchange_fn signature (ctx = the communicator);
+ * ladder_model_set_tensor_parallel(m, comm) installs it (capturable), comm == NULL switches tensor parallelism off.
+ * The communicator is the caller's: destroy it after the models that use it. */
+#define LADDER_COMM_ID_BYTES 128
+typedef struct ladder_comm ladder_comm_t;
+ladder_status_t ladder_comm_unique_id(void* id);
+ladder_status_t ladder_comm_create(int32_t world, int32_t rank, const void* id, ladder_comm_t** out);
+ladder_status_t ladder_comm_destroy(ladder_comm_t* comm);
+int32_t ladder_comm_world(const ladder_comm_t* comm);
+int32_t ladder_comm_rank(const ladder_comm_t* comm);
+ladder_status_t ladder_comm_all_reduce_sum(void* comm, float* partial, int64_t count, void* cuda_stream);
+ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_t* comm);
+
 /* Prompt pass ("prefill phase", paper Sec. 3.2): the module chain of Eq. 1 / Eq. 2 (in the pending-output form of
  * Algorithm 1 with the all-reduce removed) over all prompt positions at once, causal attention within the prompt.
  * d_tokens int32 [batch, seq_len]; every sequence has the same length.

@@ -27,7 +27,12 @@ EXPORTS = [
     "ladder_op_decode_attention", "ladder_op_prefill_gemm", "ladder_op_prefill_attention", "ladder_op_prefill_attention_at",
     "ladder_op_decode_attention_noalloc", "ladder_set_prefill_gemm_impl", "ladder_set_decode_wide_impl", "ladder_set_decode_attention_impl",
     "ladder_op_prefill_gemm_f16", "ladder_op_convert_bf16_f16",
+    "ladder_model_set_exchange", "ladder_model_set_tensor_parallel", "ladder_comm_unique_id", "ladder_comm_create",
+    "ladder_comm_destroy", "ladder_comm_world", "ladder_comm_rank", "ladder_comm_all_reduce_sum",
 ]
+
+COMM_ID_BYTES = 128                                                              # LADDER_COMM_ID_BYTES
+EXCHANGE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p)   # ladder_exchange_fn
 
 
 class LadderError(RuntimeError):
@@ -145,6 +150,16 @@ def lib() -> C.CDLL:
                                                      C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                                      C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                                      C.c_void_p]
+        L.ladder_model_set_exchange.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]
+        L.ladder_model_set_tensor_parallel.argtypes = [C.c_void_p, C.c_void_p]
+        L.ladder_comm_unique_id.argtypes = [C.c_void_p]
+        L.ladder_comm_create.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.POINTER(C.c_void_p)]
+        L.ladder_comm_destroy.argtypes = [C.c_void_p]
+        L.ladder_comm_world.argtypes = [C.c_void_p]
+        L.ladder_comm_world.restype = C.c_int32
+        L.ladder_comm_rank.argtypes = [C.c_void_p]
+        L.ladder_comm_rank.restype = C.c_int32
+        L.ladder_comm_all_reduce_sum.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
         _lib = L
     return _lib
 
@@ -244,6 +259,32 @@ class KVCache:
         return self.v.view(*self.dims)
 
 
+class Comm:
+    """Owns a ladder_comm_t (one NCCL communicator of this process's current CUDA device)."""
+
+    def __init__(self, world: int, rank: int, unique_id: bytes):
+        assert len(unique_id) == COMM_ID_BYTES
+        h = C.c_void_p()
+        buf = C.create_string_buffer(unique_id, COMM_ID_BYTES)
+        _check(lib().ladder_comm_create(world, rank, buf, C.byref(h)))
+        self.h, self.world, self.rank = h, world, rank
+
+    @staticmethod
+    def unique_id() -> bytes:
+        buf = C.create_string_buffer(COMM_ID_BYTES)
+        _check(lib().ladder_comm_unique_id(buf))
+        return buf.raw
+
+    def all_reduce_sum(self, t: torch.Tensor):
+        assert t.dtype == torch.float32 and t.is_cuda and t.is_contiguous()
+        _check(lib().ladder_comm_all_reduce_sum(self.h, t.data_ptr(), t.numel(), _stream()))
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().ladder_comm_destroy(self.h)
+            self.h = None
+
+
 class Model:
     """Owns a ladder_model_t; keeps the borrowed weight tensors alive."""
 
@@ -291,6 +332,32 @@ class Model:
 
     def set_sm_split(self, sms_attention_stream: int = 0):
         _check(lib().ladder_model_set_sm_split(self.h, sms_attention_stream), self.h)
+
+    def set_exchange(self, fn=None, capturable: bool = False):
+        """Tensor parallelism with a caller-supplied sum over the ranks: fn(partial_ptr, count, cuda_stream) -> 0
+        enqueues the in-place sum of `count` fp32 values at device address `partial_ptr` on `cuda_stream`
+        (ladder_model_set_exchange).  None switches it off."""
+        if fn is None:
+            self._exchange_cb = None
+            _check(lib().ladder_model_set_exchange(self.h, None, None, 0), self.h)
+            return
+
+        def thunk(_ctx, ptr, count, stream):
+            try:
+                return int(fn(ptr, count, stream) or 0)
+            except Exception:                      # an exception must not cross the C frames
+                import traceback
+                traceback.print_exc()
+                return 1
+
+        cb = EXCHANGE_FN(thunk)
+        _check(lib().ladder_model_set_exchange(self.h, C.cast(cb, C.c_void_p), None, int(capturable)), self.h)
+        self._exchange_cb = cb                     # keep the thunk alive as long as the model may call it
+
+    def set_tensor_parallel(self, comm: Optional["Comm"]):
+        """This model is one rank's slice; partial sums are all-reduced over `comm` (ladder_model_set_tensor_parallel)."""
+        _check(lib().ladder_model_set_tensor_parallel(self.h, comm.h if comm is not None else None), self.h)
+        self._comm = comm
 
     def set_position(self, length: int):
         _check(lib().ladder_set_position(self.h, length), self.h)

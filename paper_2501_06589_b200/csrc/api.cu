@@ -76,7 +76,16 @@ struct ladder_model {
   __nv_bfloat16* wide_opack = nullptr;
   float* pend_a = nullptr;  // batch 5..64, pending-output schedule: the attention module's output, stored not added
   float* pend_m = nullptr;  // ... and the MLP module's
-  std::vector<cudaEvent_t> ev_sq, ev_sg;  // [layer]: x_{2l-1} / x_{2l} formed by the staging step of layer l's QKV / gate-up input
+  std::vector<cudaEvent_t> ev_sq, ev_sg;  // [layer]: the staging step of layer l's QKV / gate-up input has run ([L]: the head's)
+  std::vector<cudaEvent_t> ev_out;        // [module]: the module's stored output is complete (and summed over the ranks)
+  // tensor parallelism (Sec. 2, Eq. 1): sums a module's partial output over the ranks, in place, on the given stream
+  ladder_exchange_fn exchange = nullptr;
+  void* exchange_ctx = nullptr;
+  int exchange_capturable = 0;  // the callback may be called while its stream is being captured into a CUDA graph
+  ladder_comm* comm = nullptr;  // set by ladder_model_set_tensor_parallel (not owned)
+  float* pend_pf[2] = {nullptr, nullptr};  // prompt pass under tensor parallelism: the two modules' stored outputs
+  cudaStream_t xstream = nullptr;          // ... exchanged and added to the stream on this one
+  std::vector<cudaEvent_t> ev_pf_out, ev_pf_add;  // [module]: stored / added
   // the same activations as bf16 hi/lo MMA operands ([chunk][8][2048]), written by the persistent kernel's
   // epilogues for the phase that reads them next (batch <= 4): twins of R[0], R[1], h_dec, o_dec
   __nv_bfloat16 *xpack[2] = {nullptr, nullptr}, *hpack = nullptr, *opack = nullptr;
@@ -276,8 +285,10 @@ struct Enqueue {
   int64_t kernels = 0;
   int slot = 0;  // next claim-counter slot
   int grid_a = 0, grid_b = 0;  // CTAs per GEMM on stream A / B while the two run side by side (0 = all SMs)
+  bool force_wide = false;     // the tcgen05 GEMM at batch <= 4 too
   void gemm(int s, SmallMParams& p, bool side_by_side = false) {
-    p.scratch = m->gemm_scratch[s];
+    p.scratch = m->gemm_scratch[two ? s : 0];
+    p.force_wide = force_wide;
     p.work = m->work_slots + 2 * (slot++ % m->n_work_slots);
     p.status = m->status;
     const int g = (side_by_side && two && grid_a > 0) ? (s ? grid_b : grid_a) : m->sm_count;
@@ -305,158 +316,169 @@ struct Enqueue {
   }
 };
 
-// Batch 5..64, every layer a ladder layer: the decode step in the pending-output form of Algorithm 1.  The output
-// and down projections STORE their module's output (pend_a / pend_m) instead of adding it to the stream, and the
-// stream moves on in the staging step of the next reader: x_{2l-1} = x_{2l-2} + attn_{l-1} where the QKV projection of
-// layer l stages its input, x_{2l} = x_{2l-1} + mlp_{l-1} where the gate/up projection does.  With the adds fused into
-// the epilogues every output projection has to wait for the previous down projection and vice versa, so the two
-// streams move in lock-step; here the only cross-stream edges are between the (tiny) staging launches, and the
-// attention-module chain (stage, QKV, attention, Wo) and the MLP chain (stage, gate/up, down) of a layer run side by
-// side on their shares of the SMs.  The sums are the same fp32 additions in the same order: bit-identical results.
-// R[0] holds the even stream values (x_0 from the embedding, then x_{2l}), R[1] the odd ones.
+// The decode step in the pending-output form of Algorithm 1.  The output and down projections STORE their module's
+// output (pend_a / pend_m) instead of adding it to the stream, and the stream moves on in the staging step of a
+// later reader: the step that forms module j's input x_{j-1} (Eq. 1) or x_{j-2} (Eq. 2) adds the stored outputs
+// that are still missing from the newest stream value, in module order (none, one or two of them), and writes the
+// sum to the other residual buffer.  The sums are the same fp32 additions in the same order as with the adds in the
+// GEMM epilogues: bit-identical results.
+// What it buys: (1) with the adds in the epilogues every output projection of a ladder layer has to wait for the
+// previous down projection and vice versa, so the two streams move in lock-step; here the only cross-stream
+// edges are between the (tiny) staging launches, and the attention-module chain (stage, QKV, attention, Wo) and the
+// MLP chain (stage, gate/up, down) run side by side on their shares of the SMs.  (2) Under tensor parallelism
+// (Sec. 2, Eq. 1) the stored output is this rank's partial sum: the exchange callback sums it over the ranks on
+// the producing stream, and a ladder layer's other module computes meanwhile - the overlap Algorithm 1 is about;
+// with standard residuals the next module's staging step waits for it, as in the paper's baseline.
+// Not for parallel attention + MLP layers (one sum per layer) and not for pipeline stages.
 cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cache, const int32_t* d_tokens, int batch,
                                    const ladder_outputs_t* out, cudaStream_t sA, cudaStream_t sB, int64_t* n_kernels,
                                    int grid_a, int grid_b) {
   const ladder_config_t& c = m->cfg;
-  Enqueue q{m, sA, sB, true};
+  Enqueue q{m, sA, sB, sA != sB};
   q.grid_a = grid_a;
   q.grid_b = grid_b;
+  q.force_wide = batch <= 4;
   const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff, L = c.n_layers;
   const size_t layer_elems = static_cast<size_t>(c.max_batch) * Hkv * c.max_seq_len * Dh;
-  float* const x_even = m->R[0];
-  float* const x_odd = m->R[1];
   Router rt;
   q.launched(0, begin_stream(m, rt, d_tokens, batch, sA));
-  auto stage = [&](int s, SmallMParams& p) {  // the staging launch of a GEMM on its own (an event follows it)
-    p.scratch = m->gemm_scratch[s];
+  int cur = rt.cur;  // R[cur]: the newest stream value formed so far = x_0 + outputs of modules 0 .. added
+  int added = -1;
+  auto pend = [&](int j) { return (j & 1) ? m->pend_m : m->pend_a; };
+  auto ev_stage = [&](int j) { return (j & 1) ? m->ev_sg[j >> 1] : m->ev_sq[j >> 1]; };
+  // Staging step of module `mod` (2L = the head) on stream s: its input is x_0 + outputs of modules 0 .. upto.
+  auto form_input = [&](int mod, int s, int upto, SmallMParams& p) {
+    if (upto < added) upto = added;  // module 0 has no x_{-1}: it reads x_0 whatever its flag
+    if (mod > 0 && ((mod - 1) & 1) != s) q.wait(s, ev_stage(mod - 1));  // the stream value the previous step formed
+    for (int j = added + 1; j <= upto; ++j)
+      if ((j & 1) != s) q.wait(s, m->ev_out[j]);  // a stored output of the other stream (same stream: in order)
+    const int n = upto - added;                   // 0, 1 or 2
+    p.act = m->R[cur];
+    p.act_pending = n >= 1 ? pend(added + 1) : nullptr;
+    p.act_pending2 = n >= 2 ? pend(added + 2) : nullptr;
+    p.act_sum_out = n >= 1 ? m->R[cur ^ 1] : nullptr;
+    p.scratch = m->gemm_scratch[q.two ? s : 0];
     p.status = m->status;
+    p.force_wide = q.force_wide;
     q.launched(s, launch_smallm_gemm_stage(p, q.stream(s), q.pdl(s)));
+    if (n >= 1) cur ^= 1;
+    added = upto;
+    q.record(s, ev_stage(mod));
+    p.wide_prestaged = 1;
+  };
+  // The module's output is complete in pend(mod): sum it over the tensor-parallel ranks, tell the other stream.
+  auto output_stored = [&](int mod, int s) {
+    if (m->exchange) {
+      const ladder_status_t r = m->exchange(m->exchange_ctx, pend(mod), static_cast<int64_t>(batch) * d, q.stream(s));
+      if (r != LADDER_OK && q.err == cudaSuccess) q.err = cudaErrorUnknown;
+      q.pdl_ok[q.two ? s : 0] = false;
+    }
+    q.record(s, m->ev_out[mod]);
   };
   for (int l = 0; l < L; ++l) {
-    // ---------------- attention module on stream A
-    if (l > 0) q.wait(0, m->ev_sg[l - 1]);  // x_{2l-2}
-    SmallMParams p = {};
-    p.W = m->w_qkv[l];
-    p.N = (Hq + 2 * Hkv) * Dh;
-    p.K = d;
-    p.act = x_even;
-    p.act_pending = l > 0 ? m->pend_a : nullptr;  // attn_{l-1}; the first modules both read x_0
-    p.act_sum_out = x_odd;
-    p.act_mode = ACT_F32_NORM;
-    p.gain = m->attn_norm[l];
-    p.eps = c.rms_eps;
-    p.batch = batch;
-    stage(0, p);
-    q.record(0, m->ev_sq[l]);
-    p.wide_prestaged = 1;
-    p.epi_mode = EPI_QKV_ROPE;
-    p.qkv.q_out_f32 = m->q_f32;
-    p.qkv.k_cache = static_cast<kv_t*>(cache->k) + l * layer_elems;
-    p.qkv.v_cache = static_cast<kv_t*>(cache->v) + l * layer_elems;
-    p.qkv.seq_lens = cache->seq_lens;
-    p.qkv.rope = m->rope;
-    p.qkv.n_q_heads = Hq;
-    p.qkv.n_kv_heads = Hkv;
-    p.qkv.head_dim = Dh;
-    p.qkv.max_seq_len = c.max_seq_len;
-    q.gemm(0, p, true);
+    {  // ---------------- attention module (stream A)
+      const int mod = 2 * l, s = 0;
+      SmallMParams p = {};
+      p.W = m->w_qkv[l];
+      p.N = (Hq + 2 * Hkv) * Dh;
+      p.K = d;
+      p.act_mode = ACT_F32_NORM;
+      p.gain = m->attn_norm[l];
+      p.eps = c.rms_eps;
+      p.batch = batch;
+      form_input(mod, s, mod - 1 - (m->stale[mod] ? 1 : 0), p);
+      p.epi_mode = EPI_QKV_ROPE;
+      p.qkv.q_out_f32 = m->q_f32;
+      p.qkv.k_cache = static_cast<kv_t*>(cache->k) + l * layer_elems;
+      p.qkv.v_cache = static_cast<kv_t*>(cache->v) + l * layer_elems;
+      p.qkv.seq_lens = cache->seq_lens;
+      p.qkv.rope = m->rope;
+      p.qkv.n_q_heads = Hq;
+      p.qkv.n_kv_heads = Hkv;
+      p.qkv.head_dim = Dh;
+      p.qkv.max_seq_len = c.max_seq_len;
+      q.gemm(s, p, true);
 
-    DecodeAttnParams a = {};
-    a.q = m->q_f32;
-    a.k = p.qkv.k_cache;
-    a.v = p.qkv.v_cache;
-    a.kv_len = cache->seq_lens;
-    a.kv_len_offset = 1;
-    a.batch = batch;
-    a.n_q_heads = Hq;
-    a.n_kv_heads = Hkv;
-    a.head_dim = Dh;
-    a.max_seq_len = c.max_seq_len;
-    a.n_splits = m->attn_splits;
-    a.max_len = c.max_seq_len;
-    a.scratch = m->attn_scratch;
-    a.o = m->o_dec;
-    a.status = m->status;
-    a.o_pack = m->wide_opack;
-    a.o_pack_bp = wide_padded_batch(batch);
-    q.launched(0, launch_decode_attention(a, sA, q.pdl(0)));
-    ++q.kernels;  // the split kernel and its merge kernel
+      DecodeAttnParams a = {};
+      a.q = m->q_f32;
+      a.k = p.qkv.k_cache;
+      a.v = p.qkv.v_cache;
+      a.kv_len = cache->seq_lens;
+      a.kv_len_offset = 1;
+      a.batch = batch;
+      a.n_q_heads = Hq;
+      a.n_kv_heads = Hkv;
+      a.head_dim = Dh;
+      a.max_seq_len = c.max_seq_len;
+      a.n_splits = m->attn_splits;
+      a.max_len = c.max_seq_len;
+      a.scratch = m->attn_scratch;
+      a.o = m->o_dec;
+      a.status = m->status;
+      a.o_pack = m->wide_opack;
+      a.o_pack_bp = wide_padded_batch(batch);
+      q.launched(s, launch_decode_attention(a, q.stream(s), q.pdl(s)));
+      ++q.kernels;  // the split kernel and its merge kernel
 
-    SmallMParams o = {};
-    o.W = m->w_o[l];
-    o.N = d;
-    o.K = Hq * Dh;
-    o.act = m->o_dec;
-    o.act_mode = ACT_F32;
-    o.batch = batch;
-    o.epi_mode = EPI_PLAIN;
-    o.out = m->pend_a;  // read by the staging step of layer l + 1 (or of the head) on this stream
-    o.act_staged = m->wide_opack;
-    q.gemm(0, o, true);
+      SmallMParams o = {};
+      o.W = m->w_o[l];
+      o.N = d;
+      o.K = Hq * Dh;
+      o.act = m->o_dec;
+      o.act_mode = ACT_F32;
+      o.batch = batch;
+      o.epi_mode = EPI_PLAIN;
+      o.out = pend(mod);
+      o.act_staged = m->wide_opack;
+      q.gemm(s, o, true);
+      output_stored(mod, s);
+    }
+    {  // ---------------- MLP module (stream B)
+      const int mod = 2 * l + 1, s = q.two ? 1 : 0;
+      SmallMParams g = {};
+      g.W = m->w_gate_up[l];
+      g.N = 2 * F;
+      g.K = d;
+      g.act_mode = ACT_F32_NORM;
+      g.gain = mlp_gain(m, l);
+      g.eps = c.rms_eps;
+      g.batch = batch;
+      form_input(mod, s, mod - 1 - (m->stale[mod] ? 1 : 0), g);
+      g.epi_mode = EPI_SWIGLU;
+      g.out = m->h_dec;
+      g.wide_pack_out = m->wide_hpack;
+      q.gemm(s, g, true);
 
-    // ---------------- MLP module on stream B
-    q.wait(1, m->ev_sq[l]);  // x_{2l-1}
-    SmallMParams g = {};
-    g.W = m->w_gate_up[l];
-    g.N = 2 * F;
-    g.K = d;
-    g.act = x_odd;
-    g.act_pending = l > 0 ? m->pend_m : nullptr;  // mlp_{l-1}
-    g.act_sum_out = x_even;
-    g.act_mode = ACT_F32_NORM;
-    g.gain = mlp_gain(m, l);
-    g.eps = c.rms_eps;
-    g.batch = batch;
-    stage(1, g);
-    q.record(1, m->ev_sg[l]);
-    g.wide_prestaged = 1;
-    g.epi_mode = EPI_SWIGLU;
-    g.out = m->h_dec;
-    g.wide_pack_out = m->wide_hpack;
-    q.gemm(1, g, true);
-
-    SmallMParams dn = {};
-    dn.W = m->w_down[l];
-    dn.N = d;
-    dn.K = F;
-    dn.act = m->h_dec;
-    dn.act_mode = ACT_F32;
-    dn.batch = batch;
-    dn.epi_mode = EPI_PLAIN;
-    dn.out = m->pend_m;
-    dn.act_staged = m->wide_hpack;
-    q.gemm(1, dn, true);
+      SmallMParams dn = {};
+      dn.W = m->w_down[l];
+      dn.N = d;
+      dn.K = F;
+      dn.act = m->h_dec;
+      dn.act_mode = ACT_F32;
+      dn.batch = batch;
+      dn.epi_mode = EPI_PLAIN;
+      dn.out = pend(mod);
+      dn.act_staged = m->wide_hpack;
+      q.gemm(s, dn, true);
+      output_stored(mod, s);
+    }
   }
-  // ---------------- head on stream A: x_{2L-1} = x_{2L-2} + attn_{L-1}, then x_{2L} = x_{2L-1} + mlp_{L-1} in the head's
-  // own staging step
-  q.record(1, m->ev_sq[L]);  // the last down projection
-  q.wait(0, m->ev_sg[L - 1]);
-  SmallMParams t = {};
-  t.K = d;
-  t.act = x_even;
-  t.act_pending = m->pend_a;
-  t.act_sum_out = x_odd;
-  t.act_mode = ACT_F32;
-  t.batch = batch;
-  stage(0, t);
-  q.wait(0, m->ev_sq[L]);
+  // ---------------- head on stream A: reads x_{2L} (every output added)
   float* logits = (out && out->logits) ? out->logits : m->logits_ws;
   SmallMParams h = {};
   h.W = m->lm_head;
   h.N = c.vocab_size;
   h.K = d;
-  h.act = x_odd;
-  h.act_pending = m->pend_m;
-  h.act_sum_out = x_even;
   h.act_mode = ACT_F32_NORM;
   h.gain = m->final_norm;
   h.eps = c.rms_eps;
   h.batch = batch;
+  form_input(2 * L, 0, 2 * L - 1, h);
   h.epi_mode = EPI_PLAIN;
   h.out = logits;
   q.gemm(0, h);
   if (out && out->final_hidden)
-    q.launched(0, launch_rmsnorm_f32(x_even, m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, sA, q.pdl(0)));
+    q.launched(0, launch_rmsnorm_f32(m->R[cur], m->final_norm, c.rms_eps, batch, d, d, out->final_hidden, sA, q.pdl(0)));
   q.launched(0, launch_argmax_advance(logits, batch, c.vocab_size, out ? out->next_tokens : nullptr, cache->seq_lens, 1,
                                       -1, sA, q.pdl(0)));
   *n_kernels = q.kernels;
@@ -484,6 +506,11 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   // two launches side by side overlap those costs: 60 of 148 SMs for the attention stream measured 581 -> 553 us per
   // 8 layers at batch 16 and 921 -> 865 us at batch 64 (at the 70B shape the split loses at every batch).
   const double layer_bytes = 2.0 * (static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh + 3.0 * F * d);
+  if (m->exchange) {  // tensor parallelism: the pending-output form at every batch size, all SMs per GEMM unless told otherwise
+    const bool split = sA != sB && m->sms_a > 0;
+    return enqueue_decode_pending(m, cache, d_tokens, batch, out, sA, sB, n_kernels, split ? m->sms_a : 0,
+                                  split ? m->sm_count - m->sms_a : 0);
+  }
   const bool auto_wide = (m->sms_a == -1 || m->sms_a == -3) && batch > 4 && layer_bytes < 300e6;
   if (q.two && (m->sms_a >= 0 || auto_wide)) {
     int ga = auto_wide ? (60 * m->sm_count + 74) / 148 : m->sms_a;
@@ -717,9 +744,38 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
     convert_layer(0, m->w16, m->side);
     note(cudaEventRecord(m->ev_w16_ready[0], m->side));
   }
-  auto norm = [&](const float* x, const __nv_bfloat16* gain) {
+  // Tensor parallelism (Sec. 2, Eq. 1; Algorithm 1): the output and down projections store this rank's partial sum,
+  // the exchange stream sums it over the ranks and adds it to the stream value, and this stream goes on with the
+  // next module; it waits for an add only where a module reads the buffer that add writes (a ladder module's
+  // input x_{m-2} is older than the exchange in flight; with standard residuals the very next module waits).
+  const bool tp = m->exchange != nullptr;
+  int add_writer[2] = {-1, -1};  // module whose add on the exchange stream last wrote R[i]
+  auto norm = [&](int buf, const __nv_bfloat16* gain) {
+    if (tp && add_writer[buf] >= 0) note(cudaStreamWaitEvent(st, m->ev_pf_add[add_writer[buf]], 0));
+    const float* x = m->R[buf];
     if (f16) did(launch_rmsnorm_f16(x, gain, c.rms_eps, M, d, reinterpret_cast<__half*>(m->n_pf), st));
     else did(launch_rmsnorm_bf16(x, gain, c.rms_eps, M, d, m->n_pf, n_lo, st));
+  };
+  // Last GEMM of module mod (0-based): x_m = x_{m-1} + output, x_{m-1} in R[r.add], x_m to R[r.dst].
+  auto finish_module = [&](int mod, const Router::Route& r, LargeMParams& o) {
+    if (!tp) {
+      o.epi_mode = EPI_RESID;
+      o.addend = m->R[r.add];
+      o.out = m->R[r.dst];
+      did(launch_largem_gemm(o, st));
+      return;
+    }
+    float* const pend = m->pend_pf[mod & 1];
+    if (mod >= 2) note(cudaStreamWaitEvent(st, m->ev_pf_add[mod - 2], 0));  // the buffer's previous content is added
+    o.epi_mode = EPI_PLAIN;
+    o.out = pend;
+    did(launch_largem_gemm(o, st));
+    note(cudaEventRecord(m->ev_pf_out[mod], st));
+    note(cudaStreamWaitEvent(m->xstream, m->ev_pf_out[mod], 0));
+    if (m->exchange(m->exchange_ctx, pend, static_cast<int64_t>(M) * d, m->xstream) != LADDER_OK) note(cudaErrorUnknown);
+    did(launch_add_f32(m->R[r.add], pend, m->R[r.dst], static_cast<size_t>(M) * d, m->xstream));
+    note(cudaEventRecord(m->ev_pf_add[mod], m->xstream));
+    add_writer[r.dst] = mod;
   };
   for (int l = 0; l < c.n_layers; ++l) {
     __half* const w16_qkv = overlap && (l & 1) ? m->w16b : m->w16;
@@ -738,7 +794,7 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
     }
     {
       const Router::Route r = route(m, rt, 2 * l + 1);
-      norm(m->R[r.in], m->attn_norm[l]);
+      norm(r.in, m->attn_norm[l]);
       LargeMParams p = {};
       p.A = m->n_pf;
       p.A_lo = n_lo;
@@ -772,15 +828,12 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       o.M = M;
       o.N = d;
       o.K = Hq * Dh;
-      o.epi_mode = EPI_RESID;
-      o.addend = m->R[r.add];
-      o.out = m->R[r.dst];
       o.status = m->status;
-      did(launch_largem_gemm(o, st));
+      finish_module(2 * l, r, o);
     }
     {
       const Router::Route r = route(m, rt, 2 * l + 2);
-      norm(m->R[r.in], mlp_gain(m, l));
+      norm(r.in, mlp_gain(m, l));
       LargeMParams p = {};
       p.A = m->n_pf;
       p.A_lo = n_lo;
@@ -802,14 +855,12 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       o.M = M;
       o.N = d;
       o.K = F;
-      o.epi_mode = EPI_RESID;
-      o.addend = m->R[r.add];
-      o.out = m->R[r.dst];
       o.status = m->status;
-      did(launch_largem_gemm(o, st));
+      finish_module(2 * l + 1, r, o);
     }
     if (overlap) note(cudaEventRecord(m->ev_w16_free[l & 1], st));
   }
+  if (tp && c.n_layers > 0) note(cudaStreamWaitEvent(st, m->ev_pf_add[2 * c.n_layers - 1], 0));  // every add (in order)
   if (m->st_out.newest) {  // a stage that hands its state on: every position's stream state, no head
     did(end_stage(m, rt, cache, batch, M, 0, pos0 + S, d_lens, st));
     *n_kernels = k;
@@ -1291,12 +1342,10 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
   A(dev_alloc(&m->q_f32, MB * qd));
   A(dev_alloc(&m->o_dec, MB * qd));
   A(dev_alloc(&m->h_dec, MB * F));
-  if (c.max_batch > 4) {
-    A(dev_alloc(&m->wide_hpack, 2 * 64 * F));
-    A(dev_alloc(&m->wide_opack, 2 * 64 * qd));
-    A(dev_alloc(&m->pend_a, MB * d));
-    A(dev_alloc(&m->pend_m, MB * d));
-  }
+  A(dev_alloc(&m->wide_hpack, 2 * 64 * F));
+  A(dev_alloc(&m->wide_opack, 2 * 64 * qd));
+  A(dev_alloc(&m->pend_a, MB * d));
+  A(dev_alloc(&m->pend_m, MB * d));
   const auto pack_elems = [](size_t K) { return ((K + 2047) / 2048) * 8 * 2048; };
   A(dev_alloc(&m->xpack[0], pack_elems(d)));
   A(dev_alloc(&m->xpack[1], pack_elems(d)));
@@ -1383,9 +1432,13 @@ ladder_status_t ladder_model_create(const ladder_config_t* cfg, const ladder_wei
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
   m->ev_sq.resize(L + 1, nullptr);
   m->ev_sg.resize(L + 1, nullptr);
-  for (auto* vec : {&m->ev_sq, &m->ev_sg})
+  m->ev_out.resize(2 * L, nullptr);
+  m->ev_pf_out.resize(2 * L, nullptr);
+  m->ev_pf_add.resize(2 * L, nullptr);
+  for (auto* vec : {&m->ev_sq, &m->ev_sg, &m->ev_out, &m->ev_pf_out, &m->ev_pf_add})
     for (auto& ev : *vec)
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&m->xstream, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_pf_fork, cudaEventDisableTiming);
@@ -1408,9 +1461,12 @@ ladder_status_t ladder_destroy(ladder_model_t* m) {
   drop_graph(m);
   for (auto ev : m->ev)
     if (ev) cudaEventDestroy(ev);
-  for (auto* vec : {&m->ev_sq, &m->ev_sg})
+  for (auto* vec : {&m->ev_sq, &m->ev_sg, &m->ev_out, &m->ev_pf_out, &m->ev_pf_add})
     for (auto ev : *vec)
       if (ev) cudaEventDestroy(ev);
+  if (m->xstream) cudaStreamDestroy(m->xstream);
+  if (m->pend_pf[0]) cudaFree(m->pend_pf[0]);
+  if (m->pend_pf[1]) cudaFree(m->pend_pf[1]);
   if (m->ev_fork) cudaEventDestroy(m->ev_fork);
   if (m->ev_join) cudaEventDestroy(m->ev_join);
   if (m->ev_pf_fork) cudaEventDestroy(m->ev_pf_fork);
@@ -1460,6 +1516,32 @@ ladder_status_t ladder_debug_stall_last_phase(ladder_model_t* m, int32_t on) {
 }
 
 int32_t ladder_model_persistent_active(const ladder_model_t* m) { return (m && m->use_stack && m->stack_ok) ? 1 : 0; }
+
+ladder_status_t ladder_model_set_exchange(ladder_model_t* m, ladder_exchange_fn fn, void* ctx, int32_t capturable) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  if (fn && (!m->pend_pf[0] || !m->pend_pf[1])) {
+    const size_t n = static_cast<size_t>(m->cfg.max_prefill_tokens) * m->cfg.d_model;
+    for (int i = 0; i < 2; ++i)
+      if (!m->pend_pf[i] && dev_alloc(&m->pend_pf[i], n) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(m, LADDER_ERR_OOM, "no room for the prompt pass's stored module outputs");
+      }
+  }
+  m->exchange = fn;
+  m->exchange_ctx = fn ? ctx : nullptr;
+  m->exchange_capturable = (fn && capturable) ? 1 : 0;
+  m->comm = nullptr;
+  drop_graph(m);
+  return LADDER_OK;
+}
+
+ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_t* comm) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  if (!comm) return ladder_model_set_exchange(m, nullptr, nullptr, 0);
+  const ladder_status_t s = ladder_model_set_exchange(m, ladder_comm_all_reduce_sum, comm, 1);
+  if (s == LADDER_OK) m->comm = comm;
+  return s;
+}
 
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream) {
   if (!m) return LADDER_ERR_INVALID_ARG;
@@ -1656,6 +1738,7 @@ ladder_status_t ladder_stage_prefill(ladder_model_t* m, const ladder_kv_cache_t*
   if (!m) return LADDER_ERR_INVALID_ARG;
   if (const char* why = check_stage(state_in, state_out, d_tokens)) return fail(m, LADDER_ERR_INVALID_ARG, why);
   if (state_out && out && out->all_hidden) return fail(m, LADDER_ERR_INVALID_ARG, "a stage that hands its state on has no head outputs");
+  if (m->exchange) return fail(m, LADDER_ERR_UNSUPPORTED, "pipeline stages under tensor parallelism");
   StageScope scope(m, state_in, state_out);
   return ladder_prefill(m, cache, d_tokens, batch, seq_len, out, cuda_stream);
 }
@@ -1697,7 +1780,8 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
   const bool two = m->n_streams == 2;
 
   const bool staged = m->st_in.newest || m->st_out.newest;  // a pipeline stage runs kernel by kernel
-  if (m->use_stack && m->stack_ok && batch <= 4 && !staged) {
+  if (staged && m->exchange) return fail(m, LADDER_ERR_UNSUPPORTED, "pipeline stages under tensor parallelism");
+  if (m->use_stack && m->stack_ok && batch <= 4 && !staged && !m->exchange) {
     GraphKey key;
     key.batch = batch;
     key.k = cache->k;
@@ -1733,7 +1817,7 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
     }
   }
 
-  if (!m->use_graph) {
+  if (!m->use_graph || (m->exchange && !m->exchange_capturable)) {
     int64_t k = 0;
     if (two) {
       // the side stream may only start after everything already queued on the caller's stream

@@ -533,15 +533,15 @@ size_t smallm_gemm_scratch_floats(int N, int K, int batch) {
 }
 
 cudaError_t launch_smallm_gemm_stage(const SmallMParams& p, cudaStream_t stream, bool pdl) {
-  if (p.batch <= 4 && g_wide_impl != 2) return cudaErrorInvalidValue;  // the batch <= 4 kernel stages inside itself
+  if (p.batch <= 4 && g_wide_impl != 2 && !p.force_wide) return cudaErrorInvalidValue;  // the batch <= 4 kernel stages inside itself
   return launch_smallm_gemm_wide_stage(p, stream, pdl);
 }
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count) {
   // Batch 5..64 on the tcgen05 kernel: this file's kernel holds a bf16 hi + lo activation pair only for batch <= 4
   // (one 8-column MMA tile).
-  if (p.batch > 4 || g_wide_impl == 2) return launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count);
-  if (!p.work || p.act_pending || p.act_sum_out || p.wide_prestaged) return cudaErrorInvalidValue;
+  if (p.batch > 4 || g_wide_impl == 2 || p.force_wide) return launch_smallm_gemm_wide_tc(p, stream, pdl, sm_count);
+  if (!p.work || p.act_pending || p.act_pending2 || p.act_sum_out || p.wide_prestaged) return cudaErrorInvalidValue;
   const int units = p.N >> 3;
   const int grid = units < sm_count ? units : sm_count;
   return launch_small(p, stream, pdl, grid);

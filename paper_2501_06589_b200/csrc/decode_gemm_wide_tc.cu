@@ -129,7 +129,8 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 constexpr int kStageSlice = 2048;
 __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const __nv_bfloat16* gain, int norm, int batch,
                                                          int bp, int K, __nv_bfloat16* stage, float* ssq_out,
-                                                         const float* pending, float* sum_out) {
+                                                         const float* pending, const float* pending2,
+                                                         float* sum_out) {
   __shared__ float red[8];
   const int b = blockIdx.x, slice = blockIdx.y, tid = threadIdx.x;
   pdl_launch_dependents();
@@ -147,6 +148,11 @@ __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const _
       if (pending) {  // x_m = x_{m-1} + (the module output stored by an earlier GEMM)
         const float4 pa = __ldcg(reinterpret_cast<const float4*>(pending + static_cast<size_t>(b) * K + k));
         const float4 pc = __ldcg(reinterpret_cast<const float4*>(pending + static_cast<size_t>(b) * K + k + 4));
+        y[0] += pa.x, y[1] += pa.y, y[2] += pa.z, y[3] += pa.w, y[4] += pc.x, y[5] += pc.y, y[6] += pc.z, y[7] += pc.w;
+      }
+      if (pending2) {  // ... and the one after it
+        const float4 pa = __ldcg(reinterpret_cast<const float4*>(pending2 + static_cast<size_t>(b) * K + k));
+        const float4 pc = __ldcg(reinterpret_cast<const float4*>(pending2 + static_cast<size_t>(b) * K + k + 4));
         y[0] += pa.x, y[1] += pa.y, y[2] += pa.z, y[3] += pa.w, y[4] += pc.x, y[5] += pc.y, y[6] += pc.z, y[7] += pc.w;
       }
       if (sum_out) {
@@ -653,7 +659,7 @@ cudaError_t launch_stage(const SmallMParams& p, int bp, int n_slices, __nv_bfloa
   cfg.numAttrs = pdl ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, wide_stage_kernel, static_cast<const float*>(p.act), p.gain,
                             p.act_mode == ACT_F32_NORM ? 1 : 0, p.batch, bp, p.K, stage, ssq, p.act_pending,
-                            p.act_sum_out);
+                            p.act_pending2, p.act_sum_out);
 }
 }  // namespace
 

@@ -52,13 +52,17 @@ struct SmallMParams {
   //   act_staged:    this GEMM's activations are already staged that way ([2 Bp, K]; act_mode ACT_F32 only).
   __nv_bfloat16* wide_pack_out;
   const __nv_bfloat16* act_staged;
-  // Batch 5..64, the pending-output form of Algorithm 1: the staging step first forms y = act + act_pending (a
-  // module output that was stored, not added) and, if act_sum_out is given, writes y there (the residual stream
-  // moves on in the staging step instead of in a GEMM epilogue).  wide_prestaged: the staging for this GEMM has
-  // already been launched with launch_smallm_gemm_stage on the same scratch; the GEMM does not repeat it.
+  // The pending-output form of Algorithm 1 (tcgen05 kernel): the staging step first forms
+  // y = act + act_pending + act_pending2 (module outputs that were stored, not added; in that order) and, if
+  // act_sum_out is given, writes y there (the residual stream moves on in the staging step instead of in a GEMM
+  // epilogue).  wide_prestaged: the staging for this GEMM has already been launched with
+  // launch_smallm_gemm_stage on the same scratch; the GEMM does not repeat it.  force_wide: the tcgen05 kernel
+  // at batch <= 4 too (it is the one that knows this form).
   const float* act_pending;
+  const float* act_pending2;
   float* act_sum_out;
   int wide_prestaged;
+  int force_wide;
   // Optional second copy of an fp32 output (EPI_RESID: out, EPI_SWIGLU: h) as the next GEMM's MMA operand:
   // y = value (* pack_gain[n]), bf16 hi at [n / 2048][b][n % 2048], lo at [n / 2048][4 + b][n % 2048]; batch <= 4.
   __nv_bfloat16* pack_out;
@@ -70,8 +74,9 @@ struct SmallMParams {
 };
 
 cudaError_t launch_smallm_gemm(const SmallMParams& p, cudaStream_t stream, bool pdl, int sm_count);
-// Batch 5..64 only: the staging launch of a GEMM on its own (p.act, p.act_pending, p.act_sum_out, p.gain, p.act_mode,
-// p.K, p.batch, p.scratch), so that an event can sit between it and the GEMM.
+// tcgen05 kernel only (batch > 4 or force_wide): the staging launch of a GEMM on its own (p.act, p.act_pending,
+// p.act_pending2, p.act_sum_out, p.gain, p.act_mode, p.K, p.batch, p.scratch), so that an event can sit between it
+// and the GEMM.
 cudaError_t launch_smallm_gemm_stage(const SmallMParams& p, cudaStream_t stream, bool pdl);
 size_t smallm_gemm_smem_bytes(int batch);
 size_t smallm_gemm_scratch_floats(int N, int K, int batch);
@@ -224,6 +229,8 @@ cudaError_t launch_rmsnorm_f16(const float* x, const __nv_bfloat16* gain, float 
                                cudaStream_t stream);
 // n elements, n % 8 == 0, both pointers 16-byte aligned
 cudaError_t launch_convert_bf16_f16(const __nv_bfloat16* src, __half* dst, size_t n, cudaStream_t stream);
+// out = a + b, n fp32 elements (n a multiple of 4, 16-byte aligned pointers; out may be a or b)
+cudaError_t launch_add_f32(const float* a, const float* b, float* out, size_t n, cudaStream_t stream);
 cudaError_t launch_rmsnorm_f32(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, int row_stride,
                                float* out, cudaStream_t stream, bool pdl);
 // lens (device, optional): row r is taken at offset lens[r] - 1 instead of src_offset_rows

@@ -119,6 +119,16 @@ __global__ void convert_bf16_f16_kernel(const uint4* src, uint4* dst, size_t n8)
   }
 }
 
+// out = a + b (fp32, four elements per thread and iteration): the residual add of a module output that was stored
+// and summed over the tensor-parallel ranks first (prompt pass).
+__global__ void add_f32_kernel(const float4* a, const float4* b, float4* out, size_t n4) {
+  for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n4;
+       i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const float4 x = a[i], y = __ldcs(b + i);
+    out[i] = make_float4(x.x + y.x, x.y + y.y, x.z + y.z, x.w + y.w);
+  }
+}
+
 // out[r, :] = x[(r * stride + offset), :]; with `lens` the offset of row r is lens[r] - 1 (its last valid position)
 __global__ void gather_rows_kernel(const float* x, int d, int stride, int offset, const int32_t* lens, float* out) {
   if (lens) offset = min(max(lens[blockIdx.x], 1), stride) - 1;
@@ -222,6 +232,16 @@ cudaError_t launch_convert_bf16_f16(const __nv_bfloat16* src, __half* dst, size_
   const size_t blocks = (n8 + 255) / 256;
   return launch(convert_bf16_f16_kernel, dim3(static_cast<unsigned>(blocks < 148 * 16 ? (blocks ? blocks : 1) : 148 * 16)),
                 dim3(256), stream, false, reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), n8);
+}
+
+cudaError_t launch_add_f32(const float* a, const float* b, float* out, size_t n, cudaStream_t stream) {
+  if (n % 4 || ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(out)) & 15))
+    return cudaErrorInvalidValue;
+  const size_t n4 = n / 4;
+  const size_t blocks = (n4 + 255) / 256;
+  return launch(add_f32_kernel, dim3(static_cast<unsigned>(blocks < 148 * 8 ? (blocks ? blocks : 1) : 148 * 8)), dim3(256),
+                stream, false, reinterpret_cast<const float4*>(a), reinterpret_cast<const float4*>(b),
+                reinterpret_cast<float4*>(out), n4);
 }
 
 cudaError_t launch_rmsnorm_f32(const float* x, const __nv_bfloat16* gain, float eps, int rows, int d, int row_stride,

@@ -22,6 +22,7 @@ def L():
 def test_every_declared_symbol_is_exported(L):
     header = open(os.path.join(ROOT, "include", "ladder.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    header = re.sub(r"typedef[^;{]*\(\*[^;]*;", "", header)          # function-pointer types are not entry points
     declared = set(re.findall(r"\b(ladder_[a-z0-9_]+)\s*\(", header))
     assert declared, "no declarations parsed"
     for name in sorted(declared):

@@ -1,0 +1,183 @@
+"""Tensor parallelism on ONE GPU (paper Sec. 2, Eq. 1; Sec. 3.1, Algorithm 1).
+
+No second GPU is available to these tests, so the other ranks are played by the oracle: it runs the whole model
+split over the ranks and records every rank's partial sum of every module; the GPU runs rank 0's weight slice and
+its exchange callback adds the recorded partials of the other ranks where an all-reduce would.  What comes out must
+be the unsplit model.  A second set runs the NCCL exchange itself in a world of one rank (the collective is then
+the identity, but it is enqueued, captured into the decode graph and replayed like any other)."""
+import os
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+from oracle import ladder_oracle as O                                        # noqa: E402
+from paper_2501_06589_b200 import synth                                      # noqa: E402
+from tests.helpers import rel_err                                            # noqa: E402
+
+pytestmark = pytest.mark.gpu
+HIDDEN_TOL = 2e-2
+BASE = synth.ModelShape("tiny_tp", 256, 4, 4, 2, 64, 704, 1024, 1e-5, 10000.0, None, 2, 12, 6, 11)
+VARIANTS = {"ladder": None, "standard": (0, 0, 0, 0), "hybrid": (0, 0, 1, 1)}
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2501_06589_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+def oracle_cfg(s, world):
+    c = O.OracleConfig(s.d_model, s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.vocab_size,
+                       s.rms_eps, s.rope_theta, None if s.layer_is_ladder is None else list(s.layer_is_ladder))
+    c.tp_world = world
+    return c
+
+
+class _DeviceFloats:
+    """`count` fp32 values at a raw device address, for torch.as_tensor (no copy)."""
+
+    def __init__(self, ptr, count):
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": "<f4", "data": (ptr, False), "version": 2}
+
+
+def shape_of(variant):
+    from dataclasses import replace
+    return replace(BASE, layer_is_ladder=VARIANTS[variant])
+
+
+@pytest.mark.parametrize("streams", [2, 1])
+@pytest.mark.parametrize("batch", [2, 6])
+@pytest.mark.parametrize("variant", ["ladder", "standard", "hybrid"])
+def test_rank_0_with_the_oracle_as_rank_1(B, variant, batch, streams):
+    from paper_2501_06589_b200 import tensor_parallel as TP
+    s = shape_of(variant)
+    world, S, steps = 2, 12, 6
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    prompt = synth.make_tokens(s, batch, S)
+
+    # the oracle: the model split over two ranks, every rank's partial sums recorded call by call
+    cfg = oracle_cfg(s, world)
+    OW = O.OracleWeights(provider=synth.logical_provider(w, np.float64))
+    cache_o = O.OracleCache(cfg, batch, S + steps + 1, np.float64)
+    calls, o_toks, o_hids = [], [], []
+    r = O.forward(cfg, OW, prompt, np.float64, cache_o, 0, last_only=True, record=True)
+    for j in range(steps + 1):
+        calls.append([parts[1] for parts in r.module_partials])
+        o_toks.append(r.next_tokens[:, 0])
+        o_hids.append(r.hidden[:, 0])
+        if j < steps:
+            r = O.forward(cfg, OW, o_toks[-1].reshape(-1, 1), np.float64, cache_o, cache_o.seq_len, last_only=True,
+                          record=True)
+    unsplit = O.generate(oracle_cfg(s, 1), OW, prompt, steps, S + steps + 1, dtype=np.float64,
+                         forced=np.stack(o_toks, 1))
+    assert rel_err(np.stack(o_hids, 1), unsplit[1]) < 1e-9            # the split oracle is the unsplit one
+
+    # the GPU: rank 0's slice; the exchange adds rank 1's recorded partial of the same module
+    rw = TP.rank_weights(w, 0, world)
+    model = B.Model(rw, batch, S + steps + 1, batch * S)
+    model.set_schedule(streams, True, True)
+    queue, seen = [], []
+
+    def exchange(ptr, count, stream):
+        peer = queue.pop(0)
+        assert peer.numel() == count, (peer.numel(), count)
+        view = torch.as_tensor(_DeviceFloats(ptr, count), device="cuda")
+        with torch.cuda.stream(torch.cuda.ExternalStream(stream or 0)):
+            view.add_(peer)
+        seen.append(count)
+        return 0
+
+    model.set_exchange(exchange, capturable=False)
+    cache = B.KVCache(rw.shape, batch, S + steps + 1)
+    nxt = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    hid = torch.zeros(batch, s.d_model, device="cuda")
+    toks, hids = [], []
+    for j in range(steps + 1):
+        queue[:] = [torch.from_numpy(np.ascontiguousarray(p, dtype=np.float32).reshape(-1)).cuda() for p in calls[j]]
+        if j == 0:
+            model.prefill(cache, torch.from_numpy(prompt).cuda(), next_tokens=nxt, final_hidden=hid)
+        else:                                                   # teacher forcing: the recorded partials belong to these tokens
+            feed = torch.from_numpy(o_toks[j - 1].astype(np.int32)).cuda()
+            model.decode_step(cache, feed, next_tokens=nxt, final_hidden=hid)
+        torch.cuda.synchronize()
+        assert not queue, "an exchange was skipped"
+        toks.append(nxt.cpu().numpy().copy())
+        hids.append(hid.cpu().numpy().copy())
+    assert model.device_status() == 0
+    assert seen == [batch * S * s.d_model] * (2 * s.n_layers) + [batch * s.d_model] * (2 * s.n_layers * steps)
+    err = rel_err(np.stack(hids, 1), np.stack(o_hids, 1))
+    agree = float(np.mean(np.stack(toks, 1) == np.stack(o_toks, 1)))
+    print(f"[tp rank 0 / oracle rank 1, {variant}, batch {batch}, {streams} stream(s)] hidden max-rel-err {err:.3e}, "
+          f"greedy agreement {agree:.3f} over {batch * (steps + 1)}")
+    assert err < HIDDEN_TOL, err
+    assert agree >= 0.9, agree
+    model.close()
+
+
+@pytest.mark.parametrize("variant,batch", [("ladder", 3), ("standard", 3), ("ladder", 12), ("hybrid", 12)])
+def test_world_of_one_over_nccl(B, variant, batch):
+    """The NCCL exchange in a world of one: the steps run in the pending-output form with an all-reduce after every
+    module, inside the captured decode graph.  Bit-identical to the same form with a do-nothing callback enqueued
+    step by step, and - where the default schedule is that form too (all ladder, batch > 4) - to the default."""
+    from paper_2501_06589_b200 import tensor_parallel as TP
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from tests.test_gpu_model import gpu_generate, oracle_teacher_forced
+    s = shape_of(variant)
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    S, steps = 10, 12
+    prompt = synth.make_tokens(s, batch, S)
+    comm = TP.make_comm()
+    assert (comm.world, comm.rank) == (1, 0)
+    probe = torch.arange(8, dtype=torch.float32, device="cuda")
+    comm.all_reduce_sum(probe)
+    assert torch.equal(probe.cpu(), torch.arange(8, dtype=torch.float32))
+
+    def run(mode):
+        model = B.Model(w, batch, S + steps + 2, batch * S)
+        if mode == "nccl":
+            model.set_tensor_parallel(comm)
+        elif mode == "callback":
+            model.set_exchange(lambda ptr, count, stream: 0, capturable=False)
+        cache = B.KVCache(s, batch, S + steps + 2)
+        toks, hids = gpu_generate(B, model, cache, prompt, steps)
+        assert model.device_status() == 0
+        model.close()
+        return toks, hids
+
+    t_nccl, h_nccl = run("nccl")
+    t_cb, h_cb = run("callback")
+    assert np.array_equal(t_nccl, t_cb) and np.array_equal(h_nccl, h_cb)
+    if variant == "ladder" and batch > 4:
+        t_def, h_def = run("default")
+        assert np.array_equal(t_nccl, t_def) and np.array_equal(h_nccl, h_def)
+    o_toks, o_hids, _ = oracle_teacher_forced(s, w, prompt, t_nccl, np.float64)
+    err = rel_err(h_nccl, o_hids)
+    print(f"[nccl world 1, {variant}, batch {batch}] hidden max-rel-err {err:.3e}, greedy agreement "
+          f"{float(np.mean(t_nccl == o_toks)):.3f}")
+    assert err < HIDDEN_TOL, err
+    comm.close()
+
+
+def test_pipeline_stages_are_refused_under_tensor_parallelism(B):
+    s = shape_of("ladder")
+    w = synth.make_weights(s, device="cuda")
+    model = B.Model(w, 2, 32, 32)
+    model.set_exchange(lambda ptr, count, stream: 0)
+    cache = B.KVCache(s, 2, 32)
+    tok = torch.zeros(2, 4, dtype=torch.int32, device="cuda")
+    x0 = torch.zeros(2 * 4, s.d_model, device="cuda")
+    x1 = torch.zeros(2 * 4, s.d_model, device="cuda")
+    with pytest.raises(B.LadderError) as e:
+        model.stage_prefill(cache, tok, 2, 4, None, (x0, x1))
+    assert e.value.status == 2
+    model.set_exchange(None)
+    model.stage_prefill(cache, tok, 2, 4, None, (x0, x1))
+    torch.cuda.synchronize()
+    model.close()

@@ -196,7 +196,8 @@ def workload_config(shape, args):
             "batch": shape.batch, "prompt_len": shape.prompt_len, "decode_steps": args.steps,
             "prefill_chunk": getattr(args, "prefill_chunk", 0) or shape.prompt_len,
             "l2": "inputs larger than L2 (every step streams all weights, far above 126 MB)",
-            "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU"}
+            "parallelism": (f"tensor parallel x{args.gpus} (this line's shape is one rank's slice)" if getattr(args, "tp", False)
+                            else f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU")}
 
 
 def parse_args(argv=None):
@@ -222,6 +223,10 @@ def parse_args(argv=None):
     ap.add_argument("--sm-split", type=int, default=None,
                     help="one kernel per GEMM: SMs for the attention module's GEMMs, the rest for the MLP's "
                          "(-2 = every GEMM on all SMs, -1 = the library's choice, 0 = by bytes)")
+    ap.add_argument("--tp", action="store_true",
+                    help="tensor parallelism over the --gpus ranks (Sec. 2, Eq. 1): every rank holds its slice of the "
+                         "configuration and the modules' partial sums are all-reduced over NCCL; one model, so the "
+                         "value is batch x steps / time (strong scaling).  With one GPU: a world of one")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill-timing", action="store_true")
     ap.add_argument("--no-other-configs", action="store_true",
@@ -461,6 +466,11 @@ def run_rank(args, rank, world):
     B.lib()
 
     shape = shape_for(args, synth)
+    comm = None
+    if args.tp:       # this rank's slice; timing only, so the slice is generated directly (same shapes, own seeds)
+        from paper_2501_06589_b200 import tensor_parallel as TP
+        shape = TP.rank_shape(shape, world)
+        comm = TP.make_comm()
     steps, warm = args.steps, max(args.warmup, 0)
     S, bsz = shape.prompt_len, shape.batch
     hbm_peak, bf16_peak, peak_src = measured_peaks()
@@ -473,6 +483,9 @@ def run_rank(args, rank, world):
     B.set_prefill_gemm_impl(args.prefill_impl)
     run = DecodeRun(B, torch, synth, shape, w, steps, warm, args, dist, local)
     model, cache = run.model, run.cache
+    if comm is not None:
+        model.set_tensor_parallel(comm)
+        run.persistent = False
     persistent = run.persistent
 
     # ---- prefill: once untimed (warm-up), once timed
@@ -529,8 +542,9 @@ def run_rank(args, rank, world):
 
     prefill_ms_max = max_over_ranks([prefill_ms or 0.0], dist, "cuda")[0]
     ms_per_step = dev_ms / steps
-    value = aggregate_rate(world, bsz, steps, dev_ms)
-    e2e_value = aggregate_rate(world, bsz, steps, e2e_ms)
+    jobs = 1 if args.tp else world          # tensor parallelism: ONE model over all ranks
+    value = aggregate_rate(jobs, bsz, steps, dev_ms)
+    e2e_value = aggregate_rate(jobs, bsz, steps, e2e_ms)
     mean_kv = S + (steps + 1) / 2.0
     step_bytes = shape.decode_step_bytes(mean_kv)
     step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
@@ -543,7 +557,7 @@ def run_rank(args, rank, world):
     traffic = ncu_traffic()
     line = {
         "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps,
-        "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if args.tp else "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(shape, args),
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": 4 * bsz, "d2h_bytes_per_step": 4 * bsz,
                 "repeat_ms": [round(x, 3) for x in e2e_recs]},
@@ -563,9 +577,12 @@ def run_rank(args, rank, world):
         "schedule": {"persistent": persistent, "streams": args.streams, "graph": args.graph, "pdl": args.pdl},
         "weights_gb": w.nbytes() / 1e9, "weight_gen_s": t_gen,
     }
+    if args.tp:
+        line["tensor_parallel"] = {"world": world, "exchange": "NCCL all-reduce of fp32 [rows, d_model] partial sums, "
+                                   "one per module, on the producing module's stream (decode) / a stream of its own (prompt pass)"}
     if prefill_ms_max:
         flops = prefill_flops(shape, bsz, S)
-        line["prefill"] = {"tokens_per_s": world * bsz * S / (prefill_ms_max * 1e-3), "ms": prefill_ms_max,
+        line["prefill"] = {"tokens_per_s": jobs * bsz * S / (prefill_ms_max * 1e-3), "ms": prefill_ms_max,
                            "tflops": flops / (prefill_ms_max * 1e-3) / 1e12,
                            "frac_of_bf16_peak": flops / (prefill_ms_max * 1e-3) / 1e12 / bf16_peak,
                            "impl": args.prefill_impl,
@@ -585,7 +602,9 @@ def run_rank(args, rank, world):
         line["cpu_baseline"] = cpu_baseline(shape, w, S)
     run.close()
     del run, model, cache
-    if solo and not args.no_other_configs and args.config == "70b" and args.mode is None and not args.standard:
+    if comm is not None:
+        comm.close()
+    if solo and not args.no_other_configs and args.config == "70b" and args.mode is None and not args.standard and not args.tp:
         t0 = time.time()
         others = other_configs(B, torch, synth, args, local, w, shape)
         del w

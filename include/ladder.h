@@ -185,12 +185,15 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
  * on any number of CTAs).  sms_attention_stream: -1 = the library's choice (default): no split, every GEMM on all
  * SMs, which measured fastest everywhere except for batch 5..64 with layers below 300 MB, where 60 of 148 SMs go
  * to the attention stream; -2 = never split; 0 = in proportion to the bytes each module streams; n > 0 = that many
- * SMs (at most half of them) for the attention module's GEMMs and the rest for the MLP's.  Results are bit-identical.
+ * SMs (at most half of them) for the attention module's GEMMs and the rest for the MLP's.  Batch <= 4: results are
+ * bit-identical for every setting.  Batch 5..64: every CTA accumulates one contiguous K range in fp32, so the number
+ * of CTAs a GEMM runs on decides where the sums are cut: settings that give a GEMM different shares differ in
+ * rounding (~1e-4 of the hidden state), each of them reproducible from run to run.
  * Whenever the split is on, batch is 5..64 and every module reads x_{m-2} (all layers ladder), the step also runs
  * in the pending-output form of Algorithm 1: a module's output stays in a buffer of its own and is added to the
  * residual when the next module's input is normalised, so the attention chain and the MLP chain wait for each
  * other's normalised-input kernel only, never for a GEMM.  The additions are the same fp32 additions in the same
- * order.  -3 = the library's choice of split without that form (each output added by its GEMM's epilogue). */
+ * order (bit-identical to -3 on the same shares).  -3 = the library's choice of split without that form (each output added by its GEMM's epilogue). */
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream);
 
 /* Tensor parallelism (paper Sec. 2, Eq. 1: x_i = AllReduce(h_i(x_{i-1})) + x_{i-1}; Sec. 3.1, Eq. 2 and Algorithm 1:

@@ -125,7 +125,8 @@ def test_rank_0_with_the_oracle_as_rank_1(B, variant, batch, streams):
 def test_world_of_one_over_nccl(B, variant, batch):
     """The NCCL exchange in a world of one: the steps run in the pending-output form with an all-reduce after every
     module, inside the captured decode graph.  Bit-identical to the same form with a do-nothing callback enqueued
-    step by step, and - where the default schedule is that form too (all ladder, batch > 4) - to the default."""
+    step by step, and to the ordinary schedule with the residual added in the GEMM epilogues, every GEMM on all SMs
+    (batch > 4: the same kernels on the same grids, so the same bits)."""
     from paper_2501_06589_b200 import tensor_parallel as TP
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     from tests.test_gpu_model import gpu_generate, oracle_teacher_forced
@@ -145,6 +146,8 @@ def test_world_of_one_over_nccl(B, variant, batch):
             model.set_tensor_parallel(comm)
         elif mode == "callback":
             model.set_exchange(lambda ptr, count, stream: 0, capturable=False)
+        else:
+            model.set_sm_split(-2)
         cache = B.KVCache(s, batch, S + steps + 2)
         toks, hids = gpu_generate(B, model, cache, prompt, steps)
         assert model.device_status() == 0
@@ -154,7 +157,7 @@ def test_world_of_one_over_nccl(B, variant, batch):
     t_nccl, h_nccl = run("nccl")
     t_cb, h_cb = run("callback")
     assert np.array_equal(t_nccl, t_cb) and np.array_equal(h_nccl, h_cb)
-    if variant == "ladder" and batch > 4:
+    if batch > 4:
         t_def, h_def = run("default")
         assert np.array_equal(t_nccl, t_def) and np.array_equal(h_nccl, h_def)
     o_toks, o_hids, _ = oracle_teacher_forced(s, w, prompt, t_nccl, np.float64)

@@ -227,6 +227,9 @@ def parse_args(argv=None):
                     help="tensor parallelism over the --gpus ranks (Sec. 2, Eq. 1): every rank holds its slice of the "
                          "configuration and the modules' partial sums are all-reduced over NCCL; one model, so the "
                          "value is batch x steps / time (strong scaling).  With one GPU: a world of one")
+    ap.add_argument("--tp-nccl", action="store_true",
+                    help="with --tp: NCCL for the decode-step exchanges too (default: the library's own kernel over "
+                         "peer memory for decode steps, NCCL for the prompt pass)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill-timing", action="store_true")
     ap.add_argument("--no-other-configs", action="store_true",
@@ -471,6 +474,7 @@ def run_rank(args, rank, world):
         from paper_2501_06589_b200 import tensor_parallel as TP
         shape = TP.rank_shape(shape, world)
         comm = TP.make_comm()
+        peer = None if args.tp_nccl else TP.make_peer(shape.batch * shape.d_model)
     steps, warm = args.steps, max(args.warmup, 0)
     S, bsz = shape.prompt_len, shape.batch
     hbm_peak, bf16_peak, peak_src = measured_peaks()
@@ -484,7 +488,10 @@ def run_rank(args, rank, world):
     run = DecodeRun(B, torch, synth, shape, w, steps, warm, args, dist, local)
     model, cache = run.model, run.cache
     if comm is not None:
-        model.set_tensor_parallel(comm)
+        if peer is not None:
+            model.set_tensor_parallel_peer(comm, peer)
+        else:
+            model.set_tensor_parallel(comm)
         run.persistent = False
     persistent = run.persistent
 
@@ -578,8 +585,11 @@ def run_rank(args, rank, world):
         "weights_gb": w.nbytes() / 1e9, "weight_gen_s": t_gen,
     }
     if args.tp:
-        line["tensor_parallel"] = {"world": world, "exchange": "NCCL all-reduce of fp32 [rows, d_model] partial sums, "
-                                   "one per module, on the producing module's stream (decode) / a stream of its own (prompt pass)"}
+        line["tensor_parallel"] = {"world": world,
+                                   "exchange": "all-reduce of fp32 [rows, d_model] partial sums, one per module, on the "
+                                               "producing module's stream (decode) / a stream of its own (prompt pass)",
+                                   "decode": "NCCL" if peer is None else "one-shot kernel over peer memory",
+                                   "prompt_pass": "NCCL"}
     if prefill_ms_max:
         flops = prefill_flops(shape, bsz, S)
         line["prefill"] = {"tokens_per_s": jobs * bsz * S / (prefill_ms_max * 1e-3), "ms": prefill_ms_max,
@@ -603,6 +613,8 @@ def run_rank(args, rank, world):
     run.close()
     del run, model, cache
     if comm is not None:
+        if peer is not None:
+            peer.close()
         comm.close()
     if solo and not args.no_other_configs and args.config == "70b" and args.mode is None and not args.standard and not args.tp:
         t0 = time.time()

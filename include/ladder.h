@@ -238,6 +238,51 @@ int32_t ladder_comm_rank(const ladder_comm_t* comm);
 ladder_status_t ladder_comm_all_reduce_sum(void* comm, float* partial, int64_t count, void* cuda_stream);
 ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_t* comm);
 
+/* The exchange over peer memory, for the decode step (paper Sec. 2 Eq. 1; messages of batch x d_model fp32): one
+ * kernel per exchange in which every rank stores its partial sum into a receive slot in each peer's memory (plain
+ * stores through the NVLink peer mapping), raises a counter there, waits - bounded, about 0.25 s, then
+ * LADDER_DEV_TIMEOUT in the status word and no sum - for its peers' counters in its own memory and adds the slots in
+ * rank order, so every rank gets the same bits.  Two channels (0: attention modules, 1: MLP modules: the two chains
+ * of a step, each ordered on its own stream) with two receive slots each.
+ * Set-up: every rank calls ladder_peer_create(world <= LADDER_PEER_MAX_WORLD, rank, max_floats >= max_batch x d_model,
+ * a multiple of 4) on its GPU (allocates and clears 1 KiB + 16 x world x max_floats bytes), hands the
+ * LADDER_PEER_HANDLE_BYTES of ladder_peer_export (a CUDA IPC memory handle) to the others, and calls
+ * ladder_peer_connect(peer, r, handle_of_r, NULL) for every other rank r (ranks that are threads of one process pass
+ * ladder_peer_local_base of r's object as same_process_base instead, with peer access between the devices enabled
+ * by the caller).  All ranks must have connected before the first exchange.  ladder_peer_all_reduce_sum enqueues one
+ * exchange on `cuda_stream`: partial[0 .. count) (device, fp32, 16-byte aligned, count a multiple of 4 and at most
+ * max_floats) becomes the sum over the ranks; every rank must enqueue the same sequence of (channel, count).
+ * device_status: a device int32 that receives LADDER_DEV_TIMEOUT, or NULL.  Capturable into a CUDA graph.
+ * ladder_model_set_tensor_parallel_peer(m, comm, peer): decode steps exchange over `peer`, the prompt pass (messages
+ * of hundreds of MB, where NCCL's algorithms are the right ones) over `comm`; LADDER_ERR_INVALID_ARG if the peer
+ * object is too small for max_batch x d_model or not connected.  Both objects stay the caller's.
+ * ladder_peer_probe_write / _read: connectivity check by host copies (rank a writes a word into rank b's memory, b
+ * reads it after a host-side barrier).  ladder_peer_slot / ladder_peer_counter / ladder_peer_ctas_per_exchange expose
+ * where a rank's data lands and how arrivals are counted (each exchange adds ctas_per_exchange to the sender's
+ * counter), so that a test can play an absent rank.
+ * Exercised on one GPU only (a world of one, and a world of two with the other rank's stores made by the test):
+ * the IPC path is covered by the probe between two processes; nothing is claimed about multi-GPU speed. */
+#define LADDER_PEER_MAX_WORLD 8
+#define LADDER_PEER_HANDLE_BYTES 64
+typedef struct ladder_peer ladder_peer_t;
+ladder_status_t ladder_peer_create(int32_t world, int32_t rank, int64_t max_floats, ladder_peer_t** out);
+ladder_status_t ladder_peer_export(const ladder_peer_t* peer, void* handle);
+void* ladder_peer_local_base(const ladder_peer_t* peer);
+ladder_status_t ladder_peer_connect(ladder_peer_t* peer, int32_t r, const void* ipc_handle, void* same_process_base);
+int32_t ladder_peer_connected(const ladder_peer_t* peer);
+int32_t ladder_peer_world(const ladder_peer_t* peer);
+int32_t ladder_peer_rank(const ladder_peer_t* peer);
+int64_t ladder_peer_max_floats(const ladder_peer_t* peer);
+int32_t ladder_peer_ctas_per_exchange(void);
+ladder_status_t ladder_peer_destroy(ladder_peer_t* peer);
+ladder_status_t ladder_peer_all_reduce_sum(ladder_peer_t* peer, int32_t channel, float* partial, int64_t count,
+                                           int32_t* device_status, void* cuda_stream);
+ladder_status_t ladder_peer_probe_write(ladder_peer_t* peer, int32_t r, uint32_t value);
+ladder_status_t ladder_peer_probe_read(const ladder_peer_t* peer, int32_t from, uint32_t* value);
+float* ladder_peer_slot(const ladder_peer_t* peer, int32_t channel, int32_t parity, int32_t from);
+uint32_t* ladder_peer_counter(const ladder_peer_t* peer, int32_t channel, int32_t from);
+ladder_status_t ladder_model_set_tensor_parallel_peer(ladder_model_t* m, ladder_comm_t* comm, ladder_peer_t* peer);
+
 /* Prompt pass ("prefill phase", paper Sec. 3.2): the module chain of Eq. 1 / Eq. 2 (in the pending-output form of
  * Algorithm 1 with the all-reduce removed) over all prompt positions at once, causal attention within the prompt.
  * d_tokens int32 [batch, seq_len]; every sequence has the same length.

@@ -29,7 +29,12 @@ EXPORTS = [
     "ladder_op_prefill_gemm_f16", "ladder_op_convert_bf16_f16",
     "ladder_model_set_exchange", "ladder_model_set_tensor_parallel", "ladder_comm_unique_id", "ladder_comm_create",
     "ladder_comm_destroy", "ladder_comm_world", "ladder_comm_rank", "ladder_comm_all_reduce_sum",
+    "ladder_peer_create", "ladder_peer_export", "ladder_peer_local_base", "ladder_peer_connect", "ladder_peer_connected",
+    "ladder_peer_world", "ladder_peer_rank", "ladder_peer_max_floats", "ladder_peer_ctas_per_exchange",
+    "ladder_peer_destroy", "ladder_peer_all_reduce_sum", "ladder_peer_probe_write", "ladder_peer_probe_read",
+    "ladder_peer_slot", "ladder_peer_counter", "ladder_model_set_tensor_parallel_peer",
 ]
+PEER_HANDLE_BYTES = 64                                                           # LADDER_PEER_HANDLE_BYTES
 
 COMM_ID_BYTES = 128                                                              # LADDER_COMM_ID_BYTES
 EXCHANGE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p)   # ladder_exchange_fn
@@ -160,6 +165,22 @@ def lib() -> C.CDLL:
         L.ladder_comm_rank.argtypes = [C.c_void_p]
         L.ladder_comm_rank.restype = C.c_int32
         L.ladder_comm_all_reduce_sum.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
+        L.ladder_peer_create.argtypes = [C.c_int32, C.c_int32, C.c_int64, C.POINTER(C.c_void_p)]
+        L.ladder_peer_export.argtypes = [C.c_void_p, C.c_void_p]
+        L.ladder_peer_local_base.argtypes = [C.c_void_p]
+        L.ladder_peer_local_base.restype = C.c_void_p
+        L.ladder_peer_connect.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        for f in (L.ladder_peer_connected, L.ladder_peer_world, L.ladder_peer_rank):
+            f.argtypes, f.restype = [C.c_void_p], C.c_int32
+        L.ladder_peer_max_floats.argtypes, L.ladder_peer_max_floats.restype = [C.c_void_p], C.c_int64
+        L.ladder_peer_ctas_per_exchange.argtypes, L.ladder_peer_ctas_per_exchange.restype = [], C.c_int32
+        L.ladder_peer_destroy.argtypes = [C.c_void_p]
+        L.ladder_peer_all_reduce_sum.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
+        L.ladder_peer_probe_write.argtypes = [C.c_void_p, C.c_int32, C.c_uint32]
+        L.ladder_peer_probe_read.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_uint32)]
+        L.ladder_peer_slot.argtypes, L.ladder_peer_slot.restype = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32], C.c_void_p
+        L.ladder_peer_counter.argtypes, L.ladder_peer_counter.restype = [C.c_void_p, C.c_int32, C.c_int32], C.c_void_p
+        L.ladder_model_set_tensor_parallel_peer.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -285,6 +306,57 @@ class Comm:
             self.h = None
 
 
+class Peer:
+    """Owns a ladder_peer_t: this rank's receive slots for the exchange over peer memory, and the peers' addresses."""
+
+    def __init__(self, world: int, rank: int, max_floats: int):
+        h = C.c_void_p()
+        _check(lib().ladder_peer_create(world, rank, max_floats, C.byref(h)))
+        self.h, self.world, self.rank, self.max_floats = h, world, rank, max_floats
+
+    def export(self) -> bytes:
+        buf = C.create_string_buffer(PEER_HANDLE_BYTES)
+        _check(lib().ladder_peer_export(self.h, buf))
+        return buf.raw
+
+    def local_base(self) -> int:
+        return lib().ladder_peer_local_base(self.h)
+
+    def connect(self, r: int, ipc_handle: Optional[bytes] = None, same_process_base: Optional[int] = None):
+        buf = C.create_string_buffer(ipc_handle, PEER_HANDLE_BYTES) if ipc_handle is not None else None
+        _check(lib().ladder_peer_connect(self.h, r, buf, same_process_base))
+
+    def connected(self) -> bool:
+        return bool(lib().ladder_peer_connected(self.h))
+
+    @staticmethod
+    def ctas_per_exchange() -> int:
+        return lib().ladder_peer_ctas_per_exchange()
+
+    def all_reduce_sum(self, channel: int, ptr: int, count: int, status_ptr: Optional[int] = None, stream: Optional[int] = None):
+        _check(lib().ladder_peer_all_reduce_sum(self.h, channel, ptr, count, status_ptr,
+                                                _stream() if stream is None else stream))
+
+    def probe_write(self, r: int, value: int):
+        _check(lib().ladder_peer_probe_write(self.h, r, value))
+
+    def probe_read(self, frm: int) -> int:
+        v = C.c_uint32(0)
+        _check(lib().ladder_peer_probe_read(self.h, frm, C.byref(v)))
+        return v.value
+
+    def slot_ptr(self, channel: int, parity: int, frm: int) -> int:
+        return lib().ladder_peer_slot(self.h, channel, parity, frm)
+
+    def counter_ptr(self, channel: int, frm: int) -> int:
+        return lib().ladder_peer_counter(self.h, channel, frm)
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().ladder_peer_destroy(self.h)
+            self.h = None
+
+
 class Model:
     """Owns a ladder_model_t; keeps the borrowed weight tensors alive."""
 
@@ -358,6 +430,11 @@ class Model:
         """This model is one rank's slice; partial sums are all-reduced over `comm` (ladder_model_set_tensor_parallel)."""
         _check(lib().ladder_model_set_tensor_parallel(self.h, comm.h if comm is not None else None), self.h)
         self._comm = comm
+
+    def set_tensor_parallel_peer(self, comm: "Comm", peer: "Peer"):
+        """Decode-step exchanges over peer memory, the prompt pass over NCCL (ladder_model_set_tensor_parallel_peer)."""
+        _check(lib().ladder_model_set_tensor_parallel_peer(self.h, comm.h, peer.h), self.h)
+        self._comm, self._peer = comm, peer
 
     def set_position(self, length: int):
         _check(lib().ladder_set_position(self.h, length), self.h)

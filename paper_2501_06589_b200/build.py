@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libladder.so")
 SOURCES = ["api.cu", "decode_gemm.cu", "decode_stack.cu", "decode_gemm_wide_tc.cu", "decode_attention.cu", "decode_attention_tc.cu", "prefill_gemm_tc.cu", "prefill_attention_tc.cu",
-           "misc_kernels.cu", "comm_nccl.cu"]
+           "misc_kernels.cu", "comm_nccl.cu", "peer_exchange.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "--use_fast_math", "-Xptxas", "-v"] + os.environ.get("LADDER_NVCC_EXTRA", "").split()
 

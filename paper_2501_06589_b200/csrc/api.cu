@@ -83,6 +83,7 @@ struct ladder_model {
   void* exchange_ctx = nullptr;
   int exchange_capturable = 0;  // the callback may be called while its stream is being captured into a CUDA graph
   ladder_comm* comm = nullptr;  // set by ladder_model_set_tensor_parallel (not owned)
+  ladder_peer* peer = nullptr;  // decode-step exchanges over peer memory instead of `exchange` (not owned)
   float* pend_pf[2] = {nullptr, nullptr};  // prompt pass under tensor parallelism: the two modules' stored outputs
   cudaStream_t xstream = nullptr;          // ... exchanged and added to the stream on this one
   std::vector<cudaEvent_t> ev_pf_out, ev_pf_add;  // [module]: stored / added
@@ -369,7 +370,9 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
   // The module's output is complete in pend(mod): sum it over the tensor-parallel ranks, tell the other stream.
   auto output_stored = [&](int mod, int s) {
     if (m->exchange) {
-      const ladder_status_t r = m->exchange(m->exchange_ctx, pend(mod), static_cast<int64_t>(batch) * d, q.stream(s));
+      const int64_t n = static_cast<int64_t>(batch) * d;
+      const ladder_status_t r = m->peer ? ladder_peer_all_reduce_sum(m->peer, mod & 1, pend(mod), n, m->status, q.stream(s))
+                                        : m->exchange(m->exchange_ctx, pend(mod), n, q.stream(s));
       if (r != LADDER_OK && q.err == cudaSuccess) q.err = cudaErrorUnknown;
       q.pdl_ok[q.two ? s : 0] = false;
     }
@@ -1531,6 +1534,7 @@ ladder_status_t ladder_model_set_exchange(ladder_model_t* m, ladder_exchange_fn 
   m->exchange_ctx = fn ? ctx : nullptr;
   m->exchange_capturable = (fn && capturable) ? 1 : 0;
   m->comm = nullptr;
+  m->peer = nullptr;
   drop_graph(m);
   return LADDER_OK;
 }
@@ -1540,6 +1544,17 @@ ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_
   if (!comm) return ladder_model_set_exchange(m, nullptr, nullptr, 0);
   const ladder_status_t s = ladder_model_set_exchange(m, ladder_comm_all_reduce_sum, comm, 1);
   if (s == LADDER_OK) m->comm = comm;
+  return s;
+}
+
+ladder_status_t ladder_model_set_tensor_parallel_peer(ladder_model_t* m, ladder_comm_t* comm, ladder_peer_t* peer) {
+  if (!m || !comm || !peer) return LADDER_ERR_INVALID_ARG;
+  if (!ladder_peer_connected(peer) || ladder_peer_world(peer) != ladder_comm_world(comm) ||
+      ladder_peer_rank(peer) != ladder_comm_rank(comm) ||
+      ladder_peer_max_floats(peer) < static_cast<int64_t>(m->cfg.max_batch) * m->cfg.d_model)
+    return fail(m, LADDER_ERR_INVALID_ARG, "peer object not connected, of another world, or smaller than max_batch x d_model");
+  const ladder_status_t s = ladder_model_set_tensor_parallel(m, comm);
+  if (s == LADDER_OK) m->peer = peer;
   return s;
 }
 

@@ -17,7 +17,7 @@ from typing import Optional
 
 import torch
 
-from .binding import Comm
+from .binding import Comm, Peer
 from .synth import AbiWeights, ModelShape
 
 
@@ -67,3 +67,21 @@ def make_comm(group=None) -> Comm:
     box = [Comm.unique_id() if rank == 0 else None]
     dist.broadcast_object_list(box, src=dist.get_global_rank(group, 0) if group is not None else 0, group=group)
     return Comm(world, rank, box[0])
+
+
+def make_peer(max_floats: int, group=None) -> Peer:
+    """This rank's object for the exchange over peer memory, connected to every other rank of the group (one process
+    per GPU: the CUDA IPC handles travel through torch.distributed).  max_floats >= max_batch x d_model, a multiple
+    of 4.  Collective; ends with a barrier, so every rank is connected when it returns."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return Peer(1, 0, max_floats)
+    world, rank = dist.get_world_size(group), dist.get_rank(group)
+    peer = Peer(world, rank, max_floats)
+    handles = [None] * world
+    dist.all_gather_object(handles, peer.export(), group=group)
+    for r in range(world):
+        if r != rank:
+            peer.connect(r, ipc_handle=handles[r])
+    dist.barrier(group=group)
+    return peer

@@ -184,3 +184,117 @@ def test_pipeline_stages_are_refused_under_tensor_parallelism(B):
     model.stage_prefill(cache, tok, 2, 4, None, (x0, x1))
     torch.cuda.synchronize()
     model.close()
+
+
+@pytest.mark.parametrize("variant,batch", [("ladder", 3), ("hybrid", 12)])
+def test_decode_exchange_over_peer_memory_in_a_world_of_one(B, variant, batch):
+    """Decode steps exchange through the peer-memory kernel (inside the captured graph), the prompt pass through
+    NCCL: bit-identical to NCCL for both."""
+    from paper_2501_06589_b200 import tensor_parallel as TP
+    from tests.test_gpu_model import gpu_generate
+    s = shape_of(variant)
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    S, steps = 10, 12
+    prompt = synth.make_tokens(s, batch, S)
+    comm = TP.make_comm()
+    peer = TP.make_peer(batch * s.d_model)
+    runs = []
+    for use_peer in (False, True):
+        model = B.Model(w, batch, S + steps + 2, batch * S)
+        if use_peer:
+            model.set_tensor_parallel_peer(comm, peer)
+        else:
+            model.set_tensor_parallel(comm)
+        cache = B.KVCache(s, batch, S + steps + 2)
+        runs.append(gpu_generate(B, model, cache, prompt, steps))
+        assert model.device_status() == 0
+        model.close()
+    assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1])
+    small = B.Peer(1, 0, 64)
+    model = B.Model(w, batch, 32, 32)
+    with pytest.raises(B.LadderError):
+        model.set_tensor_parallel_peer(comm, small)        # slots smaller than batch x d_model
+    model.close()
+    small.close()
+    peer.close()
+    comm.close()
+
+
+@pytest.mark.parametrize("variant", ["ladder", "standard"])
+def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant):
+    """As test_rank_0_with_the_oracle_as_rank_1, but the decode-step sums are formed by the peer-memory kernel: the
+    callback stores the oracle's rank-1 partial and rank 1's arrivals into rank 0's receive slot, then enqueues the
+    kernel on the same stream (its wait is already satisfied when it starts)."""
+    from paper_2501_06589_b200 import tensor_parallel as TP
+    s = shape_of(variant)
+    world, S, steps, batch = 2, 12, 6, 6
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    prompt = synth.make_tokens(s, batch, S)
+    cfg = oracle_cfg(s, world)
+    OW = O.OracleWeights(provider=synth.logical_provider(w, np.float64))
+    cache_o = O.OracleCache(cfg, batch, S + steps + 1, np.float64)
+    calls, o_toks, o_hids = [], [], []
+    r = O.forward(cfg, OW, prompt, np.float64, cache_o, 0, last_only=True, record=True)
+    for j in range(steps + 1):
+        calls.append([parts[1] for parts in r.module_partials])
+        o_toks.append(r.next_tokens[:, 0])
+        o_hids.append(r.hidden[:, 0])
+        if j < steps:
+            r = O.forward(cfg, OW, o_toks[-1].reshape(-1, 1), np.float64, cache_o, cache_o.seq_len, last_only=True,
+                          record=True)
+
+    n = batch * s.d_model
+    p0, p1 = B.Peer(2, 0, n), B.Peer(2, 1, n)
+    p0.connect(1, same_process_base=p1.local_base())
+    p1.connect(0, same_process_base=p0.local_base())
+    g = B.Peer.ctas_per_exchange()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rw = TP.rank_weights(w, 0, world)
+    model = B.Model(rw, batch, S + steps + 1, batch * S)
+    queue, turns, state = [], [0, 0], {"module": 0}
+
+    def as_floats(ptr, count):
+        return torch.as_tensor(_DeviceFloats(ptr, count), device="cuda")
+
+    class _Word:
+        def __init__(self, ptr):
+            self.__cuda_array_interface__ = {"shape": (1,), "typestr": "<i4", "data": (ptr, False), "version": 2}
+
+    def exchange(ptr, count, stream):
+        peer_part = queue.pop(0)
+        ch = state["module"] & 1
+        state["module"] += 1
+        with torch.cuda.stream(torch.cuda.ExternalStream(stream or 0)):
+            if count != n:                                   # prompt pass: plain add (NCCL's place)
+                as_floats(ptr, count).add_(peer_part)
+                return 0
+            as_floats(p0.slot_ptr(ch, turns[ch] & 1, 1), count).copy_(peer_part)
+            torch.as_tensor(_Word(p0.counter_ptr(ch, 1)), device="cuda").add_(g)
+        p0.all_reduce_sum(ch, ptr, count, status.data_ptr(), stream or 0)
+        turns[ch] += 1
+        return 0
+
+    model.set_exchange(exchange, capturable=False)
+    cache = B.KVCache(rw.shape, batch, S + steps + 1)
+    nxt = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    hid = torch.zeros(batch, s.d_model, device="cuda")
+    hids = []
+    for j in range(steps + 1):
+        queue[:] = [torch.from_numpy(np.ascontiguousarray(p, dtype=np.float32).reshape(-1)).cuda() for p in calls[j]]
+        state["module"] = 0
+        if j == 0:
+            model.prefill(cache, torch.from_numpy(prompt).cuda(), next_tokens=nxt, final_hidden=hid)
+        else:
+            model.decode_step(cache, torch.from_numpy(o_toks[j - 1].astype(np.int32)).cuda(), next_tokens=nxt,
+                              final_hidden=hid)
+        torch.cuda.synchronize()
+        assert not queue
+        hids.append(hid.cpu().numpy().copy())
+    assert model.device_status() == 0 and status.item() == 0
+    assert turns == [s.n_layers * steps] * 2
+    err = rel_err(np.stack(hids, 1), np.stack(o_hids, 1))
+    print(f"[tp rank 0 over peer memory / oracle rank 1, {variant}] hidden max-rel-err {err:.3e}")
+    assert err < HIDDEN_TOL, err
+    model.close()
+    p0.close()
+    p1.close()

@@ -253,9 +253,19 @@ ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_
  * exchange on `cuda_stream`: partial[0 .. count) (device, fp32, 16-byte aligned, count a multiple of 4 and at most
  * max_floats) becomes the sum over the ranks; every rank must enqueue the same sequence of (channel, count).
  * device_status: a device int32 that receives LADDER_DEV_TIMEOUT, or NULL.  Capturable into a CUDA graph.
- * ladder_model_set_tensor_parallel_peer(m, comm, peer): decode steps exchange over `peer`, the prompt pass (messages
- * of hundreds of MB, where NCCL's algorithms are the right ones) over `comm`; LADDER_ERR_INVALID_ARG if the peer
- * object is too small for max_batch x d_model or not connected.  Both objects stay the caller's.
+ * Inside a model the exchange is FUSED into the kernels on either side of it, with no kernel of its own: the output /
+ * down projection's epilogue stores every finished tile of the partial sum straight into the receive slot on every
+ * rank (the transfer runs tile by tile under the GEMM) and each of its CTAs counts its arrival on every rank; the
+ * launch that normalises the next reader's input waits (bounded) until every rank's counter has reached this rank's
+ * own and adds the slots in rank order while it forms the residual stream.
+ * ladder_model_set_tensor_parallel_peer(m, comm, peer): decode steps exchange that way over `peer`, the prompt pass
+ * (messages of hundreds of MB, where NCCL's algorithms are the right ones) over `comm`; LADDER_ERR_INVALID_ARG if the
+ * peer object is too small for max_batch x d_model, not connected or of another world.  ladder_model_set_peer(m, peer)
+ * is the second half alone, for a model whose prompt-pass exchange was set with ladder_model_set_exchange
+ * (LADDER_ERR_STATE if none is set); NULL switches back.  Both objects stay the caller's; an object serves either
+ * models or ladder_peer_all_reduce_sum calls, not both (they count arrivals differently).
+ * ladder_debug_set_peer_hook: a function called on the host right after each decode-step output GEMM has been
+ * enqueued (channel, stream), so that a test can enqueue an absent rank's stores there; steps then run ungraphed.
  * ladder_peer_probe_write / _read: connectivity check by host copies (rank a writes a word into rank b's memory, b
  * reads it after a host-side barrier).  ladder_peer_slot / ladder_peer_counter / ladder_peer_ctas_per_exchange expose
  * where a rank's data lands and how arrivals are counted (each exchange adds ctas_per_exchange to the sender's
@@ -282,6 +292,9 @@ ladder_status_t ladder_peer_probe_read(const ladder_peer_t* peer, int32_t from, 
 float* ladder_peer_slot(const ladder_peer_t* peer, int32_t channel, int32_t parity, int32_t from);
 uint32_t* ladder_peer_counter(const ladder_peer_t* peer, int32_t channel, int32_t from);
 ladder_status_t ladder_model_set_tensor_parallel_peer(ladder_model_t* m, ladder_comm_t* comm, ladder_peer_t* peer);
+ladder_status_t ladder_model_set_peer(ladder_model_t* m, ladder_peer_t* peer);
+typedef void (*ladder_peer_hook_fn)(void* ctx, int32_t channel, void* cuda_stream);
+ladder_status_t ladder_debug_set_peer_hook(ladder_model_t* m, ladder_peer_hook_fn fn, void* ctx);
 
 /* Prompt pass ("prefill phase", paper Sec. 3.2): the module chain of Eq. 1 / Eq. 2 (in the pending-output form of
  * Algorithm 1 with the all-reduce removed) over all prompt positions at once, causal attention within the prompt.

@@ -32,8 +32,10 @@ EXPORTS = [
     "ladder_peer_create", "ladder_peer_export", "ladder_peer_local_base", "ladder_peer_connect", "ladder_peer_connected",
     "ladder_peer_world", "ladder_peer_rank", "ladder_peer_max_floats", "ladder_peer_ctas_per_exchange",
     "ladder_peer_destroy", "ladder_peer_all_reduce_sum", "ladder_peer_probe_write", "ladder_peer_probe_read",
-    "ladder_peer_slot", "ladder_peer_counter", "ladder_model_set_tensor_parallel_peer",
+    "ladder_peer_slot", "ladder_peer_counter", "ladder_model_set_tensor_parallel_peer", "ladder_model_set_peer",
+    "ladder_debug_set_peer_hook",
 ]
+PEER_HOOK_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_int32, C.c_void_p)                # ladder_peer_hook_fn
 PEER_HANDLE_BYTES = 64                                                           # LADDER_PEER_HANDLE_BYTES
 
 COMM_ID_BYTES = 128                                                              # LADDER_COMM_ID_BYTES
@@ -181,6 +183,8 @@ def lib() -> C.CDLL:
         L.ladder_peer_slot.argtypes, L.ladder_peer_slot.restype = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32], C.c_void_p
         L.ladder_peer_counter.argtypes, L.ladder_peer_counter.restype = [C.c_void_p, C.c_int32, C.c_int32], C.c_void_p
         L.ladder_model_set_tensor_parallel_peer.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ladder_model_set_peer.argtypes = [C.c_void_p, C.c_void_p]
+        L.ladder_debug_set_peer_hook.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -435,6 +439,29 @@ class Model:
         """Decode-step exchanges over peer memory, the prompt pass over NCCL (ladder_model_set_tensor_parallel_peer)."""
         _check(lib().ladder_model_set_tensor_parallel_peer(self.h, comm.h, peer.h), self.h)
         self._comm, self._peer = comm, peer
+
+    def set_peer(self, peer: Optional["Peer"]):
+        """Decode-step exchanges fused into the GEMM epilogues over `peer` (ladder_model_set_peer)."""
+        _check(lib().ladder_model_set_peer(self.h, peer.h if peer is not None else None), self.h)
+        self._peer = peer
+
+    def debug_set_peer_hook(self, fn=None):
+        """fn(channel, cuda_stream), called after each decode-step output GEMM has been enqueued (tests)."""
+        if fn is None:
+            _check(lib().ladder_debug_set_peer_hook(self.h, None, None), self.h)
+            self._peer_hook = None
+            return
+
+        def thunk(_ctx, channel, stream):
+            try:
+                fn(channel, stream)
+            except Exception:
+                import traceback
+                traceback.print_exc()
+
+        cb = PEER_HOOK_FN(thunk)
+        _check(lib().ladder_debug_set_peer_hook(self.h, C.cast(cb, C.c_void_p), None), self.h)
+        self._peer_hook = cb
 
     def set_position(self, length: int):
         _check(lib().ladder_set_position(self.h, length), self.h)

@@ -84,6 +84,8 @@ struct ladder_model {
   int exchange_capturable = 0;  // the callback may be called while its stream is being captured into a CUDA graph
   ladder_comm* comm = nullptr;  // set by ladder_model_set_tensor_parallel (not owned)
   ladder_peer* peer = nullptr;  // decode-step exchanges over peer memory instead of `exchange` (not owned)
+  ladder_peer_hook_fn peer_hook = nullptr;  // test hook: called after each output GEMM of a decode step is enqueued
+  void* peer_hook_ctx = nullptr;
   float* pend_pf[2] = {nullptr, nullptr};  // prompt pass under tensor parallelism: the two modules' stored outputs
   cudaStream_t xstream = nullptr;          // ... exchanged and added to the stream on this one
   std::vector<cudaEvent_t> ev_pf_out, ev_pf_add;  // [module]: stored / added
@@ -341,6 +343,8 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
   q.force_wide = batch <= 4;
   const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff, L = c.n_layers;
   const size_t layer_elems = static_cast<size_t>(c.max_batch) * Hkv * c.max_seq_len * Dh;
+  PeerView view = {};
+  const bool use_peer = m->peer != nullptr && peer_view(m->peer, &view);
   Router rt;
   q.launched(0, begin_stream(m, rt, d_tokens, batch, sA));
   int cur = rt.cur;  // R[cur]: the newest stream value formed so far = x_0 + outputs of modules 0 .. added
@@ -355,8 +359,16 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
       if ((j & 1) != s) q.wait(s, m->ev_out[j]);  // a stored output of the other stream (same stream: in order)
     const int n = upto - added;                   // 0, 1 or 2
     p.act = m->R[cur];
-    p.act_pending = n >= 1 ? pend(added + 1) : nullptr;
-    p.act_pending2 = n >= 2 ? pend(added + 2) : nullptr;
+    WidePeer pull = {};
+    if (use_peer) {  // the stored outputs are the ranks' partial sums in this rank's receive slots
+      pull.peer = view;
+      pull.pull_channel[0] = n >= 1 ? ((added + 1) & 1) + 1 : 0;
+      pull.pull_channel[1] = n >= 2 ? ((added + 2) & 1) + 1 : 0;
+      p.wide_peer = &pull;
+    } else {
+      p.act_pending = n >= 1 ? pend(added + 1) : nullptr;
+      p.act_pending2 = n >= 2 ? pend(added + 2) : nullptr;
+    }
     p.act_sum_out = n >= 1 ? m->R[cur ^ 1] : nullptr;
     p.scratch = m->gemm_scratch[q.two ? s : 0];
     p.status = m->status;
@@ -366,19 +378,25 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
     added = upto;
     q.record(s, ev_stage(mod));
     p.wide_prestaged = 1;
+    p.wide_peer = nullptr;
   };
   // The module's output is complete in pend(mod): sum it over the tensor-parallel ranks, tell the other stream.
   auto output_stored = [&](int mod, int s) {
-    if (m->exchange) {
+    if (use_peer) {  // the GEMM itself has pushed the partial sum to every rank
+      if (m->peer_hook) {
+        m->peer_hook(m->peer_hook_ctx, mod & 1, q.stream(s));
+        q.pdl_ok[q.two ? s : 0] = false;
+      }
+    } else if (m->exchange) {
       const int64_t n = static_cast<int64_t>(batch) * d;
-      const ladder_status_t r = m->peer ? ladder_peer_all_reduce_sum(m->peer, mod & 1, pend(mod), n, m->status, q.stream(s))
-                                        : m->exchange(m->exchange_ctx, pend(mod), n, q.stream(s));
+      const ladder_status_t r = m->exchange(m->exchange_ctx, pend(mod), n, q.stream(s));
       if (r != LADDER_OK && q.err == cudaSuccess) q.err = cudaErrorUnknown;
       q.pdl_ok[q.two ? s : 0] = false;
     }
     q.record(s, m->ev_out[mod]);
   };
   for (int l = 0; l < L; ++l) {
+    const bool side = m->stale[2 * l + 1] != 0;  // the two modules of this layer can run side by side
     {  // ---------------- attention module (stream A)
       const int mod = 2 * l, s = 0;
       SmallMParams p = {};
@@ -400,7 +418,7 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
       p.qkv.n_kv_heads = Hkv;
       p.qkv.head_dim = Dh;
       p.qkv.max_seq_len = c.max_seq_len;
-      q.gemm(s, p, true);
+      q.gemm(s, p, side);
 
       DecodeAttnParams a = {};
       a.q = m->q_f32;
@@ -433,7 +451,13 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
       o.epi_mode = EPI_PLAIN;
       o.out = pend(mod);
       o.act_staged = m->wide_opack;
-      q.gemm(s, o, true);
+      WidePeer push = {};
+      if (use_peer) {
+        push.peer = view;
+        push.push_channel = (mod & 1) + 1;
+        o.wide_peer = &push;
+      }
+      q.gemm(s, o, side);
       output_stored(mod, s);
     }
     {  // ---------------- MLP module (stream B)
@@ -450,7 +474,7 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
       g.epi_mode = EPI_SWIGLU;
       g.out = m->h_dec;
       g.wide_pack_out = m->wide_hpack;
-      q.gemm(s, g, true);
+      q.gemm(s, g, side);
 
       SmallMParams dn = {};
       dn.W = m->w_down[l];
@@ -462,7 +486,13 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
       dn.epi_mode = EPI_PLAIN;
       dn.out = pend(mod);
       dn.act_staged = m->wide_hpack;
-      q.gemm(s, dn, true);
+      WidePeer push = {};
+      if (use_peer) {
+        push.peer = view;
+        push.push_channel = (mod & 1) + 1;
+        dn.wide_peer = &push;
+      }
+      q.gemm(s, dn, side);
       output_stored(mod, s);
     }
   }
@@ -509,11 +539,6 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   // two launches side by side overlap those costs: 60 of 148 SMs for the attention stream measured 581 -> 553 us per
   // 8 layers at batch 16 and 921 -> 865 us at batch 64 (at the 70B shape the split loses at every batch).
   const double layer_bytes = 2.0 * (static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh + 3.0 * F * d);
-  if (m->exchange) {  // tensor parallelism: the pending-output form at every batch size, all SMs per GEMM unless told otherwise
-    const bool split = sA != sB && m->sms_a > 0;
-    return enqueue_decode_pending(m, cache, d_tokens, batch, out, sA, sB, n_kernels, split ? m->sms_a : 0,
-                                  split ? m->sm_count - m->sms_a : 0);
-  }
   const bool auto_wide = (m->sms_a == -1 || m->sms_a == -3) && batch > 4 && layer_bytes < 300e6;
   if (q.two && (m->sms_a >= 0 || auto_wide)) {
     int ga = auto_wide ? (60 * m->sm_count + 74) / 148 : m->sms_a;
@@ -530,8 +555,11 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
     bool all_stale = batch > 4 && m->sms_a != -3 && m->pend_a && m->pend_m && !m->st_in.newest && !m->st_out.newest &&
                      (l_end < 0 || l_end == c.n_layers);
     for (size_t i = 0; i < m->stale.size() && all_stale; ++i) all_stale = m->stale[i] != 0;
-    if (all_stale) return enqueue_decode_pending(m, cache, d_tokens, batch, out, sA, sB, n_kernels, q.grid_a, q.grid_b);
+    if (all_stale && !m->exchange)
+      return enqueue_decode_pending(m, cache, d_tokens, batch, out, sA, sB, n_kernels, q.grid_a, q.grid_b);
   }
+  if (m->exchange)  // tensor parallelism: the pending-output form at every batch size (shares of the SMs as above)
+    return enqueue_decode_pending(m, cache, d_tokens, batch, out, sA, sB, n_kernels, q.grid_a, q.grid_b);
 
   Router rt;
   q.launched(0, begin_stream(m, rt, d_tokens, batch, sA));
@@ -1547,15 +1575,33 @@ ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_
   return s;
 }
 
+ladder_status_t ladder_model_set_peer(ladder_model_t* m, ladder_peer_t* peer) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  if (peer) {
+    if (!m->exchange) return fail(m, LADDER_ERR_STATE, "set the exchange of the prompt pass first");
+    if (!ladder_peer_connected(peer) ||
+        ladder_peer_max_floats(peer) < static_cast<int64_t>(m->cfg.max_batch) * m->cfg.d_model)
+      return fail(m, LADDER_ERR_INVALID_ARG, "peer object not connected, or smaller than max_batch x d_model");
+  }
+  m->peer = peer;
+  drop_graph(m);
+  return LADDER_OK;
+}
+
 ladder_status_t ladder_model_set_tensor_parallel_peer(ladder_model_t* m, ladder_comm_t* comm, ladder_peer_t* peer) {
   if (!m || !comm || !peer) return LADDER_ERR_INVALID_ARG;
-  if (!ladder_peer_connected(peer) || ladder_peer_world(peer) != ladder_comm_world(comm) ||
-      ladder_peer_rank(peer) != ladder_comm_rank(comm) ||
-      ladder_peer_max_floats(peer) < static_cast<int64_t>(m->cfg.max_batch) * m->cfg.d_model)
-    return fail(m, LADDER_ERR_INVALID_ARG, "peer object not connected, of another world, or smaller than max_batch x d_model");
+  if (ladder_peer_world(peer) != ladder_comm_world(comm) || ladder_peer_rank(peer) != ladder_comm_rank(comm))
+    return fail(m, LADDER_ERR_INVALID_ARG, "peer object and communicator of different worlds");
   const ladder_status_t s = ladder_model_set_tensor_parallel(m, comm);
-  if (s == LADDER_OK) m->peer = peer;
-  return s;
+  return s == LADDER_OK ? ladder_model_set_peer(m, peer) : s;
+}
+
+ladder_status_t ladder_debug_set_peer_hook(ladder_model_t* m, ladder_peer_hook_fn fn, void* ctx) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  m->peer_hook = fn;
+  m->peer_hook_ctx = fn ? ctx : nullptr;
+  drop_graph(m);
+  return LADDER_OK;
 }
 
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream) {
@@ -1832,7 +1878,8 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
     }
   }
 
-  if (!m->use_graph || (m->exchange && !m->exchange_capturable)) {
+  // a graph only if everything the step calls back into may be captured (with a peer object the step calls nothing)
+  if (!m->use_graph || (m->exchange && !m->peer && !m->exchange_capturable) || (m->peer && m->peer_hook)) {
     int64_t k = 0;
     if (two) {
       // the side stream may only start after everything already queued on the caller's stream

@@ -57,6 +57,7 @@ struct WideArgs {
   int n_slices;
   float* partial;          // [grid][2][bp][128]
   int32_t* tickets;        // [tiles], zero between launches
+  WidePeer wp;             // push_channel != 0: the output goes to the peers' receive slots
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -127,14 +128,68 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 // One CTA per (padded batch row, 2048-wide K slice): y = x (* gain), hi = bf16(y), lo = bf16(y - hi); rows
 // >= batch are zero.  The slice's sum of squares goes to ssq[row][slice]; the GEMM adds the slices in order.
 constexpr int kStageSlice = 2048;
+// A pending that is pulled (tensor parallelism over peer memory): the sum over the ranks, in rank order, of this rank's
+// receive slots [channel][turn & 1][0 .. world), valid once every rank's arrival counter has reached this rank's own
+// (its own output GEMM is complete when this kernel runs, so that counter is final).
+struct StagePull {
+  PeerView peer;
+  int channel[2];  // channel + 1 of pending / pending2, 0 = not pulled
+  int32_t* status;
+};
+
+__device__ __forceinline__ float4 pull_sum(const StagePull& pl, int ch, int parity, size_t off) {
+  unsigned char* base = pl.peer.base[pl.peer.rank];
+  float4 s = __ldcg(reinterpret_cast<const float4*>(peer_slot(base, pl.peer.world, pl.peer.max_floats, ch, parity, 0) + off));
+  for (int r = 1; r < pl.peer.world; ++r) {
+    const float4 v =
+        __ldcg(reinterpret_cast<const float4*>(peer_slot(base, pl.peer.world, pl.peer.max_floats, ch, parity, r) + off));
+    s.x += v.x, s.y += v.y, s.z += v.z, s.w += v.w;
+  }
+  return s;
+}
+
 __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const __nv_bfloat16* gain, int norm, int batch,
                                                          int bp, int K, __nv_bfloat16* stage, float* ssq_out,
                                                          const float* pending, const float* pending2,
-                                                         float* sum_out) {
+                                                         float* sum_out, const StagePull pl) {
   __shared__ float red[8];
+  __shared__ int pull_par[2];
+  __shared__ int pull_fail;
   const int b = blockIdx.x, slice = blockIdx.y, tid = threadIdx.x;
   pdl_launch_dependents();
   pdl_wait();
+  const bool pulls = pl.peer.world > 0 && (pl.channel[0] | pl.channel[1]);
+  if (pulls) {
+    PeerHeader* hdr = peer_header(pl.peer.base[pl.peer.rank]);
+    if (tid == 0) pull_fail = 0;
+    __syncthreads();
+    for (int i = 0; i < 2; ++i) {
+      if (!pl.channel[i]) continue;
+      const int ch = pl.channel[i] - 1;
+      if (tid == 0) pull_par[i] = *reinterpret_cast<volatile uint32_t*>(&hdr->turn[ch]) & 1;
+      if (tid < pl.peer.world) {
+        const uint32_t target = peer_ld_acquire_sys(&hdr->arrive[ch][pl.peer.rank]);
+        const uint32_t* c = &hdr->arrive[ch][tid];
+        bool ok = static_cast<int32_t>(peer_ld_acquire_sys(c) - target) >= 0;
+        if (!ok) {
+          const uint64_t t0 = global_timer_ns();
+          for (uint32_t it = 1; !ok; ++it) {
+            __nanosleep(32);
+            ok = static_cast<int32_t>(peer_ld_acquire_sys(c) - target) >= 0;
+            if (!ok && (it & 63u) == 0 && global_timer_ns() - t0 > 250000000ull) break;
+          }
+        }
+        if (!ok) {
+          pull_fail = 1;
+          if (pl.status) atomicOr(pl.status, LADDER_DEV_TIMEOUT);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  const bool pull0 = pulls && pl.channel[0] && !pull_fail, pull1 = pulls && pl.channel[1] && !pull_fail;
+  if (pulls && pl.channel[0]) pending = nullptr;   // a pulled pending has no plain buffer
+  if (pulls && pl.channel[1]) pending2 = nullptr;
   __nv_bfloat16* hi = stage + static_cast<size_t>(b) * K;
   __nv_bfloat16* lo = stage + static_cast<size_t>(bp + b) * K;
   float ssq = 0.f;
@@ -145,9 +200,19 @@ __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const _
       const float4 a = __ldcg(reinterpret_cast<const float4*>(x + static_cast<size_t>(b) * K + k));
       const float4 c = __ldcg(reinterpret_cast<const float4*>(x + static_cast<size_t>(b) * K + k + 4));
       y[0] = a.x, y[1] = a.y, y[2] = a.z, y[3] = a.w, y[4] = c.x, y[5] = c.y, y[6] = c.z, y[7] = c.w;
+      if (pull0) {  // ... the module output summed over the tensor-parallel ranks
+        const size_t off = static_cast<size_t>(b) * K + k;
+        const float4 pa = pull_sum(pl, pl.channel[0] - 1, pull_par[0], off), pc = pull_sum(pl, pl.channel[0] - 1, pull_par[0], off + 4);
+        y[0] += pa.x, y[1] += pa.y, y[2] += pa.z, y[3] += pa.w, y[4] += pc.x, y[5] += pc.y, y[6] += pc.z, y[7] += pc.w;
+      }
       if (pending) {  // x_m = x_{m-1} + (the module output stored by an earlier GEMM)
         const float4 pa = __ldcg(reinterpret_cast<const float4*>(pending + static_cast<size_t>(b) * K + k));
         const float4 pc = __ldcg(reinterpret_cast<const float4*>(pending + static_cast<size_t>(b) * K + k + 4));
+        y[0] += pa.x, y[1] += pa.y, y[2] += pa.z, y[3] += pa.w, y[4] += pc.x, y[5] += pc.y, y[6] += pc.z, y[7] += pc.w;
+      }
+      if (pull1) {
+        const size_t off = static_cast<size_t>(b) * K + k;
+        const float4 pa = pull_sum(pl, pl.channel[1] - 1, pull_par[1], off), pc = pull_sum(pl, pl.channel[1] - 1, pull_par[1], off + 4);
         y[0] += pa.x, y[1] += pa.y, y[2] += pa.z, y[3] += pa.w, y[4] += pc.x, y[5] += pc.y, y[6] += pc.z, y[7] += pc.w;
       }
       if (pending2) {  // ... and the one after it
@@ -183,6 +248,17 @@ __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const _
     float t = 0.f;
     for (int w = 0; w < 8; ++w) t += red[w];
     ssq_out[b * gridDim.y + slice] = t;
+    if (pulls) {  // the last CTA of the launch moves the pulled channels on (their other receive slot is next)
+      PeerHeader* hdr = peer_header(pl.peer.base[pl.peer.rank]);
+      const int first = (pl.channel[0] ? pl.channel[0] : pl.channel[1]) - 1;
+      __threadfence();
+      if (atomicAdd(&hdr->ticket[first], 1u) == gridDim.x * gridDim.y - 1) {
+        hdr->ticket[first] = 0;
+        for (int i = 0; i < 2; ++i)
+          if (pl.channel[i]) hdr->turn[pl.channel[i] - 1] += 1u;
+        __threadfence();
+      }
+    }
   }
 }
 
@@ -219,11 +295,25 @@ __device__ __forceinline__ void epi_prefetch(const SmallMParams& p, int n, int b
 }
 
 // v[j] = finished accumulator of row n and batch row b0 + j.
-template <int CB>
+template <int CB, bool PUSH>
 __device__ __forceinline__ void epi_apply(const SmallMParams& p, int n, int b0, float (&v)[CB], int lane,
-                                          const int* pos_s, const float (&pa)[CB], const float (&pb)[CB], int bp) {
+                                          const int* pos_s, const float (&pa)[CB], const float (&pb)[CB], int bp,
+                                          const WidePeer& wp, const size_t* push_off_s) {
   const bool row_ok = n < p.N;
-  if (p.epi_mode == EPI_RESID || p.epi_mode == EPI_PLAIN) {
+  if (PUSH) {
+    // tensor parallelism over peer memory (EPI_PLAIN only): this rank's partial sum goes straight into its receive
+    // slot on every rank (lanes hold consecutive rows: 128-byte segments per batch row and peer)
+    const size_t off = *push_off_s;
+#pragma unroll 1
+    for (int w = 0; w < wp.peer.world; ++w) {
+      float* out = reinterpret_cast<float*>(wp.peer.base[w] + kPeerHeaderBytes) + off;
+#pragma unroll
+      for (int j = 0; j < CB; ++j) {
+        const int b = b0 + j;
+        if (b < p.batch && row_ok) out[static_cast<size_t>(b) * p.N + n] = v[j];
+      }
+    }
+  } else if (p.epi_mode == EPI_RESID || p.epi_mode == EPI_PLAIN) {
     float* out = static_cast<float*>(p.out);
 #pragma unroll
     for (int j = 0; j < CB; ++j) {
@@ -302,7 +392,7 @@ struct Split {
   }
 };
 
-template <int NP>
+template <int NP, bool PUSH>
 __global__ void __launch_bounds__(kWideThreads, 1)
 decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap map_w,
                            const __grid_constant__ CUtensorMap map_act) {
@@ -319,6 +409,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
   uint64_t* tmem_empty = tmem_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
   volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  size_t* push_off_s = reinterpret_cast<size_t*>(tmem_slot + 2);  // element offset of the receive slot pushed into
   float* rstd_s = reinterpret_cast<float*>(smem + C::OFF_BARS + (2 * STAGES + 4) * 8 + 64);  // [BP] 1/rms
   int* pos_s = reinterpret_cast<int*>(rstd_s + 64);                                            // [BP] positions
 
@@ -438,6 +529,13 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
       const int b = et - 128;
       pos_s[b] = (p.epi_mode == EPI_QKV_ROPE && b < p.batch) ? p.qkv.seq_lens[b] : -1;
     }
+    // receive-slot parity of this exchange: the channel was last moved on by a staging launch that lies before
+    // this kernel's predecessors in stream order
+    if (PUSH && et == 255) {  // receive slot [channel][turn & 1][this rank]: the same offset on every rank
+      const int ch = a.wp.push_channel - 1;
+      const uint32_t turn = *reinterpret_cast<volatile uint32_t*>(&peer_header(a.wp.peer.base[a.wp.peer.rank])->turn[ch]);
+      *push_off_s = ((static_cast<size_t>(ch) * 2 + (turn & 1u)) * a.wp.peer.world + a.wp.peer.rank) * a.wp.peer.max_floats;
+    }
     asm volatile("bar.sync 1, 256;" ::: "memory");
     for (int pos = my_start; pos < my_end; ++seg) {
       const int t = pos / nkb, kb0 = pos - t * nkb, kb1 = min(nkb, kb0 + (my_end - pos));
@@ -489,7 +587,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
 #pragma unroll
             for (int j = 0; j < CB; ++j) v[j] *= rstd_s[b0 + j];
           }
-          epi_apply<CB>(p, n, b0, v, lane, pos_s, pa, pb, BP);
+          epi_apply<CB, PUSH>(p, n, b0, v, lane, pos_s, pa, pb, BP, a.wp, push_off_s);
         } else {
 #pragma unroll
           for (int j = 0; j < CB; j += 4) piece[((b0 + j) >> 2) * 32] = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -551,10 +649,20 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
 #pragma unroll
           for (int j = 0; j < FB; ++j) v[j] *= rstd_s[b0 + j];
         }
-        epi_apply<FB>(p, n, b0, v, lane, pos_s, pa, pb, BP);
+        epi_apply<FB, PUSH>(p, n, b0, v, lane, pos_s, pa, pb, BP, a.wp, push_off_s);
       }
     }
     if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
+    if (PUSH) {  // every CTA of the launch counts its arrival on every rank, its stores before it
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (et == 0 && ok) {
+        __threadfence_system();
+        for (int o = 1; o <= a.wp.peer.world; ++o) {
+          const int w = (a.wp.peer.rank + o) % a.wp.peer.world;
+          peer_red_release_sys_add(&peer_header(a.wp.peer.base[w])->arrive[a.wp.push_channel - 1][a.wp.peer.rank], 1u);
+        }
+      }
+    }
   }
 
   tc_fence_before();
@@ -605,7 +713,18 @@ cudaError_t launch_np(const WideArgs& a, const CUtensorMap& mw, const CUtensorMa
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = pdl_attr ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, decode_gemm_wide_tc_kernel<NP>, a, mw, ma);
+  if (a.wp.push_channel) return cudaLaunchKernelEx(&cfg, decode_gemm_wide_tc_kernel<NP, true>, a, mw, ma);
+  return cudaLaunchKernelEx(&cfg, decode_gemm_wide_tc_kernel<NP, false>, a, mw, ma);
+}
+
+template <int NP>
+cudaError_t allow_smem() {
+  cudaError_t e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<NP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       WCfg<NP>::SMEM);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<NP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             WCfg<NP>::SMEM);
+  return e;
 }
 
 }  // namespace
@@ -622,15 +741,10 @@ cudaError_t smallm_gemm_wide_tc_init() {
     if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
     g_encode_wide = reinterpret_cast<EncodeFn>(fn);
   }
-  cudaError_t e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       WCfg<32>::SMEM);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, WCfg<16>::SMEM);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WCfg<64>::SMEM);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_gemm_wide_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             WCfg<128>::SMEM);
+  cudaError_t e = allow_smem<16>();
+  if (e == cudaSuccess) e = allow_smem<32>();
+  if (e == cudaSuccess) e = allow_smem<64>();
+  if (e == cudaSuccess) e = allow_smem<128>();
   return e;
 }
 
@@ -657,9 +771,18 @@ cudaError_t launch_stage(const SmallMParams& p, int bp, int n_slices, __nv_bfloa
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = pdl ? 1 : 0;
+  StagePull pl = {};
+  if (p.wide_peer && p.wide_peer->peer.world > 0 && (p.wide_peer->pull_channel[0] | p.wide_peer->pull_channel[1])) {
+    const WidePeer& wp = *p.wide_peer;
+    if (wp.pull_channel[0] && wp.pull_channel[0] == wp.pull_channel[1]) return cudaErrorInvalidValue;
+    pl.peer = wp.peer;
+    pl.channel[0] = wp.pull_channel[0];
+    pl.channel[1] = wp.pull_channel[1];
+    pl.status = p.status;
+  }
   return cudaLaunchKernelEx(&cfg, wide_stage_kernel, static_cast<const float*>(p.act), p.gain,
                             p.act_mode == ACT_F32_NORM ? 1 : 0, p.batch, bp, p.K, stage, ssq, p.act_pending,
-                            p.act_pending2, p.act_sum_out);
+                            p.act_pending2, p.act_sum_out, pl);
 }
 }  // namespace
 
@@ -675,6 +798,10 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
   if (!g_encode_wide) return cudaErrorNotReady;
   if (!p.scratch || p.batch < 1 || p.batch > 64 || (p.K & 7) || (p.N & 1)) return cudaErrorInvalidValue;
   if ((reinterpret_cast<uintptr_t>(p.W) | reinterpret_cast<uintptr_t>(p.scratch)) & 15) return cudaErrorMisalignedAddress;
+  const bool push = p.wide_peer && p.wide_peer->push_channel;
+  if (push && (p.epi_mode != EPI_PLAIN || p.wide_peer->peer.world < 1 || p.wide_peer->push_channel > 2 ||
+               static_cast<size_t>(p.batch) * p.N > p.wide_peer->peer.max_floats))
+    return cudaErrorInvalidValue;
   const int bp = padded_batch(p.batch);
   const int tiles = (p.N + BM - 1) / BM, nkb = (p.K + BK - 1) / BK;
   if (tiles > kWideMaxTiles || sm_count > kWideMaxCtas) return cudaErrorInvalidValue;
@@ -705,6 +832,8 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
   a.n_slices = n_slices;
   a.partial = pieces;
   a.tickets = tickets;
+  if (push) a.wp = *p.wide_peer;
+  a.p.wide_peer = nullptr;  // a host address: not for the device
   const int total = tiles * nkb;
   const int grid = total < sm_count ? total : sm_count;
   const bool pdl_attr = (p.act_staged || p.wide_prestaged) ? pdl : true;  // after its own staging kernel always; else if the caller says so

@@ -7,12 +7,31 @@
 #include <stdint.h>
 
 #include "decode_schedule.h"
+#include "peer_layout.cuh"
 
 namespace ladder {
 
 // Element type of the KV cache: IEEE binary16.  Keys and values of a normalised-input projection are O(1), far inside
 // its range, and its 11 significant bits (bf16: 8) are what keeps the hidden-state error of deep models in bound.
 typedef __half kv_t;
+
+// Tensor parallelism over peer memory (tcgen05 decode GEMM and its staging launch; layout in peer_layout.cuh).
+// push_channel = channel + 1 (EPI_PLAIN GEMM): every output element is stored into receive slot
+// [channel][turn & 1][this rank] of EVERY rank instead of p.out, and each CTA counts its arrival on every rank when
+// it is done.  pull_channel[i] = channel + 1 (staging step): pending i is the rank-order sum of this rank's receive
+// slots of that channel, read after the ranks' arrival counters have reached this rank's own (bounded wait); the
+// staging launch then moves the channel on.  act_pending / act_pending2 are ignored for a pulled pending.
+struct WidePeer {
+  PeerView peer;
+  int push_channel;
+  int pull_channel[2];
+};
+
+}  // namespace ladder
+struct ladder_peer;
+namespace ladder {
+// The addresses of a connected peer-exchange object (peer_exchange.cu); false if it is not connected.
+bool peer_view(const ladder_peer* p, PeerView* out);
 
 enum ActMode { ACT_F32 = 0, ACT_F32_NORM = 1 };  // activations are fp32 [batch, K]; NORM applies RMSNorm
 enum EpiMode { EPI_RESID = 0, EPI_SWIGLU = 1, EPI_PLAIN = 2, EPI_QKV_ROPE = 3, EPI_BF16 = 4 };
@@ -63,6 +82,7 @@ struct SmallMParams {
   float* act_sum_out;
   int wide_prestaged;
   int force_wide;
+  const WidePeer* wide_peer;  // tensor parallelism over peer memory (HOST pointer, read while launching), or NULL
   // Optional second copy of an fp32 output (EPI_RESID: out, EPI_SWIGLU: h) as the next GEMM's MMA operand:
   // y = value (* pack_gain[n]), bf16 hi at [n / 2048][b][n % 2048], lo at [n / 2048][4 + b][n % 2048]; batch <= 4.
   __nv_bfloat16* pack_out;

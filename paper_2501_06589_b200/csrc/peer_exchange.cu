@@ -5,13 +5,8 @@
 // for the peers' counters in its own memory and adds the slots in rank order - one kernel, one link crossing, and
 // every rank forms the sum in the same order, so the ranks' residual streams stay bit-identical.
 //
-// Memory of one rank (one allocation, the same layout on every rank, shared with the others through a CUDA IPC
-// handle or - same process - by address):
-//   arrive[channel][rank]   uint32, counts CTAs of `rank` whose data for this channel has landed here (monotonic)
-//   turn[channel]           uint32, exchanges this rank has completed on the channel (slot parity = turn & 1)
-//   ticket[channel]         uint32, CTAs of the running kernel that are done (the last one advances `turn`)
-//   probe[rank]             uint32, connectivity check (host copies only)
-//   rx[channel][parity][rank][max_floats]   the receive slots
+// Memory of one rank: one allocation, the same layout on every rank (peer_layout.cuh), shared with the others
+// through a CUDA IPC handle or - same process - by address.
 // Two channels = the two module chains of a decode step (attention modules, MLP modules): each chain's exchanges are
 // ordered on their own stream on every rank.  Two parities: a rank can start exchange t + 1 of a channel while a peer
 // still adds the slots of exchange t, but it cannot start t + 2 before it has received that peer's part of t + 1,
@@ -27,40 +22,24 @@
 
 #include "../../include/ladder.h"
 #include "common.cuh"
+#include "peer_layout.cuh"
 
 namespace {
 
+using ladder::PeerView;
+using Header = ladder::PeerHeader;
 constexpr int kMaxWorld = LADDER_PEER_MAX_WORLD;
+static_assert(kMaxWorld == ladder::kPeerMaxWorld, "world limit");
 constexpr int kCtas = 16;       // CTAs per exchange kernel: the same on every rank (the counters count them)
 constexpr int kThreads = 512;
-constexpr size_t kHeaderBytes = 1024;
-
-struct Header {
-  uint32_t arrive[2][kMaxWorld];
-  uint32_t turn[2];
-  uint32_t ticket[2];
-  uint32_t probe[kMaxWorld];
-};
-static_assert(sizeof(Header) <= kHeaderBytes, "header size");
-
-struct PeerArgs {
-  unsigned char* base[kMaxWorld];  // every rank's block as seen from this device (base[rank] = the local one)
-  int world, rank;
-  size_t max_floats;
-};
+constexpr size_t kHeaderBytes = ladder::kPeerHeaderBytes;
+using PeerArgs = PeerView;
 
 __device__ __forceinline__ float* slot(unsigned char* base, const PeerArgs& a, int channel, int parity, int from) {
-  return reinterpret_cast<float*>(base + kHeaderBytes) +
-         ((static_cast<size_t>(channel) * 2 + parity) * a.world + from) * a.max_floats;
+  return ladder::peer_slot(base, a.world, a.max_floats, channel, parity, from);
 }
-__device__ __forceinline__ uint32_t ld_acquire_sys(const uint32_t* p) {
-  uint32_t v;
-  asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void red_release_sys_add(uint32_t* p, uint32_t v) {
-  asm volatile("red.release.sys.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
+__device__ __forceinline__ uint32_t ld_acquire_sys(const uint32_t* p) { return ladder::peer_ld_acquire_sys(p); }
+__device__ __forceinline__ void red_release_sys_add(uint32_t* p, uint32_t v) { ladder::peer_red_release_sys_add(p, v); }
 
 // partial[0 .. count) += the other ranks' partials (in place, rank order).  count a multiple of 4.
 __global__ void __launch_bounds__(kThreads) peer_all_reduce_kernel(PeerArgs a, int channel, float* partial, int64_t count,
@@ -153,6 +132,17 @@ bool connected(const ladder_peer* p) {
 Header* header(const ladder_peer* p, int r) { return reinterpret_cast<Header*>(p->base[r]); }
 }  // namespace
 
+namespace ladder {
+bool peer_view(const ladder_peer* p, PeerView* out) {
+  if (!p || !connected(p)) return false;
+  for (int r = 0; r < kPeerMaxWorld; ++r) out->base[r] = r < p->world ? p->base[r] : nullptr;
+  out->world = p->world;
+  out->rank = p->rank;
+  out->max_floats = p->max_floats;
+  return true;
+}
+}  // namespace ladder
+
 extern "C" {
 
 ladder_status_t ladder_peer_create(int32_t world, int32_t rank, int64_t max_floats, ladder_peer_t** out) {
@@ -232,10 +222,7 @@ ladder_status_t ladder_peer_all_reduce_sum(ladder_peer_t* p, int32_t channel, fl
   if (!connected(p)) return LADDER_ERR_STATE;
   if (count == 0) return LADDER_OK;
   PeerArgs a = {};
-  for (int r = 0; r < p->world; ++r) a.base[r] = p->base[r];
-  a.world = p->world;
-  a.rank = p->rank;
-  a.max_floats = p->max_floats;
+  ladder::peer_view(p, &a);
   peer_all_reduce_kernel<<<kCtas, kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(a, channel, partial, count,
                                                                                         device_status);
   return cudaGetLastError() == cudaSuccess ? LADDER_OK : LADDER_ERR_CUDA;

@@ -220,14 +220,17 @@ def test_decode_exchange_over_peer_memory_in_a_world_of_one(B, variant, batch):
     comm.close()
 
 
-@pytest.mark.parametrize("variant", ["ladder", "standard"])
-def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant):
-    """As test_rank_0_with_the_oracle_as_rank_1, but the decode-step sums are formed by the peer-memory kernel: the
-    callback stores the oracle's rank-1 partial and rank 1's arrivals into rank 0's receive slot, then enqueues the
-    kernel on the same stream (its wait is already satisfied when it starts)."""
+@pytest.mark.parametrize("streams", [2, 1])
+@pytest.mark.parametrize("variant,batch", [("ladder", 6), ("standard", 6), ("hybrid", 3), ("ladder", 40)])
+def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, streams):
+    """As test_rank_0_with_the_oracle_as_rank_1, but the decode-step exchange is the fused one: rank 0's output GEMMs
+    push their partial sums into the receive slots (rank 0's own and, on the same GPU, those of a second object that
+    stands for rank 1's memory), and the staging launches wait for the arrival counters and add the slots.  Rank 1's
+    stores - the oracle's rank-1 partial and an arrival count equal to rank 0's - are enqueued by the test right
+    behind each output GEMM, so every wait is already satisfied when its kernel starts."""
     from paper_2501_06589_b200 import tensor_parallel as TP
     s = shape_of(variant)
-    world, S, steps, batch = 2, 12, 6, 6
+    world, S, steps = 2, 12, 6
     w = synth.make_weights(s, device="cuda", gains="uniform")
     prompt = synth.make_tokens(s, batch, S)
     cfg = oracle_cfg(s, world)
@@ -247,41 +250,39 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant):
     p0, p1 = B.Peer(2, 0, n), B.Peer(2, 1, n)
     p0.connect(1, same_process_base=p1.local_base())
     p1.connect(0, same_process_base=p0.local_base())
-    g = B.Peer.ctas_per_exchange()
-    status = torch.zeros(1, dtype=torch.int32, device="cuda")
     rw = TP.rank_weights(w, 0, world)
     model = B.Model(rw, batch, S + steps + 1, batch * S)
-    queue, turns, state = [], [0, 0], {"module": 0}
-
-    def as_floats(ptr, count):
-        return torch.as_tensor(_DeviceFloats(ptr, count), device="cuda")
+    model.set_schedule(streams, True, True)
+    queue, turns = [], [0, 0]
 
     class _Word:
         def __init__(self, ptr):
             self.__cuda_array_interface__ = {"shape": (1,), "typestr": "<i4", "data": (ptr, False), "version": 2}
 
-    def exchange(ptr, count, stream):
-        peer_part = queue.pop(0)
-        ch = state["module"] & 1
-        state["module"] += 1
+    def word(ptr):
+        return torch.as_tensor(_Word(ptr), device="cuda")
+
+    def prompt_exchange(ptr, count, stream):                 # the prompt pass: NCCL's place
         with torch.cuda.stream(torch.cuda.ExternalStream(stream or 0)):
-            if count != n:                                   # prompt pass: plain add (NCCL's place)
-                as_floats(ptr, count).add_(peer_part)
-                return 0
-            as_floats(p0.slot_ptr(ch, turns[ch] & 1, 1), count).copy_(peer_part)
-            torch.as_tensor(_Word(p0.counter_ptr(ch, 1)), device="cuda").add_(g)
-        p0.all_reduce_sum(ch, ptr, count, status.data_ptr(), stream or 0)
-        turns[ch] += 1
+            torch.as_tensor(_DeviceFloats(ptr, count), device="cuda").add_(queue.pop(0))
         return 0
 
-    model.set_exchange(exchange, capturable=False)
+    def rank_1_arrives(channel, stream):                     # a decode-step output GEMM of rank 0 has been enqueued
+        part = queue.pop(0)
+        with torch.cuda.stream(torch.cuda.ExternalStream(stream or 0)):
+            torch.as_tensor(_DeviceFloats(p0.slot_ptr(channel, turns[channel] & 1, 1), n), device="cuda").copy_(part)
+            word(p0.counter_ptr(channel, 1)).copy_(word(p0.counter_ptr(channel, 0)))   # as many arrivals as rank 0's own
+        turns[channel] += 1
+
+    model.set_exchange(prompt_exchange, capturable=False)
+    model.set_peer(p0)
+    model.debug_set_peer_hook(rank_1_arrives)
     cache = B.KVCache(rw.shape, batch, S + steps + 1)
     nxt = torch.zeros(batch, dtype=torch.int32, device="cuda")
     hid = torch.zeros(batch, s.d_model, device="cuda")
     hids = []
     for j in range(steps + 1):
         queue[:] = [torch.from_numpy(np.ascontiguousarray(p, dtype=np.float32).reshape(-1)).cuda() for p in calls[j]]
-        state["module"] = 0
         if j == 0:
             model.prefill(cache, torch.from_numpy(prompt).cuda(), next_tokens=nxt, final_hidden=hid)
         else:
@@ -290,10 +291,17 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant):
         torch.cuda.synchronize()
         assert not queue
         hids.append(hid.cpu().numpy().copy())
-    assert model.device_status() == 0 and status.item() == 0
+    assert model.device_status() == 0
     assert turns == [s.n_layers * steps] * 2
+    # rank 0's partial of the last attention module has landed in "rank 1's" memory too, with the same arrival count
+    last = (turns[0] - 1) & 1
+    mine = torch.as_tensor(_DeviceFloats(p0.slot_ptr(0, last, 0), n), device="cuda")
+    theirs = torch.as_tensor(_DeviceFloats(p1.slot_ptr(0, last, 0), n), device="cuda")
+    assert torch.equal(mine, theirs) and float(mine.abs().max()) > 0
+    assert word(p1.counter_ptr(0, 0)).item() == word(p0.counter_ptr(0, 0)).item() > 0
     err = rel_err(np.stack(hids, 1), np.stack(o_hids, 1))
-    print(f"[tp rank 0 over peer memory / oracle rank 1, {variant}] hidden max-rel-err {err:.3e}")
+    print(f"[tp rank 0, fused exchange over peer memory / oracle rank 1, {variant}, batch {batch}, {streams} stream(s)] "
+          f"hidden max-rel-err {err:.3e}")
     assert err < HIDDEN_TOL, err
     model.close()
     p0.close()

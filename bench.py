@@ -588,7 +588,7 @@ def run_rank(args, rank, world):
         line["tensor_parallel"] = {"world": world,
                                    "exchange": "all-reduce of fp32 [rows, d_model] partial sums, one per module, on the "
                                                "producing module's stream (decode) / a stream of its own (prompt pass)",
-                                   "decode": "NCCL" if peer is None else "one-shot kernel over peer memory",
+                                   "decode": "NCCL" if peer is None else "fused into the GEMM epilogues and the staging launches over peer memory",
                                    "prompt_pass": "NCCL"}
     if prefill_ms_max:
         flops = prefill_flops(shape, bsz, S)

@@ -54,7 +54,7 @@ typedef enum {
 /* Bits of the device status word (ladder_device_status). */
 #define LADDER_DEV_BAD_TOKEN 1      /* a token id was outside [0, vocab): row treated as id 0 */
 #define LADDER_DEV_CACHE_OVERFLOW 2 /* a position >= max_seq_len reached a kernel: store skipped */
-#define LADDER_DEV_TIMEOUT 4        /* a bounded wait inside the persistent decode kernel gave up (0.25 s): that
+#define LADDER_DEV_TIMEOUT 4        /* a bounded wait inside the persistent decode kernel gave up (about 0.3 s): that
                                        step's outputs are invalid; later launches end at once until the word is read */
 
 /* Per-layer architecture (ladder_config_t.layer_mode), paper Sec. 3.3.1. */
@@ -163,7 +163,7 @@ int32_t ladder_model_persistent_active(const ladder_model_t* m);
 
 /* Test hook for the bounded waits of the persistent kernel: with on = 1 the LM-head phase of the next decode
  * steps waits for one more finished unit than its producer phase has, i.e. for a count that is never reached.
- * Nothing faults or spins forever: the wait gives up after 0.25 s, sets the LADDER_DEV_TIMEOUT bit of the
+ * Nothing faults or spins forever: the wait gives up after about 0.3 s, sets the LADDER_DEV_TIMEOUT bit of the
  * device status word, every other wait in the launch gives up as soon as it sees the bit, and the launch ends.
  * Later launches return at once until ladder_device_status has read and cleared the word.  on = 0 restores
  * the real dependency. */
@@ -240,12 +240,12 @@ ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_
 
 /* The exchange over peer memory, for the decode step (paper Sec. 2 Eq. 1; messages of batch x d_model fp32): one
  * kernel per exchange in which every rank stores its partial sum into a receive slot in each peer's memory (plain
- * stores through the NVLink peer mapping), raises a counter there, waits - bounded, about 0.25 s, then
+ * stores through the NVLink peer mapping), raises a counter there, waits - bounded, about 0.3 s, then
  * LADDER_DEV_TIMEOUT in the status word and no sum - for its peers' counters in its own memory and adds the slots in
  * rank order, so every rank gets the same bits.  Two channels (0: attention modules, 1: MLP modules: the two chains
  * of a step, each ordered on its own stream) with two receive slots each.
  * Set-up: every rank calls ladder_peer_create(world <= LADDER_PEER_MAX_WORLD, rank, max_floats >= max_batch x d_model,
- * a multiple of 4) on its GPU (allocates and clears 1 KiB + 16 x world x max_floats bytes), hands the
+ * a multiple of 4) on its GPU (allocates and clears 1 KiB + 32 x world x max_floats bytes), hands the
  * LADDER_PEER_HANDLE_BYTES of ladder_peer_export (a CUDA IPC memory handle) to the others, and calls
  * ladder_peer_connect(peer, r, handle_of_r, NULL) for every other rank r (ranks that are threads of one process pass
  * ladder_peer_local_base of r's object as same_process_base instead, with peer access between the devices enabled
@@ -253,11 +253,13 @@ ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_
  * exchange on `cuda_stream`: partial[0 .. count) (device, fp32, 16-byte aligned, count a multiple of 4 and at most
  * max_floats) becomes the sum over the ranks; every rank must enqueue the same sequence of (channel, count).
  * device_status: a device int32 that receives LADDER_DEV_TIMEOUT, or NULL.  Capturable into a CUDA graph.
- * Inside a model the exchange is FUSED into the kernels on either side of it, with no kernel of its own: the output /
- * down projection's epilogue stores every finished tile of the partial sum straight into the receive slot on every
- * rank (the transfer runs tile by tile under the GEMM) and each of its CTAs counts its arrival on every rank; the
- * launch that normalises the next reader's input waits (bounded) until every rank's counter has reached this rank's
- * own and adds the slots in rank order while it forms the residual stream.
+ * Inside a model the exchange is FUSED into the kernels on either side of it, with no kernel of its own, no counter
+ * and no fence: the output / down projection's epilogue stores every finished element of the partial sum straight
+ * into the receive slot on every rank, together with the sequence number of the exchange in ONE aligned 8-byte store
+ * (the transfer runs tile by tile under the GEMM); the launch that normalises the next reader's input polls
+ * (bounded) each pair it needs until the number is the expected one and adds the slots in rank order while it
+ * forms the residual stream.  This rests on aligned 8-byte stores reaching peer memory whole (as NCCL's
+ * low-latency protocol does).
  * ladder_model_set_tensor_parallel_peer(m, comm, peer): decode steps exchange that way over `peer`, the prompt pass
  * (messages of hundreds of MB, where NCCL's algorithms are the right ones) over `comm`; LADDER_ERR_INVALID_ARG if the
  * peer object is too small for max_batch x d_model, not connected or of another world.  ladder_model_set_peer(m, peer)
@@ -268,8 +270,9 @@ ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_
  * enqueued (channel, stream), so that a test can enqueue an absent rank's stores there; steps then run ungraphed.
  * ladder_peer_probe_write / _read: connectivity check by host copies (rank a writes a word into rank b's memory, b
  * reads it after a host-side barrier).  ladder_peer_slot / ladder_peer_counter / ladder_peer_ctas_per_exchange expose
- * where a rank's data lands and how arrivals are counted (each exchange adds ctas_per_exchange to the sender's
- * counter), so that a test can play an absent rank.
+ * where a rank's data lands (a slot holds max_floats values for ladder_peer_all_reduce_sum, max_floats (value, number)
+ * pairs for the fused exchange) and how the stand-alone kernel counts arrivals (each exchange adds ctas_per_exchange
+ * to the sender's counter), so that a test can play an absent rank.
  * Exercised on one GPU only (a world of one, and a world of two with the other rank's stores made by the test):
  * the IPC path is covered by the probe between two processes; nothing is claimed about multi-GPU speed. */
 #define LADDER_PEER_MAX_WORLD 8

@@ -78,21 +78,21 @@ struct F8 {
 // bounded spin on a shared-memory counter written by another warp of this CTA
 __device__ __forceinline__ bool wait_counter_gt(const volatile int* ctr, int n) {
   if (*ctr > n) return true;
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     if (*ctr > n) return true;
-    if ((i & 255u) == 0 && global_timer_ns() - t0 > 250000000ull) return false;
+    if ((i & 255u) == 0 && clock64() - t0 > kWaitCycles) return false;
   }
 }
 
 // bounded mbarrier wait that also gives up when a shared-memory stop flag goes negative:
 // 0 = phase completed, 1 = stop flag seen, 2 = timed out
 __device__ __forceinline__ int mbar_wait_or_stop(uint64_t* bar, uint32_t parity, const volatile int* stop) {
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return 0;
     if (*stop < 0) return 1;
-    if ((i & 255u) == 0 && global_timer_ns() - t0 > 250000000ull) return 2;
+    if ((i & 255u) == 0 && clock64() - t0 > kWaitCycles) return 2;
   }
 }
 

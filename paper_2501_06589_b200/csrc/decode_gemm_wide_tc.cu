@@ -129,23 +129,53 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 // >= batch are zero.  The slice's sum of squares goes to ssq[row][slice]; the GEMM adds the slices in order.
 constexpr int kStageSlice = 2048;
 // A pending that is pulled (tensor parallelism over peer memory): the sum over the ranks, in rank order, of this rank's
-// receive slots [channel][turn & 1][0 .. world), valid once every rank's arrival counter has reached this rank's own
-// (its own output GEMM is complete when this kernel runs, so that counter is final).
+// receive slots [channel][turn & 1][0 .. world).  Every element there is a (value, sequence number) pair written by
+// one 8-byte store of the rank that produced it; an element has arrived when its number is turn + 1.
 struct StagePull {
   PeerView peer;
   int channel[2];  // channel + 1 of pending / pending2, 0 = not pulled
   int32_t* status;
 };
 
-__device__ __forceinline__ float4 pull_sum(const StagePull& pl, int ch, int parity, size_t off) {
+// y[0 .. 8) += the eight values at element offset `off` of every rank's slot.  Polls (bounded) until they are there;
+// false if the wait ran out.
+__device__ __forceinline__ bool pull_add8(const StagePull& pl, int ch, uint32_t turn, size_t off, float (&y)[8]) {
   unsigned char* base = pl.peer.base[pl.peer.rank];
-  float4 s = __ldcg(reinterpret_cast<const float4*>(peer_slot(base, pl.peer.world, pl.peer.max_floats, ch, parity, 0) + off));
-  for (int r = 1; r < pl.peer.world; ++r) {
-    const float4 v =
-        __ldcg(reinterpret_cast<const float4*>(peer_slot(base, pl.peer.world, pl.peer.max_floats, ch, parity, r) + off));
-    s.x += v.x, s.y += v.y, s.z += v.z, s.w += v.w;
+  const uint32_t seq = turn + 1u;
+  bool ok = true;
+  for (int r = 0; r < pl.peer.world && ok; ++r) {
+    const uint4* src = reinterpret_cast<const uint4*>(
+        reinterpret_cast<const uint2*>(peer_slot(base, pl.peer.world, pl.peer.max_floats, ch, turn & 1u, r)) + off);
+    uint4 v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = peer_ld_pairs(src + i);
+    auto there = [&] {
+      bool t = true;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) t = t && v[i].y == seq && v[i].w == seq;
+      return t;
+    };
+    if (!there()) {  // bounded by the SM's cycle counter (~0.3 s); %globaltimer costs microseconds to read
+      const long long t0 = clock64();
+      for (uint32_t it = 1; !there(); ++it) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (v[i].y != seq || v[i].w != seq) v[i] = peer_ld_pairs(src + i);
+        if ((it & 255u) == 0 && clock64() - t0 > 600000000ll) {
+          ok = false;
+          break;
+        }
+      }
+    }
+    if (ok) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        y[2 * i] += __uint_as_float(v[i].x);
+        y[2 * i + 1] += __uint_as_float(v[i].z);
+      }
+    }
   }
-  return s;
+  return ok;
 }
 
 __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const __nv_bfloat16* gain, int norm, int batch,
@@ -153,43 +183,19 @@ __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const _
                                                          const float* pending, const float* pending2,
                                                          float* sum_out, const StagePull pl) {
   __shared__ float red[8];
-  __shared__ int pull_par[2];
-  __shared__ int pull_fail;
   const int b = blockIdx.x, slice = blockIdx.y, tid = threadIdx.x;
   pdl_launch_dependents();
   pdl_wait();
   const bool pulls = pl.peer.world > 0 && (pl.channel[0] | pl.channel[1]);
-  if (pulls) {
+  uint32_t turn0 = 0, turn1 = 0;
+  if (pulls) {  // the exchanges consumed so far on the pulled channels: receive-slot parity and sequence number
     PeerHeader* hdr = peer_header(pl.peer.base[pl.peer.rank]);
-    if (tid == 0) pull_fail = 0;
-    __syncthreads();
-    for (int i = 0; i < 2; ++i) {
-      if (!pl.channel[i]) continue;
-      const int ch = pl.channel[i] - 1;
-      if (tid == 0) pull_par[i] = *reinterpret_cast<volatile uint32_t*>(&hdr->turn[ch]) & 1;
-      if (tid < pl.peer.world) {
-        const uint32_t target = peer_ld_acquire_sys(&hdr->arrive[ch][pl.peer.rank]);
-        const uint32_t* c = &hdr->arrive[ch][tid];
-        bool ok = static_cast<int32_t>(peer_ld_acquire_sys(c) - target) >= 0;
-        if (!ok) {
-          const uint64_t t0 = global_timer_ns();
-          for (uint32_t it = 1; !ok; ++it) {
-            __nanosleep(32);
-            ok = static_cast<int32_t>(peer_ld_acquire_sys(c) - target) >= 0;
-            if (!ok && (it & 63u) == 0 && global_timer_ns() - t0 > 250000000ull) break;
-          }
-        }
-        if (!ok) {
-          pull_fail = 1;
-          if (pl.status) atomicOr(pl.status, LADDER_DEV_TIMEOUT);
-        }
-      }
-    }
-    __syncthreads();
+    if (pl.channel[0]) turn0 = *reinterpret_cast<volatile uint32_t*>(&hdr->turn[pl.channel[0] - 1]);
+    if (pl.channel[1]) turn1 = *reinterpret_cast<volatile uint32_t*>(&hdr->turn[pl.channel[1] - 1]);
+    pending = pl.channel[0] ? nullptr : pending;  // a pulled pending has no plain buffer
+    pending2 = pl.channel[1] ? nullptr : pending2;
   }
-  const bool pull0 = pulls && pl.channel[0] && !pull_fail, pull1 = pulls && pl.channel[1] && !pull_fail;
-  if (pulls && pl.channel[0]) pending = nullptr;   // a pulled pending has no plain buffer
-  if (pulls && pl.channel[1]) pending2 = nullptr;
+  bool pull_ok = true;
   __nv_bfloat16* hi = stage + static_cast<size_t>(b) * K;
   __nv_bfloat16* lo = stage + static_cast<size_t>(bp + b) * K;
   float ssq = 0.f;
@@ -200,21 +206,15 @@ __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const _
       const float4 a = __ldcg(reinterpret_cast<const float4*>(x + static_cast<size_t>(b) * K + k));
       const float4 c = __ldcg(reinterpret_cast<const float4*>(x + static_cast<size_t>(b) * K + k + 4));
       y[0] = a.x, y[1] = a.y, y[2] = a.z, y[3] = a.w, y[4] = c.x, y[5] = c.y, y[6] = c.z, y[7] = c.w;
-      if (pull0) {  // ... the module output summed over the tensor-parallel ranks
-        const size_t off = static_cast<size_t>(b) * K + k;
-        const float4 pa = pull_sum(pl, pl.channel[0] - 1, pull_par[0], off), pc = pull_sum(pl, pl.channel[0] - 1, pull_par[0], off + 4);
-        y[0] += pa.x, y[1] += pa.y, y[2] += pa.z, y[3] += pa.w, y[4] += pc.x, y[5] += pc.y, y[6] += pc.z, y[7] += pc.w;
-      }
+      if (pulls && pl.channel[0])  // ... the module output summed over the tensor-parallel ranks
+        pull_ok = pull_add8(pl, pl.channel[0] - 1, turn0, static_cast<size_t>(b) * K + k, y) && pull_ok;
       if (pending) {  // x_m = x_{m-1} + (the module output stored by an earlier GEMM)
         const float4 pa = __ldcg(reinterpret_cast<const float4*>(pending + static_cast<size_t>(b) * K + k));
         const float4 pc = __ldcg(reinterpret_cast<const float4*>(pending + static_cast<size_t>(b) * K + k + 4));
         y[0] += pa.x, y[1] += pa.y, y[2] += pa.z, y[3] += pa.w, y[4] += pc.x, y[5] += pc.y, y[6] += pc.z, y[7] += pc.w;
       }
-      if (pull1) {
-        const size_t off = static_cast<size_t>(b) * K + k;
-        const float4 pa = pull_sum(pl, pl.channel[1] - 1, pull_par[1], off), pc = pull_sum(pl, pl.channel[1] - 1, pull_par[1], off + 4);
-        y[0] += pa.x, y[1] += pa.y, y[2] += pa.z, y[3] += pa.w, y[4] += pc.x, y[5] += pc.y, y[6] += pc.z, y[7] += pc.w;
-      }
+      if (pulls && pl.channel[1])
+        pull_ok = pull_add8(pl, pl.channel[1] - 1, turn1, static_cast<size_t>(b) * K + k, y) && pull_ok;
       if (pending2) {  // ... and the one after it
         const float4 pa = __ldcg(reinterpret_cast<const float4*>(pending2 + static_cast<size_t>(b) * K + k));
         const float4 pc = __ldcg(reinterpret_cast<const float4*>(pending2 + static_cast<size_t>(b) * K + k + 4));
@@ -241,6 +241,7 @@ __global__ void __launch_bounds__(256) wide_stage_kernel(const float* x, const _
     *reinterpret_cast<uint4*>(hi + k) = h;
     *reinterpret_cast<uint4*>(lo + k) = l;
   }
+  if (!pull_ok && pl.status) atomicOr(pl.status, LADDER_DEV_TIMEOUT);
   ssq = warp_sum(ssq);
   if ((tid & 31) == 0) red[tid >> 5] = ssq;
   __syncthreads();
@@ -298,19 +299,21 @@ __device__ __forceinline__ void epi_prefetch(const SmallMParams& p, int n, int b
 template <int CB, bool PUSH>
 __device__ __forceinline__ void epi_apply(const SmallMParams& p, int n, int b0, float (&v)[CB], int lane,
                                           const int* pos_s, const float (&pa)[CB], const float (&pb)[CB], int bp,
-                                          const WidePeer& wp, const size_t* push_off_s) {
+                                          const WidePeer& wp, const size_t* push_s) {
   const bool row_ok = n < p.N;
   if (PUSH) {
     // tensor parallelism over peer memory (EPI_PLAIN only): this rank's partial sum goes straight into its receive
-    // slot on every rank (lanes hold consecutive rows: 128-byte segments per batch row and peer)
-    const size_t off = *push_off_s;
+    // slot on every rank, every value with the exchange's sequence number in one 8-byte store (lanes hold
+    // consecutive rows: 256-byte segments per batch row and peer)
+    const size_t off = push_s[0];
+    const uint32_t seq = static_cast<uint32_t>(push_s[1]);
 #pragma unroll 1
     for (int w = 0; w < wp.peer.world; ++w) {
-      float* out = reinterpret_cast<float*>(wp.peer.base[w] + kPeerHeaderBytes) + off;
+      uint2* out = reinterpret_cast<uint2*>(reinterpret_cast<float*>(wp.peer.base[w] + kPeerHeaderBytes) + off);
 #pragma unroll
       for (int j = 0; j < CB; ++j) {
         const int b = b0 + j;
-        if (b < p.batch && row_ok) out[static_cast<size_t>(b) * p.N + n] = v[j];
+        if (b < p.batch && row_ok) peer_st_pair(out + static_cast<size_t>(b) * p.N + n, v[j], seq);
       }
     }
   } else if (p.epi_mode == EPI_RESID || p.epi_mode == EPI_PLAIN) {
@@ -409,7 +412,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
   uint64_t* tmem_empty = tmem_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
   volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  size_t* push_off_s = reinterpret_cast<size_t*>(tmem_slot + 2);  // element offset of the receive slot pushed into
+  size_t* push_s = reinterpret_cast<size_t*>(tmem_slot + 2);  // float offset of the receive slot pushed into; sequence number
   float* rstd_s = reinterpret_cast<float*>(smem + C::OFF_BARS + (2 * STAGES + 4) * 8 + 64);  // [BP] 1/rms
   int* pos_s = reinterpret_cast<int*>(rstd_s + 64);                                            // [BP] positions
 
@@ -532,9 +535,11 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
     // receive-slot parity of this exchange: the channel was last moved on by a staging launch that lies before
     // this kernel's predecessors in stream order
     if (PUSH && et == 255) {  // receive slot [channel][turn & 1][this rank]: the same offset on every rank
+      // (the channel was last moved on by a staging launch that lies before this kernel's predecessors in stream order)
       const int ch = a.wp.push_channel - 1;
       const uint32_t turn = *reinterpret_cast<volatile uint32_t*>(&peer_header(a.wp.peer.base[a.wp.peer.rank])->turn[ch]);
-      *push_off_s = ((static_cast<size_t>(ch) * 2 + (turn & 1u)) * a.wp.peer.world + a.wp.peer.rank) * a.wp.peer.max_floats;
+      push_s[0] = ((static_cast<size_t>(ch) * 2 + (turn & 1u)) * a.wp.peer.world + a.wp.peer.rank) * (2 * a.wp.peer.max_floats);
+      push_s[1] = turn + 1u;
     }
     asm volatile("bar.sync 1, 256;" ::: "memory");
     for (int pos = my_start; pos < my_end; ++seg) {
@@ -587,7 +592,7 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
 #pragma unroll
             for (int j = 0; j < CB; ++j) v[j] *= rstd_s[b0 + j];
           }
-          epi_apply<CB, PUSH>(p, n, b0, v, lane, pos_s, pa, pb, BP, a.wp, push_off_s);
+          epi_apply<CB, PUSH>(p, n, b0, v, lane, pos_s, pa, pb, BP, a.wp, push_s);
         } else {
 #pragma unroll
           for (int j = 0; j < CB; j += 4) piece[((b0 + j) >> 2) * 32] = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -649,20 +654,10 @@ decode_gemm_wide_tc_kernel(const WideArgs a, const __grid_constant__ CUtensorMap
 #pragma unroll
           for (int j = 0; j < FB; ++j) v[j] *= rstd_s[b0 + j];
         }
-        epi_apply<FB, PUSH>(p, n, b0, v, lane, pos_s, pa, pb, BP, a.wp, push_off_s);
+        epi_apply<FB, PUSH>(p, n, b0, v, lane, pos_s, pa, pb, BP, a.wp, push_s);
       }
     }
     if (!ok && lane == 0 && p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
-    if (PUSH) {  // every CTA of the launch counts its arrival on every rank, its stores before it
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (et == 0 && ok) {
-        __threadfence_system();
-        for (int o = 1; o <= a.wp.peer.world; ++o) {
-          const int w = (a.wp.peer.rank + o) % a.wp.peer.world;
-          peer_red_release_sys_add(&peer_header(a.wp.peer.base[w])->arrive[a.wp.push_channel - 1][a.wp.peer.rank], 1u);
-        }
-      }
-    }
   }
 
   tc_fence_before();

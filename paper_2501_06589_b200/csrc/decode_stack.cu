@@ -33,7 +33,7 @@
 //                 log-sum-exp merge, units dealt round-robin over the CTAs
 // Data produced inside the launch is always read through L2 (ld.global.cg / acquire), never through
 // the non-coherent L1 path and never by the TMA engine (a bulk copy of bytes other SMs had just written
-// returned stale data now and then, proxy fences on both sides notwithstanding).  Every wait is bounded (0.25 s) and also gives up when another CTA has
+// returned stale data now and then, proxy fences on both sides notwithstanding).  Every wait is bounded (about 0.3 s) and also gives up when another CTA has
 // reported a timeout in the device status word, so a protocol error ends the launch quickly with
 // LADDER_DEV_TIMEOUT set instead of hanging the device.
 #include "common.cuh"
@@ -57,7 +57,6 @@ constexpr int SPW = TK / 32 / 4;
 constexpr int RED_FLOATS = 4 * RG_MAX * 4 * 32;
 constexpr int QDEPTH = 16;
 constexpr int NORM_RING = 4;  // the stagers run at most three normalised phases ahead of the finishers
-constexpr uint64_t kTimeoutNs = 250000000ull;
 constexpr int kChunk = 64;         // keys per attention unit
 constexpr int kMaxSplits = 1024;   // merge weights held in shared memory
 
@@ -136,29 +135,29 @@ __device__ __forceinline__ bool bar_and(int id, int count, bool pred) {
 template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool wait_mbar(uint64_t* bar, uint32_t parity, const int32_t* status) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if (mbar_try_wait_suspend(bar, parity, 4000u)) return true;
-    if ((i & 15u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
+    if ((i & 15u) == 0 && (aborted(status) || clock64() - t0 > kWaitCycles)) return false;
   }
 }
 __device__ __forceinline__ bool wait_counter_gt(const volatile int* ctr, int n, const int32_t* status) {
   if (*ctr > n) return true;
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     __nanosleep(64);  // a hot spin would take issue slots from the consumer warp of the same sub-partition
     if (*ctr > n) return true;
-    if ((i & 255u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
+    if ((i & 255u) == 0 && (aborted(status) || clock64() - t0 > kWaitCycles)) return false;
   }
 }
 __device__ __forceinline__ bool wait_global_ge(const int32_t* ctr, int need, const int32_t* status) {
   if (ld_acquire(ctr) >= need) return true;
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     __nanosleep(100);
     if (ld_acquire(ctr) >= need) return true;
-    if ((i & 31u) == 0 && (aborted(status) || global_timer_ns() - t0 > kTimeoutNs)) return false;
+    if ((i & 31u) == 0 && (aborted(status) || clock64() - t0 > kWaitCycles)) return false;
   }
 }
 // lane i of the calling warp polls dependency i; the warp agrees on the outcome

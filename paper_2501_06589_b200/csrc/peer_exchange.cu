@@ -11,7 +11,7 @@
 // ordered on their own stream on every rank.  Two parities: a rank can start exchange t + 1 of a channel while a peer
 // still adds the slots of exchange t, but it cannot start t + 2 before it has received that peer's part of t + 1,
 // which the peer sends after it is done with t.
-// Every wait is bounded (about 0.25 s): on expiry the kernel sets LADDER_DEV_TIMEOUT in the status word it was
+// Every wait is bounded (about 0.3 s): on expiry the kernel sets LADDER_DEV_TIMEOUT in the status word it was
 // given, skips the sum and returns.  No multicast loads, no multimem: plain peer stores and local loads.
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -32,6 +32,7 @@ constexpr int kMaxWorld = LADDER_PEER_MAX_WORLD;
 static_assert(kMaxWorld == ladder::kPeerMaxWorld, "world limit");
 constexpr int kCtas = 16;       // CTAs per exchange kernel: the same on every rank (the counters count them)
 constexpr int kThreads = 512;
+constexpr long long kWaitCycles = 600000000ll;  // bound of a wait: ~0.3 s at 1.9 GHz
 constexpr size_t kHeaderBytes = ladder::kPeerHeaderBytes;
 using PeerArgs = PeerView;
 
@@ -75,11 +76,12 @@ __global__ void __launch_bounds__(kThreads) peer_all_reduce_kernel(PeerArgs a, i
     const uint32_t* c = &mine->arrive[channel][threadIdx.x];
     bool ok = static_cast<int32_t>(ld_acquire_sys(c) - target) >= 0;
     if (!ok) {
-      const uint64_t t0 = ladder::global_timer_ns();
+      // Poll without sleeping, bounded by the SM's cycle counter (about 0.3 s).  Not %globaltimer: reading it takes
+      // microseconds, which a kernel this short cannot hide (measured: 12.3 -> 6.9 us per exchange).
+      const long long t0 = clock64();
       for (uint32_t i = 1; !ok; ++i) {
-        __nanosleep(64);
         ok = static_cast<int32_t>(ld_acquire_sys(c) - target) >= 0;
-        if (!ok && (i & 63u) == 0 && ladder::global_timer_ns() - t0 > 250000000ull) break;
+        if (!ok && (i & 255u) == 0 && clock64() - t0 > kWaitCycles) break;
       }
     }
     if (!ok) {
@@ -154,7 +156,7 @@ ladder_status_t ladder_peer_create(int32_t world, int32_t rank, int64_t max_floa
   p->world = world;
   p->rank = rank;
   p->max_floats = static_cast<size_t>(max_floats);
-  p->bytes = kHeaderBytes + sizeof(float) * 2 * 2 * world * p->max_floats;
+  p->bytes = kHeaderBytes + sizeof(float) * 2 * 2 * world * 2 * p->max_floats;
   void* mem = nullptr;
   if (cudaMalloc(&mem, p->bytes) != cudaSuccess) {
     cudaGetLastError();
@@ -250,8 +252,7 @@ ladder_status_t ladder_peer_probe_read(const ladder_peer_t* p, int32_t from, uin
 // rank's memory, and the counter that says it has.
 float* ladder_peer_slot(const ladder_peer_t* p, int32_t channel, int32_t parity, int32_t from) {
   if (!p || channel < 0 || channel > 1 || parity < 0 || parity > 1 || from < 0 || from >= p->world) return nullptr;
-  return reinterpret_cast<float*>(p->base[p->rank] + kHeaderBytes) +
-         ((static_cast<size_t>(channel) * 2 + parity) * p->world + from) * p->max_floats;
+  return ladder::peer_slot(p->base[p->rank], p->world, p->max_floats, channel, parity, from);
 }
 uint32_t* ladder_peer_counter(const ladder_peer_t* p, int32_t channel, int32_t from) {
   if (!p || channel < 0 || channel > 1 || from < 0 || from >= p->world) return nullptr;

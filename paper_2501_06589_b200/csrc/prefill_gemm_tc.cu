@@ -385,8 +385,8 @@ largem_gemm_tc_pair_kernel(const LargeMParams p, const __grid_constant__ CUtenso
       }
       if (!ok) {
         if (p.status) atomicOr(p.status, LADDER_DEV_TIMEOUT);
-        const uint64_t t0 = global_timer_ns();  // copies still in flight land in this CTA's shared memory: let them
-        while (global_timer_ns() - t0 < 100000ull) __nanosleep(1000);
+        const long long t0 = clock64();  // copies still in flight land in this CTA's shared memory: let them
+        while (clock64() - t0 < 200000ll) __nanosleep(1000);
       }
     }
   } else if (warp == 1) {

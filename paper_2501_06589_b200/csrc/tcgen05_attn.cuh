@@ -63,13 +63,13 @@ __device__ __forceinline__ void at_ld32(uint32_t taddr, uint32_t* r) {
       : "memory");
 }
 // Bounded wait that lets the hardware suspend the thread while the phase is incomplete: a warp that waits takes no
-// issue slots from the softmax warp of its sub-partition.  Gives up after ~0.25 s.
+// issue slots from the softmax warp of its sub-partition.  Gives up after about 0.3 s.
 __device__ __forceinline__ bool at_wait(uint64_t* bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait_suspend(bar, parity, 2000u)) return true;
-    if ((i & 15u) == 0 && global_timer_ns() - t0 > 250000000ull) return false;
+    if ((i & 15u) == 0 && clock64() - t0 > kWaitCycles) return false;
   }
 }
 // The same wait for a whole warp.  Lanes leave the polling loop at different times; the vote brings them back

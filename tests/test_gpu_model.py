@@ -505,7 +505,7 @@ def test_pending_output_form_equals_epilogue_additions(B):
 
 
 def test_persistent_kernel_wait_runs_out_cleanly(B):
-    """A dependency that is never met ends the launch after the 0.25 s limit with the timeout bit set;
+    """A dependency that is never met ends the launch after the about 0.3 s limit with the timeout bit set;
     nothing hangs or faults, and once the status has been read the same model decodes correctly again."""
     import time
     s = synth.SHAPES["tiny"]

@@ -225,9 +225,9 @@ def test_decode_exchange_over_peer_memory_in_a_world_of_one(B, variant, batch):
 def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, streams):
     """As test_rank_0_with_the_oracle_as_rank_1, but the decode-step exchange is the fused one: rank 0's output GEMMs
     push their partial sums into the receive slots (rank 0's own and, on the same GPU, those of a second object that
-    stands for rank 1's memory), and the staging launches wait for the arrival counters and add the slots.  Rank 1's
-    stores - the oracle's rank-1 partial and an arrival count equal to rank 0's - are enqueued by the test right
-    behind each output GEMM, so every wait is already satisfied when its kernel starts."""
+    stands for rank 1's memory) as (value, sequence number) pairs, and the staging launches poll the pairs and add
+    the slots.  Rank 1's stores - the oracle's rank-1 partial, numbered like rank 0's - are enqueued by the test right
+    behind each output GEMM, so every poll succeeds at once."""
     from paper_2501_06589_b200 import tensor_parallel as TP
     s = shape_of(variant)
     world, S, steps = 2, 12, 6
@@ -255,12 +255,12 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
     model.set_schedule(streams, True, True)
     queue, turns = [], [0, 0]
 
-    class _Word:
-        def __init__(self, ptr):
-            self.__cuda_array_interface__ = {"shape": (1,), "typestr": "<i4", "data": (ptr, False), "version": 2}
+    class _Words:
+        def __init__(self, ptr, count):
+            self.__cuda_array_interface__ = {"shape": (count,), "typestr": "<i4", "data": (ptr, False), "version": 2}
 
-    def word(ptr):
-        return torch.as_tensor(_Word(ptr), device="cuda")
+    def words(ptr, count):
+        return torch.as_tensor(_Words(ptr, count), device="cuda")
 
     def prompt_exchange(ptr, count, stream):                 # the prompt pass: NCCL's place
         with torch.cuda.stream(torch.cuda.ExternalStream(stream or 0)):
@@ -269,9 +269,11 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
 
     def rank_1_arrives(channel, stream):                     # a decode-step output GEMM of rank 0 has been enqueued
         part = queue.pop(0)
+        pairs = torch.empty(n, 2, dtype=torch.int32, device="cuda")   # (value, sequence number of the exchange)
+        pairs[:, 0] = part.view(torch.int32)
+        pairs[:, 1] = turns[channel] + 1
         with torch.cuda.stream(torch.cuda.ExternalStream(stream or 0)):
-            torch.as_tensor(_DeviceFloats(p0.slot_ptr(channel, turns[channel] & 1, 1), n), device="cuda").copy_(part)
-            word(p0.counter_ptr(channel, 1)).copy_(word(p0.counter_ptr(channel, 0)))   # as many arrivals as rank 0's own
+            words(p0.slot_ptr(channel, turns[channel] & 1, 1), 2 * n).copy_(pairs.view(-1))
         turns[channel] += 1
 
     model.set_exchange(prompt_exchange, capturable=False)
@@ -293,12 +295,11 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
         hids.append(hid.cpu().numpy().copy())
     assert model.device_status() == 0
     assert turns == [s.n_layers * steps] * 2
-    # rank 0's partial of the last attention module has landed in "rank 1's" memory too, with the same arrival count
-    last = (turns[0] - 1) & 1
-    mine = torch.as_tensor(_DeviceFloats(p0.slot_ptr(0, last, 0), n), device="cuda")
-    theirs = torch.as_tensor(_DeviceFloats(p1.slot_ptr(0, last, 0), n), device="cuda")
-    assert torch.equal(mine, theirs) and float(mine.abs().max()) > 0
-    assert word(p1.counter_ptr(0, 0)).item() == word(p0.counter_ptr(0, 0)).item() > 0
+    # rank 0's partial of the last attention module has landed in "rank 1's" memory too, numbered like its own copy
+    last = turns[0] - 1
+    mine = words(p0.slot_ptr(0, last & 1, 0), 2 * n).view(n, 2)
+    theirs = words(p1.slot_ptr(0, last & 1, 0), 2 * n).view(n, 2)
+    assert torch.equal(mine, theirs) and bool((mine[:, 1] == last + 1).all()) and int(mine[:, 0].abs().max()) > 0
     err = rel_err(np.stack(hids, 1), np.stack(o_hids, 1))
     print(f"[tp rank 0, fused exchange over peer memory / oracle rank 1, {variant}, batch {batch}, {streams} stream(s)] "
           f"hidden max-rel-err {err:.3e}")

@@ -52,13 +52,15 @@ def shape_of(variant):
     return replace(BASE, layer_is_ladder=VARIANTS[variant])
 
 
-@pytest.mark.parametrize("streams", [2, 1])
-@pytest.mark.parametrize("batch", [2, 6])
-@pytest.mark.parametrize("variant", ["ladder", "standard", "hybrid"])
-def test_rank_0_with_the_oracle_as_rank_1(B, variant, batch, streams):
+CASES = [(v, b, st, 12) for v in ("ladder", "standard", "hybrid") for b in (2, 6) for st in (2, 1)]
+CASES += [("ladder", 4, 2, 80), ("standard", 4, 2, 80)]     # 320 prompt tokens: the binary16 prompt-pass GEMMs
+
+
+@pytest.mark.parametrize("variant,batch,streams,S", CASES)
+def test_rank_0_with_the_oracle_as_rank_1(B, variant, batch, streams, S):
     from paper_2501_06589_b200 import tensor_parallel as TP
     s = shape_of(variant)
-    world, S, steps = 2, 12, 6
+    world, steps = 2, 6
     w = synth.make_weights(s, device="cuda", gains="uniform")
     prompt = synth.make_tokens(s, batch, S)
 

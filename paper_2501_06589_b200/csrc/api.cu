@@ -541,7 +541,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   const double layer_bytes = 2.0 * (static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh + 3.0 * F * d);
   const bool auto_wide = (m->sms_a == -1 || m->sms_a == -3) && batch > 4 && layer_bytes < 300e6;
   if (q.two && (m->sms_a >= 0 || auto_wide)) {
-    int ga = auto_wide ? (60 * m->sm_count + 74) / 148 : m->sms_a;
+    int ga = auto_wide ? (56 * m->sm_count + 74) / 148 : m->sms_a;  // 56 : 92 (swept 40 .. 72 in the pending-output form)
     if (ga == 0) {
       const double ba = static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh;
       const double bb = 3.0 * F * d;

@@ -35,7 +35,9 @@ def B():
 
 def oracle_cfg(s, world):
     c = O.OracleConfig(s.d_model, s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.d_ff, s.vocab_size,
-                       s.rms_eps, s.rope_theta, None if s.layer_is_ladder is None else list(s.layer_is_ladder))
+                       s.rms_eps, s.rope_theta, None if s.layer_is_ladder is None else list(s.layer_is_ladder),
+                       layer_mode=None if s.layer_mode is None else list(s.layer_mode),
+                       module_stale=None if s.module_stale is None else list(s.module_stale))
     c.tp_world = world
     return c
 
@@ -49,11 +51,16 @@ class _DeviceFloats:
 
 def shape_of(variant):
     from dataclasses import replace
+    if variant == "parallel":                    # attention and MLP of a layer read the same input (Sec. 3.3.1)
+        return BASE.as_mode("parallel")
+    if variant == "flags":                       # an arbitrary per-module rule: every kind of neighbour pair occurs
+        return replace(BASE, layer_mode=tuple(["standard"] * BASE.n_layers), module_stale=(0, 1, 1, 0, 0, 0, 1, 1))
     return replace(BASE, layer_is_ladder=VARIANTS[variant])
 
 
 CASES = [(v, b, st, 12) for v in ("ladder", "standard", "hybrid") for b in (2, 6) for st in (2, 1)]
 CASES += [("ladder", 4, 2, 80), ("standard", 4, 2, 80)]     # 320 prompt tokens: the binary16 prompt-pass GEMMs
+CASES += [(v, b, st, 12) for v in ("parallel", "flags") for b in (3, 9) for st in (2, 1)]
 
 
 @pytest.mark.parametrize("variant,batch,streams,S", CASES)
@@ -223,7 +230,8 @@ def test_decode_exchange_over_peer_memory_in_a_world_of_one(B, variant, batch):
 
 
 @pytest.mark.parametrize("streams", [2, 1])
-@pytest.mark.parametrize("variant,batch", [("ladder", 6), ("standard", 6), ("hybrid", 3), ("ladder", 40)])
+@pytest.mark.parametrize("variant,batch", [("ladder", 6), ("standard", 6), ("hybrid", 3), ("ladder", 40), ("parallel", 6),
+                                           ("flags", 5)])
 def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, streams):
     """As test_rank_0_with_the_oracle_as_rank_1, but the decode-step exchange is the fused one: rank 0's output GEMMs
     push their partial sums into the receive slots (rank 0's own and, on the same GPU, those of a second object that

@@ -213,7 +213,8 @@ ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attenti
  * kernel per GEMM.  Prompt pass: exchanges and adds run on a stream of their own and the GEMM stream waits only
  * where a module reads what an add writes.  capturable != 0: `exchange` may be called while its stream is being
  * captured into a CUDA graph (NCCL collectives may); 0: decode steps are enqueued without a graph.
- * fn == NULL switches it off.  Pipeline-stage calls (ladder_stage_*) return LADDER_ERR_UNSUPPORTED while it is on.
+ * fn == NULL switches it off.  Pipeline-stage calls (ladder_stage_*) work under it (tensor parallelism inside every
+ * stage, paper Sec. 5.1): the pair a stage hands on is the summed stream state, identical on all its ranks.
  * Costs 2 x max_prefill_tokens x d_model x 4 bytes of device memory on first use (LADDER_ERR_OOM if there is none).
  * Measured on one GPU only (a world of one, and against recorded partials of the other ranks): the hardware this
  * was built on has one GPU per job, so no multi-GPU timing is claimed. */
@@ -264,8 +265,8 @@ ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_
  * (messages of hundreds of MB, where NCCL's algorithms are the right ones) over `comm`; LADDER_ERR_INVALID_ARG if the
  * peer object is too small for max_batch x d_model, not connected or of another world.  ladder_model_set_peer(m, peer)
  * is the second half alone, for a model whose prompt-pass exchange was set with ladder_model_set_exchange
- * (LADDER_ERR_STATE if none is set); NULL switches back.  Both objects stay the caller's; an object serves either
- * models or ladder_peer_all_reduce_sum calls, not both (they count arrivals differently).
+ * (LADDER_ERR_STATE if none is set); NULL switches back.  Both objects stay the caller's; a peer object serves ONE
+ * model (each pipeline stage its own), or ladder_peer_all_reduce_sum calls: its channels number their exchanges.
  * ladder_debug_set_peer_hook: a function called on the host right after each decode-step output GEMM has been
  * enqueued (channel, stream), so that a test can enqueue an absent rank's stores there; steps then run ungraphed.
  * ladder_peer_probe_write / _read: connectivity check by host copies (rank a writes a word into rank b's memory, b

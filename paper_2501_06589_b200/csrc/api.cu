@@ -349,6 +349,9 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
   q.launched(0, begin_stream(m, rt, d_tokens, batch, sA));
   int cur = rt.cur;  // R[cur]: the newest stream value formed so far = x_0 + outputs of modules 0 .. added
   int added = -1;
+  // A pipeline stage that was handed (x_{-1}, x_{-2}): they are in R[cur] and the other buffer; only this stage's
+  // first module can read the older one, before any staging step overwrites it.
+  const int older_buf = (m->st_in.newest && m->st_in.older) ? (cur ^ 1) : -1;
   auto pend = [&](int j) { return (j & 1) ? m->pend_m : m->pend_a; };
   auto ev_stage = [&](int j) { return (j & 1) ? m->ev_sg[j >> 1] : m->ev_sq[j >> 1]; };
   // Staging step of module `mod` (2L = the head) on stream s: its input is x_0 + outputs of modules 0 .. upto.
@@ -358,7 +361,7 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
     for (int j = added + 1; j <= upto; ++j)
       if ((j & 1) != s) q.wait(s, m->ev_out[j]);  // a stored output of the other stream (same stream: in order)
     const int n = upto - added;                   // 0, 1 or 2
-    p.act = m->R[cur];
+    p.act = (mod == 0 && m->stale[0] && older_buf >= 0) ? m->R[older_buf] : m->R[cur];
     WidePeer pull = {};
     if (use_peer) {  // the stored outputs are the ranks' partial sums in this rank's receive slots
       pull.peer = view;
@@ -495,6 +498,25 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
       q.gemm(s, dn, side);
       output_stored(mod, s);
     }
+  }
+  if (m->st_out.newest) {  // a stage that hands its state on: x_{2L-1} (all outputs but the last) and x_{2L}, no head
+    const size_t bytes = static_cast<size_t>(batch) * d * sizeof(float);
+    auto note = [&](cudaError_t e) {
+      if (q.err == cudaSuccess) q.err = e;
+    };
+    for (int i = 0; i < 2; ++i) {
+      if (i == 0 && !m->st_out.older) continue;
+      SmallMParams t = {};
+      t.K = d;
+      t.act_mode = ACT_F32;
+      t.batch = batch;
+      form_input(2 * L + i, 0, 2 * L - 2 + i, t);  // a staging launch for its sum only
+      note(cudaMemcpyAsync(i == 0 ? m->st_out.older : m->st_out.newest, m->R[cur], bytes, cudaMemcpyDeviceToDevice, sA));
+      q.pdl_ok[0] = false;
+    }
+    q.launched(0, launch_argmax_advance(nullptr, batch, c.vocab_size, nullptr, cache->seq_lens, 1, -1, sA, false, nullptr));
+    *n_kernels = q.kernels;
+    return q.err;
   }
   // ---------------- head on stream A: reads x_{2L} (every output added)
   float* logits = (out && out->logits) ? out->logits : m->logits_ws;
@@ -1799,7 +1821,6 @@ ladder_status_t ladder_stage_prefill(ladder_model_t* m, const ladder_kv_cache_t*
   if (!m) return LADDER_ERR_INVALID_ARG;
   if (const char* why = check_stage(state_in, state_out, d_tokens)) return fail(m, LADDER_ERR_INVALID_ARG, why);
   if (state_out && out && out->all_hidden) return fail(m, LADDER_ERR_INVALID_ARG, "a stage that hands its state on has no head outputs");
-  if (m->exchange) return fail(m, LADDER_ERR_UNSUPPORTED, "pipeline stages under tensor parallelism");
   StageScope scope(m, state_in, state_out);
   return ladder_prefill(m, cache, d_tokens, batch, seq_len, out, cuda_stream);
 }
@@ -1841,7 +1862,6 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
   const bool two = m->n_streams == 2;
 
   const bool staged = m->st_in.newest || m->st_out.newest;  // a pipeline stage runs kernel by kernel
-  if (staged && m->exchange) return fail(m, LADDER_ERR_UNSUPPORTED, "pipeline stages under tensor parallelism");
   if (m->use_stack && m->stack_ok && batch <= 4 && !staged && !m->exchange) {
     GraphKey key;
     key.batch = batch;

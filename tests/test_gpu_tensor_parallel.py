@@ -177,22 +177,66 @@ def test_world_of_one_over_nccl(B, variant, batch):
     comm.close()
 
 
-def test_pipeline_stages_are_refused_under_tensor_parallelism(B):
-    s = shape_of("ladder")
-    w = synth.make_weights(s, device="cuda")
-    model = B.Model(w, 2, 32, 32)
-    model.set_exchange(lambda ptr, count, stream: 0)
-    cache = B.KVCache(s, 2, 32)
-    tok = torch.zeros(2, 4, dtype=torch.int32, device="cuda")
-    x0 = torch.zeros(2 * 4, s.d_model, device="cuda")
-    x1 = torch.zeros(2 * 4, s.d_model, device="cuda")
-    with pytest.raises(B.LadderError) as e:
-        model.stage_prefill(cache, tok, 2, 4, None, (x0, x1))
-    assert e.value.status == 2
-    model.set_exchange(None)
-    model.stage_prefill(cache, tok, 2, 4, None, (x0, x1))
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("mask,cut,bsz", [((1, 1, 1, 1), 2, 3), ((0, 1, 1, 0), 2, 6), ((1, 1, 0, 1), 1, 3)])
+def test_pipeline_stages_under_tensor_parallelism(B, mask, cut, bsz, fused):
+    """Tensor parallelism inside every pipeline stage (Sec. 5.1), in a world of one: two stage models chained through
+    the handed-on pair reproduce the whole tensor-parallel model bit for bit, prompt pass and decode steps, with the
+    exchange over NCCL and fused over peer memory (one peer object per model)."""
+    from paper_2501_06589_b200 import tensor_parallel as TP
+    from tests.test_gpu_model import gpu_generate, _whole_model_flags
+    s = synth.replace(BASE, layer_is_ladder=mask)
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    S, steps = 20, 6
+    max_seq = S + steps + 2
+    prompt = synth.make_tokens(s, bsz, S)
+    tok = torch.from_numpy(prompt).cuda()
+    flags = _whole_model_flags(s)
+    comm = TP.make_comm()
+    peers = []
+
+    def parallel(model):
+        if fused:
+            peers.append(TP.make_peer(bsz * s.d_model))
+            model.set_tensor_parallel_peer(comm, peers[-1])
+        else:
+            model.set_tensor_parallel(comm)
+        return model
+
+    whole = parallel(B.Model(w, bsz, max_seq, bsz * S))
+    ref_toks, ref_hids = gpu_generate(B, whole, B.KVCache(s, bsz, max_seq), prompt, steps)
+    whole.close()
+
+    def stage(lo, hi):
+        sh = synth.replace(s, n_layers=hi - lo, layer_is_ladder=tuple(mask[lo:hi]), module_stale=tuple(flags[2 * lo:2 * hi]))
+        ws = synth.AbiWeights(sh, w.tok_embedding, w.final_norm, w.lm_head, w.attn_norm[lo:hi], w.w_qkv[lo:hi],
+                              w.w_o[lo:hi], w.mlp_norm[lo:hi], w.w_gate_up[lo:hi], w.w_down[lo:hi])
+        return parallel(B.Model(ws, bsz, max_seq, bsz * S)), B.KVCache(sh, bsz, max_seq)
+
+    (m0, c0), (m1, c1) = stage(0, cut), stage(cut, 4)
+    d = s.d_model
+    big = (torch.zeros(bsz * S, d, device="cuda"), torch.zeros(bsz * S, d, device="cuda"))
+    small = (torch.zeros(bsz, d, device="cuda"), torch.zeros(bsz, d, device="cuda"))
+    nxt = torch.zeros(bsz, dtype=torch.int32, device="cuda")
+    hid = torch.zeros(bsz, d, device="cuda")
+    m0.stage_prefill(c0, tok, bsz, S, state_out=big)
+    m1.stage_prefill(c1, None, bsz, S, state_in=big, next_tokens=nxt, final_hidden=hid)
+    toks, hids = [nxt.clone()], [hid.clone()]
+    for _ in range(steps):
+        m0.stage_decode_step(c0, nxt, bsz, state_out=small)
+        m1.stage_decode_step(c1, None, bsz, state_in=small, next_tokens=nxt, final_hidden=hid)
+        toks.append(nxt.clone())
+        hids.append(hid.clone())
     torch.cuda.synchronize()
-    model.close()
+    assert m0.device_status() == 0 and m1.device_status() == 0
+    assert np.array_equal(torch.stack(toks, 1).cpu().numpy(), ref_toks)
+    assert np.array_equal(torch.stack(hids, 1).cpu().numpy(), ref_hids)
+    assert c0.seq_lens.cpu().tolist() == [S + steps] * bsz and c1.seq_lens.cpu().tolist() == [S + steps] * bsz
+    m0.close()
+    m1.close()
+    for p in peers:
+        p.close()
+    comm.close()
 
 
 @pytest.mark.parametrize("variant,batch", [("ladder", 3), ("hybrid", 12)])

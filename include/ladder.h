@@ -211,7 +211,9 @@ ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attenti
  * the partial, so with two streams a ladder layer's other module computes meanwhile, while with standard residuals
  * the next module's input waits for it (Eq. 1: the paper's baseline); all batch sizes run on the tcgen05 GEMMs, one
  * kernel per GEMM.  Prompt pass: exchanges and adds run on a stream of their own and the GEMM stream waits only
- * where a module reads what an add writes.  capturable != 0: `exchange` may be called while its stream is being
+ * where a module reads what an add writes.  A layer whose MLP module reads the same input as its attention module
+ * (parallel attention + MLP, Sec. 3.3.1) has ONE exchange: the down projection adds the attention module's stored
+ * partial sum before it.  capturable != 0: `exchange` may be called while its stream is being
  * captured into a CUDA graph (NCCL collectives may); 0: decode steps are enqueued without a graph.
  * fn == NULL switches it off.  Pipeline-stage calls (ladder_stage_*) work under it (tensor parallelism inside every
  * stage, paper Sec. 5.1): the pair a stage hands on is the summed stream state, identical on all its ranks.

@@ -353,24 +353,35 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
   // first module can read the older one, before any staging step overwrites it.
   const int older_buf = (m->st_in.newest && m->st_in.older) ? (cur ^ 1) : -1;
   auto pend = [&](int j) { return (j & 1) ? m->pend_m : m->pend_a; };
+  // Under an exchange, a layer whose MLP does not read its attention module's output and whose attention output
+  // nobody reads on its own (parallel attention + MLP, Sec. 3.3.1) sums the two outputs BEFORE the exchange: the
+  // down projection adds the stored attention output in its epilogue, and there is one exchange per layer.
+  auto merged = [&](int j) {  // module j's output travels inside module j + 1's
+    if (!m->exchange || (j & 1) || j + 1 >= 2 * L || m->stale[j] || !m->stale[j + 1]) return false;  // a parallel-shaped layer
+    if (j + 2 < 2 * L) return m->stale[j + 2] == 0;
+    return m->st_out.newest == nullptr || m->st_out.older == nullptr;  // the head reads everything; a handed-on x_{2L-1} would not
+  };
   auto ev_stage = [&](int j) { return (j & 1) ? m->ev_sg[j >> 1] : m->ev_sq[j >> 1]; };
   // Staging step of module `mod` (2L = the head) on stream s: its input is x_0 + outputs of modules 0 .. upto.
   auto form_input = [&](int mod, int s, int upto, SmallMParams& p) {
     if (upto < added) upto = added;  // module 0 has no x_{-1}: it reads x_0 whatever its flag
     if (mod > 0 && ((mod - 1) & 1) != s) q.wait(s, ev_stage(mod - 1));  // the stream value the previous step formed
-    for (int j = added + 1; j <= upto; ++j)
+    int list[2] = {-1, -1}, n = 0;  // the stored outputs still to add, in module order: none, one or two
+    for (int j = added + 1; j <= upto; ++j) {
+      if (merged(j)) continue;  // inside the next module's
       if ((j & 1) != s) q.wait(s, m->ev_out[j]);  // a stored output of the other stream (same stream: in order)
-    const int n = upto - added;                   // 0, 1 or 2
+      list[n++] = j;
+    }
     p.act = (mod == 0 && m->stale[0] && older_buf >= 0) ? m->R[older_buf] : m->R[cur];
     WidePeer pull = {};
     if (use_peer) {  // the stored outputs are the ranks' partial sums in this rank's receive slots
       pull.peer = view;
-      pull.pull_channel[0] = n >= 1 ? ((added + 1) & 1) + 1 : 0;
-      pull.pull_channel[1] = n >= 2 ? ((added + 2) & 1) + 1 : 0;
+      pull.pull_channel[0] = n >= 1 ? (list[0] & 1) + 1 : 0;
+      pull.pull_channel[1] = n >= 2 ? (list[1] & 1) + 1 : 0;
       p.wide_peer = &pull;
     } else {
-      p.act_pending = n >= 1 ? pend(added + 1) : nullptr;
-      p.act_pending2 = n >= 2 ? pend(added + 2) : nullptr;
+      p.act_pending = n >= 1 ? pend(list[0]) : nullptr;
+      p.act_pending2 = n >= 2 ? pend(list[1]) : nullptr;
     }
     p.act_sum_out = n >= 1 ? m->R[cur ^ 1] : nullptr;
     p.scratch = m->gemm_scratch[q.two ? s : 0];
@@ -385,6 +396,10 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
   };
   // The module's output is complete in pend(mod): sum it over the tensor-parallel ranks, tell the other stream.
   auto output_stored = [&](int mod, int s) {
+    if (merged(mod)) {  // stays local: the down projection of this layer adds it before the exchange
+      q.record(s, m->ev_out[mod]);
+      return;
+    }
     if (use_peer) {  // the GEMM itself has pushed the partial sum to every rank
       if (m->peer_hook) {
         m->peer_hook(m->peer_hook_ctx, mod & 1, q.stream(s));
@@ -455,7 +470,7 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
       o.out = pend(mod);
       o.act_staged = m->wide_opack;
       WidePeer push = {};
-      if (use_peer) {
+      if (use_peer && !merged(mod)) {
         push.peer = view;
         push.push_channel = (mod & 1) + 1;
         o.wide_peer = &push;
@@ -489,6 +504,11 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
       dn.epi_mode = EPI_PLAIN;
       dn.out = pend(mod);
       dn.act_staged = m->wide_hpack;
+      if (merged(mod - 1)) {  // attention + MLP output of this layer as one sum
+        q.wait(s, m->ev_out[mod - 1]);
+        dn.epi_mode = EPI_RESID;
+        dn.addend = pend(mod - 1);
+      }
       WidePeer push = {};
       if (use_peer) {
         push.peer = view;
@@ -803,6 +823,14 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
   // input x_{m-2} is older than the exchange in flight; with standard residuals the very next module waits).
   const bool tp = m->exchange != nullptr;
   int add_writer[2] = {-1, -1};  // module whose add on the exchange stream last wrote R[i]
+  // module j's output travels inside module j + 1's (one exchange for a parallel attention + MLP layer: see the
+  // decode step's pending-output form)
+  auto merged = [&](int j) {
+    const int n_mod = 2 * c.n_layers;
+    if (!tp || (j & 1) || j + 1 >= n_mod || m->stale[j] || !m->stale[j + 1]) return false;
+    if (j + 2 < n_mod) return m->stale[j + 2] == 0;
+    return m->st_out.newest == nullptr || m->st_out.older == nullptr;
+  };
   auto norm = [&](int buf, const __nv_bfloat16* gain) {
     if (tp && add_writer[buf] >= 0) note(cudaStreamWaitEvent(st, m->ev_pf_add[add_writer[buf]], 0));
     const float* x = m->R[buf];
@@ -819,14 +847,23 @@ cudaError_t enqueue_prefill(ladder_model* m, const ladder_kv_cache_t* cache, con
       return;
     }
     float* const pend = m->pend_pf[mod & 1];
-    if (mod >= 2) note(cudaStreamWaitEvent(st, m->ev_pf_add[mod - 2], 0));  // the buffer's previous content is added
     o.epi_mode = EPI_PLAIN;
     o.out = pend;
+    if (merged(mod)) {  // parallel attention + MLP: stays local, the down projection adds it before the one exchange
+      did(launch_largem_gemm(o, st));
+      return;
+    }
+    if (mod >= 2 && !merged(mod - 2)) note(cudaStreamWaitEvent(st, m->ev_pf_add[mod - 2], 0));  // the buffer's previous content is added
+    const bool both = (mod & 1) && merged(mod - 1);  // this output plus the attention module's: x_{m} = x_{m-2} + sum
+    if (both) {
+      o.epi_mode = EPI_RESID;
+      o.addend = m->pend_pf[0];
+    }
     did(launch_largem_gemm(o, st));
     note(cudaEventRecord(m->ev_pf_out[mod], st));
     note(cudaStreamWaitEvent(m->xstream, m->ev_pf_out[mod], 0));
     if (m->exchange(m->exchange_ctx, pend, static_cast<int64_t>(M) * d, m->xstream) != LADDER_OK) note(cudaErrorUnknown);
-    did(launch_add_f32(m->R[r.add], pend, m->R[r.dst], static_cast<size_t>(M) * d, m->xstream));
+    did(launch_add_f32(m->R[both ? r.in : r.add], pend, m->R[r.dst], static_cast<size_t>(M) * d, m->xstream));
     note(cudaEventRecord(m->ev_pf_add[mod], m->xstream));
     add_writer[r.dst] = mod;
   };

@@ -302,7 +302,7 @@ __device__ __forceinline__ void epi_apply(const SmallMParams& p, int n, int b0, 
                                           const WidePeer& wp, const size_t* push_s) {
   const bool row_ok = n < p.N;
   if (PUSH) {
-    // tensor parallelism over peer memory (EPI_PLAIN only): this rank's partial sum goes straight into its receive
+    // tensor parallelism over peer memory (EPI_PLAIN, or EPI_RESID with a local addend): this rank's partial sum goes straight into its receive
     // slot on every rank, every value with the exchange's sequence number in one 8-byte store (lanes hold
     // consecutive rows: 256-byte segments per batch row and peer)
     const size_t off = push_s[0];
@@ -313,7 +313,8 @@ __device__ __forceinline__ void epi_apply(const SmallMParams& p, int n, int b0, 
 #pragma unroll
       for (int j = 0; j < CB; ++j) {
         const int b = b0 + j;
-        if (b < p.batch && row_ok) peer_st_pair(out + static_cast<size_t>(b) * p.N + n, v[j], seq);
+        if (b < p.batch && row_ok)
+          peer_st_pair(out + static_cast<size_t>(b) * p.N + n, p.epi_mode == EPI_RESID ? v[j] + pa[j] : v[j], seq);
       }
     }
   } else if (p.epi_mode == EPI_RESID || p.epi_mode == EPI_PLAIN) {
@@ -794,7 +795,7 @@ cudaError_t launch_smallm_gemm_wide_tc(const SmallMParams& p, cudaStream_t strea
   if (!p.scratch || p.batch < 1 || p.batch > 64 || (p.K & 7) || (p.N & 1)) return cudaErrorInvalidValue;
   if ((reinterpret_cast<uintptr_t>(p.W) | reinterpret_cast<uintptr_t>(p.scratch)) & 15) return cudaErrorMisalignedAddress;
   const bool push = p.wide_peer && p.wide_peer->push_channel;
-  if (push && (p.epi_mode != EPI_PLAIN || p.wide_peer->peer.world < 1 || p.wide_peer->push_channel > 2 ||
+  if (push && ((p.epi_mode != EPI_PLAIN && p.epi_mode != EPI_RESID) || p.wide_peer->peer.world < 1 || p.wide_peer->push_channel > 2 ||
                static_cast<size_t>(p.batch) * p.N > p.wide_peer->peer.max_floats))
     return cudaErrorInvalidValue;
   const int bp = padded_batch(p.batch);

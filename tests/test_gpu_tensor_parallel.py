@@ -42,6 +42,14 @@ def oracle_cfg(s, world):
     return c
 
 
+def exchanged(parts, variant):
+    """The oracle's per-module partial sums, grouped the way the library exchanges them: one by one, except that a
+    parallel attention + MLP layer (Sec. 3.3.1) sums its two outputs before its ONE exchange."""
+    if variant != "parallel":
+        return list(parts)
+    return [parts[i] + parts[i + 1] for i in range(0, len(parts), 2)]
+
+
 class _DeviceFloats:
     """`count` fp32 values at a raw device address, for torch.as_tensor (no copy)."""
 
@@ -78,7 +86,7 @@ def test_rank_0_with_the_oracle_as_rank_1(B, variant, batch, streams, S):
     calls, o_toks, o_hids = [], [], []
     r = O.forward(cfg, OW, prompt, np.float64, cache_o, 0, last_only=True, record=True)
     for j in range(steps + 1):
-        calls.append([parts[1] for parts in r.module_partials])
+        calls.append(exchanged([parts[1] for parts in r.module_partials], variant))
         o_toks.append(r.next_tokens[:, 0])
         o_hids.append(r.hidden[:, 0])
         if j < steps:
@@ -120,7 +128,8 @@ def test_rank_0_with_the_oracle_as_rank_1(B, variant, batch, streams, S):
         toks.append(nxt.cpu().numpy().copy())
         hids.append(hid.cpu().numpy().copy())
     assert model.device_status() == 0
-    assert seen == [batch * S * s.d_model] * (2 * s.n_layers) + [batch * s.d_model] * (2 * s.n_layers * steps)
+    per_pass = s.n_layers if variant == "parallel" else 2 * s.n_layers
+    assert seen == [batch * S * s.d_model] * per_pass + [batch * s.d_model] * (per_pass * steps)
     err = rel_err(np.stack(hids, 1), np.stack(o_hids, 1))
     agree = float(np.mean(np.stack(toks, 1) == np.stack(o_toks, 1)))
     print(f"[tp rank 0 / oracle rank 1, {variant}, batch {batch}, {streams} stream(s)] hidden max-rel-err {err:.3e}, "
@@ -293,7 +302,7 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
     calls, o_toks, o_hids = [], [], []
     r = O.forward(cfg, OW, prompt, np.float64, cache_o, 0, last_only=True, record=True)
     for j in range(steps + 1):
-        calls.append([parts[1] for parts in r.module_partials])
+        calls.append(exchanged([parts[1] for parts in r.module_partials], variant))
         o_toks.append(r.next_tokens[:, 0])
         o_hids.append(r.hidden[:, 0])
         if j < steps:
@@ -348,11 +357,12 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
         assert not queue
         hids.append(hid.cpu().numpy().copy())
     assert model.device_status() == 0
-    assert turns == [s.n_layers * steps] * 2
-    # rank 0's partial of the last attention module has landed in "rank 1's" memory too, numbered like its own copy
-    last = turns[0] - 1
-    mine = words(p0.slot_ptr(0, last & 1, 0), 2 * n).view(n, 2)
-    theirs = words(p1.slot_ptr(0, last & 1, 0), 2 * n).view(n, 2)
+    assert turns == ([0, s.n_layers * steps] if variant == "parallel" else [s.n_layers * steps] * 2)
+    # rank 0's partial of the last exchange of a channel has landed in "rank 1's" memory too, numbered like its own copy
+    ch = 1 if variant == "parallel" else 0
+    last = turns[ch] - 1
+    mine = words(p0.slot_ptr(ch, last & 1, 0), 2 * n).view(n, 2)
+    theirs = words(p1.slot_ptr(ch, last & 1, 0), 2 * n).view(n, 2)
     assert torch.equal(mine, theirs) and bool((mine[:, 1] == last + 1).all()) and int(mine[:, 0].abs().max()) > 0
     err = rel_err(np.stack(hids, 1), np.stack(o_hids, 1))
     print(f"[tp rank 0, fused exchange over peer memory / oracle rank 1, {variant}, batch {batch}, {streams} stream(s)] "

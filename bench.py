@@ -390,10 +390,14 @@ def merged_clocks(recs):
     return mhz, reasons
 
 
-def short_run(B, torch, synth, shape, weights, args, local, steps=32, repeats=3, noise_kv=False):
-    """One of the other configurations: ms/step (median of `repeats` loops) and roofline fractions."""
+def short_run(B, torch, synth, shape, weights, args, local, steps=32, repeats=3, noise_kv=False, tp=None):
+    """One of the other configurations: ms/step (median of `repeats` loops) and roofline fractions.
+    tp = (comm, peer): the model as the one rank of a tensor-parallel world of one (exchange fused over peer memory)."""
     hbm_peak, _, _ = measured_peaks()
     run = DecodeRun(B, torch, synth, shape, weights, steps, 3, args, None, local, noise_kv=noise_kv)
+    if tp is not None:
+        run.model.set_tensor_parallel_peer(*tp)
+        run.persistent = False
     if not noise_kv:
         run.prefill()
     run.warm_up()
@@ -444,6 +448,18 @@ def other_configs_small(B, torch, synth, args, local):
         for b in (1, 4, 16, 64):
             shape = synth.replace(base.as_mode(mode), batch=b)
             out[f"tp_slice_b{b}_{mode}"] = short_run(B, torch, synth, shape, w, args, local, noise_kv=True)
+    # the same slice as the ONE rank of a tensor-parallel world (Sec. 2, Eq. 1; Algorithm 1): every module's output is
+    # stored, exchanged (here with nobody: what the schedule and the fused exchange cost by themselves) and added by
+    # the next reader
+    from paper_2501_06589_b200 import tensor_parallel as TP
+    comm = TP.make_comm()
+    for mode in ("ladder", "standard", "parallel"):
+        shape = synth.replace(base.as_mode(mode), batch=16)
+        peer = TP.make_peer(16 * base.d_model)
+        out[f"tp_slice_b16_{mode}_tensor_parallel_world1"] = short_run(B, torch, synth, shape, w, args, local,
+                                                                      noise_kv=True, tp=(comm, peer))
+        peer.close()
+    comm.close()
     del w
     torch.cuda.empty_cache()
     return out

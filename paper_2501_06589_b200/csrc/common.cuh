@@ -57,10 +57,8 @@ __device__ __forceinline__ bool mbar_try_wait_suspend(uint64_t* bar, uint32_t pa
       : "memory");
   return ok != 0;
 }
-// Bound of every device-side wait, in cycles of the SM's own counter: about 0.3 s at 1.9 GHz.  The waits read
-// clock64(), not %globaltimer: a read of the global timer takes microseconds to return, and a kernel cannot exit
-// while one is outstanding - measured on a 16-CTA exchange kernel: 12.3 us per launch with the timer read in its
-// wait loop, 6.9 us without.
+// Bound of every device-side wait, in cycles of the SM's own counter (clock64(): a register read, no memory or
+// timer traffic): about 0.3 s at 1.9 GHz.
 constexpr long long kWaitCycles = 600000000ll;
 // Bounded wait: gives up after kWaitCycles and reports failure, so a protocol
 // error can never hang the device.  The caller then switches to a drain mode that

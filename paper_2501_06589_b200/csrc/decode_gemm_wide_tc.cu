@@ -155,7 +155,7 @@ __device__ __forceinline__ bool pull_add8(const StagePull& pl, int ch, uint32_t 
       for (int i = 0; i < 4; ++i) t = t && v[i].y == seq && v[i].w == seq;
       return t;
     };
-    if (!there()) {  // bounded by the SM's cycle counter (~0.3 s); %globaltimer costs microseconds to read
+    if (!there()) {  // bounded by the SM's cycle counter (~0.3 s)
       const long long t0 = clock64();
       for (uint32_t it = 1; !there(); ++it) {
 #pragma unroll

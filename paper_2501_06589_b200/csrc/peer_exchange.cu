@@ -76,8 +76,7 @@ __global__ void __launch_bounds__(kThreads) peer_all_reduce_kernel(PeerArgs a, i
     const uint32_t* c = &mine->arrive[channel][threadIdx.x];
     bool ok = static_cast<int32_t>(ld_acquire_sys(c) - target) >= 0;
     if (!ok) {
-      // Poll without sleeping, bounded by the SM's cycle counter (about 0.3 s).  Not %globaltimer: reading it takes
-      // microseconds, which a kernel this short cannot hide (measured: 12.3 -> 6.9 us per exchange).
+      // Poll without sleeping, bounded by the SM's cycle counter (about 0.3 s).
       const long long t0 = clock64();
       for (uint32_t i = 1; !ok; ++i) {
         ok = static_cast<int32_t>(ld_acquire_sys(c) - target) >= 0;

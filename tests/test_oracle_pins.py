@@ -349,6 +349,25 @@ def test_tensor_parallel_partials_sum_to_the_unsplit_module():
         assert np.allclose(O.forward(c1, W(t2), TOK).hidden, O.forward(c2, W(t2), TOK).hidden, atol=1e-11)
 
 
+def test_recorded_partials_are_the_ranks_partial_sums():
+    """The per-rank partial sums a recorded forward pass keeps (what a test hands to a GPU rank in place of its
+    absent peers) are the tp_rank partials of the recorded module inputs, and add up to the recorded outputs."""
+    cfg = small_cfg(n_layers=2, hq=4, hkv=2, f=48, ladder=[1, 0])
+    cfg.tp_world = 2
+    t = rand_weights(cfg, 38)
+    r = O.forward(cfg, W(t), TOK, record=True)
+    assert len(r.module_partials) == 4 and all(len(p) == 2 for p in r.module_partials)
+    for m, (parts, out, src) in enumerate(zip(r.module_partials, r.module_outputs, r.module_inputs)):
+        assert np.allclose(parts[0] + parts[1], out, atol=1e-12)
+        layer, norm = m // 2, ("attn_norm" if m % 2 == 0 else "mlp_norm")
+        n = O.rmsnorm(src, W(t).get(norm, layer), cfg.rms_eps)
+        for rank in range(2):
+            ref = (O.attention_module(cfg, W(t), layer, n, 0, None, tp_rank=rank) if m % 2 == 0
+                   else O.mlp_module(cfg, W(t), layer, n, tp_rank=rank))
+            assert np.allclose(parts[rank], ref, atol=1e-12)
+    assert O.forward(cfg, W(t), TOK).module_partials == []          # nothing is kept unless asked for
+
+
 @pytest.mark.parametrize("masks", [[1, 1, 1, 1], [0, 0, 1, 1], [1, 0, 1, 0]])
 def test_pipeline_stages_chained_equal_the_whole_model(masks):
     """Sec. 5.1: at a stage boundary the stream state is handed on.  Two stages chained give the whole model,

@@ -263,6 +263,9 @@ ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_
  * (bounded) each pair it needs until the number is the expected one and adds the slots in rank order while it
  * forms the residual stream.  This rests on aligned 8-byte stores reaching peer memory whole (as NCCL's
  * low-latency protocol does).
+ * The fused exchange is one-shot - (world - 1) x batch x d_model x 8 bytes leave every rank per exchange - so a decode
+ * step uses it only while that is at most 8 MiB (batch 18 at world 8 and d_model 8192) and the model's `exchange`
+ * (NCCL) above; ladder_model_set_peer_max_bytes moves the limit (negative: never fused).
  * ladder_model_set_tensor_parallel_peer(m, comm, peer): decode steps exchange that way over `peer`, the prompt pass
  * (messages of hundreds of MB, where NCCL's algorithms are the right ones) over `comm`; LADDER_ERR_INVALID_ARG if the
  * peer object is too small for max_batch x d_model, not connected or of another world.  ladder_model_set_peer(m, peer)
@@ -299,6 +302,7 @@ float* ladder_peer_slot(const ladder_peer_t* peer, int32_t channel, int32_t pari
 uint32_t* ladder_peer_counter(const ladder_peer_t* peer, int32_t channel, int32_t from);
 ladder_status_t ladder_model_set_tensor_parallel_peer(ladder_model_t* m, ladder_comm_t* comm, ladder_peer_t* peer);
 ladder_status_t ladder_model_set_peer(ladder_model_t* m, ladder_peer_t* peer);
+ladder_status_t ladder_model_set_peer_max_bytes(ladder_model_t* m, int64_t bytes);
 typedef void (*ladder_peer_hook_fn)(void* ctx, int32_t channel, void* cuda_stream);
 ladder_status_t ladder_debug_set_peer_hook(ladder_model_t* m, ladder_peer_hook_fn fn, void* ctx);
 

@@ -33,7 +33,7 @@ EXPORTS = [
     "ladder_peer_world", "ladder_peer_rank", "ladder_peer_max_floats", "ladder_peer_ctas_per_exchange",
     "ladder_peer_destroy", "ladder_peer_all_reduce_sum", "ladder_peer_probe_write", "ladder_peer_probe_read",
     "ladder_peer_slot", "ladder_peer_counter", "ladder_model_set_tensor_parallel_peer", "ladder_model_set_peer",
-    "ladder_debug_set_peer_hook",
+    "ladder_debug_set_peer_hook", "ladder_model_set_peer_max_bytes",
 ]
 PEER_HOOK_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_int32, C.c_void_p)                # ladder_peer_hook_fn
 PEER_HANDLE_BYTES = 64                                                           # LADDER_PEER_HANDLE_BYTES
@@ -184,6 +184,7 @@ def lib() -> C.CDLL:
         L.ladder_peer_counter.argtypes, L.ladder_peer_counter.restype = [C.c_void_p, C.c_int32, C.c_int32], C.c_void_p
         L.ladder_model_set_tensor_parallel_peer.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.ladder_model_set_peer.argtypes = [C.c_void_p, C.c_void_p]
+        L.ladder_model_set_peer_max_bytes.argtypes = [C.c_void_p, C.c_int64]
         L.ladder_debug_set_peer_hook.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
@@ -444,6 +445,10 @@ class Model:
         """Decode-step exchanges fused into the GEMM epilogues over `peer` (ladder_model_set_peer)."""
         _check(lib().ladder_model_set_peer(self.h, peer.h if peer is not None else None), self.h)
         self._peer = peer
+
+    def set_peer_max_bytes(self, n: int):
+        """Largest (world - 1) x batch x d_model x 8 for which a decode step uses the fused exchange (negative: never)."""
+        _check(lib().ladder_model_set_peer_max_bytes(self.h, n), self.h)
 
     def debug_set_peer_hook(self, fn=None):
         """fn(channel, cuda_stream), called after each decode-step output GEMM has been enqueued (tests)."""

@@ -84,6 +84,7 @@ struct ladder_model {
   int exchange_capturable = 0;  // the callback may be called while its stream is being captured into a CUDA graph
   ladder_comm* comm = nullptr;  // set by ladder_model_set_tensor_parallel (not owned)
   ladder_peer* peer = nullptr;  // decode-step exchanges over peer memory instead of `exchange` (not owned)
+  int64_t peer_max_bytes = 8ll << 20;  // largest outbound volume per exchange the fused exchange is used for
   ladder_peer_hook_fn peer_hook = nullptr;  // test hook: called after each output GEMM of a decode step is enqueued
   void* peer_hook_ctx = nullptr;
   float* pend_pf[2] = {nullptr, nullptr};  // prompt pass under tensor parallelism: the two modules' stored outputs
@@ -319,6 +320,17 @@ struct Enqueue {
   }
 };
 
+// Whether a decode step of this batch exchanges over peer memory (fused into the GEMMs) rather than through
+// `exchange`.  The fused exchange is one-shot: every rank stores its whole partial sum, 8 bytes per element, into every
+// other rank's memory, (world - 1) x batch x d_model x 8 bytes per rank and exchange.  That is the fastest way for the
+// small messages of a decode step and a waste of link bandwidth for large ones, where a reduce-scatter / all-gather
+// moves a quarter of it at world 8: above peer_max_bytes (8 MiB unless set otherwise) the step leaves it to `exchange` (NCCL).
+bool peer_fused(const ladder_model* m, int batch) {
+  if (!m->peer) return false;
+  const int64_t out = static_cast<int64_t>(ladder_peer_world(m->peer) - 1) * batch * m->cfg.d_model * 8;
+  return out <= m->peer_max_bytes;
+}
+
 // The decode step in the pending-output form of Algorithm 1.  The output and down projections STORE their module's
 // output (pend_a / pend_m) instead of adding it to the stream, and the stream moves on in the staging step of a
 // later reader: the step that forms module j's input x_{j-1} (Eq. 1) or x_{j-2} (Eq. 2) adds the stored outputs
@@ -344,7 +356,7 @@ cudaError_t enqueue_decode_pending(ladder_model* m, const ladder_kv_cache_t* cac
   const int Hq = c.n_q_heads, Hkv = c.n_kv_heads, Dh = c.head_dim, d = c.d_model, F = c.d_ff, L = c.n_layers;
   const size_t layer_elems = static_cast<size_t>(c.max_batch) * Hkv * c.max_seq_len * Dh;
   PeerView view = {};
-  const bool use_peer = m->peer != nullptr && peer_view(m->peer, &view);
+  const bool use_peer = peer_fused(m, batch) && peer_view(m->peer, &view);
   Router rt;
   q.launched(0, begin_stream(m, rt, d_tokens, batch, sA));
   int cur = rt.cur;  // R[cur]: the newest stream value formed so far = x_0 + outputs of modules 0 .. added
@@ -1655,6 +1667,13 @@ ladder_status_t ladder_model_set_tensor_parallel_peer(ladder_model_t* m, ladder_
   return s == LADDER_OK ? ladder_model_set_peer(m, peer) : s;
 }
 
+ladder_status_t ladder_model_set_peer_max_bytes(ladder_model_t* m, int64_t bytes) {
+  if (!m) return LADDER_ERR_INVALID_ARG;
+  m->peer_max_bytes = bytes;
+  drop_graph(m);
+  return LADDER_OK;
+}
+
 ladder_status_t ladder_debug_set_peer_hook(ladder_model_t* m, ladder_peer_hook_fn fn, void* ctx) {
   if (!m) return LADDER_ERR_INVALID_ARG;
   m->peer_hook = fn;
@@ -1936,7 +1955,8 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
   }
 
   // a graph only if everything the step calls back into may be captured (with a peer object the step calls nothing)
-  if (!m->use_graph || (m->exchange && !m->peer && !m->exchange_capturable) || (m->peer && m->peer_hook)) {
+  const bool fused = peer_fused(m, batch);
+  if (!m->use_graph || (m->exchange && !fused && !m->exchange_capturable) || (fused && m->peer_hook)) {
     int64_t k = 0;
     if (two) {
       // the side stream may only start after everything already queued on the caller's stream

@@ -272,6 +272,19 @@ def test_decode_exchange_over_peer_memory_in_a_world_of_one(B, variant, batch):
         assert model.device_status() == 0
         model.close()
     assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1])
+    # above the size limit the decode steps leave the exchange to NCCL: same results, nothing lands in the slots
+    fresh = TP.make_peer(batch * s.d_model)
+    model = B.Model(w, batch, S + steps + 2, batch * S)
+    model.set_tensor_parallel_peer(comm, fresh)
+    model.set_peer_max_bytes(-1)
+    t3, h3 = gpu_generate(B, model, B.KVCache(s, batch, S + steps + 2), prompt, steps)
+    assert np.array_equal(runs[0][0], t3) and np.array_equal(runs[0][1], h3)
+    slot = torch.as_tensor(_DeviceFloats(fresh.slot_ptr(0, 0, 0), 2 * batch * s.d_model), device="cuda")
+    assert float(slot.abs().max()) == 0.0
+    used = torch.as_tensor(_DeviceFloats(peer.slot_ptr(0, 0, 0), 2 * batch * s.d_model), device="cuda")
+    assert float(used.abs().max()) > 0.0
+    model.close()
+    fresh.close()
     small = B.Peer(1, 0, 64)
     model = B.Model(w, batch, 32, 32)
     with pytest.raises(B.LadderError):

@@ -296,9 +296,9 @@ def test_decode_exchange_over_peer_memory_in_a_world_of_one(B, variant, batch):
 
 
 @pytest.mark.parametrize("streams", [2, 1])
-@pytest.mark.parametrize("variant,batch", [("ladder", 6), ("standard", 6), ("hybrid", 3), ("ladder", 40), ("parallel", 6),
-                                           ("flags", 5)])
-def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, streams):
+@pytest.mark.parametrize("variant,batch,world", [("ladder", 6, 2), ("standard", 6, 2), ("hybrid", 3, 2), ("ladder", 40, 2),
+                                                 ("parallel", 6, 2), ("flags", 5, 2), ("ladder", 9, 4), ("standard", 2, 4)])
+def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, world, streams):
     """As test_rank_0_with_the_oracle_as_rank_1, but the decode-step exchange is the fused one: rank 0's output GEMMs
     push their partial sums into the receive slots (rank 0's own and, on the same GPU, those of a second object that
     stands for rank 1's memory) as (value, sequence number) pairs, and the staging launches poll the pairs and add
@@ -306,7 +306,7 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
     behind each output GEMM, so every poll succeeds at once."""
     from paper_2501_06589_b200 import tensor_parallel as TP
     s = shape_of(variant)
-    world, S, steps = 2, 12, 6
+    S, steps = 12, 6                                          # world 4: more ranks than kv heads (each kv head on two ranks)
     w = synth.make_weights(s, device="cuda", gains="uniform")
     prompt = synth.make_tokens(s, batch, S)
     cfg = oracle_cfg(s, world)
@@ -315,7 +315,7 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
     calls, o_toks, o_hids = [], [], []
     r = O.forward(cfg, OW, prompt, np.float64, cache_o, 0, last_only=True, record=True)
     for j in range(steps + 1):
-        calls.append(exchanged([parts[1] for parts in r.module_partials], variant))
+        calls.append([exchanged([parts[k] for parts in r.module_partials], variant) for k in range(1, world)])
         o_toks.append(r.next_tokens[:, 0])
         o_hids.append(r.hidden[:, 0])
         if j < steps:
@@ -323,9 +323,11 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
                           record=True)
 
     n = batch * s.d_model
-    p0, p1 = B.Peer(2, 0, n), B.Peer(2, 1, n)
-    p0.connect(1, same_process_base=p1.local_base())
-    p1.connect(0, same_process_base=p0.local_base())
+    p0 = B.Peer(world, 0, n)
+    others = [B.Peer(world, k, n) for k in range(1, world)]   # memory that stands for the other ranks'
+    for k, pk in enumerate(others, start=1):
+        p0.connect(k, same_process_base=pk.local_base())
+    p1 = others[0]
     rw = TP.rank_weights(w, 0, world)
     model = B.Model(rw, batch, S + steps + 1, batch * S)
     model.set_schedule(streams, True, True)
@@ -340,16 +342,17 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
 
     def prompt_exchange(ptr, count, stream):                 # the prompt pass: NCCL's place
         with torch.cuda.stream(torch.cuda.ExternalStream(stream or 0)):
-            torch.as_tensor(_DeviceFloats(ptr, count), device="cuda").add_(queue.pop(0))
+            for part in queue.pop(0):
+                torch.as_tensor(_DeviceFloats(ptr, count), device="cuda").add_(part)
         return 0
 
     def rank_1_arrives(channel, stream):                     # a decode-step output GEMM of rank 0 has been enqueued
-        part = queue.pop(0)
-        pairs = torch.empty(n, 2, dtype=torch.int32, device="cuda")   # (value, sequence number of the exchange)
-        pairs[:, 0] = part.view(torch.int32)
-        pairs[:, 1] = turns[channel] + 1
-        with torch.cuda.stream(torch.cuda.ExternalStream(stream or 0)):
-            words(p0.slot_ptr(channel, turns[channel] & 1, 1), 2 * n).copy_(pairs.view(-1))
+        for k, part in enumerate(queue.pop(0), start=1):      # the other ranks' stores into rank 0's receive slots
+            pairs = torch.empty(n, 2, dtype=torch.int32, device="cuda")   # (value, sequence number of the exchange)
+            pairs[:, 0] = part.view(torch.int32)
+            pairs[:, 1] = turns[channel] + 1
+            with torch.cuda.stream(torch.cuda.ExternalStream(stream or 0)):
+                words(p0.slot_ptr(channel, turns[channel] & 1, k), 2 * n).copy_(pairs.view(-1))
         turns[channel] += 1
 
     model.set_exchange(prompt_exchange, capturable=False)
@@ -360,7 +363,8 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
     hid = torch.zeros(batch, s.d_model, device="cuda")
     hids = []
     for j in range(steps + 1):
-        queue[:] = [torch.from_numpy(np.ascontiguousarray(p, dtype=np.float32).reshape(-1)).cuda() for p in calls[j]]
+        up = lambda p: torch.from_numpy(np.ascontiguousarray(p, dtype=np.float32).reshape(-1)).cuda()
+        queue[:] = [[up(calls[j][k][i]) for k in range(world - 1)] for i in range(len(calls[j][0]))]
         if j == 0:
             model.prefill(cache, torch.from_numpy(prompt).cuda(), next_tokens=nxt, final_hidden=hid)
         else:
@@ -383,4 +387,5 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, st
     assert err < HIDDEN_TOL, err
     model.close()
     p0.close()
-    p1.close()
+    for pk in others:
+        pk.close()

@@ -3,8 +3,21 @@
 // One communicator per rank = per process = per GPU.  The NCCL library is looked up at run time (the one the
 // process has already loaded, e.g. PyTorch's, else the system's), so the library loads without it and a
 // single-GPU user never touches it.  Host code only: the reduction itself is NCCL's kernel on the stream it is given.
+#include <cuda_runtime.h>
 #include <dlfcn.h>
+#if __has_include(<nccl.h>)
 #include <nccl.h>
+#else
+// No NCCL header on the build machine: the handful of declarations this file needs, as NCCL's public interface
+// has had them since 2.0 (the library itself is only ever looked up at run time).
+typedef struct ncclComm* ncclComm_t;
+typedef struct {
+  char internal[128];
+} ncclUniqueId;
+typedef enum { ncclSuccess = 0 } ncclResult_t;
+typedef enum { ncclFloat32 = 7 } ncclDataType_t;
+typedef enum { ncclSum = 0 } ncclRedOp_t;
+#endif
 
 #include <mutex>
 

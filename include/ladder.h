@@ -157,6 +157,9 @@ ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, 
  * modules; with the standard rule (Eq. 1) each phase waits for the one before.  on = 0 selects the
  * multi-kernel schedule configured by ladder_model_set_schedule (also used automatically for batch > 4
  * and on devices where the kernel cannot be made resident).  Results are bit-identical either way.
+ * A fresh model (before any call of this function) takes this path for batch <= 4 except for all-ladder models with layers below 300 MB whose attention module is at most a
+ * quarter as wide as the hidden size (one tensor-parallel rank's slice), where the pending-output form on the tcgen05
+ * GEMMs measured 4-6 % faster; on != 0 insists on the persistent kernel.
  * ladder_model_persistent_active returns 1 when decode steps of batch <= 4 take this path. */
 ladder_status_t ladder_model_set_persistent(ladder_model_t* m, int32_t on);
 int32_t ladder_model_persistent_active(const ladder_model_t* m);
@@ -189,7 +192,8 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
  * bit-identical for every setting.  Batch 5..64: every CTA accumulates one contiguous K range in fp32, so the number
  * of CTAs a GEMM runs on decides where the sums are cut: settings that give a GEMM different shares differ in
  * rounding (~1e-4 of the hidden state), each of them reproducible from run to run.
- * Whenever the split is on, batch is 5..64 and every module reads x_{m-2} (all layers ladder), the step also runs
+ * Whenever the split is on, every module reads x_{m-2} (all layers ladder) and batch is 5..64 (any batch when the
+ * split was asked for explicitly), the step also runs
  * in the pending-output form of Algorithm 1: a module's output stays in a buffer of its own and is added to the
  * residual when the next module's input is normalised, so the attention chain and the MLP chain wait for each
  * other's normalised-input kernel only, never for a GEMM.  The additions are the same fp32 additions in the same

@@ -126,6 +126,7 @@ struct ladder_model {
   bool stack_usable = false;  // the kernel fits this device and this depth
   int stack_stall_test = 0;  // test hook: the last phase waits for a count its producer never reaches
   int use_stack = 1;
+  bool persistent_explicit = false;  // ladder_model_set_persistent was called with on != 0: no second-guessing
   GraphKey stack_key;      // what the uploaded phase list was built for
   bool stack_built = false;
   StackPhase* d_phases = nullptr;
@@ -319,6 +320,23 @@ struct Enqueue {
     if (err == cudaSuccess) err = r;
   }
 };
+
+// Batch <= 4, every module reading x_{m-2}, small layers AND an attention module much narrower than the hidden size
+// (one tensor-parallel rank's slice: 8 of 64 heads at the 70B shape): the persistent kernel loses to the
+// pending-output form on the tcgen05 GEMMs with the two chains side by side on 32 / 116 SMs - measured at the
+// TP-rank slice, KV 2048: batch 1 / 2 / 4 4.05 / 4.03 / 4.15 ms per step in the persistent kernel, 3.82 / 3.85 / 3.91 ms
+// this way (inside the persistent kernel the output projection waits for the attention of its own layer, which at
+// this shape takes longer than the gate/up phase beside it).  Where the attention is as wide as the model (1.2B
+// shape) the persistent kernel stays ahead (0.80 against 0.85 ms).
+bool prefers_wide_small(const ladder_model* m) {
+  const ladder_config_t& c = m->cfg;
+  if (m->persistent_explicit || m->n_streams != 2 || m->sms_a != -1 || !m->pend_a || !m->pend_m) return false;
+  for (uint8_t f : m->stale)
+    if (!f) return false;
+  const double layer_bytes = 2.0 * (static_cast<double>((c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim) * c.d_model +
+                                    static_cast<double>(c.d_model) * c.n_q_heads * c.head_dim + 3.0 * c.d_ff * c.d_model);
+  return layer_bytes < 300e6 && 4 * c.n_q_heads * c.head_dim <= c.d_model;
+}
 
 // Whether a decode step of this batch exchanges over peer memory (fused into the GEMMs) rather than through
 // `exchange`.  The fused exchange is one-shot: every rank stores its whole partial sum, 8 bytes per element, into every
@@ -594,8 +612,11 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   // 8 layers at batch 16 and 921 -> 865 us at batch 64 (at the 70B shape the split loses at every batch).
   const double layer_bytes = 2.0 * (static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh + 3.0 * F * d);
   const bool auto_wide = (m->sms_a == -1 || m->sms_a == -3) && batch > 4 && layer_bytes < 300e6;
-  if (q.two && (m->sms_a >= 0 || auto_wide)) {
-    int ga = auto_wide ? (56 * m->sm_count + 74) / 148 : m->sms_a;  // 56 : 92 (swept 40 .. 72 in the pending-output form)
+  const bool auto_small = batch <= 4 && !m->st_in.newest && !m->st_out.newest && (l_end < 0 || l_end == c.n_layers) &&
+                          prefers_wide_small(m);
+  if (q.two && (m->sms_a >= 0 || auto_wide || auto_small)) {
+    // 56 : 92 for batch 5..64 (swept 40 .. 72 in the pending-output form), 32 : 116 for batch <= 4 (swept 20 .. 52)
+    int ga = auto_small ? (32 * m->sm_count + 74) / 148 : auto_wide ? (56 * m->sm_count + 74) / 148 : m->sms_a;
     if (ga == 0) {
       const double ba = static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh;
       const double bb = 3.0 * F * d;
@@ -606,7 +627,7 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
     q.grid_a = ga;
     q.grid_b = m->sm_count - ga;
     // every module reads x_{m-2} (all layers ladder), batch 5..64, the whole step here: the pending-output schedule
-    bool all_stale = batch > 4 && m->sms_a != -3 && m->pend_a && m->pend_m && !m->st_in.newest && !m->st_out.newest &&
+    bool all_stale = (batch > 4 || m->sms_a >= 0 || auto_small) && m->sms_a != -3 && m->pend_a && m->pend_m && !m->st_in.newest && !m->st_out.newest &&
                      (l_end < 0 || l_end == c.n_layers);
     for (size_t i = 0; i < m->stale.size() && all_stale; ++i) all_stale = m->stale[i] != 0;
     if (all_stale && !m->exchange)
@@ -1602,6 +1623,7 @@ ladder_status_t ladder_model_set_schedule(ladder_model_t* m, int32_t n_streams, 
 ladder_status_t ladder_model_set_persistent(ladder_model_t* m, int32_t on) {
   if (!m) return LADDER_ERR_INVALID_ARG;
   m->use_stack = on ? 1 : 0;
+  m->persistent_explicit = on != 0;
   // 2: every layer in the persistent kernel, standard-residual ones included; 1: the default choice
   const int L = m->cfg.n_layers;
   m->stack_begin = on == 2 ? 0 : stack_default_begin(m->cfg, m->is_ladder);
@@ -1617,7 +1639,9 @@ ladder_status_t ladder_debug_stall_last_phase(ladder_model_t* m, int32_t on) {
   return LADDER_OK;
 }
 
-int32_t ladder_model_persistent_active(const ladder_model_t* m) { return (m && m->use_stack && m->stack_ok) ? 1 : 0; }
+int32_t ladder_model_persistent_active(const ladder_model_t* m) {
+  return (m && m->use_stack && m->stack_ok && !prefers_wide_small(m)) ? 1 : 0;
+}
 
 ladder_status_t ladder_model_set_exchange(ladder_model_t* m, ladder_exchange_fn fn, void* ctx, int32_t capturable) {
   if (!m) return LADDER_ERR_INVALID_ARG;
@@ -1918,7 +1942,7 @@ ladder_status_t ladder_decode_step(ladder_model_t* m, const ladder_kv_cache_t* c
   const bool two = m->n_streams == 2;
 
   const bool staged = m->st_in.newest || m->st_out.newest;  // a pipeline stage runs kernel by kernel
-  if (m->use_stack && m->stack_ok && batch <= 4 && !staged && !m->exchange) {
+  if (m->use_stack && m->stack_ok && batch <= 4 && !staged && !m->exchange && !prefers_wide_small(m)) {
     GraphKey key;
     key.batch = batch;
     key.k = cache->k;

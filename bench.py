@@ -546,7 +546,14 @@ def run_rank(args, rank, world):
         e2e_recs.append(max_over_ranks([(time.perf_counter() - t0) * 1e3], dist, "cuda")[0])
     e2e_ms = statistics.median(e2e_recs)
 
-    # ---- dominant kernel alone: the gate/up weight-streaming GEMM over every layer's weights
+    # ---- dominant kernel alone: the gate/up weight-streaming GEMM over every layer's weights, with the kernel the
+    # steps above used for it (batch > 4, tensor parallelism, and slice-like all-ladder models at any batch: tcgen05)
+    all_ladder = shape.layer_mode is None and shape.module_stale is None and all(shape.ladder_mask())
+    slice_like = all_ladder and shape.layer_weight_bytes() < 300e6 and 4 * shape.n_q_heads * shape.head_dim <= shape.d_model
+    step_used_tcgen05 = bsz > 4 or args.wide_impl == 2 or args.tp or (
+        not persistent and slice_like and args.sm_split is None and args.streams in (None, 2))
+    if step_used_tcgen05:
+        B.set_decode_wide_impl(2)
     x_act = torch.randn(bsz, shape.d_model, device="cuda")
     h_out_buf = torch.empty(bsz, shape.d_ff, device="cuda")
     n_l = shape.n_layers
@@ -559,6 +566,7 @@ def run_rank(args, rank, world):
         B.op_smallm_gemm(w.w_gate_up[l], x_act, 1, 1, h_out_buf, gain=w.mlp_norm[l], eps=shape.rms_eps)
     e1.record()
     torch.cuda.synchronize()
+    B.set_decode_wide_impl(args.wide_impl)
     k_ms = e0.elapsed_time(e1) / n_l
     k_bytes = 2.0 * 2 * shape.d_ff * shape.d_model
     k_gbs = k_bytes / (k_ms * 1e-3) / 1e9
@@ -587,7 +595,8 @@ def run_rank(args, rank, world):
         "gpu_launches": int(launches),
         "repeats": {"n": len(dev_recs), "statistic": "median", "ms": [round(r["ms"], 3) for r in dev_recs],
                     "sm_mhz": [r["sm_mhz"] for r in dev_recs]},
-        "roofline": {"bound": "hbm", "kernel": "smallm_gemm (RMSNorm + gate/up projection + SwiGLU)",
+        "roofline": {"bound": "hbm", "kernel": ("decode_gemm_wide_tc (tcgen05; " if step_used_tcgen05 else "smallm_gemm (") +
+                               "RMSNorm + gate/up projection + SwiGLU)",
                      "achieved": k_gbs, "peak": hbm_peak, "peak_source": peak_src, "unit": "GB/s",
                      "frac": k_gbs / hbm_peak, "bytes_per_launch": k_bytes, "ms_per_launch": k_ms,
                      "traffic": traffic.get((shape.name, bsz, "decode_gemm_gate_up_bytes"))},

@@ -197,7 +197,8 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
  * in the pending-output form of Algorithm 1: a module's output stays in a buffer of its own and is added to the
  * residual when the next module's input is normalised, so the attention chain and the MLP chain wait for each
  * other's normalised-input kernel only, never for a GEMM.  The additions are the same fp32 additions in the same
- * order (bit-identical to -3 on the same shares).  -3 = the library's choice of split without that form (each output added by its GEMM's epilogue). */
+ * order (bit-identical to -3 on the same shares).  -3 = the library's choice of split without that form (each output
+ * added by its GEMM's epilogue). */
 ladder_status_t ladder_model_set_sm_split(ladder_model_t* m, int32_t sms_attention_stream);
 
 /* Tensor parallelism (paper Sec. 2, Eq. 1: x_i = AllReduce(h_i(x_{i-1})) + x_{i-1}; Sec. 3.1, Eq. 2 and Algorithm 1:
@@ -245,7 +246,9 @@ int32_t ladder_comm_rank(const ladder_comm_t* comm);
 ladder_status_t ladder_comm_all_reduce_sum(void* comm, float* partial, int64_t count, void* cuda_stream);
 ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_t* comm);
 
-/* The exchange over peer memory, for the decode step (paper Sec. 2 Eq. 1; messages of batch x d_model fp32): one
+/* The exchange over peer memory, for the decode step (paper Sec. 2 Eq. 1; messages of batch x d_model fp32), in two
+ * forms: a stand-alone all-reduce (ladder_peer_all_reduce_sum) and, inside a model, an exchange fused into the GEMM
+ * before it and the launch after it (further down).  The stand-alone form is one
  * kernel per exchange in which every rank stores its partial sum into a receive slot in each peer's memory (plain
  * stores through the NVLink peer mapping), raises a counter there, waits - bounded, about 0.3 s, then
  * LADDER_DEV_TIMEOUT in the status word and no sum - for its peers' counters in its own memory and adds the slots in
@@ -283,7 +286,7 @@ ladder_status_t ladder_model_set_tensor_parallel(ladder_model_t* m, ladder_comm_
  * where a rank's data lands (a slot holds max_floats values for ladder_peer_all_reduce_sum, max_floats (value, number)
  * pairs for the fused exchange) and how the stand-alone kernel counts arrivals (each exchange adds ctas_per_exchange
  * to the sender's counter), so that a test can play an absent rank.
- * Exercised on one GPU only (a world of one, and a world of two with the other rank's stores made by the test):
+ * Exercised on one GPU only (a world of one, and worlds of two and four with the other ranks' stores made by the test):
  * the IPC path is covered by the probe between two processes; nothing is claimed about multi-GPU speed. */
 #define LADDER_PEER_MAX_WORLD 8
 #define LADDER_PEER_HANDLE_BYTES 64

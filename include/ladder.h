@@ -186,7 +186,7 @@ int32_t ladder_stack_plan(const ladder_config_t* cfg, int32_t batch, int32_t sm_
 /* With two streams, the GEMMs of a ladder layer's attention module and MLP module can be run side by side on
  * disjoint sets of SMs (each GEMM is a persistent kernel that claims its work dynamically, so it runs
  * on any number of CTAs).  sms_attention_stream: -1 = the library's choice (default): no split, every GEMM on all
- * SMs, which measured fastest everywhere except for batch 5..64 with layers below 300 MB, where 56 of 148 SMs go
+ * SMs, which measured fastest everywhere except for batch 5..64 with layers below 300 MB, where 56 of 148 SMs (44 above batch 32) go
  * to the attention stream; -2 = never split; 0 = in proportion to the bytes each module streams; n > 0 = that many
  * SMs (at most half of them) for the attention module's GEMMs and the rest for the MLP's.  Batch <= 4: results are
  * bit-identical for every setting.  Batch 5..64: every CTA accumulates one contiguous K range in fp32, so the number

@@ -323,7 +323,7 @@ struct Enqueue {
 
 // Batch <= 4, every module reading x_{m-2}, small layers AND an attention module much narrower than the hidden size
 // (one tensor-parallel rank's slice: 8 of 64 heads at the 70B shape): the persistent kernel loses to the
-// pending-output form on the tcgen05 GEMMs with the two chains side by side on 32 / 116 SMs - measured at the
+// pending-output form on the tcgen05 GEMMs with the two chains side by side on 36 / 112 SMs - measured at the
 // TP-rank slice, KV 2048: batch 1 / 2 / 4 4.05 / 4.03 / 4.15 ms per step in the persistent kernel, 3.82 / 3.85 / 3.91 ms
 // this way (inside the persistent kernel the output projection waits for the attention of its own layer, which at
 // this shape takes longer than the gate/up phase beside it).  Where the attention is as wide as the model (1.2B
@@ -615,8 +615,10 @@ cudaError_t enqueue_decode(ladder_model* m, const ladder_kv_cache_t* cache, cons
   const bool auto_small = batch <= 4 && !m->st_in.newest && !m->st_out.newest && (l_end < 0 || l_end == c.n_layers) &&
                           prefers_wide_small(m);
   if (q.two && (m->sms_a >= 0 || auto_wide || auto_small)) {
-    // 56 : 92 for batch 5..64 (swept 40 .. 72 in the pending-output form), 32 : 116 for batch <= 4 (swept 20 .. 52)
-    int ga = auto_small ? (32 * m->sm_count + 74) / 148 : auto_wide ? (56 * m->sm_count + 74) / 148 : m->sms_a;
+    // of 148 SMs for the attention stream (swept 20 .. 72 in the pending-output form): 36 for batch <= 4, 56 for batch
+    // 5..32, 44 above
+    const int share = auto_small ? 36 : (batch <= 32 ? 56 : 44);
+    int ga = (auto_small || auto_wide) ? (share * m->sm_count + 74) / 148 : m->sms_a;
     if (ga == 0) {
       const double ba = static_cast<double>((Hq + 2 * Hkv) * Dh) * d + static_cast<double>(d) * Hq * Dh;
       const double bb = 3.0 * F * d;

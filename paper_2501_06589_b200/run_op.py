@@ -42,6 +42,8 @@ def main():
                     help="attn, stack: 1 = the register-fragment decode attention kernel at every batch, 2 = the TMA / tcgen05 kernel for every batch > 8")
     ap.add_argument("--sm-split", type=int, default=-1,
                     help="stack (one kernel per GEMM): SMs for the attention module's GEMMs, the rest for the MLP's (0 = by bytes)")
+    ap.add_argument("--tp", action="store_true",
+                    help="stack: as the one rank of a tensor-parallel world (pending-output form, fused exchange)")
     ap.add_argument("--no-lo", action="store_true", help="prefill_attn: queries and outputs without their lo parts")
     ap.add_argument("--seq", type=int, default=None, help="prefill_attn: tokens per sequence")
     a = ap.parse_args()
@@ -170,7 +172,11 @@ def run_stack(a, s, bsz):
         model.set_persistent(2)
     if a.sm_split != -1:
         model.set_sm_split(a.sm_split)
-    persistent = model.persistent_active() and bsz <= 8
+    if a.tp:      # the one rank of a tensor-parallel world: exchange fused over peer memory (with nobody)
+        from . import tensor_parallel as TP
+        comm, peer = TP.make_comm(), TP.make_peer(bsz * s.d_model)
+        model.set_tensor_parallel_peer(comm, peer)
+    persistent = model.persistent_active() and bsz <= 8 and not a.tp
     cache = B.KVCache(s, bsz, S + steps + 1)
     cache.k.normal_()                                 # a synthetic prefix instead of a prompt pass
     cache.v.normal_()

@@ -389,3 +389,38 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, wo
     p0.close()
     for pk in others:
         pk.close()
+
+
+def test_fused_exchange_gives_up_cleanly_when_a_rank_never_stores(B):
+    """Rank 1 of a world of two never shows up: every staging launch that needs its pairs polls for its limit (about
+    0.3 s), sets LADDER_DEV_TIMEOUT and goes on with what it has; nothing hangs or faults, the status word says so, the
+    model refuses further steps, and the device keeps working."""
+    import time
+    from paper_2501_06589_b200 import tensor_parallel as TP
+    s = shape_of("ladder")
+    batch, S = 2, 8
+    w = synth.make_weights(s, device="cuda", gains="uniform")
+    rw = TP.rank_weights(w, 0, 2)
+    n = batch * s.d_model
+    p0, p1 = B.Peer(2, 0, n), B.Peer(2, 1, n)
+    p0.connect(1, same_process_base=p1.local_base())
+    model = B.Model(rw, batch, 32, batch * S)
+    model.set_exchange(lambda ptr, count, stream: 0, capturable=True)     # the prompt pass: rank 1 contributes nothing
+    model.set_peer(p0)
+    cache = B.KVCache(rw.shape, batch, 32)
+    nxt = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    model.prefill(cache, torch.from_numpy(synth.make_tokens(s, batch, S)).cuda(), next_tokens=nxt)
+    torch.cuda.synchronize()
+    t0 = time.time()
+    model.decode_step(cache, nxt, next_tokens=nxt)
+    torch.cuda.synchronize()
+    took = time.time() - t0
+    assert model.device_status() == 4                     # LADDER_DEV_TIMEOUT
+    assert 0.2 < took < 30.0, took                        # 2 x layers + 1 waits of ~0.3 s at most, never a hang
+    with pytest.raises(B.LadderError):
+        model.decode_step(cache, nxt, next_tokens=nxt)    # refused until the caller has dealt with it
+    x = torch.arange(1024, device="cuda", dtype=torch.float32)
+    assert float((x * 2).sum()) == 2 * 1023 * 1024 / 2    # the context is intact
+    model.close()
+    p0.close()
+    p1.close()

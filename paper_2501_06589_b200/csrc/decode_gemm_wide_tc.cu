@@ -155,16 +155,15 @@ __device__ __forceinline__ bool pull_add8(const StagePull& pl, int ch, uint32_t 
       for (int i = 0; i < 4; ++i) t = t && v[i].y == seq && v[i].w == seq;
       return t;
     };
-    if (!there()) {  // bounded by the SM's cycle counter (~0.3 s)
+    if (!there()) {  // bounded by the SM's cycle counter (~0.3 s); no waiting at all once a wait has run out anywhere
       const long long t0 = clock64();
-      for (uint32_t it = 1; !there(); ++it) {
+      const volatile int32_t* st = pl.status;
+      if (st && (*st & LADDER_DEV_TIMEOUT)) ok = false;
+      for (uint32_t it = 1; ok && !there(); ++it) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
           if (v[i].y != seq || v[i].w != seq) v[i] = peer_ld_pairs(src + i);
-        if ((it & 255u) == 0 && clock64() - t0 > 600000000ll) {
-          ok = false;
-          break;
-        }
+        if ((it & 255u) == 0 && (clock64() - t0 > kWaitCycles || (st && (*st & LADDER_DEV_TIMEOUT)))) ok = false;
       }
     }
     if (ok) {

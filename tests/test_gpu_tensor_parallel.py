@@ -392,8 +392,8 @@ def test_rank_0_over_peer_memory_with_the_oracle_as_rank_1(B, variant, batch, wo
 
 
 def test_fused_exchange_gives_up_cleanly_when_a_rank_never_stores(B):
-    """Rank 1 of a world of two never shows up: every staging launch that needs its pairs polls for its limit (about
-    0.3 s), sets LADDER_DEV_TIMEOUT and goes on with what it has; nothing hangs or faults, the status word says so, the
+    """Rank 1 of a world of two never shows up: the first staging launch that needs its pairs polls for its limit
+    (about 0.3 s), sets LADDER_DEV_TIMEOUT, and from then on nothing waits any more; nothing hangs or faults, the status word says so, the
     model refuses further steps, and the device keeps working."""
     import time
     from paper_2501_06589_b200 import tensor_parallel as TP
@@ -416,7 +416,7 @@ def test_fused_exchange_gives_up_cleanly_when_a_rank_never_stores(B):
     torch.cuda.synchronize()
     took = time.time() - t0
     assert model.device_status() == 4                     # LADDER_DEV_TIMEOUT
-    assert 0.2 < took < 30.0, took                        # 2 x layers + 1 waits of ~0.3 s at most, never a hang
+    assert 0.2 < took < 5.0, took                         # one wait of ~0.3 s; the launches behind it do not wait again
     with pytest.raises(B.LadderError):
         model.decode_step(cache, nxt, next_tokens=nxt)    # refused until the caller has dealt with it
     x = torch.arange(1024, device="cuda", dtype=torch.float32)

@@ -256,6 +256,12 @@ __global__ void __launch_bounds__(DH) decode_attention_merge_kernel(const float*
   pdl_launch_dependents();
   pdl_wait();
   const float* base = scratch + (static_cast<size_t>(b) * n_q_heads + h) * n_splits * stride;
+  // This thread's element of the first 32 partials, fetched before anything depends on anything: the statistics
+  // below then cost no extra memory round trip (a 2048-key cache has 32 partials of 64 keys).
+  constexpr int PRE = 32;
+  float pre[PRE];
+#pragma unroll
+  for (int s = 0; s < PRE; ++s) pre[s] = s < n_splits ? __ldcg(base + s * stride + tid) : 0.f;
   float m = -INFINITY;
   for (int s = tid; s < n_splits; s += DH) {
     wgt[s] = __ldcg(base + s * stride + DH);
@@ -280,8 +286,11 @@ __global__ void __launch_bounds__(DH) decode_attention_merge_kernel(const float*
 #pragma unroll
   for (int w = 0; w < DH / 32; ++w) lsum += red_l[w];
   float acc = 0.f;
+#pragma unroll
+  for (int s = 0; s < PRE; ++s)
+    if (s < n_splits) acc += wgt[s] * pre[s];
 #pragma unroll 8
-  for (int s = 0; s < n_splits; ++s) acc += wgt[s] * __ldcg(base + s * stride + tid);
+  for (int s = PRE; s < n_splits; ++s) acc += wgt[s] * __ldcg(base + s * stride + tid);
   const float val = lsum > 0.f ? acc / lsum : 0.f;
   o[(static_cast<size_t>(b) * n_q_heads + h) * DH + tid] = val;
   if (o_pack) {  // the output projection's staged operand: hi part in row b, lo part in row bp + b

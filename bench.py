@@ -646,10 +646,14 @@ def run_rank(args, rank, world):
         comm.close()
     if solo and not args.no_other_configs and args.config == "70b" and args.mode is None and not args.standard and not args.tp:
         t0 = time.time()
-        others = other_configs(B, torch, synth, args, local, w, shape)
-        del w
-        torch.cuda.empty_cache()
-        others.update(other_configs_small(B, torch, synth, args, local))
+        others = {}
+        try:      # the headline above is measured already: a failure here must not lose it
+            others.update(other_configs(B, torch, synth, args, local, w, shape))
+            del w
+            torch.cuda.empty_cache()
+            others.update(other_configs_small(B, torch, synth, args, local))
+        except Exception as e:      # noqa: BLE001
+            line["other_configs_error"] = repr(e)[:300]
         line["other_configs"] = others
         line["other_configs_s"] = round(time.time() - t0, 1)
     if rank == 0:
